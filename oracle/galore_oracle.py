@@ -1,0 +1,342 @@
+"""CPU oracle for the GaLore-Adam optimizer step.  TEST INFRASTRUCTURE ONLY.
+
+This module is the slow, plain fp64 statement of what the method computes.  It
+exists so that the CUDA library can be checked against it; nothing in the
+product path imports it, and it imports nothing from the CUDA package.  Only
+the tests, the smoke check and the CPU-baseline leg of the benchmark use it.
+
+What it follows (GaLore, arXiv 2403.03507):
+  * Algorithm 1 ("Adam with GaLore") for the step, read as follows where the
+    text leaves a choice:
+      - the moments M, V have the shape of the projected gradient R;
+      - the refresh test uses the number k of completed steps (k mod T == 0, so
+        the first step refreshes) and the bias correction uses t = k + 1;
+      - the bias-corrected moments are temporaries, the stored moments stay
+        uncorrected;
+      - epsilon is added outside the square root (Eq. 15);
+      - the caller passes the gradient (not its negative) and the update is
+        subtracted, which is the same trajectory;
+      - the moments are kept unchanged across a projector refresh.
+  * Sec. 4.2 ("Reducing memory usage of projection matrices") for the side:
+    R = P^T G when m <= n, R = G Q otherwise.
+  * Eq. 12-13 for the projector: the r leading left (right) singular vectors
+    of the current gradient.
+  * Sec. 4.3 ("8-bit optimizers") names block-wise 8-bit Adam states without
+    giving a format.  The format used here is this project's own and is
+    spelled out at `dynamic_code`; it is PARITY UNPINNED against the paper
+    (the paper fixes nothing to pin it to) and pinned only by its own
+    invariants in the tests.
+
+Storage emulation: arithmetic is always fp64; values are rounded when they are
+*stored* (weights to bf16 or fp32, moments to fp32 or to 8-bit codes), because
+that is part of what the step computes when the paper's BF16 / 8-bit settings
+are used.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SVD_SRC = os.path.join(_HERE, "jacobi_svd.c")
+_SVD_LIB = os.path.join(_HERE, "libjacobi_svd.so")
+_svd_handle = None
+
+
+def build_native(force: bool = False) -> str:
+    """Compile the Jacobi SVD (plain C, gcc) next to its source."""
+    if force or not os.path.exists(_SVD_LIB) or os.path.getmtime(_SVD_LIB) < os.path.getmtime(_SVD_SRC):
+        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", _SVD_LIB, _SVD_SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _SVD_LIB
+
+
+def _svd_lib():
+    global _svd_handle
+    if _svd_handle is None:
+        lib = ctypes.CDLL(build_native())
+        lib.jacobi_svd_rows.restype = ctypes.c_int
+        lib.jacobi_svd_rows.argtypes = [
+            ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
+            ctypes.c_void_p, ctypes.c_double, ctypes.c_int, ctypes.c_int]
+        _svd_handle = lib
+    return _svd_handle
+
+
+# --------------------------------------------------------------------------
+# Singular value decomposition and the projector (Eq. 12-13)
+# --------------------------------------------------------------------------
+
+def jacobi_svd(A, want_vt: bool = True, num_threads: int = 0):
+    """Full SVD A = U diag(S) Vt by one-sided Jacobi in fp64 (no LAPACK).
+
+    Returns U (a x k), S (k, descending), Vt (k x b) with k = min(a, b).
+    The native routine wants the short dimension as rows, so a tall input is
+    decomposed through its transpose (A^T = V S U^T).
+    """
+    A = np.ascontiguousarray(A, dtype=np.float64)
+    a, b = A.shape
+    if a > b:
+        V, S, Ut = jacobi_svd(A.T, want_vt=True, num_threads=num_threads)
+        return np.ascontiguousarray(Ut.T), S, np.ascontiguousarray(V.T)
+    U = np.empty((a, a), dtype=np.float64)
+    S = np.empty((a,), dtype=np.float64)
+    Vt = np.empty((a, b), dtype=np.float64) if want_vt else None
+    rc = _svd_lib().jacobi_svd_rows(
+        A.ctypes.data, a, b, U.ctypes.data, S.ctypes.data,
+        Vt.ctypes.data if want_vt else None, 1e-15, 60, num_threads)
+    if rc < 0:
+        raise RuntimeError(f"jacobi_svd_rows failed or did not converge (rc={rc})")
+    return U, S, Vt
+
+
+def top_r_projector(G, r: int, side: str, method: str = "jacobi"):
+    """Eq. 12-13: P = [u_1..u_r] (side 'left', m x r) or Q = [v_1..v_r] ('right', n x r).
+
+    method 'jacobi' is the oracle's own SVD.  method 'lapack' calls the library
+    SVD as a single step; it is for matrices too large for the Jacobi code to
+    finish in test time, and the tests check the two against each other.
+    Returns (projector, singular values).
+    """
+    G = np.asarray(G, dtype=np.float64)
+    if method == "jacobi":
+        U, S, Vt = jacobi_svd(G, want_vt=(side == "right"))
+    elif method == "lapack":
+        U, S, Vt = np.linalg.svd(G, full_matrices=False)
+    else:
+        raise ValueError(method)
+    if side == "left":
+        return np.ascontiguousarray(U[:, :r]), S
+    return np.ascontiguousarray(Vt[:r, :].T), S
+
+
+def largest_principal_angle(P_a, P_b) -> float:
+    """Largest principal angle (rad) between the column spans of two orthonormal bases.
+
+    cos of the principal angles are the singular values of P_a^T P_b; the
+    largest angle is taken from the sine, sqrt(lambda_max(I - C^T C)), so that
+    small angles are resolved (the arccos of a value near 1 is not).
+    """
+    P_a = np.asarray(P_a, dtype=np.float64)
+    P_b = np.asarray(P_b, dtype=np.float64)
+    # residual of P_b outside span(P_a); its largest singular value is sin(theta_max)
+    resid = P_b - P_a @ (P_a.T @ P_b)
+    s = np.linalg.norm(resid, 2)
+    return float(np.arcsin(min(1.0, s)))
+
+
+# --------------------------------------------------------------------------
+# Storage rounding
+# --------------------------------------------------------------------------
+
+def round_bf16(x):
+    """Round fp64 values to the nearest bfloat16 (8 significand bits, ties to even)."""
+    x = np.asarray(x, dtype=np.float64)
+    mant, expo = np.frexp(x)                      # x = mant * 2**expo, 0.5 <= |mant| < 1
+    mant = np.rint(mant * 256.0) / 256.0          # keep 8 significant bits; rint ties to even
+    return np.ldexp(mant, expo)
+
+
+def round_f32(x):
+    return np.asarray(x, dtype=np.float64).astype(np.float32).astype(np.float64)
+
+
+def _store(x, kind: str):
+    if kind == "f64":
+        return np.asarray(x, dtype=np.float64)
+    if kind == "f32":
+        return round_f32(x)
+    if kind == "bf16":
+        return round_bf16(x)
+    raise ValueError(kind)
+
+
+# --------------------------------------------------------------------------
+# 8-bit block-wise states (Sec. 4.3 names them; the format below is ours)
+# --------------------------------------------------------------------------
+
+def dynamic_code(signed: bool) -> np.ndarray:
+    """The 256 fp32 code values, ascending.
+
+    A non-uniform "dynamic" code on [-1, 1] (signed, first moment) or [0, 1]
+    (unsigned, second moment): decade e = 0, 1, 2, ... carries 2**f linearly
+    spaced magnitudes in (10**-(e+1), 10**-e], with f shrinking by one per
+    decade, so resolution follows magnitude.  Magnitude (e, j), j = 0..2**f-1:
+
+        (2**f + 9 (j + 1)) / (2**f * 10**(e + 1))          [one fp64 division]
+
+    unsigned: f = 7 - e, e = 0..7   -> 255 magnitudes, plus 0            = 256
+    signed  : f = 6 - e, e = 0..6   -> 127 magnitudes, both signs, plus 0
+              and one extra positive value 1e-7                          = 256
+    Both contain 0 and 1 exactly (signed also -1).
+    """
+    top = 7 if not signed else 6
+    mags = []
+    for e in range(top + 1):
+        f = top - e
+        for j in range(2 ** f):
+            mags.append((2 ** f + 9 * (j + 1)) / (2 ** f * 10 ** (e + 1)))
+    mags = sorted(mags)
+    if signed:
+        vals = [-v for v in reversed(mags)] + [0.0, 1.0 / 10 ** 7] + mags
+    else:
+        vals = [0.0] + mags
+    code = np.array(vals, dtype=np.float64).astype(np.float32)
+    assert code.shape == (256,)
+    return code
+
+
+def code_midpoints(code: np.ndarray) -> np.ndarray:
+    """fp32 decision thresholds between neighbouring code values."""
+    c = code.astype(np.float64)
+    return (0.5 * (c[:-1] + c[1:])).astype(np.float32)
+
+
+def quantize_blockwise(x, signed: bool, block: int = 2048):
+    """fp32 array -> (uint8 codes, fp32 absmax per block).
+
+    Blocks are runs of `block` consecutive elements of the flattened
+    (row-major) array; the last block may be shorter.  Per block:
+    absmax = max |x|;  y = x / absmax in fp32 (IEEE division);  the code is the
+    number of thresholds <= y, i.e. the nearest code value with ties going to
+    the larger index.  A block whose absmax is 0 stores the code of 0.
+    """
+    x32 = np.asarray(x, dtype=np.float32).reshape(-1)
+    n = x32.size
+    code = dynamic_code(signed)
+    mids = code_midpoints(code)
+    zero_code = int(np.nonzero(code == 0.0)[0][0])
+    nblk = (n + block - 1) // block
+    codes = np.empty(n, dtype=np.uint8)
+    absmax = np.zeros(nblk, dtype=np.float32)
+    for b in range(nblk):
+        seg = x32[b * block:(b + 1) * block]
+        a = np.float32(np.max(np.abs(seg))) if seg.size else np.float32(0)
+        absmax[b] = a
+        if a == 0:
+            codes[b * block:(b + 1) * block] = zero_code
+            continue
+        y = (seg / a).astype(np.float32)          # fp32 / fp32 -> IEEE fp32 quotient
+        codes[b * block:(b + 1) * block] = np.searchsorted(mids, y, side="right").astype(np.uint8)
+    return codes, absmax
+
+
+def dequantize_blockwise(codes, absmax, signed: bool, block: int = 2048):
+    """(codes, absmax) -> fp32 values: code value times the block's absmax, in fp32."""
+    codes = np.asarray(codes, dtype=np.uint8).reshape(-1)
+    code = dynamic_code(signed)
+    scale = np.repeat(np.asarray(absmax, dtype=np.float32), block)[:codes.size]
+    return (code[codes] * scale).astype(np.float32)
+
+
+# --------------------------------------------------------------------------
+# Algorithm 1
+# --------------------------------------------------------------------------
+
+class GaLoreOracle:
+    """One 2-D weight's GaLore-Adam state and step (Algorithm 1), in fp64.
+
+    w_store : 'f64' | 'f32' | 'bf16'   rounding applied to W when it is written
+    state   : 'f64' | 'f32' | 'q8'     how M, V are kept between steps
+    n_store : 'f64' | 'f32' | 'bf16'   rounding applied to the normalised update
+                                        before it is projected back (the CUDA
+                                        path feeds its tensor cores bf16)
+    inner   : 'adam' | 'identity'      the regulariser rho_t; 'identity' is the
+                                        rho_t = 1 case of Sec. 3.3 used by one pin
+    """
+
+    def __init__(self, m, n, rank, alpha, refresh_gap, beta1=0.9, beta2=0.999, eps=1e-8,
+                 side="auto", w_store="f64", state="f64", n_store="f64", q_block=2048,
+                 inner="adam", svd_method="jacobi"):
+        if side == "auto":
+            side = "left" if m <= n else "right"       # Sec. 4.2; m == n goes left
+        if rank < 1 or rank > min(m, n):
+            raise ValueError("rank must lie in [1, min(m, n)]")
+        self.m, self.n, self.r = int(m), int(n), int(rank)
+        self.alpha, self.T = float(alpha), int(refresh_gap)
+        self.beta1, self.beta2, self.eps = float(beta1), float(beta2), float(eps)
+        self.side, self.w_store, self.state, self.n_store = side, w_store, state, n_store
+        self.q_block, self.inner, self.svd_method = int(q_block), inner, svd_method
+        self.k = 0                                      # completed steps
+        self.proj = None                                # P (m x r) or Q (n x r)
+        self.sigma = None
+        shape = (self.r, self.n) if side == "left" else (self.m, self.r)
+        self.state_shape = shape
+        if state == "q8":
+            nel = shape[0] * shape[1]
+            nblk = (nel + self.q_block - 1) // self.q_block
+            zc_s = int(np.nonzero(dynamic_code(True) == 0.0)[0][0])
+            zc_u = int(np.nonzero(dynamic_code(False) == 0.0)[0][0])
+            self.M_codes = np.full(nel, zc_s, dtype=np.uint8)
+            self.V_codes = np.full(nel, zc_u, dtype=np.uint8)
+            self.M_absmax = np.zeros(nblk, dtype=np.float32)
+            self.V_absmax = np.zeros(nblk, dtype=np.float32)
+        else:
+            self.M = np.zeros(shape, dtype=np.float64)
+            self.V = np.zeros(shape, dtype=np.float64)
+        self.refreshes = 0
+
+    # -- state accessors ----------------------------------------------------
+    def moments(self):
+        """Stored (uncorrected) M, V as fp64 arrays of the state's shape."""
+        if self.state == "q8":
+            M = dequantize_blockwise(self.M_codes, self.M_absmax, True, self.q_block)
+            V = dequantize_blockwise(self.V_codes, self.V_absmax, False, self.q_block)
+            return (M.astype(np.float64).reshape(self.state_shape),
+                    V.astype(np.float64).reshape(self.state_shape))
+        return self.M, self.V
+
+    def optimizer_state_elements(self) -> int:
+        """Elements held besides W: projector plus two moments (Sec. 4.2: mr + 2nr for m <= n)."""
+        proj = (self.m if self.side == "left" else self.n) * self.r
+        return proj + 2 * self.state_shape[0] * self.state_shape[1]
+
+    def set_projector(self, proj):
+        proj = np.array(proj, dtype=np.float64)
+        want = (self.m if self.side == "left" else self.n, self.r)
+        if proj.shape != want:
+            raise ValueError(f"projector shape {proj.shape}, expected {want}")
+        self.proj = proj
+
+    # -- the refresh (Algorithm 1, the 't mod T = 0' branch; Eq. 12-13) ------
+    def refresh(self, G):
+        self.proj, self.sigma = top_r_projector(G, self.r, self.side, self.svd_method)
+        self.refreshes += 1
+        return self.proj
+
+    # -- one iteration of Algorithm 1 ---------------------------------------
+    def step(self, W, G, lr, auto_refresh=True):
+        W = np.asarray(W, dtype=np.float64)
+        G = np.asarray(G, dtype=np.float64)
+        if auto_refresh and self.k % self.T == 0:
+            self.refresh(G)
+        if self.proj is None:
+            raise RuntimeError("no projector: refresh or set_projector first")
+        P = self.proj
+        # project the gradient into the compact space
+        R = P.T @ G if self.side == "left" else G @ P
+        if self.inner == "identity":
+            N = R
+        else:
+            M_prev, V_prev = self.moments()
+            M = self.beta1 * M_prev + (1.0 - self.beta1) * R
+            V = self.beta2 * V_prev + (1.0 - self.beta2) * (R * R)
+            t = self.k + 1
+            M_hat = M / (1.0 - self.beta1 ** t)
+            V_hat = V / (1.0 - self.beta2 ** t)
+            N = M_hat / (np.sqrt(V_hat) + self.eps)
+            if self.state == "q8":
+                self.M_codes, self.M_absmax = quantize_blockwise(M, True, self.q_block)
+                self.V_codes, self.V_absmax = quantize_blockwise(V, False, self.q_block)
+            else:
+                self.M, self.V = _store(M, self.state), _store(V, self.state)
+        N = _store(N, self.n_store)
+        self.last_R, self.last_N = R, N
+        # project back and apply
+        G_tilde = self.alpha * (P @ N if self.side == "left" else N @ P.T)
+        W_new = _store(W - lr * G_tilde, self.w_store)
+        self.k += 1
+        return W_new
