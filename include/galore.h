@@ -1,0 +1,206 @@
+/*
+ * galore.h -- C ABI of the B200-native GaLore-Adam optimizer step.
+ *
+ * Implements, per 2-D weight W (m x n) with gradient G, one iteration of
+ * "Adam with GaLore" (arXiv 2403.03507, Algorithm 1):
+ *
+ *   refresh (every T steps)  P <- r leading left singular vectors of G      (Eq. 12-13)
+ *   project                  R <- P^T G           (m <= n, "left")          (Algorithm 1)
+ *                            R <- G Q             (m >  n, "right")         (Sec. 4.2)
+ *   Adam on R                M <- b1 M + (1-b1) R ; V <- b2 V + (1-b2) R*R
+ *                            N <- [M/(1-b1^t)] / (sqrt(V/(1-b2^t)) + eps)   (Eq. 15)
+ *   project back and apply   W <- W - lr * alpha * P N   (right: N Q^T)     (Algorithm 1)
+ *
+ * Conventions
+ *   - All matrix arguments are DEVICE pointers to row-major storage with a
+ *     leading dimension given in ELEMENTS, unless an argument says "host".
+ *   - The caller passes the gradient (not its negative) and the update is
+ *     subtracted.
+ *   - The library allocates no device memory: the optimizer state and a
+ *     scratch workspace are caller-allocated device buffers whose sizes come
+ *     from galore_query_bytes() and which must outlive the handle.  A
+ *     workspace may be shared by several layers that are never stepped
+ *     concurrently.
+ *   - A handle is used from one stream at a time.  Calls enqueue work on the
+ *     given stream (a cudaStream_t passed as void*; NULL = default stream) and
+ *     return without synchronising, except where stated.
+ *   - Every entry point returns a galore_status_t: 0 ok, > 0 warning, < 0
+ *     error.  Nothing throws or aborts across this boundary.  Conditions
+ *     detected on the device (non-finite values, a bounded wait that ran out)
+ *     are latched in a status word read by galore_device_status().
+ */
+#ifndef GALORE_H_
+#define GALORE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct galore_layer galore_layer_t; /* opaque, host memory, library-owned */
+
+typedef enum {
+  GALORE_OK = 0,
+  GALORE_WARN_NOT_CONVERGED = 1, /* refresh stopped at its iteration cap */
+  GALORE_ERR_INVALID_ARG = -1,
+  GALORE_ERR_SHAPE = -2,         /* rank outside [1, min(m, n)], non-positive sizes */
+  GALORE_ERR_ALIGNMENT = -3,     /* pointer or leading dimension not usable by the requested path */
+  GALORE_ERR_BUFFER_TOO_SMALL = -4,
+  GALORE_ERR_CUDA = -5,          /* a CUDA runtime/driver call failed; see galore_last_cuda_error() */
+  GALORE_ERR_STATE = -6,         /* e.g. a step without a projector when auto_refresh is off */
+  GALORE_ERR_NONFINITE = -7,
+  GALORE_ERR_TIMEOUT = -8,
+  GALORE_ERR_UNIMPLEMENTED = -9
+} galore_status_t;
+
+typedef enum { GALORE_SIDE_AUTO = 0, GALORE_SIDE_LEFT = 1, GALORE_SIDE_RIGHT = 2 } galore_side_t;
+typedef enum { GALORE_F32 = 0, GALORE_BF16 = 1 } galore_dtype_t;
+typedef enum { GALORE_STATE_F32 = 0, GALORE_STATE_Q8_BLOCK = 1 } galore_state_fmt_t;
+/* which kernels carry the two projections */
+typedef enum {
+  GALORE_PATH_AUTO = 0,   /* tensor cores when dtypes/alignment allow, else the fp32 path */
+  GALORE_PATH_FP32 = 1,   /* fp32 FMA kernels: any dtype, any leading dimension */
+  GALORE_PATH_TENSOR = 2  /* tcgen05 kernels; init fails with GALORE_ERR_ALIGNMENT/UNIMPLEMENTED if not eligible */
+} galore_path_t;
+
+/* Bits of the device status word. */
+enum {
+  GALORE_DEV_NONFINITE = 1,     /* a non-finite projected gradient was seen */
+  GALORE_DEV_WAIT_EXPIRED = 2,  /* a bounded device-side wait ran out */
+  GALORE_DEV_BOUNDS = 4         /* an internal index check failed */
+};
+
+/* Hyper-parameters of Algorithm 1 (rank r, scale alpha, refresh gap T, Adam's
+ * beta1/beta2/eps; the step size is a per-call argument because it follows a
+ * schedule) and the storage choices.  Zero-initialise, then fill. */
+typedef struct {
+  int64_t m, n;            /* W and G are m x n */
+  int32_t rank;            /* r, 1 <= r <= min(m, n) */
+  float alpha;             /* scale factor, not divided by r (Sec. 4.4) */
+  int32_t refresh_gap;     /* T >= 1 */
+  float beta1, beta2, eps;
+  int32_t side;            /* galore_side_t; AUTO = left iff m <= n (Sec. 4.2) */
+  int32_t w_dtype;         /* galore_dtype_t of W */
+  int32_t g_dtype;         /* galore_dtype_t of G */
+  int32_t p_dtype;         /* galore_dtype_t the projector is stored in */
+  int32_t state_fmt;       /* galore_state_fmt_t of M, V */
+  int32_t q_block;         /* elements per quantisation block: 256, 512, 1024, 2048 or 4096 (0 = 2048) */
+  int32_t auto_refresh;    /* 1: galore_step refreshes P when (completed steps) mod T == 0 */
+  int32_t path;            /* galore_path_t */
+  /* refresh: block subspace iteration on a block of rank + refresh_oversample
+   * columns (clipped to min(m, n); 0 = rank more columns, negative = none),
+   * stopped when the predicted subspace error (theta_b / theta_r)^iterations
+   * falls below refresh_tol or after refresh_max_iters power iterations.
+   * 0 = defaults (1e-4, 64). */
+  float refresh_tol;
+  int32_t refresh_max_iters;
+  int32_t refresh_oversample;
+  uint64_t seed;           /* start block of the subspace iteration */
+  int32_t reserved[8];
+} galore_config_t;
+
+/* Result of one refresh (host struct, filled after the refresh's stream work has completed). */
+typedef struct {
+  int32_t iterations;        /* power iterations run */
+  int32_t block;             /* columns iterated (rank + oversample, clipped) */
+  int32_t jacobi_sweeps;     /* sweeps of the last Rayleigh-Ritz eigen-solve */
+  int32_t converged;         /* 1 when the stated criterion was met */
+  double predicted_error;    /* (theta_b / theta_r)^iterations */
+  double residual;           /* || (G G^T) P - P Theta ||_F / (theta_1 sqrt(r)) for the kept Ritz pairs */
+  double sigma_r;            /* sqrt of the r-th Ritz value */
+  double sigma_next;         /* sqrt of the (r+1)-th Ritz value, 0 if block == rank */
+  double sigma_1;
+} galore_refresh_info_t;
+
+/* Sizes of the two caller-allocated device buffers for one layer.
+ * state_bytes covers P (rows x r, p_dtype), M and V (shape of R: r x n left,
+ * m x r right; fp32, or uint8 codes plus one fp32 absmax per block) -- the
+ * paper's  m r + 2 n r  elements for m <= n (Sec. 4.2).  Both buffers must be
+ * 256-byte aligned.  Host-only; touches no device. */
+galore_status_t galore_query_bytes(const galore_config_t* cfg, size_t* state_bytes, size_t* workspace_bytes);
+
+/* Creates a layer: validates cfg, lays out state_buf, zeroes M and V (stream
+ * work), sets the step counter to 0.  The projector is undefined until the
+ * first refresh or galore_set_projector().  *out is host memory owned by the
+ * library until galore_free(). */
+galore_status_t galore_init_layer(const galore_config_t* cfg, void* state_buf, size_t state_bytes,
+                                  void* workspace, size_t workspace_bytes, void* stream,
+                                  galore_layer_t** out);
+
+/* One iteration of Algorithm 1 on W (read and written in place) with gradient G
+ * (read only).  With auto_refresh the projector is refreshed from G first when
+ * the number of completed steps is a multiple of T (so the first step
+ * refreshes); a refresh synchronises the stream.  Increments the step counter. */
+galore_status_t galore_step(galore_layer_t* layer, void* W, int64_t ldw, const void* G, int64_t ldg,
+                            float lr, void* stream);
+
+/* Same step with W and G in HOST memory (pinned for asynchronous copies):
+ * copies both into the caller's device staging buffers (same dtype, packed,
+ * leading dimension n), steps, copies W back, all on `stream`. */
+galore_status_t galore_step_host(galore_layer_t* layer, void* W_host, const void* G_host,
+                                 void* W_dev_staging, void* G_dev_staging, float lr, void* stream);
+
+/* Steps `count` layers on one stream, layer i with W[i], G[i] (device pointers; host arrays of
+ * pointers and leading dimensions).  Equivalent to calling galore_step on each in order. */
+galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W, const int64_t* ldw,
+                                  const void* const* G, const int64_t* ldg, int32_t count, float lr,
+                                  void* stream);
+
+/* Recomputes the projector as the top-r singular subspace of G (Eq. 12-13) by
+ * block subspace iteration with a final Rayleigh-Ritz rotation, so that the
+ * stored columns approximate singular vectors in descending order of
+ * singular value.  M, V and the step counter are left untouched.
+ * Synchronises the stream.  info may be NULL.  Returns
+ * GALORE_WARN_NOT_CONVERGED when the iteration cap was reached first. */
+galore_status_t galore_refresh_projector(galore_layer_t* layer, const void* G, int64_t ldg, void* stream,
+                                         galore_refresh_info_t* info);
+
+/* Releases the host handle.  Device buffers stay with the caller. */
+galore_status_t galore_free(galore_layer_t* layer);
+
+/* ---- accessors (tests, checkpoint/resume) -------------------------------- */
+
+/* Projector as fp32, rows x r row-major packed (rows = m left, n right), device memory. */
+galore_status_t galore_get_projector(galore_layer_t* layer, float* dst, size_t dst_bytes, void* stream);
+galore_status_t galore_set_projector(galore_layer_t* layer, const float* src, size_t src_bytes, void* stream);
+/* Stored (uncorrected) moments as fp32, shape of R row-major packed, device memory (8-bit states are dequantised). */
+galore_status_t galore_get_moments(galore_layer_t* layer, float* M, float* V, size_t bytes_each, void* stream);
+/* Raw 8-bit state: codes (uint8, shape of R) and per-block absmax (fp32); device memory. */
+galore_status_t galore_get_q8_state(galore_layer_t* layer, uint8_t* M_codes, float* M_absmax,
+                                    uint8_t* V_codes, float* V_absmax, void* stream);
+/* Completed steps k.  A checkpoint is the caller's state buffer plus this counter. */
+galore_status_t galore_get_step_count(const galore_layer_t* layer, int64_t* k);
+galore_status_t galore_set_step_count(galore_layer_t* layer, int64_t k);
+/* Resolved side (galore_side_t), whether the tensor-core path is in use, and the state shape. */
+galore_status_t galore_layer_info(const galore_layer_t* layer, int32_t* side, int32_t* uses_tensor_path,
+                                  int64_t* state_rows, int64_t* state_cols);
+/* Synchronises `stream`, returns the device status bits and clears them. */
+galore_status_t galore_device_status(galore_layer_t* layer, int32_t* flags, void* stream);
+
+/* ---- 8-bit block-wise state format (Sec. 4.3 names 8-bit Adam states; the
+ *      format is this library's) ------------------------------------------- */
+
+/* The 256 fp32 code values, ascending, into host memory. is_signed != 0: the
+ * first-moment code on [-1, 1]; 0: the second-moment code on [0, 1]. */
+galore_status_t galore_q8_codebook(int32_t is_signed, float* out256_host);
+/* x (fp32, count elements, device) -> codes (uint8) and absmax (fp32, one per
+ * block of `block` consecutive elements, last block may be short).
+ * code = nearest code value to fp32(x / absmax), ties to the larger index. */
+galore_status_t galore_q8_quantize(const float* x, int64_t count, int32_t is_signed, int32_t block,
+                                   uint8_t* codes, float* absmax, void* stream);
+galore_status_t galore_q8_dequantize(const uint8_t* codes, const float* absmax, int64_t count,
+                                     int32_t is_signed, int32_t block, float* out, void* stream);
+
+/* ---- diagnostics ---------------------------------------------------------- */
+const char* galore_status_string(galore_status_t s);
+/* Text of the last CUDA error seen by this thread's calls into the library ("" if none). */
+const char* galore_last_cuda_error(void);
+/* Number of kernel launches issued by the library in this process (all layers). */
+int64_t galore_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GALORE_H_ */
