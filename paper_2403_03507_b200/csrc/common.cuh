@@ -1,0 +1,60 @@
+// Shared host/device helpers of the GaLore CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/galore.h"
+
+namespace galore {
+
+// ---- error plumbing ---------------------------------------------------------
+void note_cuda_error(cudaError_t e, const char* where);   // stores text for galore_last_cuda_error()
+void count_launch(int n = 1);
+
+#define GALORE_CUDA_TRY(expr)                                   \
+  do {                                                          \
+    cudaError_t e__ = (expr);                                   \
+    if (e__ != cudaSuccess) {                                   \
+      ::galore::note_cuda_error(e__, #expr);                    \
+      return GALORE_ERR_CUDA;                                   \
+    }                                                           \
+  } while (0)
+
+#define GALORE_TRY(expr)                          \
+  do {                                            \
+    galore_status_t s__ = (expr);                 \
+    if (s__ < 0) return s__;                      \
+  } while (0)
+
+// after a kernel launch: counts it and converts a launch failure into a status
+#define GALORE_LAUNCH_CHECK()                                   \
+  do {                                                          \
+    ::galore::count_launch();                                   \
+    cudaError_t e__ = cudaGetLastError();                       \
+    if (e__ != cudaSuccess) {                                   \
+      ::galore::note_cuda_error(e__, "kernel launch");          \
+      return GALORE_ERR_CUDA;                                   \
+    }                                                           \
+  } while (0)
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline size_t dtype_size(int32_t dt) { return dt == GALORE_BF16 ? 2 : 4; }
+
+// ---- element conversion -----------------------------------------------------
+template <typename To, typename From>
+__host__ __device__ __forceinline__ To cvt(From x) { return static_cast<To>(x); }
+template <> __device__ __forceinline__ float cvt<float, __nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <> __device__ __forceinline__ double cvt<double, __nv_bfloat16>(__nv_bfloat16 x) { return (double)__bfloat162float(x); }
+template <> __device__ __forceinline__ __nv_bfloat16 cvt<__nv_bfloat16, float>(float x) { return __float2bfloat16_rn(x); }
+template <> __device__ __forceinline__ __nv_bfloat16 cvt<__nv_bfloat16, double>(double x) { return __float2bfloat16_rn((float)x); }
+
+// Status word in the workspace (first 256 bytes).
+struct DeviceStatus {
+  int32_t flags;
+  int32_t pad[63];
+};
+
+}  // namespace galore

@@ -1,0 +1,170 @@
+// Stride-general FMA GEMM with a pluggable epilogue.
+//
+// C(i, j) = sum_k A(i, k) * B(k, j),  A(i, k) = A[i*sAi + k*sAk],  B(k, j) = B[k*sBk + j*sBj]
+//
+// This is the library's fp32/fp64 path: it takes any operand dtype, any
+// leading dimension and both transpositions, accumulates in TAcc (float or
+// double) and hands each finished element to an epilogue functor
+// epi(i, j, acc, split).  It carries the projections when the inputs are fp32
+// (where bf16 tensor-core inputs would break the fp32 tolerance) or not
+// TMA-aligned, and all fp64 work of the projector refresh.
+// blockIdx.z selects a K slice of `kchunk` elements (split-K).
+#pragma once
+
+#include "common.cuh"
+
+namespace galore {
+
+template <typename TA, typename TB, typename TAcc, int BM, int BN, int BK, int TM, int TN, class Epi>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN))
+gemm_simt_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int64_t sAk,
+                 const TB* __restrict__ B, int64_t sBk, int64_t sBj, int kchunk, Epi epi) {
+  constexpr int NT = (BM / TM) * (BN / TN);
+  constexpr int LA = BM * BK / NT;   // elements of the A tile each thread fetches
+  constexpr int LB = BN * BK / NT;
+  static_assert(BM * BK % NT == 0 && BN * BK % NT == 0, "tile/threads mismatch");
+  static_assert(TM % 4 == 0 && TN % 4 == 0, "micro-tile is built from groups of 4");
+  __shared__ TAcc As[BK][BM + 4];
+  __shared__ TAcc Bs[BK][BN + 4];
+
+  const int tid = threadIdx.x;
+  const int tx = tid % (BN / TN), ty = tid / (BN / TN);
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int k_begin = blockIdx.z * kchunk;
+  const int k_end = min(K, k_begin + kchunk);
+  const bool a_kfast = (sAk == 1);   // consecutive threads walk the contiguous direction
+  const bool b_kfast = (sBk == 1);
+
+  TAcc acc[TM][TN];
+#pragma unroll
+  for (int u = 0; u < TM; ++u)
+#pragma unroll
+    for (int v = 0; v < TN; ++v) acc[u][v] = TAcc(0);
+
+  TAcc ra[LA], rb[LB];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int e = 0; e < LA; ++e) {
+      int idx = tid + e * NT;
+      int i = a_kfast ? idx / BK : idx % BM;
+      int k = a_kfast ? idx % BK : idx / BM;
+      int gi = m0 + i, gk = k0 + k;
+      ra[e] = (gi < M && gk < k_end) ? cvt<TAcc>(A[(int64_t)gi * sAi + (int64_t)gk * sAk]) : TAcc(0);
+    }
+#pragma unroll
+    for (int e = 0; e < LB; ++e) {
+      int idx = tid + e * NT;
+      int j = b_kfast ? idx / BK : idx % BN;
+      int k = b_kfast ? idx % BK : idx / BN;
+      int gj = n0 + j, gk = k0 + k;
+      rb[e] = (gj < N && gk < k_end) ? cvt<TAcc>(B[(int64_t)gk * sBk + (int64_t)gj * sBj]) : TAcc(0);
+    }
+  };
+  auto stash = [&]() {
+#pragma unroll
+    for (int e = 0; e < LA; ++e) {
+      int idx = tid + e * NT;
+      int i = a_kfast ? idx / BK : idx % BM;
+      int k = a_kfast ? idx % BK : idx / BM;
+      As[k][i] = ra[e];
+    }
+#pragma unroll
+    for (int e = 0; e < LB; ++e) {
+      int idx = tid + e * NT;
+      int j = b_kfast ? idx / BK : idx % BN;
+      int k = b_kfast ? idx % BK : idx / BN;
+      Bs[k][j] = rb[e];
+    }
+  };
+
+  if (k_begin < k_end) fetch(k_begin);
+  for (int k0 = k_begin; k0 < k_end; k0 += BK) {
+    __syncthreads();
+    stash();
+    __syncthreads();
+    if (k0 + BK < k_end) fetch(k0 + BK);
+#pragma unroll
+    for (int k = 0; k < BK; ++k) {
+      TAcc a[TM], b[TN];
+#pragma unroll
+      for (int u = 0; u < TM; ++u) a[u] = As[k][(u / 4) * (BM / (TM / 4)) + ty * 4 + (u % 4)];
+#pragma unroll
+      for (int v = 0; v < TN; ++v) b[v] = Bs[k][(v / 4) * (BN / (TN / 4)) + tx * 4 + (v % 4)];
+#pragma unroll
+      for (int u = 0; u < TM; ++u)
+#pragma unroll
+        for (int v = 0; v < TN; ++v) acc[u][v] = fma(a[u], b[v], acc[u][v]);
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < TM; ++u) {
+    int i = m0 + (u / 4) * (BM / (TM / 4)) + ty * 4 + (u % 4);
+    if (i >= M) continue;
+#pragma unroll
+    for (int v = 0; v < TN; ++v) {
+      int j = n0 + (v / 4) * (BN / (TN / 4)) + tx * 4 + (v % 4);
+      if (j < N) epi(i, j, acc[u][v], (int)blockIdx.z);
+    }
+  }
+}
+
+// ---- epilogues ----------------------------------------------------------------
+
+// C[split][i][j] = alpha * acc  (+ beta * C when beta != 0; only with one split)
+template <typename TC, typename TAcc>
+struct EpiStore {
+  TC* C;
+  int64_t ldc;
+  int64_t split_stride;
+  TAcc alpha, beta;
+  __device__ __forceinline__ void operator()(int i, int j, TAcc acc, int z) const {
+    TC* p = C + (int64_t)z * split_stride + (int64_t)i * ldc + j;
+    TAcc v = alpha * acc;
+    if (beta != TAcc(0)) v += beta * cvt<TAcc>(*p);
+    *p = cvt<TC>(v);
+  }
+};
+
+// W[i][j] <- W[i][j] - scale * acc   (the weight update that closes Algorithm 1)
+template <typename TW>
+struct EpiApplyW {
+  TW* W;
+  int64_t ldw;
+  float scale;
+  __device__ __forceinline__ void operator()(int i, int j, float acc, int) const {
+    TW* p = W + (int64_t)i * ldw + j;
+    *p = cvt<TW>(fmaf(-scale, acc, cvt<float>(*p)));
+  }
+};
+
+template <typename TA, typename TB, typename TAcc, class Epi>
+galore_status_t launch_gemm_simt(int M, int N, int K, const TA* A, int64_t sAi, int64_t sAk, const TB* B,
+                                 int64_t sBk, int64_t sBj, int splits, Epi epi, cudaStream_t stream) {
+  if (M <= 0 || N <= 0) return GALORE_OK;
+  if (splits < 1) splits = 1;
+  int kchunk = (int)ceil_div(ceil_div(K, splits), 16) * 16;
+  if (kchunk < 16) kchunk = 16;
+  splits = (int)ceil_div(K > 0 ? K : 1, kchunk);
+  const bool small = (int64_t)M * N < (int64_t)128 * 128 * 96;
+  if (small) {
+    dim3 grid((unsigned)ceil_div(N, 64), (unsigned)ceil_div(M, 64), (unsigned)splits);
+    gemm_simt_kernel<TA, TB, TAcc, 64, 64, 16, 4, 4, Epi><<<grid, 256, 0, stream>>>(
+        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi);
+  } else {
+    dim3 grid((unsigned)ceil_div(N, 128), (unsigned)ceil_div(M, 128), (unsigned)splits);
+    gemm_simt_kernel<TA, TB, TAcc, 128, 128, 16, 8, 8, Epi><<<grid, 256, 0, stream>>>(
+        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi);
+  }
+  GALORE_LAUNCH_CHECK();
+  return GALORE_OK;
+}
+
+// number of K slices launch_gemm_simt will actually use for a request of `splits`
+inline int simt_effective_splits(int K, int splits) {
+  if (splits < 1) splits = 1;
+  int kchunk = (int)ceil_div(ceil_div(K, splits), 16) * 16;
+  if (kchunk < 16) kchunk = 16;
+  return (int)ceil_div(K > 0 ? K : 1, kchunk);
+}
+
+}  // namespace galore
