@@ -69,7 +69,8 @@ typedef enum {
 enum {
   GALORE_DEV_NONFINITE = 1,     /* a non-finite projected gradient was seen */
   GALORE_DEV_WAIT_EXPIRED = 2,  /* a bounded device-side wait ran out */
-  GALORE_DEV_BOUNDS = 4         /* an internal index check failed */
+  GALORE_DEV_BOUNDS = 4,        /* an internal index check failed */
+  GALORE_DEV_CHOLESKY = 8       /* a Gram matrix in the refresh was not positive definite */
 };
 
 /* Hyper-parameters of Algorithm 1 (rank r, scale alpha, refresh gap T, Adam's

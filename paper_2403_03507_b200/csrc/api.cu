@@ -1,0 +1,488 @@
+// C ABI of the GaLore-Adam step library: handle, buffer layout, argument
+// checks and the launch sequence of one iteration of Algorithm 1.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <atomic>
+#include <new>
+#include <string>
+
+#include "adam.cuh"
+#include "common.cuh"
+#include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+#include "refresh.cuh"
+
+namespace galore {
+
+static thread_local std::string t_last_error;
+static std::atomic<int64_t> g_launches{0};
+
+void note_cuda_error(cudaError_t e, const char* where) {
+  t_last_error = std::string(cudaGetErrorName(e)) + ": " + cudaGetErrorString(e) + " at " + where;
+}
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+template <typename TS, typename TD>
+__global__ void convert_copy_kernel(const TS* __restrict__ src, TD* __restrict__ dst, int64_t count) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+    dst[i] = cvt<TD>(src[i]);
+}
+
+}  // namespace galore
+
+using namespace galore;
+
+struct galore_layer {
+  galore_config_t cfg;
+  bool left;
+  bool tensor_path;
+  bool has_projector;
+  int64_t d;             // rows of the projector (m left, n right)
+  int64_t L;             // the other dimension of G
+  int64_t srows, scols;  // shape of R, M, V
+  int64_t nel;
+  int q_block;
+  int64_t nblk;
+  int block;             // columns of the refresh block
+  int proj_splits;       // K slices of the projection
+  int32_t n_dtype;       // dtype of the normalised update handed to the back-projection
+  int64_t k;             // completed steps
+  // device memory (all inside the caller's two buffers)
+  void* P;
+  float *M, *V;
+  uint8_t *Mc, *Vc;
+  float *Mam, *Vam;
+  int32_t* status;
+  float* Rpart;
+  void* Nbuf;
+  void* refresh_ws;
+  TensorPlan tc;         // tensor-map state of the tcgen05 path (unused on the fp32 path)
+};
+
+namespace {
+
+struct Sizes {
+  bool left;
+  int64_t d, L, srows, scols, nel, nblk;
+  int q_block, block, proj_splits;
+  bool tensor_path;
+  size_t off_P, off_M, off_V, off_Mam, off_Vam, state_bytes;
+  size_t off_status, off_R, off_N, off_refresh, ws_bytes;
+};
+
+galore_status_t resolve(const galore_config_t* c, Sizes* s) {
+  if (!c || !s) return GALORE_ERR_INVALID_ARG;
+  if (c->m <= 0 || c->n <= 0 || c->m > 0x7fffffff || c->n > 0x7fffffff) return GALORE_ERR_SHAPE;
+  if (c->rank < 1 || c->rank > std::min(c->m, c->n)) return GALORE_ERR_SHAPE;
+  if (c->refresh_gap < 1) return GALORE_ERR_INVALID_ARG;
+  if (!(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f) || !(c->eps >= 0.f))
+    return GALORE_ERR_INVALID_ARG;
+  if (c->side < GALORE_SIDE_AUTO || c->side > GALORE_SIDE_RIGHT) return GALORE_ERR_INVALID_ARG;
+  for (int32_t dt : {c->w_dtype, c->g_dtype, c->p_dtype})
+    if (dt != GALORE_F32 && dt != GALORE_BF16) return GALORE_ERR_INVALID_ARG;
+  if (c->state_fmt != GALORE_STATE_F32 && c->state_fmt != GALORE_STATE_Q8_BLOCK) return GALORE_ERR_INVALID_ARG;
+  if (c->path < GALORE_PATH_AUTO || c->path > GALORE_PATH_TENSOR) return GALORE_ERR_INVALID_ARG;
+  s->q_block = c->q_block == 0 ? 2048 : c->q_block;
+  if (s->q_block != 256 && s->q_block != 512 && s->q_block != 1024 && s->q_block != 2048 && s->q_block != 4096)
+    return GALORE_ERR_INVALID_ARG;
+  s->left = c->side == GALORE_SIDE_AUTO ? (c->m <= c->n) : (c->side == GALORE_SIDE_LEFT);
+  const int r = c->rank;
+  s->d = s->left ? c->m : c->n;
+  s->L = s->left ? c->n : c->m;
+  s->srows = s->left ? r : c->m;
+  s->scols = s->left ? c->n : r;
+  s->nel = s->srows * s->scols;
+  s->nblk = ceil_div(s->nel, s->q_block);
+  int over = c->refresh_oversample == 0 ? r : std::max(0, c->refresh_oversample);
+  s->block = (int)std::min<int64_t>(s->d, (int64_t)r + over);
+
+  const bool eligible = tensor_path_eligible(*c);
+  if (c->path == GALORE_PATH_TENSOR && !eligible) return GALORE_ERR_UNIMPLEMENTED;
+  s->tensor_path = eligible && c->path != GALORE_PATH_FP32;
+
+  // K slices of the projection: enough CTAs to fill the machine when R is small
+  if (s->tensor_path) {
+    s->proj_splits = tensor_proj_splits(*c, s->left);
+  } else {
+    const bool small = s->nel < (int64_t)128 * 128 * 96;
+    const int64_t t = small ? 64 : 128;
+    const int64_t tiles = ceil_div(s->srows, t) * ceil_div(s->scols, t);
+    int want = (int)std::min<int64_t>(16, std::max<int64_t>(1, ceil_div(2 * 148, tiles)));
+    want = (int)std::min<int64_t>(want, std::max<int64_t>(1, s->d / 64));
+    s->proj_splits = simt_effective_splits((int)s->d, want);
+  }
+
+  size_t o = 0;
+  s->off_P = o; o += align_up((size_t)s->d * r * dtype_size(c->p_dtype), 256);
+  if (c->state_fmt == GALORE_STATE_F32) {
+    s->off_M = o; o += align_up((size_t)s->nel * 4, 256);
+    s->off_V = o; o += align_up((size_t)s->nel * 4, 256);
+    s->off_Mam = s->off_Vam = o;
+  } else {
+    s->off_M = o; o += align_up((size_t)s->nel, 256);
+    s->off_V = o; o += align_up((size_t)s->nel, 256);
+    s->off_Mam = o; o += align_up((size_t)s->nblk * 4, 256);
+    s->off_Vam = o; o += align_up((size_t)s->nblk * 4, 256);
+  }
+  s->state_bytes = o;
+
+  o = 0;
+  s->off_status = o; o += 256;
+  s->off_R = o; o += align_up((size_t)s->proj_splits * s->nel * 4, 256);
+  s->off_N = o; o += align_up((size_t)s->nel * 4, 256);
+  s->off_refresh = o; o += refresh_workspace_bytes(s->d, s->L, r, s->block);
+  s->ws_bytes = o;
+  return GALORE_OK;
+}
+
+template <typename TS, typename TD>
+galore_status_t convert_copy(const TS* src, TD* dst, int64_t count, cudaStream_t st) {
+  if (count <= 0) return GALORE_OK;
+  unsigned grid = (unsigned)std::min<int64_t>(ceil_div(count, 256), 148 * 8);
+  convert_copy_kernel<TS, TD><<<grid, 256, 0, st>>>(src, dst, count);
+  GALORE_LAUNCH_CHECK();
+  return GALORE_OK;
+}
+
+// ---- the two projections on the fp32 path ------------------------------------------
+
+template <typename TP, typename TG>
+galore_status_t project_simt(galore_layer* l, const void* G, int64_t ldg, cudaStream_t st) {
+  const int r = l->cfg.rank;
+  EpiStore<float, float> epi{l->Rpart, l->scols, l->nel, 1.f, 0.f};
+  if (l->left)   // R (r x n) = P^T G
+    return launch_gemm_simt<TP, TG, float>(r, (int)l->cfg.n, (int)l->cfg.m, (const TP*)l->P, 1, r, (const TG*)G, ldg, 1,
+                                           l->proj_splits, epi, st);
+  // R (m x r) = G Q
+  return launch_gemm_simt<TG, TP, float>((int)l->cfg.m, r, (int)l->cfg.n, (const TG*)G, ldg, 1, (const TP*)l->P, r, 1,
+                                         l->proj_splits, epi, st);
+}
+
+template <typename TP, typename TW>
+galore_status_t back_project_simt(galore_layer* l, void* W, int64_t ldw, float scale, cudaStream_t st) {
+  const int r = l->cfg.rank;
+  const int m = (int)l->cfg.m, n = (int)l->cfg.n;
+  EpiApplyW<TW> epi{(TW*)W, ldw, scale};
+  const float* N = (const float*)l->Nbuf;
+  if (l->left)   // W -= scale * P N,  N is r x n
+    return launch_gemm_simt<TP, float, float>(m, n, r, (const TP*)l->P, r, 1, N, n, 1, 1, epi, st);
+  // W -= scale * N Q^T,  N is m x r
+  return launch_gemm_simt<float, TP, float>(m, n, r, N, r, 1, (const TP*)l->P, 1, r, 1, epi, st);
+}
+
+galore_status_t step_simt(galore_layer* l, void* W, int64_t ldw, const void* G, int64_t ldg, float lr,
+                          const AdamParams& ap, cudaStream_t st) {
+  const bool pb = l->cfg.p_dtype == GALORE_BF16, gb = l->cfg.g_dtype == GALORE_BF16, wb = l->cfg.w_dtype == GALORE_BF16;
+  if (pb && gb) GALORE_TRY((project_simt<__nv_bfloat16, __nv_bfloat16>(l, G, ldg, st)));
+  else if (pb) GALORE_TRY((project_simt<__nv_bfloat16, float>(l, G, ldg, st)));
+  else if (gb) GALORE_TRY((project_simt<float, __nv_bfloat16>(l, G, ldg, st)));
+  else GALORE_TRY((project_simt<float, float>(l, G, ldg, st)));
+
+  if (l->cfg.state_fmt == GALORE_STATE_F32)
+    GALORE_TRY(launch_adam_f32(l->Rpart, l->proj_splits, l->nel, l->nel, l->M, l->V, l->Nbuf, GALORE_F32, ap, l->status, st));
+  else
+    GALORE_TRY(launch_adam_q8(l->Rpart, l->proj_splits, l->nel, l->nel, l->Mc, l->Mam, l->Vc, l->Vam, l->q_block, l->Nbuf,
+                              GALORE_F32, ap, l->status, st));
+
+  const float scale = lr * l->cfg.alpha;
+  if (pb && wb) return back_project_simt<__nv_bfloat16, __nv_bfloat16>(l, W, ldw, scale, st);
+  if (pb) return back_project_simt<__nv_bfloat16, float>(l, W, ldw, scale, st);
+  if (wb) return back_project_simt<float, __nv_bfloat16>(l, W, ldw, scale, st);
+  return back_project_simt<float, float>(l, W, ldw, scale, st);
+}
+
+galore_status_t do_refresh(galore_layer* l, const void* G, int64_t ldg, cudaStream_t st, galore_refresh_info_t* info) {
+  RefreshProblem pr;
+  pr.G = G;
+  pr.g_dtype = l->cfg.g_dtype;
+  pr.ldg = ldg;
+  pr.m = l->cfg.m;
+  pr.n = l->cfg.n;
+  pr.left = l->left;
+  pr.rank = l->cfg.rank;
+  pr.block = l->block;
+  pr.P = l->P;
+  pr.p_dtype = l->cfg.p_dtype;
+  pr.seed = l->cfg.seed;
+  pr.tol = l->cfg.refresh_tol > 0.f ? (double)l->cfg.refresh_tol : 1e-4;
+  pr.max_iters = l->cfg.refresh_max_iters > 0 ? l->cfg.refresh_max_iters : 64;
+  pr.first_iters = 6;
+  galore_status_t s = refresh_projector(pr, l->refresh_ws, l->status, info, st);
+  if (s >= 0) l->has_projector = true;
+  return s;
+}
+
+}  // namespace
+
+extern "C" {
+
+galore_status_t galore_query_bytes(const galore_config_t* cfg, size_t* state_bytes, size_t* workspace_bytes) {
+  Sizes s;
+  GALORE_TRY(resolve(cfg, &s));
+  if (state_bytes) *state_bytes = s.state_bytes;
+  if (workspace_bytes) *workspace_bytes = s.ws_bytes;
+  return GALORE_OK;
+}
+
+galore_status_t galore_init_layer(const galore_config_t* cfg, void* state_buf, size_t state_bytes, void* workspace,
+                                  size_t workspace_bytes, void* stream, galore_layer_t** out) {
+  if (!out) return GALORE_ERR_INVALID_ARG;
+  *out = nullptr;
+  Sizes s;
+  GALORE_TRY(resolve(cfg, &s));
+  if (!state_buf || !workspace) return GALORE_ERR_INVALID_ARG;
+  if (((uintptr_t)state_buf | (uintptr_t)workspace) & 255) return GALORE_ERR_ALIGNMENT;
+  if (state_bytes < s.state_bytes || workspace_bytes < s.ws_bytes) return GALORE_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  galore_layer* l = new (std::nothrow) galore_layer();
+  if (!l) return GALORE_ERR_INVALID_ARG;
+  l->cfg = *cfg;
+  l->left = s.left;
+  l->tensor_path = s.tensor_path;
+  l->has_projector = false;
+  l->d = s.d; l->L = s.L; l->srows = s.srows; l->scols = s.scols; l->nel = s.nel;
+  l->q_block = s.q_block; l->nblk = s.nblk; l->block = s.block; l->proj_splits = s.proj_splits;
+  l->n_dtype = s.tensor_path ? GALORE_BF16 : GALORE_F32;
+  l->k = 0;
+  char* sb = (char*)state_buf;
+  char* ws = (char*)workspace;
+  l->P = sb + s.off_P;
+  l->M = l->V = nullptr; l->Mc = l->Vc = nullptr; l->Mam = l->Vam = nullptr;
+  if (cfg->state_fmt == GALORE_STATE_F32) {
+    l->M = (float*)(sb + s.off_M);
+    l->V = (float*)(sb + s.off_V);
+  } else {
+    l->Mc = (uint8_t*)(sb + s.off_M);
+    l->Vc = (uint8_t*)(sb + s.off_V);
+    l->Mam = (float*)(sb + s.off_Mam);
+    l->Vam = (float*)(sb + s.off_Vam);
+  }
+  l->status = (int32_t*)(ws + s.off_status);
+  l->Rpart = (float*)(ws + s.off_R);
+  l->Nbuf = ws + s.off_N;
+  l->refresh_ws = ws + s.off_refresh;
+
+  cudaError_t e = cudaSuccess;
+  if (cfg->state_fmt == GALORE_STATE_F32) {
+    e = cudaMemsetAsync(l->M, 0, (size_t)l->nel * 4, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(l->V, 0, (size_t)l->nel * 4, st);
+  } else {
+    e = cudaMemsetAsync(l->Mc, 127, (size_t)l->nel, st);   // 127 and 0 are the codes of the value 0
+    if (e == cudaSuccess) e = cudaMemsetAsync(l->Vc, 0, (size_t)l->nel, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(l->Mam, 0, (size_t)l->nblk * 4, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(l->Vam, 0, (size_t)l->nblk * 4, st);
+  }
+  if (e == cudaSuccess) e = cudaMemsetAsync(l->status, 0, 256, st);
+  if (e != cudaSuccess) {
+    note_cuda_error(e, "cudaMemsetAsync(state)");
+    delete l;
+    return GALORE_ERR_CUDA;
+  }
+  if (l->tensor_path) {
+    galore_status_t ts = tensor_plan_init(&l->tc, *cfg, l->left, l->P, l->Nbuf, l->Rpart, l->proj_splits);
+    if (ts < 0) {
+      delete l;
+      return ts;
+    }
+  }
+  *out = l;
+  return GALORE_OK;
+}
+
+galore_status_t galore_refresh_projector(galore_layer_t* l, const void* G, int64_t ldg, void* stream,
+                                         galore_refresh_info_t* info) {
+  if (!l || !G) return GALORE_ERR_INVALID_ARG;
+  if (ldg < l->cfg.n) return GALORE_ERR_INVALID_ARG;
+  return do_refresh(l, G, ldg, (cudaStream_t)stream, info);
+}
+
+galore_status_t galore_step(galore_layer_t* l, void* W, int64_t ldw, const void* G, int64_t ldg, float lr, void* stream) {
+  if (!l || !W || !G) return GALORE_ERR_INVALID_ARG;
+  if (ldw < l->cfg.n || ldg < l->cfg.n) return GALORE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  galore_status_t warn = GALORE_OK;
+  if (l->cfg.auto_refresh && l->k % l->cfg.refresh_gap == 0) {
+    galore_status_t s = do_refresh(l, G, ldg, st, nullptr);
+    if (s < 0) return s;
+    warn = s;
+  }
+  if (!l->has_projector) return GALORE_ERR_STATE;
+  const double t = (double)(l->k + 1);
+  AdamParams ap;
+  ap.b1 = l->cfg.beta1;
+  ap.b2 = l->cfg.beta2;
+  ap.omb1 = (float)(1.0 - (double)l->cfg.beta1);
+  ap.omb2 = (float)(1.0 - (double)l->cfg.beta2);
+  ap.eps = l->cfg.eps;
+  ap.inv_bc1 = (float)(1.0 / (1.0 - pow((double)l->cfg.beta1, t)));
+  ap.inv_bc2 = (float)(1.0 / (1.0 - pow((double)l->cfg.beta2, t)));
+  galore_status_t s;
+  if (l->tensor_path) {
+    if (!tensor_operands_aligned(l->cfg, W, ldw, G, ldg)) return GALORE_ERR_ALIGNMENT;
+    s = step_tensor(&l->tc, l->cfg, l->left, W, ldw, G, ldg, lr * l->cfg.alpha, ap, l->M, l->V, l->Mc, l->Mam, l->Vc,
+                    l->Vam, l->q_block, l->nel, l->status, st);
+  } else {
+    s = step_simt(l, W, ldw, G, ldg, lr, ap, st);
+  }
+  if (s < 0) return s;
+  l->k += 1;
+  return warn;
+}
+
+galore_status_t galore_step_host(galore_layer_t* l, void* W_host, const void* G_host, void* W_dev, void* G_dev, float lr,
+                                 void* stream) {
+  if (!l || !W_host || !G_host || !W_dev || !G_dev) return GALORE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t wb = (size_t)l->cfg.m * l->cfg.n * dtype_size(l->cfg.w_dtype);
+  const size_t gb = (size_t)l->cfg.m * l->cfg.n * dtype_size(l->cfg.g_dtype);
+  GALORE_CUDA_TRY(cudaMemcpyAsync(W_dev, W_host, wb, cudaMemcpyHostToDevice, st));
+  GALORE_CUDA_TRY(cudaMemcpyAsync(G_dev, G_host, gb, cudaMemcpyHostToDevice, st));
+  galore_status_t s = galore_step(l, W_dev, l->cfg.n, G_dev, l->cfg.n, lr, stream);
+  if (s < 0) return s;
+  GALORE_CUDA_TRY(cudaMemcpyAsync(W_host, W_dev, wb, cudaMemcpyDeviceToHost, st));
+  return s;
+}
+
+galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W, const int64_t* ldw, const void* const* G,
+                                  const int64_t* ldg, int32_t count, float lr, void* stream) {
+  if (count < 0 || (count > 0 && (!layers || !W || !ldw || !G || !ldg))) return GALORE_ERR_INVALID_ARG;
+  galore_status_t worst = GALORE_OK;
+  for (int32_t i = 0; i < count; ++i) {
+    galore_status_t s = galore_step(layers[i], W[i], ldw[i], G[i], ldg[i], lr, stream);
+    if (s < 0) return s;
+    if (s > worst) worst = s;
+  }
+  return worst;
+}
+
+galore_status_t galore_free(galore_layer_t* l) {
+  if (!l) return GALORE_ERR_INVALID_ARG;
+  delete l;
+  return GALORE_OK;
+}
+
+galore_status_t galore_get_projector(galore_layer_t* l, float* dst, size_t dst_bytes, void* stream) {
+  if (!l || !dst) return GALORE_ERR_INVALID_ARG;
+  const int64_t count = l->d * l->cfg.rank;
+  if (dst_bytes < (size_t)count * 4) return GALORE_ERR_BUFFER_TOO_SMALL;
+  if (!l->has_projector) return GALORE_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (l->cfg.p_dtype == GALORE_BF16) return convert_copy((const __nv_bfloat16*)l->P, dst, count, st);
+  GALORE_CUDA_TRY(cudaMemcpyAsync(dst, l->P, (size_t)count * 4, cudaMemcpyDeviceToDevice, st));
+  return GALORE_OK;
+}
+
+galore_status_t galore_set_projector(galore_layer_t* l, const float* src, size_t src_bytes, void* stream) {
+  if (!l || !src) return GALORE_ERR_INVALID_ARG;
+  const int64_t count = l->d * l->cfg.rank;
+  if (src_bytes < (size_t)count * 4) return GALORE_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (l->cfg.p_dtype == GALORE_BF16) {
+    GALORE_TRY(convert_copy(src, (__nv_bfloat16*)l->P, count, st));
+  } else {
+    GALORE_CUDA_TRY(cudaMemcpyAsync(l->P, src, (size_t)count * 4, cudaMemcpyDeviceToDevice, st));
+  }
+  l->has_projector = true;
+  return GALORE_OK;
+}
+
+galore_status_t galore_get_moments(galore_layer_t* l, float* M, float* V, size_t bytes_each, void* stream) {
+  if (!l || !M || !V) return GALORE_ERR_INVALID_ARG;
+  if (bytes_each < (size_t)l->nel * 4) return GALORE_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (l->cfg.state_fmt == GALORE_STATE_F32) {
+    GALORE_CUDA_TRY(cudaMemcpyAsync(M, l->M, (size_t)l->nel * 4, cudaMemcpyDeviceToDevice, st));
+    GALORE_CUDA_TRY(cudaMemcpyAsync(V, l->V, (size_t)l->nel * 4, cudaMemcpyDeviceToDevice, st));
+    return GALORE_OK;
+  }
+  GALORE_TRY(launch_q8_dequantize(l->Mc, l->Mam, l->nel, 1, l->q_block, M, st));
+  return launch_q8_dequantize(l->Vc, l->Vam, l->nel, 0, l->q_block, V, st);
+}
+
+galore_status_t galore_get_q8_state(galore_layer_t* l, uint8_t* Mc, float* Mam, uint8_t* Vc, float* Vam, void* stream) {
+  if (!l || !Mc || !Mam || !Vc || !Vam) return GALORE_ERR_INVALID_ARG;
+  if (l->cfg.state_fmt != GALORE_STATE_Q8_BLOCK) return GALORE_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  GALORE_CUDA_TRY(cudaMemcpyAsync(Mc, l->Mc, (size_t)l->nel, cudaMemcpyDeviceToDevice, st));
+  GALORE_CUDA_TRY(cudaMemcpyAsync(Vc, l->Vc, (size_t)l->nel, cudaMemcpyDeviceToDevice, st));
+  GALORE_CUDA_TRY(cudaMemcpyAsync(Mam, l->Mam, (size_t)l->nblk * 4, cudaMemcpyDeviceToDevice, st));
+  GALORE_CUDA_TRY(cudaMemcpyAsync(Vam, l->Vam, (size_t)l->nblk * 4, cudaMemcpyDeviceToDevice, st));
+  return GALORE_OK;
+}
+
+galore_status_t galore_get_step_count(const galore_layer_t* l, int64_t* k) {
+  if (!l || !k) return GALORE_ERR_INVALID_ARG;
+  *k = l->k;
+  return GALORE_OK;
+}
+
+galore_status_t galore_set_step_count(galore_layer_t* l, int64_t k) {
+  if (!l || k < 0) return GALORE_ERR_INVALID_ARG;
+  l->k = k;
+  return GALORE_OK;
+}
+
+galore_status_t galore_layer_info(const galore_layer_t* l, int32_t* side, int32_t* uses_tensor_path, int64_t* state_rows,
+                                  int64_t* state_cols) {
+  if (!l) return GALORE_ERR_INVALID_ARG;
+  if (side) *side = l->left ? GALORE_SIDE_LEFT : GALORE_SIDE_RIGHT;
+  if (uses_tensor_path) *uses_tensor_path = l->tensor_path ? 1 : 0;
+  if (state_rows) *state_rows = l->srows;
+  if (state_cols) *state_cols = l->scols;
+  return GALORE_OK;
+}
+
+galore_status_t galore_device_status(galore_layer_t* l, int32_t* flags, void* stream) {
+  if (!l || !flags) return GALORE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t f = 0;
+  GALORE_CUDA_TRY(cudaMemcpyAsync(&f, l->status, sizeof(f), cudaMemcpyDeviceToHost, st));
+  GALORE_CUDA_TRY(cudaMemsetAsync(l->status, 0, sizeof(f), st));
+  GALORE_CUDA_TRY(cudaStreamSynchronize(st));
+  *flags = f;
+  return GALORE_OK;
+}
+
+galore_status_t galore_q8_codebook(int32_t is_signed, float* out256_host) {
+  if (!out256_host) return GALORE_ERR_INVALID_ARG;
+  q8_host_codebook(is_signed != 0, out256_host);
+  return GALORE_OK;
+}
+
+galore_status_t galore_q8_quantize(const float* x, int64_t count, int32_t is_signed, int32_t block, uint8_t* codes,
+                                   float* absmax, void* stream) {
+  if (count < 0 || (count > 0 && (!x || !codes || !absmax))) return GALORE_ERR_INVALID_ARG;
+  return launch_q8_quantize(x, count, is_signed, block == 0 ? 2048 : block, codes, absmax, (cudaStream_t)stream);
+}
+
+galore_status_t galore_q8_dequantize(const uint8_t* codes, const float* absmax, int64_t count, int32_t is_signed,
+                                     int32_t block, float* out, void* stream) {
+  if (count < 0 || (count > 0 && (!codes || !absmax || !out))) return GALORE_ERR_INVALID_ARG;
+  return launch_q8_dequantize(codes, absmax, count, is_signed, block == 0 ? 2048 : block, out, (cudaStream_t)stream);
+}
+
+const char* galore_status_string(galore_status_t s) {
+  switch (s) {
+    case GALORE_OK: return "ok";
+    case GALORE_WARN_NOT_CONVERGED: return "refresh reached its iteration cap before the stated convergence";
+    case GALORE_ERR_INVALID_ARG: return "invalid argument";
+    case GALORE_ERR_SHAPE: return "invalid shape or rank";
+    case GALORE_ERR_ALIGNMENT: return "pointer or leading dimension not aligned for this path";
+    case GALORE_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+    case GALORE_ERR_CUDA: return "CUDA call failed";
+    case GALORE_ERR_STATE: return "layer state does not allow this call";
+    case GALORE_ERR_NONFINITE: return "non-finite values";
+    case GALORE_ERR_TIMEOUT: return "a bounded device wait ran out";
+    case GALORE_ERR_UNIMPLEMENTED: return "not implemented for this configuration";
+  }
+  return "unknown status";
+}
+
+const char* galore_last_cuda_error(void) { return t_last_error.c_str(); }
+
+int64_t galore_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

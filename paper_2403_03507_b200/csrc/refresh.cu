@@ -1,0 +1,525 @@
+// Projector refresh: the top-r singular subspace of the current gradient
+// (Algorithm 1, the "t mod T = 0" branch; Eq. 12-13), computed on the GPU by
+// block subspace iteration instead of a full SVD.
+//
+// With A = G (left projector, d = m, L = n) or A = G^T (right, d = n, L = m):
+//
+//   Y (d x b) random, b = r + oversample                     start block
+//   repeat:  Z = A^T Y ;  Y' = A Z + delta Y ;  Y = orth(Y')  power step on A A^T + delta I,
+//                                                            never forming A A^T
+//   Rayleigh-Ritz:  Y orthonormalised in fp64;  Z = A^T Y;  H = Z^T Z = Y^T A A^T Y;
+//                   H = S Theta S^T by parallel one-sided Jacobi;  P = Y S[:, top r]
+//
+// orth() is CholeskyQR (Gram matrix in fp64, blocked Cholesky, blocked
+// triangular solve).  The tiny shift delta keeps Y at full column rank when G
+// itself has rank < b (it moves every eigenvalue by delta and no eigenvector).
+// The power steps only have to bring span(Y) close to the wanted subspace, so
+// they run in fp32; what fixes the accuracy of P is the last orthonormalisation
+// and the Rayleigh-Ritz step, which run in fp64.
+//
+// Stated convergence: after q power steps the error of the top-r subspace
+// decays like (theta_b / theta_r)^q (theta = Ritz values, descending); the
+// iteration stops when that prediction is below the tolerance, or at the cap.
+#include "refresh.cuh"
+
+#include <math.h>
+
+#include <algorithm>
+#include <vector>
+
+#include "gemm_simt.cuh"
+
+namespace galore {
+
+// ---------------------------------------------------------------------------
+// small kernels
+// ---------------------------------------------------------------------------
+
+__device__ __forceinline__ uint64_t mix64(uint64_t x) {   // splitmix64 finaliser
+  x += 0x9E3779B97F4A7C15ull;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  return x ^ (x >> 31);
+}
+
+// standard normal start block from a counter-based hash (Box-Muller)
+__global__ void fill_normal_kernel(float* __restrict__ Y, int64_t count, uint64_t seed) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x) {
+    uint64_t h = mix64(seed ^ mix64((uint64_t)i));
+    float u1 = ((uint32_t)(h >> 40) + 1u) * (1.0f / 16777217.0f);   // (0, 1)
+    float u2 = (uint32_t)(h & 0xFFFFFFu) * (1.0f / 16777216.0f);    // [0, 1)
+    Y[i] = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
+  }
+}
+
+__global__ void set_identity_kernel(double* __restrict__ A, int n) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < (int64_t)n * n; i += (int64_t)gridDim.x * blockDim.x)
+    A[i] = (i / n == i % n) ? 1.0 : 0.0;
+}
+
+template <typename TS, typename TD>
+__global__ void convert_kernel(const TS* __restrict__ src, TD* __restrict__ dst, int64_t count) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+    dst[i] = cvt<TD>(src[i]);
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// every thread of a 256-thread CTA gets the sum
+__device__ __forceinline__ double block_sum_256(double v, double* red) {
+  v = warp_sum(v);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  double r = 0.0;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) r += red[w];
+  __syncthreads();
+  return r;
+}
+
+// scal[0] += sum of squares
+__global__ void __launch_bounds__(256) sumsq_kernel(const float* __restrict__ x, int64_t count, double* __restrict__ scal) {
+  __shared__ double red[8];
+  double s = 0.0;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x) {
+    double v = x[i];
+    s += v * v;
+  }
+  s = block_sum_256(s, red);
+  if (threadIdx.x == 0) atomicAdd(scal, s);
+}
+
+// Ynew += delta * Yold,  delta = max(1e-4 * rms column norm of Ynew, 1e-30)
+__global__ void shift_kernel(float* __restrict__ Ynew, const float* __restrict__ Yold, int64_t count, int cols,
+                             const double* __restrict__ scal) {
+  const float delta = fmaxf((float)(1e-4 * sqrt(scal[0] / (double)cols)), 1e-30f);
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+    Ynew[i] = fmaf(delta, Yold[i], Ynew[i]);
+}
+
+// ---- Cholesky of one diagonal block (nb <= 64) and the inverse of its factor ----
+// C: the block inside a row-major matrix with leading dimension ld (lower triangle used and
+// overwritten with L).  Linv: 64 x 64 row-major, lower triangular, zero elsewhere.
+__global__ void __launch_bounds__(256) potf2_inv_kernel(double* __restrict__ C, int ld, int nb, double* __restrict__ Linv,
+                                                        int32_t* __restrict__ status) {
+  __shared__ double L[64][65];
+  const int tid = threadIdx.x;
+  for (int idx = tid; idx < 64 * 64; idx += 256) {
+    int i = idx / 64, j = idx % 64;
+    L[i][j] = (i < nb && j <= i) ? C[(int64_t)i * ld + j] : 0.0;
+    Linv[idx] = 0.0;
+  }
+  __syncthreads();
+  for (int j = 0; j < nb; ++j) {
+    if (tid == 0) {
+      double piv = L[j][j];
+      if (!(piv > 0.0)) {              // not positive definite: keep going with a usable pivot, latch the fact
+        atomicOr(status, GALORE_DEV_CHOLESKY);
+        piv = fabs(piv) + 1e-300;
+      }
+      L[j][j] = sqrt(piv);
+    }
+    __syncthreads();
+    const double inv = 1.0 / L[j][j];
+    for (int i = j + 1 + tid; i < nb; i += 256) L[i][j] *= inv;
+    __syncthreads();
+    // trailing update of the lower triangle: L[i][k] -= L[i][j] * L[k][j], j < k <= i
+    const int rem = nb - j - 1;
+    for (int idx = tid; idx < rem * rem; idx += 256) {
+      int i = j + 1 + idx / rem, k = j + 1 + idx % rem;
+      if (k <= i) L[i][k] -= L[i][j] * L[k][j];
+    }
+    __syncthreads();
+  }
+  // inverse by forward substitution, one column per thread (L x = e_c); each thread reads back
+  // only its own column of Linv
+  if (tid < nb) {
+    const int c = tid;
+    for (int i = c; i < nb; ++i) {
+      double s = (i == c) ? 1.0 : 0.0;
+      for (int k = c; k < i; ++k) s -= L[i][k] * Linv[k * 64 + c];
+      Linv[i * 64 + c] = s / L[i][i];
+    }
+  }
+  for (int idx = tid; idx < 64 * 64; idx += 256) {
+    int i = idx / 64, j = idx % 64;
+    if (i < nb && j <= i) C[(int64_t)i * ld + j] = L[i][j];
+  }
+}
+
+// dst = src - acc   (one panel step of the blocked triangular solve)
+template <typename TS>
+struct EpiResidual {
+  const TS* src;
+  int64_t ldsrc;
+  double* dst;
+  int64_t lddst;
+  __device__ __forceinline__ void operator()(int i, int j, double acc, int) const {
+    dst[(int64_t)i * lddst + j] = cvt<double>(src[(int64_t)i * ldsrc + j]) - acc;
+  }
+};
+
+// ---- parallel one-sided Jacobi on a symmetric matrix -------------------------------
+// X starts as H, Vt as the identity.  A rotation of rows (p, q) that makes the
+// two rows of X orthogonal is applied to X and to Vt; at convergence
+// X = Theta V^T, so row norms are the eigenvalues and rows of Vt the eigenvectors.
+// One launch handles one round of the round-robin schedule: np/2 disjoint pairs.
+__global__ void __launch_bounds__(256) jacobi_round_kernel(double* __restrict__ X, double* __restrict__ Vt, int b, int np,
+                                                           int round, double tol, int* __restrict__ rotations) {
+  __shared__ double red[8];
+  const int k = blockIdx.x;
+  auto player = [&](int pos) { return pos == 0 ? 0 : 1 + (((pos - 1 - round) % (np - 1)) + (np - 1)) % (np - 1); };
+  int p = player(k), q = player(np - 1 - k);
+  if (p >= b || q >= b) return;
+  if (p > q) { int t = p; p = q; q = t; }
+  double* xp = X + (int64_t)p * b;
+  double* xq = X + (int64_t)q * b;
+  double app = 0.0, aqq = 0.0, apq = 0.0;
+  for (int j = threadIdx.x; j < b; j += 256) {
+    double a = xp[j], c = xq[j];
+    app += a * a;
+    aqq += c * c;
+    apq += a * c;
+  }
+  app = block_sum_256(app, red);
+  aqq = block_sum_256(aqq, red);
+  apq = block_sum_256(apq, red);
+  if (apq == 0.0 || fabs(apq) <= tol * sqrt(app * aqq)) return;
+  const double zeta = (aqq - app) / (2.0 * apq);
+  const double t = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+  const double c = 1.0 / sqrt(1.0 + t * t);
+  const double s = c * t;
+  double* vp = Vt + (int64_t)p * b;
+  double* vq = Vt + (int64_t)q * b;
+  for (int j = threadIdx.x; j < b; j += 256) {
+    double a = xp[j], d = xq[j];
+    xp[j] = c * a - s * d;
+    xq[j] = s * a + c * d;
+    a = vp[j];
+    d = vq[j];
+    vp[j] = c * a - s * d;
+    vq[j] = s * a + c * d;
+  }
+  if (threadIdx.x == 0) atomicAdd(rotations, 1);
+}
+
+__global__ void __launch_bounds__(256) row_norm_kernel(const double* __restrict__ X, int b, double* __restrict__ lam) {
+  __shared__ double red[8];
+  const double* x = X + (int64_t)blockIdx.x * b;
+  double s = 0.0;
+  for (int j = threadIdx.x; j < b; j += 256) s += x[j] * x[j];
+  s = block_sum_256(s, red);
+  if (threadIdx.x == 0) lam[blockIdx.x] = sqrt(s);
+}
+
+// descending order by counting: theta[rank] = lam[i], order[rank] = i
+__global__ void rank_desc_kernel(const double* __restrict__ lam, int b, double* __restrict__ theta, int* __restrict__ order) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= b) return;
+  const double li = lam[i];
+  int rank = 0;
+  for (int j = 0; j < b; ++j) {
+    double lj = lam[j];
+    rank += (lj > li) || (lj == li && j < i);
+  }
+  theta[rank] = li;
+  order[rank] = i;
+}
+
+__global__ void gather_rows_kernel(const double* __restrict__ Vt, const int* __restrict__ order, int b,
+                                   double* __restrict__ Vsel) {
+  const double* src = Vt + (int64_t)order[blockIdx.x] * b;
+  double* dst = Vsel + (int64_t)blockIdx.x * b;
+  for (int j = threadIdx.x; j < b; j += blockDim.x) dst[j] = src[j];
+}
+
+// scal[1] += || T2 - P diag(theta) ||_F^2
+__global__ void __launch_bounds__(256) residual_kernel(const double* __restrict__ T2, const double* __restrict__ P,
+                                                       const double* __restrict__ theta, int64_t rows, int r,
+                                                       double* __restrict__ scal) {
+  __shared__ double red[8];
+  double s = 0.0;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < rows * r; i += (int64_t)gridDim.x * blockDim.x) {
+    double d = T2[i] - theta[i % r] * P[i];
+    s += d * d;
+  }
+  s = block_sum_256(s, red);
+  if (threadIdx.x == 0) atomicAdd(scal + 1, s);
+}
+
+static inline unsigned grid_for(int64_t count) { return (unsigned)std::min<int64_t>(ceil_div(count, 256), 148 * 8); }
+
+// ---------------------------------------------------------------------------
+// workspace
+// ---------------------------------------------------------------------------
+
+struct RefreshBuffers {
+  float* Ya;      // d x b
+  float* Yb;      // d x b
+  void* Zu;       // L x b, fp32 during power steps, fp64 during Rayleigh-Ritz
+  double* Y64;    // d x b
+  double* C;      // b x b  Gram / Cholesky factor
+  double* H;      // b x b  Jacobi working matrix
+  double* Vt;     // b x b
+  double* P64;    // d x r
+  double* Vsel;   // r x b
+  double* tmp;    // d x 64
+  double* Linv;   // 64 x 64
+  double* lam;    // b
+  double* theta;  // b
+  int* order;     // b
+  double* scal;   // 4 scalars
+  int* counter;   // 1
+};
+
+static size_t carve(char*& p, size_t bytes) {
+  size_t a = align_up(bytes, 256);
+  p += a;
+  return a;
+}
+
+size_t refresh_workspace_bytes(int64_t d, int64_t L, int r, int b) {
+  size_t t = 0;
+  t += align_up((size_t)d * b * 4, 256) * 2;
+  t += align_up((size_t)L * b * 8, 256);
+  t += align_up((size_t)d * b * 8, 256);
+  t += align_up((size_t)b * b * 8, 256) * 3;
+  t += align_up((size_t)d * r * 8, 256);
+  t += align_up((size_t)r * b * 8, 256);
+  t += align_up((size_t)d * 64 * 8, 256);
+  t += align_up((size_t)64 * 64 * 8, 256);
+  t += align_up((size_t)b * 8, 256) * 2;
+  t += align_up((size_t)b * 4, 256);
+  t += 256 * 2;
+  return t;
+}
+
+static RefreshBuffers layout(void* base, int64_t d, int64_t L, int r, int b) {
+  RefreshBuffers w;
+  char* p = (char*)base;
+  w.Ya = (float*)p; carve(p, (size_t)d * b * 4);
+  w.Yb = (float*)p; carve(p, (size_t)d * b * 4);
+  w.Zu = (void*)p; carve(p, (size_t)L * b * 8);
+  w.Y64 = (double*)p; carve(p, (size_t)d * b * 8);
+  w.C = (double*)p; carve(p, (size_t)b * b * 8);
+  w.H = (double*)p; carve(p, (size_t)b * b * 8);
+  w.Vt = (double*)p; carve(p, (size_t)b * b * 8);
+  w.P64 = (double*)p; carve(p, (size_t)d * r * 8);
+  w.Vsel = (double*)p; carve(p, (size_t)r * b * 8);
+  w.tmp = (double*)p; carve(p, (size_t)d * 64 * 8);
+  w.Linv = (double*)p; carve(p, (size_t)64 * 64 * 8);
+  w.lam = (double*)p; carve(p, (size_t)b * 8);
+  w.theta = (double*)p; carve(p, (size_t)b * 8);
+  w.order = (int*)p; carve(p, (size_t)b * 4);
+  w.scal = (double*)p; carve(p, 256);
+  w.counter = (int*)p; carve(p, 256);
+  return w;
+}
+
+// ---------------------------------------------------------------------------
+// building blocks
+// ---------------------------------------------------------------------------
+
+// C (b x b, fp64) = Y^T Y
+template <typename TY>
+static galore_status_t gram(const TY* Y, int64_t d, int b, double* C, cudaStream_t st) {
+  EpiStore<double, double> epi{C, b, 0, 1.0, 0.0};
+  return launch_gemm_simt<TY, TY, double>(b, b, (int)d, Y, 1, b, Y, b, 1, 1, epi, st);
+}
+
+// In-place blocked Cholesky of the b x b matrix C (lower), and Y <- Y L^-T.
+template <typename TY>
+static galore_status_t cholesky_solve(TY* Y, int64_t d, int b, double* C, const RefreshBuffers& w, int32_t* status,
+                                      cudaStream_t st) {
+  for (int j0 = 0; j0 < b; j0 += 64) {
+    const int nb = std::min(64, b - j0);
+    const int j1 = j0 + nb;
+    // solve for the panel of Y first needs L[J, <J], which earlier panels completed
+    if (j0 > 0) {
+      // tmp = Y[:, J] - Y[:, <J] L[J, <J]^T
+      EpiResidual<TY> epi{Y + j0, b, w.tmp, 64};
+      GALORE_TRY((launch_gemm_simt<TY, double, double>((int)d, nb, j0, Y, b, 1, C + (int64_t)j0 * b, 1, b, 1, epi, st)));
+    } else {
+      EpiResidual<TY> epi{Y, b, w.tmp, 64};
+      GALORE_TRY((launch_gemm_simt<TY, double, double>((int)d, nb, 0, Y, b, 1, C, 1, b, 1, epi, st)));
+    }
+    potf2_inv_kernel<<<1, 256, 0, st>>>(C + (int64_t)j0 * b + j0, b, nb, w.Linv, status);
+    GALORE_LAUNCH_CHECK();
+    // Y[:, J] = tmp Linv^T
+    {
+      EpiStore<TY, double> epi{Y + j0, b, 0, 1.0, 0.0};
+      GALORE_TRY((launch_gemm_simt<double, double, double>((int)d, nb, nb, w.tmp, 64, 1, w.Linv, 1, 64, 1, epi, st)));
+    }
+    if (j1 < b) {
+      const int rem = b - j1;
+      // L[rest, J] = C[rest, J] Linv^T   (in place: one CTA column covers all nb columns)
+      EpiStore<double, double> epi{C + (int64_t)j1 * b + j0, b, 0, 1.0, 0.0};
+      GALORE_TRY((launch_gemm_simt<double, double, double>(rem, nb, nb, C + (int64_t)j1 * b + j0, b, 1, w.Linv, 1, 64, 1, epi, st)));
+      // C[rest, rest] -= L[rest, J] L[rest, J]^T
+      EpiStore<double, double> upd{C + (int64_t)j1 * b + j1, b, 0, -1.0, 1.0};
+      GALORE_TRY((launch_gemm_simt<double, double, double>(rem, rem, nb, C + (int64_t)j1 * b + j0, b, 1,
+                                                           C + (int64_t)j1 * b + j0, 1, b, 1, upd, st)));
+    }
+  }
+  return GALORE_OK;
+}
+
+template <typename TY>
+static galore_status_t orthonormalise(TY* Y, int64_t d, int b, const RefreshBuffers& w, int32_t* status, cudaStream_t st) {
+  GALORE_TRY(gram(Y, d, b, w.C, st));
+  return cholesky_solve(Y, d, b, w.C, w, status, st);
+}
+
+template <typename TG>
+static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, int32_t* status,
+                                     galore_refresh_info_t* info, cudaStream_t st) {
+  const TG* G = (const TG*)pr.G;
+  const int64_t d = pr.left ? pr.m : pr.n;
+  const int64_t L = pr.left ? pr.n : pr.m;
+  const int64_t sAi = pr.left ? pr.ldg : 1;    // A(i, l) = G[i*sAi + l*sAl]
+  const int64_t sAl = pr.left ? 1 : pr.ldg;
+  const int r = pr.rank, b = pr.block;
+  RefreshBuffers w = layout(workspace, d, L, r, b);
+  galore_refresh_info_t local = {};
+  local.block = b;
+
+  float* Y = w.Ya;
+  float* Yn = w.Yb;
+  const int64_t yb = d * b;
+  int q_done = 0;
+  std::vector<double> theta(b);
+  const bool full_space = (b == d);
+
+  if (!full_space) {
+    fill_normal_kernel<<<grid_for(yb), 256, 0, st>>>(Y, yb, pr.seed);
+    GALORE_LAUNCH_CHECK();
+    GALORE_TRY(orthonormalise(Y, d, b, w, status, st));
+  }
+  int q_target = full_space ? 0 : std::min(pr.max_iters, std::max(1, pr.first_iters));
+  double predicted = 0.0;
+  bool converged = full_space;
+
+  for (;;) {
+    // ---- power steps ---------------------------------------------------------
+    for (; q_done < q_target; ++q_done) {
+      float* Z = (float*)w.Zu;
+      {  // Z = A^T Y   (L x b)
+        EpiStore<float, float> epi{Z, b, 0, 1.f, 0.f};
+        GALORE_TRY((launch_gemm_simt<TG, float, float>((int)L, b, (int)d, G, sAl, sAi, Y, b, 1, 1, epi, st)));
+      }
+      {  // Y' = A Z     (d x b)
+        EpiStore<float, float> epi{Yn, b, 0, 1.f, 0.f};
+        GALORE_TRY((launch_gemm_simt<TG, float, float>((int)d, b, (int)L, G, sAi, sAl, Z, b, 1, 1, epi, st)));
+      }
+      GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
+      sumsq_kernel<<<grid_for(yb), 256, 0, st>>>(Yn, yb, w.scal);
+      GALORE_LAUNCH_CHECK();
+      shift_kernel<<<grid_for(yb), 256, 0, st>>>(Yn, Y, yb, b, w.scal);
+      GALORE_LAUNCH_CHECK();
+      std::swap(Y, Yn);
+      GALORE_TRY(orthonormalise(Y, d, b, w, status, st));
+    }
+    // ---- Rayleigh-Ritz in fp64 --------------------------------------------------
+    if (full_space) {
+      set_identity_kernel<<<grid_for(yb), 256, 0, st>>>(w.Y64, (int)d);
+      GALORE_LAUNCH_CHECK();
+    } else {
+      GALORE_TRY(orthonormalise(Y, d, b, w, status, st));     // second CholeskyQR pass in fp32 storage
+      convert_kernel<float, double><<<grid_for(yb), 256, 0, st>>>(Y, w.Y64, yb);
+      GALORE_LAUNCH_CHECK();
+      GALORE_TRY(orthonormalise(w.Y64, d, b, w, status, st));
+    }
+    double* Z64 = (double*)w.Zu;
+    {  // Z = A^T Y   (L x b), fp64
+      EpiStore<double, double> epi{Z64, b, 0, 1.0, 0.0};
+      GALORE_TRY((launch_gemm_simt<TG, double, double>((int)L, b, (int)d, G, sAl, sAi, w.Y64, b, 1, 1, epi, st)));
+    }
+    GALORE_TRY(gram(Z64, L, b, w.H, st));                     // H = Z^T Z
+    set_identity_kernel<<<grid_for((int64_t)b * b), 256, 0, st>>>(w.Vt, b);
+    GALORE_LAUNCH_CHECK();
+    const int np = b + (b & 1);
+    int sweeps = 0;
+    for (; sweeps < 40 && np > 1; ++sweeps) {
+      GALORE_CUDA_TRY(cudaMemsetAsync(w.counter, 0, sizeof(int), st));
+      for (int round = 0; round < np - 1; ++round) {
+        jacobi_round_kernel<<<np / 2, 256, 0, st>>>(w.H, w.Vt, b, np, round, 1e-13, w.counter);
+        GALORE_LAUNCH_CHECK();
+      }
+      int rot = 0;
+      GALORE_CUDA_TRY(cudaMemcpyAsync(&rot, w.counter, sizeof(int), cudaMemcpyDeviceToHost, st));
+      GALORE_CUDA_TRY(cudaStreamSynchronize(st));
+      if (rot == 0) { ++sweeps; break; }
+    }
+    local.jacobi_sweeps = sweeps;
+    row_norm_kernel<<<b, 256, 0, st>>>(w.H, b, w.lam);
+    GALORE_LAUNCH_CHECK();
+    rank_desc_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(w.lam, b, w.theta, w.order);
+    GALORE_LAUNCH_CHECK();
+    GALORE_CUDA_TRY(cudaMemcpyAsync(theta.data(), w.theta, sizeof(double) * b, cudaMemcpyDeviceToHost, st));
+    GALORE_CUDA_TRY(cudaStreamSynchronize(st));
+
+    if (!full_space) {
+      const double th_r = theta[r - 1], th_b = theta[b - 1];
+      const double ratio = (b > r && th_r > 0.0) ? th_b / th_r : 1.0;
+      predicted = (ratio < 1.0) ? pow(ratio, (double)q_done) : 1.0;
+      converged = predicted <= pr.tol;
+      if (!converged && q_done < pr.max_iters && ratio < 1.0 && ratio > 0.0) {
+        int need = (int)ceil(log(pr.tol) / log(ratio)) + 2;
+        q_target = std::min(pr.max_iters, std::max(need, q_done + 1));
+        continue;                                              // more power steps, then Rayleigh-Ritz again
+      }
+    }
+    break;
+  }
+
+  // ---- P = Y S[:, top r] ------------------------------------------------------------
+  gather_rows_kernel<<<r, 256, 0, st>>>(w.Vt, w.order, b, w.Vsel);
+  GALORE_LAUNCH_CHECK();
+  {
+    EpiStore<double, double> epi{w.P64, r, 0, 1.0, 0.0};
+    GALORE_TRY((launch_gemm_simt<double, double, double>((int)d, r, b, w.Y64, b, 1, w.Vsel, 1, b, 1, epi, st)));
+  }
+  const int64_t pc = d * r;
+  if (pr.p_dtype == GALORE_BF16)
+    convert_kernel<double, __nv_bfloat16><<<grid_for(pc), 256, 0, st>>>(w.P64, (__nv_bfloat16*)pr.P, pc);
+  else
+    convert_kernel<double, float><<<grid_for(pc), 256, 0, st>>>(w.P64, (float*)pr.P, pc);
+  GALORE_LAUNCH_CHECK();
+
+  // ---- a-posteriori residual of the kept Ritz pairs -----------------------------------
+  {
+    double* T1 = (double*)w.Zu;   // L x r
+    double* T2 = w.Y64;           // d x r (Y64 is no longer needed)
+    EpiStore<double, double> e1{T1, r, 0, 1.0, 0.0};
+    GALORE_TRY((launch_gemm_simt<TG, double, double>((int)L, r, (int)d, G, sAl, sAi, w.P64, r, 1, 1, e1, st)));
+    EpiStore<double, double> e2{T2, r, 0, 1.0, 0.0};
+    GALORE_TRY((launch_gemm_simt<TG, double, double>((int)d, r, (int)L, G, sAi, sAl, T1, r, 1, 1, e2, st)));
+    GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
+    residual_kernel<<<grid_for(pc), 256, 0, st>>>(T2, w.P64, w.theta, d, r, w.scal);
+    GALORE_LAUNCH_CHECK();
+    double sc[2] = {0, 0};
+    GALORE_CUDA_TRY(cudaMemcpyAsync(sc, w.scal, sizeof(sc), cudaMemcpyDeviceToHost, st));
+    GALORE_CUDA_TRY(cudaStreamSynchronize(st));
+    local.residual = theta[0] > 0.0 ? sqrt(sc[1]) / (theta[0] * sqrt((double)r)) : 0.0;
+  }
+  local.iterations = q_done;
+  local.converged = converged ? 1 : 0;
+  local.predicted_error = predicted;
+  local.sigma_1 = sqrt(theta[0]);
+  local.sigma_r = sqrt(theta[r - 1]);
+  local.sigma_next = (b > r) ? sqrt(theta[r]) : 0.0;
+  if (info) *info = local;
+  return converged ? GALORE_OK : GALORE_WARN_NOT_CONVERGED;
+}
+
+galore_status_t refresh_projector(const RefreshProblem& pr, void* workspace, int32_t* status,
+                                  galore_refresh_info_t* info, cudaStream_t st) {
+  if (pr.g_dtype == GALORE_BF16) return refresh_typed<__nv_bfloat16>(pr, workspace, status, info, st);
+  return refresh_typed<float>(pr, workspace, status, info, st);
+}
+
+}  // namespace galore

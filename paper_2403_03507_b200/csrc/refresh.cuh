@@ -1,0 +1,31 @@
+// Projector refresh (Eq. 12-13 by block subspace iteration): declarations.
+#pragma once
+
+#include "common.cuh"
+
+namespace galore {
+
+struct RefreshProblem {
+  const void* G;        // m x n, row-major
+  int32_t g_dtype;
+  int64_t ldg;
+  int64_t m, n;
+  bool left;            // true: P = leading left singular vectors (m x r); false: right (n x r)
+  int rank;
+  int block;            // columns iterated, rank <= block <= min(m, n)
+  void* P;              // output, rows x rank row-major in p_dtype
+  int32_t p_dtype;
+  uint64_t seed;
+  double tol;
+  int max_iters;
+  int first_iters;      // power steps before the first Rayleigh-Ritz
+};
+
+// d = rows of the projector, L = the other dimension of G
+size_t refresh_workspace_bytes(int64_t d, int64_t L, int r, int b);
+
+// Synchronises the stream (reads Ritz values back to decide on convergence).
+galore_status_t refresh_projector(const RefreshProblem& pr, void* workspace, int32_t* status,
+                                  galore_refresh_info_t* info, cudaStream_t st);
+
+}  // namespace galore
