@@ -1,0 +1,271 @@
+"""Thin ctypes binding of the C ABI in include/galore.h.
+
+Argument marshalling only: every step of the path runs in the CUDA library.
+Loading fails loudly when the library has not been built; there is no
+fallback of any kind.  torch is used for device buffers and streams.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgalore.so")
+
+OK, WARN_NOT_CONVERGED = 0, 1
+ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL = -1, -2, -3, -4
+ERR_CUDA, ERR_STATE, ERR_NONFINITE, ERR_TIMEOUT, ERR_UNIMPLEMENTED = -5, -6, -7, -8, -9
+SIDE_AUTO, SIDE_LEFT, SIDE_RIGHT = 0, 1, 2
+F32, BF16 = 0, 1
+STATE_F32, STATE_Q8_BLOCK = 0, 1
+PATH_AUTO, PATH_FP32, PATH_TENSOR = 0, 1, 2
+DEV_NONFINITE, DEV_WAIT_EXPIRED, DEV_BOUNDS, DEV_CHOLESKY = 1, 2, 4, 8
+
+_DTYPES = {"f32": F32, "bf16": BF16, torch.float32: F32, torch.bfloat16: BF16}
+_TORCH = {F32: torch.float32, BF16: torch.bfloat16}
+
+
+class Config(C.Structure):
+    _fields_ = [
+        ("m", C.c_int64), ("n", C.c_int64), ("rank", C.c_int32), ("alpha", C.c_float),
+        ("refresh_gap", C.c_int32), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+        ("side", C.c_int32), ("w_dtype", C.c_int32), ("g_dtype", C.c_int32), ("p_dtype", C.c_int32),
+        ("state_fmt", C.c_int32), ("q_block", C.c_int32), ("auto_refresh", C.c_int32), ("path", C.c_int32),
+        ("refresh_tol", C.c_float), ("refresh_max_iters", C.c_int32), ("refresh_oversample", C.c_int32),
+        ("seed", C.c_uint64), ("reserved", C.c_int32 * 8),
+    ]
+
+
+class RefreshInfo(C.Structure):
+    _fields_ = [
+        ("iterations", C.c_int32), ("block", C.c_int32), ("jacobi_sweeps", C.c_int32), ("converged", C.c_int32),
+        ("predicted_error", C.c_double), ("residual", C.c_double), ("sigma_r", C.c_double),
+        ("sigma_next", C.c_double), ("sigma_1", C.c_double),
+    ]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class GaloreError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        msg = lib().galore_status_string(status).decode()
+        cuda = lib().galore_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} ({status})" + (f" [{cuda}]" if status == ERR_CUDA and cuda else ""))
+
+
+_lib = None
+
+_PROTOTYPES = {
+    "galore_query_bytes": (C.c_int, [C.POINTER(Config), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
+    "galore_init_layer": (C.c_int, [C.POINTER(Config), C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p,
+                                    C.POINTER(C.c_void_p)]),
+    "galore_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_float, C.c_void_p]),
+    "galore_step_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
+    "galore_step_batch": (C.c_int, [C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_int64),
+                                    C.POINTER(C.c_void_p), C.POINTER(C.c_int64), C.c_int32, C.c_float, C.c_void_p]),
+    "galore_refresh_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.POINTER(RefreshInfo)]),
+    "galore_free": (C.c_int, [C.c_void_p]),
+    "galore_get_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "galore_set_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "galore_get_moments": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "galore_get_q8_state": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "galore_get_step_count": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
+    "galore_set_step_count": (C.c_int, [C.c_void_p, C.c_int64]),
+    "galore_layer_info": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int64),
+                                    C.POINTER(C.c_int64)]),
+    "galore_device_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32), C.c_void_p]),
+    "galore_q8_codebook": (C.c_int, [C.c_int32, C.POINTER(C.c_float)]),
+    "galore_q8_quantize": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "galore_q8_dequantize": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
+    "galore_status_string": (C.c_char_p, [C.c_int]),
+    "galore_last_cuda_error": (C.c_char_p, []),
+    "galore_launch_count": (C.c_int64, []),
+}
+
+
+def lib():
+    """The loaded C library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2403_03507_b200.build`")
+        handle = C.CDLL(LIB_PATH)
+        for name, (res, args) in _PROTOTYPES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def _check(status, where):
+    if status < 0:
+        raise GaloreError(status, where)
+    return status
+
+
+def _stream_ptr(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def make_config(m, n, rank, alpha=0.25, refresh_gap=200, beta1=0.9, beta2=0.999, eps=1e-8, side=SIDE_AUTO,
+                w_dtype="bf16", g_dtype="bf16", p_dtype=None, state_fmt="f32", q_block=2048, auto_refresh=True,
+                path=PATH_AUTO, refresh_tol=0.0, refresh_max_iters=0, refresh_oversample=0, seed=0) -> Config:
+    c = Config()
+    c.m, c.n, c.rank, c.alpha, c.refresh_gap = m, n, rank, alpha, refresh_gap
+    c.beta1, c.beta2, c.eps = beta1, beta2, eps
+    c.side = side
+    c.w_dtype, c.g_dtype = _DTYPES[w_dtype], _DTYPES[g_dtype]
+    if p_dtype is None:   # bf16 projector only where the gradient is bf16 too (tensor-core operands)
+        p_dtype = "bf16" if c.g_dtype == BF16 else "f32"
+    c.p_dtype = _DTYPES[p_dtype]
+    c.state_fmt = {"f32": STATE_F32, "q8": STATE_Q8_BLOCK, STATE_F32: STATE_F32, STATE_Q8_BLOCK: STATE_Q8_BLOCK}[state_fmt]
+    c.q_block, c.auto_refresh, c.path = q_block, int(bool(auto_refresh)), path
+    c.refresh_tol, c.refresh_max_iters, c.refresh_oversample, c.seed = refresh_tol, refresh_max_iters, refresh_oversample, seed
+    return c
+
+
+def galore_query_bytes(cfg: Config):
+    sb, wb = C.c_size_t(0), C.c_size_t(0)
+    _check(lib().galore_query_bytes(C.byref(cfg), C.byref(sb), C.byref(wb)), "galore_query_bytes")
+    return sb.value, wb.value
+
+
+def galore_q8_codebook(is_signed: bool):
+    out = (C.c_float * 256)()
+    _check(lib().galore_q8_codebook(int(is_signed), out), "galore_q8_codebook")
+    return list(out)
+
+
+def galore_q8_quantize(x: torch.Tensor, is_signed: bool, block: int = 2048, stream=None):
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    n = x.numel()
+    codes = torch.empty(n, dtype=torch.uint8, device=x.device)
+    absmax = torch.empty((n + block - 1) // block, dtype=torch.float32, device=x.device)
+    _check(lib().galore_q8_quantize(x.data_ptr(), n, int(is_signed), block, codes.data_ptr(), absmax.data_ptr(),
+                                    _stream_ptr(stream)), "galore_q8_quantize")
+    return codes, absmax
+
+
+def galore_q8_dequantize(codes: torch.Tensor, absmax: torch.Tensor, is_signed: bool, block: int = 2048, stream=None):
+    out = torch.empty(codes.numel(), dtype=torch.float32, device=codes.device)
+    _check(lib().galore_q8_dequantize(codes.data_ptr(), absmax.data_ptr(), codes.numel(), int(is_signed), block,
+                                      out.data_ptr(), _stream_ptr(stream)), "galore_q8_dequantize")
+    return out
+
+
+def galore_launch_count() -> int:
+    return int(lib().galore_launch_count())
+
+
+class Layer:
+    """One 2-D weight's GaLore state: owns the two device buffers (torch) and the C handle."""
+
+    def __init__(self, cfg: Config, device="cuda:0", workspace: torch.Tensor | None = None, stream=None):
+        self.cfg = cfg
+        self.device = torch.device(device)
+        self.state_bytes, self.workspace_bytes = galore_query_bytes(cfg)
+        self.state = torch.empty(self.state_bytes, dtype=torch.uint8, device=self.device)
+        if workspace is None:
+            workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=self.device)
+        if workspace.numel() < self.workspace_bytes:
+            raise ValueError("shared workspace too small")
+        self.workspace = workspace
+        h = C.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(lib().galore_init_layer(C.byref(cfg), self.state.data_ptr(), self.state.numel(),
+                                           workspace.data_ptr(), workspace.numel(), _stream_ptr(stream), C.byref(h)),
+                   "galore_init_layer")
+        self.handle = h
+        side, tp, sr, sc = C.c_int32(), C.c_int32(), C.c_int64(), C.c_int64()
+        _check(lib().galore_layer_info(h, C.byref(side), C.byref(tp), C.byref(sr), C.byref(sc)), "galore_layer_info")
+        self.side, self.uses_tensor_path, self.state_shape = side.value, bool(tp.value), (sr.value, sc.value)
+        self.proj_rows = cfg.m if self.side == SIDE_LEFT else cfg.n
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().galore_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the hot path ---------------------------------------------------------
+    def galore_step(self, W: torch.Tensor, G: torch.Tensor, lr: float, stream=None) -> int:
+        return _check(lib().galore_step(self.handle, W.data_ptr(), W.stride(0), G.data_ptr(), G.stride(0), lr,
+                                        _stream_ptr(stream)), "galore_step")
+
+    def galore_step_host(self, W_host, G_host, W_dev, G_dev, lr: float, stream=None) -> int:
+        return _check(lib().galore_step_host(self.handle, W_host.data_ptr(), G_host.data_ptr(), W_dev.data_ptr(),
+                                             G_dev.data_ptr(), lr, _stream_ptr(stream)), "galore_step_host")
+
+    def galore_refresh_projector(self, G: torch.Tensor, stream=None):
+        info = RefreshInfo()
+        st = _check(lib().galore_refresh_projector(self.handle, G.data_ptr(), G.stride(0), _stream_ptr(stream),
+                                                   C.byref(info)), "galore_refresh_projector")
+        return st, info
+
+    # -- accessors ------------------------------------------------------------
+    def get_projector(self, stream=None) -> torch.Tensor:
+        out = torch.empty(self.proj_rows, self.cfg.rank, dtype=torch.float32, device=self.device)
+        _check(lib().galore_get_projector(self.handle, out.data_ptr(), out.numel() * 4, _stream_ptr(stream)),
+               "galore_get_projector")
+        return out
+
+    def set_projector(self, P: torch.Tensor, stream=None):
+        P = P.to(device=self.device, dtype=torch.float32).contiguous()
+        assert tuple(P.shape) == (self.proj_rows, self.cfg.rank)
+        _check(lib().galore_set_projector(self.handle, P.data_ptr(), P.numel() * 4, _stream_ptr(stream)),
+               "galore_set_projector")
+        torch.cuda.current_stream().synchronize() if stream is None else stream.synchronize()
+
+    def get_moments(self, stream=None):
+        M = torch.empty(self.state_shape, dtype=torch.float32, device=self.device)
+        V = torch.empty(self.state_shape, dtype=torch.float32, device=self.device)
+        _check(lib().galore_get_moments(self.handle, M.data_ptr(), V.data_ptr(), M.numel() * 4, _stream_ptr(stream)),
+               "galore_get_moments")
+        return M, V
+
+    def get_q8_state(self, stream=None):
+        nel = self.state_shape[0] * self.state_shape[1]
+        qb = self.cfg.q_block or 2048
+        nblk = (nel + qb - 1) // qb
+        Mc = torch.empty(nel, dtype=torch.uint8, device=self.device)
+        Vc = torch.empty(nel, dtype=torch.uint8, device=self.device)
+        Ma = torch.empty(nblk, dtype=torch.float32, device=self.device)
+        Va = torch.empty(nblk, dtype=torch.float32, device=self.device)
+        _check(lib().galore_get_q8_state(self.handle, Mc.data_ptr(), Ma.data_ptr(), Vc.data_ptr(), Va.data_ptr(),
+                                         _stream_ptr(stream)), "galore_get_q8_state")
+        return Mc, Ma, Vc, Va
+
+    @property
+    def step_count(self) -> int:
+        k = C.c_int64()
+        _check(lib().galore_get_step_count(self.handle, C.byref(k)), "galore_get_step_count")
+        return k.value
+
+    @step_count.setter
+    def step_count(self, k: int):
+        _check(lib().galore_set_step_count(self.handle, k), "galore_set_step_count")
+
+    def device_status(self, stream=None) -> int:
+        f = C.c_int32()
+        _check(lib().galore_device_status(self.handle, C.byref(f), _stream_ptr(stream)), "galore_device_status")
+        return f.value
+
+
+def galore_step_batch(layers, Ws, Gs, lr: float, stream=None) -> int:
+    n = len(layers)
+    hs = (C.c_void_p * n)(*[l.handle for l in layers])
+    wp = (C.c_void_p * n)(*[w.data_ptr() for w in Ws])
+    gp = (C.c_void_p * n)(*[g.data_ptr() for g in Gs])
+    lw = (C.c_int64 * n)(*[w.stride(0) for w in Ws])
+    lg = (C.c_int64 * n)(*[g.stride(0) for g in Gs])
+    return _check(lib().galore_step_batch(hs, wp, lw, gp, lg, n, lr, _stream_ptr(stream)), "galore_step_batch")

@@ -81,8 +81,9 @@ __device__ __forceinline__ double block_sum_256(double v, double* red) {
   return r;
 }
 
-// scal[0] += sum of squares
-__global__ void __launch_bounds__(256) sumsq_kernel(const float* __restrict__ x, int64_t count, double* __restrict__ scal) {
+// part[blockIdx.x] = this CTA's share of the sum of squares (fixed grid, so the total is reproducible)
+constexpr int kSumsqBlocks = 592;
+__global__ void __launch_bounds__(256) sumsq_kernel(const float* __restrict__ x, int64_t count, double* __restrict__ part) {
   __shared__ double red[8];
   double s = 0.0;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x) {
@@ -90,13 +91,17 @@ __global__ void __launch_bounds__(256) sumsq_kernel(const float* __restrict__ x,
     s += v * v;
   }
   s = block_sum_256(s, red);
-  if (threadIdx.x == 0) atomicAdd(scal, s);
+  if (threadIdx.x == 0) part[blockIdx.x] = s;
 }
 
 // Ynew += delta * Yold,  delta = max(1e-4 * rms column norm of Ynew, 1e-30)
-__global__ void shift_kernel(float* __restrict__ Ynew, const float* __restrict__ Yold, int64_t count, int cols,
-                             const double* __restrict__ scal) {
-  const float delta = fmaxf((float)(1e-4 * sqrt(scal[0] / (double)cols)), 1e-30f);
+__global__ void __launch_bounds__(256) shift_kernel(float* __restrict__ Ynew, const float* __restrict__ Yold, int64_t count,
+                                                    int cols, const double* __restrict__ part) {
+  __shared__ double red[8];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < kSumsqBlocks; i += 256) s += part[i];
+  s = block_sum_256(s, red);
+  const float delta = fmaxf((float)(1e-4 * sqrt(s / (double)cols)), 1e-30f);
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
     Ynew[i] = fmaf(delta, Yold[i], Ynew[i]);
 }
@@ -273,6 +278,7 @@ struct RefreshBuffers {
   double* theta;  // b
   int* order;     // b
   double* scal;   // 4 scalars
+  double* part;   // kSumsqBlocks partial sums
   int* counter;   // 1
 };
 
@@ -294,7 +300,7 @@ size_t refresh_workspace_bytes(int64_t d, int64_t L, int r, int b) {
   t += align_up((size_t)64 * 64 * 8, 256);
   t += align_up((size_t)b * 8, 256) * 2;
   t += align_up((size_t)b * 4, 256);
-  t += 256 * 2;
+  t += 256 * 2 + 8 * 1024;
   return t;
 }
 
@@ -316,6 +322,7 @@ static RefreshBuffers layout(void* base, int64_t d, int64_t L, int r, int b) {
   w.theta = (double*)p; carve(p, (size_t)b * 8);
   w.order = (int*)p; carve(p, (size_t)b * 4);
   w.scal = (double*)p; carve(p, 256);
+  w.part = (double*)p; carve(p, 8 * 1024);
   w.counter = (int*)p; carve(p, 256);
   return w;
 }
@@ -415,10 +422,9 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
         EpiStore<float, float> epi{Yn, b, 0, 1.f, 0.f};
         GALORE_TRY((launch_gemm_simt<TG, float, float>((int)d, b, (int)L, G, sAi, sAl, Z, b, 1, 1, epi, st)));
       }
-      GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
-      sumsq_kernel<<<grid_for(yb), 256, 0, st>>>(Yn, yb, w.scal);
+      sumsq_kernel<<<kSumsqBlocks, 256, 0, st>>>(Yn, yb, w.part);
       GALORE_LAUNCH_CHECK();
-      shift_kernel<<<grid_for(yb), 256, 0, st>>>(Yn, Y, yb, b, w.scal);
+      shift_kernel<<<grid_for(yb), 256, 0, st>>>(Yn, Y, yb, b, w.part);
       GALORE_LAUNCH_CHECK();
       std::swap(Y, Yn);
       GALORE_TRY(orthonormalise(Y, d, b, w, status, st));

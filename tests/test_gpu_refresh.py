@@ -1,0 +1,94 @@
+"""Parity of the refreshed projector with the oracle's top-r singular subspace."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import galore_oracle as go
+from paper_2403_03507_b200 import binding as gb
+from paper_2403_03507_b200 import workloads as wl
+
+from gpu_util import to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+ANGLE_TOL = 1e-3      # largest principal angle, rad
+
+
+def _refresh(G, r, g_dtype="f32", **kw):
+    m, n = G.shape
+    cfg = gb.make_config(m, n, r, w_dtype="f32", g_dtype=g_dtype, p_dtype="f32", auto_refresh=False, **kw)
+    layer = gb.Layer(cfg)
+    st, info = layer.galore_refresh_projector(to_dev(G, g_dtype))
+    P = to_host(layer.get_projector())
+    assert layer.device_status() == 0
+    return st, info.as_dict(), P, layer
+
+
+@pytest.mark.parametrize("m,n,r", [(96, 200, 8), (200, 96, 8), (128, 128, 32), (150, 310, 70)])
+def test_gapped_spectrum_recovers_planted_subspace(m, n, r):
+    k = min(m, n)
+    spectrum = np.concatenate([np.linspace(10, 5, r), np.linspace(0.5, 0.01, k - r)])
+    G, U, V = wl.make_planted(m, n, seed=5, spectrum=spectrum, dtype="f32")
+    st, info, P, layer = _refresh(G, r)
+    side = "left" if m <= n else "right"
+    P_orc, S = go.top_r_projector(G, r, side)
+    assert st == gb.OK and info["converged"] == 1
+    assert np.max(np.abs(P.T @ P - np.eye(r))) < 1e-5
+    assert go.largest_principal_angle(P_orc, P) < ANGLE_TOL
+    assert go.largest_principal_angle((U if side == "left" else V)[:, :r], P) < ANGLE_TOL
+    # columns are singular vectors in descending order (distinct singular values): |<p_i, u_i>| = 1
+    assert np.allclose(np.abs(np.sum(P * P_orc, axis=0)), 1.0, atol=1e-4)
+    assert abs(info["sigma_r"] - S[r - 1]) < 1e-5 * S[0] and abs(info["sigma_1"] - S[0]) < 1e-5 * S[0]
+    assert info["residual"] < 1e-5
+
+
+def test_exactly_low_rank_gradient():
+    # rank(G) = r < block: P P^T G = G must hold although the iterated block is rank-deficient
+    m, n, r = 120, 260, 10
+    G, U, V = wl.make_planted(m, n, seed=3, spectrum=np.linspace(4, 1, r), dtype="f64")
+    G = wl.round_to(G, "f32")
+    st, info, P, _ = _refresh(G, r)
+    assert np.max(np.abs(P.T @ P - np.eye(r))) < 1e-5
+    assert np.linalg.norm(P @ (P.T @ G) - G) / np.linalg.norm(G) < 1e-5
+
+
+def test_rank_equal_to_min_dimension_and_zero_gradient():
+    G = wl.make_gradient(40, 72, 1, 1.0, 0.01, "f32")
+    st, info, P, _ = _refresh(G, 40)
+    assert np.max(np.abs(P.T @ P - np.eye(40))) < 1e-5 and info["block"] == 40
+    assert np.linalg.norm(P @ (P.T @ G) - G) / np.linalg.norm(G) < 1e-5
+    st, info, P, _ = _refresh(np.zeros((24, 40)), 6)
+    assert np.all(np.isfinite(P)) and np.max(np.abs(P.T @ P - np.eye(6))) < 1e-4
+
+
+@pytest.mark.parametrize("m,n,r,g_dtype", [(512, 1376, 128, "f32"), (1376, 512, 128, "f32"), (256, 704, 64, "bf16")])
+def test_workload_spectrum_noise_dominated(m, n, r, g_dtype):
+    # the decaying-spectrum-plus-noise recipe: sigma_{r+1}/sigma_r is about 0.999
+    G = wl.make_gradient(m, n, wl.sub_seed(wl.BASE_SEED, 0), 1.0, 0.01, g_dtype)
+    st, info, P, _ = _refresh(G, r, g_dtype)
+    side = "left" if m <= n else "right"
+    P_orc, S = go.top_r_projector(G, r, side)
+    angle = go.largest_principal_angle(P_orc, P)
+    print(f"{m}x{n} r={r}: angle {angle:.2e} rad, sigma_r {S[r-1]:.4f}, sigma_r+1/sigma_r {S[r]/S[r-1]:.5f}, info {info}")
+    assert np.max(np.abs(P.T @ P - np.eye(r))) < 1e-5
+    assert angle < ANGLE_TOL
+    # Ritz basis: P^T G G^T P is diagonal with the leading sigma^2 on it
+    A = G if side == "left" else G.T
+    T = P.T @ A @ A.T @ P
+    off = T - np.diag(np.diag(T))
+    assert np.max(np.abs(off)) < 1e-4 * S[0] ** 2
+    assert np.allclose(np.sqrt(np.diag(T)), S[:r], rtol=1e-4)
+
+
+def test_iteration_cap_gives_a_warning_not_an_error():
+    G = wl.make_gradient(128, 300, 2, 1.0, 0.01, "f32")
+    st, info, P, _ = _refresh(G, 32, refresh_max_iters=1, refresh_oversample=-1)
+    assert st == gb.WARN_NOT_CONVERGED and info["converged"] == 0 and info["iterations"] == 1
+    assert np.max(np.abs(P.T @ P - np.eye(32))) < 1e-5
+
+
+def test_same_seed_same_projector():
+    G = wl.make_gradient(96, 160, 2, 1.0, 0.01, "f32")
+    _, _, P1, _ = _refresh(G, 12, seed=7)
+    _, _, P2, _ = _refresh(G, 12, seed=7)
+    assert np.array_equal(P1, P2)
