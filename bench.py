@@ -1,0 +1,410 @@
+#!/usr/bin/env python
+"""Benchmark of the GaLore-Adam optimizer step (parameters updated per second).
+
+A "step" is one pass of the whole path (projection, Adam on R with the
+configured state format, back-projection, weight write) over every matrix of
+the workload's layer set, on synthetic gradients already resident in HBM.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+N > 1 (under torch.distributed.run) runs N independent replicas of the same
+workload, one per GPU: the path has no exchange step, so nothing is sharded
+and no collective is on the data path; only the timing is reduced over ranks.
+`--impl reference` times the CPU oracle on the host cores on a bounded sample.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "galore_adam_step_params_per_sec"
+UNIT = "params/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# fp32 FMA peak of the part: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (unit counts and max clock)
+FP32_FMA_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+def elem_bytes(dt):
+    return 2 if dt == "bf16" else 4
+
+
+def algorithmic_cost(w, m, n):
+    """Bytes the method must move and flops it must do for one matrix and one step."""
+    r = w.rank
+    left = m <= n
+    d, big = (m, n) if left else (n, m)
+    nel = r * big
+    state = 4 * nel * 4 if w.state_fmt == "f32" else 4 * nel + 4 * 4 * ((nel + w.q_block - 1) // w.q_block)
+    by = m * n * elem_bytes(w.g_dtype) + 2 * m * n * elem_bytes(w.w_dtype) + state + d * r * elem_bytes(p_dtype_of(w))
+    return by, 4 * m * n * r
+
+
+def p_dtype_of(w):
+    return "bf16" if w.g_dtype == "bf16" else "f32"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return res
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 8:
+                    continue
+                try:
+                    sm.append(float(parts[0]))
+                    mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[4:8]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            res.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return res
+
+
+def cpu_oracle_sample(w, steps=1):
+    """Times the oracle, as it stands, on one matrix of each distinct shape of the workload."""
+    import numpy as np
+    from oracle import galore_oracle as go
+    from paper_2403_03507_b200 import workloads as wl
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    total_params, total_time = 0, 0.0
+    rng = np.random.default_rng(0)
+    for (m, n, _count) in w.shapes:
+        side = "left" if m <= n else "right"
+        orc = go.GaLoreOracle(m, n, w.rank, w.alpha, w.refresh_gap, w.beta1, w.beta2, w.eps, w_store=w.w_dtype,
+                              state=w.state_fmt, q_block=w.q_block)
+        d = m if side == "left" else n
+        P, _ = np.linalg.qr(rng.standard_normal((d, w.rank)))       # any orthonormal projector: timing only
+        orc.set_projector(P)
+        G = wl.round_to(rng.standard_normal((m, n)) * 0.05, w.g_dtype)
+        W = wl.round_to(rng.standard_normal((m, n)) * 0.02, w.w_dtype)
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            W = orc.step(W, G, w.lr, auto_refresh=False)
+        total_time += time.perf_counter() - t0
+        total_params += m * n * steps
+    return total_params / total_time, cores, total_time
+
+
+def run_reference(args, w):
+    value, cores, _ = None, None, None
+    times = []
+    for i in range(args.warmup + args.steps):
+        v, cores, t = cpu_oracle_sample(w, 1)
+        if i >= args.warmup:
+            times.append((v, t))
+    value = sum(v for v, _ in times) / len(times)
+    ms = 1e3 * sum(t for _, t in times) / len(times)
+    sample = f"1 oracle step on one matrix of each distinct shape ({len(w.shapes)} of {w.matrices} matrices), given projector"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": {"workload": w.name, "rank": w.rank, "state_fmt": w.state_fmt},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="llama_7b_q8")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--extra-workloads", default="", help="comma-separated workloads also timed (device-resident only)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else max(args.warmup, 0)
+
+    from paper_2403_03507_b200 import workloads as wl
+    w = wl.WORKLOADS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, w)
+        return 0
+
+    import torch
+    from paper_2403_03507_b200 import binding as gb
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the step has no CPU path")
+    gb.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    res = time_workload(w, args, dev, dist, world, rank, full=True)
+    if rank == 0:
+        extras = []
+        for name in [x for x in args.extra_workloads.split(",") if x]:
+            extras.append(time_workload(wl.WORKLOADS[name], args, dev, None, 1, 0, full=False))
+        if extras:
+            res["other_workloads"] = extras
+        print(json.dumps(res), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def time_workload(w, args, dev, dist, world, rank, full):
+    import torch
+    from paper_2403_03507_b200 import binding as gb
+    from paper_2403_03507_b200 import workloads as wl
+
+    tdt = {"f32": torch.float32, "bf16": torch.bfloat16}
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream()
+
+    def padded(m, n, dtype):
+        ld = (n + 7) // 8 * 8          # 16-byte rows so that TMA can address bf16 operands
+        buf = torch.empty(m, ld, dtype=dtype, device=dev)
+        return buf[:, :n]
+
+    # ---- build the layer set -------------------------------------------------------------------
+    layers, Ws, Gs, shapes_of = [], [], [], []
+    refresh_info = []
+    max_ws = 0
+    cfgs = {}
+    for (m, n, count) in w.shapes:
+        cfg = gb.make_config(m, n, w.rank, alpha=w.alpha, refresh_gap=w.refresh_gap, beta1=w.beta1, beta2=w.beta2,
+                             eps=w.eps, w_dtype=w.w_dtype, g_dtype=w.g_dtype, state_fmt=w.state_fmt,
+                             q_block=w.q_block, auto_refresh=False, seed=w.seed)
+        cfgs[(m, n)] = cfg
+        max_ws = max(max_ws, gb.galore_query_bytes(cfg)[1])
+    workspace = torch.empty(max_ws, dtype=torch.uint8, device=dev)      # shared: layers step one after another
+    bytes_alg, flops_alg = 0, 0
+    for si, (m, n, count) in enumerate(w.shapes):
+        pool = []
+        for j in range(2):                                             # two gradients per distinct shape, cycled
+            g = wl.make_gradient_torch(m, n, wl.sub_seed(w.seed, si, j) & 0x7FFFFFFF, w.spectrum_p, w.noise, dev,
+                                       tdt[w.g_dtype])
+            gp = padded(m, n, tdt[w.g_dtype])
+            gp.copy_(g)
+            pool.append(gp)
+            del g
+        first = None
+        for c in range(count):
+            layer = gb.Layer(cfgs[(m, n)], device=dev, workspace=workspace)
+            if first is None:
+                t0 = torch.cuda.Event(enable_timing=True)
+                t1 = torch.cuda.Event(enable_timing=True)
+                t0.record()
+                st, info = layer.galore_refresh_projector(pool[0])
+                t1.record()
+                torch.cuda.synchronize()
+                refresh_info.append({"shape": [m, n], "ms": t0.elapsed_time(t1), "status": st, **info.as_dict()})
+                first = layer.get_projector()
+            else:
+                layer.set_projector(first)                              # timing does not depend on P's values
+            Wt = padded(m, n, tdt[w.w_dtype])
+            Wt.copy_(torch.randn(m, n, device=dev) * 0.02)
+            layers.append(layer)
+            Ws.append(Wt)
+            Gs.append(pool[c % 2])
+            shapes_of.append((m, n))
+            by, fl = algorithmic_cost(w, m, n)
+            bytes_alg += by
+            flops_alg += fl
+    torch.cuda.synchronize()
+
+    def one_step(lr=w.lr):
+        for layer, Wt, Gt in zip(layers, Ws, Gs):
+            layer.galore_step(Wt, Gt, lr, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ----------------------------------------------------------------
+    for _ in range(args.warmup):
+        one_step()
+    barrier()
+    sampler = ClockSampler(dev.index if dev.index is not None else 0)
+    sampler.start()
+    launches0 = gb.galore_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        one_step()
+    e1.record(stream)
+    barrier()
+    launches = gb.galore_launch_count() - launches0
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * w.params / (ms_step * 1e-3)
+
+    # ---- per-phase timing with events on the launching stream (separate instrumented pass) -------
+    gb.galore_profile_enable(True)
+    prof_steps = max(1, min(args.steps, 3))
+    for _ in range(prof_steps):
+        one_step()
+    torch.cuda.synchronize()
+    gb.galore_profile_enable(False)
+    phase_ms, phase_cnt = gb.galore_profile_read()
+    uses_tc = all(l.uses_tensor_path for l in layers)
+    gemm_ms = phase_ms[0] + phase_ms[2]
+    gemm_launches = phase_cnt[0] + phase_cnt[2]
+    # dominant kernels: the two projection GEMMs (2 m n r flops each)
+    t_hbm = bytes_alg / (peaks["hbm_gbs"] * 1e9)
+    tc_peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    t_tc = flops_alg / (tc_peak * 1e12)
+    achieved_tflops = (flops_alg * prof_steps) / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
+    if uses_tc:
+        roof = {"bound": "tensor", "achieved": achieved_tflops, "peak": tc_peak, "unit": "TFLOP/s",
+                "frac": achieved_tflops / tc_peak if achieved_tflops else None, "traffic": None,
+                "peak_source": peaks["source"] + " (sustained bf16 GEMM)"}
+    else:
+        roof = {"bound": "alu", "achieved": achieved_tflops, "peak": FP32_FMA_TFLOPS, "unit": "TFLOP/s",
+                "frac": achieved_tflops / FP32_FMA_TFLOPS if achieved_tflops else None, "traffic": None,
+                "peak_source": "148 SMs x 128 fp32 lanes x 2 x 1.965 GHz"}
+    roof["kernel"] = "projection + back-projection GEMMs"
+    roof["avg_launch_ms"] = gemm_ms / gemm_launches if gemm_launches else None
+    roof["phase_ms_per_step"] = {"projection": phase_ms[0] / prof_steps, "adam": phase_ms[1] / prof_steps,
+                                 "back_projection": phase_ms[2] / prof_steps}
+    roof["step_roofline_ms"] = {"hbm": t_hbm * 1e3, "tensor": t_tc * 1e3}
+    roof["step_frac_of_roofline"] = max(t_hbm, t_tc) * 1e3 / ms_step
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if uses_tc else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "matrices": w.matrices, "params": w.params, "rank": w.rank,
+                   "state_fmt": w.state_fmt, "w_dtype": w.w_dtype, "g_dtype": w.g_dtype, "alpha": w.alpha,
+                   "refresh_gap": w.refresh_gap, "tensor_path": uses_tc, "parallelism": f"replicas x{world}",
+                   "l2": "inputs larger than L2 (whole layer set streamed each step)"},
+        "clocks": clocks, "gpu_launches": launches, "roofline": roof,
+        "refresh": refresh_info,
+    }
+    if not full:
+        return {k: out[k] for k in ("value", "ms_per_step", "config", "roofline", "refresh", "gpu_launches")}
+
+    # ---- end to end through the host-buffer entry point -------------------------------------------
+    if not args.no_e2e:
+        host = {}
+        for (m, n, _c) in w.shapes:
+            hw = torch.empty(m, n, dtype=tdt[w.w_dtype]).pin_memory()
+            hg = torch.empty(m, n, dtype=tdt[w.g_dtype]).pin_memory()
+            hw.normal_(0, 0.02)
+            hg.normal_(0, 0.05)
+            dw = torch.empty(m, n, dtype=tdt[w.w_dtype], device=dev)
+            dg = torch.empty(m, n, dtype=tdt[w.g_dtype], device=dev)
+            host[(m, n)] = (hw, hg, dw, dg)
+        e2e_steps = max(1, min(args.steps, 3))
+        h2d = sum(m * n * (elem_bytes(w.w_dtype) + elem_bytes(w.g_dtype)) for (m, n) in shapes_of)
+        d2h = sum(m * n * elem_bytes(w.w_dtype) for (m, n) in shapes_of)
+
+        def e2e_step():
+            for layer, sh in zip(layers, shapes_of):
+                hw, hg, dw, dg = host[sh]
+                layer.galore_step_host(hw, hg, dw, dg, w.lr, stream)
+
+        e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        ms = a.elapsed_time(b) / e2e_steps
+        if dist is not None:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        out["e2e"] = {"value": world * w.params / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                      "d2h_bytes_per_step": d2h, "ms_per_step": ms, "steps": e2e_steps,
+                      "host_buffers": "one pinned W and G per distinct shape, reused by the layers of that shape"}
+    flags = 0
+    for layer in layers[:1]:
+        flags |= layer.device_status()
+    out["device_status"] = flags
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, cores, t = cpu_oracle_sample(w, 1)
+        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                               "sample": f"1 oracle step on one matrix of each distinct shape ({len(w.shapes)} of "
+                                         f"{w.matrices} matrices), given projector, {t:.1f} s"}
+    return out
+
+
+if __name__ == "__main__":
+    sys.exit(main())

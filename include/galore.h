@@ -200,6 +200,12 @@ const char* galore_status_string(galore_status_t s);
 const char* galore_last_cuda_error(void);
 /* Number of kernel launches issued by the library in this process (all layers). */
 int64_t galore_launch_count(void);
+/* Phase timing for benchmarks.  While enabled (process-wide), galore_step brackets its three
+ * phases with CUDA events on the step's stream: 0 projection, 1 Adam on R, 2 back-projection + weight
+ * write.  galore_profile_read synchronises on the recorded events, adds the elapsed milliseconds and
+ * the number of brackets per phase into ms3 / count3 (host arrays of 3) and forgets the events. */
+galore_status_t galore_profile_enable(int32_t on);
+galore_status_t galore_profile_read(double* ms3, int64_t* count3);
 
 #ifdef __cplusplus
 }

@@ -84,6 +84,8 @@ _PROTOTYPES = {
     "galore_status_string": (C.c_char_p, [C.c_int]),
     "galore_last_cuda_error": (C.c_char_p, []),
     "galore_launch_count": (C.c_int64, []),
+    "galore_profile_enable": (C.c_int, [C.c_int32]),
+    "galore_profile_read": (C.c_int, [C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
 }
 
 
@@ -160,6 +162,18 @@ def galore_q8_dequantize(codes: torch.Tensor, absmax: torch.Tensor, is_signed: b
 
 def galore_launch_count() -> int:
     return int(lib().galore_launch_count())
+
+
+def galore_profile_enable(on: bool):
+    _check(lib().galore_profile_enable(int(on)), "galore_profile_enable")
+
+
+def galore_profile_read():
+    """Accumulated (milliseconds, brackets) per phase: projection, Adam on R, back-projection."""
+    ms = (C.c_double * 3)(0, 0, 0)
+    cnt = (C.c_int64 * 3)(0, 0, 0)
+    _check(lib().galore_profile_read(ms, cnt), "galore_profile_read")
+    return list(ms), list(cnt)
 
 
 class Layer:

@@ -6,7 +6,9 @@
 
 #include <algorithm>
 #include <atomic>
+#include <mutex>
 #include <new>
+#include <vector>
 #include <string>
 
 #include "adam.cuh"
@@ -24,6 +26,30 @@ void note_cuda_error(cudaError_t e, const char* where) {
   t_last_error = std::string(cudaGetErrorName(e)) + ": " + cudaGetErrorString(e) + " at " + where;
 }
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// ---- optional phase timing (benchmarks) ------------------------------------------
+struct PhaseEvent { int phase; cudaEvent_t a, b; };
+static std::atomic<int> g_profile{0};
+static std::mutex g_profile_mutex;
+static std::vector<PhaseEvent> g_phase_events;
+
+struct PhaseTimer {
+  bool on;
+  PhaseEvent ev;
+  cudaStream_t st;
+  PhaseTimer(int phase, cudaStream_t s) : on(g_profile.load(std::memory_order_relaxed) != 0), st(s) {
+    if (!on) return;
+    ev.phase = phase;
+    if (cudaEventCreate(&ev.a) != cudaSuccess || cudaEventCreate(&ev.b) != cudaSuccess) { on = false; return; }
+    cudaEventRecord(ev.a, st);
+  }
+  ~PhaseTimer() {
+    if (!on) return;
+    cudaEventRecord(ev.b, st);
+    std::lock_guard<std::mutex> lock(g_profile_mutex);
+    g_phase_events.push_back(ev);
+  }
+};
 
 template <typename TS, typename TD>
 __global__ void convert_copy_kernel(const TS* __restrict__ src, TD* __restrict__ dst, int64_t count) {
@@ -176,17 +202,22 @@ galore_status_t back_project_simt(galore_layer* l, void* W, int64_t ldw, float s
 galore_status_t step_simt(galore_layer* l, void* W, int64_t ldw, const void* G, int64_t ldg, float lr,
                           const AdamParams& ap, cudaStream_t st) {
   const bool pb = l->cfg.p_dtype == GALORE_BF16, gb = l->cfg.g_dtype == GALORE_BF16, wb = l->cfg.w_dtype == GALORE_BF16;
-  if (pb && gb) GALORE_TRY((project_simt<__nv_bfloat16, __nv_bfloat16>(l, G, ldg, st)));
-  else if (pb) GALORE_TRY((project_simt<__nv_bfloat16, float>(l, G, ldg, st)));
-  else if (gb) GALORE_TRY((project_simt<float, __nv_bfloat16>(l, G, ldg, st)));
-  else GALORE_TRY((project_simt<float, float>(l, G, ldg, st)));
-
-  if (l->cfg.state_fmt == GALORE_STATE_F32)
-    GALORE_TRY(launch_adam_f32(l->Rpart, l->proj_splits, l->nel, l->nel, l->M, l->V, l->Nbuf, GALORE_F32, ap, l->status, st));
-  else
-    GALORE_TRY(launch_adam_q8(l->Rpart, l->proj_splits, l->nel, l->nel, l->Mc, l->Mam, l->Vc, l->Vam, l->q_block, l->Nbuf,
-                              GALORE_F32, ap, l->status, st));
-
+  {
+    PhaseTimer pt(0, st);
+    if (pb && gb) GALORE_TRY((project_simt<__nv_bfloat16, __nv_bfloat16>(l, G, ldg, st)));
+    else if (pb) GALORE_TRY((project_simt<__nv_bfloat16, float>(l, G, ldg, st)));
+    else if (gb) GALORE_TRY((project_simt<float, __nv_bfloat16>(l, G, ldg, st)));
+    else GALORE_TRY((project_simt<float, float>(l, G, ldg, st)));
+  }
+  {
+    PhaseTimer pt(1, st);
+    if (l->cfg.state_fmt == GALORE_STATE_F32)
+      GALORE_TRY(launch_adam_f32(l->Rpart, l->proj_splits, l->nel, l->nel, l->M, l->V, l->Nbuf, GALORE_F32, ap, l->status, st));
+    else
+      GALORE_TRY(launch_adam_q8(l->Rpart, l->proj_splits, l->nel, l->nel, l->Mc, l->Mam, l->Vc, l->Vam, l->q_block, l->Nbuf,
+                                GALORE_F32, ap, l->status, st));
+  }
+  PhaseTimer pt(2, st);
   const float scale = lr * l->cfg.alpha;
   if (pb && wb) return back_project_simt<__nv_bfloat16, __nv_bfloat16>(l, W, ldw, scale, st);
   if (pb) return back_project_simt<__nv_bfloat16, float>(l, W, ldw, scale, st);
@@ -484,5 +515,35 @@ const char* galore_status_string(galore_status_t s) {
 const char* galore_last_cuda_error(void) { return t_last_error.c_str(); }
 
 int64_t galore_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+galore_status_t galore_profile_enable(int32_t on) {
+  g_profile.store(on ? 1 : 0);
+  return GALORE_OK;
+}
+
+galore_status_t galore_profile_read(double* ms3, int64_t* count3) {
+  if (!ms3 || !count3) return GALORE_ERR_INVALID_ARG;
+  std::vector<PhaseEvent> evs;
+  {
+    std::lock_guard<std::mutex> lock(g_profile_mutex);
+    evs.swap(g_phase_events);
+  }
+  galore_status_t rc = GALORE_OK;
+  for (PhaseEvent& e : evs) {
+    float ms = 0.f;
+    cudaError_t err = cudaEventSynchronize(e.b);
+    if (err == cudaSuccess) err = cudaEventElapsedTime(&ms, e.a, e.b);
+    if (err != cudaSuccess) {
+      note_cuda_error(err, "profile event");
+      rc = GALORE_ERR_CUDA;
+    } else if (e.phase >= 0 && e.phase < 3) {
+      ms3[e.phase] += ms;
+      count3[e.phase] += 1;
+    }
+    cudaEventDestroy(e.a);
+    cudaEventDestroy(e.b);
+  }
+  return rc;
+}
 
 }  // extern "C"
