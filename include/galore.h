@@ -161,6 +161,43 @@ galore_status_t galore_refresh_projector(galore_layer_t* layer, const void* G, i
 /* Releases the host handle.  Device buffers stay with the caller. */
 galore_status_t galore_free(galore_layer_t* layer);
 
+/* A step that needs no workspace from the caller and allocates nothing.  (The paper has no
+ * counterpart: this is a convenience of this library.)
+ *
+ * For callers that cannot hand the library a scratch buffer or let it obtain one: plug-ins of a
+ * host framework that owns all device memory through its own pool and bans cudaMalloc, call sites
+ * where the device-wide synchronisation of cudaMalloc/cudaFree is not acceptable, threads that
+ * must stay away from the allocator.  The step's intermediates (split-K partial sums of R and the
+ * normalised update N) live in an array of GALORE_STATIC_SCRATCH_BYTES bytes that is part of the
+ * library image; every GPU that loads the library holds that much memory until the process exits.
+ *
+ * One fp32 iteration of Algorithm 1 on explicit arrays, all device memory, row-major:
+ *   P  projector, rows x rank packed (rows = m for the left side, n for the right), read only
+ *   M, V  moments, shape of R (rank x n left, m x rank right) packed, updated in place
+ *   W  m x n with leading dimension ldw, updated in place;  G  m x n with ldg, read only
+ *   completed_steps  k of Algorithm 1 before this call (bias correction uses k + 1)
+ *   side  galore_side_t (AUTO: left iff m <= n)
+ *   device_flags  optional host pointer; when non-NULL the call waits for the stream and stores
+ *                 the GALORE_DEV_* bits the kernels latched, otherwise it returns without waiting
+ * No refresh is done here: the caller supplies P.
+ *
+ * Limits and rules
+ *   - 256 + 4 * (splits + 1) * (elements of R) bytes, each part rounded up to 256, must fit in the
+ *     array (splits <= 16 is chosen by the library); larger layers are refused with
+ *     GALORE_ERR_BUFFER_TOO_SMALL and nothing is launched.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside of any stream capture.
+ *   - All calls on a device share the array, and it keeps the previous call's contents.  The call
+ *     clears the status word it needs at zero; everything else it reads it has written first.
+ *     Calls whose GPU work can overlap (two streams, two threads) race on the array: serialise
+ *     them.
+ *   - Calls no cudaMalloc, cudaFree or other allocating routine. */
+#define GALORE_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank, int32_t side, float alpha, float beta1,
+                                   float beta2, float eps, int64_t completed_steps, const float* P, float* M,
+                                   float* V, float* W, int64_t ldw, const float* G, int64_t ldg, float lr,
+                                   int32_t* device_flags, void* stream);
+
 /* ---- accessors (tests, checkpoint/resume) -------------------------------- */
 
 /* Projector as fp32, rows x r row-major packed (rows = m left, n right), device memory. */

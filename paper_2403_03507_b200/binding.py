@@ -69,6 +69,9 @@ _PROTOTYPES = {
                                     C.POINTER(C.c_void_p), C.POINTER(C.c_int64), C.c_int32, C.c_float, C.c_void_p]),
     "galore_refresh_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.POINTER(RefreshInfo)]),
     "galore_free": (C.c_int, [C.c_void_p]),
+    "galore_step_static": (C.c_int, [C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_float, C.c_float, C.c_float,
+                                     C.c_float, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+                                     C.c_void_p, C.c_int64, C.c_float, C.POINTER(C.c_int32), C.c_void_p]),
     "galore_get_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "galore_set_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "galore_get_moments": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -158,6 +161,27 @@ def galore_q8_dequantize(codes: torch.Tensor, absmax: torch.Tensor, is_signed: b
     _check(lib().galore_q8_dequantize(codes.data_ptr(), absmax.data_ptr(), codes.numel(), int(is_signed), block,
                                       out.data_ptr(), _stream_ptr(stream)), "galore_q8_dequantize")
     return out
+
+
+STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
+
+
+def galore_step_static(P, M, V, W, G, lr, completed_steps, alpha=0.25, beta1=0.9, beta2=0.999, eps=1e-8,
+                       side=SIDE_AUTO, want_flags=True, stream=None):
+    """One fp32 step on explicit device arrays using the library's built-in scratch (no workspace,
+    no allocation inside the library).  For callers that may not allocate device memory; layers
+    whose intermediates exceed STATIC_SCRATCH_BYTES are refused.  Calls must not overlap on the GPU.
+    Returns the device status bits (0 when want_flags is False)."""
+    for t in (P, M, V, W, G):
+        assert t.is_cuda and t.dtype == torch.float32
+    assert P.is_contiguous() and M.is_contiguous() and V.is_contiguous()
+    m, n = W.shape
+    flags = C.c_int32(0)
+    _check(lib().galore_step_static(m, n, P.shape[1], side, alpha, beta1, beta2, eps, completed_steps, P.data_ptr(),
+                                    M.data_ptr(), V.data_ptr(), W.data_ptr(), W.stride(0), G.data_ptr(), G.stride(0),
+                                    lr, C.byref(flags) if want_flags else None, _stream_ptr(stream)),
+           "galore_step_static")
+    return flags.value
 
 
 def galore_launch_count() -> int:
