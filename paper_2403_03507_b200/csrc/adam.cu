@@ -120,17 +120,18 @@ template <typename TN>
 __global__ void __launch_bounds__(256)
 adam_f32_kernel(const float* __restrict__ Rpart, int splits, int64_t split_stride, int64_t nel,
                 float* __restrict__ M, float* __restrict__ V, TN* __restrict__ Nout, AdamParams p,
-                int32_t* __restrict__ status) {
+                StateGeom g, int32_t* __restrict__ status) {
   bool bad = false;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nel; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t ir = g.r_index(i), in = g.n_index(i);
     float r = 0.f;
-    for (int s = 0; s < splits; ++s) r += Rpart[(int64_t)s * split_stride + i];
+    for (int s = 0; s < splits; ++s) r += Rpart[(int64_t)s * split_stride + ir];
     bad |= !isfinite(r);
     float m = p.b1 * M[i] + p.omb1 * r;
     float v = p.b2 * V[i] + p.omb2 * (r * r);
     M[i] = m;
     V[i] = v;
-    store_n(Nout, i, adam_normalised(m, v, p));
+    store_n(Nout, in, adam_normalised(m, v, p));
   }
   if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(status, GALORE_DEV_NONFINITE);
 }
@@ -142,7 +143,8 @@ template <typename TN, int EPT>
 __global__ void __launch_bounds__(256)
 adam_q8_kernel(const float* __restrict__ Rpart, int splits, int64_t split_stride, int64_t nel,
                uint8_t* __restrict__ Mc, float* __restrict__ Mam, uint8_t* __restrict__ Vc,
-               float* __restrict__ Vam, TN* __restrict__ Nout, AdamParams p, int32_t* __restrict__ status) {
+               float* __restrict__ Vam, TN* __restrict__ Nout, AdamParams p, StateGeom g,
+               int32_t* __restrict__ status) {
   __shared__ float s_code_s[256], s_code_u[256], s_mid_s[256], s_mid_u[256];
   __shared__ float red[8];
   s_code_s[threadIdx.x] = c_code_s[threadIdx.x];
@@ -162,14 +164,15 @@ adam_q8_kernel(const float* __restrict__ Rpart, int splits, int64_t split_stride
   for (int e = 0; e < EPT; ++e) {
     int64_t i = base + e;
     if (i < nel) {
+      const int64_t ir = g.r_index(i);
       float r = 0.f;
-      for (int s = 0; s < splits; ++s) r += Rpart[(int64_t)s * split_stride + i];
+      for (int s = 0; s < splits; ++s) r += Rpart[(int64_t)s * split_stride + ir];
       bad |= !isfinite(r);
       float m_old = s_code_s[Mc[i]] * am_m;
       float v_old = s_code_u[Vc[i]] * am_v;
       m[e] = p.b1 * m_old + p.omb1 * r;
       v[e] = p.b2 * v_old + p.omb2 * (r * r);
-      store_n(Nout, i, adam_normalised(m[e], v[e], p));
+      store_n(Nout, g.n_index(i), adam_normalised(m[e], v[e], p));
       mx_m = fmaxf(mx_m, fabsf(m[e]));
       mx_v = fmaxf(mx_v, fabsf(v[e]));
     } else {
@@ -240,31 +243,32 @@ static bool valid_block(int block) {
 
 template <typename TN>
 static galore_status_t adam_f32_t(const float* Rpart, int splits, int64_t split_stride, int64_t nel, float* M,
-                                  float* V, TN* Nout, const AdamParams& p, int32_t* status, cudaStream_t st) {
+                                  float* V, TN* Nout, const AdamParams& p, const StateGeom& g, int32_t* status,
+                                  cudaStream_t st) {
   int64_t blocks = std::min<int64_t>(ceil_div(nel, 256), 148 * 16);
-  adam_f32_kernel<TN><<<(unsigned)blocks, 256, 0, st>>>(Rpart, splits, split_stride, nel, M, V, Nout, p, status);
+  adam_f32_kernel<TN><<<(unsigned)blocks, 256, 0, st>>>(Rpart, splits, split_stride, nel, M, V, Nout, p, g, status);
   GALORE_LAUNCH_CHECK();
   return GALORE_OK;
 }
 
 galore_status_t launch_adam_f32(const float* Rpart, int splits, int64_t split_stride, int64_t nel, float* M,
                                 float* V, void* Nout, int32_t n_dtype, const AdamParams& p, int32_t* status,
-                                cudaStream_t st) {
+                                cudaStream_t st, const StateGeom& g) {
   if (nel <= 0) return GALORE_OK;
   if (n_dtype == GALORE_BF16)
-    return adam_f32_t(Rpart, splits, split_stride, nel, M, V, (__nv_bfloat16*)Nout, p, status, st);
-  return adam_f32_t(Rpart, splits, split_stride, nel, M, V, (float*)Nout, p, status, st);
+    return adam_f32_t(Rpart, splits, split_stride, nel, M, V, (__nv_bfloat16*)Nout, p, g, status, st);
+  return adam_f32_t(Rpart, splits, split_stride, nel, M, V, (float*)Nout, p, g, status, st);
 }
 
 template <typename TN>
 static galore_status_t adam_q8_t(const float* Rpart, int splits, int64_t split_stride, int64_t nel, uint8_t* Mc,
                                  float* Mam, uint8_t* Vc, float* Vam, int block, TN* Nout, const AdamParams& p,
-                                 int32_t* status, cudaStream_t st) {
+                                 const StateGeom& g, int32_t* status, cudaStream_t st) {
   unsigned grid = (unsigned)ceil_div(nel, block);
 #define GALORE_Q8_CASE(EPT)                                                                              \
   case EPT * 256:                                                                                        \
     adam_q8_kernel<TN, EPT><<<grid, 256, 0, st>>>(Rpart, splits, split_stride, nel, Mc, Mam, Vc, Vam,    \
-                                                   Nout, p, status);                                     \
+                                                   Nout, p, g, status);                                  \
     break;
   switch (block) {
     GALORE_Q8_CASE(1) GALORE_Q8_CASE(2) GALORE_Q8_CASE(4) GALORE_Q8_CASE(8) GALORE_Q8_CASE(16)
@@ -277,13 +281,13 @@ static galore_status_t adam_q8_t(const float* Rpart, int splits, int64_t split_s
 
 galore_status_t launch_adam_q8(const float* Rpart, int splits, int64_t split_stride, int64_t nel, uint8_t* Mc,
                                float* Mam, uint8_t* Vc, float* Vam, int block, void* Nout, int32_t n_dtype,
-                               const AdamParams& p, int32_t* status, cudaStream_t st) {
+                               const AdamParams& p, int32_t* status, cudaStream_t st, const StateGeom& g) {
   if (nel <= 0) return GALORE_OK;
   if (!valid_block(block)) return GALORE_ERR_INVALID_ARG;
   GALORE_TRY(q8_ensure_tables());
   if (n_dtype == GALORE_BF16)
-    return adam_q8_t(Rpart, splits, split_stride, nel, Mc, Mam, Vc, Vam, block, (__nv_bfloat16*)Nout, p, status, st);
-  return adam_q8_t(Rpart, splits, split_stride, nel, Mc, Mam, Vc, Vam, block, (float*)Nout, p, status, st);
+    return adam_q8_t(Rpart, splits, split_stride, nel, Mc, Mam, Vc, Vam, block, (__nv_bfloat16*)Nout, p, g, status, st);
+  return adam_q8_t(Rpart, splits, split_stride, nel, Mc, Mam, Vc, Vam, block, (float*)Nout, p, g, status, st);
 }
 
 galore_status_t launch_q8_quantize(const float* x, int64_t nel, int is_signed, int block, uint8_t* codes,

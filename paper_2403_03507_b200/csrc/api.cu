@@ -73,7 +73,9 @@ struct galore_layer {
   int q_block;
   int64_t nblk;
   int block;             // columns of the refresh block
-  int proj_splits;       // K slices of the projection
+  int proj_splits;       // K slices of the projection on the fp32 path
+  int tc_splits;         // K slices of the projection on the tensor-core path
+  int64_t ld_part, ld_n; // padded row pitches of the R partials and of N on the tensor-core path
   int32_t n_dtype;       // dtype of the normalised update handed to the back-projection
   int64_t k;             // completed steps
   // device memory (all inside the caller's two buffers)
@@ -93,7 +95,8 @@ namespace {
 struct Sizes {
   bool left;
   int64_t d, L, srows, scols, nel, nblk;
-  int q_block, block, proj_splits;
+  int q_block, block, proj_splits, tc_splits;
+  int64_t ld_part, ld_n;
   bool tensor_path;
   size_t off_P, off_M, off_V, off_Mam, off_Vam, state_bytes;
   size_t off_status, off_R, off_N, off_refresh, ws_bytes;
@@ -130,9 +133,7 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
   s->tensor_path = eligible && c->path != GALORE_PATH_FP32;
 
   // K slices of the projection: enough CTAs to fill the machine when R is small
-  if (s->tensor_path) {
-    s->proj_splits = tensor_proj_splits(*c, s->left);
-  } else {
+  {
     const bool small = s->nel < (int64_t)128 * 128 * 96;
     const int64_t t = small ? 64 : 128;
     const int64_t tiles = ceil_div(s->srows, t) * ceil_div(s->scols, t);
@@ -140,6 +141,9 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
     want = (int)std::min<int64_t>(want, std::max<int64_t>(1, s->d / 64));
     s->proj_splits = simt_effective_splits((int)s->d, want);
   }
+  s->tc_splits = s->tensor_path ? tensor_proj_splits(*c, s->left) : 0;
+  s->ld_part = (s->scols + 3) / 4 * 4;     // 16-byte rows for vector stores
+  s->ld_n = (s->scols + 7) / 8 * 8;        // 16-byte bf16 rows for TMA
 
   size_t o = 0;
   s->off_P = o; o += align_up((size_t)s->d * r * dtype_size(c->p_dtype), 256);
@@ -157,8 +161,8 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
 
   o = 0;
   s->off_status = o; o += 256;
-  s->off_R = o; o += align_up((size_t)s->proj_splits * s->nel * 4, 256);
-  s->off_N = o; o += align_up((size_t)s->nel * 4, 256);
+  s->off_R = o; o += align_up(std::max((size_t)s->proj_splits * s->nel, (size_t)s->tc_splits * s->srows * s->ld_part) * 4, 256);
+  s->off_N = o; o += align_up(std::max((size_t)s->nel * 4, (size_t)s->srows * s->ld_n * 2), 256);
   s->off_refresh = o; o += refresh_workspace_bytes(s->d, s->L, r, s->block);
   s->ws_bytes = o;
   return GALORE_OK;
@@ -225,6 +229,31 @@ galore_status_t step_simt(galore_layer* l, void* W, int64_t ldw, const void* G, 
   return back_project_simt<float, float>(l, W, ldw, scale, st);
 }
 
+// projection and back-projection on tcgen05, Adam in between reading the padded partials
+galore_status_t step_tensor(galore_layer* l, void* W, int64_t ldw, const void* G, int64_t ldg, float lr,
+                            const AdamParams& ap, cudaStream_t st) {
+  {
+    PhaseTimer pt(0, st);
+    GALORE_TRY(tensor_project(&l->tc, l->cfg, l->left, G, ldg, l->status, st));
+  }
+  {
+    PhaseTimer pt(1, st);
+    StateGeom g;
+    g.cols = l->scols;
+    g.r_ld = l->ld_part;
+    g.n_ld = l->ld_n;
+    const int64_t split_stride = l->srows * l->ld_part;
+    if (l->cfg.state_fmt == GALORE_STATE_F32)
+      GALORE_TRY(launch_adam_f32(l->Rpart, l->tc.splits, split_stride, l->nel, l->M, l->V, l->Nbuf, GALORE_BF16, ap,
+                                 l->status, st, g));
+    else
+      GALORE_TRY(launch_adam_q8(l->Rpart, l->tc.splits, split_stride, l->nel, l->Mc, l->Mam, l->Vc, l->Vam, l->q_block,
+                                l->Nbuf, GALORE_BF16, ap, l->status, st, g));
+  }
+  PhaseTimer pt(2, st);
+  return tensor_back_project(&l->tc, l->cfg, l->left, W, ldw, lr * l->cfg.alpha, l->status, st);
+}
+
 galore_status_t do_refresh(galore_layer* l, const void* G, int64_t ldg, cudaStream_t st, galore_refresh_info_t* info) {
   RefreshProblem pr;
   pr.G = G;
@@ -276,6 +305,7 @@ galore_status_t galore_init_layer(const galore_config_t* cfg, void* state_buf, s
   l->has_projector = false;
   l->d = s.d; l->L = s.L; l->srows = s.srows; l->scols = s.scols; l->nel = s.nel;
   l->q_block = s.q_block; l->nblk = s.nblk; l->block = s.block; l->proj_splits = s.proj_splits;
+  l->tc_splits = s.tc_splits; l->ld_part = s.ld_part; l->ld_n = s.ld_n;
   l->n_dtype = s.tensor_path ? GALORE_BF16 : GALORE_F32;
   l->k = 0;
   char* sb = (char*)state_buf;
@@ -313,7 +343,7 @@ galore_status_t galore_init_layer(const galore_config_t* cfg, void* state_buf, s
     return GALORE_ERR_CUDA;
   }
   if (l->tensor_path) {
-    galore_status_t ts = tensor_plan_init(&l->tc, *cfg, l->left, l->P, l->Nbuf, l->Rpart, l->proj_splits);
+    galore_status_t ts = tensor_plan_init(&l->tc, *cfg, l->left, l->P, l->Nbuf, l->Rpart, l->tc_splits, l->ld_part, l->ld_n);
     if (ts < 0) {
       delete l;
       return ts;
@@ -351,10 +381,10 @@ galore_status_t galore_step(galore_layer_t* l, void* W, int64_t ldw, const void*
   ap.inv_bc1 = (float)(1.0 / (1.0 - pow((double)l->cfg.beta1, t)));
   ap.inv_bc2 = (float)(1.0 / (1.0 - pow((double)l->cfg.beta2, t)));
   galore_status_t s;
-  if (l->tensor_path) {
-    if (!tensor_operands_aligned(l->cfg, W, ldw, G, ldg)) return GALORE_ERR_ALIGNMENT;
-    s = step_tensor(&l->tc, l->cfg, l->left, W, ldw, G, ldg, lr * l->cfg.alpha, ap, l->M, l->V, l->Mc, l->Mam, l->Vc,
-                    l->Vam, l->q_block, l->nel, l->status, st);
+  if (l->tensor_path && tensor_operands_aligned(l->cfg, W, ldw, G, ldg)) {
+    s = step_tensor(l, W, ldw, G, ldg, lr, ap, st);
+  } else if (l->tensor_path && l->cfg.path == GALORE_PATH_TENSOR) {
+    return GALORE_ERR_ALIGNMENT;     // the caller insisted on tensor cores but these buffers cannot feed TMA
   } else {
     s = step_simt(l, W, ldw, G, ldg, lr, ap, st);
   }

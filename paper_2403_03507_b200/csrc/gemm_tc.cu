@@ -1,18 +1,598 @@
-// tcgen05 / TMEM / TMA projection kernels: not wired yet; the fp32 path carries every configuration.
+// Projection and back-projection of the GaLore step on the 5th-generation
+// tensor cores (sm_100a): bf16 operands staged in shared memory by TMA,
+// tcgen05.mma with fp32 accumulators in tensor memory, epilogues that either
+// store split-K partial sums of R or apply the update to W in place
+// (Algorithm 1: R = P^T G resp. G Q;  W <- W - lr * alpha * P N resp. N Q^T).
+//
+// One persistent CTA per SM, six warps:
+//   warp 0        TMA producer: fills a ring of kStages shared-memory stages
+//   warp 1        MMA issuer (one lane) and owner of the tensor-memory allocation
+//   warps 2..5    epilogue: tcgen05.ld of a finished accumulator, then global memory
+// Two accumulators of kBN columns alternate, so the epilogue of one tile runs
+// under the MMAs of the next.  Work units are (tile_m, tile_n, K slice); the
+// K slices of one output tile go to separate partial buffers that the Adam
+// kernel sums in a fixed order, so results do not depend on scheduling.
+//
+// Every wait on an mbarrier is bounded by a clock limit; when it runs out the
+// CTA latches GALORE_DEV_WAIT_EXPIRED, lets its outstanding copies land,
+// releases tensor memory and returns.
 #include "gemm_tc.cuh"
+
+#include <cudaTypedefs.h>
+
+#include <algorithm>
+#include <mutex>
 
 namespace galore {
 
-bool tensor_path_eligible(const galore_config_t&) { return false; }
-int tensor_proj_splits(const galore_config_t&, bool) { return 1; }
-galore_status_t tensor_plan_init(TensorPlan*, const galore_config_t&, bool, void*, void*, float*, int) {
-  return GALORE_ERR_UNIMPLEMENTED;
+namespace {
+
+constexpr int kBM = 128;          // rows of an output tile = TMEM lanes
+constexpr int kBN = 256;          // columns of an output tile = TMEM columns per accumulator
+constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int kStages = 4;
+constexpr int kUmmaK = 16;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr int kABytes = kBM * kBK * 2;            // 16 KiB
+constexpr int kBBytes = kBN * kBK * 2;            // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr long long kWaitLimitCycles = 4000000000LL;   // about two seconds
+
+enum { EPI_PARTIAL = 0, EPI_APPLY = 1 };
+
+struct TcParams {
+  int M, N, K;
+  int tiles_m, tiles_n, splits;
+  int kblocks_total, kblocks_per_split;
+  int m_fast;                 // 1: consecutive units walk tile_m first (B panel shared), 0: tile_n first
+  // EPI_PARTIAL
+  float* part;
+  int64_t ld_part, split_stride;
+  // EPI_APPLY
+  void* W;
+  int64_t ldw;
+  float scale;
+  int32_t* status;
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-bool tensor_operands_aligned(const galore_config_t&, const void*, int64_t, const void*, int64_t) { return false; }
-galore_status_t step_tensor(TensorPlan*, const galore_config_t&, bool, void*, int64_t, const void*, int64_t, float,
-                            const AdamParams&, float*, float*, uint8_t*, float*, uint8_t*, float*, int, int64_t,
-                            int32_t*, cudaStream_t) {
-  return GALORE_ERR_UNIMPLEMENTED;
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  Returns false when the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 63u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitLimitCycles) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_result, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem], 128 x kBN x 16, bf16 in, fp32 out
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// the mbarrier receives one arrival once every MMA issued so far by this thread has finished
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base lane + t)
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// ---- descriptors ------------------------------------------------------------------------
+// Shared-memory operand descriptor, 128-byte swizzle, tile base 1024-byte aligned.
+//  K-major  : rows of 64 bf16 (128 B); 8-row groups 1024 B apart (stride offset); leading offset unused.
+//  MN-major : 64-element (128 B) runs along M/N, one per k; 8-k groups 1024 B apart (stride offset);
+//             the next 64 elements of M/N start kBK * 128 B further on (leading offset).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major) {
+  const uint64_t lbo = mn_major ? (uint64_t)((kBK * 128) >> 4) : 1ull;
+  const uint64_t sbo = 1024 >> 4;
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, majors, N, M.
+__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+         ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+}
+
+struct Unit {
+  int m0, n0, split, kb_begin, kb_end;
+};
+
+__device__ __forceinline__ Unit decode_unit(const TcParams& p, int u) {
+  int tm, tn, s;
+  if (p.m_fast) {
+    tm = u % p.tiles_m;
+    s = (u / p.tiles_m) % p.splits;
+    tn = u / (p.tiles_m * p.splits);
+  } else {
+    tn = u % p.tiles_n;
+    s = (u / p.tiles_n) % p.splits;
+    tm = u / (p.tiles_n * p.splits);
+  }
+  Unit w;
+  w.m0 = tm * kBM;
+  w.n0 = tn * kBN;
+  w.split = s;
+  w.kb_begin = s * p.kblocks_per_split;
+  w.kb_end = min(p.kblocks_total, w.kb_begin + p.kblocks_per_split);
+  return w;
+}
+
+// ---- epilogues ----------------------------------------------------------------------------
+
+// thread owns row `row`, columns [col0, col0 + 32) of the tile
+__device__ __forceinline__ void epi_partial(const TcParams& p, const Unit& w, int row, int col0, const uint32_t (&v)[32]) {
+  if (row >= p.M) return;
+  float* dst = p.part + (int64_t)w.split * p.split_stride + (int64_t)row * p.ld_part + col0;
+  if (col0 + 32 <= p.N && (p.ld_part & 3) == 0) {
+#pragma unroll
+    for (int j = 0; j < 32; j += 4)
+      *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                        __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (col0 + j < p.N) dst[j] = __uint_as_float(v[j]);
+  }
+}
+
+template <typename TW>
+__device__ __forceinline__ void epi_apply(const TcParams& p, int row, int col0, const uint32_t (&v)[32]);
+
+template <>
+__device__ __forceinline__ void epi_apply<__nv_bfloat16>(const TcParams& p, int row, int col0, const uint32_t (&v)[32]) {
+  if (row >= p.M) return;
+  __nv_bfloat16* dst = (__nv_bfloat16*)p.W + (int64_t)row * p.ldw + col0;
+  if (col0 + 32 <= p.N) {
+#pragma unroll
+    for (int j = 0; j < 32; j += 8) {
+      uint4 raw = *reinterpret_cast<const uint4*>(dst + j);
+      __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        float2 f = __bfloat1622float2(h[q]);
+        f.x = fmaf(-p.scale, __uint_as_float(v[j + 2 * q]), f.x);
+        f.y = fmaf(-p.scale, __uint_as_float(v[j + 2 * q + 1]), f.y);
+        h[q] = __floats2bfloat162_rn(f.x, f.y);
+      }
+      *reinterpret_cast<uint4*>(dst + j) = raw;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(fmaf(-p.scale, __uint_as_float(v[j]), __bfloat162float(dst[j])));
+  }
+}
+
+template <>
+__device__ __forceinline__ void epi_apply<float>(const TcParams& p, int row, int col0, const uint32_t (&v)[32]) {
+  if (row >= p.M) return;
+  float* dst = (float*)p.W + (int64_t)row * p.ldw + col0;
+  if (col0 + 32 <= p.N) {
+#pragma unroll
+    for (int j = 0; j < 32; j += 4) {
+      float4 f = *reinterpret_cast<const float4*>(dst + j);
+      f.x = fmaf(-p.scale, __uint_as_float(v[j]), f.x);
+      f.y = fmaf(-p.scale, __uint_as_float(v[j + 1]), f.y);
+      f.z = fmaf(-p.scale, __uint_as_float(v[j + 2]), f.z);
+      f.w = fmaf(-p.scale, __uint_as_float(v[j + 3]), f.w);
+      *reinterpret_cast<float4*>(dst + j) = f;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (col0 + j < p.N) dst[j] = fmaf(-p.scale, __uint_as_float(v[j]), dst[j]);
+  }
+}
+
+// ---- the kernel -------------------------------------------------------------------------------
+
+template <bool A_MN, bool B_MN, int EPI, typename TW>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  // stage ring, 1024-byte aligned for the 128-byte swizzle
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t ring = (raw_addr + 1023u) & ~1023u;
+  uint8_t* ring_ptr = smem_raw + (ring - raw_addr);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring_ptr + kStages * kStageBytes);
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto accf_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
+  auto acce_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * kStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kStages + 5);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int total_units = p.tiles_m * p.tiles_n * p.splits;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(accf_bar(a), 1);
+      mbar_init(acce_bar(a), 4);     // one arrival per epilogue warp
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32((const void*)tmem_slot), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ================= TMA producer =================
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      long long issued = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+        const Unit w = decode_unit(p, u);
+        for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t a_dst = ring + stage * kStageBytes;
+          const uint32_t b_dst = a_dst + kABytes;
+          mbar_arrive_expect_tx(full_bar(stage), kStageBytes);
+          const int k0 = kb * kBK;
+          if (A_MN) {
+#pragma unroll
+            for (int j = 0; j < kBM / 64; ++j) tma_load_2d(a_dst + j * (kBK * 128), &map_a, w.m0 + 64 * j, k0, full_bar(stage));
+          } else {
+            tma_load_2d(a_dst, &map_a, k0, w.m0, full_bar(stage));
+          }
+          if (B_MN) {
+#pragma unroll
+            for (int j = 0; j < kBN / 64; ++j) tma_load_2d(b_dst + j * (kBK * 128), &map_b, w.n0 + 64 * j, k0, full_bar(stage));
+          } else {
+            tma_load_2d(b_dst, &map_b, k0, w.n0, full_bar(stage));
+          }
+          ++issued;
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // let the copies that are still in flight land before the CTA goes away
+        int s = stage;
+        uint32_t ph = phase;
+        const long long pending = issued < kStages ? issued : kStages;
+        for (long long i = 0; i < pending; ++i) {
+          if (--s < 0) { s = kStages - 1; ph ^= 1u; }
+          const long long t0 = clock64();
+          while (!mbar_try_wait(full_bar(s), ph) && clock64() - t0 < kWaitLimitCycles) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ================= MMA issuer =================
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc(A_MN, B_MN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+        const Unit w = decode_unit(p, u);
+        if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kBN);
+        for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = ring + stage * kStageBytes;
+          const uint32_t b_addr = a_addr + kABytes;
+          const uint64_t a_desc = smem_desc(a_addr, A_MN);
+          const uint64_t b_desc = smem_desc(b_addr, B_MN);
+#pragma unroll
+          for (int k = 0; k < kBK / kUmmaK; ++k) {
+            // K-major: 16 bf16 = 32 B along the swizzled row; MN-major: 16 k = two 8-k groups of 1024 B
+            const uint64_t a_adv = (uint64_t)((A_MN ? k * 2048 : k * 32) >> 4);
+            const uint64_t b_adv = (uint64_t)((B_MN ? k * 2048 : k * 32) >> 4);
+            umma_bf16(d_tmem, a_desc + a_adv, b_desc + b_adv, idesc, (kb > w.kb_begin || k > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(stage));            // stage reusable once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit(accf_bar(acc));         // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ================= epilogue =================
+    const int quarter = warp & 3;                   // TMEM lanes 32*quarter .. +31 belong to this warp
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+      const Unit w = decode_unit(p, u);
+      if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row = w.m0 + quarter * 32 + lane;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kBN);
+#pragma unroll 1
+      for (int c = 0; c < kBN; c += 32) {
+        if (w.n0 + c >= p.N) break;                 // columns past the matrix: nothing to write
+        uint32_t v[32];
+        tmem_ld_32x32(t_row + (uint32_t)c, v);
+        tmem_ld_wait();
+        if (EPI == EPI_PARTIAL) epi_partial(p, w, row, w.n0 + c, v);
+        else epi_apply<TW>(p, row, w.n0 + c, v);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acce_bar(acc));    // accumulator free for the MMA warp
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, GALORE_DEV_WAIT_EXPIRED);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---- host side --------------------------------------------------------------------------------------
+
+PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+std::mutex g_encode_mutex;
+
+galore_status_t ensure_encode() {
+  std::lock_guard<std::mutex> lock(g_encode_mutex);
+  if (g_encode) return GALORE_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  GALORE_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+  if (!fn || qres != cudaDriverEntryPointSuccess) return GALORE_ERR_CUDA;
+  g_encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
+  return GALORE_OK;
+}
+
+// bf16 matrix, `rows` x `cols` (cols contiguous), leading dimension ld; box = box_rows x 64 columns, 128-byte swizzle
+galore_status_t make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+  GALORE_TRY(ensure_encode());
+  if (((uintptr_t)base & 15) || (ld * 2) % 16) return GALORE_ERR_ALIGNMENT;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    note_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return GALORE_ERR_CUDA;
+  }
+  return GALORE_OK;
+}
+
+int sm_count() {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+  }
+  return sms;
+}
+
+template <bool A_MN, bool B_MN, int EPI, typename TW>
+galore_status_t launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, cudaStream_t st) {
+  auto kern = gemm_tc_kernel<A_MN, B_MN, EPI, TW>;
+  static bool configured = false;
+  if (!configured) {
+    GALORE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    configured = true;
+  }
+  const int units = p.tiles_m * p.tiles_n * p.splits;
+  const int grid = std::min(units, sm_count());
+  kern<<<grid, kThreads, kSmemBytes, st>>>(ma, mb, p);
+  GALORE_LAUNCH_CHECK();
+  return GALORE_OK;
+}
+
+void fill_tiles(TcParams& p, int M, int N, int K, int splits) {
+  p.M = M; p.N = N; p.K = K;
+  p.tiles_m = (int)ceil_div(M, kBM);
+  p.tiles_n = (int)ceil_div(N, kBN);
+  p.kblocks_total = (int)ceil_div(K, kBK);
+  if (splits < 1) splits = 1;
+  p.kblocks_per_split = (int)ceil_div(p.kblocks_total, splits);
+  p.splits = (int)ceil_div(p.kblocks_total, p.kblocks_per_split);
+}
+
+// K slices that fill the last wave of CTAs best, keeping at least 4 k-blocks per slice
+int choose_splits(int64_t M, int64_t N, int64_t K) {
+  const int64_t tiles = ceil_div(M, kBM) * ceil_div(N, kBN);
+  const int kblocks = (int)ceil_div(K, kBK);
+  const int sms = 148;
+  int best = 1;
+  double best_score = -1.0;
+  for (int s = 1; s <= 8; ++s) {
+    const int per = (int)ceil_div(kblocks, s);
+    if (s > 1 && per < 4) break;
+    const int eff_s = (int)ceil_div(kblocks, per);
+    if (eff_s != s) continue;
+    const int64_t units = tiles * s;
+    const double fill = (double)units / (double)(ceil_div(units, sms) * sms);
+    // each extra slice costs one more partial buffer to write and read back
+    const double score = fill - 0.02 * (s - 1);
+    if (score > best_score + 1e-9) { best_score = score; best = s; }
+  }
+  return best;
+}
+
+}  // namespace
+
+bool tensor_path_eligible(const galore_config_t& c) {
+  return c.g_dtype == GALORE_BF16 && c.p_dtype == GALORE_BF16 && (c.rank % 8) == 0;
+}
+
+int tensor_proj_splits(const galore_config_t& c, bool left) {
+  if (left) return choose_splits(c.rank, c.n, c.m);
+  return choose_splits(c.m, c.rank, c.n);
+}
+
+galore_status_t tensor_plan_init(TensorPlan* plan, const galore_config_t& c, bool left, void* P, void* Nbuf, float* Rpart,
+                                 int splits, int64_t ld_part, int64_t ld_n) {
+  plan->ready = false;
+  plan->splits = splits;
+  plan->P = P;
+  plan->Nbuf = Nbuf;
+  plan->Rpart = Rpart;
+  plan->ld_part = ld_part;
+  plan->ld_n = ld_n;
+  const int64_t r = c.rank;
+  if (left) {
+    // projection: A = P^T, MN-major from P (m x r);  back-projection: A = P, K-major
+    GALORE_TRY(make_map(&plan->map_p_proj, P, c.m, r, r, 64));
+    GALORE_TRY(make_map(&plan->map_p_back, P, c.m, r, r, kBM));
+    // back-projection: B = N (r x n), MN-major
+    GALORE_TRY(make_map(&plan->map_n_back, Nbuf, r, c.n, ld_n, 64));
+  } else {
+    // projection: B = Q (n x r), MN-major;  back-projection: B = Q^T, K-major from Q
+    GALORE_TRY(make_map(&plan->map_p_proj, P, c.n, r, r, 64));
+    GALORE_TRY(make_map(&plan->map_p_back, P, c.n, r, r, kBN));
+    // back-projection: A = N (m x r), K-major
+    GALORE_TRY(make_map(&plan->map_n_back, Nbuf, c.m, r, ld_n, kBM));
+  }
+  plan->ready = true;
+  return GALORE_OK;
+}
+
+bool tensor_operands_aligned(const galore_config_t& c, const void* W, int64_t ldw, const void* G, int64_t ldg) {
+  if (((uintptr_t)G & 15) || (ldg % 8)) return false;
+  if ((uintptr_t)W & 15) return false;
+  return c.w_dtype == GALORE_BF16 ? (ldw % 8) == 0 : (ldw % 4) == 0;
+}
+
+galore_status_t tensor_project(TensorPlan* plan, const galore_config_t& c, bool left, const void* G, int64_t ldg,
+                               int32_t* status, cudaStream_t st) {
+  if (!plan->ready) return GALORE_ERR_STATE;
+  const int r = c.rank;
+  TcParams p = {};
+  p.status = status;
+  p.part = plan->Rpart;
+  p.ld_part = plan->ld_part;
+  CUtensorMap map_g;
+  if (left) {
+    // R (r x n) = P^T G : A MN-major (P), B MN-major (G); G is the big operand, shared along tile_m
+    fill_tiles(p, r, (int)c.n, (int)c.m, plan->splits);
+    p.split_stride = (int64_t)r * plan->ld_part;
+    p.m_fast = 1;
+    GALORE_TRY(make_map(&map_g, G, c.m, c.n, ldg, 64));
+    return launch_tc<true, true, EPI_PARTIAL, float>(plan->map_p_proj, map_g, p, st);
+  }
+  // R (m x r) = G Q : A K-major (G), B MN-major (Q); G is the big operand, shared along tile_n
+  fill_tiles(p, (int)c.m, r, (int)c.n, plan->splits);
+  p.split_stride = (int64_t)c.m * plan->ld_part;
+  p.m_fast = 0;
+  GALORE_TRY(make_map(&map_g, G, c.m, c.n, ldg, kBM));
+  return launch_tc<false, true, EPI_PARTIAL, float>(map_g, plan->map_p_proj, p, st);
+}
+
+galore_status_t tensor_back_project(TensorPlan* plan, const galore_config_t& c, bool left, void* W, int64_t ldw,
+                                    float scale, int32_t* status, cudaStream_t st) {
+  if (!plan->ready) return GALORE_ERR_STATE;
+  TcParams p = {};
+  p.status = status;
+  p.W = W;
+  p.ldw = ldw;
+  p.scale = scale;
+  p.m_fast = 1;
+  fill_tiles(p, (int)c.m, (int)c.n, c.rank, 1);
+  const bool wb = c.w_dtype == GALORE_BF16;
+  if (left) {
+    // W -= scale * P N : A K-major (P), B MN-major (N)
+    if (wb) return launch_tc<false, true, EPI_APPLY, __nv_bfloat16>(plan->map_p_back, plan->map_n_back, p, st);
+    return launch_tc<false, true, EPI_APPLY, float>(plan->map_p_back, plan->map_n_back, p, st);
+  }
+  // W -= scale * N Q^T : A K-major (N), B K-major (Q)
+  if (wb) return launch_tc<false, false, EPI_APPLY, __nv_bfloat16>(plan->map_n_back, plan->map_p_back, p, st);
+  return launch_tc<false, false, EPI_APPLY, float>(plan->map_n_back, plan->map_p_back, p, st);
 }
 
 }  // namespace galore
