@@ -81,7 +81,7 @@ typedef struct {
   int32_t rank;            /* r, 1 <= r <= min(m, n) */
   float alpha;             /* scale factor, not divided by r (Sec. 4.4) */
   int32_t refresh_gap;     /* T >= 1 */
-  float beta1, beta2, eps;
+  double beta1, beta2, eps; /* Adam; doubles so that 1 - beta is formed from the exact decimal the caller means */
   int32_t side;            /* galore_side_t; AUTO = left iff m <= n (Sec. 4.2) */
   int32_t w_dtype;         /* galore_dtype_t of W */
   int32_t g_dtype;         /* galore_dtype_t of G */
@@ -193,8 +193,8 @@ galore_status_t galore_free(galore_layer_t* layer);
  *     them.
  *   - Calls no cudaMalloc, cudaFree or other allocating routine. */
 #define GALORE_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
-galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank, int32_t side, float alpha, float beta1,
-                                   float beta2, float eps, int64_t completed_steps, const float* P, float* M,
+galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank, int32_t side, float alpha, double beta1,
+                                   double beta2, double eps, int64_t completed_steps, const float* P, float* M,
                                    float* V, float* W, int64_t ldw, const float* G, int64_t ldg, float lr,
                                    int32_t* device_flags, void* stream);
 
@@ -232,6 +232,8 @@ galore_status_t galore_q8_dequantize(const uint8_t* codes, const float* absmax, 
                                      int32_t is_signed, int32_t block, float* out, void* stream);
 
 /* ---- diagnostics ---------------------------------------------------------- */
+/* sizeof(galore_config_t) and sizeof(galore_refresh_info_t) as compiled, for bindings to check their marshalling. */
+galore_status_t galore_abi_sizes(size_t* config_bytes, size_t* refresh_info_bytes);
 const char* galore_status_string(galore_status_t s);
 /* Text of the last CUDA error seen by this thread's calls into the library ("" if none). */
 const char* galore_last_cuda_error(void);

@@ -30,7 +30,7 @@ _TORCH = {F32: torch.float32, BF16: torch.bfloat16}
 class Config(C.Structure):
     _fields_ = [
         ("m", C.c_int64), ("n", C.c_int64), ("rank", C.c_int32), ("alpha", C.c_float),
-        ("refresh_gap", C.c_int32), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+        ("refresh_gap", C.c_int32), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
         ("side", C.c_int32), ("w_dtype", C.c_int32), ("g_dtype", C.c_int32), ("p_dtype", C.c_int32),
         ("state_fmt", C.c_int32), ("q_block", C.c_int32), ("auto_refresh", C.c_int32), ("path", C.c_int32),
         ("refresh_tol", C.c_float), ("refresh_max_iters", C.c_int32), ("refresh_oversample", C.c_int32),
@@ -69,8 +69,8 @@ _PROTOTYPES = {
                                     C.POINTER(C.c_void_p), C.POINTER(C.c_int64), C.c_int32, C.c_float, C.c_void_p]),
     "galore_refresh_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.POINTER(RefreshInfo)]),
     "galore_free": (C.c_int, [C.c_void_p]),
-    "galore_step_static": (C.c_int, [C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_float, C.c_float, C.c_float,
-                                     C.c_float, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+    "galore_step_static": (C.c_int, [C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_float, C.c_double, C.c_double,
+                                     C.c_double, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                      C.c_void_p, C.c_int64, C.c_float, C.POINTER(C.c_int32), C.c_void_p]),
     "galore_get_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "galore_set_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -84,6 +84,7 @@ _PROTOTYPES = {
     "galore_q8_codebook": (C.c_int, [C.c_int32, C.POINTER(C.c_float)]),
     "galore_q8_quantize": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "galore_q8_dequantize": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
+    "galore_abi_sizes": (C.c_int, [C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
     "galore_status_string": (C.c_char_p, [C.c_int]),
     "galore_last_cuda_error": (C.c_char_p, []),
     "galore_launch_count": (C.c_int64, []),
@@ -102,6 +103,10 @@ def lib():
         for name, (res, args) in _PROTOTYPES.items():
             fn = getattr(handle, name)
             fn.restype, fn.argtypes = res, args
+        a, b = C.c_size_t(), C.c_size_t()
+        handle.galore_abi_sizes(C.byref(a), C.byref(b))
+        if (a.value, b.value) != (C.sizeof(Config), C.sizeof(RefreshInfo)):
+            raise ImportError("libgalore.so and binding.py disagree on the struct layout: rebuild the library")
         _lib = handle
     return _lib
 

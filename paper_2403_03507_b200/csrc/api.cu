@@ -107,7 +107,7 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
   if (c->m <= 0 || c->n <= 0 || c->m > 0x7fffffff || c->n > 0x7fffffff) return GALORE_ERR_SHAPE;
   if (c->rank < 1 || c->rank > std::min(c->m, c->n)) return GALORE_ERR_SHAPE;
   if (c->refresh_gap < 1) return GALORE_ERR_INVALID_ARG;
-  if (!(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f) || !(c->eps >= 0.f))
+  if (!(c->beta1 >= 0.0 && c->beta1 < 1.0) || !(c->beta2 >= 0.0 && c->beta2 < 1.0) || !(c->eps >= 0.0))
     return GALORE_ERR_INVALID_ARG;
   if (c->side < GALORE_SIDE_AUTO || c->side > GALORE_SIDE_RIGHT) return GALORE_ERR_INVALID_ARG;
   for (int32_t dt : {c->w_dtype, c->g_dtype, c->p_dtype})
@@ -373,13 +373,13 @@ galore_status_t galore_step(galore_layer_t* l, void* W, int64_t ldw, const void*
   if (!l->has_projector) return GALORE_ERR_STATE;
   const double t = (double)(l->k + 1);
   AdamParams ap;
-  ap.b1 = l->cfg.beta1;
-  ap.b2 = l->cfg.beta2;
-  ap.omb1 = (float)(1.0 - (double)l->cfg.beta1);
-  ap.omb2 = (float)(1.0 - (double)l->cfg.beta2);
-  ap.eps = l->cfg.eps;
-  ap.inv_bc1 = (float)(1.0 / (1.0 - pow((double)l->cfg.beta1, t)));
-  ap.inv_bc2 = (float)(1.0 / (1.0 - pow((double)l->cfg.beta2, t)));
+  ap.b1 = (float)l->cfg.beta1;
+  ap.b2 = (float)l->cfg.beta2;
+  ap.omb1 = (float)(1.0 - l->cfg.beta1);
+  ap.omb2 = (float)(1.0 - l->cfg.beta2);
+  ap.eps = (float)l->cfg.eps;
+  ap.inv_bc1 = (float)(1.0 / (1.0 - pow(l->cfg.beta1, t)));
+  ap.inv_bc2 = (float)(1.0 / (1.0 - pow(l->cfg.beta2, t)));
   galore_status_t s;
   if (l->tensor_path && tensor_operands_aligned(l->cfg, W, ldw, G, ldg)) {
     s = step_tensor(l, W, ldw, G, ldg, lr, ap, st);
@@ -540,6 +540,12 @@ const char* galore_status_string(galore_status_t s) {
     case GALORE_ERR_UNIMPLEMENTED: return "not implemented for this configuration";
   }
   return "unknown status";
+}
+
+galore_status_t galore_abi_sizes(size_t* config_bytes, size_t* refresh_info_bytes) {
+  if (config_bytes) *config_bytes = sizeof(galore_config_t);
+  if (refresh_info_bytes) *refresh_info_bytes = sizeof(galore_refresh_info_t);
+  return GALORE_OK;
 }
 
 const char* galore_last_cuda_error(void) { return t_last_error.c_str(); }

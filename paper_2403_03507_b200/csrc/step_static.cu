@@ -50,7 +50,7 @@ static galore_status_t static_scratch(void** out) {
 using namespace galore;
 
 extern "C" galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank, int32_t side, float alpha,
-                                               float beta1, float beta2, float eps, int64_t completed_steps,
+                                               double beta1, double beta2, double eps, int64_t completed_steps,
                                                const float* P, float* M, float* V, float* W, int64_t ldw,
                                                const float* G, int64_t ldg, float lr, int32_t* device_flags,
                                                void* stream) {
@@ -59,7 +59,7 @@ extern "C" galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank
   if (rank < 1 || rank > (m < n ? m : n)) return GALORE_ERR_SHAPE;
   if (ldw < n || ldg < n || completed_steps < 0) return GALORE_ERR_INVALID_ARG;
   if (side < GALORE_SIDE_AUTO || side > GALORE_SIDE_RIGHT) return GALORE_ERR_INVALID_ARG;
-  if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps >= 0.f)) return GALORE_ERR_INVALID_ARG;
+  if (!(beta1 >= 0.0 && beta1 < 1.0) || !(beta2 >= 0.0 && beta2 < 1.0) || !(eps >= 0.0)) return GALORE_ERR_INVALID_ARG;
   const bool left = side == GALORE_SIDE_AUTO ? (m <= n) : (side == GALORE_SIDE_LEFT);
   const int r = rank;
   const int64_t d = left ? m : n;
@@ -94,13 +94,13 @@ extern "C" galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank
 
   const double t = (double)(completed_steps + 1);
   AdamParams ap;
-  ap.b1 = beta1;
-  ap.b2 = beta2;
-  ap.omb1 = (float)(1.0 - (double)beta1);
-  ap.omb2 = (float)(1.0 - (double)beta2);
-  ap.eps = eps;
-  ap.inv_bc1 = (float)(1.0 / (1.0 - pow((double)beta1, t)));
-  ap.inv_bc2 = (float)(1.0 / (1.0 - pow((double)beta2, t)));
+  ap.b1 = (float)beta1;
+  ap.b2 = (float)beta2;
+  ap.omb1 = (float)(1.0 - beta1);
+  ap.omb2 = (float)(1.0 - beta2);
+  ap.eps = (float)eps;
+  ap.inv_bc1 = (float)(1.0 / (1.0 - pow(beta1, t)));
+  ap.inv_bc2 = (float)(1.0 / (1.0 - pow(beta2, t)));
   GALORE_TRY(launch_adam_f32(Rpart, splits, nel, nel, M, V, Nbuf, GALORE_F32, ap, status, st));
 
   EpiApplyW<float> apply{W, ldw, lr * alpha};

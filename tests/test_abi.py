@@ -31,7 +31,10 @@ def test_library_exports_every_declared_symbol():
 
 def test_config_struct_layout_matches_header():
     # the header's galore_config_t: field order and sizes as marshalled by the binding
-    assert C.sizeof(gb.Config) == 128
+    assert C.sizeof(gb.Config) == 144
+    a, b = C.c_size_t(), C.c_size_t()
+    assert gb.lib().galore_abi_sizes(C.byref(a), C.byref(b)) == 0
+    assert (a.value, b.value) == (C.sizeof(gb.Config), C.sizeof(gb.RefreshInfo))
     assert gb.Config.seed.offset % 8 == 0
     assert C.sizeof(gb.RefreshInfo) == 56
 
