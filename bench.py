@@ -178,6 +178,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--projector", default="refresh", choices=["refresh", "random"],
+                    help="refresh: one real refresh per distinct shape (timed, reported); random: a random orthonormal "
+                         "projector (step timing does not depend on P's values; for short profiling runs)")
     ap.add_argument("--extra-workloads", default="", help="comma-separated workloads also timed (device-resident only)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else max(args.warmup, 0)
@@ -258,7 +261,11 @@ def time_workload(w, args, dev, dist, world, rank, full):
         first = None
         for c in range(count):
             layer = gb.Layer(cfgs[(m, n)], device=dev, workspace=workspace)
-            if first is None:
+            if first is None and args.projector == "random":
+                d = m if m <= n else n
+                first = torch.linalg.qr(torch.randn(d, w.rank, device=dev))[0].contiguous()
+                layer.set_projector(first)
+            elif first is None:
                 t0 = torch.cuda.Event(enable_timing=True)
                 t1 = torch.cuda.Event(enable_timing=True)
                 t0.record()

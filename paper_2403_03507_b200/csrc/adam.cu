@@ -138,7 +138,8 @@ adam_f32_kernel(const float* __restrict__ Rpart, int splits, int64_t split_strid
 
 // ---- 8-bit block-wise moments ---------------------------------------------------
 // One CTA per quantisation block of EPT * 256 elements; thread t owns elements
-// [t*EPT, (t+1)*EPT) of the block.
+// t, t + 256, t + 512, ... of the block, so every warp-level access is one
+// contiguous run whatever the alignment of the block.
 template <typename TN, int EPT>
 __global__ void __launch_bounds__(256)
 adam_q8_kernel(const float* __restrict__ Rpart, int splits, int64_t split_stride, int64_t nel,
@@ -155,35 +156,47 @@ adam_q8_kernel(const float* __restrict__ Rpart, int splits, int64_t split_stride
 
   constexpr int QB = EPT * 256;
   const int64_t blk = blockIdx.x;
-  const int64_t base = blk * QB + (int64_t)threadIdx.x * EPT;
+  const int64_t base = blk * QB + threadIdx.x;
   const float am_m = Mam[blk], am_v = Vam[blk];
+  // position of the thread's first element in the padded R / N buffers; advanced by 256 per element
+  const bool packed = (g.cols == 0) || (g.r_ld == g.cols && g.n_ld == g.cols);
+  int64_t row = 0, col = 0;
+  if (!packed) {
+    row = base / g.cols;
+    col = base - row * g.cols;
+  }
   float m[EPT], v[EPT];
   bool bad = false;
   float mx_m = 0.f, mx_v = 0.f;
 #pragma unroll
   for (int e = 0; e < EPT; ++e) {
-    int64_t i = base + e;
+    const int64_t i = base + (int64_t)e * 256;
     if (i < nel) {
-      const int64_t ir = g.r_index(i);
-      float r = 0.f;
-      for (int s = 0; s < splits; ++s) r += Rpart[(int64_t)s * split_stride + ir];
+      const int64_t ir = packed ? i : row * g.r_ld + col;
+      const int64_t in = packed ? i : row * g.n_ld + col;
+      float r = Rpart[ir];
+      for (int s = 1; s < splits; ++s) r += Rpart[(int64_t)s * split_stride + ir];
       bad |= !isfinite(r);
       float m_old = s_code_s[Mc[i]] * am_m;
       float v_old = s_code_u[Vc[i]] * am_v;
       m[e] = p.b1 * m_old + p.omb1 * r;
       v[e] = p.b2 * v_old + p.omb2 * (r * r);
-      store_n(Nout, g.n_index(i), adam_normalised(m[e], v[e], p));
+      store_n(Nout, in, adam_normalised(m[e], v[e], p));
       mx_m = fmaxf(mx_m, fabsf(m[e]));
       mx_v = fmaxf(mx_v, fabsf(v[e]));
     } else {
       m[e] = v[e] = 0.f;
+    }
+    if (!packed) {
+      col += 256;
+      while (col >= g.cols) { col -= g.cols; ++row; }
     }
   }
   mx_m = block_max_256(mx_m, red);
   mx_v = block_max_256(mx_v, red);
 #pragma unroll
   for (int e = 0; e < EPT; ++e) {
-    int64_t i = base + e;
+    const int64_t i = base + (int64_t)e * 256;
     if (i < nel) {
       Mc[i] = (mx_m == 0.f) ? (uint8_t)127 : (uint8_t)q8_encode(__fdiv_rn(m[e], mx_m), s_mid_s);
       Vc[i] = (mx_v == 0.f) ? (uint8_t)0 : (uint8_t)q8_encode(__fdiv_rn(v[e], mx_v), s_mid_u);
@@ -207,12 +220,12 @@ q8_quantize_kernel(const float* __restrict__ x, int64_t nel, int is_signed, uint
   __syncthreads();
   constexpr int QB = EPT * 256;
   const int64_t blk = blockIdx.x;
-  const int64_t base = blk * QB + (int64_t)threadIdx.x * EPT;
+  const int64_t base = blk * QB + threadIdx.x;
   float val[EPT];
   float mx = 0.f;
 #pragma unroll
   for (int e = 0; e < EPT; ++e) {
-    int64_t i = base + e;
+    int64_t i = base + (int64_t)e * 256;
     val[e] = (i < nel) ? x[i] : 0.f;
     mx = fmaxf(mx, fabsf(val[e]));
   }
@@ -220,7 +233,7 @@ q8_quantize_kernel(const float* __restrict__ x, int64_t nel, int is_signed, uint
   const uint8_t zero_code = is_signed ? 127 : 0;
 #pragma unroll
   for (int e = 0; e < EPT; ++e) {
-    int64_t i = base + e;
+    int64_t i = base + (int64_t)e * 256;
     if (i < nel) codes[i] = (mx == 0.f) ? zero_code : (uint8_t)q8_encode(__fdiv_rn(val[e], mx), s_mid);
   }
   if (threadIdx.x == 0) absmax[blk] = mx;
