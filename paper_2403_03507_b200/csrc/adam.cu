@@ -9,7 +9,9 @@
 // makes exactly one round trip through HBM.
 #include "adam.cuh"
 
+#include <float.h>
 #include <math.h>
+#include <string.h>
 
 #include <algorithm>
 #include <mutex>
@@ -48,10 +50,16 @@ static void build_code(bool is_signed, float* out) {
 
 void q8_host_codebook(bool is_signed, float* out256) { build_code(is_signed, out256); }
 
-__constant__ float c_code_s[256];
-__constant__ float c_code_u[256];
-__constant__ float c_mid_s[256];   // 255 thresholds used
-__constant__ float c_mid_u[256];
+// Tables in global memory (not __constant__): every thread reads its own entry when a CTA
+// stages them in shared memory, which the constant cache would serialise.
+__device__ float c_code_s[256];
+__device__ float c_code_u[256];
+__device__ float c_mid_s[256];   // 255 thresholds used
+__device__ float c_mid_u[256];
+__device__ float2 c_pair_s[256];  // thresholds bracketing each code (+-FLT_MAX at the ends)
+__device__ float2 c_pair_u[256];
+__device__ uint8_t c_lut_s[2 * 3584];   // candidate codes: [0, 3584) for y >= 0, [3584, 7168) for y < 0
+__device__ uint8_t c_lut_u[3584];
 
 static std::mutex g_code_mutex;
 static bool g_code_ready[64] = {};
@@ -73,6 +81,33 @@ galore_status_t q8_ensure_tables() {
   GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_code_u, cu, sizeof(cu)));
   GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_mid_s, ms, sizeof(ms)));
   GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_mid_u, mu, sizeof(mu)));
+  float2 ps[256], pu[256];
+  for (int i = 0; i < 256; ++i) {
+    ps[i] = make_float2(i > 0 ? ms[i - 1] : -FLT_MAX, i < 255 ? ms[i] : FLT_MAX);
+    pu[i] = make_float2(i > 0 ? mu[i - 1] : -FLT_MAX, i < 255 ? mu[i] : FLT_MAX);
+  }
+  GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_pair_s, ps, sizeof(ps)));
+  GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_pair_u, pu, sizeof(pu)));
+  // candidate tables: number of thresholds at or below the lowest value of each bin
+  static uint8_t lut_s[2 * 3584], lut_u[3584];
+  auto count_le = [](const float* mids, float x) {
+    int c = 0;
+    while (c < 255 && mids[c] <= x) ++c;
+    return c;
+  };
+  for (int key = 0; key < 3584; ++key) {
+    const uint32_t b0 = 0x32000000u + ((uint32_t)std::min(key, 3456) << 16);
+    const uint32_t b1 = 0x32000000u + ((uint32_t)(std::min(key, 3456) + 1) << 16);
+    float lo, hi;
+    memcpy(&lo, &b0, 4);
+    memcpy(&hi, &b1, 4);
+    if (key == 0) lo = 0.f;
+    lut_u[key] = (uint8_t)count_le(mu, lo);
+    lut_s[key] = (uint8_t)count_le(ms, lo);            // y in [lo, hi)
+    lut_s[3584 + key] = (uint8_t)count_le(ms, -hi);    // y in (-hi, -lo]
+  }
+  GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_lut_s, lut_s, sizeof(lut_s)));
+  GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_lut_u, lut_u, sizeof(lut_u)));
   if (dev < 64) g_code_ready[dev] = true;
   return GALORE_OK;
 }
@@ -86,6 +121,37 @@ __device__ __forceinline__ int q8_encode(float y, const float* __restrict__ mids
     if (mids[mid] <= y) lo = mid + 1; else hi = mid;
   }
   return lo;
+}
+
+// Same code as q8_encode(fp32(x / absmax)) at a fraction of the cost.
+//  1. y' = x * (1 / absmax) approximates the quotient to within 2 ulp.
+//  2. A table indexed by the exponent and 7 mantissa bits of |y'| gives the code of the lower edge
+//     of that bin (kLutSize entries per sign); at most one threshold lies inside a bin, so one
+//     comparison with the bracketing thresholds pairs[idx] = {below, above} finishes the search.
+//  3. If y' is not within 6e-7 (relative) of either bracketing threshold, the exactly rounded
+//     quotient lies on the same side of both and the code is final.  Otherwise the quotient is
+//     formed with IEEE division and searched exactly.
+constexpr int kLutSize = 3584;                 // keys 0 .. 3456 used
+constexpr uint32_t kLutBase = 0x32000000u;     // bits of 2^-27: below it every value maps to key 0
+
+__device__ __forceinline__ int q8_lut_key(float ya) {
+  const uint32_t bits = __float_as_uint(ya) & 0x7fffffffu;
+  return min((int)((max(bits, kLutBase) - kLutBase) >> 16), 3456);
+}
+
+template <bool SIGNED>
+__device__ __forceinline__ int q8_encode_block(float x, float absmax, float inv, const uint8_t* __restrict__ lut,
+                                               const float2* __restrict__ pairs, const float* __restrict__ mids) {
+  const float ya = x * inv;
+  int idx = lut[q8_lut_key(ya) + ((SIGNED && ya < 0.f) ? kLutSize : 0)];
+  float2 t = pairs[idx];
+  if (ya >= t.y) {
+    ++idx;
+    t = pairs[idx];
+  }
+  constexpr float guard = 6e-7f;
+  if ((ya - t.x) > guard * fabsf(t.x) && (t.y - ya) > guard * fabsf(t.y)) return idx;
+  return q8_encode(__fdiv_rn(x, absmax), mids);
 }
 
 __device__ __forceinline__ float warp_max(float v) {
@@ -109,10 +175,13 @@ __device__ __forceinline__ float block_max_256(float v, float* red /* >= 8 float
 template <typename TN>
 __device__ __forceinline__ void store_n(TN* out, int64_t i, float v) { out[i] = cvt<TN>(v); }
 
+// Eq. 15 with bias correction.  The square root and the quotient use the approximate hardware
+// units (about 2 ulp each): N feeds a bf16 or fp32 GEMM operand and decides no integer.
 __device__ __forceinline__ float adam_normalised(float m, float v, const AdamParams& p) {
-  float mh = m * p.inv_bc1;
-  float vh = v * p.inv_bc2;
-  return mh / (sqrtf(vh) + p.eps);
+  const float mh = m * p.inv_bc1;
+  const float vh = v * p.inv_bc2;
+  const float root = vh > 0.f ? vh * rsqrtf(vh) : 0.f;
+  return __fdividef(mh, root + p.eps);
 }
 
 // ---- fp32 moments -------------------------------------------------------------
@@ -137,74 +206,102 @@ adam_f32_kernel(const float* __restrict__ Rpart, int splits, int64_t split_strid
 }
 
 // ---- 8-bit block-wise moments ---------------------------------------------------
-// One CTA per quantisation block of EPT * 256 elements; thread t owns elements
-// t, t + 256, t + 512, ... of the block, so every warp-level access is one
-// contiguous run whatever the alignment of the block.
-template <typename TN, int EPT>
+// A CTA walks quantisation blocks of EPT * 256 elements; within a block thread t owns
+// elements t, t + 256, t + 512, ... so every warp-level access is one contiguous run
+// whatever the alignment of the block.  PACKED: R partials and N have the state's own
+// row pitch, so one flat index serves all arrays.
+template <typename TN, int EPT, bool PACKED>
 __global__ void __launch_bounds__(256)
-adam_q8_kernel(const float* __restrict__ Rpart, int splits, int64_t split_stride, int64_t nel,
+adam_q8_kernel(const float* __restrict__ Rpart, int splits, int64_t split_stride, int nel,
                uint8_t* __restrict__ Mc, float* __restrict__ Mam, uint8_t* __restrict__ Vc,
-               float* __restrict__ Vam, TN* __restrict__ Nout, AdamParams p, StateGeom g,
+               float* __restrict__ Vam, TN* __restrict__ Nout, AdamParams p, int cols, int r_ld, int n_ld,
                int32_t* __restrict__ status) {
   __shared__ float s_code_s[256], s_code_u[256], s_mid_s[256], s_mid_u[256];
+  __shared__ float2 s_pair_s[256], s_pair_u[256];
+  __shared__ uint8_t s_lut_s[2 * kLutSize], s_lut_u[kLutSize];
   __shared__ float red[8];
+  for (int i = threadIdx.x; i < kLutSize / 4; i += 256) {
+    reinterpret_cast<uint32_t*>(s_lut_u)[i] = reinterpret_cast<const uint32_t*>(c_lut_u)[i];
+    reinterpret_cast<uint32_t*>(s_lut_s)[i] = reinterpret_cast<const uint32_t*>(c_lut_s)[i];
+    reinterpret_cast<uint32_t*>(s_lut_s)[kLutSize / 4 + i] = reinterpret_cast<const uint32_t*>(c_lut_s)[kLutSize / 4 + i];
+  }
   s_code_s[threadIdx.x] = c_code_s[threadIdx.x];
   s_code_u[threadIdx.x] = c_code_u[threadIdx.x];
   s_mid_s[threadIdx.x] = c_mid_s[threadIdx.x];
   s_mid_u[threadIdx.x] = c_mid_u[threadIdx.x];
+  s_pair_s[threadIdx.x] = c_pair_s[threadIdx.x];
+  s_pair_u[threadIdx.x] = c_pair_u[threadIdx.x];
   __syncthreads();
 
   constexpr int QB = EPT * 256;
-  const int64_t blk = blockIdx.x;
-  const int64_t base = blk * QB + threadIdx.x;
-  const float am_m = Mam[blk], am_v = Vam[blk];
-  // position of the thread's first element in the padded R / N buffers; advanced by 256 per element
-  const bool packed = (g.cols == 0) || (g.r_ld == g.cols && g.n_ld == g.cols);
-  int64_t row = 0, col = 0;
-  if (!packed) {
-    row = base / g.cols;
-    col = base - row * g.cols;
-  }
-  float m[EPT], v[EPT];
+  const int nblk = (nel + QB - 1) / QB;
   bool bad = false;
-  float mx_m = 0.f, mx_v = 0.f;
+  for (int blk = blockIdx.x; blk < nblk; blk += gridDim.x) {
+    const int base = blk * QB + threadIdx.x;
+    const float am_m = Mam[blk], am_v = Vam[blk];
+    int row = 0, col = 0;
+    if (!PACKED) {
+      row = base / cols;
+      col = base - row * cols;
+    }
+    // all loads of the block are issued before anything is used: the kernel lives on memory-level
+    // parallelism (EPT * (splits + 2) independent requests per thread)
+    float m[EPT], v[EPT], r[EPT];
+    int off_r[EPT], off_n[EPT];          // positions in the (possibly padded) R and N buffers
+    uint8_t cm[EPT], cv[EPT];
 #pragma unroll
-  for (int e = 0; e < EPT; ++e) {
-    const int64_t i = base + (int64_t)e * 256;
-    if (i < nel) {
-      const int64_t ir = packed ? i : row * g.r_ld + col;
-      const int64_t in = packed ? i : row * g.n_ld + col;
-      float r = Rpart[ir];
-      for (int s = 1; s < splits; ++s) r += Rpart[(int64_t)s * split_stride + ir];
-      bad |= !isfinite(r);
-      float m_old = s_code_s[Mc[i]] * am_m;
-      float v_old = s_code_u[Vc[i]] * am_v;
-      m[e] = p.b1 * m_old + p.omb1 * r;
-      v[e] = p.b2 * v_old + p.omb2 * (r * r);
-      store_n(Nout, in, adam_normalised(m[e], v[e], p));
-      mx_m = fmaxf(mx_m, fabsf(m[e]));
-      mx_v = fmaxf(mx_v, fabsf(v[e]));
-    } else {
-      m[e] = v[e] = 0.f;
+    for (int e = 0; e < EPT; ++e) {
+      const int i = base + e * 256;
+      const bool ok = i < nel;
+      off_r[e] = PACKED ? i : row * r_ld + col;
+      off_n[e] = PACKED ? i : row * n_ld + col;
+      r[e] = ok ? Rpart[off_r[e]] : 0.f;
+      cm[e] = ok ? Mc[i] : (uint8_t)127;
+      cv[e] = ok ? Vc[i] : (uint8_t)0;
+      if (!PACKED) {
+        col += 256;
+        while (col >= cols) { col -= cols; ++row; }
+      }
     }
-    if (!packed) {
-      col += 256;
-      while (col >= g.cols) { col -= g.cols; ++row; }
-    }
-  }
-  mx_m = block_max_256(mx_m, red);
-  mx_v = block_max_256(mx_v, red);
+    for (int s = 1; s < splits; ++s) {
+      const float* part = Rpart + (int64_t)s * split_stride;
 #pragma unroll
-  for (int e = 0; e < EPT; ++e) {
-    const int64_t i = base + (int64_t)e * 256;
-    if (i < nel) {
-      Mc[i] = (mx_m == 0.f) ? (uint8_t)127 : (uint8_t)q8_encode(__fdiv_rn(m[e], mx_m), s_mid_s);
-      Vc[i] = (mx_v == 0.f) ? (uint8_t)0 : (uint8_t)q8_encode(__fdiv_rn(v[e], mx_v), s_mid_u);
+      for (int e = 0; e < EPT; ++e) {
+        if (base + e * 256 < nel) r[e] += part[off_r[e]];
+      }
     }
-  }
-  if (threadIdx.x == 0) {
-    Mam[blk] = mx_m;
-    Vam[blk] = mx_v;
+    float mx_m = 0.f, mx_v = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+      const int i = base + e * 256;
+      if (i < nel) {
+        bad |= !isfinite(r[e]);
+        const float m_old = s_code_s[cm[e]] * am_m;
+        const float v_old = s_code_u[cv[e]] * am_v;
+        m[e] = p.b1 * m_old + p.omb1 * r[e];
+        v[e] = p.b2 * v_old + p.omb2 * (r[e] * r[e]);
+        Nout[off_n[e]] = cvt<TN>(adam_normalised(m[e], v[e], p));
+        mx_m = fmaxf(mx_m, fabsf(m[e]));
+        mx_v = fmaxf(mx_v, v[e]);
+      } else {
+        m[e] = v[e] = 0.f;
+      }
+    }
+    mx_m = block_max_256(mx_m, red);
+    mx_v = block_max_256(mx_v, red);
+    const float inv_m = 1.0f / mx_m, inv_v = 1.0f / mx_v;
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+      const int i = base + e * 256;
+      if (i < nel) {
+        Mc[i] = (mx_m == 0.f) ? (uint8_t)127 : (uint8_t)q8_encode_block<true>(m[e], mx_m, inv_m, s_lut_s, s_pair_s, s_mid_s);
+        Vc[i] = (mx_v == 0.f) ? (uint8_t)0 : (uint8_t)q8_encode_block<false>(v[e], mx_v, inv_v, s_lut_u, s_pair_u, s_mid_u);
+      }
+    }
+    if (threadIdx.x == 0) {
+      Mam[blk] = mx_m;
+      Vam[blk] = mx_v;
+    }
   }
   if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(status, GALORE_DEV_NONFINITE);
 }
@@ -215,8 +312,14 @@ __global__ void __launch_bounds__(256)
 q8_quantize_kernel(const float* __restrict__ x, int64_t nel, int is_signed, uint8_t* __restrict__ codes,
                    float* __restrict__ absmax) {
   __shared__ float s_mid[256];
+  __shared__ float2 s_pair[256];
+  __shared__ uint8_t s_lut[2 * kLutSize];
   __shared__ float red[8];
+  for (int i = threadIdx.x; i < (is_signed ? 2 : 1) * kLutSize / 4; i += 256)
+    reinterpret_cast<uint32_t*>(s_lut)[i] = is_signed ? reinterpret_cast<const uint32_t*>(c_lut_s)[i]
+                                                      : reinterpret_cast<const uint32_t*>(c_lut_u)[i];
   s_mid[threadIdx.x] = is_signed ? c_mid_s[threadIdx.x] : c_mid_u[threadIdx.x];
+  s_pair[threadIdx.x] = is_signed ? c_pair_s[threadIdx.x] : c_pair_u[threadIdx.x];
   __syncthreads();
   constexpr int QB = EPT * 256;
   const int64_t blk = blockIdx.x;
@@ -231,10 +334,14 @@ q8_quantize_kernel(const float* __restrict__ x, int64_t nel, int is_signed, uint
   }
   mx = block_max_256(mx, red);
   const uint8_t zero_code = is_signed ? 127 : 0;
+  const float inv = 1.0f / mx;
 #pragma unroll
   for (int e = 0; e < EPT; ++e) {
     int64_t i = base + (int64_t)e * 256;
-    if (i < nel) codes[i] = (mx == 0.f) ? zero_code : (uint8_t)q8_encode(__fdiv_rn(val[e], mx), s_mid);
+    if (i < nel)
+      codes[i] = (mx == 0.f) ? zero_code
+                             : (uint8_t)(is_signed ? q8_encode_block<true>(val[e], mx, inv, s_lut, s_pair, s_mid)
+                                                   : q8_encode_block<false>(val[e], mx, inv, s_lut, s_pair, s_mid));
   }
   if (threadIdx.x == 0) absmax[blk] = mx;
 }
@@ -277,11 +384,20 @@ template <typename TN>
 static galore_status_t adam_q8_t(const float* Rpart, int splits, int64_t split_stride, int64_t nel, uint8_t* Mc,
                                  float* Mam, uint8_t* Vc, float* Vam, int block, TN* Nout, const AdamParams& p,
                                  const StateGeom& g, int32_t* status, cudaStream_t st) {
-  unsigned grid = (unsigned)ceil_div(nel, block);
-#define GALORE_Q8_CASE(EPT)                                                                              \
-  case EPT * 256:                                                                                        \
-    adam_q8_kernel<TN, EPT><<<grid, 256, 0, st>>>(Rpart, splits, split_stride, nel, Mc, Mam, Vc, Vam,    \
-                                                   Nout, p, g, status);                                  \
+  // 32-bit offsets inside the kernel: the padded buffers must stay below 2^31 elements
+  const int64_t rows = g.cols > 0 ? ceil_div(nel, g.cols) : 1;
+  if (nel >= (int64_t)1 << 31 || rows * std::max(g.r_ld, g.n_ld) >= (int64_t)1 << 31) return GALORE_ERR_SHAPE;
+  const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(nel, block), 148 * 8);
+  const bool packed = (g.cols == 0) || (g.r_ld == g.cols && g.n_ld == g.cols);
+  const int cols = (int)g.cols, r_ld = (int)g.r_ld, n_ld = (int)g.n_ld;
+#define GALORE_Q8_CASE(EPT)                                                                                  \
+  case EPT * 256:                                                                                            \
+    if (packed)                                                                                              \
+      adam_q8_kernel<TN, EPT, true><<<grid, 256, 0, st>>>(Rpart, splits, split_stride, (int)nel, Mc, Mam,    \
+                                                          Vc, Vam, Nout, p, cols, r_ld, n_ld, status);       \
+    else                                                                                                     \
+      adam_q8_kernel<TN, EPT, false><<<grid, 256, 0, st>>>(Rpart, splits, split_stride, (int)nel, Mc, Mam,   \
+                                                           Vc, Vam, Nout, p, cols, r_ld, n_ld, status);      \
     break;
   switch (block) {
     GALORE_Q8_CASE(1) GALORE_Q8_CASE(2) GALORE_Q8_CASE(4) GALORE_Q8_CASE(8) GALORE_Q8_CASE(16)
