@@ -21,7 +21,9 @@
 #include <cudaTypedefs.h>
 
 #include <algorithm>
+#include <memory>
 #include <mutex>
+#include <new>
 
 namespace galore {
 
@@ -42,8 +44,11 @@ constexpr long long kWaitLimitCycles = 4000000000LL;   // about two seconds
 
 enum { EPI_PARTIAL = 0, EPI_APPLY = 1 };
 
+constexpr int kMaxGroup = 32;     // problems one launch can carry (its arguments travel as kernel parameters)
+
 struct TcParams {
   int M, N, K;
+  int a_mn, b_mn;             // operand majors in shared memory: 1 = M/N contiguous, 0 = K contiguous
   int tiles_m, tiles_n, splits;
   int kblocks_total, kblocks_per_split;
   int m_fast;                 // 1: consecutive units walk tile_m first (B panel shared), 0: tile_n first
@@ -55,6 +60,15 @@ struct TcParams {
   int64_t ldw;
   float scale;
   int32_t* status;
+};
+
+// One launch = up to kMaxGroup independent problems; work units are numbered across them.
+struct TcGroup {
+  CUtensorMap map_a[kMaxGroup];
+  CUtensorMap map_b[kMaxGroup];
+  TcParams p[kMaxGroup];
+  int unit_end[kMaxGroup];    // running total of units: problem i owns [unit_end[i-1], unit_end[i])
+  int count;
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------
@@ -158,7 +172,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major) {
 }
 
 // Instruction descriptor: fp32 accumulate, bf16 x bf16, majors, N, M.
-__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn) {
+__host__ __device__ constexpr uint32_t instr_desc(int a_mn, int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
          ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 }
@@ -167,7 +181,11 @@ struct Unit {
   int m0, n0, split, kb_begin, kb_end;
 };
 
-__device__ __forceinline__ Unit decode_unit(const TcParams& p, int u) {
+__device__ __forceinline__ Unit decode_unit(const TcGroup& g, int u, int& pi) {
+  pi = 0;
+  while (pi + 1 < g.count && u >= g.unit_end[pi]) ++pi;
+  if (pi > 0) u -= g.unit_end[pi - 1];
+  const TcParams& p = g.p[pi];
   int tm, tn, s;
   if (p.m_fast) {
     tm = u % p.tiles_m;
@@ -256,9 +274,9 @@ __device__ __forceinline__ void epi_apply<float>(const TcParams& p, int row, int
 
 // ---- the kernel -------------------------------------------------------------------------------
 
-template <bool A_MN, bool B_MN, int EPI, typename TW>
+template <int EPI, typename TW>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcParams p) {
+gemm_tc_kernel(const __grid_constant__ TcGroup g) {
   extern __shared__ uint8_t smem_raw[];
   // stage ring, 1024-byte aligned for the 128-byte swizzle
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -276,7 +294,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int total_units = p.tiles_m * p.tiles_n * p.splits;
+  const int total_units = g.unit_end[g.count - 1];
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -308,7 +326,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       long long issued = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
-        const Unit w = decode_unit(p, u);
+        int pi;
+        const Unit w = decode_unit(g, u, pi);
+        const bool A_MN = g.p[pi].a_mn != 0, B_MN = g.p[pi].b_mn != 0;
+        const CUtensorMap* map_a = &g.map_a[pi];
+        const CUtensorMap* map_b = &g.map_b[pi];
         for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t a_dst = ring + stage * kStageBytes;
@@ -317,15 +339,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int k0 = kb * kBK;
           if (A_MN) {
 #pragma unroll
-            for (int j = 0; j < kBM / 64; ++j) tma_load_2d(a_dst + j * (kBK * 128), &map_a, w.m0 + 64 * j, k0, full_bar(stage));
+            for (int j = 0; j < kBM / 64; ++j) tma_load_2d(a_dst + j * (kBK * 128), map_a, w.m0 + 64 * j, k0, full_bar(stage));
           } else {
-            tma_load_2d(a_dst, &map_a, k0, w.m0, full_bar(stage));
+            tma_load_2d(a_dst, map_a, k0, w.m0, full_bar(stage));
           }
           if (B_MN) {
 #pragma unroll
-            for (int j = 0; j < kBN / 64; ++j) tma_load_2d(b_dst + j * (kBK * 128), &map_b, w.n0 + 64 * j, k0, full_bar(stage));
+            for (int j = 0; j < kBN / 64; ++j) tma_load_2d(b_dst + j * (kBK * 128), map_b, w.n0 + 64 * j, k0, full_bar(stage));
           } else {
-            tma_load_2d(b_dst, &map_b, k0, w.n0, full_bar(stage));
+            tma_load_2d(b_dst, map_b, k0, w.n0, full_bar(stage));
           }
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -346,14 +368,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else if (warp == 1) {
     // ================= MMA issuer =================
     if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc(A_MN, B_MN);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
-        const Unit w = decode_unit(p, u);
+        int pi;
+        const Unit w = decode_unit(g, u, pi);
+        const bool A_MN = g.p[pi].a_mn != 0, B_MN = g.p[pi].b_mn != 0;
+        const uint32_t idesc = instr_desc(g.p[pi].a_mn, g.p[pi].b_mn);
         if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kBN);
@@ -385,7 +409,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
-      const Unit w = decode_unit(p, u);
+      int pi;
+      const Unit w = decode_unit(g, u, pi);
+      const TcParams& p = g.p[pi];
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int row = w.m0 + quarter * 32 + lane;
@@ -408,7 +434,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, GALORE_DEV_WAIT_EXPIRED);
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(g.p[0].status, GALORE_DEV_WAIT_EXPIRED);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
@@ -459,19 +485,30 @@ int sm_count() {
   return sms;
 }
 
-template <bool A_MN, bool B_MN, int EPI, typename TW>
-galore_status_t launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, cudaStream_t st) {
-  auto kern = gemm_tc_kernel<A_MN, B_MN, EPI, TW>;
+template <int EPI, typename TW>
+galore_status_t launch_tc(const TcGroup& g, cudaStream_t st) {
+  auto kern = gemm_tc_kernel<EPI, TW>;
   static bool configured = false;
   if (!configured) {
     GALORE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     configured = true;
   }
-  const int units = p.tiles_m * p.tiles_n * p.splits;
+  if (g.count < 1 || g.count > kMaxGroup) return GALORE_ERR_INVALID_ARG;
+  const int units = g.unit_end[g.count - 1];
+  if (units <= 0) return GALORE_OK;
   const int grid = std::min(units, sm_count());
-  kern<<<grid, kThreads, kSmemBytes, st>>>(ma, mb, p);
+  kern<<<grid, kThreads, kSmemBytes, st>>>(g);
   GALORE_LAUNCH_CHECK();
   return GALORE_OK;
+}
+
+// appends one problem to a group
+void group_add(TcGroup& g, const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p) {
+  const int i = g.count++;
+  g.map_a[i] = ma;
+  g.map_b[i] = mb;
+  g.p[i] = p;
+  g.unit_end[i] = (i > 0 ? g.unit_end[i - 1] : 0) + p.tiles_m * p.tiles_n * p.splits;
 }
 
 void fill_tiles(TcParams& p, int M, int N, int K, int splits) {
@@ -549,50 +586,137 @@ bool tensor_operands_aligned(const galore_config_t& c, const void* W, int64_t ld
   return c.w_dtype == GALORE_BF16 ? (ldw % 8) == 0 : (ldw % 4) == 0;
 }
 
-galore_status_t tensor_project(TensorPlan* plan, const galore_config_t& c, bool left, const void* G, int64_t ldg,
-                               int32_t* status, cudaStream_t st) {
+// ---- problems -----------------------------------------------------------------------------------
+
+// R partials <- P^T G (left) / G Q (right)
+static galore_status_t project_problem(const TensorPlan* plan, const galore_config_t& c, bool left, const void* G,
+                                       int64_t ldg, float* part, int64_t ld_part, int splits, int32_t* status,
+                                       TcParams* p, CUtensorMap* ma, CUtensorMap* mb) {
   if (!plan->ready) return GALORE_ERR_STATE;
   const int r = c.rank;
-  TcParams p = {};
-  p.status = status;
-  p.part = plan->Rpart;
-  p.ld_part = plan->ld_part;
-  CUtensorMap map_g;
+  *p = TcParams{};
+  p->status = status;
+  p->part = part;
+  p->ld_part = ld_part;
   if (left) {
-    // R (r x n) = P^T G : A MN-major (P), B MN-major (G); G is the big operand, shared along tile_m
-    fill_tiles(p, r, (int)c.n, (int)c.m, plan->splits);
-    p.split_stride = (int64_t)r * plan->ld_part;
-    p.m_fast = 1;
-    GALORE_TRY(make_map(&map_g, G, c.m, c.n, ldg, 64));
-    return launch_tc<true, true, EPI_PARTIAL, float>(plan->map_p_proj, map_g, p, st);
+    // A = P^T, M/N-major from P; B = G, M/N-major.  G is the big operand: units sharing a G panel run together
+    fill_tiles(*p, r, (int)c.n, (int)c.m, splits);
+    p->split_stride = (int64_t)r * ld_part;
+    p->m_fast = 1;
+    p->a_mn = 1;
+    p->b_mn = 1;
+    *ma = plan->map_p_proj;
+    return make_map(mb, G, c.m, c.n, ldg, 64);
   }
-  // R (m x r) = G Q : A K-major (G), B MN-major (Q); G is the big operand, shared along tile_n
-  fill_tiles(p, (int)c.m, r, (int)c.n, plan->splits);
-  p.split_stride = (int64_t)c.m * plan->ld_part;
-  p.m_fast = 0;
-  GALORE_TRY(make_map(&map_g, G, c.m, c.n, ldg, kBM));
-  return launch_tc<false, true, EPI_PARTIAL, float>(map_g, plan->map_p_proj, p, st);
+  // A = G, K-major; B = Q, M/N-major
+  fill_tiles(*p, (int)c.m, r, (int)c.n, splits);
+  p->split_stride = (int64_t)c.m * ld_part;
+  p->m_fast = 0;
+  p->a_mn = 0;
+  p->b_mn = 1;
+  *mb = plan->map_p_proj;
+  return make_map(ma, G, c.m, c.n, ldg, kBM);
+}
+
+// W <- W - scale * P N (left) / N Q^T (right); map_n addresses the normalised update
+static galore_status_t back_problem(const TensorPlan* plan, const galore_config_t& c, bool left, const CUtensorMap& map_n,
+                                    void* W, int64_t ldw, float scale, int32_t* status, TcParams* p, CUtensorMap* ma,
+                                    CUtensorMap* mb) {
+  if (!plan->ready) return GALORE_ERR_STATE;
+  *p = TcParams{};
+  p->status = status;
+  p->W = W;
+  p->ldw = ldw;
+  p->scale = scale;
+  p->m_fast = 1;
+  fill_tiles(*p, (int)c.m, (int)c.n, c.rank, 1);
+  if (left) {   // A = P K-major, B = N M/N-major
+    p->a_mn = 0;
+    p->b_mn = 1;
+    *ma = plan->map_p_back;
+    *mb = map_n;
+  } else {      // A = N K-major, B = Q^T K-major from Q
+    p->a_mn = 0;
+    p->b_mn = 0;
+    *ma = map_n;
+    *mb = plan->map_p_back;
+  }
+  return GALORE_OK;
+}
+
+galore_status_t tensor_project(TensorPlan* plan, const galore_config_t& c, bool left, const void* G, int64_t ldg,
+                               int32_t* status, cudaStream_t st) {
+  TcParams p;
+  CUtensorMap ma, mb;
+  GALORE_TRY(project_problem(plan, c, left, G, ldg, plan->Rpart, plan->ld_part, plan->splits, status, &p, &ma, &mb));
+  std::unique_ptr<TcGroup> g(new TcGroup);
+  g->count = 0;
+  group_add(*g, ma, mb, p);
+  return launch_tc<EPI_PARTIAL, float>(*g, st);
 }
 
 galore_status_t tensor_back_project(TensorPlan* plan, const galore_config_t& c, bool left, void* W, int64_t ldw,
                                     float scale, int32_t* status, cudaStream_t st) {
-  if (!plan->ready) return GALORE_ERR_STATE;
-  TcParams p = {};
-  p.status = status;
-  p.W = W;
-  p.ldw = ldw;
-  p.scale = scale;
-  p.m_fast = 1;
-  fill_tiles(p, (int)c.m, (int)c.n, c.rank, 1);
-  const bool wb = c.w_dtype == GALORE_BF16;
-  if (left) {
-    // W -= scale * P N : A K-major (P), B MN-major (N)
-    if (wb) return launch_tc<false, true, EPI_APPLY, __nv_bfloat16>(plan->map_p_back, plan->map_n_back, p, st);
-    return launch_tc<false, true, EPI_APPLY, float>(plan->map_p_back, plan->map_n_back, p, st);
-  }
-  // W -= scale * N Q^T : A K-major (N), B K-major (Q)
-  if (wb) return launch_tc<false, false, EPI_APPLY, __nv_bfloat16>(plan->map_n_back, plan->map_p_back, p, st);
-  return launch_tc<false, false, EPI_APPLY, float>(plan->map_n_back, plan->map_p_back, p, st);
+  TcParams p;
+  CUtensorMap ma, mb;
+  GALORE_TRY(back_problem(plan, c, left, plan->map_n_back, W, ldw, scale, status, &p, &ma, &mb));
+  std::unique_ptr<TcGroup> g(new TcGroup);
+  g->count = 0;
+  group_add(*g, ma, mb, p);
+  if (c.w_dtype == GALORE_BF16) return launch_tc<EPI_APPLY, __nv_bfloat16>(*g, st);
+  return launch_tc<EPI_APPLY, float>(*g, st);
+}
+
+// ---- groups: many layers per launch ------------------------------------------------------------------
+
+struct TensorGroup {
+  TcGroup g;
+};
+
+TensorGroup* tensor_group_new() {
+  TensorGroup* t = new (std::nothrow) TensorGroup;
+  if (t) t->g.count = 0;
+  return t;
+}
+void tensor_group_free(TensorGroup* t) { delete t; }
+void tensor_group_reset(TensorGroup* t) { t->g.count = 0; }
+int tensor_group_count(const TensorGroup* t) { return t->g.count; }
+int tensor_group_capacity() { return kMaxGroup; }
+
+galore_status_t tensor_group_add_project(TensorGroup* t, const TensorPlan* plan, const galore_config_t& c, bool left,
+                                         const void* G, int64_t ldg, float* part, int64_t ld_part, int splits,
+                                         int32_t* status) {
+  if (t->g.count >= kMaxGroup) return GALORE_ERR_BUFFER_TOO_SMALL;
+  TcParams p;
+  CUtensorMap ma, mb;
+  GALORE_TRY(project_problem(plan, c, left, G, ldg, part, ld_part, splits, status, &p, &ma, &mb));
+  group_add(t->g, ma, mb, p);
+  return GALORE_OK;
+}
+
+galore_status_t tensor_group_add_back(TensorGroup* t, const TensorPlan* plan, const galore_config_t& c, bool left,
+                                      const void* Nbuf, int64_t ld_n, void* W, int64_t ldw, float scale,
+                                      int32_t* status) {
+  if (t->g.count >= kMaxGroup) return GALORE_ERR_BUFFER_TOO_SMALL;
+  CUtensorMap map_n;
+  if (left) GALORE_TRY(make_map(&map_n, Nbuf, c.rank, c.n, ld_n, 64));
+  else GALORE_TRY(make_map(&map_n, Nbuf, c.m, c.rank, ld_n, kBM));
+  TcParams p;
+  CUtensorMap ma, mb;
+  GALORE_TRY(back_problem(plan, c, left, map_n, W, ldw, scale, status, &p, &ma, &mb));
+  group_add(t->g, ma, mb, p);
+  return GALORE_OK;
+}
+
+galore_status_t tensor_group_launch_project(TensorGroup* t, cudaStream_t st) {
+  if (t->g.count == 0) return GALORE_OK;
+  return launch_tc<EPI_PARTIAL, float>(t->g, st);
+}
+
+galore_status_t tensor_group_launch_back(TensorGroup* t, int32_t w_dtype, cudaStream_t st) {
+  if (t->g.count == 0) return GALORE_OK;
+  if (w_dtype == GALORE_BF16) return launch_tc<EPI_APPLY, __nv_bfloat16>(t->g, st);
+  return launch_tc<EPI_APPLY, float>(t->g, st);
 }
 
 }  // namespace galore

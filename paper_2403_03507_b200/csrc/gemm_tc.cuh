@@ -35,4 +35,23 @@ galore_status_t tensor_project(TensorPlan* plan, const galore_config_t& cfg, boo
 galore_status_t tensor_back_project(TensorPlan* plan, const galore_config_t& cfg, bool left, void* W, int64_t ldw,
                                     float scale, int32_t* status, cudaStream_t st);
 
+
+// ---- groups: up to tensor_group_capacity() layers per launch ------------------------------------
+struct TensorGroup;   // opaque, host memory
+TensorGroup* tensor_group_new();
+void tensor_group_free(TensorGroup* t);
+void tensor_group_reset(TensorGroup* t);
+int tensor_group_count(const TensorGroup* t);
+int tensor_group_capacity();
+// the layer's projection with its R partials going to `part` (leading dimension ld_part, `splits` K slices)
+galore_status_t tensor_group_add_project(TensorGroup* t, const TensorPlan* plan, const galore_config_t& cfg, bool left,
+                                         const void* G, int64_t ldg, float* part, int64_t ld_part, int splits,
+                                         int32_t* status);
+// the layer's back-projection reading its normalised update from Nbuf (bf16, leading dimension ld_n)
+galore_status_t tensor_group_add_back(TensorGroup* t, const TensorPlan* plan, const galore_config_t& cfg, bool left,
+                                      const void* Nbuf, int64_t ld_n, void* W, int64_t ldw, float scale,
+                                      int32_t* status);
+galore_status_t tensor_group_launch_project(TensorGroup* t, cudaStream_t st);
+galore_status_t tensor_group_launch_back(TensorGroup* t, int32_t w_dtype, cudaStream_t st);
+
 }  // namespace galore
