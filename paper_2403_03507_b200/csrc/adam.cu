@@ -14,6 +14,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <memory>
 #include <mutex>
 #include <vector>
 
@@ -172,9 +173,6 @@ __device__ __forceinline__ float block_max_256(float v, float* red /* >= 8 float
   return r;
 }
 
-template <typename TN>
-__device__ __forceinline__ void store_n(TN* out, int64_t i, float v) { out[i] = cvt<TN>(v); }
-
 // Eq. 15 with bias correction.  The square root and the quotient use the approximate hardware
 // units (about 2 ulp each): N feeds a bf16 or fp32 GEMM operand and decides no integer.
 __device__ __forceinline__ float adam_normalised(float m, float v, const AdamParams& p) {
@@ -184,25 +182,83 @@ __device__ __forceinline__ float adam_normalised(float m, float v, const AdamPar
   return __fdividef(mh, root + p.eps);
 }
 
+// ---- grouped launches ------------------------------------------------------------
+// Both kernels take a group of layers (AdamGroup, passed as kernel parameters) and walk the
+// blocks of all of them with one persistent grid; a single layer is a group of one.
+
+__device__ __forceinline__ int find_item(const AdamGroup& g, int gb, int& local) {
+  int it = 0;
+  while (it + 1 < g.count && gb >= g.block_end[it]) ++it;
+  local = gb - (it > 0 ? g.block_end[it - 1] : 0);
+  return it;
+}
+
 // ---- fp32 moments -------------------------------------------------------------
-template <typename TN>
-__global__ void __launch_bounds__(256)
-adam_f32_kernel(const float* __restrict__ Rpart, int splits, int64_t split_stride, int64_t nel,
-                float* __restrict__ M, float* __restrict__ V, TN* __restrict__ Nout, AdamParams p,
-                StateGeom g, int32_t* __restrict__ status) {
-  bool bad = false;
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nel; i += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t ir = g.r_index(i), in = g.n_index(i);
-    float r = 0.f;
-    for (int s = 0; s < splits; ++s) r += Rpart[(int64_t)s * split_stride + ir];
-    bad |= !isfinite(r);
-    float m = p.b1 * M[i] + p.omb1 * r;
-    float v = p.b2 * V[i] + p.omb2 * (r * r);
-    M[i] = m;
-    V[i] = v;
-    store_n(Nout, in, adam_normalised(m, v, p));
+// work block = 2048 consecutive state elements, thread t owns t, t + 256, ...
+template <typename TN, bool PACKED>
+__device__ __forceinline__ bool adam_f32_block(const AdamItem& a, int blk) {
+  constexpr int EPT = 8;
+  const int base = blk * (EPT * 256) + threadIdx.x;
+  const AdamParams p = a.p;
+  float* __restrict__ M = a.M;
+  float* __restrict__ V = a.V;
+  TN* __restrict__ Nout = (TN*)a.Nout;
+  int row = 0, col = 0;
+  if (!PACKED) {
+    row = base / a.cols;
+    col = base - row * a.cols;
   }
-  if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(status, GALORE_DEV_NONFINITE);
+  float r[EPT], m[EPT], v[EPT];
+  int off_r[EPT], off_n[EPT];
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    const int i = base + e * 256;
+    const bool ok = i < a.nel;
+    off_r[e] = PACKED ? i : row * a.r_ld + col;
+    off_n[e] = PACKED ? i : row * a.n_ld + col;
+    r[e] = ok ? a.Rpart[off_r[e]] : 0.f;
+    m[e] = ok ? M[i] : 0.f;
+    v[e] = ok ? V[i] : 0.f;
+    if (!PACKED) {
+      col += 256;
+      while (col >= a.cols) { col -= a.cols; ++row; }
+    }
+  }
+  for (int s = 1; s < a.splits; ++s) {
+    const float* part = a.Rpart + (int64_t)s * a.split_stride;
+#pragma unroll
+    for (int e = 0; e < EPT; ++e)
+      if (base + e * 256 < a.nel) r[e] += part[off_r[e]];
+  }
+  bool bad = false;
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    const int i = base + e * 256;
+    if (i < a.nel) {
+      bad |= !isfinite(r[e]);
+      const float mn = p.b1 * m[e] + p.omb1 * r[e];
+      const float vn = p.b2 * v[e] + p.omb2 * (r[e] * r[e]);
+      M[i] = mn;
+      V[i] = vn;
+      Nout[off_n[e]] = cvt<TN>(adam_normalised(mn, vn, p));
+    }
+  }
+  return bad;
+}
+
+template <typename TN>
+__global__ void __launch_bounds__(256) adam_f32_kernel(const __grid_constant__ AdamGroup g) {
+  const int total = g.block_end[g.count - 1];
+  int bad_item = -1;
+  for (int gb = blockIdx.x; gb < total; gb += gridDim.x) {
+    int blk;
+    const int it = find_item(g, gb, blk);
+    const AdamItem& a = g.item[it];
+    const bool packed = (a.r_ld == a.cols && a.n_ld == a.cols);
+    const bool bad = packed ? adam_f32_block<TN, true>(a, blk) : adam_f32_block<TN, false>(a, blk);
+    if (bad) bad_item = it;
+  }
+  if (bad_item >= 0) atomicOr(g.item[bad_item].status, GALORE_DEV_NONFINITE);
 }
 
 // ---- 8-bit block-wise moments ---------------------------------------------------
@@ -210,100 +266,116 @@ adam_f32_kernel(const float* __restrict__ Rpart, int splits, int64_t split_strid
 // elements t, t + 256, t + 512, ... so every warp-level access is one contiguous run
 // whatever the alignment of the block.  PACKED: R partials and N have the state's own
 // row pitch, so one flat index serves all arrays.
+struct Q8Tables {
+  float code_s[256], code_u[256], mid_s[256], mid_u[256];
+  float2 pair_s[256], pair_u[256];
+  uint8_t lut_s[2 * kLutSize], lut_u[kLutSize];
+  float red[8];
+};
+
 template <typename TN, int EPT, bool PACKED>
-__global__ void __launch_bounds__(256)
-adam_q8_kernel(const float* __restrict__ Rpart, int splits, int64_t split_stride, int nel,
-               uint8_t* __restrict__ Mc, float* __restrict__ Mam, uint8_t* __restrict__ Vc,
-               float* __restrict__ Vam, TN* __restrict__ Nout, AdamParams p, int cols, int r_ld, int n_ld,
-               int32_t* __restrict__ status) {
-  __shared__ float s_code_s[256], s_code_u[256], s_mid_s[256], s_mid_u[256];
-  __shared__ float2 s_pair_s[256], s_pair_u[256];
-  __shared__ uint8_t s_lut_s[2 * kLutSize], s_lut_u[kLutSize];
-  __shared__ float red[8];
-  for (int i = threadIdx.x; i < kLutSize / 4; i += 256) {
-    reinterpret_cast<uint32_t*>(s_lut_u)[i] = reinterpret_cast<const uint32_t*>(c_lut_u)[i];
-    reinterpret_cast<uint32_t*>(s_lut_s)[i] = reinterpret_cast<const uint32_t*>(c_lut_s)[i];
-    reinterpret_cast<uint32_t*>(s_lut_s)[kLutSize / 4 + i] = reinterpret_cast<const uint32_t*>(c_lut_s)[kLutSize / 4 + i];
+__device__ __forceinline__ bool adam_q8_block(const AdamItem& a, int blk, Q8Tables& t) {
+  constexpr int QB = EPT * 256;
+  const int nel = a.nel;
+  const AdamParams p = a.p;
+  uint8_t* __restrict__ Mc = a.Mc;
+  uint8_t* __restrict__ Vc = a.Vc;
+  TN* __restrict__ Nout = (TN*)a.Nout;
+  const int base = blk * QB + threadIdx.x;
+  const float am_m = a.Mam[blk], am_v = a.Vam[blk];
+  int row = 0, col = 0;
+  if (!PACKED) {
+    row = base / a.cols;
+    col = base - row * a.cols;
   }
-  s_code_s[threadIdx.x] = c_code_s[threadIdx.x];
-  s_code_u[threadIdx.x] = c_code_u[threadIdx.x];
-  s_mid_s[threadIdx.x] = c_mid_s[threadIdx.x];
-  s_mid_u[threadIdx.x] = c_mid_u[threadIdx.x];
-  s_pair_s[threadIdx.x] = c_pair_s[threadIdx.x];
-  s_pair_u[threadIdx.x] = c_pair_u[threadIdx.x];
+  // all loads of the block are issued before anything is used: the kernel lives on memory-level
+  // parallelism (EPT * (splits + 2) independent requests per thread)
+  float m[EPT], v[EPT], r[EPT];
+  int off_r[EPT], off_n[EPT];          // positions in the (possibly padded) R and N buffers
+  uint8_t cm[EPT], cv[EPT];
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    const int i = base + e * 256;
+    const bool ok = i < nel;
+    off_r[e] = PACKED ? i : row * a.r_ld + col;
+    off_n[e] = PACKED ? i : row * a.n_ld + col;
+    r[e] = ok ? a.Rpart[off_r[e]] : 0.f;
+    cm[e] = ok ? Mc[i] : (uint8_t)127;
+    cv[e] = ok ? Vc[i] : (uint8_t)0;
+    if (!PACKED) {
+      col += 256;
+      while (col >= a.cols) { col -= a.cols; ++row; }
+    }
+  }
+  for (int s = 1; s < a.splits; ++s) {
+    const float* part = a.Rpart + (int64_t)s * a.split_stride;
+#pragma unroll
+    for (int e = 0; e < EPT; ++e)
+      if (base + e * 256 < nel) r[e] += part[off_r[e]];
+  }
+  bool bad = false;
+  float mx_m = 0.f, mx_v = 0.f;
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    const int i = base + e * 256;
+    if (i < nel) {
+      bad |= !isfinite(r[e]);
+      const float m_old = t.code_s[cm[e]] * am_m;
+      const float v_old = t.code_u[cv[e]] * am_v;
+      m[e] = p.b1 * m_old + p.omb1 * r[e];
+      v[e] = p.b2 * v_old + p.omb2 * (r[e] * r[e]);
+      Nout[off_n[e]] = cvt<TN>(adam_normalised(m[e], v[e], p));
+      mx_m = fmaxf(mx_m, fabsf(m[e]));
+      mx_v = fmaxf(mx_v, v[e]);
+    } else {
+      m[e] = v[e] = 0.f;
+    }
+  }
+  mx_m = block_max_256(mx_m, t.red);
+  mx_v = block_max_256(mx_v, t.red);
+  const float inv_m = 1.0f / mx_m, inv_v = 1.0f / mx_v;
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    const int i = base + e * 256;
+    if (i < nel) {
+      Mc[i] = (mx_m == 0.f) ? (uint8_t)127 : (uint8_t)q8_encode_block<true>(m[e], mx_m, inv_m, t.lut_s, t.pair_s, t.mid_s);
+      Vc[i] = (mx_v == 0.f) ? (uint8_t)0 : (uint8_t)q8_encode_block<false>(v[e], mx_v, inv_v, t.lut_u, t.pair_u, t.mid_u);
+    }
+  }
+  if (threadIdx.x == 0) {
+    a.Mam[blk] = mx_m;
+    a.Vam[blk] = mx_v;
+  }
+  return bad;
+}
+
+template <typename TN, int EPT>
+__global__ void __launch_bounds__(256) adam_q8_kernel(const __grid_constant__ AdamGroup g) {
+  __shared__ Q8Tables t;
+  for (int i = threadIdx.x; i < kLutSize / 4; i += 256) {
+    reinterpret_cast<uint32_t*>(t.lut_u)[i] = reinterpret_cast<const uint32_t*>(c_lut_u)[i];
+    reinterpret_cast<uint32_t*>(t.lut_s)[i] = reinterpret_cast<const uint32_t*>(c_lut_s)[i];
+    reinterpret_cast<uint32_t*>(t.lut_s)[kLutSize / 4 + i] = reinterpret_cast<const uint32_t*>(c_lut_s)[kLutSize / 4 + i];
+  }
+  t.code_s[threadIdx.x] = c_code_s[threadIdx.x];
+  t.code_u[threadIdx.x] = c_code_u[threadIdx.x];
+  t.mid_s[threadIdx.x] = c_mid_s[threadIdx.x];
+  t.mid_u[threadIdx.x] = c_mid_u[threadIdx.x];
+  t.pair_s[threadIdx.x] = c_pair_s[threadIdx.x];
+  t.pair_u[threadIdx.x] = c_pair_u[threadIdx.x];
   __syncthreads();
 
-  constexpr int QB = EPT * 256;
-  const int nblk = (nel + QB - 1) / QB;
-  bool bad = false;
-  for (int blk = blockIdx.x; blk < nblk; blk += gridDim.x) {
-    const int base = blk * QB + threadIdx.x;
-    const float am_m = Mam[blk], am_v = Vam[blk];
-    int row = 0, col = 0;
-    if (!PACKED) {
-      row = base / cols;
-      col = base - row * cols;
-    }
-    // all loads of the block are issued before anything is used: the kernel lives on memory-level
-    // parallelism (EPT * (splits + 2) independent requests per thread)
-    float m[EPT], v[EPT], r[EPT];
-    int off_r[EPT], off_n[EPT];          // positions in the (possibly padded) R and N buffers
-    uint8_t cm[EPT], cv[EPT];
-#pragma unroll
-    for (int e = 0; e < EPT; ++e) {
-      const int i = base + e * 256;
-      const bool ok = i < nel;
-      off_r[e] = PACKED ? i : row * r_ld + col;
-      off_n[e] = PACKED ? i : row * n_ld + col;
-      r[e] = ok ? Rpart[off_r[e]] : 0.f;
-      cm[e] = ok ? Mc[i] : (uint8_t)127;
-      cv[e] = ok ? Vc[i] : (uint8_t)0;
-      if (!PACKED) {
-        col += 256;
-        while (col >= cols) { col -= cols; ++row; }
-      }
-    }
-    for (int s = 1; s < splits; ++s) {
-      const float* part = Rpart + (int64_t)s * split_stride;
-#pragma unroll
-      for (int e = 0; e < EPT; ++e) {
-        if (base + e * 256 < nel) r[e] += part[off_r[e]];
-      }
-    }
-    float mx_m = 0.f, mx_v = 0.f;
-#pragma unroll
-    for (int e = 0; e < EPT; ++e) {
-      const int i = base + e * 256;
-      if (i < nel) {
-        bad |= !isfinite(r[e]);
-        const float m_old = s_code_s[cm[e]] * am_m;
-        const float v_old = s_code_u[cv[e]] * am_v;
-        m[e] = p.b1 * m_old + p.omb1 * r[e];
-        v[e] = p.b2 * v_old + p.omb2 * (r[e] * r[e]);
-        Nout[off_n[e]] = cvt<TN>(adam_normalised(m[e], v[e], p));
-        mx_m = fmaxf(mx_m, fabsf(m[e]));
-        mx_v = fmaxf(mx_v, v[e]);
-      } else {
-        m[e] = v[e] = 0.f;
-      }
-    }
-    mx_m = block_max_256(mx_m, red);
-    mx_v = block_max_256(mx_v, red);
-    const float inv_m = 1.0f / mx_m, inv_v = 1.0f / mx_v;
-#pragma unroll
-    for (int e = 0; e < EPT; ++e) {
-      const int i = base + e * 256;
-      if (i < nel) {
-        Mc[i] = (mx_m == 0.f) ? (uint8_t)127 : (uint8_t)q8_encode_block<true>(m[e], mx_m, inv_m, s_lut_s, s_pair_s, s_mid_s);
-        Vc[i] = (mx_v == 0.f) ? (uint8_t)0 : (uint8_t)q8_encode_block<false>(v[e], mx_v, inv_v, s_lut_u, s_pair_u, s_mid_u);
-      }
-    }
-    if (threadIdx.x == 0) {
-      Mam[blk] = mx_m;
-      Vam[blk] = mx_v;
-    }
+  const int total = g.block_end[g.count - 1];
+  int bad_item = -1;
+  for (int gb = blockIdx.x; gb < total; gb += gridDim.x) {
+    int blk;
+    const int it = find_item(g, gb, blk);
+    const AdamItem& a = g.item[it];
+    const bool packed = (a.r_ld == a.cols && a.n_ld == a.cols);
+    const bool bad = packed ? adam_q8_block<TN, EPT, true>(a, blk, t) : adam_q8_block<TN, EPT, false>(a, blk, t);
+    if (__syncthreads_or(bad)) bad_item = it;
   }
-  if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(status, GALORE_DEV_NONFINITE);
+  if (bad_item >= 0 && threadIdx.x == 0) atomicOr(g.item[bad_item].status, GALORE_DEV_NONFINITE);
 }
 
 // ---- stand-alone quantise / dequantise (same device code as the Adam kernel) ----
@@ -361,45 +433,26 @@ static bool valid_block(int block) {
   return block == 256 || block == 512 || block == 1024 || block == 2048 || block == 4096;
 }
 
-template <typename TN>
-static galore_status_t adam_f32_t(const float* Rpart, int splits, int64_t split_stride, int64_t nel, float* M,
-                                  float* V, TN* Nout, const AdamParams& p, const StateGeom& g, int32_t* status,
-                                  cudaStream_t st) {
-  int64_t blocks = std::min<int64_t>(ceil_div(nel, 256), 148 * 16);
-  adam_f32_kernel<TN><<<(unsigned)blocks, 256, 0, st>>>(Rpart, splits, split_stride, nel, M, V, Nout, p, g, status);
-  GALORE_LAUNCH_CHECK();
-  return GALORE_OK;
-}
-
-galore_status_t launch_adam_f32(const float* Rpart, int splits, int64_t split_stride, int64_t nel, float* M,
-                                float* V, void* Nout, int32_t n_dtype, const AdamParams& p, int32_t* status,
-                                cudaStream_t st, const StateGeom& g) {
-  if (nel <= 0) return GALORE_OK;
-  if (n_dtype == GALORE_BF16)
-    return adam_f32_t(Rpart, splits, split_stride, nel, M, V, (__nv_bfloat16*)Nout, p, g, status, st);
-  return adam_f32_t(Rpart, splits, split_stride, nel, M, V, (float*)Nout, p, g, status, st);
-}
-
-template <typename TN>
-static galore_status_t adam_q8_t(const float* Rpart, int splits, int64_t split_stride, int64_t nel, uint8_t* Mc,
-                                 float* Mam, uint8_t* Vc, float* Vam, int block, TN* Nout, const AdamParams& p,
-                                 const StateGeom& g, int32_t* status, cudaStream_t st) {
-  // 32-bit offsets inside the kernel: the padded buffers must stay below 2^31 elements
-  const int64_t rows = g.cols > 0 ? ceil_div(nel, g.cols) : 1;
-  if (nel >= (int64_t)1 << 31 || rows * std::max(g.r_ld, g.n_ld) >= (int64_t)1 << 31) return GALORE_ERR_SHAPE;
-  const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(nel, block), 148 * 8);
-  const bool packed = (g.cols == 0) || (g.r_ld == g.cols && g.n_ld == g.cols);
-  const int cols = (int)g.cols, r_ld = (int)g.r_ld, n_ld = (int)g.n_ld;
-#define GALORE_Q8_CASE(EPT)                                                                                  \
-  case EPT * 256:                                                                                            \
-    if (packed)                                                                                              \
-      adam_q8_kernel<TN, EPT, true><<<grid, 256, 0, st>>>(Rpart, splits, split_stride, (int)nel, Mc, Mam,    \
-                                                          Vc, Vam, Nout, p, cols, r_ld, n_ld, status);       \
-    else                                                                                                     \
-      adam_q8_kernel<TN, EPT, false><<<grid, 256, 0, st>>>(Rpart, splits, split_stride, (int)nel, Mc, Mam,   \
-                                                           Vc, Vam, Nout, p, cols, r_ld, n_ld, status);      \
+galore_status_t launch_adam_group(const AdamGroup& g, int32_t state_fmt, int q_block, int32_t n_dtype, cudaStream_t st) {
+  if (g.count < 1 || g.count > kAdamGroup) return GALORE_ERR_INVALID_ARG;
+  const int total = g.block_end[g.count - 1];
+  if (total <= 0) return GALORE_OK;
+  const unsigned grid = (unsigned)std::min(total, 148 * 8);
+  const bool nb = n_dtype == GALORE_BF16;
+  if (state_fmt == GALORE_STATE_F32) {
+    if (nb) adam_f32_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(g);
+    else adam_f32_kernel<float><<<grid, 256, 0, st>>>(g);
+    GALORE_LAUNCH_CHECK();
+    return GALORE_OK;
+  }
+  if (!valid_block(q_block)) return GALORE_ERR_INVALID_ARG;
+  GALORE_TRY(q8_ensure_tables());
+#define GALORE_Q8_CASE(EPT)                                                            \
+  case EPT * 256:                                                                      \
+    if (nb) adam_q8_kernel<__nv_bfloat16, EPT><<<grid, 256, 0, st>>>(g);               \
+    else adam_q8_kernel<float, EPT><<<grid, 256, 0, st>>>(g);                          \
     break;
-  switch (block) {
+  switch (q_block) {
     GALORE_Q8_CASE(1) GALORE_Q8_CASE(2) GALORE_Q8_CASE(4) GALORE_Q8_CASE(8) GALORE_Q8_CASE(16)
     default: return GALORE_ERR_INVALID_ARG;
   }
@@ -408,15 +461,49 @@ static galore_status_t adam_q8_t(const float* Rpart, int splits, int64_t split_s
   return GALORE_OK;
 }
 
+galore_status_t adam_group_add(AdamGroup& g, const AdamItem& item, int32_t state_fmt, int q_block) {
+  if (g.count >= kAdamGroup) return GALORE_ERR_BUFFER_TOO_SMALL;
+  AdamItem a = item;
+  if (a.cols == 0) a.cols = a.r_ld = a.n_ld = a.nel > 0 ? a.nel : 1;       // packed: one long row
+  // 32-bit offsets inside the kernels: the padded buffers must stay below 2^31 elements
+  const int64_t rows = ceil_div(a.nel, a.cols);
+  if (rows * std::max(a.r_ld, a.n_ld) >= (int64_t)1 << 31) return GALORE_ERR_SHAPE;
+  const int per_block = state_fmt == GALORE_STATE_F32 ? 2048 : q_block;
+  const int i = g.count++;
+  g.item[i] = a;
+  g.block_end[i] = (i > 0 ? g.block_end[i - 1] : 0) + (int)ceil_div(a.nel, per_block);
+  return GALORE_OK;
+}
+
+static galore_status_t single(const AdamItem& a, int32_t state_fmt, int q_block, int32_t n_dtype, cudaStream_t st) {
+  if (a.nel <= 0) return GALORE_OK;
+  std::unique_ptr<AdamGroup> g(new AdamGroup);
+  g->count = 0;
+  GALORE_TRY(adam_group_add(*g, a, state_fmt, q_block));
+  return launch_adam_group(*g, state_fmt, q_block, n_dtype, st);
+}
+
+galore_status_t launch_adam_f32(const float* Rpart, int splits, int64_t split_stride, int64_t nel, float* M,
+                                float* V, void* Nout, int32_t n_dtype, const AdamParams& p, int32_t* status,
+                                cudaStream_t st, const StateGeom& geo) {
+  if (nel >= (int64_t)1 << 31) return GALORE_ERR_SHAPE;
+  AdamItem a = {};
+  a.Rpart = Rpart; a.splits = splits; a.split_stride = split_stride; a.nel = (int)nel;
+  a.M = M; a.V = V; a.Nout = Nout; a.p = p; a.status = status;
+  a.cols = (int)geo.cols; a.r_ld = (int)geo.r_ld; a.n_ld = (int)geo.n_ld;
+  return single(a, GALORE_STATE_F32, 2048, n_dtype, st);
+}
+
 galore_status_t launch_adam_q8(const float* Rpart, int splits, int64_t split_stride, int64_t nel, uint8_t* Mc,
                                float* Mam, uint8_t* Vc, float* Vam, int block, void* Nout, int32_t n_dtype,
-                               const AdamParams& p, int32_t* status, cudaStream_t st, const StateGeom& g) {
-  if (nel <= 0) return GALORE_OK;
+                               const AdamParams& p, int32_t* status, cudaStream_t st, const StateGeom& geo) {
+  if (nel >= (int64_t)1 << 31) return GALORE_ERR_SHAPE;
   if (!valid_block(block)) return GALORE_ERR_INVALID_ARG;
-  GALORE_TRY(q8_ensure_tables());
-  if (n_dtype == GALORE_BF16)
-    return adam_q8_t(Rpart, splits, split_stride, nel, Mc, Mam, Vc, Vam, block, (__nv_bfloat16*)Nout, p, g, status, st);
-  return adam_q8_t(Rpart, splits, split_stride, nel, Mc, Mam, Vc, Vam, block, (float*)Nout, p, g, status, st);
+  AdamItem a = {};
+  a.Rpart = Rpart; a.splits = splits; a.split_stride = split_stride; a.nel = (int)nel;
+  a.Mc = Mc; a.Mam = Mam; a.Vc = Vc; a.Vam = Vam; a.Nout = Nout; a.p = p; a.status = status;
+  a.cols = (int)geo.cols; a.r_ld = (int)geo.r_ld; a.n_ld = (int)geo.n_ld;
+  return single(a, GALORE_STATE_Q8_BLOCK, block, n_dtype, st);
 }
 
 galore_status_t launch_q8_quantize(const float* x, int64_t nel, int is_signed, int block, uint8_t* codes,

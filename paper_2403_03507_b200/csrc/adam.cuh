@@ -24,6 +24,30 @@ struct StateGeom {
   }
 };
 
+// One layer's share of a grouped Adam launch.
+struct AdamItem {
+  const float* Rpart;      // split-K partials of R
+  int splits;
+  int64_t split_stride;
+  int nel;                 // state elements
+  float *M, *V;            // fp32 moments, or
+  uint8_t *Mc, *Vc;        // 8-bit codes with
+  float *Mam, *Vam;        // one absmax per quantisation block
+  void* Nout;              // normalised update (fp32 or bf16)
+  int cols, r_ld, n_ld;    // state row length and the row pitches of Rpart / Nout (cols == 0: packed)
+  AdamParams p;
+  int32_t* status;
+};
+constexpr int kAdamGroup = 32;
+struct AdamGroup {
+  AdamItem item[kAdamGroup];
+  int block_end[kAdamGroup];   // running total of work blocks
+  int count;
+};
+// all items of a group share the state format, the quantisation block and the dtype of N
+galore_status_t adam_group_add(AdamGroup& g, const AdamItem& item, int32_t state_fmt, int q_block);
+galore_status_t launch_adam_group(const AdamGroup& g, int32_t state_fmt, int q_block, int32_t n_dtype, cudaStream_t st);
+
 // R arrives as `splits` fp32 partial sums, each `split_stride` elements apart.
 galore_status_t launch_adam_f32(const float* Rpart, int splits, int64_t split_stride, int64_t nel, float* M,
                                 float* V, void* Nout, int32_t n_dtype, const AdamParams& p, int32_t* status,
