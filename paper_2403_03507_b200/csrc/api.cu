@@ -407,15 +407,166 @@ galore_status_t galore_step_host(galore_layer_t* l, void* W_host, const void* G_
   return s;
 }
 
-galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W, const int64_t* ldw, const void* const* G,
-                                  const int64_t* ldg, int32_t count, float lr, void* stream) {
-  if (count < 0 || (count > 0 && (!layers || !W || !ldw || !G || !ldg))) return GALORE_ERR_INVALID_ARG;
-  galore_status_t worst = GALORE_OK;
-  for (int32_t i = 0; i < count; ++i) {
-    galore_status_t s = galore_step(layers[i], W[i], ldw[i], G[i], ldg[i], lr, stream);
-    if (s < 0) return s;
-    if (s > worst) worst = s;
+// ---- batched step --------------------------------------------------------------------------------
+namespace {
+
+// bytes of group scratch one layer needs: R (one or tc_splits partial buffers) and N, each 256-aligned
+size_t batch_layer_bytes(const galore_layer* l, int splits) {
+  return align_up((size_t)splits * l->srows * l->ld_part * 4, 256) + align_up((size_t)l->srows * l->ld_n * 2, 256);
+}
+
+// With several layers in flight there are enough tiles to fill the machine without slicing K.
+int batch_splits(const galore_layer* l, int eligible) { return eligible >= 4 ? 1 : l->tc_splits; }
+
+bool batch_eligible(const galore_layer* l, const void* W, int64_t ldw, const void* G, int64_t ldg) {
+  return l->tensor_path && l->has_projector && tensor_operands_aligned(l->cfg, W, ldw, G, ldg);
+}
+
+AdamParams adam_params(const galore_layer* l) {
+  const double t = (double)(l->k + 1);
+  AdamParams ap;
+  ap.b1 = (float)l->cfg.beta1;
+  ap.b2 = (float)l->cfg.beta2;
+  ap.omb1 = (float)(1.0 - l->cfg.beta1);
+  ap.omb2 = (float)(1.0 - l->cfg.beta2);
+  ap.eps = (float)l->cfg.eps;
+  ap.inv_bc1 = (float)(1.0 / (1.0 - pow(l->cfg.beta1, t)));
+  ap.inv_bc2 = (float)(1.0 / (1.0 - pow(l->cfg.beta2, t)));
+  return ap;
+}
+
+struct BatchScratch {   // host-side objects reused across calls on this thread
+  TensorGroup* proj = nullptr;
+  TensorGroup* back = nullptr;
+  AdamGroup* adam = nullptr;
+  ~BatchScratch() {
+    tensor_group_free(proj);
+    tensor_group_free(back);
+    delete adam;
   }
+};
+
+}  // namespace
+
+galore_status_t galore_batch_query_bytes(galore_layer_t* const* layers, int32_t count, size_t* bytes) {
+  if (!bytes || count < 0 || (count > 0 && !layers)) return GALORE_ERR_INVALID_ARG;
+  int eligible = 0;
+  for (int32_t i = 0; i < count; ++i) {
+    if (!layers[i]) return GALORE_ERR_INVALID_ARG;
+    eligible += layers[i]->tensor_path ? 1 : 0;
+  }
+  // the largest sum over any run of `capacity` consecutive tensor-path layers
+  const int cap = std::min(tensor_group_capacity(), (int)kAdamGroup);
+  std::vector<size_t> need;
+  for (int32_t i = 0; i < count; ++i)
+    if (layers[i]->tensor_path) need.push_back(batch_layer_bytes(layers[i], batch_splits(layers[i], eligible)));
+  size_t best = 0, run = 0;
+  for (size_t i = 0; i < need.size(); ++i) {
+    run += need[i];
+    if (i >= (size_t)cap) run -= need[i - cap];
+    best = std::max(best, run);
+  }
+  *bytes = best;
+  return GALORE_OK;
+}
+
+galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W, const int64_t* ldw, const void* const* G,
+                                  const int64_t* ldg, int32_t count, float lr, void* batch_ws, size_t batch_ws_bytes,
+                                  void* stream) {
+  if (count < 0 || (count > 0 && (!layers || !W || !ldw || !G || !ldg))) return GALORE_ERR_INVALID_ARG;
+  if (batch_ws && ((uintptr_t)batch_ws & 255)) return GALORE_ERR_ALIGNMENT;
+  cudaStream_t st = (cudaStream_t)stream;
+  galore_status_t worst = GALORE_OK;
+  // refreshes that are due come first (each synchronises the stream and uses the layer's own workspace)
+  int eligible = 0;
+  for (int32_t i = 0; i < count; ++i) {
+    galore_layer* l = layers[i];
+    if (!l || !W[i] || !G[i] || ldw[i] < l->cfg.n || ldg[i] < l->cfg.n) return GALORE_ERR_INVALID_ARG;
+    if (l->cfg.auto_refresh && l->k % l->cfg.refresh_gap == 0) {
+      galore_status_t s = do_refresh(l, G[i], ldg[i], st, nullptr);
+      if (s < 0) return s;
+      worst = std::max(worst, s);
+    }
+    if (!l->has_projector) return GALORE_ERR_STATE;
+    eligible += batch_eligible(l, W[i], ldw[i], G[i], ldg[i]) ? 1 : 0;
+  }
+  static thread_local BatchScratch scratch;
+  if (!scratch.proj) scratch.proj = tensor_group_new();
+  if (!scratch.back) scratch.back = tensor_group_new();
+  if (!scratch.adam) scratch.adam = new (std::nothrow) AdamGroup;
+  if (!scratch.proj || !scratch.back || !scratch.adam) return GALORE_ERR_INVALID_ARG;
+  const int cap = std::min(tensor_group_capacity(), (int)kAdamGroup);
+
+  std::vector<int> group;          // indices of the layers in the group being assembled
+  size_t used = 0;
+  auto flush = [&]() -> galore_status_t {
+    if (group.empty()) return GALORE_OK;
+    const galore_layer* first = layers[group[0]];
+    {
+      PhaseTimer pt(0, st);
+      GALORE_TRY(tensor_group_launch_project(scratch.proj, st));
+    }
+    {
+      PhaseTimer pt(1, st);
+      GALORE_TRY(launch_adam_group(*scratch.adam, first->cfg.state_fmt, first->q_block, GALORE_BF16, st));
+    }
+    {
+      PhaseTimer pt(2, st);
+      GALORE_TRY(tensor_group_launch_back(scratch.back, first->cfg.w_dtype, st));
+    }
+    for (int i : group) layers[i]->k += 1;
+    group.clear();
+    used = 0;
+    tensor_group_reset(scratch.proj);
+    tensor_group_reset(scratch.back);
+    scratch.adam->count = 0;
+    return GALORE_OK;
+  };
+  tensor_group_reset(scratch.proj);
+  tensor_group_reset(scratch.back);
+  scratch.adam->count = 0;
+
+  for (int32_t i = 0; i < count; ++i) {
+    galore_layer* l = layers[i];
+    const bool ok = batch_ws && batch_eligible(l, W[i], ldw[i], G[i], ldg[i]);
+    const int splits = batch_splits(l, eligible);
+    const size_t need = ok ? batch_layer_bytes(l, splits) : 0;
+    if (!ok || need > batch_ws_bytes) {
+      // not groupable: plain step (its refresh, if due, is already done: auto_refresh off for this call)
+      const int32_t saved = l->cfg.auto_refresh;
+      l->cfg.auto_refresh = 0;
+      galore_status_t s = galore_step(l, W[i], ldw[i], G[i], ldg[i], lr, stream);
+      l->cfg.auto_refresh = saved;
+      if (s < 0) return s;
+      worst = std::max(worst, s);
+      continue;
+    }
+    if (!group.empty()) {
+      const galore_layer* first = layers[group[0]];
+      const bool same = first->cfg.w_dtype == l->cfg.w_dtype && first->cfg.state_fmt == l->cfg.state_fmt &&
+                        first->q_block == l->q_block;
+      if (!same || (int)group.size() >= cap || used + need > batch_ws_bytes) GALORE_TRY(flush());
+    }
+    char* base = (char*)batch_ws + used;
+    float* part = (float*)base;
+    void* nbuf = base + align_up((size_t)splits * l->srows * l->ld_part * 4, 256);
+    GALORE_TRY(tensor_group_add_project(scratch.proj, &l->tc, l->cfg, l->left, G[i], ldg[i], part, l->ld_part, splits, l->status));
+    AdamItem a = {};
+    a.Rpart = part;
+    a.splits = splits;
+    a.split_stride = l->srows * l->ld_part;
+    a.nel = (int)l->nel;
+    a.M = l->M; a.V = l->V; a.Mc = l->Mc; a.Vc = l->Vc; a.Mam = l->Mam; a.Vam = l->Vam;
+    a.Nout = nbuf;
+    a.cols = (int)l->scols; a.r_ld = (int)l->ld_part; a.n_ld = (int)l->ld_n;
+    a.p = adam_params(l);
+    a.status = l->status;
+    GALORE_TRY(adam_group_add(*scratch.adam, a, l->cfg.state_fmt, l->q_block));
+    GALORE_TRY(tensor_group_add_back(scratch.back, &l->tc, l->cfg, l->left, nbuf, l->ld_n, W[i], ldw[i], lr * l->cfg.alpha, l->status));
+    group.push_back(i);
+    used += need;
+  }
+  GALORE_TRY(flush());
   return worst;
 }
 
