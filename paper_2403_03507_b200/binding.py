@@ -65,8 +65,10 @@ _PROTOTYPES = {
                                     C.POINTER(C.c_void_p)]),
     "galore_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_float, C.c_void_p]),
     "galore_step_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
+    "galore_batch_query_bytes": (C.c_int, [C.POINTER(C.c_void_p), C.c_int32, C.POINTER(C.c_size_t)]),
     "galore_step_batch": (C.c_int, [C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_int64),
-                                    C.POINTER(C.c_void_p), C.POINTER(C.c_int64), C.c_int32, C.c_float, C.c_void_p]),
+                                    C.POINTER(C.c_void_p), C.POINTER(C.c_int64), C.c_int32, C.c_float, C.c_void_p,
+                                    C.c_size_t, C.c_void_p]),
     "galore_refresh_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.POINTER(RefreshInfo)]),
     "galore_free": (C.c_int, [C.c_void_p]),
     "galore_step_static": (C.c_int, [C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_float, C.c_double, C.c_double,
@@ -304,11 +306,45 @@ class Layer:
         return f.value
 
 
-def galore_step_batch(layers, Ws, Gs, lr: float, stream=None) -> int:
+def galore_batch_query_bytes(layers) -> int:
     n = len(layers)
-    hs = (C.c_void_p * n)(*[l.handle for l in layers])
-    wp = (C.c_void_p * n)(*[w.data_ptr() for w in Ws])
-    gp = (C.c_void_p * n)(*[g.data_ptr() for g in Gs])
-    lw = (C.c_int64 * n)(*[w.stride(0) for w in Ws])
-    lg = (C.c_int64 * n)(*[g.stride(0) for g in Gs])
-    return _check(lib().galore_step_batch(hs, wp, lw, gp, lg, n, lr, _stream_ptr(stream)), "galore_step_batch")
+    hs = (C.c_void_p * n)(*[l.handle.value for l in layers])
+    out = C.c_size_t(0)
+    _check(lib().galore_batch_query_bytes(hs, n, C.byref(out)), "galore_batch_query_bytes")
+    return out.value
+
+
+class Batch:
+    """A fixed list of layers stepped together by galore_step_batch.
+
+    Holds the batch workspace (torch) and the marshalled pointer arrays, so that a step is one
+    call into the library.  W and G tensors are bound once; rebind() swaps them.
+    """
+
+    def __init__(self, layers, Ws, Gs, workspace_bytes=None, device=None):
+        self.layers = list(layers)
+        self.n = len(self.layers)
+        self.device = device if device is not None else self.layers[0].device
+        need = galore_batch_query_bytes(self.layers)
+        self.workspace_bytes = need if workspace_bytes is None else int(workspace_bytes)
+        self.workspace = torch.empty(max(self.workspace_bytes, 256), dtype=torch.uint8, device=self.device)
+        self._hs = (C.c_void_p * self.n)(*[l.handle.value for l in self.layers])
+        self.rebind(Ws, Gs)
+
+    def rebind(self, Ws, Gs):
+        self.Ws, self.Gs = list(Ws), list(Gs)
+        n = self.n
+        self._wp = (C.c_void_p * n)(*[w.data_ptr() for w in self.Ws])
+        self._gp = (C.c_void_p * n)(*[g.data_ptr() for g in self.Gs])
+        self._lw = (C.c_int64 * n)(*[w.stride(0) for w in self.Ws])
+        self._lg = (C.c_int64 * n)(*[g.stride(0) for g in self.Gs])
+
+    def galore_step_batch(self, lr: float, stream=None) -> int:
+        return _check(lib().galore_step_batch(self._hs, self._wp, self._lw, self._gp, self._lg, self.n, lr,
+                                              self.workspace.data_ptr(), self.workspace_bytes, _stream_ptr(stream)),
+                      "galore_step_batch")
+
+
+def galore_step_batch(layers, Ws, Gs, lr: float, stream=None, workspace_bytes=None) -> int:
+    """One-off convenience: builds a Batch (allocating its workspace) and steps it once."""
+    return Batch(layers, Ws, Gs, workspace_bytes).galore_step_batch(lr, stream)

@@ -1,0 +1,128 @@
+"""galore_step_batch must give the same result as stepping each layer with galore_step."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import galore_oracle as go
+from paper_2403_03507_b200 import binding as gb
+from paper_2403_03507_b200 import workloads as wl
+
+from gpu_util import rel_err, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [(256, 512, 64), (512, 256, 64), (384, 1000, 128), (1000, 384, 128), (640, 640, 64), (200, 304, 16),
+          (256, 1096, 64), (130, 2056, 8)]
+
+
+def _make(state_fmt, w_dtype, path=gb.PATH_AUTO, g_dtype="bf16"):
+    layers, Ws, Gs, Ps, W0s, Gh = [], [], [], [], [], []
+    for i, (m, n, r) in enumerate(SHAPES):
+        cfg = gb.make_config(m, n, r, refresh_gap=1000, w_dtype=w_dtype, g_dtype=g_dtype, state_fmt=state_fmt,
+                             auto_refresh=False, path=path, q_block=256)
+        layer = gb.Layer(cfg)
+        d = m if layer.side == gb.SIDE_LEFT else n
+        P = wl.round_to(wl.random_orthonormal(d, r, np.random.default_rng(i)), g_dtype)
+        layer.set_projector(torch.from_numpy(P))
+        ld = (n + 7) // 8 * 8
+        W0 = wl.make_weight(m, n, 100 + i, w_dtype)
+        layers.append(layer)
+        Ps.append(P)
+        W0s.append(W0)
+        Ws.append(to_dev(W0, w_dtype, ld))
+    return layers, Ws, Ps, W0s
+
+
+def _grads(step, g_dtype="bf16"):
+    host = [wl.make_gradient(m, n, wl.sub_seed(7, i, step), 0.8, 0.05, g_dtype) for i, (m, n, r) in enumerate(SHAPES)]
+    dev = [to_dev(g, g_dtype, (g.shape[1] + 7) // 8 * 8) for g in host]
+    return host, dev
+
+
+@pytest.mark.parametrize("state_fmt,w_dtype", [("f32", "bf16"), ("q8", "bf16"), ("f32", "f32")])
+def test_batch_equals_per_layer_steps(state_fmt, w_dtype):
+    # The two modes slice K differently, so fp32 sums differ in the last bits; a bf16 rounding of N or
+    # of W that sits on a boundary may then flip (one bf16 ulp = 4e-3 of that element, on few elements).
+    tol = 5e-4 if w_dtype == "bf16" else 1e-5
+    la, Wa, _, _ = _make(state_fmt, w_dtype)
+    lb, Wb, _, _ = _make(state_fmt, w_dtype)
+    assert all(l.uses_tensor_path for l in la)
+    batch = None
+    for s in range(3):
+        _, G = _grads(s)
+        for l, w, g in zip(la, Wa, G):
+            l.galore_step(w, g, 1e-2)
+        if batch is None:
+            batch = gb.Batch(lb, Wb, G)
+        else:
+            batch.rebind(Wb, G)
+        batch.galore_step_batch(1e-2)
+    torch.cuda.synchronize()
+    for l1, l2, w1, w2 in zip(la, lb, Wa, Wb):
+        assert l2.step_count == 3 and l2.device_status() == 0
+        assert rel_err(to_host(w2), to_host(w1)) < tol
+        M1, V1 = l1.get_moments()
+        M2, V2 = l2.get_moments()
+        if state_fmt == "q8":   # a state on a threshold may land one code step apart
+            assert rel_err(to_host(M2), to_host(M1)) < 5e-3 and rel_err(to_host(V2), to_host(V1)) < 5e-3
+        else:
+            assert torch.allclose(M1, M2, rtol=1e-3, atol=1e-6) and torch.allclose(V1, V2, rtol=1e-3, atol=1e-9)
+
+
+def test_batch_matches_the_oracle():
+    layers, Ws, Ps, W0s = _make("q8", "bf16")
+    orcs = []
+    for (m, n, r), P in zip(SHAPES, Ps):
+        o = go.GaLoreOracle(m, n, r, 0.25, 1000, w_store="bf16", state="q8", q_block=256, n_store="bf16")
+        o.set_projector(P)
+        orcs.append(o)
+    Wo = list(W0s)
+    batch = None
+    for s in range(3):
+        Gh, Gd = _grads(s)
+        if batch is None:
+            batch = gb.Batch(layers, Ws, Gd)
+        else:
+            batch.rebind(Ws, Gd)
+        batch.galore_step_batch(1e-2)
+        Wo = [o.step(w, g, 1e-2, auto_refresh=False) for o, w, g in zip(orcs, Wo, Gh)]
+    for w_gpu, w_orc, w0 in zip(Ws, Wo, W0s):
+        assert rel_err(to_host(w_gpu), w_orc) <= 2e-2
+        assert rel_err(to_host(w_gpu) - w0, w_orc - w0) <= 5e-2
+
+
+def test_small_workspace_only_makes_groups_smaller_and_mixed_paths_work():
+    la, Wa, _, _ = _make("f32", "bf16")
+    lb, Wb, _, _ = _make("f32", "bf16")
+    _, G = _grads(0)
+    full = gb.galore_batch_query_bytes(la)
+    gb.Batch(la, Wa, G).galore_step_batch(1e-2)
+    gb.Batch(lb, Wb, G, workspace_bytes=full // 5).galore_step_batch(1e-2)      # several groups, maybe single steps
+    for w1, w2 in zip(Wa, Wb):
+        assert rel_err(to_host(w2), to_host(w1)) < 5e-4
+    # fp32 layers (not on the tensor path) inside a batch take the plain path
+    lc, Wc, _, _ = _make("f32", "f32", path=gb.PATH_FP32, g_dtype="f32")
+    ld_, Wd, _, _ = _make("f32", "f32", path=gb.PATH_FP32, g_dtype="f32")
+    _, G32 = _grads(0, "f32")
+    gb.Batch(lc, Wc, G32).galore_step_batch(1e-2)
+    for l, w, g in zip(ld_, Wd, G32):
+        l.galore_step(w, g, 1e-2)
+    for w1, w2 in zip(Wc, Wd):
+        assert torch.equal(w1, w2)
+
+
+def test_auto_refresh_inside_a_batch():
+    m, n, r = 256, 512, 32
+    cfgs = [gb.make_config(m, n, r, refresh_gap=2, auto_refresh=True, seed=3) for _ in range(4)]
+    la = [gb.Layer(c) for c in cfgs]
+    lb = [gb.Layer(c) for c in cfgs]
+    W0 = wl.make_weight(m, n, 1, "bf16")
+    Wa = [to_dev(W0, "bf16") for _ in la]
+    Wb = [to_dev(W0, "bf16") for _ in lb]
+    for s in range(3):
+        G = [to_dev(wl.make_gradient(m, n, wl.sub_seed(5, i, s), 0.8, 0.05, "bf16"), "bf16") for i in range(4)]
+        for l, w, g in zip(la, Wa, G):
+            l.galore_step(w, g, 1e-2)
+        gb.Batch(lb, Wb, G).galore_step_batch(1e-2)
+    for w1, w2 in zip(Wa, Wb):
+        assert rel_err(to_host(w2), to_host(w1)) < 5e-4
