@@ -178,6 +178,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--mode", default="batch", choices=["batch", "layer"],
+                    help="batch: galore_step_batch over the layer set (grouped launches); layer: galore_step per layer")
     ap.add_argument("--projector", default="refresh", choices=["refresh", "random"],
                     help="refresh: one real refresh per distinct shape (timed, reported); random: a random orthonormal "
                          "projector (step timing does not depend on P's values; for short profiling runs)")
@@ -287,7 +289,12 @@ def time_workload(w, args, dev, dist, world, rank, full):
             flops_alg += fl
     torch.cuda.synchronize()
 
+    batch = gb.Batch(layers, Ws, Gs, device=dev) if args.mode == "batch" else None
+
     def one_step(lr=w.lr):
+        if batch is not None:
+            batch.galore_step_batch(lr, stream)
+            return
         for layer, Wt, Gt in zip(layers, Ws, Gs):
             layer.galore_step(Wt, Gt, lr, stream)
 
@@ -356,7 +363,7 @@ def time_workload(w, args, dev, dist, world, rank, full):
         "dtype": "bf16" if uses_tc else "f32", "data": "synthetic",
         "config": {"workload": w.name, "matrices": w.matrices, "params": w.params, "rank": w.rank,
                    "state_fmt": w.state_fmt, "w_dtype": w.w_dtype, "g_dtype": w.g_dtype, "alpha": w.alpha,
-                   "refresh_gap": w.refresh_gap, "tensor_path": uses_tc, "parallelism": f"replicas x{world}",
+                   "refresh_gap": w.refresh_gap, "tensor_path": uses_tc, "mode": args.mode, "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (whole layer set streamed each step)"},
         "clocks": clocks, "gpu_launches": launches, "roofline": roof,
         "refresh": refresh_info,
