@@ -176,10 +176,10 @@ __device__ __forceinline__ float block_max_256(float v, float* red /* >= 8 float
 // Eq. 15 with bias correction.  The square root and the quotient use the approximate hardware
 // units (about 2 ulp each): N feeds a bf16 or fp32 GEMM operand and decides no integer.
 __device__ __forceinline__ float adam_normalised(float m, float v, const AdamParams& p) {
-  const float mh = m * p.inv_bc1;
-  const float vh = v * p.inv_bc2;
-  const float root = vh > 0.f ? vh * rsqrtf(vh) : 0.f;
-  return __fdividef(mh, root + p.eps);
+  float root, inv;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(root) : "f"(v * p.inv_bc2));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(root + p.eps));
+  return (m * p.inv_bc1) * inv;
 }
 
 // ---- grouped launches ------------------------------------------------------------
@@ -270,7 +270,7 @@ struct Q8Tables {
   float code_s[256], code_u[256], mid_s[256], mid_u[256];
   float2 pair_s[256], pair_u[256];
   uint8_t lut_s[2 * kLutSize], lut_u[kLutSize];
-  float red[8];
+  float red[16];
 };
 
 template <typename TN, int EPT, bool PACKED>
@@ -349,8 +349,86 @@ __device__ __forceinline__ bool adam_q8_block(const AdamItem& a, int blk, Q8Tabl
   return bad;
 }
 
+// max of two values over the CTA (256 threads) with one pair of barriers; every thread gets both
+__device__ __forceinline__ void block_max2_256(float& x, float& y, float* red /* >= 16 floats */) {
+  x = warp_max(x);
+  y = warp_max(y);
+  if ((threadIdx.x & 31) == 0) {
+    red[threadIdx.x >> 5] = x;
+    red[8 + (threadIdx.x >> 5)] = y;
+  }
+  __syncthreads();
+  float rx = red[0], ry = red[8];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) {
+    rx = fmaxf(rx, red[w]);
+    ry = fmaxf(ry, red[8 + w]);
+  }
+  __syncthreads();
+  x = rx;
+  y = ry;
+}
+
+// Full block of a layer whose R and N buffers have the state's own row pitch: every array is
+// addressed as base pointer + constant offset, no bounds checks.
 template <typename TN, int EPT>
-__global__ void __launch_bounds__(256) adam_q8_kernel(const __grid_constant__ AdamGroup g) {
+__device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q8Tables& t) {
+  const AdamParams p = a.p;
+  const int base = blk * (EPT * 256) + threadIdx.x;
+  const float* __restrict__ R = a.Rpart + base;
+  uint8_t* __restrict__ Mc = a.Mc + base;
+  uint8_t* __restrict__ Vc = a.Vc + base;
+  TN* __restrict__ Nout = (TN*)a.Nout + base;
+  const float am_m = a.Mam[blk], am_v = a.Vam[blk];
+  float r[EPT];
+  uint32_t cm[EPT], cv[EPT];
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    r[e] = R[e * 256];
+    cm[e] = Mc[e * 256];
+    cv[e] = Vc[e * 256];
+  }
+  for (int s = 1; s < a.splits; ++s) {
+    const float* __restrict__ part = R + (int64_t)s * a.split_stride;
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) r[e] += part[e * 256];
+  }
+  float m[EPT], v[EPT];
+  float mx_m = 0.f, mx_v = 0.f, poison = 0.f;
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    poison = fmaf(r[e], 0.f, poison);              // stays 0 unless some r is inf or nan
+    m[e] = p.b1 * (t.code_s[cm[e]] * am_m) + p.omb1 * r[e];
+    v[e] = p.b2 * (t.code_u[cv[e]] * am_v) + p.omb2 * (r[e] * r[e]);
+    Nout[e * 256] = cvt<TN>(adam_normalised(m[e], v[e], p));
+    mx_m = fmaxf(mx_m, fabsf(m[e]));
+    mx_v = fmaxf(mx_v, v[e]);
+  }
+  block_max2_256(mx_m, mx_v, t.red);
+  const float inv_m = 1.0f / mx_m, inv_v = 1.0f / mx_v;
+  if (mx_m == 0.f) {
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) Mc[e * 256] = (uint8_t)127;
+  } else {
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) Mc[e * 256] = (uint8_t)q8_encode_block<true>(m[e], mx_m, inv_m, t.lut_s, t.pair_s, t.mid_s);
+  }
+  if (mx_v == 0.f) {
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) Vc[e * 256] = (uint8_t)0;
+  } else {
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) Vc[e * 256] = (uint8_t)q8_encode_block<false>(v[e], mx_v, inv_v, t.lut_u, t.pair_u, t.mid_u);
+  }
+  if (threadIdx.x == 0) {
+    a.Mam[blk] = mx_m;
+    a.Vam[blk] = mx_v;
+  }
+  return poison != 0.f;
+}
+
+template <typename TN, int EPT>
+__global__ void __launch_bounds__(256, 4) adam_q8_kernel(const __grid_constant__ AdamGroup g) {
   __shared__ Q8Tables t;
   for (int i = threadIdx.x; i < kLutSize / 4; i += 256) {
     reinterpret_cast<uint32_t*>(t.lut_u)[i] = reinterpret_cast<const uint32_t*>(c_lut_u)[i];
@@ -372,7 +450,10 @@ __global__ void __launch_bounds__(256) adam_q8_kernel(const __grid_constant__ Ad
     const int it = find_item(g, gb, blk);
     const AdamItem& a = g.item[it];
     const bool packed = (a.r_ld == a.cols && a.n_ld == a.cols);
-    const bool bad = packed ? adam_q8_block<TN, EPT, true>(a, blk, t) : adam_q8_block<TN, EPT, false>(a, blk, t);
+    const bool full = (blk + 1) * (EPT * 256) <= a.nel;
+    const bool bad = (packed && full) ? adam_q8_block_full<TN, EPT>(a, blk, t)
+                     : packed         ? adam_q8_block<TN, EPT, true>(a, blk, t)
+                                      : adam_q8_block<TN, EPT, false>(a, blk, t);
     if (__syncthreads_or(bad)) bad_item = it;
   }
   if (bad_item >= 0 && threadIdx.x == 0) atomicOr(g.item[bad_item].status, GALORE_DEV_NONFINITE);
