@@ -34,7 +34,7 @@ constexpr int kBN = 256;          // columns of an output tile = TMEM columns pe
 constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int kStages = 4;
 constexpr int kUmmaK = 16;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;        // producer warp, MMA warp, two epilogue groups of four warps
 constexpr uint32_t kTmemCols = 512;
 constexpr int kABytes = kBM * kBK * 2;            // 16 KiB
 constexpr int kBBytes = kBN * kBK * 2;            // 32 KiB
@@ -272,6 +272,31 @@ __device__ __forceinline__ void epi_apply<float>(const TcParams& p, int row, int
   }
 }
 
+// one 16-byte vector of W: w <- w - scale * acc
+template <typename TW>
+__device__ __forceinline__ void apply_vec(uint4& raw, const uint32_t* acc, float scale);
+
+template <>
+__device__ __forceinline__ void apply_vec<__nv_bfloat16>(uint4& raw, const uint32_t* acc, float scale) {
+  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    float2 f = __bfloat1622float2(h[q]);
+    f.x = fmaf(-scale, __uint_as_float(acc[2 * q]), f.x);
+    f.y = fmaf(-scale, __uint_as_float(acc[2 * q + 1]), f.y);
+    h[q] = __floats2bfloat162_rn(f.x, f.y);
+  }
+}
+
+template <>
+__device__ __forceinline__ void apply_vec<float>(uint4& raw, const uint32_t* acc, float scale) {
+  float4* f = reinterpret_cast<float4*>(&raw);
+  f->x = fmaf(-scale, __uint_as_float(acc[0]), f->x);
+  f->y = fmaf(-scale, __uint_as_float(acc[1]), f->y);
+  f->z = fmaf(-scale, __uint_as_float(acc[2]), f->z);
+  f->w = fmaf(-scale, __uint_as_float(acc[3]), f->w);
+}
+
 // ---- the kernel -------------------------------------------------------------------------------
 
 template <int EPI, typename TW>
@@ -404,31 +429,73 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
     }
   } else {
     // ================= epilogue =================
+    // Two groups of four warps take the CTA's units in turn (group 0 the even ones with accumulator
+    // 0, group 1 the odd ones with accumulator 1), so that a group can start fetching the W tile of
+    // its next unit a whole unit ahead of the tensor cores.
     const int quarter = warp & 3;                   // TMEM lanes 32*quarter .. +31 belong to this warp
-    int acc = 0;
+    const int acc = (warp - 2) >> 2;                // epilogue group = accumulator it drains
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+    for (int u = blockIdx.x + acc * gridDim.x; u < total_units && ok; u += 2 * gridDim.x) {
       int pi;
       const Unit w = decode_unit(g, u, pi);
       const TcParams& p = g.p[pi];
-      if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
-      tc_fence_after();
       const int row = w.m0 + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kBN);
+      if (EPI == EPI_APPLY && w.n0 + kBN <= p.N) {
+        // Interior tile of the weight update.  The thread's stretch of its W row is fetched into
+        // registers BEFORE waiting for the accumulator: the loads do not depend on the MMAs, so the
+        // whole W tile streams in from HBM while the tensor cores are still working on it.
+        constexpr int kVec = 16 / (int)sizeof(TW);            // elements per 16-byte vector
+        constexpr int kPre = sizeof(TW) == 2 ? kBN : kBN / 2; // columns held in registers at once
+        constexpr int kNV = kPre / kVec;                      // 32 vectors = 128 registers
+        const bool row_ok = row < p.M;
+        TW* wrow = (TW*)p.W + (int64_t)(row_ok ? row : 0) * p.ldw + w.n0;
+        uint4 wv[kNV];
+        if (row_ok) {
+#pragma unroll
+          for (int j = 0; j < kNV; ++j) wv[j] = reinterpret_cast<const uint4*>(wrow)[j];
+        }
+        if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int h = 0; h < kBN / kPre; ++h) {
+          if (h > 0 && row_ok) {
+#pragma unroll
+            for (int j = 0; j < kNV; ++j) wv[j] = reinterpret_cast<const uint4*>(wrow + h * kPre)[j];
+          }
+#pragma unroll
+          for (int c = 0; c < kPre; c += 32) {
+            uint32_t v[32];
+            tmem_ld_32x32(t_row + (uint32_t)(h * kPre + c), v);
+            tmem_ld_wait();
+            if (row_ok) {
+#pragma unroll
+              for (int q = 0; q < 32 / kVec; ++q) {
+                uint4 raw = wv[c / kVec + q];
+                apply_vec<TW>(raw, &v[q * kVec], p.scale);
+                reinterpret_cast<uint4*>(wrow + h * kPre + c)[q] = raw;
+              }
+            }
+          }
+        }
+      } else {
+        if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+        tc_fence_after();
 #pragma unroll 1
-      for (int c = 0; c < kBN; c += 32) {
-        if (w.n0 + c >= p.N) break;                 // columns past the matrix: nothing to write
-        uint32_t v[32];
-        tmem_ld_32x32(t_row + (uint32_t)c, v);
-        tmem_ld_wait();
-        if (EPI == EPI_PARTIAL) epi_partial(p, w, row, w.n0 + c, v);
-        else epi_apply<TW>(p, row, w.n0 + c, v);
+        for (int c = 0; c < kBN; c += 32) {
+          if (w.n0 + c >= p.N) break;                 // columns past the matrix: nothing to write
+          uint32_t v[32];
+          tmem_ld_32x32(t_row + (uint32_t)c, v);
+          tmem_ld_wait();
+          if (EPI == EPI_PARTIAL) epi_partial(p, w, row, w.n0 + c, v);
+          else epi_apply<TW>(p, row, w.n0 + c, v);
+        }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acce_bar(acc));    // accumulator free for the MMA warp
-      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      acc_phase ^= 1u;
     }
   }
 
