@@ -544,7 +544,7 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
     if (!group.empty()) {
       const galore_layer* first = layers[group[0]];
       const bool same = first->cfg.w_dtype == l->cfg.w_dtype && first->cfg.state_fmt == l->cfg.state_fmt &&
-                        first->q_block == l->q_block;
+                        first->q_block == l->q_block && first->tc.ctas == l->tc.ctas;
       if (!same || (int)group.size() >= cap || used + need > batch_ws_bytes) GALORE_TRY(flush());
     }
     char* base = (char*)batch_ws + used;

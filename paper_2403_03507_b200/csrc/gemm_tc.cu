@@ -32,14 +32,24 @@ namespace {
 constexpr int kBM = 128;          // rows of an output tile = TMEM lanes
 constexpr int kBN = 256;          // columns of an output tile = TMEM columns per accumulator
 constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzle row
-constexpr int kStages = 4;
 constexpr int kUmmaK = 16;
 constexpr int kThreads = 320;        // producer warp, MMA warp, two epilogue groups of four warps
 constexpr uint32_t kTmemCols = 512;
-constexpr int kABytes = kBM * kBK * 2;            // 16 KiB
-constexpr int kBBytes = kBN * kBK * 2;            // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int kABytes = kBM * kBK * 2;            // 16 KiB: the 128 rows of A one CTA stages per k-block
+constexpr int kMaxStages = 6;
+
+// CTAS = 1: one CTA computes a 128 x 256 tile.  CTAS = 2: a cluster of two CTAs computes 256 x 256
+// with cta_group::2 MMAs; each CTA stages its own 128 rows of A and half (128 columns) of B, so a
+// k-block costs 32 KiB of shared-memory fill per CTA instead of 48 and the ring holds 6 stages.
+template <int CTAS>
+struct Geo {
+  static constexpr int kTileM = kBM * CTAS;
+  static constexpr int kBNcta = kBN / CTAS;
+  static constexpr int kBBytes = kBNcta * kBK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = CTAS == 1 ? 4 : 6;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+};
 constexpr long long kWaitLimitCycles = 4000000000LL;   // about two seconds
 
 enum { EPI_PARTIAL = 0, EPI_APPLY = 1 };
@@ -48,6 +58,7 @@ constexpr int kMaxGroup = 32;     // problems one launch can carry (its argument
 
 struct TcParams {
   int M, N, K;
+  int tile_m;                 // rows of a work unit: 128 (one CTA) or 256 (CTA pair)
   int a_mn, b_mn;             // operand majors in shared memory: 1 = M/N contiguous, 0 = K contiguous
   int tiles_m, tiles_n, splits;
   int kblocks_total, kblocks_per_split;
@@ -119,6 +130,56 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// ---- CTA pairs ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load of a CTA pair: data lands in this CTA, completion is signalled on the leader's barrier
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t leader_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(leader_bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_result, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D (+)= A B over the pair: 256 x kBN x 16; A rows and B columns are split between the two CTAs
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// one arrival on the barrier at this offset in both CTAs once the pair's MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_result, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(cols) : "memory");
 }
@@ -172,9 +233,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major) {
 }
 
 // Instruction descriptor: fp32 accumulate, bf16 x bf16, majors, N, M.
-__host__ __device__ constexpr uint32_t instr_desc(int a_mn, int b_mn) {
+__host__ __device__ constexpr uint32_t instr_desc(int a_mn, int b_mn, int tile_m) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-         ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+         ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
 }
 
 struct Unit {
@@ -197,7 +258,7 @@ __device__ __forceinline__ Unit decode_unit(const TcGroup& g, int u, int& pi) {
     tm = u / (p.tiles_n * p.splits);
   }
   Unit w;
-  w.m0 = tm * kBM;
+  w.m0 = tm * p.tile_m;
   w.n0 = tn * kBN;
   w.split = s;
   w.kb_begin = s * p.kblocks_per_split;
@@ -299,16 +360,20 @@ __device__ __forceinline__ void apply_vec<float>(uint4& raw, const uint32_t* acc
 
 // ---- the kernel -------------------------------------------------------------------------------
 
-template <int EPI, typename TW>
+template <int EPI, typename TW, int CTAS>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ TcGroup g) {
+  using G = Geo<CTAS>;
+  constexpr int kStages = G::kStages;
+  constexpr int kStageBytes = G::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   // stage ring, 1024-byte aligned for the 128-byte swizzle
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t ring = (raw_addr + 1023u) & ~1023u;
   uint8_t* ring_ptr = smem_raw + (ring - raw_addr);
   uint64_t* bars = reinterpret_cast<uint64_t*>(ring_ptr + kStages * kStageBytes);
-  // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty.
+  // In a CTA pair the full and accumulator-empty barriers that count are the leader's (rank 0).
   const uint32_t bar_base = smem_u32(bars);
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
@@ -320,6 +385,9 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int total_units = g.unit_end[g.count - 1];
+  const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;
+  const int team = blockIdx.x / CTAS;               // CTA or CTA pair that walks the units together
+  const int teams = gridDim.x / CTAS;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -328,57 +396,70 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(accf_bar(a), 1);
-      mbar_init(acce_bar(a), 4);     // one arrival per epilogue warp
+      mbar_init(acce_bar(a), 4 * CTAS);             // one arrival per epilogue warp of the group, from every CTA
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32((const void*)tmem_slot), kTmemCols);
-    tmem_relinquish();
+    if (CTAS == 2) {
+      tmem_alloc_pair(smem_u32((const void*)tmem_slot), kTmemCols);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(smem_u32((const void*)tmem_slot), kTmemCols);
+      tmem_relinquish();
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (CTAS == 2) cluster_sync_all();                // the peer's barriers exist before anyone signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ================= TMA producer =================
+    // ================= TMA producer (every CTA loads its own share) =================
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       long long issued = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+      for (int u = team; u < total_units && ok; u += teams) {
         int pi;
         const Unit w = decode_unit(g, u, pi);
         const bool A_MN = g.p[pi].a_mn != 0, B_MN = g.p[pi].b_mn != 0;
         const CUtensorMap* map_a = &g.map_a[pi];
         const CUtensorMap* map_b = &g.map_b[pi];
+        const int m0 = w.m0 + (int)rank * kBM;               // this CTA's rows of A
+        const int n0 = w.n0 + (int)rank * G::kBNcta;         // this CTA's columns of B
         for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t a_dst = ring + stage * kStageBytes;
           const uint32_t b_dst = a_dst + kABytes;
-          mbar_arrive_expect_tx(full_bar(stage), kStageBytes);
+          const uint32_t fbar = CTAS == 2 ? map_to_cta(full_bar(stage), 0) : full_bar(stage);
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), CTAS * kStageBytes);
           const int k0 = kb * kBK;
+          auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
+            if (CTAS == 2) tma_load_2d_pair(dst, map, x, y, fbar);
+            else tma_load_2d(dst, map, x, y, fbar);
+          };
           if (A_MN) {
 #pragma unroll
-            for (int j = 0; j < kBM / 64; ++j) tma_load_2d(a_dst + j * (kBK * 128), map_a, w.m0 + 64 * j, k0, full_bar(stage));
+            for (int j = 0; j < kBM / 64; ++j) load(a_dst + j * (kBK * 128), map_a, m0 + 64 * j, k0);
           } else {
-            tma_load_2d(a_dst, map_a, k0, w.m0, full_bar(stage));
+            load(a_dst, map_a, k0, m0);
           }
           if (B_MN) {
 #pragma unroll
-            for (int j = 0; j < kBN / 64; ++j) tma_load_2d(b_dst + j * (kBK * 128), map_b, w.n0 + 64 * j, k0, full_bar(stage));
+            for (int j = 0; j < G::kBNcta / 64; ++j) load(b_dst + j * (kBK * 128), map_b, n0 + 64 * j, k0);
           } else {
-            tma_load_2d(b_dst, map_b, k0, w.n0, full_bar(stage));
+            load(b_dst, map_b, k0, n0);
           }
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) {
+      if (!ok && CTAS == 1) {
         // let the copies that are still in flight land before the CTA goes away
         int s = stage;
         uint32_t ph = phase;
@@ -391,18 +472,18 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
       }
     }
   } else if (warp == 1) {
-    // ================= MMA issuer =================
-    if (lane == 0) {
+    // ================= MMA issuer (the leader CTA of a pair issues for both) =================
+    if (lane == 0 && rank == 0) {
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+      for (int u = team; u < total_units && ok; u += teams) {
         int pi;
         const Unit w = decode_unit(g, u, pi);
         const bool A_MN = g.p[pi].a_mn != 0, B_MN = g.p[pi].b_mn != 0;
-        const uint32_t idesc = instr_desc(g.p[pi].a_mn, g.p[pi].b_mn);
+        const uint32_t idesc = instr_desc(g.p[pi].a_mn, g.p[pi].b_mn, G::kTileM);
         if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kBN);
@@ -418,29 +499,36 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
             // K-major: 16 bf16 = 32 B along the swizzled row; MN-major: 16 k = two 8-k groups of 1024 B
             const uint64_t a_adv = (uint64_t)((A_MN ? k * 2048 : k * 32) >> 4);
             const uint64_t b_adv = (uint64_t)((B_MN ? k * 2048 : k * 32) >> 4);
-            umma_bf16(d_tmem, a_desc + a_adv, b_desc + b_adv, idesc, (kb > w.kb_begin || k > 0) ? 1u : 0u);
+            const uint32_t accum = (kb > w.kb_begin || k > 0) ? 1u : 0u;
+            if (CTAS == 2) umma_bf16_pair(d_tmem, a_desc + a_adv, b_desc + b_adv, idesc, accum);
+            else umma_bf16(d_tmem, a_desc + a_adv, b_desc + b_adv, idesc, accum);
           }
-          umma_commit(empty_bar(stage));            // stage reusable once these MMAs have read it
+          // stage reusable (in both CTAs of a pair) once these MMAs have read it
+          if (CTAS == 2) umma_commit_pair(empty_bar(stage));
+          else umma_commit(empty_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) umma_commit(accf_bar(acc));         // accumulator complete
+        if (ok) {                                     // accumulator complete
+          if (CTAS == 2) umma_commit_pair(accf_bar(acc));
+          else umma_commit(accf_bar(acc));
+        }
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
   } else {
     // ================= epilogue =================
-    // Two groups of four warps take the CTA's units in turn (group 0 the even ones with accumulator
+    // Two groups of four warps take the team's units in turn (group 0 the even ones with accumulator
     // 0, group 1 the odd ones with accumulator 1), so that a group can start fetching the W tile of
     // its next unit a whole unit ahead of the tensor cores.
     const int quarter = warp & 3;                   // TMEM lanes 32*quarter .. +31 belong to this warp
     const int acc = (warp - 2) >> 2;                // epilogue group = accumulator it drains
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int u = blockIdx.x + acc * gridDim.x; u < total_units && ok; u += 2 * gridDim.x) {
+    for (int u = team + acc * teams; u < total_units && ok; u += 2 * teams) {
       int pi;
       const Unit w = decode_unit(g, u, pi);
       const TcParams& p = g.p[pi];
-      const int row = w.m0 + quarter * 32 + lane;
+      const int row = w.m0 + (int)rank * kBM + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kBN);
       if (EPI == EPI_APPLY && w.n0 + kBN <= p.N) {
         // Interior tile of the weight update.  The thread's stretch of its W row is fetched into
@@ -494,17 +582,26 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(acce_bar(acc));    // accumulator free for the MMA warp
+      if (lane == 0) {                                // accumulator free for the MMA warp (the leader's)
+        if (rank == 0) mbar_arrive(acce_bar(acc));
+        else mbar_arrive_remote(map_to_cta(acce_bar(acc), 0));
+      }
       acc_phase ^= 1u;
     }
   }
 
+  if (CTAS == 2 && *abort_flag) {                     // gave up: let copies that are still in flight land
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) {}
+  }
   tc_fence_before();
   __syncthreads();
+  if (CTAS == 2) cluster_sync_all();                  // neither CTA leaves while the peer may still signal it
   if (threadIdx.x == 0 && *abort_flag) atomicOr(g.p[0].status, GALORE_DEV_WAIT_EXPIRED);
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
+    if (CTAS == 2) tmem_dealloc_pair(tmem_base, kTmemCols);
+    else tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -552,21 +649,43 @@ int sm_count() {
   return sms;
 }
 
-template <int EPI, typename TW>
-galore_status_t launch_tc(const TcGroup& g, cudaStream_t st) {
-  auto kern = gemm_tc_kernel<EPI, TW>;
+template <int EPI, typename TW, int CTAS>
+galore_status_t launch_tc_variant(const TcGroup& g, cudaStream_t st) {
+  auto kern = gemm_tc_kernel<EPI, TW, CTAS>;
+  constexpr int smem = Geo<CTAS>::kSmemBytes;
   static bool configured = false;
   if (!configured) {
-    GALORE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    GALORE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     configured = true;
   }
-  if (g.count < 1 || g.count > kMaxGroup) return GALORE_ERR_INVALID_ARG;
   const int units = g.unit_end[g.count - 1];
   if (units <= 0) return GALORE_OK;
-  const int grid = std::min(units, sm_count());
-  kern<<<grid, kThreads, kSmemBytes, st>>>(g);
-  GALORE_LAUNCH_CHECK();
+  const int teams = std::min(units, sm_count() / CTAS);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(teams * CTAS));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTAS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  GALORE_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, g));
+  count_launch();
   return GALORE_OK;
+}
+
+// every problem of a group was tiled for the same variant (TcParams::tile_m)
+template <int EPI, typename TW>
+galore_status_t launch_tc(const TcGroup& g, cudaStream_t st) {
+  if (g.count < 1 || g.count > kMaxGroup) return GALORE_ERR_INVALID_ARG;
+  for (int i = 1; i < g.count; ++i)
+    if (g.p[i].tile_m != g.p[0].tile_m) return GALORE_ERR_INVALID_ARG;
+  if (g.p[0].tile_m == 2 * kBM) return launch_tc_variant<EPI, TW, 2>(g, st);
+  return launch_tc_variant<EPI, TW, 1>(g, st);
 }
 
 // appends one problem to a group
@@ -578,9 +697,10 @@ void group_add(TcGroup& g, const CUtensorMap& ma, const CUtensorMap& mb, const T
   g.unit_end[i] = (i > 0 ? g.unit_end[i - 1] : 0) + p.tiles_m * p.tiles_n * p.splits;
 }
 
-void fill_tiles(TcParams& p, int M, int N, int K, int splits) {
+void fill_tiles(TcParams& p, int M, int N, int K, int splits, int ctas) {
   p.M = M; p.N = N; p.K = K;
-  p.tiles_m = (int)ceil_div(M, kBM);
+  p.tile_m = kBM * ctas;
+  p.tiles_m = (int)ceil_div(M, p.tile_m);
   p.tiles_n = (int)ceil_div(N, kBN);
   p.kblocks_total = (int)ceil_div(K, kBK);
   if (splits < 1) splits = 1;
@@ -589,10 +709,10 @@ void fill_tiles(TcParams& p, int M, int N, int K, int splits) {
 }
 
 // K slices that fill the last wave of CTAs best, keeping at least 4 k-blocks per slice
-int choose_splits(int64_t M, int64_t N, int64_t K) {
-  const int64_t tiles = ceil_div(M, kBM) * ceil_div(N, kBN);
+int choose_splits(int64_t M, int64_t N, int64_t K, int ctas) {
+  const int64_t tiles = ceil_div(M, kBM * ctas) * ceil_div(N, kBN);
   const int kblocks = (int)ceil_div(K, kBK);
-  const int sms = 148;
+  const int sms = 148 / ctas;
   int best = 1;
   double best_score = -1.0;
   for (int s = 1; s <= 8; ++s) {
@@ -615,14 +735,19 @@ bool tensor_path_eligible(const galore_config_t& c) {
   return c.g_dtype == GALORE_BF16 && c.p_dtype == GALORE_BF16 && (c.rank % 8) == 0;
 }
 
+// CTA pairs (256-row tiles) whenever every GEMM of the layer has at least 256 rows
+int tensor_ctas(const galore_config_t& c) { return c.rank >= 256 ? 2 : 1; }
+
 int tensor_proj_splits(const galore_config_t& c, bool left) {
-  if (left) return choose_splits(c.rank, c.n, c.m);
-  return choose_splits(c.m, c.rank, c.n);
+  const int ctas = tensor_ctas(c);
+  if (left) return choose_splits(c.rank, c.n, c.m, ctas);
+  return choose_splits(c.m, c.rank, c.n, ctas);
 }
 
 galore_status_t tensor_plan_init(TensorPlan* plan, const galore_config_t& c, bool left, void* P, void* Nbuf, float* Rpart,
                                  int splits, int64_t ld_part, int64_t ld_n) {
   plan->ready = false;
+  plan->ctas = tensor_ctas(c);
   plan->splits = splits;
   plan->P = P;
   plan->Nbuf = Nbuf;
@@ -639,7 +764,7 @@ galore_status_t tensor_plan_init(TensorPlan* plan, const galore_config_t& c, boo
   } else {
     // projection: B = Q (n x r), MN-major;  back-projection: B = Q^T, K-major from Q
     GALORE_TRY(make_map(&plan->map_p_proj, P, c.n, r, r, 64));
-    GALORE_TRY(make_map(&plan->map_p_back, P, c.n, r, r, kBN));
+    GALORE_TRY(make_map(&plan->map_p_back, P, c.n, r, r, kBN / plan->ctas));   // each CTA of a pair stages half of B
     // back-projection: A = N (m x r), K-major
     GALORE_TRY(make_map(&plan->map_n_back, Nbuf, c.m, r, ld_n, kBM));
   }
@@ -667,7 +792,7 @@ static galore_status_t project_problem(const TensorPlan* plan, const galore_conf
   p->ld_part = ld_part;
   if (left) {
     // A = P^T, M/N-major from P; B = G, M/N-major.  G is the big operand: units sharing a G panel run together
-    fill_tiles(*p, r, (int)c.n, (int)c.m, splits);
+    fill_tiles(*p, r, (int)c.n, (int)c.m, splits, plan->ctas);
     p->split_stride = (int64_t)r * ld_part;
     p->m_fast = 1;
     p->a_mn = 1;
@@ -676,7 +801,7 @@ static galore_status_t project_problem(const TensorPlan* plan, const galore_conf
     return make_map(mb, G, c.m, c.n, ldg, 64);
   }
   // A = G, K-major; B = Q, M/N-major
-  fill_tiles(*p, (int)c.m, r, (int)c.n, splits);
+  fill_tiles(*p, (int)c.m, r, (int)c.n, splits, plan->ctas);
   p->split_stride = (int64_t)c.m * ld_part;
   p->m_fast = 0;
   p->a_mn = 0;
@@ -696,7 +821,7 @@ static galore_status_t back_problem(const TensorPlan* plan, const galore_config_
   p->ldw = ldw;
   p->scale = scale;
   p->m_fast = 1;
-  fill_tiles(*p, (int)c.m, (int)c.n, c.rank, 1);
+  fill_tiles(*p, (int)c.m, (int)c.n, c.rank, 1, plan->ctas);
   if (left) {   // A = P K-major, B = N M/N-major
     p->a_mn = 0;
     p->b_mn = 1;

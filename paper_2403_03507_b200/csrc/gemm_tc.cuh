@@ -12,6 +12,7 @@ namespace galore {
 struct TensorPlan {
   bool ready = false;
   int splits = 1;             // K slices of the projection
+  int ctas = 1;               // 1: 128-row tiles per CTA; 2: 256-row tiles per CTA pair (cta_group::2)
   void* P = nullptr;
   void* Nbuf = nullptr;       // normalised update, bf16, leading dimension ld_n
   float* Rpart = nullptr;     // split-K partials of R, fp32, leading dimension ld_part
@@ -24,6 +25,7 @@ struct TensorPlan {
 // bf16 G and P, rank a multiple of 8 (16-byte rows for TMA).
 bool tensor_path_eligible(const galore_config_t& cfg);
 int tensor_proj_splits(const galore_config_t& cfg, bool left);
+int tensor_ctas(const galore_config_t& cfg);
 galore_status_t tensor_plan_init(TensorPlan* plan, const galore_config_t& cfg, bool left, void* P, void* Nbuf,
                                  float* Rpart, int splits, int64_t ld_part, int64_t ld_n);
 // G and W usable by this path: 16-byte aligned bases and rows.

@@ -40,7 +40,10 @@ def _run(m, n, r, w_dtype, fmt, steps=3, ldw=None, ldg=None, q_block=2048, path=
 
 
 @pytest.mark.parametrize("m,n,r", [(256, 512, 64), (512, 256, 64), (384, 1000, 128), (1000, 384, 128),
-                                   (200, 304, 16), (130, 2056, 8), (640, 640, 640), (77, 1032, 72)])
+                                   (200, 304, 16), (130, 2056, 8), (640, 640, 640), (77, 1032, 72),
+                                   # rank >= 256: CTA-pair kernels (256-row tiles), exact and ragged in every dimension
+                                   (512, 1024, 256), (1024, 512, 256), (300, 1000, 256), (1000, 300, 256),
+                                   (1100, 2600, 384)])
 @pytest.mark.parametrize("w_dtype", ["bf16", "f32"])
 def test_tensor_path_fp32_states(m, n, r, w_dtype):
     ld = (n + 7) // 8 * 8
