@@ -142,7 +142,7 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
     s->proj_splits = simt_effective_splits((int)s->d, want);
   }
   s->tc_splits = s->tensor_path ? tensor_proj_splits(*c, s->left) : 0;
-  s->ld_part = (s->scols + 3) / 4 * 4;     // 16-byte rows for vector stores
+  s->ld_part = (s->scols + 7) / 8 * 8;     // 32-byte rows for whole-sector vector stores
   s->ld_n = (s->scols + 7) / 8 * 8;        // 16-byte bf16 rows for TMA
 
   size_t o = 0;

@@ -33,7 +33,7 @@ constexpr int kBM = 128;          // rows of an output tile = TMEM lanes
 constexpr int kBN = 256;          // columns of an output tile = TMEM columns per accumulator
 constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;
-constexpr int kThreads = 320;        // producer warp, MMA warp, two epilogue groups of four warps
+constexpr int kThreads = 192;        // producer warp, MMA warp, four epilogue warps
 constexpr uint32_t kTmemCols = 512;
 constexpr int kABytes = kBM * kBK * 2;            // 16 KiB: the 128 rows of A one CTA stages per k-block
 constexpr int kMaxStages = 6;
@@ -69,6 +69,7 @@ struct TcParams {
   // EPI_APPLY
   void* W;
   int64_t ldw;
+  int vec32;                  // W base and row pitch (resp. the partial buffer's) are 32-byte aligned
   float scale;
   int32_t* status;
 };
@@ -221,6 +222,20 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32])
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// 32-byte global accesses: one request covers a whole 32-byte sector, so a thread that walks its own
+// row does not send half-filled sectors through the L1/L2 fabric.  Address must be 32-byte aligned.
+__device__ __forceinline__ void ld_global_32B(const void* ptr, uint4& a, uint4& b) {
+  asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w)
+               : "l"(ptr)
+               : "memory");
+}
+__device__ __forceinline__ void st_global_32B(void* ptr, const uint4& a, const uint4& b) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+               ::"l"(ptr), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
+               : "memory");
+}
+
 // ---- descriptors ------------------------------------------------------------------------
 // Shared-memory operand descriptor, 128-byte swizzle, tile base 1024-byte aligned.
 //  K-major  : rows of 64 bf16 (128 B); 8-row groups 1024 B apart (stride offset); leading offset unused.
@@ -272,7 +287,11 @@ __device__ __forceinline__ Unit decode_unit(const TcGroup& g, int u, int& pi) {
 __device__ __forceinline__ void epi_partial(const TcParams& p, const Unit& w, int row, int col0, const uint32_t (&v)[32]) {
   if (row >= p.M) return;
   float* dst = p.part + (int64_t)w.split * p.split_stride + (int64_t)row * p.ld_part + col0;
-  if (col0 + 32 <= p.N && (p.ld_part & 3) == 0) {
+  if (col0 + 32 <= p.N && p.vec32) {
+#pragma unroll
+    for (int j = 0; j < 32; j += 8)
+      st_global_32B(dst + j, make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]), make_uint4(v[j + 4], v[j + 5], v[j + 6], v[j + 7]));
+  } else if (col0 + 32 <= p.N && (p.ld_part & 3) == 0) {
 #pragma unroll
     for (int j = 0; j < 32; j += 4)
       *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
@@ -517,14 +536,11 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
     }
   } else {
     // ================= epilogue =================
-    // Two groups of four warps take the team's units in turn (group 0 the even ones with accumulator
-    // 0, group 1 the odd ones with accumulator 1), so that a group can start fetching the W tile of
-    // its next unit a whole unit ahead of the tensor cores.
     const int quarter = warp & 3;                   // TMEM lanes 32*quarter .. +31 belong to this warp
-    const int acc = (warp - 2) >> 2;                // epilogue group = accumulator it drains
+    int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int u = team + acc * teams; u < total_units && ok; u += 2 * teams) {
+    for (int u = team; u < total_units && ok; u += teams) {
       int pi;
       const Unit w = decode_unit(g, u, pi);
       const TcParams& p = g.p[pi];
@@ -540,29 +556,37 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
         const bool row_ok = row < p.M;
         TW* wrow = (TW*)p.W + (int64_t)(row_ok ? row : 0) * p.ldw + w.n0;
         uint4 wv[kNV];
-        if (row_ok) {
+        const bool vec32 = p.vec32 != 0;
+        auto fetch = [&](const TW* src) {
+          if (vec32) {
 #pragma unroll
-          for (int j = 0; j < kNV; ++j) wv[j] = reinterpret_cast<const uint4*>(wrow)[j];
-        }
+            for (int j = 0; j < kNV; j += 2) ld_global_32B(reinterpret_cast<const uint4*>(src) + j, wv[j], wv[j + 1]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < kNV; ++j) wv[j] = reinterpret_cast<const uint4*>(src)[j];
+          }
+        };
+        if (row_ok) fetch(wrow);
         if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
         tc_fence_after();
 #pragma unroll
         for (int h = 0; h < kBN / kPre; ++h) {
-          if (h > 0 && row_ok) {
-#pragma unroll
-            for (int j = 0; j < kNV; ++j) wv[j] = reinterpret_cast<const uint4*>(wrow + h * kPre)[j];
-          }
+          if (h > 0 && row_ok) fetch(wrow + h * kPre);
 #pragma unroll
           for (int c = 0; c < kPre; c += 32) {
             uint32_t v[32];
             tmem_ld_32x32(t_row + (uint32_t)(h * kPre + c), v);
             tmem_ld_wait();
             if (row_ok) {
+              uint4* dst = reinterpret_cast<uint4*>(wrow + h * kPre + c);
 #pragma unroll
-              for (int q = 0; q < 32 / kVec; ++q) {
-                uint4 raw = wv[c / kVec + q];
-                apply_vec<TW>(raw, &v[q * kVec], p.scale);
-                reinterpret_cast<uint4*>(wrow + h * kPre + c)[q] = raw;
+              for (int q = 0; q < 32 / kVec; ++q) apply_vec<TW>(wv[c / kVec + q], &v[q * kVec], p.scale);
+              if (vec32) {
+#pragma unroll
+                for (int q = 0; q < 32 / kVec; q += 2) st_global_32B(dst + q, wv[c / kVec + q], wv[c / kVec + q + 1]);
+              } else {
+#pragma unroll
+                for (int q = 0; q < 32 / kVec; ++q) dst[q] = wv[c / kVec + q];
               }
             }
           }
@@ -586,7 +610,7 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
         if (rank == 0) mbar_arrive(acce_bar(acc));
         else mbar_arrive_remote(map_to_cta(acce_bar(acc), 0));
       }
-      acc_phase ^= 1u;
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }
 
@@ -790,6 +814,7 @@ static galore_status_t project_problem(const TensorPlan* plan, const galore_conf
   p->status = status;
   p->part = part;
   p->ld_part = ld_part;
+  p->vec32 = (((uintptr_t)part & 31) == 0 && (ld_part % 8) == 0) ? 1 : 0;
   if (left) {
     // A = P^T, M/N-major from P; B = G, M/N-major.  G is the big operand: units sharing a G panel run together
     fill_tiles(*p, r, (int)c.n, (int)c.m, splits, plan->ctas);
@@ -819,6 +844,7 @@ static galore_status_t back_problem(const TensorPlan* plan, const galore_config_
   p->status = status;
   p->W = W;
   p->ldw = ldw;
+  p->vec32 = (((uintptr_t)W & 31) == 0 && (ldw * (int64_t)dtype_size(c.w_dtype)) % 32 == 0) ? 1 : 0;
   p->scale = scale;
   p->m_fast = 1;
   fill_tiles(*p, (int)c.m, (int)c.n, c.rank, 1, plan->ctas);
