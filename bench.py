@@ -234,7 +234,7 @@ def time_workload(w, args, dev, dist, world, rank, full):
     stream = torch.cuda.current_stream()
 
     def padded(m, n, dtype):
-        ld = (n + 7) // 8 * 8          # 16-byte rows so that TMA can address bf16 operands
+        ld = (n + 15) // 16 * 16       # 32-byte bf16 rows: TMA-addressable, and whole-sector vector accesses
         buf = torch.empty(m, ld, dtype=dtype, device=dev)
         return buf[:, :n]
 

@@ -439,11 +439,21 @@ struct BatchScratch {   // host-side objects reused across calls on this thread
   TensorGroup* proj = nullptr;
   TensorGroup* back = nullptr;
   AdamGroup* adam = nullptr;
+  cudaStream_t aux = nullptr;           // carries the Adam launches so that they overlap the GEMMs
+  int aux_device = -1;
+  std::vector<cudaEvent_t> events;
   ~BatchScratch() {
     tensor_group_free(proj);
     tensor_group_free(back);
     delete adam;
+    // stream and events are left to the driver at process exit (the context may already be gone)
   }
+};
+
+struct BatchMember {
+  int index;            // position in the caller's arrays
+  size_t offset;        // where its R partials start inside the batch workspace
+  int splits;
 };
 
 }  // namespace
@@ -455,7 +465,8 @@ galore_status_t galore_batch_query_bytes(galore_layer_t* const* layers, int32_t 
     if (!layers[i]) return GALORE_ERR_INVALID_ARG;
     eligible += layers[i]->tensor_path ? 1 : 0;
   }
-  // the largest sum over any run of `capacity` consecutive tensor-path layers
+  // the largest sum over any run of `capacity` consecutive tensor-path layers, twice: two groups are in
+  // flight at a time (the Adam pass of one overlaps the GEMMs of the next)
   const int cap = std::min(tensor_group_capacity(), (int)kAdamGroup);
   std::vector<size_t> need;
   for (int32_t i = 0; i < count; ++i)
@@ -466,7 +477,7 @@ galore_status_t galore_batch_query_bytes(galore_layer_t* const* layers, int32_t 
     if (i >= (size_t)cap) run -= need[i - cap];
     best = std::max(best, run);
   }
-  *bytes = best;
+  *bytes = need.size() > (size_t)cap ? 2 * best : best;
   return GALORE_OK;
 }
 
@@ -497,76 +508,143 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
   if (!scratch.proj || !scratch.back || !scratch.adam) return GALORE_ERR_INVALID_ARG;
   const int cap = std::min(tensor_group_capacity(), (int)kAdamGroup);
 
-  std::vector<int> group;          // indices of the layers in the group being assembled
-  size_t used = 0;
-  auto flush = [&]() -> galore_status_t {
-    if (group.empty()) return GALORE_OK;
-    const galore_layer* first = layers[group[0]];
-    {
-      PhaseTimer pt(0, st);
-      GALORE_TRY(tensor_group_launch_project(scratch.proj, st));
+  // ---- 1. partition: layers that cannot be grouped step on their own, the rest form groups ----------
+  // Two groups are in flight at a time, each in its own half of the workspace.
+  const size_t half = (batch_ws_bytes / 2) & ~(size_t)255;
+  std::vector<std::vector<BatchMember>> groups;
+  {
+    size_t used = 0;
+    for (int32_t i = 0; i < count; ++i) {
+      galore_layer* l = layers[i];
+      const bool ok = batch_ws && batch_eligible(l, W[i], ldw[i], G[i], ldg[i]);
+      const int splits = batch_splits(l, eligible);
+      const size_t need = ok ? batch_layer_bytes(l, splits) : 0;
+      if (!ok || need > half) {
+        // plain step (its refresh, if due, is already done: auto_refresh off for this call)
+        const int32_t saved = l->cfg.auto_refresh;
+        l->cfg.auto_refresh = 0;
+        galore_status_t s = galore_step(l, W[i], ldw[i], G[i], ldg[i], lr, stream);
+        l->cfg.auto_refresh = saved;
+        if (s < 0) return s;
+        worst = std::max(worst, s);
+        continue;
+      }
+      bool fresh = groups.empty();
+      if (!fresh) {
+        const galore_layer* first = layers[groups.back()[0].index];
+        const bool same = first->cfg.w_dtype == l->cfg.w_dtype && first->cfg.state_fmt == l->cfg.state_fmt &&
+                          first->q_block == l->q_block && first->tc.ctas == l->tc.ctas;
+        fresh = !same || (int)groups.back().size() >= cap || used + need > half;
+      }
+      if (fresh) {
+        groups.emplace_back();
+        used = 0;
+      }
+      groups.back().push_back(BatchMember{i, used, splits});
+      used += need;
     }
-    {
-      PhaseTimer pt(1, st);
-      GALORE_TRY(launch_adam_group(*scratch.adam, first->cfg.state_fmt, first->q_block, GALORE_BF16, st));
-    }
-    {
-      PhaseTimer pt(2, st);
-      GALORE_TRY(tensor_group_launch_back(scratch.back, first->cfg.w_dtype, st));
-    }
-    for (int i : group) layers[i]->k += 1;
-    group.clear();
-    used = 0;
+  }
+  if (groups.empty()) return worst;
+
+  // ---- 2. launch helpers -------------------------------------------------------------------------------
+  auto scratch_of = [&](size_t gi, const BatchMember& mb, float** part, void** nbuf) {
+    const galore_layer* l = layers[mb.index];
+    char* base = (char*)batch_ws + (gi & 1) * half + mb.offset;
+    *part = (float*)base;
+    *nbuf = base + align_up((size_t)mb.splits * l->srows * l->ld_part * 4, 256);
+  };
+  auto launch_proj = [&](size_t gi, cudaStream_t s) -> galore_status_t {
     tensor_group_reset(scratch.proj);
-    tensor_group_reset(scratch.back);
+    for (const BatchMember& mb : groups[gi]) {
+      galore_layer* l = layers[mb.index];
+      float* part; void* nbuf;
+      scratch_of(gi, mb, &part, &nbuf);
+      GALORE_TRY(tensor_group_add_project(scratch.proj, &l->tc, l->cfg, l->left, G[mb.index], ldg[mb.index], part,
+                                          l->ld_part, mb.splits, l->status));
+    }
+    PhaseTimer pt(0, s);
+    return tensor_group_launch_project(scratch.proj, s);
+  };
+  auto launch_adam = [&](size_t gi, cudaStream_t s) -> galore_status_t {
     scratch.adam->count = 0;
+    const galore_layer* first = layers[groups[gi][0].index];
+    for (const BatchMember& mb : groups[gi]) {
+      galore_layer* l = layers[mb.index];
+      float* part; void* nbuf;
+      scratch_of(gi, mb, &part, &nbuf);
+      AdamItem a = {};
+      a.Rpart = part;
+      a.splits = mb.splits;
+      a.split_stride = l->srows * l->ld_part;
+      a.nel = (int)l->nel;
+      a.M = l->M; a.V = l->V; a.Mc = l->Mc; a.Vc = l->Vc; a.Mam = l->Mam; a.Vam = l->Vam;
+      a.Nout = nbuf;
+      a.cols = (int)l->scols; a.r_ld = (int)l->ld_part; a.n_ld = (int)l->ld_n;
+      a.p = adam_params(l);
+      a.status = l->status;
+      GALORE_TRY(adam_group_add(*scratch.adam, a, l->cfg.state_fmt, l->q_block));
+    }
+    PhaseTimer pt(1, s);
+    return launch_adam_group(*scratch.adam, first->cfg.state_fmt, first->q_block, GALORE_BF16, s);
+  };
+  auto launch_back = [&](size_t gi, cudaStream_t s) -> galore_status_t {
+    tensor_group_reset(scratch.back);
+    const galore_layer* first = layers[groups[gi][0].index];
+    for (const BatchMember& mb : groups[gi]) {
+      galore_layer* l = layers[mb.index];
+      float* part; void* nbuf;
+      scratch_of(gi, mb, &part, &nbuf);
+      GALORE_TRY(tensor_group_add_back(scratch.back, &l->tc, l->cfg, l->left, nbuf, l->ld_n, W[mb.index], ldw[mb.index],
+                                       lr * l->cfg.alpha, l->status));
+    }
+    PhaseTimer pt(2, s);
+    GALORE_TRY(tensor_group_launch_back(scratch.back, first->cfg.w_dtype, s));
+    for (const BatchMember& mb : groups[gi]) layers[mb.index]->k += 1;
     return GALORE_OK;
   };
-  tensor_group_reset(scratch.proj);
-  tensor_group_reset(scratch.back);
-  scratch.adam->count = 0;
 
-  for (int32_t i = 0; i < count; ++i) {
-    galore_layer* l = layers[i];
-    const bool ok = batch_ws && batch_eligible(l, W[i], ldw[i], G[i], ldg[i]);
-    const int splits = batch_splits(l, eligible);
-    const size_t need = ok ? batch_layer_bytes(l, splits) : 0;
-    if (!ok || need > batch_ws_bytes) {
-      // not groupable: plain step (its refresh, if due, is already done: auto_refresh off for this call)
-      const int32_t saved = l->cfg.auto_refresh;
-      l->cfg.auto_refresh = 0;
-      galore_status_t s = galore_step(l, W[i], ldw[i], G[i], ldg[i], lr, stream);
-      l->cfg.auto_refresh = saved;
-      if (s < 0) return s;
-      worst = std::max(worst, s);
-      continue;
+  // ---- 3. schedule ----------------------------------------------------------------------------------------
+  // Phase timing wants the phases back to back on one stream; so does a single group.
+  const size_t ng = groups.size();
+  const bool overlap = ng > 1 && g_profile.load(std::memory_order_relaxed) == 0;
+  if (!overlap) {
+    for (size_t gi = 0; gi < ng; ++gi) {
+      GALORE_TRY(launch_proj(gi, st));
+      GALORE_TRY(launch_adam(gi, st));
+      GALORE_TRY(launch_back(gi, st));
     }
-    if (!group.empty()) {
-      const galore_layer* first = layers[group[0]];
-      const bool same = first->cfg.w_dtype == l->cfg.w_dtype && first->cfg.state_fmt == l->cfg.state_fmt &&
-                        first->q_block == l->q_block && first->tc.ctas == l->tc.ctas;
-      if (!same || (int)group.size() >= cap || used + need > batch_ws_bytes) GALORE_TRY(flush());
-    }
-    char* base = (char*)batch_ws + used;
-    float* part = (float*)base;
-    void* nbuf = base + align_up((size_t)splits * l->srows * l->ld_part * 4, 256);
-    GALORE_TRY(tensor_group_add_project(scratch.proj, &l->tc, l->cfg, l->left, G[i], ldg[i], part, l->ld_part, splits, l->status));
-    AdamItem a = {};
-    a.Rpart = part;
-    a.splits = splits;
-    a.split_stride = l->srows * l->ld_part;
-    a.nel = (int)l->nel;
-    a.M = l->M; a.V = l->V; a.Mc = l->Mc; a.Vc = l->Vc; a.Mam = l->Mam; a.Vam = l->Vam;
-    a.Nout = nbuf;
-    a.cols = (int)l->scols; a.r_ld = (int)l->ld_part; a.n_ld = (int)l->ld_n;
-    a.p = adam_params(l);
-    a.status = l->status;
-    GALORE_TRY(adam_group_add(*scratch.adam, a, l->cfg.state_fmt, l->q_block));
-    GALORE_TRY(tensor_group_add_back(scratch.back, &l->tc, l->cfg, l->left, nbuf, l->ld_n, W[i], ldw[i], lr * l->cfg.alpha, l->status));
-    group.push_back(i);
-    used += need;
+    return worst;
   }
-  GALORE_TRY(flush());
+  // Adam is arithmetic on the CUDA cores, the GEMMs live on the tensor cores and the memory fabric:
+  // the Adam pass of group g runs on a second stream under the projection of group g+1 and the
+  // back-projection of group g-1.  Everything is joined back into the caller's stream by events.
+  int dev = 0;
+  GALORE_CUDA_TRY(cudaGetDevice(&dev));
+  if (!scratch.aux || scratch.aux_device != dev) {
+    GALORE_CUDA_TRY(cudaStreamCreateWithFlags(&scratch.aux, cudaStreamNonBlocking));
+    scratch.aux_device = dev;
+    scratch.events.clear();
+  }
+  while (scratch.events.size() < 2 * ng) {
+    cudaEvent_t e;
+    GALORE_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    scratch.events.push_back(e);
+  }
+  auto ev_proj = [&](size_t gi) { return scratch.events[2 * gi]; };
+  auto ev_adam = [&](size_t gi) { return scratch.events[2 * gi + 1]; };
+  for (size_t gi = 0; gi < ng; ++gi) {
+    GALORE_TRY(launch_proj(gi, st));
+    GALORE_CUDA_TRY(cudaEventRecord(ev_proj(gi), st));
+    GALORE_CUDA_TRY(cudaStreamWaitEvent(scratch.aux, ev_proj(gi), 0));
+    GALORE_TRY(launch_adam(gi, scratch.aux));
+    GALORE_CUDA_TRY(cudaEventRecord(ev_adam(gi), scratch.aux));
+    if (gi > 0) {
+      GALORE_CUDA_TRY(cudaStreamWaitEvent(st, ev_adam(gi - 1), 0));
+      GALORE_TRY(launch_back(gi - 1, st));
+    }
+  }
+  GALORE_CUDA_TRY(cudaStreamWaitEvent(st, ev_adam(ng - 1), 0));
+  GALORE_TRY(launch_back(ng - 1, st));
   return worst;
 }
 
