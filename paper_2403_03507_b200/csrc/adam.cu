@@ -370,55 +370,87 @@ __device__ __forceinline__ void block_max2_256(float& x, float& y, float* red /*
 }
 
 // Full block of a layer whose R and N buffers have the state's own row pitch: every array is
-// addressed as base pointer + constant offset, no bounds checks.
+// addressed as base pointer + constant offset, no bounds checks, and each thread owns runs of four
+// consecutive elements (one 16-byte load of R, one 4-byte load / store per code array, one 8- or
+// 16-byte store of N per run).  Run j of thread t starts at element 1024 j + 4 t of the block.
+template <typename TN>
+__device__ __forceinline__ void store_n4(TN* dst, float a, float b, float c, float d);
+template <>
+__device__ __forceinline__ void store_n4<__nv_bfloat16>(__nv_bfloat16* dst, float a, float b, float c, float d) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  uint2 v;
+  v.x = *reinterpret_cast<uint32_t*>(&lo);
+  v.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(dst) = v;
+}
+template <>
+__device__ __forceinline__ void store_n4<float>(float* dst, float a, float b, float c, float d) {
+  *reinterpret_cast<float4*>(dst) = make_float4(a, b, c, d);
+}
+
 template <typename TN, int EPT>
 __device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q8Tables& t) {
+  static_assert(EPT % 4 == 0, "runs of four elements");
+  constexpr int RUNS = EPT / 4;
   const AdamParams p = a.p;
-  const int base = blk * (EPT * 256) + threadIdx.x;
+  const int base = blk * (EPT * 256) + 4 * threadIdx.x;
   const float* __restrict__ R = a.Rpart + base;
   uint8_t* __restrict__ Mc = a.Mc + base;
   uint8_t* __restrict__ Vc = a.Vc + base;
   TN* __restrict__ Nout = (TN*)a.Nout + base;
   const float am_m = a.Mam[blk], am_v = a.Vam[blk];
-  float r[EPT];
-  uint32_t cm[EPT], cv[EPT];
+  float4 r[RUNS];
+  uint32_t cm[RUNS], cv[RUNS];
 #pragma unroll
-  for (int e = 0; e < EPT; ++e) {
-    r[e] = R[e * 256];
-    cm[e] = Mc[e * 256];
-    cv[e] = Vc[e * 256];
+  for (int j = 0; j < RUNS; ++j) {
+    r[j] = *reinterpret_cast<const float4*>(R + j * 1024);
+    cm[j] = *reinterpret_cast<const uint32_t*>(Mc + j * 1024);
+    cv[j] = *reinterpret_cast<const uint32_t*>(Vc + j * 1024);
   }
   for (int s = 1; s < a.splits; ++s) {
     const float* __restrict__ part = R + (int64_t)s * a.split_stride;
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) r[e] += part[e * 256];
+    for (int j = 0; j < RUNS; ++j) {
+      const float4 q = *reinterpret_cast<const float4*>(part + j * 1024);
+      r[j].x += q.x; r[j].y += q.y; r[j].z += q.z; r[j].w += q.w;
+    }
   }
   float m[EPT], v[EPT];
   float mx_m = 0.f, mx_v = 0.f, poison = 0.f;
 #pragma unroll
-  for (int e = 0; e < EPT; ++e) {
-    poison = fmaf(r[e], 0.f, poison);              // stays 0 unless some r is inf or nan
-    m[e] = p.b1 * (t.code_s[cm[e]] * am_m) + p.omb1 * r[e];
-    v[e] = p.b2 * (t.code_u[cv[e]] * am_v) + p.omb2 * (r[e] * r[e]);
-    Nout[e * 256] = cvt<TN>(adam_normalised(m[e], v[e], p));
-    mx_m = fmaxf(mx_m, fabsf(m[e]));
-    mx_v = fmaxf(mx_v, v[e]);
+  for (int j = 0; j < RUNS; ++j) {
+    const float rr[4] = {r[j].x, r[j].y, r[j].z, r[j].w};
+    float nn[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int e = 4 * j + k;
+      poison = fmaf(rr[k], 0.f, poison);             // stays 0 unless some r is inf or nan
+      m[e] = p.b1 * (t.code_s[(cm[j] >> (8 * k)) & 0xffu] * am_m) + p.omb1 * rr[k];
+      v[e] = p.b2 * (t.code_u[(cv[j] >> (8 * k)) & 0xffu] * am_v) + p.omb2 * (rr[k] * rr[k]);
+      nn[k] = adam_normalised(m[e], v[e], p);
+      mx_m = fmaxf(mx_m, fabsf(m[e]));
+      mx_v = fmaxf(mx_v, v[e]);
+    }
+    store_n4<TN>(Nout + j * 1024, nn[0], nn[1], nn[2], nn[3]);
   }
   block_max2_256(mx_m, mx_v, t.red);
   const float inv_m = 1.0f / mx_m, inv_v = 1.0f / mx_v;
-  if (mx_m == 0.f) {
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) Mc[e * 256] = (uint8_t)127;
-  } else {
+  for (int j = 0; j < RUNS; ++j) {
+    uint32_t pm = 0x7f7f7f7fu, pv = 0u;              // codes of the value 0
+    if (mx_m != 0.f) {
+      pm = 0u;
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) Mc[e * 256] = (uint8_t)q8_encode_block<true>(m[e], mx_m, inv_m, t.lut_s, t.pair_s, t.mid_s);
-  }
-  if (mx_v == 0.f) {
+      for (int k = 0; k < 4; ++k)
+        pm |= (uint32_t)q8_encode_block<true>(m[4 * j + k], mx_m, inv_m, t.lut_s, t.pair_s, t.mid_s) << (8 * k);
+    }
+    if (mx_v != 0.f) {
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) Vc[e * 256] = (uint8_t)0;
-  } else {
-#pragma unroll
-    for (int e = 0; e < EPT; ++e) Vc[e * 256] = (uint8_t)q8_encode_block<false>(v[e], mx_v, inv_v, t.lut_u, t.pair_u, t.mid_u);
+      for (int k = 0; k < 4; ++k)
+        pv |= (uint32_t)q8_encode_block<false>(v[4 * j + k], mx_v, inv_v, t.lut_u, t.pair_u, t.mid_u) << (8 * k);
+    }
+    *reinterpret_cast<uint32_t*>(Mc + j * 1024) = pm;
+    *reinterpret_cast<uint32_t*>(Vc + j * 1024) = pv;
   }
   if (threadIdx.x == 0) {
     a.Mam[blk] = mx_m;
@@ -451,9 +483,14 @@ __global__ void __launch_bounds__(256, 4) adam_q8_kernel(const __grid_constant__
     const AdamItem& a = g.item[it];
     const bool packed = (a.r_ld == a.cols && a.n_ld == a.cols);
     const bool full = (blk + 1) * (EPT * 256) <= a.nel;
-    const bool bad = (packed && full) ? adam_q8_block_full<TN, EPT>(a, blk, t)
-                     : packed         ? adam_q8_block<TN, EPT, true>(a, blk, t)
-                                      : adam_q8_block<TN, EPT, false>(a, blk, t);
+    bool bad;
+    if constexpr (EPT % 4 == 0) {
+      bad = (packed && full && a.aligned16) ? adam_q8_block_full<TN, EPT>(a, blk, t)
+            : packed                        ? adam_q8_block<TN, EPT, true>(a, blk, t)
+                                            : adam_q8_block<TN, EPT, false>(a, blk, t);
+    } else {
+      bad = packed ? adam_q8_block<TN, EPT, true>(a, blk, t) : adam_q8_block<TN, EPT, false>(a, blk, t);
+    }
     if (__syncthreads_or(bad)) bad_item = it;
   }
   if (bad_item >= 0 && threadIdx.x == 0) atomicOr(g.item[bad_item].status, GALORE_DEV_NONFINITE);
@@ -550,6 +587,8 @@ galore_status_t adam_group_add(AdamGroup& g, const AdamItem& item, int32_t state
   const int64_t rows = ceil_div(a.nel, a.cols);
   if (rows * std::max(a.r_ld, a.n_ld) >= (int64_t)1 << 31) return GALORE_ERR_SHAPE;
   const int per_block = state_fmt == GALORE_STATE_F32 ? 2048 : q_block;
+  a.aligned16 = ((((uintptr_t)a.Rpart | (uintptr_t)a.Nout | (uintptr_t)a.Mc | (uintptr_t)a.Vc) & 15) == 0 &&
+                 (a.split_stride % 4) == 0) ? 1 : 0;
   const int i = g.count++;
   g.item[i] = a;
   g.block_end[i] = (i > 0 ? g.block_end[i - 1] : 0) + (int)ceil_div(a.nel, per_block);

@@ -35,6 +35,7 @@ struct AdamItem {
   float *Mam, *Vam;        // one absmax per quantisation block
   void* Nout;              // normalised update (fp32 or bf16)
   int cols, r_ld, n_ld;    // state row length and the row pitches of Rpart / Nout (cols == 0: packed)
+  int aligned16;           // set by adam_group_add: all arrays allow 16-byte vector accesses
   AdamParams p;
   int32_t* status;
 };
