@@ -66,6 +66,23 @@ def p_dtype_of(w):
     return "bf16" if w.g_dtype == "bf16" else "f32"
 
 
+# DRAM bytes per parameter moved by the two tcgen05 launches of a step (projection + back-projection),
+# from the ncu capture summarised in profiles/gemm_tc_and_adam_single_4096x11008_r1024.md (one
+# 4096 x 11008 matrix, r = 1024: 355 MB for 45.09 M parameters).  Traffic grows with the parameters a
+# launch covers; set to None whenever those kernels change after the capture.
+GEMM_DRAM_BYTES_PER_PARAM = 7.88
+
+
+def max_over_ranks(value: float, dist, device) -> float:
+    """The slowest rank's time: every multi-GPU number is a maximum over ranks."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -183,7 +200,9 @@ def main():
     ap.add_argument("--projector", default="refresh", choices=["refresh", "random"],
                     help="refresh: one real refresh per distinct shape (timed, reported); random: a random orthonormal "
                          "projector (step timing does not depend on P's values; for short profiling runs)")
-    ap.add_argument("--extra-workloads", default="", help="comma-separated workloads also timed (device-resident only)")
+    ap.add_argument("--extra-workloads", default="llama_1b_q8,llama_1b_f32",
+                    help="comma-separated workloads also timed, device-resident only, reported under other_workloads "
+                         "(only with the default workload; empty string to skip)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else max(args.warmup, 0)
 
@@ -213,7 +232,8 @@ def main():
     res = time_workload(w, args, dev, dist, world, rank, full=True)
     if rank == 0:
         extras = []
-        for name in [x for x in args.extra_workloads.split(",") if x]:
+        names = [x for x in args.extra_workloads.split(",") if x] if args.workload == "llama_7b_q8" and world == 1 else []
+        for name in names:
             extras.append(time_workload(wl.WORKLOADS[name], args, dev, None, 1, 0, full=False))
         if extras:
             res["other_workloads"] = extras
@@ -318,11 +338,7 @@ def time_workload(w, args, dev, dist, world, rank, full):
     barrier()
     launches = gb.galore_launch_count() - launches0
     clocks = sampler.stop()
-    ms_total = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(e0.elapsed_time(e1), dist, dev)
     ms_step = ms_total / args.steps
     value = world * w.params / (ms_step * 1e-3)
 
@@ -344,7 +360,10 @@ def time_workload(w, args, dev, dist, world, rank, full):
     achieved_tflops = (flops_alg * prof_steps) / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
     if uses_tc:
         roof = {"bound": "tensor", "achieved": achieved_tflops, "peak": tc_peak, "unit": "TFLOP/s",
-                "frac": achieved_tflops / tc_peak if achieved_tflops else None, "traffic": None,
+                "frac": achieved_tflops / tc_peak if achieved_tflops else None,
+                "traffic": (GEMM_DRAM_BYTES_PER_PARAM * w.params * prof_steps / gemm_launches
+                            if GEMM_DRAM_BYTES_PER_PARAM and gemm_launches and w.rank == 1024 else None),
+                "traffic_unit": "bytes per launch, scaled from a one-matrix ncu capture by parameters covered",
                 "peak_source": peaks["source"] + " (sustained bf16 GEMM)"}
     else:
         roof = {"bound": "alu", "achieved": achieved_tflops, "peak": FP32_FMA_TFLOPS, "unit": "TFLOP/s",
@@ -399,11 +418,7 @@ def time_workload(w, args, dev, dist, world, rank, full):
             e2e_step()
         b.record(stream)
         barrier()
-        ms = a.elapsed_time(b) / e2e_steps
-        if dist is not None:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(a.elapsed_time(b) / e2e_steps, dist, dev)
         out["e2e"] = {"value": world * w.params / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                       "d2h_bytes_per_step": d2h, "ms_per_step": ms, "steps": e2e_steps,
                       "host_buffers": "one pinned W and G per distinct shape, reused by the layers of that shape"}
