@@ -926,6 +926,33 @@ galore_status_t tensor_group_add_back(TensorGroup* t, const TensorPlan* plan, co
   return GALORE_OK;
 }
 
+// A plain GEMM problem for the group: C (M x N, fp32, leading dimension ldc) = op(A) op(B), bf16
+// operands.  a_mn = 1: A is stored K rows x M contiguous, 0: M rows x K contiguous; b_mn likewise
+// (K x N contiguous resp. N x K contiguous).  All problems of a group must have M on the same side
+// of 256 (they share the tile shape).
+galore_status_t tensor_group_add_gemm(TensorGroup* t, const void* A, int64_t lda, int a_mn, const void* B, int64_t ldb,
+                                      int b_mn, int M, int N, int K, float* C, int64_t ldc, int32_t* status) {
+  if (t->g.count >= kMaxGroup) return GALORE_ERR_BUFFER_TOO_SMALL;
+  const int ctas = M >= 2 * kBM ? 2 : 1;
+  TcParams p = {};
+  p.status = status;
+  p.part = C;
+  p.ld_part = ldc;
+  p.split_stride = 0;
+  p.vec32 = (((uintptr_t)C & 31) == 0 && (ldc % 8) == 0) ? 1 : 0;
+  p.a_mn = a_mn ? 1 : 0;
+  p.b_mn = b_mn ? 1 : 0;
+  p.m_fast = 1;
+  fill_tiles(p, M, N, K, 1, ctas);
+  CUtensorMap ma, mb;
+  if (a_mn) GALORE_TRY(make_map(&ma, A, K, M, lda, 64));
+  else GALORE_TRY(make_map(&ma, A, M, K, lda, kBM));
+  if (b_mn) GALORE_TRY(make_map(&mb, B, K, N, ldb, 64));
+  else GALORE_TRY(make_map(&mb, B, N, K, ldb, kBN / ctas));
+  group_add(t->g, ma, mb, p);
+  return GALORE_OK;
+}
+
 galore_status_t tensor_group_launch_project(TensorGroup* t, cudaStream_t st) {
   if (t->g.count == 0) return GALORE_OK;
   return launch_tc<EPI_PARTIAL, float>(t->g, st);

@@ -53,6 +53,10 @@ galore_status_t tensor_group_add_project(TensorGroup* t, const TensorPlan* plan,
 galore_status_t tensor_group_add_back(TensorGroup* t, const TensorPlan* plan, const galore_config_t& cfg, bool left,
                                       const void* Nbuf, int64_t ld_n, void* W, int64_t ldw, float scale,
                                       int32_t* status);
+// a plain GEMM: C (M x N fp32, ldc) = op(A) op(B), bf16 operands; *_mn = 1 when the operand is stored
+// with M (resp. N) contiguous, 0 when K is contiguous.  Launch with tensor_group_launch_project.
+galore_status_t tensor_group_add_gemm(TensorGroup* t, const void* A, int64_t lda, int a_mn, const void* B, int64_t ldb,
+                                      int b_mn, int M, int N, int K, float* C, int64_t ldc, int32_t* status);
 galore_status_t tensor_group_launch_project(TensorGroup* t, cudaStream_t st);
 galore_status_t tensor_group_launch_back(TensorGroup* t, int32_t w_dtype, cudaStream_t st);
 
