@@ -113,6 +113,10 @@ typedef struct {
   double sigma_r;            /* sqrt of the r-th Ritz value */
   double sigma_next;         /* sqrt of the (r+1)-th Ritz value, 0 if block == rank */
   double sigma_1;
+  double ms_total;           /* wall time of the refresh, with its parts: */
+  double ms_power;           /* power steps and their orthonormalisations */
+  double ms_ritz;            /* final orthonormalisation, fp64 products, sorting, P = Y S (without the eigen-solve) */
+  double ms_jacobi;          /* Jacobi eigen-solves */
 } galore_refresh_info_t;
 
 /* Sizes of the two caller-allocated device buffers for one layer.

@@ -43,6 +43,7 @@ class RefreshInfo(C.Structure):
         ("iterations", C.c_int32), ("block", C.c_int32), ("jacobi_sweeps", C.c_int32), ("converged", C.c_int32),
         ("predicted_error", C.c_double), ("residual", C.c_double), ("sigma_r", C.c_double),
         ("sigma_next", C.c_double), ("sigma_1", C.c_double),
+        ("ms_total", C.c_double), ("ms_power", C.c_double), ("ms_ritz", C.c_double), ("ms_jacobi", C.c_double),
     ]
 
     def as_dict(self):

@@ -270,6 +270,7 @@ galore_status_t do_refresh(galore_layer* l, const void* G, int64_t ldg, cudaStre
   pr.tol = l->cfg.refresh_tol > 0.f ? (double)l->cfg.refresh_tol : 1e-4;
   pr.max_iters = l->cfg.refresh_max_iters > 0 ? l->cfg.refresh_max_iters : 64;
   pr.first_iters = 6;
+  pr.use_tensor = l->tensor_path;
   galore_status_t s = refresh_projector(pr, l->refresh_ws, l->status, info, st);
   if (s >= 0) l->has_projector = true;
   return s;

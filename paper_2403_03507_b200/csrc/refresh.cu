@@ -25,9 +25,11 @@
 #include <math.h>
 
 #include <algorithm>
+#include <chrono>
 #include <vector>
 
 #include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
 
 namespace galore {
 
@@ -104,6 +106,77 @@ __global__ void __launch_bounds__(256) shift_kernel(float* __restrict__ Ynew, co
   const float delta = fmaxf((float)(1e-4 * sqrt(s / (double)cols)), 1e-30f);
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
     Ynew[i] = fmaf(delta, Yold[i], Ynew[i]);
+}
+
+// ---- helpers of the tensor-core power step -----------------------------------------------------
+// A value x is carried to the tensor cores as two bf16 numbers, hi = bf16(x) and lo = bf16(x - hi):
+// products with exactly representable bf16 gradients then keep about 16 significant bits.
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+  hi = __float2bfloat16_rn(x);
+  lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+// out = x0 + x1 (+ x2); optionally stored as fp32 and always as a hi/lo pair
+__global__ void sum_split_kernel(const float* __restrict__ x0, const float* __restrict__ x1, const float* __restrict__ x2,
+                                 float* __restrict__ out, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                 int64_t count) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x) {
+    float v = x0[i] + x1[i];
+    if (x2) v += x2[i];
+    if (out) out[i] = v;
+    split_bf16(v, hi[i], lo[i]);
+  }
+}
+
+// x0 += x1, and this CTA's share of the sum of squares of the result (fixed grid)
+__global__ void __launch_bounds__(256) add_sumsq_kernel(float* __restrict__ x0, const float* __restrict__ x1, int64_t count,
+                                                        double* __restrict__ part) {
+  __shared__ double red[8];
+  double s = 0.0;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x) {
+    const float v = x0[i] + x1[i];
+    x0[i] = v;
+    s += (double)v * v;
+  }
+  s = block_sum_256(s, red);
+  if (threadIdx.x == 0) part[blockIdx.x] = s;
+}
+
+// Ynew += delta * Yold, then the hi/lo pair of Ynew.  delta = 1e-2 x rms column norm here (1e-4 on
+// the fp32 path): the pair carries about 16 bits, so directions kept alive only by the shift must
+// stay well above 2^-16 of the dominant ones for the Gram matrix to remain positive definite.
+__global__ void __launch_bounds__(256) shift_split_kernel(float* __restrict__ Ynew, const float* __restrict__ Yold,
+                                                          int64_t count, int cols, const double* __restrict__ part,
+                                                          __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  __shared__ double red[8];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < kSumsqBlocks; i += 256) s += part[i];
+  s = block_sum_256(s, red);
+  const float delta = fmaxf((float)(1e-2 * sqrt(s / (double)cols)), 1e-30f);
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x) {
+    const float v = fmaf(delta, Yold[i], Ynew[i]);
+    Ynew[i] = v;
+    split_bf16(v, hi[i], lo[i]);
+  }
+}
+
+// C (fp64) = g0 + g1 + g2 : the three bf16-pair products that make up a Gram matrix
+__global__ void gram_sum_kernel(const float* __restrict__ g0, const float* __restrict__ g1, const float* __restrict__ g2,
+                                double* __restrict__ C, int64_t count) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+    C[i] = (double)g0[i] + (double)g1[i] + (double)g2[i];
+}
+
+__global__ void split_kernel(const float* __restrict__ x, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                             int64_t count) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+    split_bf16(x[i], hi[i], lo[i]);
+}
+
+__global__ void split_double_kernel(const double* __restrict__ x, __nv_bfloat16* __restrict__ hi,
+                                    __nv_bfloat16* __restrict__ lo, int64_t count) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+    split_bf16((float)x[i], hi[i], lo[i]);
 }
 
 // ---- Cholesky of one diagonal block (nb <= 64) and the inverse of its factor ----
@@ -280,6 +353,11 @@ struct RefreshBuffers {
   double* scal;   // 4 scalars
   double* part;   // kSumsqBlocks partial sums
   int* counter;   // 1
+  // tensor-core power steps
+  float* Yc;                 // d x b, third fp32 block
+  __nv_bfloat16 *Yhi, *Ylo;  // d x b
+  __nv_bfloat16 *Zhi, *Zlo;  // L x b
+  __nv_bfloat16 *Thi, *Tlo;  // b x b, inverse Cholesky factor
 };
 
 static size_t carve(char*& p, size_t bytes) {
@@ -301,6 +379,8 @@ size_t refresh_workspace_bytes(int64_t d, int64_t L, int r, int b) {
   t += align_up((size_t)b * 8, 256) * 2;
   t += align_up((size_t)b * 4, 256);
   t += 256 * 2 + 8 * 1024;
+  t += align_up((size_t)d * b * 4, 256) + 2 * align_up((size_t)d * b * 2, 256) + 2 * align_up((size_t)L * b * 2, 256) +
+       2 * align_up((size_t)b * b * 2, 256);
   return t;
 }
 
@@ -324,6 +404,13 @@ static RefreshBuffers layout(void* base, int64_t d, int64_t L, int r, int b) {
   w.scal = (double*)p; carve(p, 256);
   w.part = (double*)p; carve(p, 8 * 1024);
   w.counter = (int*)p; carve(p, 256);
+  w.Yc = (float*)p; carve(p, (size_t)d * b * 4);
+  w.Yhi = (__nv_bfloat16*)p; carve(p, (size_t)d * b * 2);
+  w.Ylo = (__nv_bfloat16*)p; carve(p, (size_t)d * b * 2);
+  w.Zhi = (__nv_bfloat16*)p; carve(p, (size_t)L * b * 2);
+  w.Zlo = (__nv_bfloat16*)p; carve(p, (size_t)L * b * 2);
+  w.Thi = (__nv_bfloat16*)p; carve(p, (size_t)b * b * 2);
+  w.Tlo = (__nv_bfloat16*)p; carve(p, (size_t)b * b * 2);
   return w;
 }
 
@@ -381,6 +468,76 @@ static galore_status_t orthonormalise(TY* Y, int64_t d, int b, const RefreshBuff
   return cholesky_solve(Y, d, b, w.C, w, status, st);
 }
 
+// ---- power step on the tensor cores -------------------------------------------------------------
+// The block Y lives as an fp32 master (one of three d x b buffers) plus its bf16 hi/lo pair.  Every
+// product below is a tcgen05 GEMM on bf16 operands with fp32 output; a product with a hi/lo operand
+// is two (or three) problems of one grouped launch whose outputs are added afterwards.
+
+struct TensorRefresh {
+  TensorGroup* tg;
+  float* F[3];          // fp32 d x b buffers; F[master] holds Y
+  int master;
+  int32_t* status;
+};
+
+// Y <- Y L^-T with L L^T = Y^T Y: CholeskyQR whose two big products run on the tensor cores.
+// In: hi/lo pair of Y valid (the fp32 master itself is not read).  Out: master and pair updated.
+static galore_status_t orth_tensor(TensorRefresh& t, const RefreshBuffers& w, int64_t d, int b, cudaStream_t st) {
+  const int64_t bb = (int64_t)b * b, yb = d * b;
+  float* g0 = (float*)w.H;
+  float* g1 = g0 + bb;
+  float* g2 = (float*)w.Y64;
+  tensor_group_reset(t.tg);   // Gram = (hi + lo)^T (hi + lo) without the lo^T lo term
+  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 1, w.Yhi, b, 1, b, b, (int)d, g0, b, t.status));
+  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 1, w.Ylo, b, 1, b, b, (int)d, g1, b, t.status));
+  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Ylo, b, 1, w.Yhi, b, 1, b, b, (int)d, g2, b, t.status));
+  GALORE_TRY(tensor_group_launch_project(t.tg, st));
+  gram_sum_kernel<<<grid_for(bb), 256, 0, st>>>(g0, g1, g2, w.C, bb);
+  GALORE_LAUNCH_CHECK();
+  // T = L^-T from the blocked Cholesky solve applied to the identity (b x b instead of d x b)
+  set_identity_kernel<<<grid_for(bb), 256, 0, st>>>(w.Vt, b);
+  GALORE_LAUNCH_CHECK();
+  GALORE_TRY(cholesky_solve(w.Vt, (int64_t)b, b, w.C, w, t.status, st));
+  split_double_kernel<<<grid_for(bb), 256, 0, st>>>(w.Vt, w.Thi, w.Tlo, bb);
+  GALORE_LAUNCH_CHECK();
+  const int m = t.master, s1 = (m + 1) % 3, s2 = (m + 2) % 3;
+  tensor_group_reset(t.tg);   // Y T = hi Thi + hi Tlo + lo Thi
+  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 0, w.Thi, b, 1, (int)d, b, b, t.F[m], b, t.status));
+  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 0, w.Tlo, b, 1, (int)d, b, b, t.F[s1], b, t.status));
+  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Ylo, b, 0, w.Thi, b, 1, (int)d, b, b, t.F[s2], b, t.status));
+  GALORE_TRY(tensor_group_launch_project(t.tg, st));
+  sum_split_kernel<<<grid_for(yb), 256, 0, st>>>(t.F[m], t.F[s1], t.F[s2], t.F[m], w.Yhi, w.Ylo, yb);
+  GALORE_LAUNCH_CHECK();
+  return GALORE_OK;
+}
+
+// Z = A^T Y ; Y' = A Z + delta Y ; Y = orth(Y')
+static galore_status_t power_step_tensor(TensorRefresh& t, const RefreshProblem& pr, const RefreshBuffers& w, int64_t d,
+                                         int64_t L, int b, cudaStream_t st) {
+  const int64_t zb = L * b, yb = d * b;
+  float* z0 = (float*)w.Zu;
+  float* z1 = z0 + zb;
+  const int at_mn = pr.left ? 1 : 0;   // A^T as the first operand: G^T (left) is M-contiguous in G, G (right) is K-contiguous
+  const int a_mn = pr.left ? 0 : 1;    // A as the first operand
+  tensor_group_reset(t.tg);
+  GALORE_TRY(tensor_group_add_gemm(t.tg, pr.G, pr.ldg, at_mn, w.Yhi, b, 1, (int)L, b, (int)d, z0, b, t.status));
+  GALORE_TRY(tensor_group_add_gemm(t.tg, pr.G, pr.ldg, at_mn, w.Ylo, b, 1, (int)L, b, (int)d, z1, b, t.status));
+  GALORE_TRY(tensor_group_launch_project(t.tg, st));
+  sum_split_kernel<<<grid_for(zb), 256, 0, st>>>(z0, z1, nullptr, nullptr, w.Zhi, w.Zlo, zb);
+  GALORE_LAUNCH_CHECK();
+  const int m = t.master, s1 = (m + 1) % 3, s2 = (m + 2) % 3;
+  tensor_group_reset(t.tg);
+  GALORE_TRY(tensor_group_add_gemm(t.tg, pr.G, pr.ldg, a_mn, w.Zhi, b, 1, (int)d, b, (int)L, t.F[s1], b, t.status));
+  GALORE_TRY(tensor_group_add_gemm(t.tg, pr.G, pr.ldg, a_mn, w.Zlo, b, 1, (int)d, b, (int)L, t.F[s2], b, t.status));
+  GALORE_TRY(tensor_group_launch_project(t.tg, st));
+  add_sumsq_kernel<<<kSumsqBlocks, 256, 0, st>>>(t.F[s1], t.F[s2], yb, w.part);
+  GALORE_LAUNCH_CHECK();
+  shift_split_kernel<<<grid_for(yb), 256, 0, st>>>(t.F[s1], t.F[m], yb, b, w.part, w.Yhi, w.Ylo);
+  GALORE_LAUNCH_CHECK();
+  t.master = s1;
+  return orth_tensor(t, w, d, b, st);
+}
+
 template <typename TG>
 static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, int32_t* status,
                                      galore_refresh_info_t* info, cudaStream_t st) {
@@ -393,6 +550,14 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
   RefreshBuffers w = layout(workspace, d, L, r, b);
   galore_refresh_info_t local = {};
   local.block = b;
+  // phase clock: host time at points where the stream is synchronised anyway
+  using clk = std::chrono::steady_clock;
+  auto now_synced = [&]() {
+    cudaStreamSynchronize(st);
+    return clk::now();
+  };
+  auto ms_between = [](clk::time_point a, clk::time_point b2) { return std::chrono::duration<double, std::milli>(b2 - a).count(); };
+  const clk::time_point t_begin = now_synced();
 
   float* Y = w.Ya;
   float* Yn = w.Yb;
@@ -401,10 +566,29 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
   std::vector<double> theta(b);
   const bool full_space = (b == d);
 
+  // tensor cores carry the power steps when the gradient is bf16 and everything is TMA-addressable
+  const bool tensor = pr.use_tensor && !full_space && sizeof(TG) == 2 && (b % 8) == 0 && (pr.ldg % 8) == 0 &&
+                      (((uintptr_t)pr.G) & 15) == 0;
+  TensorRefresh tr = {};
+  struct GroupGuard {
+    TensorGroup* g;
+    ~GroupGuard() { tensor_group_free(g); }
+  } guard{nullptr};
   if (!full_space) {
     fill_normal_kernel<<<grid_for(yb), 256, 0, st>>>(Y, yb, pr.seed);
     GALORE_LAUNCH_CHECK();
-    GALORE_TRY(orthonormalise(Y, d, b, w, status, st));
+    if (tensor) {
+      guard.g = tr.tg = tensor_group_new();
+      if (!tr.tg) return GALORE_ERR_INVALID_ARG;
+      tr.F[0] = w.Ya; tr.F[1] = w.Yb; tr.F[2] = w.Yc;
+      tr.master = 0;
+      tr.status = status;
+      split_kernel<<<grid_for(yb), 256, 0, st>>>(Y, w.Yhi, w.Ylo, yb);
+      GALORE_LAUNCH_CHECK();
+      GALORE_TRY(orth_tensor(tr, w, d, b, st));
+    } else {
+      GALORE_TRY(orthonormalise(Y, d, b, w, status, st));
+    }
   }
   int q_target = full_space ? 0 : std::min(pr.max_iters, std::max(1, pr.first_iters));
   double predicted = 0.0;
@@ -412,6 +596,14 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
 
   for (;;) {
     // ---- power steps ---------------------------------------------------------
+    if (tensor && q_done > 0 && q_done < q_target) {   // the Rayleigh-Ritz pass re-orthonormalised the master in place
+      split_kernel<<<grid_for(yb), 256, 0, st>>>(Y, w.Yhi, w.Ylo, yb);
+      GALORE_LAUNCH_CHECK();
+    }
+    for (; tensor && q_done < q_target; ++q_done) {
+      GALORE_TRY(power_step_tensor(tr, pr, w, d, L, b, st));
+      Y = tr.F[tr.master];
+    }
     for (; q_done < q_target; ++q_done) {
       float* Z = (float*)w.Zu;
       {  // Z = A^T Y   (L x b)
@@ -430,6 +622,8 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
       GALORE_TRY(orthonormalise(Y, d, b, w, status, st));
     }
     // ---- Rayleigh-Ritz in fp64 --------------------------------------------------
+    const clk::time_point t_rr = now_synced();
+    local.ms_power = ms_between(t_begin, t_rr) - local.ms_ritz - local.ms_jacobi;
     if (full_space) {
       set_identity_kernel<<<grid_for(yb), 256, 0, st>>>(w.Y64, (int)d);
       GALORE_LAUNCH_CHECK();
@@ -448,6 +642,7 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
     set_identity_kernel<<<grid_for((int64_t)b * b), 256, 0, st>>>(w.Vt, b);
     GALORE_LAUNCH_CHECK();
     const int np = b + (b & 1);
+    const clk::time_point t_jac = now_synced();
     int sweeps = 0;
     for (; sweeps < 40 && np > 1; ++sweeps) {
       GALORE_CUDA_TRY(cudaMemsetAsync(w.counter, 0, sizeof(int), st));
@@ -461,6 +656,9 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
       if (rot == 0) { ++sweeps; break; }
     }
     local.jacobi_sweeps = sweeps;
+    const clk::time_point t_jac_end = now_synced();
+    local.ms_jacobi += ms_between(t_jac, t_jac_end);
+    local.ms_ritz += ms_between(t_rr, t_jac);
     row_norm_kernel<<<b, 256, 0, st>>>(w.H, b, w.lam);
     GALORE_LAUNCH_CHECK();
     rank_desc_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(w.lam, b, w.theta, w.order);
@@ -512,6 +710,8 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
     GALORE_CUDA_TRY(cudaStreamSynchronize(st));
     local.residual = theta[0] > 0.0 ? sqrt(sc[1]) / (theta[0] * sqrt((double)r)) : 0.0;
   }
+  local.ms_total = ms_between(t_begin, now_synced());
+  local.ms_ritz = local.ms_total - local.ms_power - local.ms_jacobi;
   local.iterations = q_done;
   local.converged = converged ? 1 : 0;
   local.predicted_error = predicted;

@@ -19,6 +19,7 @@ struct RefreshProblem {
   double tol;
   int max_iters;
   int first_iters;      // power steps before the first Rayleigh-Ritz
+  bool use_tensor;      // power steps on the tensor cores when G is bf16 and TMA-addressable
 };
 
 // d = rows of the projector, L = the other dimension of G

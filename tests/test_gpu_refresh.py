@@ -92,3 +92,50 @@ def test_same_seed_same_projector():
     _, _, P1, _ = _refresh(G, 12, seed=7)
     _, _, P2, _ = _refresh(G, 12, seed=7)
     assert np.array_equal(P1, P2)
+
+
+# ---- power steps on the tensor cores (bf16 gradient and projector) -----------------------------------
+
+def _refresh_tc(G, r, **kw):
+    m, n = G.shape
+    cfg = gb.make_config(m, n, r, w_dtype="bf16", g_dtype="bf16", auto_refresh=False, **kw)
+    layer = gb.Layer(cfg)
+    assert layer.uses_tensor_path
+    ld = (n + 7) // 8 * 8
+    st, info = layer.galore_refresh_projector(to_dev(G, "bf16", ld))
+    P = to_host(layer.get_projector())
+    assert layer.device_status() == 0
+    return st, info.as_dict(), P
+
+
+@pytest.mark.parametrize("m,n,r", [(512, 1376, 128), (1376, 512, 128), (768, 2048, 256), (300, 1001, 72)])
+def test_tensor_core_refresh_noise_dominated(m, n, r):
+    G = wl.make_gradient(m, n, wl.sub_seed(wl.BASE_SEED, 1), 1.0, 0.01, "bf16")
+    st, info, P = _refresh_tc(G, r)
+    side = "left" if m <= n else "right"
+    P_orc, S = go.top_r_projector(G, r, side)
+    P_orc_b = wl.round_to(P_orc, "bf16")      # the stored projector is bf16: compare with the same rounding applied
+    angle = go.largest_principal_angle(P_orc, P)
+    floor = go.largest_principal_angle(P_orc, np.linalg.qr(P_orc_b)[0])
+    print(f"{m}x{n} r={r}: angle {angle:.2e} (bf16 storage alone gives {floor:.2e}), {info}")
+    assert st == gb.OK and info["converged"] == 1
+    # bf16 storage of P limits the angle of the *stored* basis; the iteration itself must be far below 1e-3
+    assert angle < max(ANGLE_TOL, 3 * floor)
+    assert info["residual"] < 1e-4
+    assert abs(info["sigma_r"] - S[r - 1]) < 1e-4 * S[0]
+
+
+def test_tensor_core_refresh_gapped_and_low_rank():
+    m, n, r = 384, 896, 32
+    k = min(m, n)
+    spectrum = np.concatenate([np.linspace(10, 5, r), np.linspace(0.5, 0.01, k - r)])
+    G, U, V = wl.make_planted(m, n, seed=5, spectrum=spectrum, dtype="bf16")
+    st, info, P = _refresh_tc(G, r)
+    P_orc, S = go.top_r_projector(G, r, "left")
+    assert st == gb.OK
+    assert go.largest_principal_angle(P_orc, P) < 5e-3          # bf16 storage of P: about 2e-3
+    assert abs(info["sigma_1"] - S[0]) < 1e-4 * S[0]
+    # rank(G) = r (up to bf16 rounding of G): the iterated block is numerically rank-deficient
+    G2, _, _ = wl.make_planted(m, n, seed=6, spectrum=np.linspace(4, 1, r), dtype="bf16")
+    st, info, P = _refresh_tc(G2, r)
+    assert np.linalg.norm(P @ (P.T @ G2) - G2) / np.linalg.norm(G2) < 2e-2
