@@ -152,12 +152,37 @@ __global__ void __launch_bounds__(256) shift_split_kernel(float* __restrict__ Yn
   double s = 0.0;
   for (int i = threadIdx.x; i < kSumsqBlocks; i += 256) s += part[i];
   s = block_sum_256(s, red);
-  const float delta = fmaxf((float)(1e-2 * sqrt(s / (double)cols)), 1e-30f);
+  const float rms = (float)sqrt(s / (double)cols);
+  const float delta = fmaxf(1e-2f * rms, 1e-30f);
+  const float scale = rms > 1e-30f ? 1.0f / rms : 1.0f;      // keeps magnitudes near 1 when steps are chained
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x) {
-    const float v = fmaf(delta, Yold[i], Ynew[i]);
+    const float v = fmaf(delta, Yold[i], Ynew[i]) * scale;
     Ynew[i] = v;
     split_bf16(v, hi[i], lo[i]);
   }
+}
+
+// Rayleigh quotients of the block: ||z_i||^2 with Z = A^T Y (+ second partial of a hi/lo product).
+// Slice s of kColSlices sums rows s, s + kColSlices, ...; slices are added in order afterwards.
+constexpr int kColSlices = 64;
+__global__ void colsumsq_partial_kernel(const float* __restrict__ z0, const float* __restrict__ z1, int64_t rows, int cols,
+                                        double* __restrict__ part /* kColSlices x cols */) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= cols) return;
+  double s = 0.0;
+  for (int64_t i = blockIdx.y; i < rows; i += kColSlices) {
+    float v = z0[i * cols + c];
+    if (z1) v += z1[i * cols + c];
+    s += (double)v * v;
+  }
+  part[(int64_t)blockIdx.y * cols + c] = s;
+}
+__global__ void colsumsq_final_kernel(const double* __restrict__ part, int cols, double* __restrict__ out) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= cols) return;
+  double s = 0.0;
+  for (int k = 0; k < kColSlices; ++k) s += part[(int64_t)k * cols + c];
+  out[c] = s;
 }
 
 // C (fp64) = g0 + g1 + g2 : the three bf16-pair products that make up a Gram matrix
@@ -513,7 +538,7 @@ static galore_status_t orth_tensor(TensorRefresh& t, const RefreshBuffers& w, in
 
 // Z = A^T Y ; Y' = A Z + delta Y ; Y = orth(Y')
 static galore_status_t power_step_tensor(TensorRefresh& t, const RefreshProblem& pr, const RefreshBuffers& w, int64_t d,
-                                         int64_t L, int b, cudaStream_t st) {
+                                         int64_t L, int b, bool orth, cudaStream_t st) {
   const int64_t zb = L * b, yb = d * b;
   float* z0 = (float*)w.Zu;
   float* z1 = z0 + zb;
@@ -535,7 +560,7 @@ static galore_status_t power_step_tensor(TensorRefresh& t, const RefreshProblem&
   shift_split_kernel<<<grid_for(yb), 256, 0, st>>>(t.F[s1], t.F[m], yb, b, w.part, w.Yhi, w.Ylo);
   GALORE_LAUNCH_CHECK();
   t.master = s1;
-  return orth_tensor(t, w, d, b, st);
+  return orth ? orth_tensor(t, w, d, b, st) : GALORE_OK;
 }
 
 template <typename TG>
@@ -590,36 +615,84 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
       GALORE_TRY(orthonormalise(Y, d, b, w, status, st));
     }
   }
-  int q_target = full_space ? 0 : std::min(pr.max_iters, std::max(1, pr.first_iters));
   double predicted = 0.0;
   bool converged = full_space;
 
+  // one power step, Z = A^T Y ; Y' = A Z + delta Y ; optionally Y = orth(Y')
+  auto one_step = [&](bool orth) -> galore_status_t {
+    if (tensor) {
+      GALORE_TRY(power_step_tensor(tr, pr, w, d, L, b, orth, st));
+      Y = tr.F[tr.master];
+      return GALORE_OK;
+    }
+    float* Z = (float*)w.Zu;
+    {  // Z = A^T Y   (L x b)
+      EpiStore<float, float> epi{Z, b, 0, 1.f, 0.f};
+      GALORE_TRY((launch_gemm_simt<TG, float, float>((int)L, b, (int)d, G, sAl, sAi, Y, b, 1, 1, epi, st)));
+    }
+    {  // Y' = A Z     (d x b)
+      EpiStore<float, float> epi{Yn, b, 0, 1.f, 0.f};
+      GALORE_TRY((launch_gemm_simt<TG, float, float>((int)d, b, (int)L, G, sAi, sAl, Z, b, 1, 1, epi, st)));
+    }
+    sumsq_kernel<<<kSumsqBlocks, 256, 0, st>>>(Yn, yb, w.part);
+    GALORE_LAUNCH_CHECK();
+    shift_kernel<<<grid_for(yb), 256, 0, st>>>(Yn, Y, yb, b, w.part);
+    GALORE_LAUNCH_CHECK();
+    std::swap(Y, Yn);
+    return orthonormalise(Y, d, b, w, status, st);
+  };
+
+  // ---- first steps, then a cheap look at the spectrum ------------------------------------------
+  // After a step from an orthonormal Y, ||z_i||^2 (Z = A^T Y) are the Rayleigh quotients of the
+  // block's columns.  Sorted, they stand in for the Ritz values: enough to size the iteration
+  // (their spread is narrower than the spectrum's, which errs towards more steps) and to decide
+  // how many steps may be chained before the block has to be orthonormalised again.
+  int q_target = 0;
+  int orth_every = 1;
+  if (!full_space) {
+    const int q0 = std::min(pr.max_iters, std::max(1, pr.first_iters));
+    for (; q_done < q0; ++q_done) GALORE_TRY(one_step(true));
+    q_target = q_done;
+    if (b > r && q_done < pr.max_iters) {
+      double* slices = (double*)w.Y64;                      // kColSlices x b doubles, Y64 is idle here
+      const float* z0 = (const float*)w.Zu;
+      const float* z1 = tensor ? z0 + L * b : nullptr;
+      colsumsq_partial_kernel<<<dim3((unsigned)ceil_div(b, 128), kColSlices), 128, 0, st>>>(z0, z1, L, b, slices);
+      GALORE_LAUNCH_CHECK();
+      colsumsq_final_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(slices, b, w.lam);
+      GALORE_LAUNCH_CHECK();
+      rank_desc_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(w.lam, b, w.theta, w.order);
+      GALORE_LAUNCH_CHECK();
+      GALORE_CUDA_TRY(cudaMemcpyAsync(theta.data(), w.theta, sizeof(double) * b, cudaMemcpyDeviceToHost, st));
+      GALORE_CUDA_TRY(cudaStreamSynchronize(st));
+      const double ratio = theta[r - 1] > 0.0 ? theta[b - 1] / theta[r - 1] : 1.0;
+      if (ratio > 0.0 && ratio < 1.0) {
+        const int need = (int)ceil(log(pr.tol) / log(ratio)) + 1;
+        q_target = std::min(pr.max_iters, std::max(need, q_done));
+      } else if (ratio >= 1.0) {
+        q_target = pr.max_iters;
+      }
+      if (tensor && theta[b - 1] > 0.0) {
+        // chained steps multiply the block's condition number by theta_1/theta_b each; the bf16 pair
+        // carries 16 bits and the Gram matrix squares the product, so keep it below about 100
+        const double spread = theta[0] / theta[b - 1];
+        orth_every = spread > 1.0 ? (int)floor(log(100.0) / log(spread)) : 8;
+        orth_every = std::max(1, std::min(orth_every, 8));
+      }
+    }
+  }
+  bool pair_stale = false;
+
   for (;;) {
     // ---- power steps ---------------------------------------------------------
-    if (tensor && q_done > 0 && q_done < q_target) {   // the Rayleigh-Ritz pass re-orthonormalised the master in place
+    if (tensor && pair_stale && q_done < q_target) {   // the Rayleigh-Ritz pass re-orthonormalised the master in place
       split_kernel<<<grid_for(yb), 256, 0, st>>>(Y, w.Yhi, w.Ylo, yb);
       GALORE_LAUNCH_CHECK();
-    }
-    for (; tensor && q_done < q_target; ++q_done) {
-      GALORE_TRY(power_step_tensor(tr, pr, w, d, L, b, st));
-      Y = tr.F[tr.master];
+      pair_stale = false;
     }
     for (; q_done < q_target; ++q_done) {
-      float* Z = (float*)w.Zu;
-      {  // Z = A^T Y   (L x b)
-        EpiStore<float, float> epi{Z, b, 0, 1.f, 0.f};
-        GALORE_TRY((launch_gemm_simt<TG, float, float>((int)L, b, (int)d, G, sAl, sAi, Y, b, 1, 1, epi, st)));
-      }
-      {  // Y' = A Z     (d x b)
-        EpiStore<float, float> epi{Yn, b, 0, 1.f, 0.f};
-        GALORE_TRY((launch_gemm_simt<TG, float, float>((int)d, b, (int)L, G, sAi, sAl, Z, b, 1, 1, epi, st)));
-      }
-      sumsq_kernel<<<kSumsqBlocks, 256, 0, st>>>(Yn, yb, w.part);
-      GALORE_LAUNCH_CHECK();
-      shift_kernel<<<grid_for(yb), 256, 0, st>>>(Yn, Y, yb, b, w.part);
-      GALORE_LAUNCH_CHECK();
-      std::swap(Y, Yn);
-      GALORE_TRY(orthonormalise(Y, d, b, w, status, st));
+      const bool orth = ((q_target - 1 - q_done) % orth_every) == 0;      // the last step always ends orthonormal
+      GALORE_TRY(one_step(orth));
     }
     // ---- Rayleigh-Ritz in fp64 --------------------------------------------------
     const clk::time_point t_rr = now_synced();
@@ -674,6 +747,7 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
       if (!converged && q_done < pr.max_iters && ratio < 1.0 && ratio > 0.0) {
         int need = (int)ceil(log(pr.tol) / log(ratio)) + 2;
         q_target = std::min(pr.max_iters, std::max(need, q_done + 1));
+        pair_stale = true;
         continue;                                              // more power steps, then Rayleigh-Ritz again
       }
     }
