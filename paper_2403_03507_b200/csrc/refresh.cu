@@ -21,6 +21,7 @@
 // decays like (theta_b / theta_r)^q (theta = Ritz values, descending); the
 // iteration stops when that prediction is below the tolerance, or at the cap.
 #include "refresh.cuh"
+#include "eig_jacobi.cuh"
 
 #include <math.h>
 
@@ -207,50 +208,61 @@ __global__ void split_double_kernel(const double* __restrict__ x, __nv_bfloat16*
 // ---- Cholesky of one diagonal block (nb <= 64) and the inverse of its factor ----
 // C: the block inside a row-major matrix with leading dimension ld (lower triangle used and
 // overwritten with L).  Linv: 64 x 64 row-major, lower triangular, zero elsewhere.
-__global__ void __launch_bounds__(256) potf2_inv_kernel(double* __restrict__ C, int ld, int nb, double* __restrict__ Linv,
-                                                        int32_t* __restrict__ status) {
+//
+// Left-looking, one thread per row: at column j row i subtracts its dot product with row j over
+// the columns already done, then divides by the new pivot.  The strict upper triangle of the same
+// shared array then receives Linv^T (entry (k, c) of the inverse sits at [c][k]), so thread c
+// walks its own row while it substitutes forward; the reciprocal pivots live in a side array.
+__global__ void __launch_bounds__(64) potf2_inv_kernel(double* __restrict__ C, int ld, int nb, double* __restrict__ Linv,
+                                                       int32_t* __restrict__ status) {
   __shared__ double L[64][65];
-  const int tid = threadIdx.x;
-  for (int idx = tid; idx < 64 * 64; idx += 256) {
-    int i = idx / 64, j = idx % 64;
-    L[i][j] = (i < nb && j <= i) ? C[(int64_t)i * ld + j] : 0.0;
-    Linv[idx] = 0.0;
-  }
+  __shared__ double rdiag[64];
+  const int i = threadIdx.x;
+  for (int j = 0; j < 64; ++j) L[i][j] = (i < nb && j <= i) ? C[(int64_t)i * ld + j] : 0.0;
   __syncthreads();
   for (int j = 0; j < nb; ++j) {
-    if (tid == 0) {
-      double piv = L[j][j];
-      if (!(piv > 0.0)) {              // not positive definite: keep going with a usable pivot, latch the fact
-        atomicOr(status, GALORE_DEV_CHOLESKY);
-        piv = fabs(piv) + 1e-300;
+    double s0 = L[i][j], s1 = 0.0;
+    if (i >= j) {
+      int k = 0;
+      for (; k + 1 < j; k += 2) {
+        s0 = fma(-L[i][k], L[j][k], s0);
+        s1 = fma(-L[i][k + 1], L[j][k + 1], s1);
       }
-      L[j][j] = sqrt(piv);
+      if (k < j) s0 = fma(-L[i][k], L[j][k], s0);
+      s0 += s1;
+    }
+    if (i == j) {
+      if (!(s0 > 0.0)) {                  // not positive definite: keep going with a usable pivot, latch the fact
+        atomicOr(status, GALORE_DEV_CHOLESKY);
+        s0 = fabs(s0) + 1e-300;
+      }
+      const double piv = sqrt(s0);
+      L[j][j] = piv;
+      rdiag[j] = 1.0 / piv;
     }
     __syncthreads();
-    const double inv = 1.0 / L[j][j];
-    for (int i = j + 1 + tid; i < nb; i += 256) L[i][j] *= inv;
-    __syncthreads();
-    // trailing update of the lower triangle: L[i][k] -= L[i][j] * L[k][j], j < k <= i
-    const int rem = nb - j - 1;
-    for (int idx = tid; idx < rem * rem; idx += 256) {
-      int i = j + 1 + idx / rem, k = j + 1 + idx % rem;
-      if (k <= i) L[i][k] -= L[i][j] * L[k][j];
-    }
-    __syncthreads();
+    if (i > j) L[i][j] = s0 * rdiag[j];
+    __syncthreads();                      // column j is complete before anyone reads it
   }
-  // inverse by forward substitution, one column per thread (L x = e_c); each thread reads back
-  // only its own column of Linv
-  if (tid < nb) {
-    const int c = tid;
-    for (int i = c; i < nb; ++i) {
-      double s = (i == c) ? 1.0 : 0.0;
-      for (int k = c; k < i; ++k) s -= L[i][k] * Linv[k * 64 + c];
-      Linv[i * 64 + c] = s / L[i][i];
+  // inverse by forward substitution, one column per thread: x_i = (e_c - sum_{c<=k<i} L[i][k] x_k) / L[i][i]
+  if (i < nb) {
+    const int c = i;
+    const double xc = rdiag[c];
+    for (int r = c + 1; r < nb; ++r) {
+      double s = -L[r][c] * xc;
+      for (int k = c + 1; k < r; ++k) s = fma(-L[r][k], L[c][k], s);
+      L[c][r] = s * rdiag[r];
     }
   }
-  for (int idx = tid; idx < 64 * 64; idx += 256) {
-    int i = idx / 64, j = idx % 64;
-    if (i < nb && j <= i) C[(int64_t)i * ld + j] = L[i][j];
+  __syncthreads();
+  for (int j = 0; j < 64; ++j) {
+    // row i of the outputs: L below the diagonal, Linv(i, j) = [j][i] of the shared array for j < i
+    double inv = 0.0;
+    if (i < nb && j <= i) {
+      inv = (j == i) ? rdiag[i] : L[j][i];
+      C[(int64_t)i * ld + j] = L[i][j];
+    }
+    Linv[i * 64 + j] = inv;
   }
 }
 
@@ -340,6 +352,16 @@ __global__ void gather_rows_kernel(const double* __restrict__ Vt, const int* __r
   for (int j = threadIdx.x; j < b; j += blockDim.x) dst[j] = src[j];
 }
 
+// rows of X = Theta V^T divided by their norms: the eigenvectors themselves
+__global__ void gather_rows_scaled_kernel(const double* __restrict__ X, const double* __restrict__ lam,
+                                          const int* __restrict__ order, int b, double* __restrict__ Vsel) {
+  const int i = order[blockIdx.x];
+  const double* src = X + (int64_t)i * b;
+  const double inv = lam[i] > 0.0 ? 1.0 / lam[i] : 0.0;
+  double* dst = Vsel + (int64_t)blockIdx.x * b;
+  for (int j = threadIdx.x; j < b; j += blockDim.x) dst[j] = src[j] * inv;
+}
+
 // scal[1] += || T2 - P diag(theta) ||_F^2
 __global__ void __launch_bounds__(256) residual_kernel(const double* __restrict__ T2, const double* __restrict__ P,
                                                        const double* __restrict__ theta, int64_t rows, int r,
@@ -378,6 +400,7 @@ struct RefreshBuffers {
   double* scal;   // 4 scalars
   double* part;   // kSumsqBlocks partial sums
   int* counter;   // 1
+  void* jac;      // scratch of the Jacobi eigensolver
   // tensor-core power steps
   float* Yc;                 // d x b, third fp32 block
   __nv_bfloat16 *Yhi, *Ylo;  // d x b
@@ -404,6 +427,7 @@ size_t refresh_workspace_bytes(int64_t d, int64_t L, int r, int b) {
   t += align_up((size_t)b * 8, 256) * 2;
   t += align_up((size_t)b * 4, 256);
   t += 256 * 2 + 8 * 1024;
+  t += align_up(jacobi_scratch_bytes(b), 256);
   t += align_up((size_t)d * b * 4, 256) + 2 * align_up((size_t)d * b * 2, 256) + 2 * align_up((size_t)L * b * 2, 256) +
        2 * align_up((size_t)b * b * 2, 256);
   return t;
@@ -429,6 +453,7 @@ static RefreshBuffers layout(void* base, int64_t d, int64_t L, int r, int b) {
   w.scal = (double*)p; carve(p, 256);
   w.part = (double*)p; carve(p, 8 * 1024);
   w.counter = (int*)p; carve(p, 256);
+  w.jac = (void*)p; carve(p, jacobi_scratch_bytes(b));
   w.Yc = (float*)p; carve(p, (size_t)d * b * 4);
   w.Yhi = (__nv_bfloat16*)p; carve(p, (size_t)d * b * 2);
   w.Ylo = (__nv_bfloat16*)p; carve(p, (size_t)d * b * 2);
@@ -466,7 +491,7 @@ static galore_status_t cholesky_solve(TY* Y, int64_t d, int b, double* C, const 
       EpiResidual<TY> epi{Y, b, w.tmp, 64};
       GALORE_TRY((launch_gemm_simt<TY, double, double>((int)d, nb, 0, Y, b, 1, C, 1, b, 1, epi, st)));
     }
-    potf2_inv_kernel<<<1, 256, 0, st>>>(C + (int64_t)j0 * b + j0, b, nb, w.Linv, status);
+    potf2_inv_kernel<<<1, 64, 0, st>>>(C + (int64_t)j0 * b + j0, b, nb, w.Linv, status);
     GALORE_LAUNCH_CHECK();
     // Y[:, J] = tmp Linv^T
     {
@@ -682,6 +707,7 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
     }
   }
   bool pair_stale = false;
+  bool with_vt = false;
 
   for (;;) {
     // ---- power steps ---------------------------------------------------------
@@ -711,33 +737,29 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
       EpiStore<double, double> epi{Z64, b, 0, 1.0, 0.0};
       GALORE_TRY((launch_gemm_simt<TG, double, double>((int)L, b, (int)d, G, sAl, sAi, w.Y64, b, 1, 1, epi, st)));
     }
-    GALORE_TRY(gram(Z64, L, b, w.H, st));                     // H = Z^T Z
-    set_identity_kernel<<<grid_for((int64_t)b * b), 256, 0, st>>>(w.Vt, b);
-    GALORE_LAUNCH_CHECK();
-    const int np = b + (b & 1);
     const clk::time_point t_jac = now_synced();
-    int sweeps = 0;
-    for (; sweeps < 40 && np > 1; ++sweeps) {
-      GALORE_CUDA_TRY(cudaMemsetAsync(w.counter, 0, sizeof(int), st));
-      for (int round = 0; round < np - 1; ++round) {
-        jacobi_round_kernel<<<np / 2, 256, 0, st>>>(w.H, w.Vt, b, np, round, 1e-13, w.counter);
+    local.ms_ritz += ms_between(t_rr, t_jac);
+    // Eigenvectors are read off the rotated rows Theta V^T; only when wanted eigenvalues are tiny
+    // against the largest (a gradient of rank below r) are the rotations accumulated separately.
+    for (;;) {
+      GALORE_TRY(gram(Z64, L, b, w.H, st));                   // H = Z^T Z
+      if (with_vt) {
+        set_identity_kernel<<<grid_for((int64_t)b * b), 256, 0, st>>>(w.Vt, b);
         GALORE_LAUNCH_CHECK();
       }
-      int rot = 0;
-      GALORE_CUDA_TRY(cudaMemcpyAsync(&rot, w.counter, sizeof(int), cudaMemcpyDeviceToHost, st));
+      int sweeps = 0;
+      GALORE_TRY(jacobi_eigh(w.H, with_vt ? w.Vt : nullptr, b, w.jac, w.counter, 1e-13, 40, &sweeps, st));
+      local.jacobi_sweeps = sweeps;
+      row_norm_kernel<<<b, 256, 0, st>>>(w.H, b, w.lam);
+      GALORE_LAUNCH_CHECK();
+      rank_desc_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(w.lam, b, w.theta, w.order);
+      GALORE_LAUNCH_CHECK();
+      GALORE_CUDA_TRY(cudaMemcpyAsync(theta.data(), w.theta, sizeof(double) * b, cudaMemcpyDeviceToHost, st));
       GALORE_CUDA_TRY(cudaStreamSynchronize(st));
-      if (rot == 0) { ++sweeps; break; }
+      if (with_vt || theta[r - 1] > 1e-8 * theta[0]) break;
+      with_vt = true;
     }
-    local.jacobi_sweeps = sweeps;
-    const clk::time_point t_jac_end = now_synced();
-    local.ms_jacobi += ms_between(t_jac, t_jac_end);
-    local.ms_ritz += ms_between(t_rr, t_jac);
-    row_norm_kernel<<<b, 256, 0, st>>>(w.H, b, w.lam);
-    GALORE_LAUNCH_CHECK();
-    rank_desc_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(w.lam, b, w.theta, w.order);
-    GALORE_LAUNCH_CHECK();
-    GALORE_CUDA_TRY(cudaMemcpyAsync(theta.data(), w.theta, sizeof(double) * b, cudaMemcpyDeviceToHost, st));
-    GALORE_CUDA_TRY(cudaStreamSynchronize(st));
+    local.ms_jacobi += ms_between(t_jac, now_synced());
 
     if (!full_space) {
       const double th_r = theta[r - 1], th_b = theta[b - 1];
@@ -755,7 +777,10 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
   }
 
   // ---- P = Y S[:, top r] ------------------------------------------------------------
-  gather_rows_kernel<<<r, 256, 0, st>>>(w.Vt, w.order, b, w.Vsel);
+  if (with_vt)
+    gather_rows_kernel<<<r, 256, 0, st>>>(w.Vt, w.order, b, w.Vsel);
+  else
+    gather_rows_scaled_kernel<<<r, 256, 0, st>>>(w.H, w.lam, w.order, b, w.Vsel);
   GALORE_LAUNCH_CHECK();
   {
     EpiStore<double, double> epi{w.P64, r, 0, 1.0, 0.0};
