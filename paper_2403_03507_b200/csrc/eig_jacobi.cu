@@ -153,25 +153,38 @@ __global__ void __launch_bounds__(256) jb_sweep_kernel(const double* __restrict_
     return;
   }
   const double* src = part + (int64_t)pair * chunks * (kPairRows * kPairRows);
-  for (int idx = tid; idx < kPairRows * kPairRows; idx += 256) {
-    double s = 0.0;
-    for (int c = 0; c < chunks; ++c) s += src[(int64_t)c * (kPairRows * kPairRows) + idx];
-    A[idx >> 6][idx & 63] = s;
-    Rot[idx >> 6][idx & 63] = ((idx >> 6) == (idx & 63)) ? 1.0 : 0.0;
+  {
+    double sum[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) sum[i] = 0.0;
+    for (int c = 0; c < chunks; ++c) {
+      const double* sc = src + (int64_t)c * (kPairRows * kPairRows);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) sum[i] += sc[tid + 256 * i];
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int idx = tid + 256 * i;
+      A[idx >> 6][idx & 63] = sum[i];
+      Rot[idx >> 6][idx & 63] = ((idx >> 6) == (idx & 63)) ? 1.0 : 0.0;
+    }
   }
   __syncthreads();
   int applied = 0;
-  const int slot = tid >> 3, l8 = tid & 7;
+  const int u = tid >> 3, l8 = tid & 7;
+  const double tol2 = tol * tol;
   for (int rr = 0; rr < kPairRows - 1; ++rr) {
     if (tid < 32) {
       int p = rr_player(tid, rr, kPairRows), q = rr_player(kPairRows - 1 - tid, rr, kPairRows);
       if (p > q) { const int x = p; p = q; q = x; }
       const double app = A[p][p], aqq = A[q][q], apq = A[p][q];
       double c = 1.0, s = 0.0;
-      if (apq != 0.0 && fabs(apq) > tol * sqrt(app * aqq)) {
-        const double zeta = (aqq - app) / (2.0 * apq);
-        const double tt = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
-        c = 1.0 / sqrt(1.0 + tt * tt);
+      if (apq != 0.0 && apq * apq > tol2 * app * aqq) {
+        // tan of the rotation angle: the smaller root of t^2 + 2 zeta t - 1 = 0, zeta = (aqq - app) / (2 apq)
+        const double d = aqq - app, o = 2.0 * apq;
+        const double h = sqrt(d * d + o * o);
+        const double tt = o / (d + (d >= 0.0 ? h : -h));
+        c = rsqrt(1.0 + tt * tt);
         s = c * tt;
         ++applied;
       }
@@ -181,29 +194,31 @@ __global__ void __launch_bounds__(256) jb_sweep_kernel(const double* __restrict_
       pq[tid][1] = q;
     }
     __syncthreads();
-    const double c = cs[slot][0], s = cs[slot][1];
-    const int p = pq[slot][0], q = pq[slot][1];
-    if (s != 0.0) {   // rows p, q of A and of Rot
+    // A <- R A R^T, one 2 x 2 block (rows of slot u, columns of slot v) at a time: blocks are disjoint,
+    // so the row and the column rotation of a block are applied together.  Rot <- R Rot alongside.
+    const double cu = cs[u][0], su = cs[u][1];
+    const int pu = pq[u][0], qu = pq[u][1];
+#pragma unroll
+    for (int vv = 0; vv < 4; ++vv) {
+      const int v = l8 + 8 * vv;
+      const double cv = cs[v][0], sv = cs[v][1];
+      if (su == 0.0 && sv == 0.0) continue;
+      const int pv = pq[v][0], qv = pq[v][1];
+      const double a00 = A[pu][pv], a01 = A[pu][qv], a10 = A[qu][pv], a11 = A[qu][qv];
+      const double r00 = cu * a00 - su * a10, r01 = cu * a01 - su * a11;
+      const double r10 = su * a00 + cu * a10, r11 = su * a01 + cu * a11;
+      A[pu][pv] = cv * r00 - sv * r01;
+      A[pu][qv] = sv * r00 + cv * r01;
+      A[qu][pv] = cv * r10 - sv * r11;
+      A[qu][qv] = sv * r10 + cv * r11;
+    }
+    if (su != 0.0) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const int col = l8 + 8 * i;
-        double x = A[p][col], y = A[q][col];
-        A[p][col] = c * x - s * y;
-        A[q][col] = s * x + c * y;
-        x = Rot[p][col];
-        y = Rot[q][col];
-        Rot[p][col] = c * x - s * y;
-        Rot[q][col] = s * x + c * y;
-      }
-    }
-    __syncthreads();
-    if (s != 0.0) {   // columns p, q of A
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int row = l8 + 8 * i;
-        const double x = A[row][p], y = A[row][q];
-        A[row][p] = c * x - s * y;
-        A[row][q] = s * x + c * y;
+        const double x = Rot[pu][col], y = Rot[qu][col];
+        Rot[pu][col] = cu * x - su * y;
+        Rot[qu][col] = su * x + cu * y;
       }
     }
     __syncthreads();
