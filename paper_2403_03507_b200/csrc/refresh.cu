@@ -22,6 +22,7 @@
 // iteration stops when that prediction is below the tolerance, or at the cap.
 #include "refresh.cuh"
 #include "eig_jacobi.cuh"
+#include "gemm_dmma.cuh"
 
 #include <math.h>
 
@@ -207,76 +208,79 @@ __global__ void split_double_kernel(const double* __restrict__ x, __nv_bfloat16*
 
 // ---- Cholesky of one diagonal block (nb <= 64) and the inverse of its factor ----
 // C: the block inside a row-major matrix with leading dimension ld (lower triangle used and
-// overwritten with L).  Linv: 64 x 64 row-major, lower triangular, zero elsewhere.
+// overwritten with L).  Linv: 64 x 64 row-major, lower triangular, zero elsewhere; rows and
+// columns past nb continue the identity.
 //
-// Left-looking, one thread per row: at column j row i subtracts its dot product with row j over
-// the columns already done, then divides by the new pivot.  The strict upper triangle of the same
-// shared array then receives Linv^T (entry (k, c) of the inverse sits at [c][k]), so thread c
-// walks its own row while it substitutes forward; the reciprocal pivots live in a side array.
+// One thread per row, the row held in registers (every index below is a compile-time constant
+// after unrolling).  Column j: the owner of the pivot publishes 1/sqrt, every row below scales its
+// entry and publishes it, then all rows subtract the rank-1 term from their remaining entries:
+// 63 - j independent FMAs per thread, no dependent chain.  The inverse is formed the same way,
+// column c of L^-1 in the registers of thread c: x_r = s_r / L_rr, then s_i -= L_ir x_r for i > r.
 __global__ void __launch_bounds__(64) potf2_inv_kernel(double* __restrict__ C, int ld, int nb, double* __restrict__ Linv,
                                                        int32_t* __restrict__ status) {
-  __shared__ double L[64][65];
+  __shared__ double Ls[64][65];
+  __shared__ double col[64];
   __shared__ double rdiag[64];
   const int i = threadIdx.x;
-  for (int j = 0; j < 64; ++j) L[i][j] = (i < nb && j <= i) ? C[(int64_t)i * ld + j] : 0.0;
+  for (int r = 0; r < 64; ++r) {      // coalesced read of row r by the threads k <= r
+    double v = (r == i) ? 1.0 : 0.0;
+    if (r < nb && i <= r) v = C[(int64_t)r * ld + i];
+    Ls[r][i] = v;
+  }
   __syncthreads();
-  for (int j = 0; j < nb; ++j) {
-    double s0 = L[i][j], s1 = 0.0;
-    if (i >= j) {
-      int k = 0;
-      for (; k + 1 < j; k += 2) {
-        s0 = fma(-L[i][k], L[j][k], s0);
-        s1 = fma(-L[i][k + 1], L[j][k + 1], s1);
-      }
-      if (k < j) s0 = fma(-L[i][k], L[j][k], s0);
-      s0 += s1;
-    }
+  double a[64];
+#pragma unroll
+  for (int k = 0; k < 64; ++k) a[k] = Ls[i][k];
+  __syncthreads();
+#pragma unroll
+  for (int j = 0; j < 64; ++j) {
     if (i == j) {
-      if (!(s0 > 0.0)) {                  // not positive definite: keep going with a usable pivot, latch the fact
+      double piv = a[j];
+      if (!(piv > 0.0)) {              // not positive definite: keep going with a usable pivot, latch the fact
         atomicOr(status, GALORE_DEV_CHOLESKY);
-        s0 = fabs(s0) + 1e-300;
+        piv = fabs(piv) + 1e-300;
       }
-      const double piv = sqrt(s0);
-      L[j][j] = piv;
-      rdiag[j] = 1.0 / piv;
+      const double sq = sqrt(piv);
+      Ls[j][j] = sq;
+      rdiag[j] = 1.0 / sq;
     }
     __syncthreads();
-    if (i > j) L[i][j] = s0 * rdiag[j];
-    __syncthreads();                      // column j is complete before anyone reads it
-  }
-  // inverse by forward substitution, one column per thread: x_i = (e_c - sum_{c<=k<i} L[i][k] x_k) / L[i][i]
-  if (i < nb) {
-    const int c = i;
-    const double xc = rdiag[c];
-    for (int r = c + 1; r < nb; ++r) {
-      double s = -L[r][c] * xc;
-      for (int k = c + 1; k < r; ++k) s = fma(-L[r][k], L[c][k], s);
-      L[c][r] = s * rdiag[r];
+    double l = 0.0;
+    if (i > j) {
+      l = a[j] * rdiag[j];
+      Ls[i][j] = l;
     }
+    col[i] = l;
+    __syncthreads();
+#pragma unroll
+    for (int k = j + 1; k < 64; ++k) a[k] = fma(-l, col[k], a[k]);
   }
   __syncthreads();
-  for (int j = 0; j < 64; ++j) {
-    // row i of the outputs: L below the diagonal, Linv(i, j) = [j][i] of the shared array for j < i
-    double inv = 0.0;
-    if (i < nb && j <= i) {
-      inv = (j == i) ? rdiag[i] : L[j][i];
-      C[(int64_t)i * ld + j] = L[i][j];
-    }
-    Linv[i * 64 + j] = inv;
+  // column i of L^-1
+#pragma unroll
+  for (int k = 0; k < 64; ++k) a[k] = (k == i) ? 1.0 : 0.0;
+#pragma unroll
+  for (int r = 0; r < 64; ++r) {
+    const double x = a[r] * rdiag[r];
+    a[r] = x;
+#pragma unroll
+    for (int k = r + 1; k < 64; ++k) a[k] = fma(-Ls[k][r], x, a[k]);
   }
+#pragma unroll
+  for (int r = 0; r < 64; ++r) Linv[r * 64 + i] = a[r];
+  for (int r = 0; r < nb; ++r)
+    if (i <= r) C[(int64_t)r * ld + i] = Ls[r][i];
 }
 
-// dst = src - acc   (one panel step of the blocked triangular solve)
-template <typename TS>
-struct EpiResidual {
-  const TS* src;
-  int64_t ldsrc;
-  double* dst;
-  int64_t lddst;
-  __device__ __forceinline__ void operator()(int i, int j, double acc, int) const {
-    dst[(int64_t)i * lddst + j] = cvt<double>(src[(int64_t)i * ldsrc + j]) - acc;
+// diagonal 64 x 64 blocks of T <- the inverses of the diagonal blocks of L (slab p = block p)
+__global__ void place_diag_inverse_kernel(const double* __restrict__ slabs, int b, double* __restrict__ T) {
+  const int p = blockIdx.x, j0 = p * 64;
+  const int nb = min(64, b - j0);
+  for (int idx = threadIdx.x; idx < 64 * 64; idx += blockDim.x) {
+    const int r = idx >> 6, c = idx & 63;
+    if (r < nb && c < nb) T[(int64_t)(j0 + r) * b + j0 + c] = slabs[(int64_t)p * 4096 + idx];
   }
-};
+}
 
 // ---- parallel one-sided Jacobi on a symmetric matrix -------------------------------
 // X starts as H, Vt as the identity.  A rotation of rows (p, q) that makes the
@@ -401,6 +405,8 @@ struct RefreshBuffers {
   double* part;   // kSumsqBlocks partial sums
   int* counter;   // 1
   void* jac;      // scratch of the Jacobi eigensolver
+  double* slabs;  // ceil(b / 64) inverses of 64 x 64 diagonal blocks
+  double* Y64b;   // d x b, second fp64 block
   // tensor-core power steps
   float* Yc;                 // d x b, third fp32 block
   __nv_bfloat16 *Yhi, *Ylo;  // d x b
@@ -428,6 +434,8 @@ size_t refresh_workspace_bytes(int64_t d, int64_t L, int r, int b) {
   t += align_up((size_t)b * 4, 256);
   t += 256 * 2 + 8 * 1024;
   t += align_up(jacobi_scratch_bytes(b), 256);
+  t += align_up((size_t)ceil_div(b, 64) * 4096 * 8, 256);
+  t += align_up((size_t)d * b * 8, 256);
   t += align_up((size_t)d * b * 4, 256) + 2 * align_up((size_t)d * b * 2, 256) + 2 * align_up((size_t)L * b * 2, 256) +
        2 * align_up((size_t)b * b * 2, 256);
   return t;
@@ -454,6 +462,8 @@ static RefreshBuffers layout(void* base, int64_t d, int64_t L, int r, int b) {
   w.part = (double*)p; carve(p, 8 * 1024);
   w.counter = (int*)p; carve(p, 256);
   w.jac = (void*)p; carve(p, jacobi_scratch_bytes(b));
+  w.slabs = (double*)p; carve(p, (size_t)ceil_div(b, 64) * 4096 * 8);
+  w.Y64b = (double*)p; carve(p, (size_t)d * b * 8);
   w.Yc = (float*)p; carve(p, (size_t)d * b * 4);
   w.Yhi = (__nv_bfloat16*)p; carve(p, (size_t)d * b * 2);
   w.Ylo = (__nv_bfloat16*)p; carve(p, (size_t)d * b * 2);
@@ -472,50 +482,70 @@ static RefreshBuffers layout(void* base, int64_t d, int64_t L, int r, int b) {
 template <typename TY>
 static galore_status_t gram(const TY* Y, int64_t d, int b, double* C, cudaStream_t st) {
   EpiStore<double, double> epi{C, b, 0, 1.0, 0.0};
-  return launch_gemm_simt<TY, TY, double>(b, b, (int)d, Y, 1, b, Y, b, 1, 1, epi, st);
+  return launch_gemm_dmma<TY, TY>(b, b, (int)d, Y, 1, b, Y, b, 1, epi, st);
 }
 
-// In-place blocked Cholesky of the b x b matrix C (lower), and Y <- Y L^-T.
-template <typename TY>
-static galore_status_t cholesky_solve(TY* Y, int64_t d, int b, double* C, const RefreshBuffers& w, int32_t* status,
-                                      cudaStream_t st) {
-  for (int j0 = 0; j0 < b; j0 += 64) {
-    const int nb = std::min(64, b - j0);
-    const int j1 = j0 + nb;
-    // solve for the panel of Y first needs L[J, <J], which earlier panels completed
-    if (j0 > 0) {
-      // tmp = Y[:, J] - Y[:, <J] L[J, <J]^T
-      EpiResidual<TY> epi{Y + j0, b, w.tmp, 64};
-      GALORE_TRY((launch_gemm_simt<TY, double, double>((int)d, nb, j0, Y, b, 1, C + (int64_t)j0 * b, 1, b, 1, epi, st)));
-    } else {
-      EpiResidual<TY> epi{Y, b, w.tmp, 64};
-      GALORE_TRY((launch_gemm_simt<TY, double, double>((int)d, nb, 0, Y, b, 1, C, 1, b, 1, epi, st)));
-    }
-    potf2_inv_kernel<<<1, 64, 0, st>>>(C + (int64_t)j0 * b + j0, b, nb, w.Linv, status);
+// Blocked Cholesky of the b x b matrix C (lower triangle, in place), then T = L^-1 (b x b, lower,
+// zero above the diagonal).
+//   factor : per 64-wide panel the diagonal block (with its inverse, kept in w.slabs), the panel
+//            below it and the trailing update;
+//   invert : the inverses of the diagonal blocks are merged pairwise, level by level,
+//            [T11 0; T21 T22] with T21 = -T22 L21 T11, every level two batched products.
+// scratch: b*b/4 doubles.
+static galore_status_t cholesky_inverse(double* C, int b, double* T, double* scratch, const RefreshBuffers& w,
+                                        int32_t* status, cudaStream_t st) {
+  const int nblk = (int)ceil_div(b, 64);
+  for (int p = 0; p < nblk; ++p) {
+    const int j0 = p * 64, nb = std::min(64, b - j0), j1 = j0 + nb;
+    double* slab = w.slabs + (int64_t)p * 4096;
+    potf2_inv_kernel<<<1, 64, 0, st>>>(C + (int64_t)j0 * b + j0, b, nb, slab, status);
     GALORE_LAUNCH_CHECK();
-    // Y[:, J] = tmp Linv^T
-    {
-      EpiStore<TY, double> epi{Y + j0, b, 0, 1.0, 0.0};
-      GALORE_TRY((launch_gemm_simt<double, double, double>((int)d, nb, nb, w.tmp, 64, 1, w.Linv, 1, 64, 1, epi, st)));
-    }
     if (j1 < b) {
       const int rem = b - j1;
+      double* panel = C + (int64_t)j1 * b + j0;
       // L[rest, J] = C[rest, J] Linv^T   (in place: one CTA column covers all nb columns)
-      EpiStore<double, double> epi{C + (int64_t)j1 * b + j0, b, 0, 1.0, 0.0};
-      GALORE_TRY((launch_gemm_simt<double, double, double>(rem, nb, nb, C + (int64_t)j1 * b + j0, b, 1, w.Linv, 1, 64, 1, epi, st)));
+      EpiStore<double, double> epi{panel, b, 0, 1.0, 0.0};
+      GALORE_TRY((launch_gemm_dmma<double, double>(rem, nb, nb, panel, b, 1, slab, 1, 64, epi, st)));
       // C[rest, rest] -= L[rest, J] L[rest, J]^T
       EpiStore<double, double> upd{C + (int64_t)j1 * b + j1, b, 0, -1.0, 1.0};
-      GALORE_TRY((launch_gemm_simt<double, double, double>(rem, rem, nb, C + (int64_t)j1 * b + j0, b, 1,
-                                                           C + (int64_t)j1 * b + j0, 1, b, 1, upd, st)));
+      GALORE_TRY((launch_gemm_dmma<double, double>(rem, rem, nb, panel, b, 1, panel, 1, b, upd, st)));
+    }
+  }
+  GALORE_CUDA_TRY(cudaMemsetAsync(T, 0, sizeof(double) * b * b, st));
+  place_diag_inverse_kernel<<<nblk, 256, 0, st>>>(w.slabs, b, T);
+  GALORE_LAUNCH_CHECK();
+  for (int64_t s = 64; s < b; s *= 2) {
+    const int64_t step = 2 * s * b + 2 * s;            // from one merged block to the next, in elements
+    const int full = (int)(b / (2 * s));               // blocks with a complete lower half
+    const int tail = (int)(b % (2 * s)) - (int)s;      // rows of a ragged last lower half (<= 0: none)
+    for (int pass = 0; pass < 2; ++pass) {
+      const int count = pass == 0 ? full : (tail > 0 ? 1 : 0);
+      if (count == 0) continue;
+      const int s2 = pass == 0 ? (int)s : tail;
+      const int64_t o = pass == 0 ? 0 : (int64_t)full * 2 * s;
+      const double* L21 = C + (o + s) * b + o;
+      const double* T11 = T + o * b + o;
+      const double* T22 = T + (o + s) * b + (o + s);
+      double* T21 = T + (o + s) * b + o;
+      // W = L21 T11
+      EpiStore<double, double> ew{scratch, s, s * s, 1.0, 0.0};
+      GALORE_TRY((launch_gemm_dmma<double, double>(s2, (int)s, (int)s, L21, b, 1, T11, b, 1, ew, st, count, step, step)));
+      // T21 = -T22 W
+      EpiStore<double, double> et{T21, b, step, -1.0, 0.0};
+      GALORE_TRY((launch_gemm_dmma<double, double>(s2, (int)s, s2, T22, b, 1, scratch, s, 1, et, st, count, step, s * s)));
     }
   }
   return GALORE_OK;
 }
 
-template <typename TY>
-static galore_status_t orthonormalise(TY* Y, int64_t d, int b, const RefreshBuffers& w, int32_t* status, cudaStream_t st) {
+// out = Y L^-T with L L^T = Y^T Y (CholeskyQR); out must not alias Y.  Uses w.C, w.Vt, w.H.
+template <typename TY, typename TO>
+static galore_status_t orthonormalise(const TY* Y, TO* out, int64_t d, int b, const RefreshBuffers& w, int32_t* status,
+                                      cudaStream_t st) {
   GALORE_TRY(gram(Y, d, b, w.C, st));
-  return cholesky_solve(Y, d, b, w.C, w, status, st);
+  GALORE_TRY(cholesky_inverse(w.C, b, w.Vt, w.H, w, status, st));
+  EpiStore<TO, double> epi{out, b, 0, 1.0, 0.0};
+  return launch_gemm_dmma<TY, double>((int)d, b, b, Y, b, 1, w.Vt, 1, b, epi, st);
 }
 
 // ---- power step on the tensor cores -------------------------------------------------------------
@@ -544,17 +574,15 @@ static galore_status_t orth_tensor(TensorRefresh& t, const RefreshBuffers& w, in
   GALORE_TRY(tensor_group_launch_project(t.tg, st));
   gram_sum_kernel<<<grid_for(bb), 256, 0, st>>>(g0, g1, g2, w.C, bb);
   GALORE_LAUNCH_CHECK();
-  // T = L^-T from the blocked Cholesky solve applied to the identity (b x b instead of d x b)
-  set_identity_kernel<<<grid_for(bb), 256, 0, st>>>(w.Vt, b);
-  GALORE_LAUNCH_CHECK();
-  GALORE_TRY(cholesky_solve(w.Vt, (int64_t)b, b, w.C, w, t.status, st));
+  // T = L^-1, split into a bf16 pair; as the second operand of Y L^-T it is read K-contiguous
+  GALORE_TRY(cholesky_inverse(w.C, b, w.Vt, w.H, w, t.status, st));
   split_double_kernel<<<grid_for(bb), 256, 0, st>>>(w.Vt, w.Thi, w.Tlo, bb);
   GALORE_LAUNCH_CHECK();
   const int m = t.master, s1 = (m + 1) % 3, s2 = (m + 2) % 3;
   tensor_group_reset(t.tg);   // Y T = hi Thi + hi Tlo + lo Thi
-  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 0, w.Thi, b, 1, (int)d, b, b, t.F[m], b, t.status));
-  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 0, w.Tlo, b, 1, (int)d, b, b, t.F[s1], b, t.status));
-  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Ylo, b, 0, w.Thi, b, 1, (int)d, b, b, t.F[s2], b, t.status));
+  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 0, w.Thi, b, 0, (int)d, b, b, t.F[m], b, t.status));
+  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 0, w.Tlo, b, 0, (int)d, b, b, t.F[s1], b, t.status));
+  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Ylo, b, 0, w.Thi, b, 0, (int)d, b, b, t.F[s2], b, t.status));
   GALORE_TRY(tensor_group_launch_project(t.tg, st));
   sum_split_kernel<<<grid_for(yb), 256, 0, st>>>(t.F[m], t.F[s1], t.F[s2], t.F[m], w.Yhi, w.Ylo, yb);
   GALORE_LAUNCH_CHECK();
@@ -637,7 +665,8 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
       GALORE_LAUNCH_CHECK();
       GALORE_TRY(orth_tensor(tr, w, d, b, st));
     } else {
-      GALORE_TRY(orthonormalise(Y, d, b, w, status, st));
+      GALORE_TRY(orthonormalise(Y, Yn, d, b, w, status, st));
+      std::swap(Y, Yn);
     }
   }
   double predicted = 0.0;
@@ -663,8 +692,7 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
     GALORE_LAUNCH_CHECK();
     shift_kernel<<<grid_for(yb), 256, 0, st>>>(Yn, Y, yb, b, w.part);
     GALORE_LAUNCH_CHECK();
-    std::swap(Y, Yn);
-    return orthonormalise(Y, d, b, w, status, st);
+    return orthonormalise(Yn, Y, d, b, w, status, st);    // the old block is no longer needed: reuse it for the result
   };
 
   // ---- first steps, then a cheap look at the spectrum ------------------------------------------
@@ -706,16 +734,10 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
       }
     }
   }
-  bool pair_stale = false;
   bool with_vt = false;
 
   for (;;) {
     // ---- power steps ---------------------------------------------------------
-    if (tensor && pair_stale && q_done < q_target) {   // the Rayleigh-Ritz pass re-orthonormalised the master in place
-      split_kernel<<<grid_for(yb), 256, 0, st>>>(Y, w.Yhi, w.Ylo, yb);
-      GALORE_LAUNCH_CHECK();
-      pair_stale = false;
-    }
     for (; q_done < q_target; ++q_done) {
       const bool orth = ((q_target - 1 - q_done) % orth_every) == 0;      // the last step always ends orthonormal
       GALORE_TRY(one_step(orth));
@@ -727,15 +749,13 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
       set_identity_kernel<<<grid_for(yb), 256, 0, st>>>(w.Y64, (int)d);
       GALORE_LAUNCH_CHECK();
     } else {
-      GALORE_TRY(orthonormalise(Y, d, b, w, status, st));     // second CholeskyQR pass in fp32 storage
-      convert_kernel<float, double><<<grid_for(yb), 256, 0, st>>>(Y, w.Y64, yb);
-      GALORE_LAUNCH_CHECK();
-      GALORE_TRY(orthonormalise(w.Y64, d, b, w, status, st));
+      GALORE_TRY(orthonormalise(Y, w.Y64b, d, b, w, status, st));     // two more CholeskyQR passes, results in fp64
+      GALORE_TRY(orthonormalise(w.Y64b, w.Y64, d, b, w, status, st));
     }
     double* Z64 = (double*)w.Zu;
     {  // Z = A^T Y   (L x b), fp64
       EpiStore<double, double> epi{Z64, b, 0, 1.0, 0.0};
-      GALORE_TRY((launch_gemm_simt<TG, double, double>((int)L, b, (int)d, G, sAl, sAi, w.Y64, b, 1, 1, epi, st)));
+      GALORE_TRY((launch_gemm_dmma<TG, double>((int)L, b, (int)d, G, sAl, sAi, w.Y64, b, 1, epi, st)));
     }
     const clk::time_point t_jac = now_synced();
     local.ms_ritz += ms_between(t_rr, t_jac);
@@ -769,7 +789,6 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
       if (!converged && q_done < pr.max_iters && ratio < 1.0 && ratio > 0.0) {
         int need = (int)ceil(log(pr.tol) / log(ratio)) + 2;
         q_target = std::min(pr.max_iters, std::max(need, q_done + 1));
-        pair_stale = true;
         continue;                                              // more power steps, then Rayleigh-Ritz again
       }
     }
@@ -784,7 +803,7 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
   GALORE_LAUNCH_CHECK();
   {
     EpiStore<double, double> epi{w.P64, r, 0, 1.0, 0.0};
-    GALORE_TRY((launch_gemm_simt<double, double, double>((int)d, r, b, w.Y64, b, 1, w.Vsel, 1, b, 1, epi, st)));
+    GALORE_TRY((launch_gemm_dmma<double, double>((int)d, r, b, w.Y64, b, 1, w.Vsel, 1, b, epi, st)));
   }
   const int64_t pc = d * r;
   if (pr.p_dtype == GALORE_BF16)
@@ -798,9 +817,9 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
     double* T1 = (double*)w.Zu;   // L x r
     double* T2 = w.Y64;           // d x r (Y64 is no longer needed)
     EpiStore<double, double> e1{T1, r, 0, 1.0, 0.0};
-    GALORE_TRY((launch_gemm_simt<TG, double, double>((int)L, r, (int)d, G, sAl, sAi, w.P64, r, 1, 1, e1, st)));
+    GALORE_TRY((launch_gemm_dmma<TG, double>((int)L, r, (int)d, G, sAl, sAi, w.P64, r, 1, e1, st)));
     EpiStore<double, double> e2{T2, r, 0, 1.0, 0.0};
-    GALORE_TRY((launch_gemm_simt<TG, double, double>((int)d, r, (int)L, G, sAi, sAl, T1, r, 1, 1, e2, st)));
+    GALORE_TRY((launch_gemm_dmma<TG, double>((int)d, r, (int)L, G, sAi, sAl, T1, r, 1, e2, st)));
     GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
     residual_kernel<<<grid_for(pc), 256, 0, st>>>(T2, w.P64, w.theta, d, r, w.scal);
     GALORE_LAUNCH_CHECK();
