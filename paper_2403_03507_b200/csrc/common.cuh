@@ -51,6 +51,20 @@ template <> __device__ __forceinline__ double cvt<double, __nv_bfloat16>(__nv_bf
 template <> __device__ __forceinline__ __nv_bfloat16 cvt<__nv_bfloat16, float>(float x) { return __float2bfloat16_rn(x); }
 template <> __device__ __forceinline__ __nv_bfloat16 cvt<__nv_bfloat16, double>(double x) { return __float2bfloat16_rn((float)x); }
 
+// 1 / sqrt(x) in double precision from the single-precision hardware estimate and two Newton steps
+// (the latency of the general routine matters in the serial parts of the factorisations).  x is
+// first scaled by an even power of two into [1, 4); outside 1e-290 .. 1e290 the general routine runs.
+__device__ __forceinline__ double rsqrt_newton(double x) {
+  if (!(x > 1e-290 && x < 1e290)) return rsqrt(x);
+  const int ex = ((((__double2hiint(x) >> 20) & 0x7ff) - 1023)) & ~1;
+  const double xs = x * __hiloint2double((1023 - ex) << 20, 0);
+  double y = (double)rsqrtf((float)xs);
+  const double h = 0.5 * xs;
+  y = fma(y, fma(-h * y, y, 0.5), y);
+  y = fma(y, fma(-h * y, y, 0.5), y);
+  return y * __hiloint2double((1023 - ex / 2) << 20, 0);
+}
+
 // Status word in the workspace (first 256 bytes).
 struct DeviceStatus {
   int32_t flags;

@@ -135,17 +135,76 @@ __global__ void __launch_bounds__(128) jb_gram_kernel(const double* __restrict__
     }
 }
 
-// One cyclic sweep over the 64 rows of a block pair, run on their Gram matrix A: a rotation of rows
-// (p, q) by (c, s) turns A into R A R^T.  Rot accumulates the rotations (Rot <- R Rot), so that the
-// rows themselves become Rot x rows.  flags[pair] = rotations applied (0: Rot is the identity).
-__global__ void __launch_bounds__(256) jb_sweep_kernel(const double* __restrict__ part, int chunks, int b, int nblk, int round,
-                                                       double tol, double* __restrict__ rot_out, int* __restrict__ flags,
-                                                       int* __restrict__ rotations) {
+// One cyclic sweep over the 64 rows of a block pair, run on their Gram matrix A, with the rotations
+// accumulated into Rot (Rot <- R Rot, so that the rows themselves become Rot x rows).
+//
+// The 64 rows sit at the 64 positions of a round-robin table; slot k pairs positions k and 63 - k.
+// After every round the rows move on by one position (position 0 stays), and the data moves with
+// them: a round reads A and Rot from one shared-memory copy and writes the other copy at the next
+// positions, so every address a thread touches is the same in all rounds and is computed once.
+// After the 63 rounds of a sweep all rows are back where they started.
+//   * A is kept as its upper triangle in position space (entry (i, j) at [min][max]).  The 32
+//     rotations of a round split it into 2 x 2 blocks (positions of slot u x positions of slot v)
+//     that transform independently, B <- R_u B R_v^T; the 528 blocks with u <= v are the work.
+//   * Rot: the two rows of a slot are rotated, 64 columns each.
+//   * The angle is computed in single precision (after scaling by the exponent of the larger of
+//     aqq - app and 2 apq) and (c, s) are then renormalised in double precision: the rotation is
+//     orthogonal to double rounding, its angle accurate to about 1e-7, which leaves the pair
+//     orthogonal to 1e-7 of what it was.
+// flags[pair] = rotations applied (0: Rot is the identity and is not written).
+constexpr int kSweepRounds = kPairRows - 1;
+constexpr int kSlots = kPairRows / 2;
+constexpr int kBlockTasks = kSlots * (kSlots + 1) / 2;
+constexpr int kSweepThreads = 512;
+constexpr int kALd = kPairRows + 1;
+constexpr size_t kSweepSmem = 4 * (size_t)kPairRows * kALd * sizeof(double);
+
+__host__ __device__ __forceinline__ int next_position(int pos) { return pos == 0 ? 0 : (pos == kPairRows - 1 ? 1 : pos + 1); }
+__host__ __device__ __forceinline__ int upper_offset(int i, int j) { return i < j ? i * kALd + j : j * kALd + i; }
+
+struct BlockTask {
+  int u, v;        // slots
+  int rd[4];       // offsets of (fu, fv), (fu, gv), (gu, fv), (gu, gv) in the current copy
+  int wr[4];       // offsets of the same entries, one position on, in the other copy
+};
+__device__ __forceinline__ BlockTask make_block_task(int task) {
+  BlockTask t;
+  int u = 0, start = 0;
+  while (u + 1 < kSlots && start + (kSlots - u) <= task) { start += kSlots - u; ++u; }
+  t.u = u;
+  t.v = min(kSlots - 1, u + (task - start));
+  const int fu = t.u, gu = kPairRows - 1 - t.u, fv = t.v, gv = kPairRows - 1 - t.v;
+  t.rd[0] = upper_offset(fu, fv);
+  t.rd[1] = upper_offset(fu, gv);
+  t.rd[2] = upper_offset(gu, fv);
+  t.rd[3] = upper_offset(gu, gv);
+  const int nfu = next_position(fu), ngu = next_position(gu), nfv = next_position(fv), ngv = next_position(gv);
+  t.wr[0] = upper_offset(nfu, nfv);
+  t.wr[1] = upper_offset(nfu, ngv);
+  t.wr[2] = upper_offset(ngu, nfv);
+  t.wr[3] = upper_offset(ngu, ngv);
+  return t;
+}
+
+__device__ __forceinline__ void block_update(const BlockTask& t, const double2* cs, const double* cur, double* nxt) {
+  const double2 ru = cs[t.u], rv = cs[t.v];
+  const double a0 = cur[t.rd[0]], a1 = cur[t.rd[1]], a2 = cur[t.rd[2]], a3 = cur[t.rd[3]];
+  // B <- R_u B R_v^T.  For u == v the two off-diagonal entries are one stored value; both results agree.
+  const double r00 = ru.x * a0 - ru.y * a2, r01 = ru.x * a1 - ru.y * a3;
+  const double r10 = ru.y * a0 + ru.x * a2, r11 = ru.y * a1 + ru.x * a3;
+  nxt[t.wr[0]] = rv.x * r00 - rv.y * r01;
+  nxt[t.wr[1]] = rv.y * r00 + rv.x * r01;
+  nxt[t.wr[2]] = rv.x * r10 - rv.y * r11;
+  nxt[t.wr[3]] = rv.y * r10 + rv.x * r11;
+}
+
+__global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* __restrict__ part, int chunks, int b, int nblk,
+                                                                 int round, double tol, double* __restrict__ rot_out,
+                                                                 int* __restrict__ flags, int* __restrict__ rotations) {
   extern __shared__ __align__(16) double jb_smem[];
-  double(*A)[65] = reinterpret_cast<double(*)[65]>(jb_smem);
-  double(*Rot)[65] = reinterpret_cast<double(*)[65]>(jb_smem + 64 * 65);
-  __shared__ double cs[32][2];
-  __shared__ int pq[32][2];
+  double* Abuf[2] = {jb_smem, jb_smem + kPairRows * kALd};
+  double* Rbuf[2] = {jb_smem + 2 * kPairRows * kALd, jb_smem + 3 * kPairRows * kALd};
+  __shared__ double2 cs[kSlots];
   const int pair = blockIdx.x, tid = threadIdx.x;
   const BlockPair bp = block_pair(pair, round, nblk);
   if (bp.I * kBlockRows >= b) {
@@ -154,83 +213,101 @@ __global__ void __launch_bounds__(256) jb_sweep_kernel(const double* __restrict_
   }
   const double* src = part + (int64_t)pair * chunks * (kPairRows * kPairRows);
   {
-    double sum[16];
+    double sum[8];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) sum[i] = 0.0;
-    for (int c = 0; c < chunks; ++c) {
-      const double* sc = src + (int64_t)c * (kPairRows * kPairRows);
+    for (int i = 0; i < 8; ++i) sum[i] = 0.0;
+    for (int c = 0; c < chunks; c += 4) {     // four partial matrices in flight
+      double v[4][8];
 #pragma unroll
-      for (int i = 0; i < 16; ++i) sum[i] += sc[tid + 256 * i];
+      for (int j = 0; j < 4; ++j) {
+        const double* sc = src + (int64_t)(c + j) * (kPairRows * kPairRows);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[j][i] = (c + j < chunks) ? sc[tid + kSweepThreads * i] : 0.0;
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sum[i] += v[j][i];
     }
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const int idx = tid + 256 * i;
-      A[idx >> 6][idx & 63] = sum[i];
-      Rot[idx >> 6][idx & 63] = ((idx >> 6) == (idx & 63)) ? 1.0 : 0.0;
+    for (int i = 0; i < 8; ++i) {
+      const int idx = tid + kSweepThreads * i;
+      Abuf[0][(idx >> 6) * kALd + (idx & 63)] = sum[i];
+      Rbuf[0][(idx >> 6) * kALd + (idx & 63)] = ((idx >> 6) == (idx & 63)) ? 1.0 : 0.0;
     }
   }
+  const BlockTask t0 = make_block_task(tid);                                   // tasks 0 .. 511
+  const bool second = tid < kBlockTasks - kSweepThreads;
+  const BlockTask t1 = make_block_task(second ? kSweepThreads + tid : 0);      // tasks 512 .. 527
+  // Rot: slot tid / 16, columns tid % 16 + 16 i
+  const int rslot = tid >> 4, rcol = tid & 15;
+  const int rf = rslot * kALd + rcol, rg = (kPairRows - 1 - rslot) * kALd + rcol;
+  const int wf = next_position(rslot) * kALd + rcol, wg = next_position(kPairRows - 1 - rslot) * kALd + rcol;
   __syncthreads();
   int applied = 0;
-  const int u = tid >> 3, l8 = tid & 7;
   const double tol2 = tol * tol;
-  for (int rr = 0; rr < kPairRows - 1; ++rr) {
-    if (tid < 32) {
-      int p = rr_player(tid, rr, kPairRows), q = rr_player(kPairRows - 1 - tid, rr, kPairRows);
-      if (p > q) { const int x = p; p = q; q = x; }
-      const double app = A[p][p], aqq = A[q][q], apq = A[p][q];
+  for (int rr = 0; rr < kSweepRounds; ++rr) {
+    const double* Ac = Abuf[rr & 1];
+    double* An = Abuf[(rr + 1) & 1];
+    const double* Rc = Rbuf[rr & 1];
+    double* Rn = Rbuf[(rr + 1) & 1];
+    if (tid < kSlots) {
+      const int f = tid, g = kPairRows - 1 - tid;
+      const double app = Ac[f * kALd + f], aqq = Ac[g * kALd + g], apq = Ac[f * kALd + g];
       double c = 1.0, s = 0.0;
       if (apq != 0.0 && apq * apq > tol2 * app * aqq) {
-        // tan of the rotation angle: the smaller root of t^2 + 2 zeta t - 1 = 0, zeta = (aqq - app) / (2 apq)
+        // tan(2 phi) = 2 apq / (aqq - app), |phi| <= pi/4.  With h = hypot(d, o): cos(2 phi) = |d| / h,
+        // c = sqrt((1 + |d|/h) / 2), s = sign(d) o / (2 h c).
         const double d = aqq - app, o = 2.0 * apq;
-        const double h = sqrt(d * d + o * o);
-        const double tt = o / (d + (d >= 0.0 ? h : -h));
-        c = rsqrt(1.0 + tt * tt);
-        s = c * tt;
-        ++applied;
+        const int ex = (__double2hiint(fmax(fabs(d), fabs(o))) >> 20) & 0x7ff;
+        if (ex >= 1 && ex <= 2045) {
+          const double sc = __hiloint2double((2046 - ex) << 20, 0);
+          const float df = (float)(d * sc), of = (float)(o * sc);
+          const float rh = rsqrtf(fmaf(df, df, of * of));
+          const float v = fmaf(0.5f * fabsf(df), rh, 0.5f);
+          const float rc = rsqrtf(v);
+          const float c0 = v * rc, s0 = (d >= 0.0 ? 0.5f : -0.5f) * of * rh * rc;
+          if (s0 != 0.0f) {
+            c = (double)c0;
+            s = (double)s0;
+            const double eps = fma(c, c, fma(s, s, -1.0));          // c0^2 + s0^2 = 1 + eps, |eps| ~ 1e-7
+            const double fix = fma(eps, fma(eps, 0.375, -0.5), 1.0);  // (1 + eps)^-1/2 to O(eps^3)
+            c *= fix;
+            s *= fix;
+            ++applied;
+          }
+        }
       }
-      cs[tid][0] = c;
-      cs[tid][1] = s;
-      pq[tid][0] = p;
-      pq[tid][1] = q;
+      cs[tid] = make_double2(c, s);
     }
     __syncthreads();
-    // A <- R A R^T, one 2 x 2 block (rows of slot u, columns of slot v) at a time: blocks are disjoint,
-    // so the row and the column rotation of a block are applied together.  Rot <- R Rot alongside.
-    const double cu = cs[u][0], su = cs[u][1];
-    const int pu = pq[u][0], qu = pq[u][1];
+    block_update(t0, cs, Ac, An);
+    if (second) block_update(t1, cs, Ac, An);
+    {
+      const double2 r = cs[rslot];
 #pragma unroll
-    for (int vv = 0; vv < 4; ++vv) {
-      const int v = l8 + 8 * vv;
-      const double cv = cs[v][0], sv = cs[v][1];
-      if (su == 0.0 && sv == 0.0) continue;
-      const int pv = pq[v][0], qv = pq[v][1];
-      const double a00 = A[pu][pv], a01 = A[pu][qv], a10 = A[qu][pv], a11 = A[qu][qv];
-      const double r00 = cu * a00 - su * a10, r01 = cu * a01 - su * a11;
-      const double r10 = su * a00 + cu * a10, r11 = su * a01 + cu * a11;
-      A[pu][pv] = cv * r00 - sv * r01;
-      A[pu][qv] = sv * r00 + cv * r01;
-      A[qu][pv] = cv * r10 - sv * r11;
-      A[qu][qv] = sv * r10 + cv * r11;
-    }
-    if (su != 0.0) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int col = l8 + 8 * i;
-        const double x = Rot[pu][col], y = Rot[qu][col];
-        Rot[pu][col] = cu * x - su * y;
-        Rot[qu][col] = su * x + cu * y;
+      for (int i = 0; i < 4; ++i) {
+        const double x = Rc[rf + 16 * i], y = Rc[rg + 16 * i];
+        Rn[wf + 16 * i] = r.x * x - r.y * y;
+        Rn[wg + 16 * i] = r.y * x + r.x * y;
       }
     }
     __syncthreads();
   }
-  double* out = rot_out + (int64_t)pair * (kPairRows * kPairRows);
-  for (int idx = tid; idx < kPairRows * kPairRows; idx += 256) out[idx] = Rot[idx >> 6][idx & 63];
   if (tid < 32) {
     for (int o = 16; o > 0; o >>= 1) applied += __shfl_xor_sync(0xffffffffu, applied, o);
+    applied = __shfl_sync(0xffffffffu, applied, 0);
     if (tid == 0) {
       flags[pair] = applied;
       if (applied) atomicAdd(rotations, applied);
     }
+    if (tid == 0) cs[0].x = (double)applied;
+  }
+  __syncthreads();
+  if (cs[0].x != 0.0) {   // all rows are back at their own positions after the 63 rounds
+    const double* Rf = Rbuf[kSweepRounds & 1];
+    double* out = rot_out + (int64_t)pair * (kPairRows * kPairRows);
+    for (int idx = tid; idx < kPairRows * kPairRows; idx += kSweepThreads) out[idx] = Rf[(idx >> 6) * kALd + (idx & 63)];
   }
 }
 
@@ -322,7 +399,6 @@ JacobiGeometry jacobi_geometry(int b) {
   return g;
 }
 
-constexpr size_t kSweepSmem = 2 * 64 * 65 * sizeof(double);
 constexpr size_t kApplySmem = (size_t)(kPairRows * kRotLd + kPairRows * kTileLd) * sizeof(double);
 
 }  // namespace
@@ -357,7 +433,7 @@ galore_status_t jacobi_eigh(double* X, double* Vt, int b, void* scratch, int* co
     for (int round = 0; round < g.nblk - 1; ++round) {
       jb_gram_kernel<<<dim3(g.pairs, g.chunks), 128, 0, st>>>(X, b, g.nblk, round, g.chunks, part);
       GALORE_LAUNCH_CHECK();
-      jb_sweep_kernel<<<g.pairs, 256, kSweepSmem, st>>>(part, g.chunks, b, g.nblk, round, tol, rot, flags, counter);
+      jb_sweep_kernel<<<g.pairs, kSweepThreads, kSweepSmem, st>>>(part, g.chunks, b, g.nblk, round, tol, rot, flags, counter);
       GALORE_LAUNCH_CHECK();
       jb_apply_kernel<<<dim3(g.pairs, g.col_tiles, Vt ? 2 : 1), 256, kApplySmem, st>>>(X, Vt, b, g.nblk, round, rot, flags);
       GALORE_LAUNCH_CHECK();
