@@ -240,9 +240,9 @@ __global__ void __launch_bounds__(64) potf2_inv_kernel(double* __restrict__ C, i
         atomicOr(status, GALORE_DEV_CHOLESKY);
         piv = fabs(piv) + 1e-300;
       }
-      const double sq = sqrt(piv);
-      Ls[j][j] = sq;
-      rdiag[j] = 1.0 / sq;
+      const double rs = rsqrt_newton(piv);
+      Ls[j][j] = piv * rs;
+      rdiag[j] = rs;
     }
     __syncthreads();
     double l = 0.0;
@@ -380,6 +380,29 @@ __global__ void __launch_bounds__(256) residual_kernel(const double* __restrict_
   if (threadIdx.x == 0) atomicAdd(scal + 1, s);
 }
 
+// the same with T2 given as two fp32 partial products
+__global__ void __launch_bounds__(256) residual_pair_kernel(const float* __restrict__ t0, const float* __restrict__ t1,
+                                                            const double* __restrict__ P, const double* __restrict__ theta,
+                                                            int64_t rows, int r, double* __restrict__ scal) {
+  __shared__ double red[8];
+  double s = 0.0;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < rows * r; i += (int64_t)gridDim.x * blockDim.x) {
+    double d = ((double)t0[i] + (double)t1[i]) - theta[i % r] * P[i];
+    s += d * d;
+  }
+  s = block_sum_256(s, red);
+  if (threadIdx.x == 0) atomicAdd(scal + 1, s);
+}
+
+// GEMM epilogue: the result as a bf16 hi/lo pair
+struct EpiSplitPair {
+  __nv_bfloat16 *hi, *lo;
+  int64_t ld;
+  __device__ __forceinline__ void operator()(int i, int j, double acc, int) const {
+    split_bf16((float)acc, hi[(int64_t)i * ld + j], lo[(int64_t)i * ld + j]);
+  }
+};
+
 static inline unsigned grid_for(int64_t count) { return (unsigned)std::min<int64_t>(ceil_div(count, 256), 148 * 8); }
 
 // ---------------------------------------------------------------------------
@@ -406,7 +429,6 @@ struct RefreshBuffers {
   int* counter;   // 1
   void* jac;      // scratch of the Jacobi eigensolver
   double* slabs;  // ceil(b / 64) inverses of 64 x 64 diagonal blocks
-  double* Y64b;   // d x b, second fp64 block
   // tensor-core power steps
   float* Yc;                 // d x b, third fp32 block
   __nv_bfloat16 *Yhi, *Ylo;  // d x b
@@ -435,7 +457,6 @@ size_t refresh_workspace_bytes(int64_t d, int64_t L, int r, int b) {
   t += 256 * 2 + 8 * 1024;
   t += align_up(jacobi_scratch_bytes(b), 256);
   t += align_up((size_t)ceil_div(b, 64) * 4096 * 8, 256);
-  t += align_up((size_t)d * b * 8, 256);
   t += align_up((size_t)d * b * 4, 256) + 2 * align_up((size_t)d * b * 2, 256) + 2 * align_up((size_t)L * b * 2, 256) +
        2 * align_up((size_t)b * b * 2, 256);
   return t;
@@ -463,7 +484,6 @@ static RefreshBuffers layout(void* base, int64_t d, int64_t L, int r, int b) {
   w.counter = (int*)p; carve(p, 256);
   w.jac = (void*)p; carve(p, jacobi_scratch_bytes(b));
   w.slabs = (double*)p; carve(p, (size_t)ceil_div(b, 64) * 4096 * 8);
-  w.Y64b = (double*)p; carve(p, (size_t)d * b * 8);
   w.Yc = (float*)p; carve(p, (size_t)d * b * 4);
   w.Yhi = (__nv_bfloat16*)p; carve(p, (size_t)d * b * 2);
   w.Ylo = (__nv_bfloat16*)p; carve(p, (size_t)d * b * 2);
@@ -749,8 +769,9 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
       set_identity_kernel<<<grid_for(yb), 256, 0, st>>>(w.Y64, (int)d);
       GALORE_LAUNCH_CHECK();
     } else {
-      GALORE_TRY(orthonormalise(Y, w.Y64b, d, b, w, status, st));     // two more CholeskyQR passes, results in fp64
-      GALORE_TRY(orthonormalise(w.Y64b, w.Y64, d, b, w, status, st));
+      // Y left the last power step orthonormal to working precision (1e-7 on the FMA path, about 1e-4 from the
+      // bf16 pairs); one CholeskyQR pass in fp64 from there is orthonormal to double rounding
+      GALORE_TRY(orthonormalise(Y, w.Y64, d, b, w, status, st));
     }
     double* Z64 = (double*)w.Zu;
     {  // Z = A^T Y   (L x b), fp64
@@ -813,7 +834,22 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
   GALORE_LAUNCH_CHECK();
 
   // ---- a-posteriori residual of the kept Ritz pairs -----------------------------------
-  {
+  // || A A^T P - P Theta ||.  It is a diagnostic: on the tensor path A^T P = Z S is formed from the
+  // products already at hand and A (A^T P) runs on the tensor cores in bf16 pairs.
+  const bool tensor_residual = tensor && (r % 8) == 0;
+  if (tensor_residual) {
+    EpiSplitPair e1{w.Zhi, w.Zlo, r};
+    GALORE_TRY((launch_gemm_dmma<double, double>((int)L, r, b, (const double*)w.Zu, b, 1, w.Vsel, 1, b, e1, st)));
+    const int a_mn = pr.left ? 0 : 1;
+    const int s1 = (tr.master + 1) % 3, s2 = (tr.master + 2) % 3;
+    tensor_group_reset(tr.tg);
+    GALORE_TRY(tensor_group_add_gemm(tr.tg, pr.G, pr.ldg, a_mn, w.Zhi, r, 1, (int)d, r, (int)L, tr.F[s1], r, status));
+    GALORE_TRY(tensor_group_add_gemm(tr.tg, pr.G, pr.ldg, a_mn, w.Zlo, r, 1, (int)d, r, (int)L, tr.F[s2], r, status));
+    GALORE_TRY(tensor_group_launch_project(tr.tg, st));
+    GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
+    residual_pair_kernel<<<grid_for(d * r), 256, 0, st>>>(tr.F[s1], tr.F[s2], w.P64, w.theta, d, r, w.scal);
+    GALORE_LAUNCH_CHECK();
+  } else {
     double* T1 = (double*)w.Zu;   // L x r
     double* T2 = w.Y64;           // d x r (Y64 is no longer needed)
     EpiStore<double, double> e1{T1, r, 0, 1.0, 0.0};
@@ -823,6 +859,8 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
     GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
     residual_kernel<<<grid_for(pc), 256, 0, st>>>(T2, w.P64, w.theta, d, r, w.scal);
     GALORE_LAUNCH_CHECK();
+  }
+  {
     double sc[2] = {0, 0};
     GALORE_CUDA_TRY(cudaMemcpyAsync(sc, w.scal, sizeof(sc), cudaMemcpyDeviceToHost, st));
     GALORE_CUDA_TRY(cudaStreamSynchronize(st));
