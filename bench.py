@@ -200,6 +200,9 @@ def main():
     ap.add_argument("--projector", default="refresh", choices=["refresh", "random"],
                     help="refresh: one real refresh per distinct shape (timed, reported); random: a random orthonormal "
                          "projector (step timing does not depend on P's values; for short profiling runs)")
+    ap.add_argument("--refresh-only", action="store_true",
+                    help="run the projector refresh of each distinct shape and print its timings; no step is timed "
+                         "(for profiling the refresh on its own)")
     ap.add_argument("--extra-workloads", default="llama_1b_q8,llama_1b_f32",
                     help="comma-separated workloads also timed, device-resident only, reported under other_workloads "
                          "(only with the default workload; empty string to skip)")
@@ -232,7 +235,7 @@ def main():
     res = time_workload(w, args, dev, dist, world, rank, full=True)
     if rank == 0:
         extras = []
-        names = [x for x in args.extra_workloads.split(",") if x] if args.workload == "llama_7b_q8" and world == 1 else []
+        names = [x for x in args.extra_workloads.split(",") if x] if args.workload == "llama_7b_q8" and world == 1 and not args.refresh_only else []
         for name in names:
             extras.append(time_workload(wl.WORKLOADS[name], args, dev, None, 1, 0, full=False))
         if extras:
@@ -290,12 +293,16 @@ def time_workload(w, args, dev, dist, world, rank, full):
             elif first is None:
                 t0 = torch.cuda.Event(enable_timing=True)
                 t1 = torch.cuda.Event(enable_timing=True)
-                t0.record()
-                st, info = layer.galore_refresh_projector(pool[0])
-                t1.record()
-                torch.cuda.synchronize()
-                refresh_info.append({"shape": [m, n], "ms": t0.elapsed_time(t1), "status": st, **info.as_dict()})
+                for rep in range(1 if args.refresh_only else 2):         # the second run is the warm one
+                    t0.record()
+                    st, info = layer.galore_refresh_projector(pool[0])
+                    t1.record()
+                    torch.cuda.synchronize()
+                refresh_info.append({"shape": [m, n], "count": count, "ms": t0.elapsed_time(t1), "status": st,
+                                     **info.as_dict()})
                 first = layer.get_projector()
+                if args.refresh_only:
+                    break
             else:
                 layer.set_projector(first)                              # timing does not depend on P's values
             Wt = padded(m, n, tdt[w.w_dtype])
@@ -308,6 +315,8 @@ def time_workload(w, args, dev, dist, world, rank, full):
             bytes_alg += by
             flops_alg += fl
     torch.cuda.synchronize()
+    if args.refresh_only:
+        return {"refresh": refresh_info, "config": {"workload": w.name, "rank": w.rank}}
 
     batch = gb.Batch(layers, Ws, Gs, device=dev) if args.mode == "batch" else None
 
@@ -387,8 +396,16 @@ def time_workload(w, args, dev, dist, world, rank, full):
         "clocks": clocks, "gpu_launches": launches, "roofline": roof,
         "refresh": refresh_info,
     }
+    if refresh_info:
+        # Algorithm 1 refreshes every matrix once per `refresh_gap` steps: the step plus its share of that
+        set_ms = sum(x["ms"] * x["count"] for x in refresh_info)
+        amortised_ms = ms_step + set_ms / w.refresh_gap
+        out["refresh_amortised"] = {"refresh_ms_whole_set": set_ms, "refresh_gap": w.refresh_gap,
+                                    "ms_per_step": amortised_ms, "value": world * w.params / (amortised_ms * 1e-3),
+                                    "unit": UNIT}
     if not full:
-        return {k: out[k] for k in ("value", "ms_per_step", "config", "roofline", "refresh", "gpu_launches")}
+        return {k: out[k] for k in ("value", "ms_per_step", "config", "roofline", "refresh", "refresh_amortised",
+                                    "gpu_launches") if k in out}
 
     # ---- end to end through the host-buffer entry point -------------------------------------------
     if not args.no_e2e:
