@@ -8,7 +8,8 @@
 // epi(i, j, acc, split).  It carries the projections when the inputs are fp32
 // (where bf16 tensor-core inputs would break the fp32 tolerance) or not
 // TMA-aligned, and all fp64 work of the projector refresh.
-// blockIdx.z selects a K slice of `kchunk` elements (split-K).
+// blockIdx.z selects a K slice of `kchunk` elements (split-K) or, when `batched`, one problem of
+// a batch whose operands lie batchA / batchB elements apart.
 #pragma once
 
 #include "common.cuh"
@@ -18,7 +19,8 @@ namespace galore {
 template <typename TA, typename TB, typename TAcc, int BM, int BN, int BK, int TM, int TN, class Epi>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN))
 gemm_simt_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int64_t sAk,
-                 const TB* __restrict__ B, int64_t sBk, int64_t sBj, int kchunk, Epi epi) {
+                 const TB* __restrict__ B, int64_t sBk, int64_t sBj, int kchunk, Epi epi, int batched = 0,
+                 int64_t batchA = 0, int64_t batchB = 0) {
   constexpr int NT = (BM / TM) * (BN / TN);
   constexpr int LA = BM * BK / NT;   // elements of the A tile each thread fetches
   constexpr int LB = BN * BK / NT;
@@ -30,8 +32,12 @@ gemm_simt_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int
   const int tid = threadIdx.x;
   const int tx = tid % (BN / TN), ty = tid / (BN / TN);
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-  const int k_begin = blockIdx.z * kchunk;
-  const int k_end = min(K, k_begin + kchunk);
+  const int k_begin = batched ? 0 : blockIdx.z * kchunk;
+  const int k_end = batched ? K : min(K, k_begin + kchunk);
+  if (batched) {
+    A += (int64_t)blockIdx.z * batchA;
+    B += (int64_t)blockIdx.z * batchB;
+  }
   const bool a_kfast = (sAk == 1);   // consecutive threads walk the contiguous direction
   const bool b_kfast = (sBk == 1);
 
@@ -139,21 +145,24 @@ struct EpiApplyW {
 
 template <typename TA, typename TB, typename TAcc, class Epi>
 galore_status_t launch_gemm_simt(int M, int N, int K, const TA* A, int64_t sAi, int64_t sAk, const TB* B,
-                                 int64_t sBk, int64_t sBj, int splits, Epi epi, cudaStream_t stream) {
+                                 int64_t sBk, int64_t sBj, int splits, Epi epi, cudaStream_t stream, int batch = 0,
+                                 int64_t batchA = 0, int64_t batchB = 0) {
   if (M <= 0 || N <= 0) return GALORE_OK;
+  if (batch > 0) splits = 1;       // a batch uses blockIdx.z for the problem index
   if (splits < 1) splits = 1;
   int kchunk = (int)ceil_div(ceil_div(K, splits), 16) * 16;
   if (kchunk < 16) kchunk = 16;
   splits = (int)ceil_div(K > 0 ? K : 1, kchunk);
-  const bool small = (int64_t)M * N < (int64_t)128 * 128 * 96;
+  const unsigned gz = batch > 0 ? (unsigned)batch : (unsigned)splits;
+  const bool small = (int64_t)M * N * (batch > 0 ? batch : 1) < (int64_t)128 * 128 * 96;
   if (small) {
-    dim3 grid((unsigned)ceil_div(N, 64), (unsigned)ceil_div(M, 64), (unsigned)splits);
+    dim3 grid((unsigned)ceil_div(N, 64), (unsigned)ceil_div(M, 64), gz);
     gemm_simt_kernel<TA, TB, TAcc, 64, 64, 16, 4, 4, Epi><<<grid, 256, 0, stream>>>(
-        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi);
+        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi, batch > 0 ? 1 : 0, batchA, batchB);
   } else {
-    dim3 grid((unsigned)ceil_div(N, 128), (unsigned)ceil_div(M, 128), (unsigned)splits);
+    dim3 grid((unsigned)ceil_div(N, 128), (unsigned)ceil_div(M, 128), gz);
     gemm_simt_kernel<TA, TB, TAcc, 128, 128, 16, 8, 8, Epi><<<grid, 256, 0, stream>>>(
-        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi);
+        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi, batch > 0 ? 1 : 0, batchA, batchB);
   }
   GALORE_LAUNCH_CHECK();
   return GALORE_OK;

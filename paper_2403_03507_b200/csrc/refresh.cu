@@ -21,6 +21,7 @@
 // decays like (theta_b / theta_r)^q (theta = Ritz values, descending); the
 // iteration stops when that prediction is below the tolerance, or at the cap.
 #include "refresh.cuh"
+#include <type_traits>
 #include "eig_jacobi.cuh"
 #include "gemm_dmma.cuh"
 
@@ -187,23 +188,17 @@ __global__ void colsumsq_final_kernel(const double* __restrict__ part, int cols,
   out[c] = s;
 }
 
-// C (fp64) = g0 + g1 + g2 : the three bf16-pair products that make up a Gram matrix
+// C = g0 + g1 + g2 : the three bf16-pair products that make up a Gram matrix
 __global__ void gram_sum_kernel(const float* __restrict__ g0, const float* __restrict__ g1, const float* __restrict__ g2,
-                                double* __restrict__ C, int64_t count) {
+                                float* __restrict__ C, int64_t count) {
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
-    C[i] = (double)g0[i] + (double)g1[i] + (double)g2[i];
+    C[i] = (float)((double)g0[i] + (double)g1[i] + (double)g2[i]);
 }
 
 __global__ void split_kernel(const float* __restrict__ x, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
                              int64_t count) {
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
     split_bf16(x[i], hi[i], lo[i]);
-}
-
-__global__ void split_double_kernel(const double* __restrict__ x, __nv_bfloat16* __restrict__ hi,
-                                    __nv_bfloat16* __restrict__ lo, int64_t count) {
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
-    split_bf16((float)x[i], hi[i], lo[i]);
 }
 
 // ---- Cholesky of one diagonal block (nb <= 64) and the inverse of its factor ----
@@ -216,36 +211,40 @@ __global__ void split_double_kernel(const double* __restrict__ x, __nv_bfloat16*
 // entry and publishes it, then all rows subtract the rank-1 term from their remaining entries:
 // 63 - j independent FMAs per thread, no dependent chain.  The inverse is formed the same way,
 // column c of L^-1 in the registers of thread c: x_r = s_r / L_rr, then s_i -= L_ir x_r for i > r.
-__global__ void __launch_bounds__(64) potf2_inv_kernel(double* __restrict__ C, int ld, int nb, double* __restrict__ Linv,
+__device__ __forceinline__ double pivot_rsqrt(double x) { return rsqrt_newton(x); }
+__device__ __forceinline__ float pivot_rsqrt(float x) { return rsqrtf(x); }
+
+template <typename T>
+__global__ void __launch_bounds__(64) potf2_inv_kernel(T* __restrict__ C, int ld, int nb, T* __restrict__ Linv,
                                                        int32_t* __restrict__ status) {
-  __shared__ double Ls[64][65];
-  __shared__ double col[64];
-  __shared__ double rdiag[64];
+  __shared__ T Ls[64][65];
+  __shared__ T col[64];
+  __shared__ T rdiag[64];
   const int i = threadIdx.x;
   for (int r = 0; r < 64; ++r) {      // coalesced read of row r by the threads k <= r
-    double v = (r == i) ? 1.0 : 0.0;
+    T v = (r == i) ? T(1) : T(0);
     if (r < nb && i <= r) v = C[(int64_t)r * ld + i];
     Ls[r][i] = v;
   }
   __syncthreads();
-  double a[64];
+  T a[64];
 #pragma unroll
   for (int k = 0; k < 64; ++k) a[k] = Ls[i][k];
   __syncthreads();
 #pragma unroll
   for (int j = 0; j < 64; ++j) {
     if (i == j) {
-      double piv = a[j];
-      if (!(piv > 0.0)) {              // not positive definite: keep going with a usable pivot, latch the fact
+      T piv = a[j];
+      if (!(piv > T(0))) {             // not positive definite: keep going with a usable pivot, latch the fact
         atomicOr(status, GALORE_DEV_CHOLESKY);
-        piv = fabs(piv) + 1e-300;
+        piv = (T)(fabs((double)piv) + 1e-30);
       }
-      const double rs = rsqrt_newton(piv);
+      const T rs = pivot_rsqrt(piv);
       Ls[j][j] = piv * rs;
       rdiag[j] = rs;
     }
     __syncthreads();
-    double l = 0.0;
+    T l = T(0);
     if (i > j) {
       l = a[j] * rdiag[j];
       Ls[i][j] = l;
@@ -258,10 +257,10 @@ __global__ void __launch_bounds__(64) potf2_inv_kernel(double* __restrict__ C, i
   __syncthreads();
   // column i of L^-1
 #pragma unroll
-  for (int k = 0; k < 64; ++k) a[k] = (k == i) ? 1.0 : 0.0;
+  for (int k = 0; k < 64; ++k) a[k] = (k == i) ? T(1) : T(0);
 #pragma unroll
   for (int r = 0; r < 64; ++r) {
-    const double x = a[r] * rdiag[r];
+    const T x = a[r] * rdiag[r];
     a[r] = x;
 #pragma unroll
     for (int k = r + 1; k < 64; ++k) a[k] = fma(-Ls[k][r], x, a[k]);
@@ -273,7 +272,8 @@ __global__ void __launch_bounds__(64) potf2_inv_kernel(double* __restrict__ C, i
 }
 
 // diagonal 64 x 64 blocks of T <- the inverses of the diagonal blocks of L (slab p = block p)
-__global__ void place_diag_inverse_kernel(const double* __restrict__ slabs, int b, double* __restrict__ T) {
+template <typename S>
+__global__ void place_diag_inverse_kernel(const S* __restrict__ slabs, int b, S* __restrict__ T) {
   const int p = blockIdx.x, j0 = p * 64;
   const int nb = min(64, b - j0);
   for (int idx = threadIdx.x; idx < 64 * 64; idx += blockDim.x) {
@@ -512,27 +512,40 @@ static galore_status_t gram(const TY* Y, int64_t d, int b, double* C, cudaStream
 //   invert : the inverses of the diagonal blocks are merged pairwise, level by level,
 //            [T11 0; T21 T22] with T21 = -T22 L21 T11, every level two batched products.
 // scratch: b*b/4 doubles.
-static galore_status_t cholesky_inverse(double* C, int b, double* T, double* scratch, const RefreshBuffers& w,
-                                        int32_t* status, cudaStream_t st) {
+// (S = double: products on the fp64 MMA unit; S = float, used between the tensor-core power steps
+// whose Gram matrices carry about 16 bits anyway: FMA products and a ten times shorter pivot chain.)
+template <typename TA, typename TB, typename S, class Epi>
+static galore_status_t gemm_scalar(int M, int N, int K, const TA* A, int64_t sAi, int64_t sAk, const TB* B, int64_t sBk,
+                                   int64_t sBj, Epi epi, cudaStream_t st, int batch = 1, int64_t bA = 0, int64_t bB = 0) {
+  if constexpr (std::is_same<S, double>::value)
+    return launch_gemm_dmma<TA, TB>(M, N, K, A, sAi, sAk, B, sBk, sBj, epi, st, batch, bA, bB);
+  else
+    return launch_gemm_simt<TA, TB, float>(M, N, K, A, sAi, sAk, B, sBk, sBj, 1, epi, st, batch, bA, bB);
+}
+
+template <typename S>
+static galore_status_t cholesky_inverse(S* C, int b, S* T, S* scratch, const RefreshBuffers& w, int32_t* status,
+                                        cudaStream_t st) {
   const int nblk = (int)ceil_div(b, 64);
+  S* slabs = (S*)w.slabs;
   for (int p = 0; p < nblk; ++p) {
     const int j0 = p * 64, nb = std::min(64, b - j0), j1 = j0 + nb;
-    double* slab = w.slabs + (int64_t)p * 4096;
-    potf2_inv_kernel<<<1, 64, 0, st>>>(C + (int64_t)j0 * b + j0, b, nb, slab, status);
+    S* slab = slabs + (int64_t)p * 4096;
+    potf2_inv_kernel<S><<<1, 64, 0, st>>>(C + (int64_t)j0 * b + j0, b, nb, slab, status);
     GALORE_LAUNCH_CHECK();
     if (j1 < b) {
       const int rem = b - j1;
-      double* panel = C + (int64_t)j1 * b + j0;
+      S* panel = C + (int64_t)j1 * b + j0;
       // L[rest, J] = C[rest, J] Linv^T   (in place: one CTA column covers all nb columns)
-      EpiStore<double, double> epi{panel, b, 0, 1.0, 0.0};
-      GALORE_TRY((launch_gemm_dmma<double, double>(rem, nb, nb, panel, b, 1, slab, 1, 64, epi, st)));
+      EpiStore<S, S> epi{panel, b, 0, S(1), S(0)};
+      GALORE_TRY((gemm_scalar<S, S, S>(rem, nb, nb, panel, b, 1, slab, 1, 64, epi, st)));
       // C[rest, rest] -= L[rest, J] L[rest, J]^T
-      EpiStore<double, double> upd{C + (int64_t)j1 * b + j1, b, 0, -1.0, 1.0};
-      GALORE_TRY((launch_gemm_dmma<double, double>(rem, rem, nb, panel, b, 1, panel, 1, b, upd, st)));
+      EpiStore<S, S> upd{C + (int64_t)j1 * b + j1, b, 0, S(-1), S(1)};
+      GALORE_TRY((gemm_scalar<S, S, S>(rem, rem, nb, panel, b, 1, panel, 1, b, upd, st)));
     }
   }
-  GALORE_CUDA_TRY(cudaMemsetAsync(T, 0, sizeof(double) * b * b, st));
-  place_diag_inverse_kernel<<<nblk, 256, 0, st>>>(w.slabs, b, T);
+  GALORE_CUDA_TRY(cudaMemsetAsync(T, 0, sizeof(S) * b * b, st));
+  place_diag_inverse_kernel<S><<<nblk, 256, 0, st>>>(slabs, b, T);
   GALORE_LAUNCH_CHECK();
   for (int64_t s = 64; s < b; s *= 2) {
     const int64_t step = 2 * s * b + 2 * s;            // from one merged block to the next, in elements
@@ -543,16 +556,16 @@ static galore_status_t cholesky_inverse(double* C, int b, double* T, double* scr
       if (count == 0) continue;
       const int s2 = pass == 0 ? (int)s : tail;
       const int64_t o = pass == 0 ? 0 : (int64_t)full * 2 * s;
-      const double* L21 = C + (o + s) * b + o;
-      const double* T11 = T + o * b + o;
-      const double* T22 = T + (o + s) * b + (o + s);
-      double* T21 = T + (o + s) * b + o;
+      const S* L21 = C + (o + s) * b + o;
+      const S* T11 = T + o * b + o;
+      const S* T22 = T + (o + s) * b + (o + s);
+      S* T21 = T + (o + s) * b + o;
       // W = L21 T11
-      EpiStore<double, double> ew{scratch, s, s * s, 1.0, 0.0};
-      GALORE_TRY((launch_gemm_dmma<double, double>(s2, (int)s, (int)s, L21, b, 1, T11, b, 1, ew, st, count, step, step)));
+      EpiStore<S, S> ew{scratch, s, s * s, S(1), S(0)};
+      GALORE_TRY((gemm_scalar<S, S, S>(s2, (int)s, (int)s, L21, b, 1, T11, b, 1, ew, st, count, step, step)));
       // T21 = -T22 W
-      EpiStore<double, double> et{T21, b, step, -1.0, 0.0};
-      GALORE_TRY((launch_gemm_dmma<double, double>(s2, (int)s, s2, T22, b, 1, scratch, s, 1, et, st, count, step, s * s)));
+      EpiStore<S, S> et{T21, b, step, S(-1), S(0)};
+      GALORE_TRY((gemm_scalar<S, S, S>(s2, (int)s, s2, T22, b, 1, scratch, s, 1, et, st, count, step, s * s)));
     }
   }
   return GALORE_OK;
@@ -563,7 +576,7 @@ template <typename TY, typename TO>
 static galore_status_t orthonormalise(const TY* Y, TO* out, int64_t d, int b, const RefreshBuffers& w, int32_t* status,
                                       cudaStream_t st) {
   GALORE_TRY(gram(Y, d, b, w.C, st));
-  GALORE_TRY(cholesky_inverse(w.C, b, w.Vt, w.H, w, status, st));
+  GALORE_TRY(cholesky_inverse<double>(w.C, b, w.Vt, w.H, w, status, st));
   EpiStore<TO, double> epi{out, b, 0, 1.0, 0.0};
   return launch_gemm_dmma<TY, double>((int)d, b, b, Y, b, 1, w.Vt, 1, b, epi, st);
 }
@@ -592,11 +605,11 @@ static galore_status_t orth_tensor(TensorRefresh& t, const RefreshBuffers& w, in
   GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 1, w.Ylo, b, 1, b, b, (int)d, g1, b, t.status));
   GALORE_TRY(tensor_group_add_gemm(t.tg, w.Ylo, b, 1, w.Yhi, b, 1, b, b, (int)d, g2, b, t.status));
   GALORE_TRY(tensor_group_launch_project(t.tg, st));
-  gram_sum_kernel<<<grid_for(bb), 256, 0, st>>>(g0, g1, g2, w.C, bb);
+  gram_sum_kernel<<<grid_for(bb), 256, 0, st>>>(g0, g1, g2, (float*)w.C, bb);
   GALORE_LAUNCH_CHECK();
   // T = L^-1, split into a bf16 pair; as the second operand of Y L^-T it is read K-contiguous
-  GALORE_TRY(cholesky_inverse(w.C, b, w.Vt, w.H, w, t.status, st));
-  split_double_kernel<<<grid_for(bb), 256, 0, st>>>(w.Vt, w.Thi, w.Tlo, bb);
+  GALORE_TRY(cholesky_inverse<float>((float*)w.C, b, (float*)w.Vt, (float*)w.H, w, t.status, st));
+  split_kernel<<<grid_for(bb), 256, 0, st>>>((const float*)w.Vt, w.Thi, w.Tlo, bb);
   GALORE_LAUNCH_CHECK();
   const int m = t.master, s1 = (m + 1) % 3, s2 = (m + 2) % 3;
   tensor_group_reset(t.tg);   // Y T = hi Thi + hi Tlo + lo Thi
