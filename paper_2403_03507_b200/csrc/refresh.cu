@@ -221,16 +221,10 @@ __global__ void __launch_bounds__(64) potf2_inv_kernel(T* __restrict__ C, int ld
   __shared__ T col[64];
   __shared__ T rdiag[64];
   const int i = threadIdx.x;
-  for (int r = 0; r < 64; ++r) {      // coalesced read of row r by the threads k <= r
-    T v = (r == i) ? T(1) : T(0);
-    if (r < nb && i <= r) v = C[(int64_t)r * ld + i];
-    Ls[r][i] = v;
-  }
-  __syncthreads();
+  // row i straight into registers: 64 independent loads in flight (rows past nb continue the identity)
   T a[64];
 #pragma unroll
-  for (int k = 0; k < 64; ++k) a[k] = Ls[i][k];
-  __syncthreads();
+  for (int k = 0; k < 64; ++k) a[k] = (i < nb && k <= i) ? C[(int64_t)i * ld + k] : ((k == i) ? T(1) : T(0));
 #pragma unroll
   for (int j = 0; j < 64; ++j) {
     if (i == j) {
