@@ -125,12 +125,16 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
   s->scols = s->left ? c->n : r;
   s->nel = s->srows * s->scols;
   s->nblk = ceil_div(s->nel, s->q_block);
-  int over = c->refresh_oversample == 0 ? r : std::max(0, c->refresh_oversample);
-  s->block = (int)std::min<int64_t>(s->d, (int64_t)r + over);
-
   const bool eligible = tensor_path_eligible(*c);
   if (c->path == GALORE_PATH_TENSOR && !eligible) return GALORE_ERR_UNIMPLEMENTED;
   s->tensor_path = eligible && c->path != GALORE_PATH_FP32;
+  // Extra columns of the refresh block.  More of them mean fewer power steps but a larger dense
+  // eigenproblem (cubic in the block); where the steps run on the tensor cores they are cheap and
+  // half the rank (at least 256) balances the two, elsewhere the block is twice the rank.
+  int over = c->refresh_oversample;
+  if (over == 0) over = (s->tensor_path && r > 256) ? std::max(256, r / 2) : r;
+  over = std::max(0, over);
+  s->block = (int)std::min<int64_t>(s->d, (int64_t)r + over);
 
   // K slices of the projection: enough CTAs to fill the machine when R is small
   {
@@ -268,7 +272,7 @@ galore_status_t do_refresh(galore_layer* l, const void* G, int64_t ldg, cudaStre
   pr.p_dtype = l->cfg.p_dtype;
   pr.seed = l->cfg.seed;
   pr.tol = l->cfg.refresh_tol > 0.f ? (double)l->cfg.refresh_tol : 1e-4;
-  pr.max_iters = l->cfg.refresh_max_iters > 0 ? l->cfg.refresh_max_iters : 64;
+  pr.max_iters = l->cfg.refresh_max_iters > 0 ? l->cfg.refresh_max_iters : 96;
   pr.first_iters = 6;
   pr.use_tensor = l->tensor_path;
   galore_status_t s = refresh_projector(pr, l->refresh_ws, l->status, info, st);
