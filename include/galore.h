@@ -172,6 +172,17 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
 galore_status_t galore_refresh_projector(galore_layer_t* layer, const void* G, int64_t ldg, void* stream,
                                          galore_refresh_info_t* info);
 
+/* The same refresh for `count` layers, one after another on `stream` (Algorithm 1 refreshes
+ * every layer at the same steps), with `workspace` (device memory, 256-byte aligned, at least
+ * galore_refresh_query_bytes() of every layer) in place of each layer's own refresh workspace,
+ * so that layers which share their workspace can be refreshed through one call.
+ * infos: NULL or `count` records.  Stops at the first error; otherwise returns
+ * GALORE_WARN_NOT_CONVERGED if any layer reached its iteration cap. */
+galore_status_t galore_refresh_query_bytes(const galore_layer_t* layer, size_t* bytes);
+galore_status_t galore_refresh_batch(galore_layer_t* const* layers, const void* const* G, const int64_t* ldg,
+                                     int32_t count, void* workspace, size_t workspace_bytes, void* stream,
+                                     galore_refresh_info_t* infos);
+
 /* Releases the host handle.  Device buffers stay with the caller. */
 galore_status_t galore_free(galore_layer_t* layer);
 

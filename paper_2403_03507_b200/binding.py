@@ -71,6 +71,9 @@ _PROTOTYPES = {
                                     C.POINTER(C.c_void_p), C.POINTER(C.c_int64), C.c_int32, C.c_float, C.c_void_p,
                                     C.c_size_t, C.c_void_p]),
     "galore_refresh_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.POINTER(RefreshInfo)]),
+    "galore_refresh_query_bytes": (C.c_int, [C.c_void_p, C.POINTER(C.c_size_t)]),
+    "galore_refresh_batch": (C.c_int, [C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_int64), C.c_int32,
+                                       C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(RefreshInfo)]),
     "galore_free": (C.c_int, [C.c_void_p]),
     "galore_step_static": (C.c_int, [C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_float, C.c_double, C.c_double,
                                      C.c_double, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
@@ -305,6 +308,30 @@ class Layer:
         f = C.c_int32()
         _check(lib().galore_device_status(self.handle, C.byref(f), _stream_ptr(stream)), "galore_device_status")
         return f.value
+
+
+def galore_refresh_query_bytes(layer) -> int:
+    out = C.c_size_t(0)
+    _check(lib().galore_refresh_query_bytes(layer.handle, C.byref(out)), "galore_refresh_query_bytes")
+    return out.value
+
+
+def galore_refresh_batch(layers, Gs, stream=None, workspace=None):
+    """Refreshes the projectors of `layers` from `Gs`, one after another, through one shared workspace.
+
+    workspace: a uint8 CUDA tensor (allocated here when None).  Returns (status, infos).
+    """
+    n = len(layers)
+    need = max(galore_refresh_query_bytes(l) for l in layers)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=layers[0].device)
+    hs = (C.c_void_p * n)(*[l.handle.value for l in layers])
+    gp = (C.c_void_p * n)(*[g.data_ptr() for g in Gs])
+    lg = (C.c_int64 * n)(*[g.stride(0) for g in Gs])
+    infos = (RefreshInfo * n)()
+    st = _check(lib().galore_refresh_batch(hs, gp, lg, n, workspace.data_ptr(), workspace.numel(), _stream_ptr(stream),
+                                           infos), "galore_refresh_batch")
+    return st, list(infos)
 
 
 def galore_batch_query_bytes(layers) -> int:

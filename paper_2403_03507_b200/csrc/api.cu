@@ -2,6 +2,7 @@
 // checks and the launch sequence of one iteration of Algorithm 1.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -258,7 +259,8 @@ galore_status_t step_tensor(galore_layer* l, void* W, int64_t ldw, const void* G
   return tensor_back_project(&l->tc, l->cfg, l->left, W, ldw, lr * l->cfg.alpha, l->status, st);
 }
 
-galore_status_t do_refresh(galore_layer* l, const void* G, int64_t ldg, cudaStream_t st, galore_refresh_info_t* info) {
+galore_status_t do_refresh(galore_layer* l, const void* G, int64_t ldg, cudaStream_t st, galore_refresh_info_t* info,
+                           void* workspace = nullptr) {
   RefreshProblem pr;
   pr.G = G;
   pr.g_dtype = l->cfg.g_dtype;
@@ -275,7 +277,7 @@ galore_status_t do_refresh(galore_layer* l, const void* G, int64_t ldg, cudaStre
   pr.max_iters = l->cfg.refresh_max_iters > 0 ? l->cfg.refresh_max_iters : 96;
   pr.first_iters = 6;
   pr.use_tensor = l->tensor_path;
-  galore_status_t s = refresh_projector(pr, l->refresh_ws, l->status, info, st);
+  galore_status_t s = refresh_projector(pr, workspace ? workspace : l->refresh_ws, l->status, info, st);
   if (s >= 0) l->has_projector = true;
   return s;
 }
@@ -363,6 +365,30 @@ galore_status_t galore_refresh_projector(galore_layer_t* l, const void* G, int64
   if (!l || !G) return GALORE_ERR_INVALID_ARG;
   if (ldg < l->cfg.n) return GALORE_ERR_INVALID_ARG;
   return do_refresh(l, G, ldg, (cudaStream_t)stream, info);
+}
+
+galore_status_t galore_refresh_query_bytes(const galore_layer_t* l, size_t* bytes) {
+  if (!l || !bytes) return GALORE_ERR_INVALID_ARG;
+  *bytes = refresh_workspace_bytes(l->d, l->L, l->cfg.rank, l->block);
+  return GALORE_OK;
+}
+
+galore_status_t galore_refresh_batch(galore_layer_t* const* layers, const void* const* G, const int64_t* ldg, int32_t count,
+                                     void* workspace, size_t workspace_bytes, void* stream, galore_refresh_info_t* infos) {
+  if (count < 0 || (count > 0 && (!layers || !G || !ldg || !workspace))) return GALORE_ERR_INVALID_ARG;
+  if ((uintptr_t)workspace & 255) return GALORE_ERR_INVALID_ARG;
+  for (int i = 0; i < count; ++i) {
+    if (!layers[i] || !G[i] || ldg[i] < layers[i]->cfg.n) return GALORE_ERR_INVALID_ARG;
+    if (refresh_workspace_bytes(layers[i]->d, layers[i]->L, layers[i]->cfg.rank, layers[i]->block) > workspace_bytes)
+      return GALORE_ERR_BUFFER_TOO_SMALL;
+  }
+  galore_status_t warn = GALORE_OK;
+  for (int i = 0; i < count; ++i) {
+    const galore_status_t s = do_refresh(layers[i], G[i], ldg[i], (cudaStream_t)stream, infos ? &infos[i] : nullptr, workspace);
+    if (s < 0) return s;
+    if (s > warn) warn = s;
+  }
+  return warn;
 }
 
 galore_status_t galore_step(galore_layer_t* l, void* W, int64_t ldw, const void* G, int64_t ldg, float lr, void* stream) {

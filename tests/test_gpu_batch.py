@@ -126,3 +126,34 @@ def test_auto_refresh_inside_a_batch():
         gb.Batch(lb, Wb, G).galore_step_batch(1e-2)
     for w1, w2 in zip(Wa, Wb):
         assert rel_err(to_host(w2), to_host(w1)) < 5e-4
+
+
+def test_refresh_batch_matches_single_refreshes():
+    """galore_refresh_batch over a shared workspace gives the projectors of one-by-one refreshes.
+
+    The refresh is deterministic for a given seed, so the two agree to rounding of the stored dtype;
+    both are also checked against the oracle's subspace for a gapped spectrum.
+    """
+    shapes = [(256, 512, 32), (512, 256, 32), (384, 1000, 64), (640, 640, 64), (256, 1096, 64), (200, 304, 16)]
+    single, batched, Gs = [], [], []
+    for i, (m, n, r) in enumerate(shapes):
+        k = min(m, n)
+        spectrum = np.concatenate([np.linspace(2.0, 1.0, r), 0.2 * np.arange(1, k - r + 1, dtype=np.float64) ** -0.5])
+        G, U, V = wl.make_planted(m, n, 50 + i, spectrum, "bf16")
+        Gs.append(to_dev(G, "bf16", (n + 7) // 8 * 8))
+        for dst in (single, batched):
+            cfg = gb.make_config(m, n, r, auto_refresh=False, p_dtype="f32", seed=11 + i)
+            dst.append(gb.Layer(cfg))
+    for layer, G in zip(single, Gs):
+        st, _info = layer.galore_refresh_projector(G)
+        assert st == 0
+    st, infos = gb.galore_refresh_batch(batched, Gs)
+    assert st == 0 and len(infos) == len(shapes)
+    for (m, n, r), a, b_, G, info in zip(shapes, single, batched, Gs, infos):
+        Pa, Pb = a.get_projector().double().cpu().numpy(), b_.get_projector().double().cpu().numpy()
+        assert info.converged == 1
+        assert np.abs(Pa - Pb).max() < 1e-6
+        Gh = to_host(G)[:, :n]
+        side = "left" if m <= n else "right"
+        Po, _sv = go.top_r_projector(Gh, r, side, method="lapack")
+        assert go.largest_principal_angle(Po, Pb) < 1e-3
