@@ -388,22 +388,48 @@ __device__ __forceinline__ void store_n4<float>(float* dst, float a, float b, fl
   *reinterpret_cast<float4*>(dst) = make_float4(a, b, c, d);
 }
 
-template <typename TN, int EPT>
+// PADDED: R and N have rows of a.cols elements at pitches a.r_ld and a.n_ld (the state itself is
+// always contiguous).  The codes keep their 4-byte accesses; the four R and N elements of a run are
+// addressed one by one, and a run may continue on the next row.
+template <typename TN, int EPT, bool PADDED>
 __device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q8Tables& t) {
   static_assert(EPT % 4 == 0, "runs of four elements");
   constexpr int RUNS = EPT / 4;
   const AdamParams p = a.p;
   const int base = blk * (EPT * 256) + 4 * threadIdx.x;
-  const float* __restrict__ R = a.Rpart + base;
+  const float* __restrict__ R = a.Rpart + (PADDED ? 0 : base);
   uint8_t* __restrict__ Mc = a.Mc + base;
   uint8_t* __restrict__ Vc = a.Vc + base;
-  TN* __restrict__ Nout = (TN*)a.Nout + base;
+  TN* __restrict__ Nout = (TN*)a.Nout + (PADDED ? 0 : base);
   const float am_m = a.Mam[blk], am_v = a.Vam[blk];
   float4 r[RUNS];
   uint32_t cm[RUNS], cv[RUNS];
+  int run_row[PADDED ? RUNS : 1], run_col[PADDED ? RUNS : 1];      // where each run starts
+  if (PADDED) {
+    int row = base / a.cols;
+    int col = base - row * a.cols;
+    const int adv_rows = 1024 / a.cols, adv_cols = 1024 - adv_rows * a.cols;   // from one run to the next
+#pragma unroll
+    for (int j = 0; j < RUNS; ++j) {
+      run_row[j] = row;
+      run_col[j] = col;
+      row += adv_rows;
+      col += adv_cols;
+      if (col >= a.cols) { col -= a.cols; ++row; }
+    }
+  }
+  // element k of run j in a buffer with row pitch ld
+  auto at = [&](int j, int k, int ld) {
+    const bool wrap = run_col[j] + k >= a.cols;
+    return (run_row[j] + (wrap ? 1 : 0)) * ld + run_col[j] + k - (wrap ? a.cols : 0);
+  };
 #pragma unroll
   for (int j = 0; j < RUNS; ++j) {
-    r[j] = *reinterpret_cast<const float4*>(R + j * 1024);
+    if (PADDED) {
+      r[j] = make_float4(R[at(j, 0, a.r_ld)], R[at(j, 1, a.r_ld)], R[at(j, 2, a.r_ld)], R[at(j, 3, a.r_ld)]);
+    } else {
+      r[j] = *reinterpret_cast<const float4*>(R + j * 1024);
+    }
     cm[j] = *reinterpret_cast<const uint32_t*>(Mc + j * 1024);
     cv[j] = *reinterpret_cast<const uint32_t*>(Vc + j * 1024);
   }
@@ -411,7 +437,9 @@ __device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q
     const float* __restrict__ part = R + (int64_t)s * a.split_stride;
 #pragma unroll
     for (int j = 0; j < RUNS; ++j) {
-      const float4 q = *reinterpret_cast<const float4*>(part + j * 1024);
+      float4 q;
+      if (PADDED) q = make_float4(part[at(j, 0, a.r_ld)], part[at(j, 1, a.r_ld)], part[at(j, 2, a.r_ld)], part[at(j, 3, a.r_ld)]);
+      else q = *reinterpret_cast<const float4*>(part + j * 1024);
       r[j].x += q.x; r[j].y += q.y; r[j].z += q.z; r[j].w += q.w;
     }
   }
@@ -431,7 +459,12 @@ __device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q
       mx_m = fmaxf(mx_m, fabsf(m[e]));
       mx_v = fmaxf(mx_v, v[e]);
     }
-    store_n4<TN>(Nout + j * 1024, nn[0], nn[1], nn[2], nn[3]);
+    if (PADDED) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) Nout[at(j, k, a.n_ld)] = cvt<TN>(nn[k]);
+    } else {
+      store_n4<TN>(Nout + j * 1024, nn[0], nn[1], nn[2], nn[3]);
+    }
   }
   block_max2_256(mx_m, mx_v, t.red);
   const float inv_m = 1.0f / mx_m, inv_v = 1.0f / mx_v;
@@ -485,7 +518,8 @@ __global__ void __launch_bounds__(256, 4) adam_q8_kernel(const __grid_constant__
     const bool full = (blk + 1) * (EPT * 256) <= a.nel;
     bool bad;
     if constexpr (EPT % 4 == 0) {
-      bad = (packed && full && a.aligned16) ? adam_q8_block_full<TN, EPT>(a, blk, t)
+      bad = (packed && full && a.aligned16) ? adam_q8_block_full<TN, EPT, false>(a, blk, t)
+            : (full && a.aligned16 && a.cols >= 4) ? adam_q8_block_full<TN, EPT, true>(a, blk, t)
             : packed                        ? adam_q8_block<TN, EPT, true>(a, blk, t)
                                             : adam_q8_block<TN, EPT, false>(a, blk, t);
     } else {
