@@ -157,3 +157,39 @@ def test_refresh_batch_matches_single_refreshes():
         side = "left" if m <= n else "right"
         Po, _sv = go.top_r_projector(Gh, r, side, method="lapack")
         assert go.largest_principal_angle(Po, Pb) < 1e-3
+
+
+def test_full_size_7b_matrices_in_the_benched_configuration():
+    """Two 4096 x 11008 matrices (and their transposed shape) at rank 1024 with 8-bit states, stepped by
+    galore_step_batch exactly as bench.py does (CTA-pair GEMMs, grouped launches), against the oracle."""
+    w = wl.WORKLOADS["llama_7b_q8"]
+    r = w.rank
+    shapes = [(4096, 11008), (11008, 4096)]
+    layers, Ws, Gd, orcs, W0s, Gh = [], [], [], [], [], []
+    for i, (m, n) in enumerate(shapes):
+        G = wl.make_gradient(m, n, wl.sub_seed(w.seed, i), w.spectrum_p, w.noise, "bf16")
+        W0 = wl.make_weight(m, n, 40 + i, "bf16")
+        d = min(m, n)
+        P = wl.round_to(wl.random_orthonormal(d, r, np.random.default_rng(i)), "bf16")
+        cfg = gb.make_config(m, n, r, alpha=w.alpha, refresh_gap=w.refresh_gap, state_fmt="q8", q_block=w.q_block,
+                             auto_refresh=False)
+        layer = gb.Layer(cfg)
+        assert layer.uses_tensor_path
+        layer.set_projector(torch.from_numpy(P))
+        o = go.GaLoreOracle(m, n, r, w.alpha, w.refresh_gap, w_store="bf16", state="q8", q_block=w.q_block, n_store="bf16")
+        o.set_projector(P)
+        ld = (n + 15) // 16 * 16
+        layers.append(layer); orcs.append(o); W0s.append(W0); Gh.append(G)
+        Ws.append(to_dev(W0, "bf16", ld)); Gd.append(to_dev(G, "bf16", ld))
+    batch = gb.Batch(layers, Ws, Gd)
+    Wo = list(W0s)
+    for s in range(2):
+        batch.galore_step_batch(w.lr)
+        Wo = [o.step(x, g, w.lr, auto_refresh=False) for o, x, g in zip(orcs, Wo, Gh)]
+    for layer, w_gpu, w_orc, w0, o in zip(layers, Ws, Wo, W0s, orcs):
+        assert layer.device_status() == 0 and layer.step_count == 2
+        assert rel_err(to_host(w_gpu), w_orc) <= 2e-2
+        assert rel_err(to_host(w_gpu) - w0, w_orc - w0) <= 5e-2
+        M, V = layer.get_moments()
+        Mo, Vo = o.moments()
+        assert rel_err(to_host(M), Mo) < 2e-2 and rel_err(to_host(V), Vo) < 2e-2
