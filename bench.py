@@ -427,23 +427,44 @@ def time_workload(w, args, dev, dist, world, rank, full):
 
     # ---- end to end through the host-buffer entry point -------------------------------------------
     if not args.no_e2e:
+        # pinned host copies: four sets per distinct shape, taken in turn, so that layers in flight
+        # together (three staging slots) never share a host buffer
         host = {}
         for (m, n, _c) in w.shapes:
-            hw = torch.empty(m, n, dtype=tdt[w.w_dtype]).pin_memory()
-            hg = torch.empty(m, n, dtype=tdt[w.g_dtype]).pin_memory()
-            hw.normal_(0, 0.02)
-            hg.normal_(0, 0.05)
-            dw = torch.empty(m, n, dtype=tdt[w.w_dtype], device=dev)
-            dg = torch.empty(m, n, dtype=tdt[w.g_dtype], device=dev)
-            host[(m, n)] = (hw, hg, dw, dg)
+            sets = []
+            for j in range(4):
+                hw = torch.empty(m, n, dtype=tdt[w.w_dtype]).pin_memory()
+                hg = torch.empty(m, n, dtype=tdt[w.g_dtype]).pin_memory()
+                hw.normal_(0, 0.02)
+                hg.normal_(0, 0.05)
+                sets.append((hw, hg))
+            host[(m, n)] = sets
+        turn = {}
+        W_hosts, G_hosts = [], []
+        for sh in shapes_of:
+            j = turn.get(sh, 0)
+            turn[sh] = j + 1
+            hw, hg = host[sh][j % 4]
+            W_hosts.append(hw)
+            G_hosts.append(hg)
         e2e_steps = max(1, min(args.steps, 3))
         h2d = sum(m * n * (elem_bytes(w.w_dtype) + elem_bytes(w.g_dtype)) for (m, n) in shapes_of)
         d2h = sum(m * n * elem_bytes(w.w_dtype) for (m, n) in shapes_of)
+        if args.mode == "batch":
+            hb = gb.HostBatch(layers, W_hosts, G_hosts, slots=3, device=dev)
+            e2e_call = "galore_step_host_batch, 3 staging slots"
 
-        def e2e_step():
-            for layer, sh in zip(layers, shapes_of):
-                hw, hg, dw, dg = host[sh]
-                layer.galore_step_host(hw, hg, dw, dg, w.lr, stream)
+            def e2e_step():
+                hb.galore_step_host_batch(w.lr, stream)
+        else:
+            dws = {sh: (torch.empty(sh[0], sh[1], dtype=tdt[w.w_dtype], device=dev),
+                        torch.empty(sh[0], sh[1], dtype=tdt[w.g_dtype], device=dev)) for sh in set(shapes_of)}
+            e2e_call = "galore_step_host per layer"
+
+            def e2e_step():
+                for layer, sh, hw, hg in zip(layers, shapes_of, W_hosts, G_hosts):
+                    dw, dg = dws[sh]
+                    layer.galore_step_host(hw, hg, dw, dg, w.lr, stream)
 
         e2e_step()
         barrier()
@@ -456,7 +477,8 @@ def time_workload(w, args, dev, dist, world, rank, full):
         ms = max_over_ranks(a.elapsed_time(b) / e2e_steps, dist, dev)
         out["e2e"] = {"value": world * w.params / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                       "d2h_bytes_per_step": d2h, "ms_per_step": ms, "steps": e2e_steps,
-                      "host_buffers": "one pinned W and G per distinct shape, reused by the layers of that shape"}
+                      "call": e2e_call,
+                      "host_buffers": "four pinned W and G per distinct shape, taken in turn by the layers of that shape"}
     flags = 0
     for layer in layers[:1]:
         flags |= layer.device_status()

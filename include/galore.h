@@ -163,6 +163,19 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
                                   const void* const* G, const int64_t* ldg, int32_t count, float lr,
                                   void* batch_ws, size_t batch_ws_bytes, void* stream);
 
+/* The step for a list of layers whose W and G live in pinned host memory (an optimizer state
+ * kept on the GPU for weights that are not).  (The paper has no counterpart: Algorithm 1 does not
+ * say where W lives.)  Layer i's W and G (row-major, rows of n elements, no padding) are copied into one
+ * of `slots` parts of `staging` (device memory, 256-byte aligned, galore_host_batch_query_bytes()),
+ * stepped there, and W is copied back.  Copies in, steps and copies out run on three streams (the
+ * steps on `stream`), so that both directions of the host link and the steps overlap across layers;
+ * 3 slots keep all three busy.  Asynchronous: work queued on `stream` after the call runs after
+ * the last copy out.  The host arrays must stay valid and untouched until then. */
+galore_status_t galore_host_batch_query_bytes(galore_layer_t* const* layers, int32_t count, int32_t slots, size_t* bytes);
+galore_status_t galore_step_host_batch(galore_layer_t* const* layers, void* const* W_host, const void* const* G_host,
+                                       int32_t count, float lr, void* staging, size_t staging_bytes, int32_t slots,
+                                       void* stream);
+
 /* Recomputes the projector as the top-r singular subspace of G (Eq. 12-13) by
  * block subspace iteration with a final Rayleigh-Ritz rotation, so that the
  * stored columns approximate singular vectors in descending order of

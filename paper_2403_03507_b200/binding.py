@@ -71,6 +71,9 @@ _PROTOTYPES = {
                                     C.POINTER(C.c_void_p), C.POINTER(C.c_int64), C.c_int32, C.c_float, C.c_void_p,
                                     C.c_size_t, C.c_void_p]),
     "galore_refresh_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.POINTER(RefreshInfo)]),
+    "galore_host_batch_query_bytes": (C.c_int, [C.POINTER(C.c_void_p), C.c_int32, C.c_int32, C.POINTER(C.c_size_t)]),
+    "galore_step_host_batch": (C.c_int, [C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.c_int32,
+                                         C.c_float, C.c_void_p, C.c_size_t, C.c_int32, C.c_void_p]),
     "galore_refresh_query_bytes": (C.c_int, [C.c_void_p, C.POINTER(C.c_size_t)]),
     "galore_refresh_batch": (C.c_int, [C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_int64), C.c_int32,
                                        C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(RefreshInfo)]),
@@ -308,6 +311,34 @@ class Layer:
         f = C.c_int32()
         _check(lib().galore_device_status(self.handle, C.byref(f), _stream_ptr(stream)), "galore_device_status")
         return f.value
+
+
+class HostBatch:
+    """Layers whose W and G stay in pinned host memory, stepped through galore_step_host_batch."""
+
+    def __init__(self, layers, W_hosts, G_hosts, slots: int = 3, device=None):
+        self.layers = list(layers)
+        self.n = len(self.layers)
+        self.slots = int(slots)
+        self.device = device if device is not None else self.layers[0].device
+        self._hs = (C.c_void_p * self.n)(*[l.handle.value for l in self.layers])
+        out = C.c_size_t(0)
+        _check(lib().galore_host_batch_query_bytes(self._hs, self.n, self.slots, C.byref(out)), "galore_host_batch_query_bytes")
+        self.staging = torch.empty(max(out.value, 256), dtype=torch.uint8, device=self.device)
+        self.rebind(W_hosts, G_hosts)
+
+    def rebind(self, W_hosts, G_hosts):
+        for t in list(W_hosts) + list(G_hosts):
+            if not (t.is_pinned() and t.is_contiguous()):
+                raise ValueError("host tensors must be pinned and contiguous")
+        self.W_hosts, self.G_hosts = list(W_hosts), list(G_hosts)
+        self._wp = (C.c_void_p * self.n)(*[w.data_ptr() for w in self.W_hosts])
+        self._gp = (C.c_void_p * self.n)(*[g.data_ptr() for g in self.G_hosts])
+
+    def galore_step_host_batch(self, lr: float, stream=None) -> int:
+        return _check(lib().galore_step_host_batch(self._hs, self._wp, self._gp, self.n, lr, self.staging.data_ptr(),
+                                                   self.staging.numel(), self.slots, _stream_ptr(stream)),
+                      "galore_step_host_batch")
 
 
 def galore_refresh_query_bytes(layer) -> int:

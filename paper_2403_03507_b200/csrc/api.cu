@@ -438,6 +438,103 @@ galore_status_t galore_step_host(galore_layer_t* l, void* W_host, const void* G_
   return s;
 }
 
+// ---- pipelined step for host-resident W and G -------------------------------------------------------
+namespace {
+
+int64_t staged_ld(const galore_layer* l) { return (l->cfg.n + 15) / 16 * 16; }   // 32-byte bf16 rows: TMA-addressable
+size_t staged_w_bytes(const galore_layer* l) { return align_up((size_t)l->cfg.m * staged_ld(l) * dtype_size(l->cfg.w_dtype), 256); }
+size_t staged_g_bytes(const galore_layer* l) { return align_up((size_t)l->cfg.m * staged_ld(l) * dtype_size(l->cfg.g_dtype), 256); }
+
+struct HostPipe {
+  int device = -1;
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr;
+  std::vector<cudaEvent_t> arrived, stepped, drained;   // per layer, per layer, per slot
+};
+
+galore_status_t host_pipe_prepare(HostPipe& hp, int dev, size_t layers, size_t slots) {
+  if (hp.device != dev) {
+    hp = HostPipe();
+    hp.device = dev;
+    GALORE_CUDA_TRY(cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking));
+    GALORE_CUDA_TRY(cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking));
+    GALORE_CUDA_TRY(cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming));
+  }
+  auto grow = [](std::vector<cudaEvent_t>& v, size_t n) -> galore_status_t {
+    while (v.size() < n) {
+      cudaEvent_t e;
+      GALORE_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+      v.push_back(e);
+    }
+    return GALORE_OK;
+  };
+  GALORE_TRY(grow(hp.arrived, layers));
+  GALORE_TRY(grow(hp.stepped, layers));
+  GALORE_TRY(grow(hp.drained, slots));
+  return GALORE_OK;
+}
+
+}  // namespace
+
+galore_status_t galore_host_batch_query_bytes(galore_layer_t* const* layers, int32_t count, int32_t slots, size_t* bytes) {
+  if (!layers || !bytes || count < 0 || slots < 1) return GALORE_ERR_INVALID_ARG;
+  size_t one = 0;
+  for (int i = 0; i < count; ++i) {
+    if (!layers[i]) return GALORE_ERR_INVALID_ARG;
+    one = std::max(one, staged_w_bytes(layers[i]) + staged_g_bytes(layers[i]));
+  }
+  *bytes = one * (size_t)slots;
+  return GALORE_OK;
+}
+
+galore_status_t galore_step_host_batch(galore_layer_t* const* layers, void* const* W_host, const void* const* G_host,
+                                       int32_t count, float lr, void* staging, size_t staging_bytes, int32_t slots,
+                                       void* stream) {
+  if (count < 0 || slots < 1 || (count > 0 && (!layers || !W_host || !G_host || !staging))) return GALORE_ERR_INVALID_ARG;
+  if (count == 0) return GALORE_OK;
+  if ((uintptr_t)staging & 255) return GALORE_ERR_INVALID_ARG;
+  size_t need = 0;
+  GALORE_TRY(galore_host_batch_query_bytes(layers, count, slots, &need));
+  if (need > staging_bytes) return GALORE_ERR_BUFFER_TOO_SMALL;
+  const size_t slot_bytes = need / (size_t)slots;
+  for (int i = 0; i < count; ++i)
+    if (!W_host[i] || !G_host[i]) return GALORE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int dev = 0;
+  GALORE_CUDA_TRY(cudaGetDevice(&dev));
+  static thread_local HostPipe hp;
+  GALORE_TRY(host_pipe_prepare(hp, dev, (size_t)count, (size_t)slots));
+  // Three lanes: copies in (hp.in), steps (the caller's stream), copies out (hp.out).  A slot of the
+  // staging buffer is filled, stepped and drained in turn; events hand it from lane to lane, so the
+  // two directions of the host link and the steps of different layers overlap.
+  GALORE_CUDA_TRY(cudaEventRecord(hp.start, st));
+  GALORE_CUDA_TRY(cudaStreamWaitEvent(hp.in, hp.start, 0));
+  galore_status_t warn = GALORE_OK;
+  for (int i = 0; i < count; ++i) {
+    galore_layer* l = layers[i];
+    const int slot = i % slots;
+    char* dW = (char*)staging + (size_t)slot * slot_bytes;
+    char* dG = dW + staged_w_bytes(l);
+    const int64_t ld = staged_ld(l);
+    const size_t we = dtype_size(l->cfg.w_dtype), ge = dtype_size(l->cfg.g_dtype);
+    const size_t wrow = (size_t)l->cfg.n * we, grow = (size_t)l->cfg.n * ge;
+    if (i >= slots) GALORE_CUDA_TRY(cudaStreamWaitEvent(hp.in, hp.drained[slot], 0));
+    GALORE_CUDA_TRY(cudaMemcpy2DAsync(dW, (size_t)ld * we, W_host[i], wrow, wrow, (size_t)l->cfg.m, cudaMemcpyHostToDevice, hp.in));
+    GALORE_CUDA_TRY(cudaMemcpy2DAsync(dG, (size_t)ld * ge, G_host[i], grow, grow, (size_t)l->cfg.m, cudaMemcpyHostToDevice, hp.in));
+    GALORE_CUDA_TRY(cudaEventRecord(hp.arrived[i], hp.in));
+    GALORE_CUDA_TRY(cudaStreamWaitEvent(st, hp.arrived[i], 0));
+    const galore_status_t s = galore_step(l, dW, ld, dG, ld, lr, stream);
+    if (s < 0) return s;
+    if (s > warn) warn = s;
+    GALORE_CUDA_TRY(cudaEventRecord(hp.stepped[i], st));
+    GALORE_CUDA_TRY(cudaStreamWaitEvent(hp.out, hp.stepped[i], 0));
+    GALORE_CUDA_TRY(cudaMemcpy2DAsync(W_host[i], wrow, dW, (size_t)ld * we, wrow, (size_t)l->cfg.m, cudaMemcpyDeviceToHost, hp.out));
+    GALORE_CUDA_TRY(cudaEventRecord(hp.drained[slot], hp.out));
+  }
+  for (int j = 0; j < std::min<int>(slots, count); ++j) GALORE_CUDA_TRY(cudaStreamWaitEvent(st, hp.drained[j], 0));
+  return warn;
+}
+
 // ---- batched step --------------------------------------------------------------------------------
 namespace {
 

@@ -193,3 +193,29 @@ def test_full_size_7b_matrices_in_the_benched_configuration():
         M, V = layer.get_moments()
         Mo, Vo = o.moments()
         assert rel_err(to_host(M), Mo) < 2e-2 and rel_err(to_host(V), Vo) < 2e-2
+
+
+@pytest.mark.parametrize("slots", [1, 3])
+def test_host_resident_batch_equals_device_steps(slots):
+    """galore_step_host_batch (W and G in pinned host memory, staged through `slots` device buffers) leaves
+    the same W as galore_step on device tensors with the same row pitch."""
+    layers_h, Wh, _, W0s = _make("q8", "bf16")
+    layers_d, Wd, _, _ = _make("q8", "bf16")
+    Wd = [to_dev(w0, "bf16", (w0.shape[1] + 15) // 16 * 16) for w0 in W0s]
+    W_host = [torch.from_numpy(np.ascontiguousarray(w0)).to(torch.bfloat16).pin_memory() for w0 in W0s]
+    hb = None
+    for s in range(3):
+        Gh, _ = _grads(s)
+        G_host = [torch.from_numpy(np.ascontiguousarray(g)).to(torch.bfloat16).pin_memory() for g in Gh]
+        if hb is None:
+            hb = gb.HostBatch(layers_h, W_host, G_host, slots=slots)
+        else:
+            hb.rebind(W_host, G_host)
+        hb.galore_step_host_batch(1e-2)
+        torch.cuda.synchronize()
+        for l, w, g in zip(layers_d, Wd, Gh):
+            l.galore_step(w, to_dev(g, "bf16", (g.shape[1] + 15) // 16 * 16), 1e-2)
+    torch.cuda.synchronize()
+    for l, wh, wd in zip(layers_h, W_host, Wd):
+        assert l.step_count == 3 and l.device_status() == 0
+        assert torch.equal(wh, wd.cpu())
