@@ -202,8 +202,10 @@ __global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* _
                                                                  int round, double tol, double* __restrict__ rot_out,
                                                                  int* __restrict__ flags, int* __restrict__ rotations) {
   extern __shared__ __align__(16) double jb_smem[];
-  double* Abuf[2] = {jb_smem, jb_smem + kPairRows * kALd};
-  double* Rbuf[2] = {jb_smem + 2 * kPairRows * kALd, jb_smem + 3 * kPairRows * kALd};
+  // the two copies of A, then the two copies of Rot (addresses computed, not looked up: an array of
+  // pointers indexed by the round would live in local memory)
+  auto Abuf = [&](int which) { return jb_smem + which * (kPairRows * kALd); };
+  auto Rbuf = [&](int which) { return jb_smem + (2 + which) * (kPairRows * kALd); };
   __shared__ double2 cs[kSlots];
   const int pair = blockIdx.x, tid = threadIdx.x;
   const BlockPair bp = block_pair(pair, round, nblk);
@@ -232,8 +234,8 @@ __global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* _
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int idx = tid + kSweepThreads * i;
-      Abuf[0][(idx >> 6) * kALd + (idx & 63)] = sum[i];
-      Rbuf[0][(idx >> 6) * kALd + (idx & 63)] = ((idx >> 6) == (idx & 63)) ? 1.0 : 0.0;
+      Abuf(0)[(idx >> 6) * kALd + (idx & 63)] = sum[i];
+      Rbuf(0)[(idx >> 6) * kALd + (idx & 63)] = ((idx >> 6) == (idx & 63)) ? 1.0 : 0.0;
     }
   }
   const BlockTask t0 = make_block_task(tid);                                   // tasks 0 .. 511
@@ -247,10 +249,10 @@ __global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* _
   int applied = 0;
   const double tol2 = tol * tol;
   for (int rr = 0; rr < kSweepRounds; ++rr) {
-    const double* Ac = Abuf[rr & 1];
-    double* An = Abuf[(rr + 1) & 1];
-    const double* Rc = Rbuf[rr & 1];
-    double* Rn = Rbuf[(rr + 1) & 1];
+    const double* Ac = Abuf(rr & 1);
+    double* An = Abuf((rr + 1) & 1);
+    const double* Rc = Rbuf(rr & 1);
+    double* Rn = Rbuf((rr + 1) & 1);
     if (tid < kSlots) {
       const int f = tid, g = kPairRows - 1 - tid;
       const double app = Ac[f * kALd + f], aqq = Ac[g * kALd + g], apq = Ac[f * kALd + g];
@@ -305,7 +307,7 @@ __global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* _
   }
   __syncthreads();
   if (cs[0].x != 0.0) {   // all rows are back at their own positions after the 63 rounds
-    const double* Rf = Rbuf[kSweepRounds & 1];
+    const double* Rf = Rbuf(kSweepRounds & 1);
     double* out = rot_out + (int64_t)pair * (kPairRows * kPairRows);
     for (int idx = tid; idx < kPairRows * kPairRows; idx += kSweepThreads) out[idx] = Rf[(idx >> 6) * kALd + (idx & 63)];
   }
