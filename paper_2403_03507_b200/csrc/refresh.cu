@@ -796,7 +796,7 @@ static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, 
         GALORE_LAUNCH_CHECK();
       }
       int sweeps = 0;
-      GALORE_TRY(jacobi_eigh(w.H, with_vt ? w.Vt : nullptr, b, w.jac, w.counter, 1e-13, 40, &sweeps, st));
+      GALORE_TRY(jacobi_eigh(w.H, with_vt ? w.Vt : nullptr, b, w.jac, w.counter, 1e-11, 40, &sweeps, st));
       local.jacobi_sweeps = sweeps;
       row_norm_kernel<<<b, 256, 0, st>>>(w.H, b, w.lam);
       GALORE_LAUNCH_CHECK();
