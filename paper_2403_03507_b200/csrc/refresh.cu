@@ -206,29 +206,37 @@ __global__ void split_kernel(const float* __restrict__ x, __nv_bfloat16* __restr
 // overwritten with L).  Linv: 64 x 64 row-major, lower triangular, zero elsewhere; rows and
 // columns past nb continue the identity.
 //
-// One thread per row, the row held in registers (every index below is a compile-time constant
-// after unrolling).  Column j: the owner of the pivot publishes 1/sqrt, every row below scales its
-// entry and publishes it, then all rows subtract the rank-1 term from their remaining entries:
-// 63 - j independent FMAs per thread, no dependent chain.  The inverse is formed the same way,
-// column c of L^-1 in the registers of thread c: x_r = s_r / L_rr, then s_i -= L_ir x_r for i > r.
+// Four threads per row: thread (row, part) keeps the 16 entries of its row in the columns
+// 4 q + part in registers, every index a compile-time constant after unrolling.  Column j: the
+// owner of the pivot publishes 1/sqrt, the rows below scale their entry and publish it, then
+// every thread subtracts the rank-1 term from its entries right of j -- independent FMAs, no
+// dependent chain.  The inverse is formed the same way: the threads of column c keep the running
+// right-hand side of column c of L^-1, x_r = s_r / L_rr goes through shared memory to the other
+// three parts, then s_k -= L_kr x_r for k > r.  (One thread per row with 64 entries each made
+// the kernel four times longer in instructions, all executed once: it waited on instruction
+// fetch.)
 __device__ __forceinline__ double pivot_rsqrt(double x) { return rsqrt_newton(x); }
 __device__ __forceinline__ float pivot_rsqrt(float x) { return rsqrtf(x); }
 
 template <typename T>
-__global__ void __launch_bounds__(64) potf2_inv_kernel(T* __restrict__ C, int ld, int nb, T* __restrict__ Linv,
-                                                       int32_t* __restrict__ status) {
-  __shared__ T Ls[64][65];
+__global__ void __launch_bounds__(256) potf2_inv_kernel(T* __restrict__ C, int ld, int nb, T* __restrict__ Linv,
+                                                        int32_t* __restrict__ status) {
+  __shared__ T Ls[64][65];       // the factor: needed again for the inverse and for the write-back
   __shared__ T col[64];
   __shared__ T rdiag[64];
-  const int i = threadIdx.x;
-  // row i straight into registers: 64 independent loads in flight (rows past nb continue the identity)
-  T a[64];
+  __shared__ T xs[2][64];
+  const int row = threadIdx.x & 63, part = threadIdx.x >> 6;
+  T a[16];
 #pragma unroll
-  for (int k = 0; k < 64; ++k) a[k] = (i < nb && k <= i) ? C[(int64_t)i * ld + k] : ((k == i) ? T(1) : T(0));
+  for (int q = 0; q < 16; ++q) {
+    const int k = 4 * q + part;
+    a[q] = (row < nb && k <= row) ? C[(int64_t)row * ld + k] : ((k == row) ? T(1) : T(0));
+  }
 #pragma unroll
   for (int j = 0; j < 64; ++j) {
-    if (i == j) {
-      T piv = a[j];
+    const int pj = j & 3, qj = j >> 2;
+    if (row == j && part == pj) {
+      T piv = a[qj];
       if (!(piv > T(0))) {             // not positive definite: keep going with a usable pivot, latch the fact
         atomicOr(status, GALORE_DEV_CHOLESKY);
         piv = (T)(fabs((double)piv) + 1e-30);
@@ -238,31 +246,46 @@ __global__ void __launch_bounds__(64) potf2_inv_kernel(T* __restrict__ C, int ld
       rdiag[j] = rs;
     }
     __syncthreads();
-    T l = T(0);
-    if (i > j) {
-      l = a[j] * rdiag[j];
-      Ls[i][j] = l;
+    if (part == pj) {
+      T l = T(0);
+      if (row > j) {
+        l = a[qj] * rdiag[j];
+        Ls[row][j] = l;
+      }
+      col[row] = l;
     }
-    col[i] = l;
     __syncthreads();
+    const T l = col[row];
 #pragma unroll
-    for (int k = j + 1; k < 64; ++k) a[k] = fma(-l, col[k], a[k]);
+    for (int q = qj; q < 16; ++q) {
+      if (q > qj || part > pj) a[q] = fma(-l, col[4 * q + part], a[q]);
+    }
   }
   __syncthreads();
-  // column i of L^-1
+  // column `row` of L^-1, entries 4 q + part
 #pragma unroll
-  for (int k = 0; k < 64; ++k) a[k] = (k == i) ? T(1) : T(0);
+  for (int q = 0; q < 16; ++q) a[q] = (4 * q + part == row) ? T(1) : T(0);
 #pragma unroll
   for (int r = 0; r < 64; ++r) {
-    const T x = a[r] * rdiag[r];
-    a[r] = x;
+    const int pr = r & 3, qr = r >> 2;
+    if (part == pr) {
+      const T x = a[qr] * rdiag[r];
+      a[qr] = x;
+      xs[r & 1][row] = x;
+    }
+    __syncthreads();
+    const T x = xs[r & 1][row];
 #pragma unroll
-    for (int k = r + 1; k < 64; ++k) a[k] = fma(-Ls[k][r], x, a[k]);
+    for (int q = qr; q < 16; ++q) {
+      if (q > qr || part > pr) a[q] = fma(-Ls[4 * q + part][r], x, a[q]);
+    }
   }
 #pragma unroll
-  for (int r = 0; r < 64; ++r) Linv[r * 64 + i] = a[r];
-  for (int r = 0; r < nb; ++r)
-    if (i <= r) C[(int64_t)r * ld + i] = Ls[r][i];
+  for (int q = 0; q < 16; ++q) Linv[(4 * q + part) * 64 + row] = a[q];
+  for (int idx = threadIdx.x; idx < 64 * 64; idx += 256) {
+    const int r = idx >> 6, c = idx & 63;
+    if (r < nb && c <= r) C[(int64_t)r * ld + c] = Ls[r][c];
+  }
 }
 
 // diagonal 64 x 64 blocks of T <- the inverses of the diagonal blocks of L (slab p = block p)
@@ -525,7 +548,7 @@ static galore_status_t cholesky_inverse(S* C, int b, S* T, S* scratch, const Ref
   for (int p = 0; p < nblk; ++p) {
     const int j0 = p * 64, nb = std::min(64, b - j0), j1 = j0 + nb;
     S* slab = slabs + (int64_t)p * 4096;
-    potf2_inv_kernel<S><<<1, 64, 0, st>>>(C + (int64_t)j0 * b + j0, b, nb, slab, status);
+    potf2_inv_kernel<S><<<1, 256, 0, st>>>(C + (int64_t)j0 * b + j0, b, nb, slab, status);
     GALORE_LAUNCH_CHECK();
     if (j1 < b) {
       const int rem = b - j1;
