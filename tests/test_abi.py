@@ -96,3 +96,18 @@ def test_codebooks_match_the_oracle_bit_for_bit():
     for signed in (True, False):
         lib_code = np.array(gb.galore_q8_codebook(signed), dtype=np.float32)
         assert np.array_equal(lib_code, go.dynamic_code(signed))
+
+
+def test_list_entry_points_validate_before_touching_the_device():
+    lib = gb.lib()
+    none = C.c_void_p(None)
+    out = C.c_size_t(7)
+    # empty lists are no-ops, negative counts and missing arrays are argument errors
+    assert lib.galore_refresh_batch(None, None, None, 0, none, 0, none, None) == 0
+    assert lib.galore_refresh_batch(None, None, None, -1, none, 0, none, None) == gb.ERR_INVALID_ARG
+    assert lib.galore_refresh_batch(None, None, None, 3, none, 0, none, None) == gb.ERR_INVALID_ARG
+    assert lib.galore_step_host_batch(None, None, None, 0, 1e-2, none, 0, 3, none) == 0
+    assert lib.galore_step_host_batch(None, None, None, 2, 1e-2, none, 0, 3, none) == gb.ERR_INVALID_ARG
+    assert lib.galore_step_host_batch(None, None, None, 0, 1e-2, none, 0, 0, none) == gb.ERR_INVALID_ARG
+    assert lib.galore_host_batch_query_bytes(None, 0, 3, C.byref(out)) == gb.ERR_INVALID_ARG
+    assert lib.galore_refresh_query_bytes(None, C.byref(out)) == gb.ERR_INVALID_ARG
