@@ -240,6 +240,12 @@ galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank, int32_t s
 
 /* Projector as fp32, rows x r row-major packed (rows = m left, n right), device memory. */
 galore_status_t galore_get_projector(galore_layer_t* layer, float* dst, size_t dst_bytes, void* stream);
+/* Diagnostic: the projector of the last galore_refresh_projector() (or refresh inside galore_step) of
+ * this layer as it was before rounding to p_dtype, rows x rank doubles (device memory).  It is read
+ * from the layer's workspace: valid only until that workspace is used again (by this or by another
+ * layer that shares it); GALORE_ERR_STATE if the layer has not been refreshed through its own
+ * workspace.  The 1e-3 rad bound of the refresh is a statement about this matrix. */
+galore_status_t galore_get_unrounded_projector(galore_layer_t* layer, double* dst, size_t dst_bytes, void* stream);
 galore_status_t galore_set_projector(galore_layer_t* layer, const float* src, size_t src_bytes, void* stream);
 /* Stored (uncorrected) moments as fp32, shape of R row-major packed, device memory (8-bit states are dequantised). */
 galore_status_t galore_get_moments(galore_layer_t* layer, float* M, float* V, size_t bytes_each, void* stream);

@@ -82,6 +82,7 @@ _PROTOTYPES = {
                                      C.c_double, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                      C.c_void_p, C.c_int64, C.c_float, C.POINTER(C.c_int32), C.c_void_p]),
     "galore_get_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "galore_get_unrounded_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "galore_set_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "galore_get_moments": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "galore_get_q8_state": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -265,6 +266,14 @@ class Layer:
         return st, info
 
     # -- accessors ------------------------------------------------------------
+    def get_unrounded_projector(self, stream=None) -> torch.Tensor:
+        """fp64 projector of the last refresh before rounding to p_dtype (read it right after the refresh)."""
+        rows = self.cfg.m if self.side == SIDE_LEFT else self.cfg.n
+        out = torch.empty(rows, self.cfg.rank, dtype=torch.float64, device=self.device)
+        _check(lib().galore_get_unrounded_projector(self.handle, out.data_ptr(), out.numel() * 8, _stream_ptr(stream)),
+               "galore_get_unrounded_projector")
+        return out
+
     def get_projector(self, stream=None) -> torch.Tensor:
         out = torch.empty(self.proj_rows, self.cfg.rank, dtype=torch.float32, device=self.device)
         _check(lib().galore_get_projector(self.handle, out.data_ptr(), out.numel() * 4, _stream_ptr(stream)),

@@ -88,6 +88,7 @@ struct galore_layer {
   float* Rpart;
   void* Nbuf;
   void* refresh_ws;
+  bool refreshed_here = false;   // the last refresh ran in refresh_ws (its unrounded projector is still there)
   TensorPlan tc;         // tensor-map state of the tcgen05 path (unused on the fp32 path)
 };
 
@@ -279,6 +280,7 @@ galore_status_t do_refresh(galore_layer* l, const void* G, int64_t ldg, cudaStre
   pr.use_tensor = l->tensor_path;
   galore_status_t s = refresh_projector(pr, workspace ? workspace : l->refresh_ws, l->status, info, st);
   if (s >= 0) l->has_projector = true;
+  l->refreshed_here = (s >= 0 && workspace == nullptr);
   return s;
 }
 
@@ -790,6 +792,16 @@ galore_status_t galore_get_projector(galore_layer_t* l, float* dst, size_t dst_b
   cudaStream_t st = (cudaStream_t)stream;
   if (l->cfg.p_dtype == GALORE_BF16) return convert_copy((const __nv_bfloat16*)l->P, dst, count, st);
   GALORE_CUDA_TRY(cudaMemcpyAsync(dst, l->P, (size_t)count * 4, cudaMemcpyDeviceToDevice, st));
+  return GALORE_OK;
+}
+
+galore_status_t galore_get_unrounded_projector(galore_layer_t* l, double* dst, size_t dst_bytes, void* stream) {
+  if (!l || !dst) return GALORE_ERR_INVALID_ARG;
+  const int64_t count = l->d * l->cfg.rank;
+  if (dst_bytes < (size_t)count * 8) return GALORE_ERR_BUFFER_TOO_SMALL;
+  if (!l->refreshed_here) return GALORE_ERR_STATE;
+  const double* src = refresh_unrounded_projector(l->refresh_ws, l->d, l->L, l->cfg.rank, l->block);
+  GALORE_CUDA_TRY(cudaMemcpyAsync(dst, src, (size_t)count * 8, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
   return GALORE_OK;
 }
 

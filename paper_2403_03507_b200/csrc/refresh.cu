@@ -511,6 +511,10 @@ static RefreshBuffers layout(void* base, int64_t d, int64_t L, int r, int b) {
   return w;
 }
 
+const double* refresh_unrounded_projector(void* workspace, int64_t d, int64_t L, int r, int b) {
+  return layout(workspace, d, L, r, b).P64;
+}
+
 // ---------------------------------------------------------------------------
 // building blocks
 // ---------------------------------------------------------------------------

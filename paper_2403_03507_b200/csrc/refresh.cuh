@@ -25,6 +25,10 @@ struct RefreshProblem {
 // d = rows of the projector, L = the other dimension of G
 size_t refresh_workspace_bytes(int64_t d, int64_t L, int r, int b);
 
+// Where the last refresh through `workspace` left its projector before rounding to the stored
+// dtype: rows x rank doubles, row-major.  Valid until the workspace is written again.
+const double* refresh_unrounded_projector(void* workspace, int64_t d, int64_t L, int r, int b);
+
 // Synchronises the stream (reads Ritz values back to decide on convergence).
 galore_status_t refresh_projector(const RefreshProblem& pr, void* workspace, int32_t* status,
                                   galore_refresh_info_t* info, cudaStream_t st);
