@@ -200,6 +200,8 @@ def main():
     ap.add_argument("--projector", default="refresh", choices=["refresh", "random"],
                     help="refresh: one real refresh per distinct shape (timed, reported); random: a random orthonormal "
                          "projector (step timing does not depend on P's values; for short profiling runs)")
+    ap.add_argument("--rank", type=int, default=0, help="override the workload's rank (rank sweep on one shape)")
+    ap.add_argument("--state-fmt", default="", choices=["", "f32", "q8"], help="override the workload's state format")
     ap.add_argument("--refresh-only", action="store_true",
                     help="run the projector refresh of each distinct shape and print its timings; no step is timed "
                          "(for profiling the refresh on its own)")
@@ -211,6 +213,9 @@ def main():
 
     from paper_2403_03507_b200 import workloads as wl
     w = wl.WORKLOADS[args.workload]
+    if args.rank or args.state_fmt:
+        import dataclasses
+        w = dataclasses.replace(w, rank=args.rank or w.rank, state_fmt=args.state_fmt or w.state_fmt)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
