@@ -91,8 +91,8 @@ typedef struct {
   int32_t auto_refresh;    /* 1: galore_step refreshes P when (completed steps) mod T == 0 */
   int32_t path;            /* galore_path_t */
   /* refresh: block subspace iteration on a block of rank + refresh_oversample
-   * columns (clipped to min(m, n); 0 = default: rank more columns, or
-   * max(256, rank / 2) on the tensor path when rank > 256; negative = none),
+   * columns (clipped to min(m, n); 0 = default: max(256, rank / 2) on the
+   * tensor path, rank more columns elsewhere; negative = none),
    * stopped when the predicted subspace error (theta_b / theta_r)^iterations
    * falls below refresh_tol or after refresh_max_iters power iterations.
    * 0 = defaults (1e-4, 96). */

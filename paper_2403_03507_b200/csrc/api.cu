@@ -132,9 +132,10 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
   s->tensor_path = eligible && c->path != GALORE_PATH_FP32;
   // Extra columns of the refresh block.  More of them mean fewer power steps but a larger dense
   // eigenproblem (cubic in the block); where the steps run on the tensor cores they are cheap and
-  // half the rank (at least 256) balances the two, elsewhere the block is twice the rank.
+  // half the rank, at least 256, balances the two (a block only twice a small rank converges
+  // slowly on flat spectra); elsewhere the block is twice the rank.
   int over = c->refresh_oversample;
-  if (over == 0) over = (s->tensor_path && r > 256) ? std::max(256, r / 2) : r;
+  if (over == 0) over = s->tensor_path ? std::max(256, r / 2) : r;
   over = std::max(0, over);
   s->block = (int)std::min<int64_t>(s->d, (int64_t)r + over);
 
