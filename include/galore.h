@@ -24,6 +24,11 @@
  *   - A handle is used from one stream at a time.  Calls enqueue work on the
  *     given stream (a cudaStream_t passed as void*; NULL = default stream) and
  *     return without synchronising, except where stated.
+ *   - Work of different handles is meant to be queued on ONE stream per
+ *     device (the list entry points add internal streams of their own, joined
+ *     by events).  Driving several handles from several host threads on
+ *     several streams at once is not supported: refreshes run that way
+ *     stalled on the test machines, and the cause was not found.
  *   - Every entry point returns a galore_status_t: 0 ok, > 0 warning, < 0
  *     error.  Nothing throws or aborts across this boundary.  Conditions
  *     detected on the device (non-finite values, a bounded wait that ran out)
