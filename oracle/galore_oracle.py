@@ -250,7 +250,7 @@ class GaLoreOracle:
 
     def __init__(self, m, n, rank, alpha, refresh_gap, beta1=0.9, beta2=0.999, eps=1e-8,
                  side="auto", w_store="f64", state="f64", n_store="f64", q_block=2048,
-                 inner="adam", svd_method="jacobi"):
+                 inner="adam", svd_method="jacobi", weight_decay=0.0):
         if side == "auto":
             side = "left" if m <= n else "right"       # Sec. 4.2; m == n goes left
         if rank < 1 or rank > min(m, n):
@@ -260,6 +260,10 @@ class GaLoreOracle:
         self.beta1, self.beta2, self.eps = float(beta1), float(beta2), float(eps)
         self.side, self.w_store, self.state, self.n_store = side, w_store, state, n_store
         self.q_block, self.inner, self.svd_method = int(q_block), inner, svd_method
+        # GaLore-AdamW (Sec. "GaLore with memory-efficient optimizers" names AdamW, no equations):
+        # decoupled weight decay as Loshchilov & Hutter define it, W <- W (1 - lr lambda) - lr G~,
+        # applied to the full-rank weight with the plain learning rate (alpha scales only G~).
+        self.weight_decay = float(weight_decay)
         self.k = 0                                      # completed steps
         self.proj = None                                # P (m x r) or Q (n x r)
         self.sigma = None
@@ -337,6 +341,6 @@ class GaLoreOracle:
         self.last_R, self.last_N = R, N
         # project back and apply
         G_tilde = self.alpha * (P @ N if self.side == "left" else N @ P.T)
-        W_new = _store(W - lr * G_tilde, self.w_store)
+        W_new = _store(W * (1.0 - lr * self.weight_decay) - lr * G_tilde, self.w_store)
         self.k += 1
         return W_new

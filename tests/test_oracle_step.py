@@ -25,6 +25,29 @@ def _torch_adam(W0, grads, lr, beta1, beta2, eps):
     return out
 
 
+def test_identity_projector_with_weight_decay_is_library_adamw():
+    """GaLore-AdamW with P = I and alpha = 1 is element-wise AdamW (decoupled decay, an independent implementation)."""
+    m, n = 10, 16
+    W = wl.make_weight(m, n, 2, "f64")
+    grads = _grads(m, n, 6, seed=3)
+    lr, wd = 3e-2, 0.2
+    orc = go.GaLoreOracle(m, n, m, alpha=1.0, refresh_gap=100, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=wd)
+    orc.set_projector(np.eye(m))
+    w = torch.nn.Parameter(torch.from_numpy(W.copy()))
+    opt = torch.optim.AdamW([w], lr=lr, betas=(0.9, 0.999), eps=1e-8, weight_decay=wd)
+    for g in grads:
+        W = orc.step(W, g, lr, auto_refresh=False)
+        w.grad = torch.from_numpy(np.ascontiguousarray(g))
+        opt.step()
+        assert np.allclose(W, w.detach().numpy(), rtol=1e-12, atol=1e-14)
+    # the decay acts on W alone: with zero gradients W shrinks geometrically and the moments stay zero
+    orc2 = go.GaLoreOracle(m, n, 4, alpha=0.25, refresh_gap=100, weight_decay=wd)
+    orc2.set_projector(np.linalg.qr(np.random.default_rng(0).standard_normal((m, 4)))[0])
+    W2 = wl.make_weight(m, n, 5, "f64")
+    W3 = orc2.step(orc2.step(W2, np.zeros((m, n)), lr, auto_refresh=False), np.zeros((m, n)), lr, auto_refresh=False)
+    assert np.allclose(W3, W2 * (1 - lr * wd) ** 2, rtol=1e-14)
+
+
 def test_identity_projector_is_elementwise_adam():
     m, n = 12, 20
     W = wl.make_weight(m, n, 1, "f64")
