@@ -200,6 +200,8 @@ def main():
     ap.add_argument("--projector", default="refresh", choices=["refresh", "random"],
                     help="refresh: one real refresh per distinct shape (timed, reported); random: a random orthonormal "
                          "projector (step timing does not depend on P's values; for short profiling runs)")
+    ap.add_argument("--weight-decay", type=float, default=0.0,
+                    help="GaLore-AdamW: decoupled weight decay folded into the weight update (0 = plain Adam)")
     ap.add_argument("--rank", type=int, default=0, help="override the workload's rank (rank sweep on one shape)")
     ap.add_argument("--state-fmt", default="", choices=["", "f32", "q8"], help="override the workload's state format")
     ap.add_argument("--refresh-only", action="store_true",
@@ -274,7 +276,7 @@ def time_workload(w, args, dev, dist, world, rank, full):
     for (m, n, count) in w.shapes:
         cfg = gb.make_config(m, n, w.rank, alpha=w.alpha, refresh_gap=w.refresh_gap, beta1=w.beta1, beta2=w.beta2,
                              eps=w.eps, w_dtype=w.w_dtype, g_dtype=w.g_dtype, state_fmt=w.state_fmt,
-                             q_block=w.q_block, auto_refresh=False, seed=w.seed)
+                             q_block=w.q_block, auto_refresh=False, seed=w.seed, weight_decay=args.weight_decay)
         cfgs[(m, n)] = cfg
         max_ws = max(max_ws, gb.galore_query_bytes(cfg)[1])
     workspace = torch.empty(max_ws, dtype=torch.uint8, device=dev)      # shared: layers step one after another
@@ -412,7 +414,7 @@ def time_workload(w, args, dev, dist, world, rank, full):
         "dtype": "bf16" if uses_tc else "f32", "data": "synthetic",
         "config": {"workload": w.name, "matrices": w.matrices, "params": w.params, "rank": w.rank,
                    "state_fmt": w.state_fmt, "w_dtype": w.w_dtype, "g_dtype": w.g_dtype, "alpha": w.alpha,
-                   "refresh_gap": w.refresh_gap, "tensor_path": uses_tc, "mode": args.mode, "parallelism": f"replicas x{world}",
+                   "refresh_gap": w.refresh_gap, "weight_decay": args.weight_decay, "tensor_path": uses_tc, "mode": args.mode, "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (whole layer set streamed each step)"},
         "clocks": clocks, "gpu_launches": launches, "roofline": roof,
         "refresh": refresh_info,

@@ -105,7 +105,11 @@ typedef struct {
   int32_t refresh_max_iters;
   int32_t refresh_oversample;
   uint64_t seed;           /* start block of the subspace iteration */
-  int32_t reserved[8];
+  /* GaLore-AdamW: decoupled weight decay lambda >= 0 (0 = plain Adam).  The paper names AdamW as a
+   * supported optimizer without equations; the reading taken is Loshchilov & Hutter's:
+   * W <- W (1 - lr lambda) - lr alpha P N, the decay on the full-rank weight with the plain lr. */
+  float weight_decay;
+  int32_t reserved[7];
 } galore_config_t;
 
 /* Result of one refresh (host struct, filled after the refresh's stream work has completed). */

@@ -111,6 +111,7 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
   if (c->refresh_gap < 1) return GALORE_ERR_INVALID_ARG;
   if (!(c->beta1 >= 0.0 && c->beta1 < 1.0) || !(c->beta2 >= 0.0 && c->beta2 < 1.0) || !(c->eps >= 0.0))
     return GALORE_ERR_INVALID_ARG;
+  if (!(c->weight_decay >= 0.0f) || !(c->weight_decay < 1e6f)) return GALORE_ERR_INVALID_ARG;
   if (c->side < GALORE_SIDE_AUTO || c->side > GALORE_SIDE_RIGHT) return GALORE_ERR_INVALID_ARG;
   for (int32_t dt : {c->w_dtype, c->g_dtype, c->p_dtype})
     if (dt != GALORE_F32 && dt != GALORE_BF16) return GALORE_ERR_INVALID_ARG;
@@ -198,11 +199,14 @@ galore_status_t project_simt(galore_layer* l, const void* G, int64_t ldg, cudaSt
                                          l->proj_splits, epi, st);
 }
 
+// GaLore-AdamW: W is multiplied by 1 - lr * lambda in the pass that subtracts the update (exactly 1 for lambda = 0)
+inline float decay_keep(const galore_layer* l, float lr) { return (float)(1.0 - (double)lr * (double)l->cfg.weight_decay); }
+
 template <typename TP, typename TW>
-galore_status_t back_project_simt(galore_layer* l, void* W, int64_t ldw, float scale, cudaStream_t st) {
+galore_status_t back_project_simt(galore_layer* l, void* W, int64_t ldw, float scale, float keep, cudaStream_t st) {
   const int r = l->cfg.rank;
   const int m = (int)l->cfg.m, n = (int)l->cfg.n;
-  EpiApplyW<TW> epi{(TW*)W, ldw, scale};
+  EpiApplyW<TW> epi{(TW*)W, ldw, scale, keep};
   const float* N = (const float*)l->Nbuf;
   if (l->left)   // W -= scale * P N,  N is r x n
     return launch_gemm_simt<TP, float, float>(m, n, r, (const TP*)l->P, r, 1, N, n, 1, 1, epi, st);
@@ -229,11 +233,11 @@ galore_status_t step_simt(galore_layer* l, void* W, int64_t ldw, const void* G, 
                                 GALORE_F32, ap, l->status, st));
   }
   PhaseTimer pt(2, st);
-  const float scale = lr * l->cfg.alpha;
-  if (pb && wb) return back_project_simt<__nv_bfloat16, __nv_bfloat16>(l, W, ldw, scale, st);
-  if (pb) return back_project_simt<__nv_bfloat16, float>(l, W, ldw, scale, st);
-  if (wb) return back_project_simt<float, __nv_bfloat16>(l, W, ldw, scale, st);
-  return back_project_simt<float, float>(l, W, ldw, scale, st);
+  const float scale = lr * l->cfg.alpha, keep = decay_keep(l, lr);
+  if (pb && wb) return back_project_simt<__nv_bfloat16, __nv_bfloat16>(l, W, ldw, scale, keep, st);
+  if (pb) return back_project_simt<__nv_bfloat16, float>(l, W, ldw, scale, keep, st);
+  if (wb) return back_project_simt<float, __nv_bfloat16>(l, W, ldw, scale, keep, st);
+  return back_project_simt<float, float>(l, W, ldw, scale, keep, st);
 }
 
 // projection and back-projection on tcgen05, Adam in between reading the padded partials
@@ -258,7 +262,7 @@ galore_status_t step_tensor(galore_layer* l, void* W, int64_t ldw, const void* G
                                 l->Nbuf, GALORE_BF16, ap, l->status, st, g));
   }
   PhaseTimer pt(2, st);
-  return tensor_back_project(&l->tc, l->cfg, l->left, W, ldw, lr * l->cfg.alpha, l->status, st);
+  return tensor_back_project(&l->tc, l->cfg, l->left, W, ldw, lr * l->cfg.alpha, decay_keep(l, lr), l->status, st);
 }
 
 galore_status_t do_refresh(galore_layer* l, const void* G, int64_t ldg, cudaStream_t st, galore_refresh_info_t* info,
@@ -726,7 +730,7 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
       float* part; void* nbuf;
       scratch_of(gi, mb, &part, &nbuf);
       GALORE_TRY(tensor_group_add_back(scratch.back, &l->tc, l->cfg, l->left, nbuf, l->ld_n, W[mb.index], ldw[mb.index],
-                                       lr * l->cfg.alpha, l->status));
+                                       lr * l->cfg.alpha, decay_keep(l, lr), l->status));
     }
     PhaseTimer pt(2, s);
     GALORE_TRY(tensor_group_launch_back(scratch.back, first->cfg.w_dtype, s));

@@ -131,15 +131,17 @@ struct EpiStore {
   }
 };
 
-// W[i][j] <- W[i][j] - scale * acc   (the weight update that closes Algorithm 1)
+// W[i][j] <- keep * W[i][j] - scale * acc   (the weight update that closes Algorithm 1; keep =
+// 1 - lr * weight_decay for GaLore-AdamW, exactly 1 otherwise)
 template <typename TW>
 struct EpiApplyW {
   TW* W;
   int64_t ldw;
   float scale;
+  float keep = 1.0f;
   __device__ __forceinline__ void operator()(int i, int j, float acc, int) const {
     TW* p = W + (int64_t)i * ldw + j;
-    *p = cvt<TW>(fmaf(-scale, acc, cvt<float>(*p)));
+    *p = cvt<TW>(fmaf(-scale, acc, keep * cvt<float>(*p)));
   }
 };
 

@@ -52,7 +52,10 @@ struct Geo {
 };
 constexpr long long kWaitLimitCycles = 4000000000LL;   // about two seconds
 
-enum { EPI_PARTIAL = 0, EPI_APPLY = 1 };
+// EPI_APPLY_DECAY is EPI_APPLY with W multiplied by TcParams::keep first (GaLore-AdamW).  It is an
+// instantiation of its own: the same code with the multiply behind a run-time test made the plain
+// update 15 % slower at K = 512.
+enum { EPI_PARTIAL = 0, EPI_APPLY = 1, EPI_APPLY_DECAY = 2 };
 
 constexpr int kMaxGroup = 32;     // problems one launch can carry (its arguments travel as kernel parameters)
 
@@ -71,6 +74,7 @@ struct TcParams {
   int64_t ldw;
   int vec32;                  // W base and row pitch (resp. the partial buffer's) are 32-byte aligned
   float scale;
+  float keep;                 // EPI_APPLY_DECAY: W is multiplied by this before the update is subtracted
   int32_t* status;
 };
 
@@ -303,78 +307,51 @@ __device__ __forceinline__ void epi_partial(const TcParams& p, const Unit& w, in
   }
 }
 
-template <typename TW>
-__device__ __forceinline__ void epi_apply(const TcParams& p, int row, int col0, const uint32_t (&v)[32]);
+// w <- w - scale * acc, or keep * w - scale * acc (decoupled weight decay)
+template <bool DECAY>
+__device__ __forceinline__ float apply_one(float w, float acc, float scale, float keep) {
+  return DECAY ? fmaf(-scale, acc, keep * w) : fmaf(-scale, acc, w);
+}
 
-template <>
-__device__ __forceinline__ void epi_apply<__nv_bfloat16>(const TcParams& p, int row, int col0, const uint32_t (&v)[32]) {
+// one 16-byte vector of W
+template <typename TW, bool DECAY>
+__device__ __forceinline__ void apply_vec(uint4& raw, const uint32_t* acc, float scale, float keep) {
+  if constexpr (sizeof(TW) == 2) {
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      float2 f = __bfloat1622float2(h[q]);
+      f.x = apply_one<DECAY>(f.x, __uint_as_float(acc[2 * q]), scale, keep);
+      f.y = apply_one<DECAY>(f.y, __uint_as_float(acc[2 * q + 1]), scale, keep);
+      h[q] = __floats2bfloat162_rn(f.x, f.y);
+    }
+  } else {
+    float4* f = reinterpret_cast<float4*>(&raw);
+    f->x = apply_one<DECAY>(f->x, __uint_as_float(acc[0]), scale, keep);
+    f->y = apply_one<DECAY>(f->y, __uint_as_float(acc[1]), scale, keep);
+    f->z = apply_one<DECAY>(f->z, __uint_as_float(acc[2]), scale, keep);
+    f->w = apply_one<DECAY>(f->w, __uint_as_float(acc[3]), scale, keep);
+  }
+}
+
+// edge tiles: thread owns row `row`, columns [col0, col0 + 32) of the tile
+template <typename TW, bool DECAY>
+__device__ __forceinline__ void epi_apply(const TcParams& p, int row, int col0, const uint32_t (&v)[32]) {
   if (row >= p.M) return;
-  __nv_bfloat16* dst = (__nv_bfloat16*)p.W + (int64_t)row * p.ldw + col0;
+  TW* dst = (TW*)p.W + (int64_t)row * p.ldw + col0;
+  constexpr int kVec = 16 / (int)sizeof(TW);
   if (col0 + 32 <= p.N) {
 #pragma unroll
-    for (int j = 0; j < 32; j += 8) {
+    for (int j = 0; j < 32; j += kVec) {
       uint4 raw = *reinterpret_cast<const uint4*>(dst + j);
-      __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        float2 f = __bfloat1622float2(h[q]);
-        f.x = fmaf(-p.scale, __uint_as_float(v[j + 2 * q]), f.x);
-        f.y = fmaf(-p.scale, __uint_as_float(v[j + 2 * q + 1]), f.y);
-        h[q] = __floats2bfloat162_rn(f.x, f.y);
-      }
+      apply_vec<TW, DECAY>(raw, &v[j], p.scale, p.keep);
       *reinterpret_cast<uint4*>(dst + j) = raw;
     }
   } else {
 #pragma unroll
     for (int j = 0; j < 32; ++j)
-      if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(fmaf(-p.scale, __uint_as_float(v[j]), __bfloat162float(dst[j])));
+      if (col0 + j < p.N) dst[j] = cvt<TW>(apply_one<DECAY>(cvt<float>(dst[j]), __uint_as_float(v[j]), p.scale, p.keep));
   }
-}
-
-template <>
-__device__ __forceinline__ void epi_apply<float>(const TcParams& p, int row, int col0, const uint32_t (&v)[32]) {
-  if (row >= p.M) return;
-  float* dst = (float*)p.W + (int64_t)row * p.ldw + col0;
-  if (col0 + 32 <= p.N) {
-#pragma unroll
-    for (int j = 0; j < 32; j += 4) {
-      float4 f = *reinterpret_cast<const float4*>(dst + j);
-      f.x = fmaf(-p.scale, __uint_as_float(v[j]), f.x);
-      f.y = fmaf(-p.scale, __uint_as_float(v[j + 1]), f.y);
-      f.z = fmaf(-p.scale, __uint_as_float(v[j + 2]), f.z);
-      f.w = fmaf(-p.scale, __uint_as_float(v[j + 3]), f.w);
-      *reinterpret_cast<float4*>(dst + j) = f;
-    }
-  } else {
-#pragma unroll
-    for (int j = 0; j < 32; ++j)
-      if (col0 + j < p.N) dst[j] = fmaf(-p.scale, __uint_as_float(v[j]), dst[j]);
-  }
-}
-
-// one 16-byte vector of W: w <- w - scale * acc
-template <typename TW>
-__device__ __forceinline__ void apply_vec(uint4& raw, const uint32_t* acc, float scale);
-
-template <>
-__device__ __forceinline__ void apply_vec<__nv_bfloat16>(uint4& raw, const uint32_t* acc, float scale) {
-  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw);
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    float2 f = __bfloat1622float2(h[q]);
-    f.x = fmaf(-scale, __uint_as_float(acc[2 * q]), f.x);
-    f.y = fmaf(-scale, __uint_as_float(acc[2 * q + 1]), f.y);
-    h[q] = __floats2bfloat162_rn(f.x, f.y);
-  }
-}
-
-template <>
-__device__ __forceinline__ void apply_vec<float>(uint4& raw, const uint32_t* acc, float scale) {
-  float4* f = reinterpret_cast<float4*>(&raw);
-  f->x = fmaf(-scale, __uint_as_float(acc[0]), f->x);
-  f->y = fmaf(-scale, __uint_as_float(acc[1]), f->y);
-  f->z = fmaf(-scale, __uint_as_float(acc[2]), f->z);
-  f->w = fmaf(-scale, __uint_as_float(acc[3]), f->w);
 }
 
 // ---- the kernel -------------------------------------------------------------------------------
@@ -546,7 +523,7 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
       const TcParams& p = g.p[pi];
       const int row = w.m0 + (int)rank * kBM + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kBN);
-      if (EPI == EPI_APPLY && w.n0 + kBN <= p.N) {
+      if (EPI != EPI_PARTIAL && w.n0 + kBN <= p.N) {
         // Interior tile of the weight update.  The thread's stretch of its W row is fetched into
         // registers BEFORE waiting for the accumulator: the loads do not depend on the MMAs, so the
         // whole W tile streams in from HBM while the tensor cores are still working on it.
@@ -580,7 +557,7 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
             if (row_ok) {
               uint4* dst = reinterpret_cast<uint4*>(wrow + h * kPre + c);
 #pragma unroll
-              for (int q = 0; q < 32 / kVec; ++q) apply_vec<TW>(wv[c / kVec + q], &v[q * kVec], p.scale);
+              for (int q = 0; q < 32 / kVec; ++q) apply_vec<TW, EPI == EPI_APPLY_DECAY>(wv[c / kVec + q], &v[q * kVec], p.scale, p.keep);
               if (vec32) {
 #pragma unroll
                 for (int q = 0; q < 32 / kVec; q += 2) st_global_32B(dst + q, wv[c / kVec + q], wv[c / kVec + q + 1]);
@@ -601,7 +578,7 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
           tmem_ld_32x32(t_row + (uint32_t)c, v);
           tmem_ld_wait();
           if (EPI == EPI_PARTIAL) epi_partial(p, w, row, w.n0 + c, v);
-          else epi_apply<TW>(p, row, w.n0 + c, v);
+          else epi_apply<TW, EPI == EPI_APPLY_DECAY>(p, row, w.n0 + c, v);
         }
       }
       tc_fence_before();
@@ -835,10 +812,19 @@ static galore_status_t project_problem(const TensorPlan* plan, const galore_conf
   return make_map(ma, G, c.m, c.n, ldg, kBM);
 }
 
-// W <- W - scale * P N (left) / N Q^T (right); map_n addresses the normalised update
+// the weight update of a group: with the decay multiply only if some problem of the group decays
+static galore_status_t launch_apply(const TcGroup& g, int32_t w_dtype, cudaStream_t st) {
+  bool decay = false;
+  for (int i = 0; i < g.count; ++i) decay = decay || g.p[i].keep != 1.0f;
+  if (w_dtype == GALORE_BF16)
+    return decay ? launch_tc<EPI_APPLY_DECAY, __nv_bfloat16>(g, st) : launch_tc<EPI_APPLY, __nv_bfloat16>(g, st);
+  return decay ? launch_tc<EPI_APPLY_DECAY, float>(g, st) : launch_tc<EPI_APPLY, float>(g, st);
+}
+
+// W <- keep * W - scale * P N (left) / N Q^T (right); map_n addresses the normalised update
 static galore_status_t back_problem(const TensorPlan* plan, const galore_config_t& c, bool left, const CUtensorMap& map_n,
-                                    void* W, int64_t ldw, float scale, int32_t* status, TcParams* p, CUtensorMap* ma,
-                                    CUtensorMap* mb) {
+                                    void* W, int64_t ldw, float scale, float keep, int32_t* status, TcParams* p,
+                                    CUtensorMap* ma, CUtensorMap* mb) {
   if (!plan->ready) return GALORE_ERR_STATE;
   *p = TcParams{};
   p->status = status;
@@ -846,6 +832,7 @@ static galore_status_t back_problem(const TensorPlan* plan, const galore_config_
   p->ldw = ldw;
   p->vec32 = (((uintptr_t)W & 31) == 0 && (ldw * (int64_t)dtype_size(c.w_dtype)) % 32 == 0) ? 1 : 0;
   p->scale = scale;
+  p->keep = keep;
   p->m_fast = 1;
   fill_tiles(*p, (int)c.m, (int)c.n, c.rank, 1, plan->ctas);
   if (left) {   // A = P K-major, B = N M/N-major
@@ -874,15 +861,14 @@ galore_status_t tensor_project(TensorPlan* plan, const galore_config_t& c, bool 
 }
 
 galore_status_t tensor_back_project(TensorPlan* plan, const galore_config_t& c, bool left, void* W, int64_t ldw,
-                                    float scale, int32_t* status, cudaStream_t st) {
+                                    float scale, float keep, int32_t* status, cudaStream_t st) {
   TcParams p;
   CUtensorMap ma, mb;
-  GALORE_TRY(back_problem(plan, c, left, plan->map_n_back, W, ldw, scale, status, &p, &ma, &mb));
+  GALORE_TRY(back_problem(plan, c, left, plan->map_n_back, W, ldw, scale, keep, status, &p, &ma, &mb));
   std::unique_ptr<TcGroup> g(new TcGroup);
   g->count = 0;
   group_add(*g, ma, mb, p);
-  if (c.w_dtype == GALORE_BF16) return launch_tc<EPI_APPLY, __nv_bfloat16>(*g, st);
-  return launch_tc<EPI_APPLY, float>(*g, st);
+  return launch_apply(*g, c.w_dtype, st);
 }
 
 // ---- groups: many layers per launch ------------------------------------------------------------------
@@ -913,7 +899,7 @@ galore_status_t tensor_group_add_project(TensorGroup* t, const TensorPlan* plan,
 }
 
 galore_status_t tensor_group_add_back(TensorGroup* t, const TensorPlan* plan, const galore_config_t& c, bool left,
-                                      const void* Nbuf, int64_t ld_n, void* W, int64_t ldw, float scale,
+                                      const void* Nbuf, int64_t ld_n, void* W, int64_t ldw, float scale, float keep,
                                       int32_t* status) {
   if (t->g.count >= kMaxGroup) return GALORE_ERR_BUFFER_TOO_SMALL;
   CUtensorMap map_n;
@@ -921,7 +907,7 @@ galore_status_t tensor_group_add_back(TensorGroup* t, const TensorPlan* plan, co
   else GALORE_TRY(make_map(&map_n, Nbuf, c.m, c.rank, ld_n, kBM));
   TcParams p;
   CUtensorMap ma, mb;
-  GALORE_TRY(back_problem(plan, c, left, map_n, W, ldw, scale, status, &p, &ma, &mb));
+  GALORE_TRY(back_problem(plan, c, left, map_n, W, ldw, scale, keep, status, &p, &ma, &mb));
   group_add(t->g, ma, mb, p);
   return GALORE_OK;
 }
@@ -960,8 +946,7 @@ galore_status_t tensor_group_launch_project(TensorGroup* t, cudaStream_t st) {
 
 galore_status_t tensor_group_launch_back(TensorGroup* t, int32_t w_dtype, cudaStream_t st) {
   if (t->g.count == 0) return GALORE_OK;
-  if (w_dtype == GALORE_BF16) return launch_tc<EPI_APPLY, __nv_bfloat16>(t->g, st);
-  return launch_tc<EPI_APPLY, float>(t->g, st);
+  return launch_apply(t->g, w_dtype, st);
 }
 
 }  // namespace galore

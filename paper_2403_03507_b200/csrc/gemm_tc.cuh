@@ -35,7 +35,7 @@ galore_status_t tensor_project(TensorPlan* plan, const galore_config_t& cfg, boo
                                int32_t* status, cudaStream_t st);
 // W <- W - scale * P N (left) / N Q^T (right), N read from plan->Nbuf
 galore_status_t tensor_back_project(TensorPlan* plan, const galore_config_t& cfg, bool left, void* W, int64_t ldw,
-                                    float scale, int32_t* status, cudaStream_t st);
+                                    float scale, float keep, int32_t* status, cudaStream_t st);
 
 
 // ---- groups: up to tensor_group_capacity() layers per launch ------------------------------------
@@ -51,7 +51,7 @@ galore_status_t tensor_group_add_project(TensorGroup* t, const TensorPlan* plan,
                                          int32_t* status);
 // the layer's back-projection reading its normalised update from Nbuf (bf16, leading dimension ld_n)
 galore_status_t tensor_group_add_back(TensorGroup* t, const TensorPlan* plan, const galore_config_t& cfg, bool left,
-                                      const void* Nbuf, int64_t ld_n, void* W, int64_t ldw, float scale,
+                                      const void* Nbuf, int64_t ld_n, void* W, int64_t ldw, float scale, float keep,
                                       int32_t* status);
 // a plain GEMM: C (M x N fp32, ldc) = op(A) op(B), bf16 operands; *_mn = 1 when the operand is stored
 // with M (resp. N) contiguous, 0 when K is contiguous.  Launch with tensor_group_launch_project.

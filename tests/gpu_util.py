@@ -29,7 +29,7 @@ def rel_err(a, b):
 
 def run_pair(m, n, r, steps, T, w_dtype="f32", g_dtype="f32", state_fmt="f32", p=1.0, noise=0.01, lr=1e-2, seed=1,
              q_block=2048, path=gb.PATH_AUTO, side=gb.SIDE_AUTO, ldw=None, ldg=None, oversample=0,
-             check_angle=None, svd_method="jacobi", same_g=False):
+             check_angle=None, svd_method="jacobi", same_g=False, weight_decay=0.0):
     """Steps the CUDA path and the oracle together.
 
     At every refresh the oracle first computes its own top-r subspace (for the
@@ -40,12 +40,13 @@ def run_pair(m, n, r, steps, T, w_dtype="f32", g_dtype="f32", state_fmt="f32", p
     """
     cfg = gb.make_config(m, n, r, alpha=0.25, refresh_gap=T, w_dtype=w_dtype, g_dtype=g_dtype, state_fmt=state_fmt,
                          q_block=q_block, auto_refresh=False, path=path, side=side, refresh_oversample=oversample,
-                         seed=seed)
+                         seed=seed, weight_decay=weight_decay)
     layer = gb.Layer(cfg)
     side_name = "left" if layer.side == gb.SIDE_LEFT else "right"
     n_store = "bf16" if layer.uses_tensor_path else "f64"
     orc = go.GaLoreOracle(m, n, r, 0.25, T, side=side_name, w_store=w_dtype, n_store=n_store,
-                          state={"f32": "f32", "q8": "q8"}[state_fmt], q_block=q_block, svd_method=svd_method)
+                          state={"f32": "f32", "q8": "q8"}[state_fmt], q_block=q_block, svd_method=svd_method,
+                          weight_decay=weight_decay)
     W0 = wl.make_weight(m, n, wl.sub_seed(seed, 999), w_dtype)
     W_orc = W0.copy()
     W_gpu = to_dev(W0, w_dtype, ldw)

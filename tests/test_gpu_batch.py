@@ -219,3 +219,36 @@ def test_host_resident_batch_equals_device_steps(slots):
     for l, wh, wd in zip(layers_h, W_host, Wd):
         assert l.step_count == 3 and l.device_status() == 0
         assert torch.equal(wh, wd.cpu())
+
+
+def test_batch_with_weight_decay_equals_per_layer_steps_and_the_oracle():
+    shapes = [(256, 512, 64), (512, 256, 64), (384, 1000, 128)]
+    la, lb, Wa, Wb, orcs, Wo, W0s = [], [], [], [], [], [], []
+    for i, (m, n, r) in enumerate(shapes):
+        P = wl.round_to(wl.random_orthonormal(min(m, n), r, np.random.default_rng(i)), "bf16")
+        W0 = wl.make_weight(m, n, 60 + i, "bf16")
+        for ls, Ws in ((la, Wa), (lb, Wb)):
+            cfg = gb.make_config(m, n, r, state_fmt="q8", q_block=256, auto_refresh=False, weight_decay=0.05)
+            layer = gb.Layer(cfg)
+            layer.set_projector(torch.from_numpy(P))
+            ls.append(layer)
+            Ws.append(to_dev(W0, "bf16", (n + 7) // 8 * 8))
+        o = go.GaLoreOracle(m, n, r, 0.25, 1000, w_store="bf16", state="q8", q_block=256, n_store="bf16", weight_decay=0.05)
+        o.set_projector(P)
+        orcs.append(o); Wo.append(W0); W0s.append(W0)
+    batch = None
+    for s in range(3):
+        Gh = [wl.make_gradient(m, n, wl.sub_seed(17, i, s), 0.8, 0.05, "bf16") for i, (m, n, r) in enumerate(shapes)]
+        Gd = [to_dev(g, "bf16", (g.shape[1] + 7) // 8 * 8) for g in Gh]
+        for l, w, g in zip(la, Wa, Gd):
+            l.galore_step(w, g, 2e-2)
+        if batch is None:
+            batch = gb.Batch(lb, Wb, Gd)
+        else:
+            batch.rebind(Wb, Gd)
+        batch.galore_step_batch(2e-2)
+        Wo = [o.step(w, g, 2e-2, auto_refresh=False) for o, w, g in zip(orcs, Wo, Gh)]
+    for w1, w2, wo, w0 in zip(Wa, Wb, Wo, W0s):
+        assert rel_err(to_host(w2), to_host(w1)) < 5e-4
+        assert rel_err(to_host(w2), wo) <= 2e-2
+        assert rel_err(to_host(w2) - w0, wo - w0) <= 5e-2

@@ -192,3 +192,20 @@ def test_full_size_matrix_of_the_1b_workload_sampled():
         assert layer.device_status() == 0
         assert rel_err(to_host(Wg), Wo) <= TOL_W_BF16
         assert rel_err(to_host(Wg) - W0, Wo - W0) <= TOL_DW_BF16_W
+
+
+@pytest.mark.parametrize("w_dtype,g_dtype,state_fmt,path", [("f32", "f32", "f32", gb.PATH_FP32), ("bf16", "bf16", "q8", gb.PATH_AUTO),
+                                                            ("bf16", "bf16", "f32", gb.PATH_AUTO)])
+def test_decoupled_weight_decay_matches_the_oracle(w_dtype, g_dtype, state_fmt, path):
+    """GaLore-AdamW: W <- W (1 - lr lambda) - lr alpha P N, the decay folded into the pass that applies the update."""
+    m, n, r = (256, 640, 32) if w_dtype == "bf16" else (200, 333, 24)
+    res = run_pair(m, n, r, 6, 4, w_dtype, g_dtype, state_fmt, seed=13, path=path, weight_decay=0.1, lr=2e-2,
+                   ldw=(n + 7) // 8 * 8, ldg=(n + 7) // 8 * 8, q_block=256)
+    assert res["flags"] == 0
+    tol_w, tol_dw = (TOL_W_F32, TOL_DW_F32) if w_dtype == "f32" else (TOL_W_BF16, TOL_DW_BF16_W)
+    assert max(res["w_err"]) <= tol_w, res["w_err"]
+    assert max(res["dw_err"]) <= tol_dw, res["dw_err"]
+    # the decay is really there: without it W would be elsewhere by about 6 steps of lr * lambda
+    res0 = run_pair(m, n, r, 6, 4, w_dtype, g_dtype, state_fmt, seed=13, path=path, weight_decay=0.0, lr=2e-2,
+                    ldw=(n + 7) // 8 * 8, ldg=(n + 7) // 8 * 8, q_block=256)
+    assert rel_err(res["W_gpu"], res0["W_gpu"]) > 5e-3
