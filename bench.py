@@ -195,11 +195,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--mode", default="batch", choices=["batch", "layer"],
-                    help="batch: galore_step_batch over the layer set (grouped launches); layer: galore_step per layer")
-    ap.add_argument("--projector", default="refresh", choices=["refresh", "random"],
-                    help="refresh: one real refresh per distinct shape (timed, reported); random: a random orthonormal "
-                         "projector (step timing does not depend on P's values; for short profiling runs)")
+    ap.add_argument("--mode", default="batch", choices=["batch", "layer", "arrive"],
+                    help="batch: galore_step_batch over the layer set (grouped launches); layer: galore_step per layer; "
+                         "arrive: galore_step per layer as its gradient arrives from a producer stream into a ring of "
+                         "--ring gradient buffers per shape (per-layer weight updates, Sec. 'Reducing memory footprint "
+                         "of gradients': the full set of gradients never exists)")
+    ap.add_argument("--ring", type=int, default=2, help="gradient buffers per distinct shape in --mode arrive")
     ap.add_argument("--weight-decay", type=float, default=0.0,
                     help="GaLore-AdamW: decoupled weight decay folded into the weight update (0 = plain Adam)")
     ap.add_argument("--rank", type=int, default=0, help="override the workload's rank (rank sweep on one shape)")
@@ -343,9 +344,40 @@ def time_workload(w, args, dev, dist, world, rank, full):
 
     batch = gb.Batch(layers, Ws, Gs, device=dev) if args.mode == "batch" else None
 
+    arrive = None
+    if args.mode == "arrive":
+        # A producer stream stands in for the backward pass: it writes layer i's gradient into the next
+        # buffer of a small ring (a device copy of a resident gradient, i.e. the write traffic of the
+        # kernel that would produce it) and signals; the step of layer i waits for that, runs on the
+        # optimizer stream and hands the buffer back.
+        prod = torch.cuda.Stream(device=dev)
+        rings = {}
+        for sh in set(shapes_of):
+            rings[sh] = [padded(sh[0], sh[1], tdt[w.g_dtype]) for _ in range(max(1, args.ring))]
+        ready = [torch.cuda.Event() for _ in layers]
+        freed = {sh: [torch.cuda.Event() for _ in rings[sh]] for sh in rings}
+        arrive = (prod, rings, ready, freed)
+
     def one_step(lr=w.lr):
         if batch is not None:
             batch.galore_step_batch(lr, stream)
+            return
+        if arrive is not None:
+            prod, rings, ready, freed = arrive
+            turn = {}
+            prod.wait_stream(stream)
+            for i, (layer, Wt, Gt, sh) in enumerate(zip(layers, Ws, Gs, shapes_of)):
+                j = turn.get(sh, 0)
+                turn[sh] = j + 1
+                slot = j % len(rings[sh])
+                with torch.cuda.stream(prod):
+                    if j >= len(rings[sh]):
+                        prod.wait_event(freed[sh][slot])
+                    rings[sh][slot].copy_(Gt, non_blocking=True)
+                    ready[i].record(prod)
+                stream.wait_event(ready[i])
+                layer.galore_step(Wt, rings[sh][slot], lr, stream)
+                freed[sh][slot].record(stream)
             return
         for layer, Wt, Gt in zip(layers, Ws, Gs):
             layer.galore_step(Wt, Gt, lr, stream)

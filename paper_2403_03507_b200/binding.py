@@ -391,13 +391,17 @@ class Batch:
     call into the library.  W and G tensors are bound once; rebind() swaps them.
     """
 
-    def __init__(self, layers, Ws, Gs, workspace_bytes=None, device=None):
+    def __init__(self, layers, Ws, Gs, workspace_bytes=None, device=None, workspace=None):
         self.layers = list(layers)
         self.n = len(self.layers)
         self.device = device if device is not None else self.layers[0].device
         need = galore_batch_query_bytes(self.layers)
-        self.workspace_bytes = need if workspace_bytes is None else int(workspace_bytes)
-        self.workspace = torch.empty(max(self.workspace_bytes, 256), dtype=torch.uint8, device=self.device)
+        if workspace is not None:          # a caller-owned buffer, e.g. shared by batches that never run together
+            self.workspace_bytes = int(workspace.numel())
+            self.workspace = workspace
+        else:
+            self.workspace_bytes = need if workspace_bytes is None else int(workspace_bytes)
+            self.workspace = torch.empty(max(self.workspace_bytes, 256), dtype=torch.uint8, device=self.device)
         self._hs = (C.c_void_p * self.n)(*[l.handle.value for l in self.layers])
         self.rebind(Ws, Gs)
 
