@@ -201,6 +201,9 @@ def main():
                          "--ring gradient buffers per shape (per-layer weight updates, Sec. 'Reducing memory footprint "
                          "of gradients': the full set of gradients never exists)")
     ap.add_argument("--ring", type=int, default=2, help="gradient buffers per distinct shape in --mode arrive")
+    ap.add_argument("--projector", default="refresh", choices=["refresh", "random"],
+                    help="refresh: one real refresh per distinct shape (timed, reported); random: a random orthonormal "
+                         "projector (step timing does not depend on P's values; for short profiling runs)")
     ap.add_argument("--weight-decay", type=float, default=0.0,
                     help="GaLore-AdamW: decoupled weight decay folded into the weight update (0 = plain Adam)")
     ap.add_argument("--rank", type=int, default=0, help="override the workload's rank (rank sweep on one shape)")
