@@ -57,10 +57,8 @@ __device__ float c_code_s[256];
 __device__ float c_code_u[256];
 __device__ float c_mid_s[256];   // 255 thresholds used
 __device__ float c_mid_u[256];
-__device__ float2 c_pair_s[256];  // thresholds bracketing each code (+-FLT_MAX at the ends)
-__device__ float2 c_pair_u[256];
-__device__ uint8_t c_lut_s[2 * 3584];   // candidate codes: [0, 3584) for y >= 0, [3584, 7168) for y < 0
-__device__ uint8_t c_lut_u[3584];
+__device__ uint32_t c_enc_s[3584];   // quantiser table, one entry per bin of |y| (see q8_encode_block)
+__device__ uint32_t c_enc_u[3584];
 
 static std::mutex g_code_mutex;
 static bool g_code_ready[64] = {};
@@ -82,33 +80,43 @@ galore_status_t q8_ensure_tables() {
   GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_code_u, cu, sizeof(cu)));
   GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_mid_s, ms, sizeof(ms)));
   GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_mid_u, mu, sizeof(mu)));
-  float2 ps[256], pu[256];
-  for (int i = 0; i < 256; ++i) {
-    ps[i] = make_float2(i > 0 ? ms[i - 1] : -FLT_MAX, i < 255 ? ms[i] : FLT_MAX);
-    pu[i] = make_float2(i > 0 ? mu[i - 1] : -FLT_MAX, i < 255 ? mu[i] : FLT_MAX);
-  }
-  GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_pair_s, ps, sizeof(ps)));
-  GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_pair_u, pu, sizeof(pu)));
-  // candidate tables: number of thresholds at or below the lowest value of each bin
-  static uint8_t lut_s[2 * 3584], lut_u[3584];
-  auto count_le = [](const float* mids, float x) {
-    int c = 0;
-    while (c < 255 && mids[c] <= x) ++c;
-    return c;
+  // Quantiser tables.  Bin `key` holds the non-negative floats whose upper 16 bits are
+  // (kLutBase >> 16) + key (bin 0 also everything below 2^-27).  With c = number of thresholds below
+  // the bin and t = lower 16 bits of the one threshold inside it (0xffff if none), the entry is
+  // (c << 16) + (0x10000 - t): adding the lower 16 bits of a value of the bin carries into the upper
+  // half exactly when the value is at or above the threshold.
+  static uint32_t enc_s[3584], enc_u[3584];
+  auto build_enc = [](const float* mids, uint32_t* enc) -> bool {
+    uint32_t tb[255];
+    int n_nonpos = 0, n_pos = 0;
+    for (int i = 0; i < 255; ++i) {
+      if (mids[i] > 0.f) memcpy(&tb[n_pos++], &mids[i], 4);     // ascending, positive: bit order = value order
+      else ++n_nonpos;
+    }
+    for (int key = 0; key < 3584; ++key) {
+      const uint32_t k = (uint32_t)std::min(key, 3456);
+      const uint32_t hi = (0x32000000u >> 16) + k;
+      uint32_t below = 0, thr = 0xffffu;
+      int inside = 0;
+      for (int i = 0; i < n_pos; ++i) {
+        const uint32_t th = tb[i] >> 16;
+        if (th < hi && k > 0) ++below;
+        else if (th == hi || (k == 0 && th < hi)) { thr = tb[i] & 0xffffu; ++inside; }
+      }
+      if (inside > 1 || (inside == 1 && thr > 0xfff0u)) return false;
+      enc[key] = (((uint32_t)n_nonpos + below) << 16) + (0x10000u - thr);
+    }
+    // a threshold within 8 ulp of its bin's lower edge needs a threshold-free bin below it, so that
+    // values just under the edge are sent to the exact search by the 0xffff entry
+    for (int key = 1; key <= 3456; ++key) {
+      const uint32_t t_here = (0x10000u - (enc[key] & 0xffffu)) & 0xffffu;       // t = 0 is stored as 0
+      if (t_here < 8u && (enc[key - 1] & 0xffffu) != 1u) return false;
+    }
+    return true;
   };
-  for (int key = 0; key < 3584; ++key) {
-    const uint32_t b0 = 0x32000000u + ((uint32_t)std::min(key, 3456) << 16);
-    const uint32_t b1 = 0x32000000u + ((uint32_t)(std::min(key, 3456) + 1) << 16);
-    float lo, hi;
-    memcpy(&lo, &b0, 4);
-    memcpy(&hi, &b1, 4);
-    if (key == 0) lo = 0.f;
-    lut_u[key] = (uint8_t)count_le(mu, lo);
-    lut_s[key] = (uint8_t)count_le(ms, lo);            // y in [lo, hi)
-    lut_s[3584 + key] = (uint8_t)count_le(ms, -hi);    // y in (-hi, -lo]
-  }
-  GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_lut_s, lut_s, sizeof(lut_s)));
-  GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_lut_u, lut_u, sizeof(lut_u)));
+  if (!build_enc(ms, enc_s) || !build_enc(mu, enc_u)) return GALORE_ERR_STATE;
+  GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_enc_s, enc_s, sizeof(enc_s)));
+  GALORE_CUDA_TRY(cudaMemcpyToSymbol(c_enc_u, enc_u, sizeof(enc_u)));
   if (dev < 64) g_code_ready[dev] = true;
   return GALORE_OK;
 }
@@ -125,33 +133,43 @@ __device__ __forceinline__ int q8_encode(float y, const float* __restrict__ mids
 }
 
 // Same code as q8_encode(fp32(x / absmax)) at a fraction of the cost.
-//  1. y' = x * (1 / absmax) approximates the quotient to within 2 ulp.
-//  2. A table indexed by the exponent and 7 mantissa bits of |y'| gives the code of the lower edge
-//     of that bin (kLutSize entries per sign); at most one threshold lies inside a bin, so one
-//     comparison with the bracketing thresholds pairs[idx] = {below, above} finishes the search.
-//  3. If y' is not within 6e-7 (relative) of either bracketing threshold, the exactly rounded
-//     quotient lies on the same side of both and the code is final.  Otherwise the quotient is
-//     formed with IEEE division and searched exactly.
+//  1. y' = x * (1 / absmax) is within 2 ulp of the correctly rounded quotient q.
+//  2. The upper 16 bits of |y'| (exponent and 7 mantissa bits) select a bin; the spacing of the
+//     thresholds is wider than a bin, so a bin holds at most one.  The bin's table entry gives the
+//     number of thresholds below the bin and the lower 16 bits of the threshold inside it
+//     (0xffff if there is none); comparing those with the lower 16 bits of |y'| finishes the search
+//     in integer arithmetic.
+//  3. If |y'| is more than 8 ulp away from the bin's threshold, q lies on the same side of it and
+//     the code is final.  Otherwise (also for the top 9 values of a bin without a threshold, which
+//     covers a threshold at the lower edge of the next bin) the quotient is formed with IEEE
+//     division and searched exactly.
+//  Signed code: its thresholds are symmetric about zero except between -1e-6 and 1e-6, so a
+//  negative y' takes 255 - (code of |y'|), and goes to the exact search below 2^-19.
 constexpr int kLutSize = 3584;                 // keys 0 .. 3456 used
 constexpr uint32_t kLutBase = 0x32000000u;     // bits of 2^-27: below it every value maps to key 0
 
-__device__ __forceinline__ int q8_lut_key(float ya) {
-  const uint32_t bits = __float_as_uint(ya) & 0x7fffffffu;
-  return min((int)((max(bits, kLutBase) - kLutBase) >> 16), 3456);
+// Fast part: the code of y' and whether it has to be confirmed by the exact search.
+template <bool SIGNED>
+__device__ __forceinline__ uint32_t q8_encode_fast(float x, float inv, const uint32_t* __restrict__ enc, bool& exact) {
+  const float ya = x * inv;
+  const uint32_t mag = SIGNED ? (__float_as_uint(ya) & 0x7fffffffu) : __float_as_uint(ya);   // unsigned code: y' >= 0
+  const uint32_t b = max(mag, kLutBase + 0x8000u);      // everything below lands mid-bin in bin 0 (no threshold there)
+  const uint32_t sum = enc[min((b - kLutBase) >> 16, 3456u)] + (b & 0xffffu);
+  uint32_t idx = sum >> 16;
+  exact = ((sum + 8u) & 0xffffu) <= 16u;          // within 8 ulp of the threshold (modulo 2^16: errs on the safe side)
+  if (SIGNED && ya < 0.f) {
+    idx = 255u - idx;
+    exact |= b < 0x36000000u;
+  }
+  return idx;
 }
 
 template <bool SIGNED>
-__device__ __forceinline__ int q8_encode_block(float x, float absmax, float inv, const uint8_t* __restrict__ lut,
-                                               const float2* __restrict__ pairs, const float* __restrict__ mids) {
-  const float ya = x * inv;
-  int idx = lut[q8_lut_key(ya) + ((SIGNED && ya < 0.f) ? kLutSize : 0)];
-  float2 t = pairs[idx];
-  if (ya >= t.y) {
-    ++idx;
-    t = pairs[idx];
-  }
-  constexpr float guard = 6e-7f;
-  if ((ya - t.x) > guard * fabsf(t.x) && (t.y - ya) > guard * fabsf(t.y)) return idx;
+__device__ __forceinline__ int q8_encode_block(float x, float absmax, float inv, const uint32_t* __restrict__ enc,
+                                               const float* __restrict__ mids) {
+  bool exact;
+  const uint32_t idx = q8_encode_fast<SIGNED>(x, inv, enc, exact);
+  if (!exact) return (int)idx;
   return q8_encode(__fdiv_rn(x, absmax), mids);
 }
 
@@ -266,10 +284,12 @@ __global__ void __launch_bounds__(256) adam_f32_kernel(const __grid_constant__ A
 // elements t, t + 256, t + 512, ... so every warp-level access is one contiguous run
 // whatever the alignment of the block.  PACKED: R partials and N have the state's own
 // row pitch, so one flat index serves all arrays.
+#ifndef GALORE_Q8_CTAS
+#define GALORE_Q8_CTAS 4          // resident CTAs per SM the kernel is compiled for (register budget)
+#endif
 struct Q8Tables {
   float code_s[256], code_u[256], mid_s[256], mid_u[256];
-  float2 pair_s[256], pair_u[256];
-  uint8_t lut_s[2 * kLutSize], lut_u[kLutSize];
+  uint32_t enc_s[kLutSize], enc_u[kLutSize];
   float red[16];
 };
 
@@ -338,8 +358,8 @@ __device__ __forceinline__ bool adam_q8_block(const AdamItem& a, int blk, Q8Tabl
   for (int e = 0; e < EPT; ++e) {
     const int i = base + e * 256;
     if (i < nel) {
-      Mc[i] = (mx_m == 0.f) ? (uint8_t)127 : (uint8_t)q8_encode_block<true>(m[e], mx_m, inv_m, t.lut_s, t.pair_s, t.mid_s);
-      Vc[i] = (mx_v == 0.f) ? (uint8_t)0 : (uint8_t)q8_encode_block<false>(v[e], mx_v, inv_v, t.lut_u, t.pair_u, t.mid_u);
+      Mc[i] = (mx_m == 0.f) ? (uint8_t)127 : (uint8_t)q8_encode_block<true>(m[e], mx_m, inv_m, t.enc_s, t.mid_s);
+      Vc[i] = (mx_v == 0.f) ? (uint8_t)0 : (uint8_t)q8_encode_block<false>(v[e], mx_v, inv_v, t.enc_u, t.mid_u);
     }
   }
   if (threadIdx.x == 0) {
@@ -423,10 +443,19 @@ __device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q
     const bool wrap = run_col[j] + k >= a.cols;
     return (run_row[j] + (wrap ? 1 : 0)) * ld + run_col[j] + k - (wrap ? a.cols : 0);
   };
+  // a run that stays inside its row (all but one or two per row) is four consecutive elements of
+  // the padded buffers as well
+  auto load_run = [&](const float* __restrict__ src, int j) {
+    if (run_col[j] + 3 < a.cols) {
+      const float* __restrict__ q = src + run_row[j] * a.r_ld + run_col[j];
+      return make_float4(q[0], q[1], q[2], q[3]);
+    }
+    return make_float4(src[at(j, 0, a.r_ld)], src[at(j, 1, a.r_ld)], src[at(j, 2, a.r_ld)], src[at(j, 3, a.r_ld)]);
+  };
 #pragma unroll
   for (int j = 0; j < RUNS; ++j) {
     if (PADDED) {
-      r[j] = make_float4(R[at(j, 0, a.r_ld)], R[at(j, 1, a.r_ld)], R[at(j, 2, a.r_ld)], R[at(j, 3, a.r_ld)]);
+      r[j] = load_run(R, j);
     } else {
       r[j] = *reinterpret_cast<const float4*>(R + j * 1024);
     }
@@ -438,13 +467,16 @@ __device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q
 #pragma unroll
     for (int j = 0; j < RUNS; ++j) {
       float4 q;
-      if (PADDED) q = make_float4(part[at(j, 0, a.r_ld)], part[at(j, 1, a.r_ld)], part[at(j, 2, a.r_ld)], part[at(j, 3, a.r_ld)]);
+      if (PADDED) q = load_run(part, j);
       else q = *reinterpret_cast<const float4*>(part + j * 1024);
       r[j].x += q.x; r[j].y += q.y; r[j].z += q.z; r[j].w += q.w;
     }
   }
   float m[EPT], v[EPT];
-  float mx_m = 0.f, mx_v = 0.f, poison = 0.f;
+  float mx_m = 0.f;
+  uint32_t mx_v_bits = 0u;                       // v >= 0: the order of the bit patterns is the order of the values,
+                                                 // and a NaN or an infinity (from a non-finite r) ends up on top
+  const float c1 = p.b1 * am_m, c2 = p.b2 * am_v;
 #pragma unroll
   for (int j = 0; j < RUNS; ++j) {
     const float rr[4] = {r[j].x, r[j].y, r[j].z, r[j].w};
@@ -452,35 +484,65 @@ __device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const int e = 4 * j + k;
-      poison = fmaf(rr[k], 0.f, poison);             // stays 0 unless some r is inf or nan
-      m[e] = p.b1 * (t.code_s[(cm[j] >> (8 * k)) & 0xffu] * am_m) + p.omb1 * rr[k];
-      v[e] = p.b2 * (t.code_u[(cv[j] >> (8 * k)) & 0xffu] * am_v) + p.omb2 * (rr[k] * rr[k]);
+      m[e] = fmaf(t.code_s[((cm[j] >> (8 * k)) & 0xffu)], c1, p.omb1 * rr[k]);
+      v[e] = fmaf(t.code_u[((cv[j] >> (8 * k)) & 0xffu)], c2, p.omb2 * (rr[k] * rr[k]));
       nn[k] = adam_normalised(m[e], v[e], p);
       mx_m = fmaxf(mx_m, fabsf(m[e]));
-      mx_v = fmaxf(mx_v, v[e]);
+      mx_v_bits = max(mx_v_bits, __float_as_uint(v[e]));
     }
     if (PADDED) {
+      if (run_col[j] + 3 < a.cols) {
+        TN* __restrict__ q = Nout + run_row[j] * a.n_ld + run_col[j];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) Nout[at(j, k, a.n_ld)] = cvt<TN>(nn[k]);
+        for (int k = 0; k < 4; ++k) q[k] = cvt<TN>(nn[k]);
+      } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) Nout[at(j, k, a.n_ld)] = cvt<TN>(nn[k]);
+      }
     } else {
       store_n4<TN>(Nout + j * 1024, nn[0], nn[1], nn[2], nn[3]);
     }
   }
+  const bool bad = mx_v_bits >= 0x7f800000u;
+  float mx_v = __uint_as_float(mx_v_bits);
   block_max2_256(mx_m, mx_v, t.red);
   const float inv_m = 1.0f / mx_m, inv_v = 1.0f / mx_v;
 #pragma unroll
   for (int j = 0; j < RUNS; ++j) {
     uint32_t pm = 0x7f7f7f7fu, pv = 0u;              // codes of the value 0
+    uint32_t need = 0u;                              // bit k: M value k of the run, bit 4 + k: V value k
     if (mx_m != 0.f) {
       pm = 0u;
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        pm |= (uint32_t)q8_encode_block<true>(m[4 * j + k], mx_m, inv_m, t.lut_s, t.pair_s, t.mid_s) << (8 * k);
+      for (int k = 0; k < 4; ++k) {
+        bool ex;
+        const uint32_t c = q8_encode_fast<true>(m[4 * j + k], inv_m, t.enc_s, ex) & 0xffu;
+        pm |= c << (8 * k);
+        need |= (ex ? 1u : 0u) << k;
+      }
     }
     if (mx_v != 0.f) {
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        pv |= (uint32_t)q8_encode_block<false>(v[4 * j + k], mx_v, inv_v, t.lut_u, t.pair_u, t.mid_u) << (8 * k);
+      for (int k = 0; k < 4; ++k) {
+        bool ex;
+        const uint32_t c = q8_encode_fast<false>(v[4 * j + k], inv_v, t.enc_u, ex) & 0xffu;
+        pv |= c << (8 * k);
+        need |= (ex ? 1u : 0u) << (4 + k);
+      }
+    }
+    // rare (about 1 value in 15 000): one branch for the eight values of the run
+    if (need != 0u) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (need & (1u << k)) {
+          const uint32_t c = (uint32_t)q8_encode(__fdiv_rn(m[4 * j + k], mx_m), t.mid_s) & 0xffu;
+          pm = (pm & ~(0xffu << (8 * k))) | (c << (8 * k));
+        }
+        if (need & (16u << k)) {
+          const uint32_t c = (uint32_t)q8_encode(__fdiv_rn(v[4 * j + k], mx_v), t.mid_u) & 0xffu;
+          pv = (pv & ~(0xffu << (8 * k))) | (c << (8 * k));
+        }
+      }
     }
     *reinterpret_cast<uint32_t*>(Mc + j * 1024) = pm;
     *reinterpret_cast<uint32_t*>(Vc + j * 1024) = pv;
@@ -489,23 +551,20 @@ __device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q
     a.Mam[blk] = mx_m;
     a.Vam[blk] = mx_v;
   }
-  return poison != 0.f;
+  return bad;
 }
 
 template <typename TN, int EPT>
-__global__ void __launch_bounds__(256, 4) adam_q8_kernel(const __grid_constant__ AdamGroup g) {
+__global__ void __launch_bounds__(256, GALORE_Q8_CTAS) adam_q8_kernel(const __grid_constant__ AdamGroup g) {
   __shared__ Q8Tables t;
-  for (int i = threadIdx.x; i < kLutSize / 4; i += 256) {
-    reinterpret_cast<uint32_t*>(t.lut_u)[i] = reinterpret_cast<const uint32_t*>(c_lut_u)[i];
-    reinterpret_cast<uint32_t*>(t.lut_s)[i] = reinterpret_cast<const uint32_t*>(c_lut_s)[i];
-    reinterpret_cast<uint32_t*>(t.lut_s)[kLutSize / 4 + i] = reinterpret_cast<const uint32_t*>(c_lut_s)[kLutSize / 4 + i];
+  for (int i = threadIdx.x; i < kLutSize; i += 256) {
+    t.enc_s[i] = c_enc_s[i];
+    t.enc_u[i] = c_enc_u[i];
   }
   t.code_s[threadIdx.x] = c_code_s[threadIdx.x];
   t.code_u[threadIdx.x] = c_code_u[threadIdx.x];
   t.mid_s[threadIdx.x] = c_mid_s[threadIdx.x];
   t.mid_u[threadIdx.x] = c_mid_u[threadIdx.x];
-  t.pair_s[threadIdx.x] = c_pair_s[threadIdx.x];
-  t.pair_u[threadIdx.x] = c_pair_u[threadIdx.x];
   __syncthreads();
 
   const int total = g.block_end[g.count - 1];
@@ -536,14 +595,10 @@ __global__ void __launch_bounds__(256)
 q8_quantize_kernel(const float* __restrict__ x, int64_t nel, int is_signed, uint8_t* __restrict__ codes,
                    float* __restrict__ absmax) {
   __shared__ float s_mid[256];
-  __shared__ float2 s_pair[256];
-  __shared__ uint8_t s_lut[2 * kLutSize];
+  __shared__ uint32_t s_enc[kLutSize];
   __shared__ float red[8];
-  for (int i = threadIdx.x; i < (is_signed ? 2 : 1) * kLutSize / 4; i += 256)
-    reinterpret_cast<uint32_t*>(s_lut)[i] = is_signed ? reinterpret_cast<const uint32_t*>(c_lut_s)[i]
-                                                      : reinterpret_cast<const uint32_t*>(c_lut_u)[i];
+  for (int i = threadIdx.x; i < kLutSize; i += 256) s_enc[i] = is_signed ? c_enc_s[i] : c_enc_u[i];
   s_mid[threadIdx.x] = is_signed ? c_mid_s[threadIdx.x] : c_mid_u[threadIdx.x];
-  s_pair[threadIdx.x] = is_signed ? c_pair_s[threadIdx.x] : c_pair_u[threadIdx.x];
   __syncthreads();
   constexpr int QB = EPT * 256;
   const int64_t blk = blockIdx.x;
@@ -564,8 +619,8 @@ q8_quantize_kernel(const float* __restrict__ x, int64_t nel, int is_signed, uint
     int64_t i = base + (int64_t)e * 256;
     if (i < nel)
       codes[i] = (mx == 0.f) ? zero_code
-                             : (uint8_t)(is_signed ? q8_encode_block<true>(val[e], mx, inv, s_lut, s_pair, s_mid)
-                                                   : q8_encode_block<false>(val[e], mx, inv, s_lut, s_pair, s_mid));
+                             : (uint8_t)(is_signed ? q8_encode_block<true>(val[e], mx, inv, s_enc, s_mid)
+                                                   : q8_encode_block<false>(val[e], mx, inv, s_enc, s_mid));
   }
   if (threadIdx.x == 0) absmax[blk] = mx;
 }
@@ -599,10 +654,18 @@ galore_status_t launch_adam_group(const AdamGroup& g, int32_t state_fmt, int q_b
   }
   if (!valid_block(q_block)) return GALORE_ERR_INVALID_ARG;
   GALORE_TRY(q8_ensure_tables());
+  // four CTAs of 32 KiB of tables each per SM: ask for the largest shared-memory carve-out
 #define GALORE_Q8_CASE(EPT)                                                            \
   case EPT * 256:                                                                      \
-    if (nb) adam_q8_kernel<__nv_bfloat16, EPT><<<grid, 256, 0, st>>>(g);               \
-    else adam_q8_kernel<float, EPT><<<grid, 256, 0, st>>>(g);                          \
+    if (nb) {                                                                          \
+      GALORE_CUDA_TRY(cudaFuncSetAttribute(adam_q8_kernel<__nv_bfloat16, EPT>,         \
+                                           cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)); \
+      adam_q8_kernel<__nv_bfloat16, EPT><<<grid, 256, 0, st>>>(g);                     \
+    } else {                                                                           \
+      GALORE_CUDA_TRY(cudaFuncSetAttribute(adam_q8_kernel<float, EPT>,                 \
+                                           cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)); \
+      adam_q8_kernel<float, EPT><<<grid, 256, 0, st>>>(g);                             \
+    }                                                                                  \
     break;
   switch (q_block) {
     GALORE_Q8_CASE(1) GALORE_Q8_CASE(2) GALORE_Q8_CASE(4) GALORE_Q8_CASE(8) GALORE_Q8_CASE(16)

@@ -193,6 +193,12 @@ def test_full_size_7b_matrices_in_the_benched_configuration():
         M, V = layer.get_moments()
         Mo, Vo = o.moments()
         assert rel_err(to_host(M), Mo) < 2e-2 and rel_err(to_host(V), Vo) < 2e-2
+        # the stored codes themselves: fp32 against fp64 arithmetic may move a value on a threshold to
+        # the neighbouring code, never further
+        Mc, _Ma, Vc, _Va = [t.cpu().numpy() for t in layer.get_q8_state()]
+        cs, cu = go.dynamic_code(True).astype(np.float64), go.dynamic_code(False).astype(np.float64)
+        assert np.mean(Mc != o.M_codes.ravel()) < 2e-3 and np.max(np.abs(cs[Mc] - cs[o.M_codes.ravel()])) <= 0.9 / 64 + 1e-6
+        assert np.mean(Vc != o.V_codes.ravel()) < 2e-3 and np.max(np.abs(cu[Vc] - cu[o.V_codes.ravel()])) <= 0.9 / 128 + 1e-6
 
 
 @pytest.mark.parametrize("slots", [1, 3])

@@ -48,6 +48,28 @@ def test_thresholds_ties_and_zero_blocks(signed):
     assert am_o[2] == 0 and np.all(codes_o[512:768] == (127 if signed else 0))
 
 
+@pytest.mark.parametrize("signed", [True, False])
+def test_quotients_next_to_thresholds_any_absmax(signed):
+    """Blocks [a, x_1 .. x_255] with x_i within a few ulp of threshold_i * a for arbitrary absmax a: the
+    cases where x * (1 / a) and the correctly rounded x / a can fall on different sides of a threshold."""
+    mids = go.code_midpoints(go.dynamic_code(signed)).astype(np.float32)
+    assert len(mids) == 255
+    rng = np.random.default_rng(5)
+    blocks = []
+    for off in range(-3, 4):
+        for _ in range(160):
+            a = np.float32(rng.uniform(1.0, 2.0) * 10.0 ** rng.uniform(-6, 3))
+            x = (mids.astype(np.float64) * float(a)).astype(np.float32)
+            x = (x.view(np.int32) + off).view(np.float32)          # same-sign neighbours: |x| moves by `off` ulp
+            blocks.append(np.concatenate([[a], x]).astype(np.float32))
+    x = np.concatenate(blocks)
+    assert np.all(np.abs(x.reshape(-1, 256)[:, 1:]) <= x.reshape(-1, 256)[:, :1])
+    codes_o, am_o = go.quantize_blockwise(x, signed, 256)
+    codes_g, am_g = gb.galore_q8_quantize(torch.from_numpy(x).cuda(), signed, 256)
+    assert np.array_equal(am_g.cpu().numpy(), am_o)
+    assert np.array_equal(codes_g.cpu().numpy(), codes_o)
+
+
 def test_empty_input():
     codes, am = gb.galore_q8_quantize(torch.zeros(0, device="cuda"), True, 2048)
     assert codes.numel() == 0 and am.numel() == 0
