@@ -207,7 +207,7 @@ __device__ __forceinline__ float adam_normalised(float m, float v, const AdamPar
 __device__ __forceinline__ int find_item(const AdamGroup& g, int gb, int& local) {
   int it = 0;
   while (it + 1 < g.count && gb >= g.block_end[it]) ++it;
-  local = gb - (it > 0 ? g.block_end[it - 1] : 0);
+  local = gb - (it > 0 ? g.block_end[it - 1] : 0) + g.item[it].first_block;
   return it;
 }
 
@@ -264,26 +264,17 @@ __device__ __forceinline__ bool adam_f32_block(const AdamItem& a, int blk) {
   return bad;
 }
 
-template <typename TN>
-__global__ void __launch_bounds__(256) adam_f32_kernel(const __grid_constant__ AdamGroup g) {
-  const int total = g.block_end[g.count - 1];
-  int bad_item = -1;
-  for (int gb = blockIdx.x; gb < total; gb += gridDim.x) {
-    int blk;
-    const int it = find_item(g, gb, blk);
-    const AdamItem& a = g.item[it];
-    const bool packed = (a.r_ld == a.cols && a.n_ld == a.cols);
-    const bool bad = packed ? adam_f32_block<TN, true>(a, blk) : adam_f32_block<TN, false>(a, blk);
-    if (bad) bad_item = it;
-  }
-  if (bad_item >= 0) atomicOr(g.item[bad_item].status, GALORE_DEV_NONFINITE);
-}
-
 // ---- 8-bit block-wise moments ---------------------------------------------------
 // A CTA walks quantisation blocks of EPT * 256 elements; within a block thread t owns
 // elements t, t + 256, t + 512, ... so every warp-level access is one contiguous run
 // whatever the alignment of the block.  PACKED: R partials and N have the state's own
 // row pitch, so one flat index serves all arrays.
+#ifndef GALORE_Q8_FAST_CTAS
+#define GALORE_Q8_FAST_CTAS 6     // the same for the kernel that holds the full-packed-block variant alone
+#endif
+#ifndef GALORE_Q8_PADDED_CTAS
+#define GALORE_Q8_PADDED_CTAS 5   // and for the one that holds the full-padded-block variant alone
+#endif
 #ifndef GALORE_Q8_CTAS
 #define GALORE_Q8_CTAS 4          // resident CTAs per SM the kernel is compiled for (register budget)
 #endif
@@ -407,6 +398,71 @@ template <>
 __device__ __forceinline__ void store_n4<float>(float* dst, float a, float b, float c, float d) {
   *reinterpret_cast<float4*>(dst) = make_float4(a, b, c, d);
 }
+
+// fp32 moments, full work block of a layer with packed, 16-byte aligned arrays: runs of four as
+// below, every access a 16-byte one (8 bytes for a bf16 N)
+template <typename TN>
+__device__ __forceinline__ bool adam_f32_block_full(const AdamItem& a, int blk) {
+  const AdamParams p = a.p;
+  const int base = blk * 2048 + 4 * threadIdx.x;
+  const float* __restrict__ R = a.Rpart + base;
+  float* __restrict__ M = a.M + base;
+  float* __restrict__ V = a.V + base;
+  TN* __restrict__ Nout = (TN*)a.Nout + base;
+  float4 r[2], m[2], v[2];
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    r[j] = *reinterpret_cast<const float4*>(R + j * 1024);
+    m[j] = *reinterpret_cast<const float4*>(M + j * 1024);
+    v[j] = *reinterpret_cast<const float4*>(V + j * 1024);
+  }
+  for (int s = 1; s < a.splits; ++s) {
+    const float* __restrict__ part = R + (int64_t)s * a.split_stride;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const float4 q = *reinterpret_cast<const float4*>(part + j * 1024);
+      r[j].x += q.x; r[j].y += q.y; r[j].z += q.z; r[j].w += q.w;
+    }
+  }
+  uint32_t top = 0u;      // largest bit pattern among the new second moments (all >= 0): a non-finite r shows here
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const float rr[4] = {r[j].x, r[j].y, r[j].z, r[j].w};
+    const float mo[4] = {m[j].x, m[j].y, m[j].z, m[j].w};
+    const float vo[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+    float mn[4], vn[4], nn[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      mn[k] = p.b1 * mo[k] + p.omb1 * rr[k];
+      vn[k] = p.b2 * vo[k] + p.omb2 * (rr[k] * rr[k]);
+      nn[k] = adam_normalised(mn[k], vn[k], p);
+      top = max(top, __float_as_uint(vn[k]));
+    }
+    *reinterpret_cast<float4*>(M + j * 1024) = make_float4(mn[0], mn[1], mn[2], mn[3]);
+    *reinterpret_cast<float4*>(V + j * 1024) = make_float4(vn[0], vn[1], vn[2], vn[3]);
+    store_n4<TN>(Nout + j * 1024, nn[0], nn[1], nn[2], nn[3]);
+  }
+  return top >= 0x7f800000u;
+}
+
+template <typename TN>
+__global__ void __launch_bounds__(256) adam_f32_kernel(const __grid_constant__ AdamGroup g) {
+  const int total = g.block_end[g.count - 1];
+  int bad_item = -1;
+  for (int gb = blockIdx.x; gb < total; gb += gridDim.x) {
+    int blk;
+    const int it = find_item(g, gb, blk);
+    const AdamItem& a = g.item[it];
+    const bool packed = (a.r_ld == a.cols && a.n_ld == a.cols);
+    const bool full = (blk + 1) * 2048 <= a.nel;
+    const bool bad = (packed && full && a.aligned16) ? adam_f32_block_full<TN>(a, blk)
+                     : packed                        ? adam_f32_block<TN, true>(a, blk)
+                                                     : adam_f32_block<TN, false>(a, blk);
+    if (bad) bad_item = it;
+  }
+  if (bad_item >= 0) atomicOr(g.item[bad_item].status, GALORE_DEV_NONFINITE);
+}
+
 
 // PADDED: R and N have rows of a.cols elements at pitches a.r_ld and a.n_ld (the state itself is
 // always contiguous).  The codes keep their 4-byte accesses; the four R and N elements of a run are
@@ -554,8 +610,36 @@ __device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q
   return bad;
 }
 
-template <typename TN, int EPT>
-__global__ void __launch_bounds__(256, GALORE_Q8_CTAS) adam_q8_kernel(const __grid_constant__ AdamGroup g) {
+// How a quantisation block is processed depends on its layer (row pitches, alignment) and on
+// whether it is a full block.  A kernel compiled with every variant inlined needs the registers of
+// the most demanding one and spills in all of them, so the kernel takes the set of variants it
+// contains as a template argument; the launcher sorts the layers of a group into launches whose
+// kernels contain what their blocks need.
+enum : int {
+  kBlockFullPacked = 1,    // full block, R and N at the state's own pitch, 16-byte aligned: vector accesses
+  kBlockFullPadded = 2,    // full block, padded R / N rows
+  kBlockAnyPacked = 4,     // tail block or unaligned arrays, packed
+  kBlockAny = 8,           // tail block or unaligned arrays, padded rows
+  kBlockAll = 15
+};
+
+template <int EPT>
+__host__ __device__ __forceinline__ int q8_block_kind(const AdamItem& a, int blk) {
+  const bool packed = (a.r_ld == a.cols && a.n_ld == a.cols);
+  const bool full = (blk + 1) * (EPT * 256) <= a.nel;
+  if (EPT % 4 == 0 && full && a.aligned16) {
+    if (packed) return kBlockFullPacked;
+    if (a.cols >= 4) return kBlockFullPadded;
+  }
+  return packed ? kBlockAnyPacked : kBlockAny;
+}
+
+constexpr int q8_ctas_per_sm(int kinds) {
+  return kinds == kBlockFullPacked ? GALORE_Q8_FAST_CTAS : kinds == kBlockFullPadded ? GALORE_Q8_PADDED_CTAS : GALORE_Q8_CTAS;
+}
+
+template <typename TN, int EPT, int KINDS>
+__global__ void __launch_bounds__(256, q8_ctas_per_sm(KINDS)) adam_q8_kernel(const __grid_constant__ AdamGroup g) {
   __shared__ Q8Tables t;
   for (int i = threadIdx.x; i < kLutSize; i += 256) {
     t.enc_s[i] = c_enc_s[i];
@@ -573,16 +657,20 @@ __global__ void __launch_bounds__(256, GALORE_Q8_CTAS) adam_q8_kernel(const __gr
     int blk;
     const int it = find_item(g, gb, blk);
     const AdamItem& a = g.item[it];
-    const bool packed = (a.r_ld == a.cols && a.n_ld == a.cols);
-    const bool full = (blk + 1) * (EPT * 256) <= a.nel;
-    bool bad;
-    if constexpr (EPT % 4 == 0) {
-      bad = (packed && full && a.aligned16) ? adam_q8_block_full<TN, EPT, false>(a, blk, t)
-            : (full && a.aligned16 && a.cols >= 4) ? adam_q8_block_full<TN, EPT, true>(a, blk, t)
-            : packed                        ? adam_q8_block<TN, EPT, true>(a, blk, t)
-                                            : adam_q8_block<TN, EPT, false>(a, blk, t);
+    bool bad = false;
+    if constexpr (KINDS == kBlockFullPacked || KINDS == kBlockFullPadded) {
+      // never launched for EPT < 4
+      if constexpr (EPT % 4 == 0) bad = adam_q8_block_full<TN, EPT, KINDS == kBlockFullPadded>(a, blk, t);
     } else {
-      bad = packed ? adam_q8_block<TN, EPT, true>(a, blk, t) : adam_q8_block<TN, EPT, false>(a, blk, t);
+      const int kind = q8_block_kind<EPT>(a, blk);           // the same for every thread of the CTA
+      if constexpr (EPT % 4 == 0 && (KINDS & kBlockFullPacked) != 0)
+        if (kind == kBlockFullPacked) bad = adam_q8_block_full<TN, EPT, false>(a, blk, t);
+      if constexpr (EPT % 4 == 0 && (KINDS & kBlockFullPadded) != 0)
+        if (kind == kBlockFullPadded) bad = adam_q8_block_full<TN, EPT, true>(a, blk, t);
+      if constexpr ((KINDS & kBlockAnyPacked) != 0)
+        if (kind == kBlockAnyPacked) bad = adam_q8_block<TN, EPT, true>(a, blk, t);
+      if constexpr ((KINDS & kBlockAny) != 0)
+        if (kind == kBlockAny) bad = adam_q8_block<TN, EPT, false>(a, blk, t);
     }
     if (__syncthreads_or(bad)) bad_item = it;
   }
@@ -636,6 +724,17 @@ q8_dequantize_kernel(const uint8_t* __restrict__ codes, const float* __restrict_
 }
 
 // ---- launchers --------------------------------------------------------------------
+// the variant the full blocks of a layer take (block 0 when the layer has a full block at all)
+static int q8_item_kind(const AdamItem& a, int q_block) {
+  switch (q_block) {
+    case 256: return q8_block_kind<1>(a, 0);
+    case 512: return q8_block_kind<2>(a, 0);
+    case 1024: return q8_block_kind<4>(a, 0);
+    case 2048: return q8_block_kind<8>(a, 0);
+    default: return q8_block_kind<16>(a, 0);
+  }
+}
+
 static bool valid_block(int block) {
   return block == 256 || block == 512 || block == 1024 || block == 2048 || block == 4096;
 }
@@ -654,17 +753,52 @@ galore_status_t launch_adam_group(const AdamGroup& g, int32_t state_fmt, int q_b
   }
   if (!valid_block(q_block)) return GALORE_ERR_INVALID_ARG;
   GALORE_TRY(q8_ensure_tables());
-  // four CTAs of 32 KiB of tables each per SM: ask for the largest shared-memory carve-out
+  // The full blocks of a layer go to the kernel that holds their variant alone (packed or padded
+  // rows); tail blocks and layers with unaligned arrays go to the kernel that holds all variants.
+  std::unique_ptr<AdamGroup> packed(new AdamGroup), padded(new AdamGroup), rest(new AdamGroup);
+  packed->count = padded->count = rest->count = 0;
+  auto append = [](AdamGroup& dst, const AdamItem& a, int first, int blocks) {
+    if (blocks <= 0) return;
+    const int j = dst.count++;
+    dst.item[j] = a;
+    dst.item[j].first_block = a.first_block + first;
+    dst.block_end[j] = (j > 0 ? dst.block_end[j - 1] : 0) + blocks;
+  };
+  for (int i = 0; i < g.count; ++i) {
+    const AdamItem& a = g.item[i];
+    const int blocks = g.block_end[i] - (i > 0 ? g.block_end[i - 1] : 0);
+    const int kind = q8_item_kind(a, q_block);
+    // whole blocks among those the item covers (it covers the layer's blocks from first_block to the last)
+    const int whole = std::min(blocks, std::max(0, a.nel / q_block - a.first_block));
+    if (kind == kBlockFullPacked || kind == kBlockFullPadded) {
+      append(kind == kBlockFullPacked ? *packed : *padded, a, 0, whole);
+      append(*rest, a, whole, blocks - whole);
+    } else {
+      append(*rest, a, 0, blocks);
+    }
+  }
+#define GALORE_Q8_LAUNCH(TN, EPT, KINDS, grp)                                                                 \
+  do {                                                                                                       \
+    GALORE_CUDA_TRY(cudaFuncSetAttribute(adam_q8_kernel<TN, EPT, KINDS>,                                     \
+                                         cudaFuncAttributePreferredSharedMemoryCarveout,                     \
+                                         cudaSharedmemCarveoutMaxShared)); /* several CTAs of 32 KiB of tables per SM */ \
+    const int blocks_ = (grp).block_end[(grp).count - 1];                                                    \
+    adam_q8_kernel<TN, EPT, KINDS><<<(unsigned)std::min(blocks_, 148 * 2 * q8_ctas_per_sm(KINDS)), 256, 0, st>>>(grp); \
+    GALORE_LAUNCH_CHECK();                                                                                   \
+  } while (0)
 #define GALORE_Q8_CASE(EPT)                                                            \
   case EPT * 256:                                                                      \
-    if (nb) {                                                                          \
-      GALORE_CUDA_TRY(cudaFuncSetAttribute(adam_q8_kernel<__nv_bfloat16, EPT>,         \
-                                           cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)); \
-      adam_q8_kernel<__nv_bfloat16, EPT><<<grid, 256, 0, st>>>(g);                     \
-    } else {                                                                           \
-      GALORE_CUDA_TRY(cudaFuncSetAttribute(adam_q8_kernel<float, EPT>,                 \
-                                           cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)); \
-      adam_q8_kernel<float, EPT><<<grid, 256, 0, st>>>(g);                             \
+    if (packed->count > 0) {                                                           \
+      if (nb) GALORE_Q8_LAUNCH(__nv_bfloat16, EPT, kBlockFullPacked, *packed);         \
+      else GALORE_Q8_LAUNCH(float, EPT, kBlockFullPacked, *packed);                    \
+    }                                                                                  \
+    if (padded->count > 0) {                                                           \
+      if (nb) GALORE_Q8_LAUNCH(__nv_bfloat16, EPT, kBlockFullPadded, *padded);         \
+      else GALORE_Q8_LAUNCH(float, EPT, kBlockFullPadded, *padded);                    \
+    }                                                                                  \
+    if (rest->count > 0) {                                                             \
+      if (nb) GALORE_Q8_LAUNCH(__nv_bfloat16, EPT, kBlockAll, *rest);                  \
+      else GALORE_Q8_LAUNCH(float, EPT, kBlockAll, *rest);                             \
     }                                                                                  \
     break;
   switch (q_block) {
@@ -672,7 +806,7 @@ galore_status_t launch_adam_group(const AdamGroup& g, int32_t state_fmt, int q_b
     default: return GALORE_ERR_INVALID_ARG;
   }
 #undef GALORE_Q8_CASE
-  GALORE_LAUNCH_CHECK();
+#undef GALORE_Q8_LAUNCH
   return GALORE_OK;
 }
 
@@ -684,7 +818,8 @@ galore_status_t adam_group_add(AdamGroup& g, const AdamItem& item, int32_t state
   const int64_t rows = ceil_div(a.nel, a.cols);
   if (rows * std::max(a.r_ld, a.n_ld) >= (int64_t)1 << 31) return GALORE_ERR_SHAPE;
   const int per_block = state_fmt == GALORE_STATE_F32 ? 2048 : q_block;
-  a.aligned16 = ((((uintptr_t)a.Rpart | (uintptr_t)a.Nout | (uintptr_t)a.Mc | (uintptr_t)a.Vc) & 15) == 0 &&
+  a.aligned16 = ((((uintptr_t)a.Rpart | (uintptr_t)a.Nout | (uintptr_t)a.Mc | (uintptr_t)a.Vc | (uintptr_t)a.M |
+                   (uintptr_t)a.V) & 15) == 0 &&
                  (a.split_stride % 4) == 0) ? 1 : 0;
   const int i = g.count++;
   g.item[i] = a;

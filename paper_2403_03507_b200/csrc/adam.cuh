@@ -36,6 +36,7 @@ struct AdamItem {
   void* Nout;              // normalised update (fp32 or bf16)
   int cols, r_ld, n_ld;    // state row length and the row pitches of Rpart / Nout (cols == 0: packed)
   int aligned16;           // set by adam_group_add: all arrays allow 16-byte vector accesses
+  int first_block;         // the item covers the layer's work blocks from this one on (0: the whole layer)
   AdamParams p;
   int32_t* status;
 };
