@@ -270,7 +270,7 @@ __device__ __forceinline__ bool adam_f32_block(const AdamItem& a, int blk) {
 // whatever the alignment of the block.  PACKED: R partials and N have the state's own
 // row pitch, so one flat index serves all arrays.
 #ifndef GALORE_Q8_FAST_CTAS
-#define GALORE_Q8_FAST_CTAS 6     // the same for the kernel that holds the full-packed-block variant alone
+#define GALORE_Q8_FAST_CTAS 5     // the same for the kernel that holds the full-packed-block variant alone
 #endif
 #ifndef GALORE_Q8_PADDED_CTAS
 #define GALORE_Q8_PADDED_CTAS 5   // and for the one that holds the full-padded-block variant alone
@@ -278,10 +278,10 @@ __device__ __forceinline__ bool adam_f32_block(const AdamItem& a, int blk) {
 #ifndef GALORE_Q8_CTAS
 #define GALORE_Q8_CTAS 4          // resident CTAs per SM the kernel is compiled for (register budget)
 #endif
-struct Q8Tables {
+struct alignas(16) Q8Tables {
   float code_s[256], code_u[256], mid_s[256], mid_u[256];
   uint32_t enc_s[kLutSize], enc_u[kLutSize];
-  float red[16];
+  float red[48];          // [0, 16): the one-value reductions; [16, 32) and [32, 48): the alternating two-value ones
 };
 
 template <typename TN, int EPT, bool PACKED>
@@ -360,8 +360,10 @@ __device__ __forceinline__ bool adam_q8_block(const AdamItem& a, int blk, Q8Tabl
   return bad;
 }
 
-// max of two values over the CTA (256 threads) with one pair of barriers; every thread gets both
-__device__ __forceinline__ void block_max2_256(float& x, float& y, float* red /* >= 16 floats */) {
+// max of two values over the CTA (256 threads) with a single barrier; every thread gets both.
+// `red` is one of two alternating 16-float buffers: a buffer is written again two calls later, and
+// the barrier of the call in between separates that from the last reads of this one.
+__device__ __forceinline__ void block_max2_256(float& x, float& y, float* red /* 16 floats */) {
   x = warp_max(x);
   y = warp_max(y);
   if ((threadIdx.x & 31) == 0) {
@@ -369,15 +371,10 @@ __device__ __forceinline__ void block_max2_256(float& x, float& y, float* red /*
     red[8 + (threadIdx.x >> 5)] = y;
   }
   __syncthreads();
-  float rx = red[0], ry = red[8];
-#pragma unroll
-  for (int w = 1; w < 8; ++w) {
-    rx = fmaxf(rx, red[w]);
-    ry = fmaxf(ry, red[8 + w]);
-  }
-  __syncthreads();
-  x = rx;
-  y = ry;
+  const float4* __restrict__ q = reinterpret_cast<const float4*>(red);      // 16-byte aligned (Q8Tables)
+  const float4 a = q[0], b = q[1], c = q[2], d = q[3];
+  x = fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w)));
+  y = fmaxf(fmaxf(fmaxf(c.x, c.y), fmaxf(c.z, c.w)), fmaxf(fmaxf(d.x, d.y), fmaxf(d.z, d.w)));
 }
 
 // Full block of a layer whose R and N buffers have the state's own row pitch: every array is
@@ -468,7 +465,7 @@ __global__ void __launch_bounds__(256) adam_f32_kernel(const __grid_constant__ A
 // always contiguous).  The codes keep their 4-byte accesses; the four R and N elements of a run are
 // addressed one by one, and a run may continue on the next row.
 template <typename TN, int EPT, bool PADDED>
-__device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q8Tables& t) {
+__device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q8Tables& t, int parity) {
   static_assert(EPT % 4 == 0, "runs of four elements");
   constexpr int RUNS = EPT / 4;
   const AdamParams p = a.p;
@@ -561,7 +558,7 @@ __device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q
   }
   const bool bad = mx_v_bits >= 0x7f800000u;
   float mx_v = __uint_as_float(mx_v_bits);
-  block_max2_256(mx_m, mx_v, t.red);
+  block_max2_256(mx_m, mx_v, t.red + 16 + 16 * parity);
   const float inv_m = 1.0f / mx_m, inv_v = 1.0f / mx_v;
 #pragma unroll
   for (int j = 0; j < RUNS; ++j) {
@@ -641,9 +638,12 @@ constexpr int q8_ctas_per_sm(int kinds) {
 template <typename TN, int EPT, int KINDS>
 __global__ void __launch_bounds__(256, q8_ctas_per_sm(KINDS)) adam_q8_kernel(const __grid_constant__ AdamGroup g) {
   __shared__ Q8Tables t;
-  for (int i = threadIdx.x; i < kLutSize; i += 256) {
-    t.enc_s[i] = c_enc_s[i];
-    t.enc_u[i] = c_enc_u[i];
+  // 32 KiB of tables per CTA: all loads in flight at once (one L2 round trip instead of fourteen)
+  static_assert(kLutSize % 256 == 0, "whole rounds");
+#pragma unroll
+  for (int i = 0; i < kLutSize / 256; ++i) {
+    t.enc_s[i * 256 + threadIdx.x] = c_enc_s[i * 256 + threadIdx.x];
+    t.enc_u[i * 256 + threadIdx.x] = c_enc_u[i * 256 + threadIdx.x];
   }
   t.code_s[threadIdx.x] = c_code_s[threadIdx.x];
   t.code_u[threadIdx.x] = c_code_u[threadIdx.x];
@@ -653,28 +653,29 @@ __global__ void __launch_bounds__(256, q8_ctas_per_sm(KINDS)) adam_q8_kernel(con
 
   const int total = g.block_end[g.count - 1];
   int bad_item = -1;
-  for (int gb = blockIdx.x; gb < total; gb += gridDim.x) {
+  int parity = 0;
+  for (int gb = blockIdx.x; gb < total; gb += gridDim.x, parity ^= 1) {
     int blk;
     const int it = find_item(g, gb, blk);
     const AdamItem& a = g.item[it];
     bool bad = false;
     if constexpr (KINDS == kBlockFullPacked || KINDS == kBlockFullPadded) {
       // never launched for EPT < 4
-      if constexpr (EPT % 4 == 0) bad = adam_q8_block_full<TN, EPT, KINDS == kBlockFullPadded>(a, blk, t);
+      if constexpr (EPT % 4 == 0) bad = adam_q8_block_full<TN, EPT, KINDS == kBlockFullPadded>(a, blk, t, parity);
     } else {
       const int kind = q8_block_kind<EPT>(a, blk);           // the same for every thread of the CTA
       if constexpr (EPT % 4 == 0 && (KINDS & kBlockFullPacked) != 0)
-        if (kind == kBlockFullPacked) bad = adam_q8_block_full<TN, EPT, false>(a, blk, t);
+        if (kind == kBlockFullPacked) bad = adam_q8_block_full<TN, EPT, false>(a, blk, t, parity);
       if constexpr (EPT % 4 == 0 && (KINDS & kBlockFullPadded) != 0)
-        if (kind == kBlockFullPadded) bad = adam_q8_block_full<TN, EPT, true>(a, blk, t);
+        if (kind == kBlockFullPadded) bad = adam_q8_block_full<TN, EPT, true>(a, blk, t, parity);
       if constexpr ((KINDS & kBlockAnyPacked) != 0)
         if (kind == kBlockAnyPacked) bad = adam_q8_block<TN, EPT, true>(a, blk, t);
       if constexpr ((KINDS & kBlockAny) != 0)
         if (kind == kBlockAny) bad = adam_q8_block<TN, EPT, false>(a, blk, t);
     }
-    if (__syncthreads_or(bad)) bad_item = it;
+    if (bad) bad_item = it;      // per thread: no barrier; a non-finite input is reported by the threads that met it
   }
-  if (bad_item >= 0 && threadIdx.x == 0) atomicOr(g.item[bad_item].status, GALORE_DEV_NONFINITE);
+  if (bad_item >= 0) atomicOr(g.item[bad_item].status, GALORE_DEV_NONFINITE);
 }
 
 // ---- stand-alone quantise / dequantise (same device code as the Adam kernel) ----
@@ -783,7 +784,7 @@ galore_status_t launch_adam_group(const AdamGroup& g, int32_t state_fmt, int q_b
                                          cudaFuncAttributePreferredSharedMemoryCarveout,                     \
                                          cudaSharedmemCarveoutMaxShared)); /* several CTAs of 32 KiB of tables per SM */ \
     const int blocks_ = (grp).block_end[(grp).count - 1];                                                    \
-    adam_q8_kernel<TN, EPT, KINDS><<<(unsigned)std::min(blocks_, 148 * 2 * q8_ctas_per_sm(KINDS)), 256, 0, st>>>(grp); \
+    adam_q8_kernel<TN, EPT, KINDS><<<(unsigned)std::min(blocks_, 148 * q8_ctas_per_sm(KINDS)), 256, 0, st>>>(grp); /* one resident wave: tables are set up once per SM slot */ \
     GALORE_LAUNCH_CHECK();                                                                                   \
   } while (0)
 #define GALORE_Q8_CASE(EPT)                                                            \
