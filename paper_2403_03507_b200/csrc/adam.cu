@@ -204,11 +204,12 @@ __device__ __forceinline__ float adam_normalised(float m, float v, const AdamPar
 // Both kernels take a group of layers (AdamGroup, passed as kernel parameters) and walk the
 // blocks of all of them with one persistent grid; a single layer is a group of one.
 
-__device__ __forceinline__ int find_item(const AdamGroup& g, int gb, int& local) {
-  int it = 0;
+// `it` is a cursor: a CTA's work blocks come in ascending order, so the search resumes where the
+// previous one ended (a group has up to 32 layers; a scan from the start for every block cost about
+// as many instructions per element as the Adam arithmetic itself).
+__device__ __forceinline__ void find_item(const AdamGroup& g, int gb, int& it, int& local) {
   while (it + 1 < g.count && gb >= g.block_end[it]) ++it;
   local = gb - (it > 0 ? g.block_end[it - 1] : 0) + g.item[it].first_block;
-  return it;
 }
 
 // ---- fp32 moments -------------------------------------------------------------
@@ -443,12 +444,12 @@ __device__ __forceinline__ bool adam_f32_block_full(const AdamItem& a, int blk) 
 }
 
 template <typename TN>
-__global__ void __launch_bounds__(256) adam_f32_kernel(const __grid_constant__ AdamGroup g) {
+__global__ void __launch_bounds__(256, 3) adam_f32_kernel(const __grid_constant__ AdamGroup g) {
   const int total = g.block_end[g.count - 1];
-  int bad_item = -1;
+  int bad_item = -1, it = 0;
   for (int gb = blockIdx.x; gb < total; gb += gridDim.x) {
     int blk;
-    const int it = find_item(g, gb, blk);
+    find_item(g, gb, it, blk);
     const AdamItem& a = g.item[it];
     const bool packed = (a.r_ld == a.cols && a.n_ld == a.cols);
     const bool full = (blk + 1) * 2048 <= a.nel;
@@ -559,29 +560,25 @@ __device__ __forceinline__ bool adam_q8_block_full(const AdamItem& a, int blk, Q
   const bool bad = mx_v_bits >= 0x7f800000u;
   float mx_v = __uint_as_float(mx_v_bits);
   block_max2_256(mx_m, mx_v, t.red + 16 + 16 * parity);
-  const float inv_m = 1.0f / mx_m, inv_v = 1.0f / mx_v;
+  // an all-zero block: with 0 in place of the reciprocal every y' is 0 and takes the code of zero
+  const float inv_m = mx_m != 0.f ? 1.0f / mx_m : 0.f, inv_v = mx_v != 0.f ? 1.0f / mx_v : 0.f;
 #pragma unroll
   for (int j = 0; j < RUNS; ++j) {
-    uint32_t pm = 0x7f7f7f7fu, pv = 0u;              // codes of the value 0
+    uint32_t pm = 0u, pv = 0u;
     uint32_t need = 0u;                              // bit k: M value k of the run, bit 4 + k: V value k
-    if (mx_m != 0.f) {
-      pm = 0u;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        bool ex;
-        const uint32_t c = q8_encode_fast<true>(m[4 * j + k], inv_m, t.enc_s, ex) & 0xffu;
-        pm |= c << (8 * k);
-        need |= (ex ? 1u : 0u) << k;
-      }
+    for (int k = 0; k < 4; ++k) {
+      bool ex;
+      const uint32_t c = q8_encode_fast<true>(m[4 * j + k], inv_m, t.enc_s, ex) & 0xffu;
+      pm |= c << (8 * k);
+      need |= (ex ? 1u : 0u) << k;
     }
-    if (mx_v != 0.f) {
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        bool ex;
-        const uint32_t c = q8_encode_fast<false>(v[4 * j + k], inv_v, t.enc_u, ex) & 0xffu;
-        pv |= c << (8 * k);
-        need |= (ex ? 1u : 0u) << (4 + k);
-      }
+    for (int k = 0; k < 4; ++k) {
+      bool ex;
+      const uint32_t c = q8_encode_fast<false>(v[4 * j + k], inv_v, t.enc_u, ex) & 0xffu;
+      pv |= c << (8 * k);
+      need |= (ex ? 1u : 0u) << (4 + k);
     }
     // rare (about 1 value in 15 000): one branch for the eight values of the run
     if (need != 0u) {
@@ -652,11 +649,11 @@ __global__ void __launch_bounds__(256, q8_ctas_per_sm(KINDS)) adam_q8_kernel(con
   __syncthreads();
 
   const int total = g.block_end[g.count - 1];
-  int bad_item = -1;
+  int bad_item = -1, it = 0;
   int parity = 0;
   for (int gb = blockIdx.x; gb < total; gb += gridDim.x, parity ^= 1) {
     int blk;
-    const int it = find_item(g, gb, blk);
+    find_item(g, gb, it, blk);
     const AdamItem& a = g.item[it];
     bool bad = false;
     if constexpr (KINDS == kBlockFullPacked || KINDS == kBlockFullPadded) {
