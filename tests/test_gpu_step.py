@@ -82,7 +82,8 @@ def test_bf16_weights(g_dtype):
     assert max(res["dw_err"]) <= TOL_DW_BF16_W, res["dw_err"]
 
 
-@pytest.mark.parametrize("m,n,r,qb", [(128, 1100, 16, 2048), (700, 96, 8, 256), (64, 96, 8, 4096)])
+@pytest.mark.parametrize("m,n,r,qb", [(128, 1100, 16, 2048), (700, 96, 8, 256), (64, 96, 8, 4096),
+                                      (96, 700, 16, 4096), (128, 1100, 16, 1024), (1100, 128, 16, 512)])
 def test_q8_states_follow_the_oracle(m, n, r, qb):
     # several quantisation blocks plus a ragged tail block; right case included
     res = run_pair(m, n, r, 6, 10, "f32", "f32", "q8", seed=11, q_block=qb, path=gb.PATH_FP32)

@@ -71,6 +71,21 @@ def test_tensor_path_q8_states(m, n, r, qb):
     assert np.mean(Vc != orc.V_codes) < 5e-3 and np.max(np.abs(cu[Vc] - cu[orc.V_codes])) <= 0.9 / 128 + 1e-6
 
 
+@pytest.mark.parametrize("m,n,r,qb", [(256, 1100, 64, 2048), (1100, 256, 64, 1024), (200, 2741, 72, 4096)])
+def test_tensor_path_q8_states_with_padded_rows(m, n, r, qb):
+    """Row lengths that are no multiple of 8: R and N have padded rows while the state stays packed, so
+    the full blocks go to the padded-row kernel and the tail block to the general one."""
+    ld = (n + 7) // 8 * 8
+    layer, orc, errs = _run(m, n, r, "bf16", "q8", steps=4, q_block=qb, ldw=ld, ldg=ld)
+    assert layer.uses_tensor_path and layer.device_status() == 0
+    assert max(e[0] for e in errs) <= TOL_W_BF16, errs
+    assert max(e[1] for e in errs) <= 5e-2, errs
+    Mc, Ma, Vc, Va = [t.cpu().numpy() for t in layer.get_q8_state()]
+    cs, cu = go.dynamic_code(True).astype(np.float64), go.dynamic_code(False).astype(np.float64)
+    assert np.mean(Mc != orc.M_codes) < 5e-3 and np.max(np.abs(cs[Mc] - cs[orc.M_codes])) <= 0.9 / 64 + 1e-6
+    assert np.mean(Vc != orc.V_codes) < 5e-3 and np.max(np.abs(cu[Vc] - cu[orc.V_codes])) <= 0.9 / 128 + 1e-6
+
+
 def test_unaligned_leading_dimension_falls_back_or_errors():
     # n = 5461 packed: rows are not 16-byte aligned, TMA cannot address them
     m, n, r = 256, 1001, 32
