@@ -270,6 +270,9 @@ __device__ __forceinline__ bool adam_f32_block(const AdamItem& a, int blk) {
 // elements t, t + 256, t + 512, ... so every warp-level access is one contiguous run
 // whatever the alignment of the block.  PACKED: R partials and N have the state's own
 // row pitch, so one flat index serves all arrays.
+#ifndef GALORE_F32_CTAS
+#define GALORE_F32_CTAS 3         // fp32-state kernel: 80 registers
+#endif
 #ifndef GALORE_Q8_FAST_CTAS
 #define GALORE_Q8_FAST_CTAS 5     // the same for the kernel that holds the full-packed-block variant alone
 #endif
@@ -444,7 +447,7 @@ __device__ __forceinline__ bool adam_f32_block_full(const AdamItem& a, int blk) 
 }
 
 template <typename TN>
-__global__ void __launch_bounds__(256, 3) adam_f32_kernel(const __grid_constant__ AdamGroup g) {
+__global__ void __launch_bounds__(256, GALORE_F32_CTAS) adam_f32_kernel(const __grid_constant__ AdamGroup g) {
   const int total = g.block_end[g.count - 1];
   int bad_item = -1, it = 0;
   for (int gb = blockIdx.x; gb < total; gb += gridDim.x) {
