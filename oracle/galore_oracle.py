@@ -23,7 +23,9 @@ What it follows (GaLore, arXiv 2403.03507):
     of the current gradient.
   * Sec. 4.3 ("8-bit optimizers") names block-wise 8-bit Adam states without
     giving a format.  The format used here is this project's own and is
-    spelled out at `dynamic_code`; it is PARITY UNPINNED against the paper
+    spelled out at `dynamic_code` (the code values) and `state_tile` (which
+    elements share an absmax: tiles of q_block / 128 rows x 128 columns of the
+    state matrix); it is PARITY UNPINNED against the paper
     (the paper fixes nothing to pin it to) and pinned only by its own
     invariants in the tests.
 
@@ -195,41 +197,79 @@ def code_midpoints(code: np.ndarray) -> np.ndarray:
     return (0.5 * (c[:-1] + c[1:])).astype(np.float32)
 
 
-def quantize_blockwise(x, signed: bool, block: int = 2048):
-    """fp32 array -> (uint8 codes, fp32 absmax per block).
+def _quantize_one_block(seg, mids, zero_code):
+    """One block of fp32 values (any shape) -> (codes of the same shape, fp32 absmax).
 
-    Blocks are runs of `block` consecutive elements of the flattened
-    (row-major) array; the last block may be shorter.  Per block:
     absmax = max |x|;  y = x / absmax in fp32 (IEEE division);  the code is the
     number of thresholds <= y, i.e. the nearest code value with ties going to
     the larger index.  A block whose absmax is 0 stores the code of 0.
     """
-    x32 = np.asarray(x, dtype=np.float32).reshape(-1)
-    n = x32.size
+    a = np.float32(np.max(np.abs(seg))) if seg.size else np.float32(0)
+    if a == 0:
+        return np.full(seg.shape, zero_code, dtype=np.uint8), a
+    y = (seg / a).astype(np.float32)              # fp32 / fp32 -> IEEE fp32 quotient
+    return np.searchsorted(mids, y, side="right").astype(np.uint8), a
+
+
+def quantize_tiles(X, signed: bool, tile_rows: int, tile_cols: int):
+    """fp32 matrix -> (uint8 codes of the same shape, fp32 absmax per tile).
+
+    The quantisation blocks are tiles of `tile_rows` x `tile_cols` elements of
+    the matrix, tile (I, J) covering rows [I tile_rows, (I+1) tile_rows) and
+    columns [J tile_cols, (J+1) tile_cols); tiles on the lower and right edges
+    are cut off at the matrix border.  absmax has one entry per tile, shape
+    (ceil(rows / tile_rows), ceil(cols / tile_cols)).
+    """
+    X32 = np.asarray(X, dtype=np.float32)
+    assert X32.ndim == 2
+    rows, cols = X32.shape
     code = dynamic_code(signed)
     mids = code_midpoints(code)
     zero_code = int(np.nonzero(code == 0.0)[0][0])
-    nblk = (n + block - 1) // block
-    codes = np.empty(n, dtype=np.uint8)
-    absmax = np.zeros(nblk, dtype=np.float32)
-    for b in range(nblk):
-        seg = x32[b * block:(b + 1) * block]
-        a = np.float32(np.max(np.abs(seg))) if seg.size else np.float32(0)
-        absmax[b] = a
-        if a == 0:
-            codes[b * block:(b + 1) * block] = zero_code
-            continue
-        y = (seg / a).astype(np.float32)          # fp32 / fp32 -> IEEE fp32 quotient
-        codes[b * block:(b + 1) * block] = np.searchsorted(mids, y, side="right").astype(np.uint8)
+    gr, gc = -(-rows // tile_rows), -(-cols // tile_cols)
+    codes = np.empty((rows, cols), dtype=np.uint8)
+    absmax = np.zeros((gr, gc), dtype=np.float32)
+    for I in range(gr):
+        for J in range(gc):
+            sl = (slice(I * tile_rows, (I + 1) * tile_rows), slice(J * tile_cols, (J + 1) * tile_cols))
+            codes[sl], absmax[I, J] = _quantize_one_block(X32[sl], mids, zero_code)
     return codes, absmax
+
+
+def dequantize_tiles(codes, absmax, signed: bool, tile_rows: int, tile_cols: int):
+    """(codes, absmax per tile) -> fp32 matrix: code value times the tile's absmax, in fp32."""
+    codes = np.asarray(codes, dtype=np.uint8)
+    rows, cols = codes.shape
+    code = dynamic_code(signed)
+    am = np.asarray(absmax, dtype=np.float32)
+    scale = np.repeat(np.repeat(am, tile_rows, axis=0)[:rows], tile_cols, axis=1)[:, :cols]
+    return (code[codes] * scale).astype(np.float32)
+
+
+def quantize_blockwise(x, signed: bool, block: int = 2048):
+    """Flat fp32 array -> (uint8 codes, fp32 absmax per block): blocks are runs of `block`
+    consecutive elements, the last one may be shorter (a one-row matrix cut into 1 x block tiles)."""
+    x32 = np.asarray(x, dtype=np.float32).reshape(1, -1)
+    codes, absmax = quantize_tiles(x32, signed, 1, block)
+    return codes.reshape(-1), absmax.reshape(-1)
 
 
 def dequantize_blockwise(codes, absmax, signed: bool, block: int = 2048):
     """(codes, absmax) -> fp32 values: code value times the block's absmax, in fp32."""
-    codes = np.asarray(codes, dtype=np.uint8).reshape(-1)
-    code = dynamic_code(signed)
-    scale = np.repeat(np.asarray(absmax, dtype=np.float32), block)[:codes.size]
-    return (code[codes] * scale).astype(np.float32)
+    codes = np.asarray(codes, dtype=np.uint8).reshape(1, -1)
+    am = np.asarray(absmax, dtype=np.float32).reshape(1, -1)
+    return dequantize_tiles(codes, am, signed, 1, block).reshape(-1)
+
+
+STATE_TILE_COLS = 128
+
+
+def state_tile(q_block: int):
+    """Shape of the quantisation blocks of the 8-bit moments: q_block elements as a tile of
+    q_block / 128 consecutive rows x 128 consecutive columns of the state matrix (2048 -> 16 x 128)."""
+    if q_block % STATE_TILE_COLS:
+        raise ValueError("q_block must be a multiple of 128")
+    return q_block // STATE_TILE_COLS, STATE_TILE_COLS
 
 
 # --------------------------------------------------------------------------
@@ -270,14 +310,14 @@ class GaLoreOracle:
         shape = (self.r, self.n) if side == "left" else (self.m, self.r)
         self.state_shape = shape
         if state == "q8":
-            nel = shape[0] * shape[1]
-            nblk = (nel + self.q_block - 1) // self.q_block
+            self.tile = state_tile(self.q_block)
+            grid = (-(-shape[0] // self.tile[0]), -(-shape[1] // self.tile[1]))
             zc_s = int(np.nonzero(dynamic_code(True) == 0.0)[0][0])
             zc_u = int(np.nonzero(dynamic_code(False) == 0.0)[0][0])
-            self.M_codes = np.full(nel, zc_s, dtype=np.uint8)
-            self.V_codes = np.full(nel, zc_u, dtype=np.uint8)
-            self.M_absmax = np.zeros(nblk, dtype=np.float32)
-            self.V_absmax = np.zeros(nblk, dtype=np.float32)
+            self.M_codes = np.full(shape, zc_s, dtype=np.uint8)
+            self.V_codes = np.full(shape, zc_u, dtype=np.uint8)
+            self.M_absmax = np.zeros(grid, dtype=np.float32)
+            self.V_absmax = np.zeros(grid, dtype=np.float32)
         else:
             self.M = np.zeros(shape, dtype=np.float64)
             self.V = np.zeros(shape, dtype=np.float64)
@@ -287,10 +327,9 @@ class GaLoreOracle:
     def moments(self):
         """Stored (uncorrected) M, V as fp64 arrays of the state's shape."""
         if self.state == "q8":
-            M = dequantize_blockwise(self.M_codes, self.M_absmax, True, self.q_block)
-            V = dequantize_blockwise(self.V_codes, self.V_absmax, False, self.q_block)
-            return (M.astype(np.float64).reshape(self.state_shape),
-                    V.astype(np.float64).reshape(self.state_shape))
+            M = dequantize_tiles(self.M_codes, self.M_absmax, True, *self.tile)
+            V = dequantize_tiles(self.V_codes, self.V_absmax, False, *self.tile)
+            return M.astype(np.float64), V.astype(np.float64)
         return self.M, self.V
 
     def optimizer_state_elements(self) -> int:
@@ -333,8 +372,8 @@ class GaLoreOracle:
             V_hat = V / (1.0 - self.beta2 ** t)
             N = M_hat / (np.sqrt(V_hat) + self.eps)
             if self.state == "q8":
-                self.M_codes, self.M_absmax = quantize_blockwise(M, True, self.q_block)
-                self.V_codes, self.V_absmax = quantize_blockwise(V, False, self.q_block)
+                self.M_codes, self.M_absmax = quantize_tiles(M, True, *self.tile)
+                self.V_codes, self.V_absmax = quantize_tiles(V, False, *self.tile)
             else:
                 self.M, self.V = _store(M, self.state), _store(V, self.state)
         N = _store(N, self.n_store)

@@ -115,7 +115,7 @@ def test_q8_states_track_fp32_states():
         Wa, Wb = a.step(Wa, g, 1e-2), b.step(Wb, g, 1e-2)
     Ma, Va = a.moments()
     Mb, Vb = b.moments()
-    assert len(b.M_absmax) == (r * n + 255) // 256
+    assert b.M_absmax.shape == ((r + 1) // 2, (n + 127) // 128)        # q_block 256 = tiles of 2 x 128
     assert np.linalg.norm(Mb - Ma) / np.linalg.norm(Ma) < 0.05
     assert np.linalg.norm((Wb - W0) - (Wa - W0)) / np.linalg.norm(Wa - W0) < 0.1
     # first step does not depend on the state format at all (states start at zero)
@@ -123,3 +123,62 @@ def test_q8_states_track_fp32_states():
     b1 = go.GaLoreOracle(m, n, r, state="q8", q_block=256, **hp)
     g = wl.make_gradient(m, n, 3, 1.0, 0.01, "f64")
     assert np.array_equal(a1.step(W0, g, 1e-2), b1.step(W0, g, 1e-2))
+
+
+@pytest.mark.parametrize("signed", [True, False])
+@pytest.mark.parametrize("rows,cols,tr,tc", [(37, 300, 16, 128), (5, 128, 2, 128), (16, 129, 16, 128), (40, 90, 8, 32)])
+def test_tiles_brute_force_geometry_and_codes(signed, rows, cols, tr, tc):
+    """Which elements share an absmax, written out with explicit index arithmetic, and the nearest code by
+    exhaustive search over the 256 values."""
+    rng = np.random.default_rng(rows * 1000 + cols)
+    X = (rng.standard_normal((rows, cols)) * 10.0 ** rng.uniform(-5, 0, (rows, cols))).astype(np.float32)
+    if not signed:
+        X = np.abs(X)
+    codes, am = go.quantize_tiles(X, signed, tr, tc)
+    assert codes.shape == X.shape and am.shape == ((rows + tr - 1) // tr, (cols + tc - 1) // tc)
+    c = go.dynamic_code(signed).astype(np.float64)
+    for i in range(rows):
+        for j in range(cols):
+            I, J = i // tr, j // tc
+            a = np.float32(0)
+            for ii in range(I * tr, min(rows, (I + 1) * tr)):
+                for jj in range(J * tc, min(cols, (J + 1) * tc)):
+                    a = max(a, abs(X[ii, jj]))
+            assert am[I, J] == a
+            y = np.float64(X[i, j] / a)                                # fp32 quotient
+            dist = np.abs(c - y)
+            cand = np.nonzero(dist <= dist.min() * (1 + 1e-6) + 1e-12)[0]
+            assert codes[i, j] in cand
+    back = go.dequantize_tiles(codes, am, signed, tr, tc)
+    for i in range(0, rows, 3):
+        for j in range(0, cols, 7):
+            assert back[i, j] == np.float32(go.dynamic_code(signed)[codes[i, j]] * am[i // tr, j // tc])
+
+
+def test_one_large_element_changes_only_its_own_tile():
+    X = np.full((40, 300), 0.01, dtype=np.float32)
+    base_codes, base_am = go.quantize_tiles(X, True, 16, 128)
+    X[17, 130] = 5.0                                                    # tile (1, 1)
+    codes, am = go.quantize_tiles(X, True, 16, 128)
+    changed = np.argwhere(codes != base_codes)
+    assert am[1, 1] == 5.0 and np.count_nonzero(am != base_am) == 1
+    assert changed[:, 0].min() == 16 and changed[:, 0].max() == 31 and changed[:, 1].min() == 128 and changed[:, 1].max() == 255
+    assert len(changed) == 16 * 128 - 1          # every other element of that tile (the large one keeps the code of 1), nothing else
+
+
+def test_flat_blocks_are_tiles_of_a_one_row_matrix():
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal(1000).astype(np.float32)
+    c1, a1 = go.quantize_blockwise(x, True, 256)
+    c2, a2 = go.quantize_tiles(x.reshape(1, -1), True, 1, 256)
+    assert np.array_equal(c1, c2.ravel()) and np.array_equal(a1, a2.ravel()) and len(a1) == 4
+
+
+def test_state_tile_shapes():
+    assert go.state_tile(2048) == (16, 128) and go.state_tile(256) == (2, 128) and go.state_tile(4096) == (32, 128)
+    with pytest.raises(ValueError):
+        go.state_tile(1000)
+    o = go.GaLoreOracle(40, 300, 24, 0.25, 10, state="q8", q_block=2048)
+    assert o.M_codes.shape == (24, 300) and o.M_absmax.shape == (2, 3)
+    o = go.GaLoreOracle(300, 40, 24, 0.25, 10, state="q8", q_block=512)          # right side: state is m x r
+    assert o.V_codes.shape == (300, 24) and o.V_absmax.shape == (75, 1)
