@@ -92,7 +92,8 @@ typedef struct {
   int32_t g_dtype;         /* galore_dtype_t of G */
   int32_t p_dtype;         /* galore_dtype_t the projector is stored in */
   int32_t state_fmt;       /* galore_state_fmt_t of M, V */
-  int32_t q_block;         /* elements per quantisation block: 256, 512, 1024, 2048 or 4096 (0 = 2048) */
+  int32_t q_block;         /* elements per quantisation block: 256, 512, 1024, 2048 or 4096 (0 = 2048); a block is a
+                              tile of q_block / 128 consecutive rows x 128 consecutive columns of the state matrix */
   int32_t auto_refresh;    /* 1: galore_step refreshes P when (completed steps) mod T == 0 */
   int32_t path;            /* galore_path_t */
   /* refresh: block subspace iteration on a block of rank + refresh_oversample
@@ -132,7 +133,8 @@ typedef struct {
 /* Sizes of the two caller-allocated device buffers for one layer.
  * state_bytes covers P (rows x r, p_dtype), M and V (shape of R: r x n left,
  * m x r right; fp32, or uint8 codes plus one fp32 absmax per block) -- the
- * paper's  m r + 2 n r  elements for m <= n (Sec. 4.2).  Both buffers must be
+ * paper's  m r + 2 n r  elements for m <= n (Sec. 4.2), with the rows of M
+ * and V padded to 32 bytes.  Both buffers must be
  * 256-byte aligned.  Host-only; touches no device. */
 galore_status_t galore_query_bytes(const galore_config_t* cfg, size_t* state_bytes, size_t* workspace_bytes);
 
@@ -258,7 +260,8 @@ galore_status_t galore_get_unrounded_projector(galore_layer_t* layer, double* ds
 galore_status_t galore_set_projector(galore_layer_t* layer, const float* src, size_t src_bytes, void* stream);
 /* Stored (uncorrected) moments as fp32, shape of R row-major packed, device memory (8-bit states are dequantised). */
 galore_status_t galore_get_moments(galore_layer_t* layer, float* M, float* V, size_t bytes_each, void* stream);
-/* Raw 8-bit state: codes (uint8, shape of R) and per-block absmax (fp32); device memory. */
+/* Raw 8-bit state: codes (uint8, shape of R, packed) and per-block absmax (fp32, tile (I, J) of the
+ * state at I * ceil(cols / 128) + J); device memory. */
 galore_status_t galore_get_q8_state(galore_layer_t* layer, uint8_t* M_codes, float* M_absmax,
                                     uint8_t* V_codes, float* V_absmax, void* stream);
 /* Completed steps k.  A checkpoint is the caller's state buffer plus this counter. */
@@ -276,13 +279,16 @@ galore_status_t galore_device_status(galore_layer_t* layer, int32_t* flags, void
 /* The 256 fp32 code values, ascending, into host memory. is_signed != 0: the
  * first-moment code on [-1, 1]; 0: the second-moment code on [0, 1]. */
 galore_status_t galore_q8_codebook(int32_t is_signed, float* out256_host);
-/* x (fp32, count elements, device) -> codes (uint8) and absmax (fp32, one per
- * block of `block` consecutive elements, last block may be short).
- * code = nearest code value to fp32(x / absmax), ties to the larger index. */
-galore_status_t galore_q8_quantize(const float* x, int64_t count, int32_t is_signed, int32_t block,
-                                   uint8_t* codes, float* absmax, void* stream);
-galore_status_t galore_q8_dequantize(const uint8_t* codes, const float* absmax, int64_t count,
-                                     int32_t is_signed, int32_t block, float* out, void* stream);
+/* x (fp32, rows x cols packed, device) -> codes (uint8, rows x cols packed) and absmax (fp32, one per
+ * quantisation block).  The blocks are tiles of tile_rows x tile_cols elements of the matrix, tile
+ * (I, J) at absmax[I * ceil(cols / tile_cols) + J]; tiles on the lower and right edges are cut off
+ * at the border.  A flat array with blocks of b consecutive elements is rows = 1, tile 1 x b.
+ * code = nearest code value to fp32(x / absmax), ties to the larger index; absmax = 0 stores the
+ * code of 0.  The moments of a layer use tiles of (q_block / 128) x 128 of the state matrix. */
+galore_status_t galore_q8_quantize(const float* x, int64_t rows, int64_t cols, int32_t is_signed, int32_t tile_rows,
+                                   int32_t tile_cols, uint8_t* codes, float* absmax, void* stream);
+galore_status_t galore_q8_dequantize(const uint8_t* codes, const float* absmax, int64_t rows, int64_t cols,
+                                     int32_t is_signed, int32_t tile_rows, int32_t tile_cols, float* out, void* stream);
 
 /* ---- diagnostics ---------------------------------------------------------- */
 /* sizeof(galore_config_t) and sizeof(galore_refresh_info_t) as compiled, for bindings to check their marshalling. */

@@ -92,8 +92,10 @@ _PROTOTYPES = {
                                     C.POINTER(C.c_int64)]),
     "galore_device_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32), C.c_void_p]),
     "galore_q8_codebook": (C.c_int, [C.c_int32, C.POINTER(C.c_float)]),
-    "galore_q8_quantize": (C.c_int, [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
-    "galore_q8_dequantize": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
+    "galore_q8_quantize": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                     C.c_void_p, C.c_void_p]),
+    "galore_q8_dequantize": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
+                                       C.c_void_p, C.c_void_p]),
     "galore_abi_sizes": (C.c_int, [C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
     "galore_status_string": (C.c_char_p, [C.c_int]),
     "galore_last_cuda_error": (C.c_char_p, []),
@@ -163,19 +165,34 @@ def galore_q8_codebook(is_signed: bool):
     return list(out)
 
 
-def galore_q8_quantize(x: torch.Tensor, is_signed: bool, block: int = 2048, stream=None):
+STATE_TILE_COLS = 128
+
+
+def _tile_of(x, block, tile):
+    """(rows, cols, tile_rows, tile_cols) of a quantiser call: a flat tensor with `block` consecutive elements
+    per block, or a matrix with tile = (tile_rows, tile_cols)."""
+    if tile is None:
+        return 1, x.numel(), 1, block
+    assert x.dim() == 2
+    return x.shape[0], x.shape[1], tile[0], tile[1]
+
+
+def galore_q8_quantize(x: torch.Tensor, is_signed: bool, block: int = 2048, tile=None, stream=None):
     assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
-    n = x.numel()
-    codes = torch.empty(n, dtype=torch.uint8, device=x.device)
-    absmax = torch.empty((n + block - 1) // block, dtype=torch.float32, device=x.device)
-    _check(lib().galore_q8_quantize(x.data_ptr(), n, int(is_signed), block, codes.data_ptr(), absmax.data_ptr(),
+    rows, cols, tr, tc = _tile_of(x, block, tile)
+    codes = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+    grid = ((rows + tr - 1) // tr, (cols + tc - 1) // tc) if x.numel() else (0, 0)
+    absmax = torch.empty(grid if tile is not None else grid[0] * grid[1], dtype=torch.float32, device=x.device)
+    _check(lib().galore_q8_quantize(x.data_ptr(), rows, cols, int(is_signed), tr, tc, codes.data_ptr(), absmax.data_ptr(),
                                     _stream_ptr(stream)), "galore_q8_quantize")
     return codes, absmax
 
 
-def galore_q8_dequantize(codes: torch.Tensor, absmax: torch.Tensor, is_signed: bool, block: int = 2048, stream=None):
-    out = torch.empty(codes.numel(), dtype=torch.float32, device=codes.device)
-    _check(lib().galore_q8_dequantize(codes.data_ptr(), absmax.data_ptr(), codes.numel(), int(is_signed), block,
+def galore_q8_dequantize(codes: torch.Tensor, absmax: torch.Tensor, is_signed: bool, block: int = 2048, tile=None,
+                         stream=None):
+    rows, cols, tr, tc = _tile_of(codes, block, tile)
+    out = torch.empty(codes.shape, dtype=torch.float32, device=codes.device)
+    _check(lib().galore_q8_dequantize(codes.data_ptr(), absmax.data_ptr(), rows, cols, int(is_signed), tr, tc,
                                       out.data_ptr(), _stream_ptr(stream)), "galore_q8_dequantize")
     return out
 
@@ -297,13 +314,13 @@ class Layer:
         return M, V
 
     def get_q8_state(self, stream=None):
-        nel = self.state_shape[0] * self.state_shape[1]
-        qb = self.cfg.q_block or 2048
-        nblk = (nel + qb - 1) // qb
-        Mc = torch.empty(nel, dtype=torch.uint8, device=self.device)
-        Vc = torch.empty(nel, dtype=torch.uint8, device=self.device)
-        Ma = torch.empty(nblk, dtype=torch.float32, device=self.device)
-        Va = torch.empty(nblk, dtype=torch.float32, device=self.device)
+        rows, cols = self.state_shape
+        tr = (self.cfg.q_block or 2048) // STATE_TILE_COLS
+        grid = ((rows + tr - 1) // tr, (cols + STATE_TILE_COLS - 1) // STATE_TILE_COLS)
+        Mc = torch.empty(rows, cols, dtype=torch.uint8, device=self.device)
+        Vc = torch.empty(rows, cols, dtype=torch.uint8, device=self.device)
+        Ma = torch.empty(grid, dtype=torch.float32, device=self.device)
+        Va = torch.empty(grid, dtype=torch.float32, device=self.device)
         _check(lib().galore_get_q8_state(self.handle, Mc.data_ptr(), Ma.data_ptr(), Vc.data_ptr(), Va.data_ptr(),
                                          _stream_ptr(stream)), "galore_get_q8_state")
         return Mc, Ma, Vc, Va

@@ -2,67 +2,57 @@
 #pragma once
 
 #include "common.cuh"
+#include "q8_code.cuh"
 
 namespace galore {
 
-struct AdamParams {
-  float b1, b2;          // beta1, beta2
-  float omb1, omb2;      // 1 - beta1, 1 - beta2
-  float eps;
-  float inv_bc1, inv_bc2;  // 1 / (1 - beta^t), t = completed steps + 1
-};
+constexpr int kStateTileCols = 128;   // a quantisation block is a tile of q_block / 128 rows x 128 columns of the state
 
-// Where element i of the packed state (row-major, `cols` wide) sits in the R partials and in N,
-// whose rows may be padded (leading dimensions r_ld, n_ld) so that TMA can address them.
-struct StateGeom {
-  int64_t cols = 0, r_ld = 0, n_ld = 0;   // cols == 0: everything is packed
-  __host__ __device__ __forceinline__ int64_t r_index(int64_t i) const {
-    return (cols == 0 || r_ld == cols) ? i : (i / cols) * r_ld + (i % cols);
-  }
-  __host__ __device__ __forceinline__ int64_t n_index(int64_t i) const {
-    return (cols == 0 || n_ld == cols) ? i : (i / cols) * n_ld + (i % cols);
-  }
-};
-
-// One layer's share of a grouped Adam launch.
+// One layer's share of a grouped Adam launch.  The state (shape of R: rows x cols) is walked in tiles
+// of tile_rows x 128; R partials, N and the state arrays are row-major with their own row pitches.
 struct AdamItem {
   const float* Rpart;      // split-K partials of R
   int splits;
   int64_t split_stride;
-  int nel;                 // state elements
+  int rows, cols;          // shape of R, M, V
+  int64_t r_ld, n_ld, s_ld;  // row pitches (elements) of Rpart, Nout and the state arrays
   float *M, *V;            // fp32 moments, or
   uint8_t *Mc, *Vc;        // 8-bit codes with
-  float *Mam, *Vam;        // one absmax per quantisation block
+  float *Mam, *Vam;        // one absmax per tile, tile (I, J) at I * tiles_c + J
   void* Nout;              // normalised update (fp32 or bf16)
-  int cols, r_ld, n_ld;    // state row length and the row pitches of Rpart / Nout (cols == 0: packed)
-  int aligned16;           // set by adam_group_add: all arrays allow 16-byte vector accesses
-  int first_block;         // the item covers the layer's work blocks from this one on (0: the whole layer)
+  int tiles_c;             // set by adam_group_add: ceil(cols / 128)
+  int vec;                 // set by adam_group_add: bases and pitches allow the vector accesses of an interior tile
   AdamParams p;
   int32_t* status;
 };
 constexpr int kAdamGroup = 32;
 struct AdamGroup {
   AdamItem item[kAdamGroup];
-  int block_end[kAdamGroup];   // running total of work blocks
+  int block_end[kAdamGroup];   // running total of tiles
   int count;
 };
 // all items of a group share the state format, the quantisation block and the dtype of N
 galore_status_t adam_group_add(AdamGroup& g, const AdamItem& item, int32_t state_fmt, int q_block);
 galore_status_t launch_adam_group(const AdamGroup& g, int32_t state_fmt, int q_block, int32_t n_dtype, cudaStream_t st);
+// one layer
+galore_status_t launch_adam(const AdamItem& item, int32_t state_fmt, int q_block, int32_t n_dtype, cudaStream_t st);
 
-// R arrives as `splits` fp32 partial sums, each `split_stride` elements apart.
-galore_status_t launch_adam_f32(const float* Rpart, int splits, int64_t split_stride, int64_t nel, float* M,
-                                float* V, void* Nout, int32_t n_dtype, const AdamParams& p, int32_t* status,
-                                cudaStream_t st, const StateGeom& g = StateGeom());
-galore_status_t launch_adam_q8(const float* Rpart, int splits, int64_t split_stride, int64_t nel, uint8_t* Mc,
-                               float* Mam, uint8_t* Vc, float* Vam, int block, void* Nout, int32_t n_dtype,
-                               const AdamParams& p, int32_t* status, cudaStream_t st,
-                               const StateGeom& g = StateGeom());
-galore_status_t launch_q8_quantize(const float* x, int64_t nel, int is_signed, int block, uint8_t* codes,
-                                   float* absmax, cudaStream_t st);
-galore_status_t launch_q8_dequantize(const uint8_t* codes, const float* absmax, int64_t nel, int is_signed,
-                                     int block, float* out, cudaStream_t st);
+// Pitches and sizes of a layer's state arrays.  fp32 moments: rows of ceil8(cols) floats; 8-bit codes:
+// rows of ceil32(cols) bytes, plus ceil(rows / (q_block / 128)) * ceil(cols / 128) absmax values.
+inline int64_t state_pitch(int32_t state_fmt, int64_t cols) {
+  return state_fmt == GALORE_STATE_F32 ? (cols + 7) / 8 * 8 : (cols + 31) / 32 * 32;
+}
+inline int64_t state_tiles(int64_t rows, int64_t cols, int q_block) {
+  return ceil_div(rows, q_block / kStateTileCols) * ceil_div(cols, kStateTileCols);
+}
+
+// x (rows x cols fp32, pitch ldx) -> codes (pitch ldc) and one absmax per tile_rows x tile_cols tile
+galore_status_t launch_q8_quantize(const float* x, int64_t rows, int64_t cols, int64_t ldx, int is_signed, int tile_rows,
+                                   int tile_cols, uint8_t* codes, int64_t ldc, float* absmax, cudaStream_t st);
+galore_status_t launch_q8_dequantize(const uint8_t* codes, int64_t ldc, const float* absmax, int64_t rows, int64_t cols,
+                                     int is_signed, int tile_rows, int tile_cols, float* out, int64_t ldo, cudaStream_t st);
 galore_status_t q8_ensure_tables();
+galore_status_t q8_table_ptrs(Q8TablePtrs* out);   // device addresses on the current device (fills the tables first)
 void q8_host_codebook(bool is_signed, float* out256);
 
 }  // namespace galore

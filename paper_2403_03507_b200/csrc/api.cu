@@ -77,6 +77,7 @@ struct galore_layer {
   int proj_splits;       // K slices of the projection on the fp32 path
   int tc_splits;         // K slices of the projection on the tensor-core path
   int64_t ld_part, ld_n; // padded row pitches of the R partials and of N on the tensor-core path
+  int64_t ld_s;          // row pitch of the state arrays (fp32 moments: floats, 8-bit codes: bytes)
   int32_t n_dtype;       // dtype of the normalised update handed to the back-projection
   int64_t k;             // completed steps
   // device memory (all inside the caller's two buffers)
@@ -98,7 +99,7 @@ struct Sizes {
   bool left;
   int64_t d, L, srows, scols, nel, nblk;
   int q_block, block, proj_splits, tc_splits;
-  int64_t ld_part, ld_n;
+  int64_t ld_part, ld_n, ld_s;
   bool tensor_path;
   size_t off_P, off_M, off_V, off_Mam, off_Vam, state_bytes;
   size_t off_status, off_R, off_N, off_refresh, ws_bytes;
@@ -127,7 +128,10 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
   s->srows = s->left ? r : c->m;
   s->scols = s->left ? c->n : r;
   s->nel = s->srows * s->scols;
-  s->nblk = ceil_div(s->nel, s->q_block);
+  s->ld_s = state_pitch(c->state_fmt, s->scols);
+  s->nblk = state_tiles(s->srows, s->scols, s->q_block);
+  // the kernels count tiles and address rows of one matrix with 32-bit integers
+  if (s->srows * std::max<int64_t>(s->ld_s, (s->scols + 7) / 8 * 8) >= ((int64_t)1 << 31) - 4096) return GALORE_ERR_SHAPE;
   const bool eligible = tensor_path_eligible(*c);
   if (c->path == GALORE_PATH_TENSOR && !eligible) return GALORE_ERR_UNIMPLEMENTED;
   s->tensor_path = eligible && c->path != GALORE_PATH_FP32;
@@ -156,12 +160,12 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
   size_t o = 0;
   s->off_P = o; o += align_up((size_t)s->d * r * dtype_size(c->p_dtype), 256);
   if (c->state_fmt == GALORE_STATE_F32) {
-    s->off_M = o; o += align_up((size_t)s->nel * 4, 256);
-    s->off_V = o; o += align_up((size_t)s->nel * 4, 256);
+    s->off_M = o; o += align_up((size_t)s->srows * s->ld_s * 4, 256);
+    s->off_V = o; o += align_up((size_t)s->srows * s->ld_s * 4, 256);
     s->off_Mam = s->off_Vam = o;
   } else {
-    s->off_M = o; o += align_up((size_t)s->nel, 256);
-    s->off_V = o; o += align_up((size_t)s->nel, 256);
+    s->off_M = o; o += align_up((size_t)s->srows * s->ld_s, 256);
+    s->off_V = o; o += align_up((size_t)s->srows * s->ld_s, 256);
     s->off_Mam = o; o += align_up((size_t)s->nblk * 4, 256);
     s->off_Vam = o; o += align_up((size_t)s->nblk * 4, 256);
   }
@@ -199,6 +203,20 @@ galore_status_t project_simt(galore_layer* l, const void* G, int64_t ldg, cudaSt
                                          l->proj_splits, epi, st);
 }
 
+// the layer's share of an Adam launch: R partials in `part` (pitch r_ld), N to `nbuf` (pitch n_ld)
+AdamItem adam_item(const galore_layer* l, const float* part, int splits, int64_t split_stride, int64_t r_ld, void* nbuf,
+                   int64_t n_ld, const AdamParams& ap) {
+  AdamItem a = {};
+  a.Rpart = part; a.splits = splits; a.split_stride = split_stride;
+  a.rows = (int)l->srows; a.cols = (int)l->scols;
+  a.r_ld = r_ld; a.n_ld = n_ld; a.s_ld = l->ld_s;
+  a.M = l->M; a.V = l->V; a.Mc = l->Mc; a.Vc = l->Vc; a.Mam = l->Mam; a.Vam = l->Vam;
+  a.Nout = nbuf;
+  a.p = ap;
+  a.status = l->status;
+  return a;
+}
+
 // GaLore-AdamW: W is multiplied by 1 - lr * lambda in the pass that subtracts the update (exactly 1 for lambda = 0)
 inline float decay_keep(const galore_layer* l, float lr) { return (float)(1.0 - (double)lr * (double)l->cfg.weight_decay); }
 
@@ -226,11 +244,8 @@ galore_status_t step_simt(galore_layer* l, void* W, int64_t ldw, const void* G, 
   }
   {
     PhaseTimer pt(1, st);
-    if (l->cfg.state_fmt == GALORE_STATE_F32)
-      GALORE_TRY(launch_adam_f32(l->Rpart, l->proj_splits, l->nel, l->nel, l->M, l->V, l->Nbuf, GALORE_F32, ap, l->status, st));
-    else
-      GALORE_TRY(launch_adam_q8(l->Rpart, l->proj_splits, l->nel, l->nel, l->Mc, l->Mam, l->Vc, l->Vam, l->q_block, l->Nbuf,
-                                GALORE_F32, ap, l->status, st));
+    GALORE_TRY(launch_adam(adam_item(l, l->Rpart, l->proj_splits, l->nel, l->scols, l->Nbuf, l->scols, ap), l->cfg.state_fmt,
+                           l->q_block, GALORE_F32, st));
   }
   PhaseTimer pt(2, st);
   const float scale = lr * l->cfg.alpha, keep = decay_keep(l, lr);
@@ -249,17 +264,8 @@ galore_status_t step_tensor(galore_layer* l, void* W, int64_t ldw, const void* G
   }
   {
     PhaseTimer pt(1, st);
-    StateGeom g;
-    g.cols = l->scols;
-    g.r_ld = l->ld_part;
-    g.n_ld = l->ld_n;
-    const int64_t split_stride = l->srows * l->ld_part;
-    if (l->cfg.state_fmt == GALORE_STATE_F32)
-      GALORE_TRY(launch_adam_f32(l->Rpart, l->tc.splits, split_stride, l->nel, l->M, l->V, l->Nbuf, GALORE_BF16, ap,
-                                 l->status, st, g));
-    else
-      GALORE_TRY(launch_adam_q8(l->Rpart, l->tc.splits, split_stride, l->nel, l->Mc, l->Mam, l->Vc, l->Vam, l->q_block,
-                                l->Nbuf, GALORE_BF16, ap, l->status, st, g));
+    GALORE_TRY(launch_adam(adam_item(l, l->Rpart, l->tc.splits, l->srows * l->ld_part, l->ld_part, l->Nbuf, l->ld_n, ap),
+                           l->cfg.state_fmt, l->q_block, GALORE_BF16, st));
   }
   PhaseTimer pt(2, st);
   return tensor_back_project(&l->tc, l->cfg, l->left, W, ldw, lr * l->cfg.alpha, decay_keep(l, lr), l->status, st);
@@ -319,7 +325,7 @@ galore_status_t galore_init_layer(const galore_config_t* cfg, void* state_buf, s
   l->has_projector = false;
   l->d = s.d; l->L = s.L; l->srows = s.srows; l->scols = s.scols; l->nel = s.nel;
   l->q_block = s.q_block; l->nblk = s.nblk; l->block = s.block; l->proj_splits = s.proj_splits;
-  l->tc_splits = s.tc_splits; l->ld_part = s.ld_part; l->ld_n = s.ld_n;
+  l->tc_splits = s.tc_splits; l->ld_part = s.ld_part; l->ld_n = s.ld_n; l->ld_s = s.ld_s;
   l->n_dtype = s.tensor_path ? GALORE_BF16 : GALORE_F32;
   l->k = 0;
   char* sb = (char*)state_buf;
@@ -342,11 +348,11 @@ galore_status_t galore_init_layer(const galore_config_t* cfg, void* state_buf, s
 
   cudaError_t e = cudaSuccess;
   if (cfg->state_fmt == GALORE_STATE_F32) {
-    e = cudaMemsetAsync(l->M, 0, (size_t)l->nel * 4, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(l->V, 0, (size_t)l->nel * 4, st);
+    e = cudaMemsetAsync(l->M, 0, (size_t)l->srows * l->ld_s * 4, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(l->V, 0, (size_t)l->srows * l->ld_s * 4, st);
   } else {
-    e = cudaMemsetAsync(l->Mc, 127, (size_t)l->nel, st);   // 127 and 0 are the codes of the value 0
-    if (e == cudaSuccess) e = cudaMemsetAsync(l->Vc, 0, (size_t)l->nel, st);
+    e = cudaMemsetAsync(l->Mc, 127, (size_t)l->srows * l->ld_s, st);   // 127 and 0 are the codes of the value 0
+    if (e == cudaSuccess) e = cudaMemsetAsync(l->Vc, 0, (size_t)l->srows * l->ld_s, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(l->Mam, 0, (size_t)l->nblk * 4, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(l->Vam, 0, (size_t)l->nblk * 4, st);
   }
@@ -703,16 +709,7 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
       galore_layer* l = layers[mb.index];
       float* part; void* nbuf;
       scratch_of(gi, mb, &part, &nbuf);
-      AdamItem a = {};
-      a.Rpart = part;
-      a.splits = mb.splits;
-      a.split_stride = l->srows * l->ld_part;
-      a.nel = (int)l->nel;
-      a.M = l->M; a.V = l->V; a.Mc = l->Mc; a.Vc = l->Vc; a.Mam = l->Mam; a.Vam = l->Vam;
-      a.Nout = nbuf;
-      a.cols = (int)l->scols; a.r_ld = (int)l->ld_part; a.n_ld = (int)l->ld_n;
-      a.p = adam_params(l);
-      a.status = l->status;
+      const AdamItem a = adam_item(l, part, mb.splits, l->srows * l->ld_part, l->ld_part, nbuf, l->ld_n, adam_params(l));
       GALORE_TRY(adam_group_add(*scratch.adam, a, l->cfg.state_fmt, l->q_block));
     }
     PhaseTimer pt(1, s);
@@ -792,20 +789,23 @@ galore_status_t galore_get_moments(galore_layer_t* l, float* M, float* V, size_t
   if (bytes_each < (size_t)l->nel * 4) return GALORE_ERR_BUFFER_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
   if (l->cfg.state_fmt == GALORE_STATE_F32) {
-    GALORE_CUDA_TRY(cudaMemcpyAsync(M, l->M, (size_t)l->nel * 4, cudaMemcpyDeviceToDevice, st));
-    GALORE_CUDA_TRY(cudaMemcpyAsync(V, l->V, (size_t)l->nel * 4, cudaMemcpyDeviceToDevice, st));
+    const size_t row = (size_t)l->scols * 4;
+    GALORE_CUDA_TRY(cudaMemcpy2DAsync(M, row, l->M, (size_t)l->ld_s * 4, row, (size_t)l->srows, cudaMemcpyDeviceToDevice, st));
+    GALORE_CUDA_TRY(cudaMemcpy2DAsync(V, row, l->V, (size_t)l->ld_s * 4, row, (size_t)l->srows, cudaMemcpyDeviceToDevice, st));
     return GALORE_OK;
   }
-  GALORE_TRY(launch_q8_dequantize(l->Mc, l->Mam, l->nel, 1, l->q_block, M, st));
-  return launch_q8_dequantize(l->Vc, l->Vam, l->nel, 0, l->q_block, V, st);
+  const int tr = l->q_block / kStateTileCols;
+  GALORE_TRY(launch_q8_dequantize(l->Mc, l->ld_s, l->Mam, l->srows, l->scols, 1, tr, kStateTileCols, M, l->scols, st));
+  return launch_q8_dequantize(l->Vc, l->ld_s, l->Vam, l->srows, l->scols, 0, tr, kStateTileCols, V, l->scols, st);
 }
 
 galore_status_t galore_get_q8_state(galore_layer_t* l, uint8_t* Mc, float* Mam, uint8_t* Vc, float* Vam, void* stream) {
   if (!l || !Mc || !Mam || !Vc || !Vam) return GALORE_ERR_INVALID_ARG;
   if (l->cfg.state_fmt != GALORE_STATE_Q8_BLOCK) return GALORE_ERR_STATE;
   cudaStream_t st = (cudaStream_t)stream;
-  GALORE_CUDA_TRY(cudaMemcpyAsync(Mc, l->Mc, (size_t)l->nel, cudaMemcpyDeviceToDevice, st));
-  GALORE_CUDA_TRY(cudaMemcpyAsync(Vc, l->Vc, (size_t)l->nel, cudaMemcpyDeviceToDevice, st));
+  const size_t row = (size_t)l->scols;
+  GALORE_CUDA_TRY(cudaMemcpy2DAsync(Mc, row, l->Mc, (size_t)l->ld_s, row, (size_t)l->srows, cudaMemcpyDeviceToDevice, st));
+  GALORE_CUDA_TRY(cudaMemcpy2DAsync(Vc, row, l->Vc, (size_t)l->ld_s, row, (size_t)l->srows, cudaMemcpyDeviceToDevice, st));
   GALORE_CUDA_TRY(cudaMemcpyAsync(Mam, l->Mam, (size_t)l->nblk * 4, cudaMemcpyDeviceToDevice, st));
   GALORE_CUDA_TRY(cudaMemcpyAsync(Vam, l->Vam, (size_t)l->nblk * 4, cudaMemcpyDeviceToDevice, st));
   return GALORE_OK;
@@ -850,16 +850,16 @@ galore_status_t galore_q8_codebook(int32_t is_signed, float* out256_host) {
   return GALORE_OK;
 }
 
-galore_status_t galore_q8_quantize(const float* x, int64_t count, int32_t is_signed, int32_t block, uint8_t* codes,
-                                   float* absmax, void* stream) {
-  if (count < 0 || (count > 0 && (!x || !codes || !absmax))) return GALORE_ERR_INVALID_ARG;
-  return launch_q8_quantize(x, count, is_signed, block == 0 ? 2048 : block, codes, absmax, (cudaStream_t)stream);
+galore_status_t galore_q8_quantize(const float* x, int64_t rows, int64_t cols, int32_t is_signed, int32_t tile_rows,
+                                   int32_t tile_cols, uint8_t* codes, float* absmax, void* stream) {
+  if (rows < 0 || cols < 0 || (rows > 0 && cols > 0 && (!x || !codes || !absmax))) return GALORE_ERR_INVALID_ARG;
+  return launch_q8_quantize(x, rows, cols, cols, is_signed, tile_rows, tile_cols, codes, cols, absmax, (cudaStream_t)stream);
 }
 
-galore_status_t galore_q8_dequantize(const uint8_t* codes, const float* absmax, int64_t count, int32_t is_signed,
-                                     int32_t block, float* out, void* stream) {
-  if (count < 0 || (count > 0 && (!codes || !absmax || !out))) return GALORE_ERR_INVALID_ARG;
-  return launch_q8_dequantize(codes, absmax, count, is_signed, block == 0 ? 2048 : block, out, (cudaStream_t)stream);
+galore_status_t galore_q8_dequantize(const uint8_t* codes, const float* absmax, int64_t rows, int64_t cols,
+                                     int32_t is_signed, int32_t tile_rows, int32_t tile_cols, float* out, void* stream) {
+  if (rows < 0 || cols < 0 || (rows > 0 && cols > 0 && (!codes || !absmax || !out))) return GALORE_ERR_INVALID_ARG;
+  return launch_q8_dequantize(codes, cols, absmax, rows, cols, is_signed, tile_rows, tile_cols, out, cols, (cudaStream_t)stream);
 }
 
 const char* galore_status_string(galore_status_t s) {

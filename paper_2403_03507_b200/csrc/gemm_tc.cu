@@ -4,10 +4,15 @@
 // store split-K partial sums of R or apply the update to W in place
 // (Algorithm 1: R = P^T G resp. G Q;  W <- W - lr * alpha * P N resp. N Q^T).
 //
-// One persistent CTA per SM, six warps:
+// With one K slice per output tile the projection's epilogue also runs Adam on its tile of R
+// (moment update, bias correction, Eq. 15, 8-bit dequantisation and requantisation of the moments)
+// and writes the normalised update N for the back-projection: R never reaches memory.
+//
+// One persistent CTA per SM:
 //   warp 0        TMA producer: fills a ring of kStages shared-memory stages
 //   warp 1        MMA issuer (one lane) and owner of the tensor-memory allocation
-//   warps 2..5    epilogue: tcgen05.ld of a finished accumulator, then global memory
+//   warps 2..     epilogue (four warps, eight when it runs Adam): tcgen05.ld of a finished
+//                 accumulator, then global memory
 // Two accumulators of kBN columns alternate, so the epilogue of one tile runs
 // under the MMAs of the next.  Work units are (tile_m, tile_n, K slice); the
 // K slices of one output tile go to separate partial buffers that the Adam
@@ -19,6 +24,8 @@
 #include "gemm_tc.cuh"
 
 #include <cudaTypedefs.h>
+
+#include "adam.cuh"
 
 #include <algorithm>
 #include <memory>
@@ -33,10 +40,8 @@ constexpr int kBM = 128;          // rows of an output tile = TMEM lanes
 constexpr int kBN = 256;          // columns of an output tile = TMEM columns per accumulator
 constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;
-constexpr int kThreads = 192;        // producer warp, MMA warp, four epilogue warps
 constexpr uint32_t kTmemCols = 512;
 constexpr int kABytes = kBM * kBK * 2;            // 16 KiB: the 128 rows of A one CTA stages per k-block
-constexpr int kMaxStages = 6;
 
 // CTAS = 1: one CTA computes a 128 x 256 tile.  CTAS = 2: a cluster of two CTAs computes 256 x 256
 // with cta_group::2 MMAs; each CTA stages its own 128 rows of A and half (128 columns) of B, so a
@@ -55,7 +60,15 @@ constexpr long long kWaitLimitCycles = 4000000000LL;   // about two seconds
 // EPI_APPLY_DECAY is EPI_APPLY with W multiplied by TcParams::keep first (GaLore-AdamW).  It is an
 // instantiation of its own: the same code with the multiply behind a run-time test made the plain
 // update 15 % slower at K = 512.
-enum { EPI_PARTIAL = 0, EPI_APPLY = 1, EPI_APPLY_DECAY = 2 };
+// EPI_ADAM_F32 / EPI_ADAM_Q8: the projection with Adam on its output tile (fp32 / 8-bit moments).
+enum { EPI_PARTIAL = 0, EPI_APPLY = 1, EPI_APPLY_DECAY = 2, EPI_ADAM_F32 = 3, EPI_ADAM_Q8 = 4 };
+constexpr bool epi_is_adam(int epi) { return epi == EPI_ADAM_F32 || epi == EPI_ADAM_Q8; }
+// Adam is instruction-heavy (about 70 per element with 8-bit moments): eight epilogue warps, two
+// per quarter of the accumulator's lanes with 128 columns each, keep every scheduler of the SM busy
+// while the tensor cores work on the next tile.
+constexpr int epi_warps(int epi) { return epi_is_adam(epi) ? 8 : 4; }
+constexpr int epi_threads(int epi) { return 64 + 32 * epi_warps(epi); }     // + producer warp and MMA warp
+constexpr int epi_smem(int epi) { return epi == EPI_ADAM_Q8 ? (int)sizeof(Q8Tables) : 0; }
 
 constexpr int kMaxGroup = 32;     // problems one launch can carry (its arguments travel as kernel parameters)
 
@@ -76,6 +89,16 @@ struct TcParams {
   float scale;
   float keep;                 // EPI_APPLY_DECAY: W is multiplied by this before the update is subtracted
   int32_t* status;
+  // EPI_ADAM_*: the state of the layer (rows x cols of the output, row pitch ld_s) and where N goes
+  float *Ms, *Vs;             // fp32 moments, or
+  uint8_t *Mc, *Vc;           // 8-bit codes with
+  float *Mam, *Vam;           // one absmax per tile of q_rows x 128 state elements, tile (I, J) at I * q_tiles_c + J
+  int64_t ld_s;
+  int q_rows, q_tiles_c;
+  __nv_bfloat16* Nout;
+  int64_t ld_n;
+  int adam_vec;               // bases and pitches of the state and of N allow 32-byte accesses
+  AdamParams ap;
 };
 
 // One launch = up to kMaxGroup independent problems; work units are numbered across them.
@@ -85,6 +108,7 @@ struct TcGroup {
   TcParams p[kMaxGroup];
   int unit_end[kMaxGroup];    // running total of units: problem i owns [unit_end[i-1], unit_end[i])
   int count;
+  Q8TablePtrs q8;             // EPI_ADAM_Q8: the code tables in global memory
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------
@@ -354,12 +378,230 @@ __device__ __forceinline__ void epi_apply(const TcParams& p, int row, int col0, 
   }
 }
 
+
+// ---- Adam in the projection's epilogue ----------------------------------------------------------
+// The thread owns row `row` of R and the 128 columns from col0 on (Algorithm 1, the update block on
+// its part of R; Eq. 15 for N).  Rows and columns outside the matrix hold exact zeros in the
+// accumulator (TMA fills out-of-range operand elements with zeros).
+
+__device__ __forceinline__ void st_n32(__nv_bfloat16* dst, const float (&n)[32], bool vec, int valid) {
+  if (vec) {
+    uint32_t w[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const __nv_bfloat162 h = __floats2bfloat162_rn(n[2 * j], n[2 * j + 1]);
+      w[j] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    st_global_32B(dst, make_uint4(w[0], w[1], w[2], w[3]), make_uint4(w[4], w[5], w[6], w[7]));
+    st_global_32B(dst + 16, make_uint4(w[8], w[9], w[10], w[11]), make_uint4(w[12], w[13], w[14], w[15]));
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (j < valid) dst[j] = __float2bfloat16_rn(n[j]);
+  }
+}
+
+// fp32 moments: one pass, 32 columns at a time
+__device__ __forceinline__ bool epi_adam_f32(const TcParams& p, int row, int col0, uint32_t t_addr, uint32_t accf,
+                                             uint32_t acc_phase, volatile int* abort_flag, bool& ok) {
+  const bool row_ok = row < p.M;
+  const int ncols = row_ok ? max(0, min(128, p.N - col0)) : 0;       // columns of this thread inside the matrix
+  const bool vec = p.adam_vec != 0;
+  const AdamParams ap = p.ap;
+  const int64_t so = (int64_t)row * p.ld_s + col0;
+  float* __restrict__ Mrow = p.Ms + so;
+  float* __restrict__ Vrow = p.Vs + so;
+  __nv_bfloat16* __restrict__ Nrow = p.Nout + (int64_t)row * p.ld_n + col0;
+  float m[32], v[32];
+  auto fetch = [&](int c) {
+    const int valid = ncols - c;
+    if (valid >= 32 && vec) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 8) {
+        uint4 a, b;
+        ld_global_32B(Mrow + c + j, a, b);
+        m[j] = __uint_as_float(a.x); m[j + 1] = __uint_as_float(a.y); m[j + 2] = __uint_as_float(a.z); m[j + 3] = __uint_as_float(a.w);
+        m[j + 4] = __uint_as_float(b.x); m[j + 5] = __uint_as_float(b.y); m[j + 6] = __uint_as_float(b.z); m[j + 7] = __uint_as_float(b.w);
+        ld_global_32B(Vrow + c + j, a, b);
+        v[j] = __uint_as_float(a.x); v[j + 1] = __uint_as_float(a.y); v[j + 2] = __uint_as_float(a.z); v[j + 3] = __uint_as_float(a.w);
+        v[j + 4] = __uint_as_float(b.x); v[j + 5] = __uint_as_float(b.y); v[j + 6] = __uint_as_float(b.z); v[j + 7] = __uint_as_float(b.w);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        m[j] = j < valid ? Mrow[c + j] : 0.f;
+        v[j] = j < valid ? Vrow[c + j] : 0.f;
+      }
+    }
+  };
+  fetch(0);                                   // does not depend on the MMAs: in flight while the tile is computed
+  // the decision is taken by the warp as a whole: what follows is warp-synchronous
+  if (!__all_sync(0xffffffffu, mbar_wait(accf, acc_phase, abort_flag))) { ok = false; return false; }
+  tc_fence_after();
+  uint32_t top = 0u;      // largest bit pattern among the new second moments (all >= 0): a non-finite r shows here
+#pragma unroll 1
+  for (int c = 0; c < 128; c += 32) {
+    const int valid = ncols - c;
+    if (!__any_sync(0xffffffffu, valid > 0)) break;      // the whole warp is past the last column
+    if (c > 0) fetch(c);
+    uint32_t acc[32];
+    tmem_ld_32x32(t_addr + (uint32_t)c, acc);
+    tmem_ld_wait();
+    float n[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const float r = __uint_as_float(acc[j]);
+      m[j] = adam_m(m[j], r, ap);
+      v[j] = adam_v(v[j], r, ap);
+      n[j] = adam_normalised(m[j], v[j], ap);
+      top = max(top, __float_as_uint(v[j]));
+    }
+    if (valid >= 32 && vec) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 8) {
+        st_global_32B(Mrow + c + j, make_uint4(__float_as_uint(m[j]), __float_as_uint(m[j + 1]), __float_as_uint(m[j + 2]), __float_as_uint(m[j + 3])),
+                      make_uint4(__float_as_uint(m[j + 4]), __float_as_uint(m[j + 5]), __float_as_uint(m[j + 6]), __float_as_uint(m[j + 7])));
+        st_global_32B(Vrow + c + j, make_uint4(__float_as_uint(v[j]), __float_as_uint(v[j + 1]), __float_as_uint(v[j + 2]), __float_as_uint(v[j + 3])),
+                      make_uint4(__float_as_uint(v[j + 4]), __float_as_uint(v[j + 5]), __float_as_uint(v[j + 6]), __float_as_uint(v[j + 7])));
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j < valid) {
+          Mrow[c + j] = m[j];
+          Vrow[c + j] = v[j];
+        }
+    }
+    st_n32(Nrow + c, n, valid >= 32 && vec, valid);
+  }
+  return top >= 0x7f800000u;
+}
+
+// 8-bit moments.  A quantisation block is a tile of q_rows x 128 state elements: q_rows lanes of this
+// warp hold all of it, so its absmax is a warp-shuffle reduction.  Two passes over the accumulator:
+// the first finds the block's absmax of the updated moments, the second recomputes them (the same
+// instructions, hence the same bits), writes N and the new codes.
+__device__ __forceinline__ bool epi_adam_q8(const TcParams& p, int row, int col0, uint32_t t_addr, uint32_t accf,
+                                            uint32_t acc_phase, volatile int* abort_flag, const Q8Tables& t, bool& ok) {
+  const bool row_ok = row < p.M;
+  const int ncols = row_ok ? max(0, min(128, p.N - col0)) : 0;
+  const bool vec = p.adam_vec != 0 && ncols == 128;
+  const AdamParams ap = p.ap;
+  const int64_t so = (int64_t)row * p.ld_s + col0;
+  uint8_t* __restrict__ Mrow = p.Mc + so;
+  uint8_t* __restrict__ Vrow = p.Vc + so;
+  __nv_bfloat16* __restrict__ Nrow = p.Nout + (int64_t)row * p.ld_n + col0;
+  const int tile = ncols > 0 ? (row / p.q_rows) * p.q_tiles_c + (col0 >> 7) : 0;
+  // old codes of the thread's 128 elements (zero codes outside the matrix) and the block's old absmax:
+  // none of it depends on the MMAs, so it is in flight while the tile is computed
+  uint32_t cm[32], cv[32];
+  if (vec) {
+#pragma unroll
+    for (int j = 0; j < 32; j += 8) {
+      uint4 a, b;
+      ld_global_32B(Mrow + 4 * j, a, b);
+      cm[j] = a.x; cm[j + 1] = a.y; cm[j + 2] = a.z; cm[j + 3] = a.w; cm[j + 4] = b.x; cm[j + 5] = b.y; cm[j + 6] = b.z; cm[j + 7] = b.w;
+      ld_global_32B(Vrow + 4 * j, a, b);
+      cv[j] = a.x; cv[j + 1] = a.y; cv[j + 2] = a.z; cv[j + 3] = a.w; cv[j + 4] = b.x; cv[j + 5] = b.y; cv[j + 6] = b.z; cv[j + 7] = b.w;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      uint32_t wm = 0u, wv = 0u;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const bool in = 4 * j + k < ncols;
+        wm |= (in ? (uint32_t)Mrow[4 * j + k] : 127u) << (8 * k);
+        wv |= (in ? (uint32_t)Vrow[4 * j + k] : 0u) << (8 * k);
+      }
+      cm[j] = wm;
+      cv[j] = wv;
+    }
+  }
+  const float am_m = ncols > 0 ? p.Mam[tile] : 0.f, am_v = ncols > 0 ? p.Vam[tile] : 0.f;
+  // the decision is taken by the warp as a whole: what follows is warp-synchronous
+  if (!__all_sync(0xffffffffu, mbar_wait(accf, acc_phase, abort_flag))) { ok = false; return false; }
+  tc_fence_after();
+  if (!__any_sync(0xffffffffu, ncols > 0)) return false;   // the warp's part of the tile lies outside the matrix
+
+  // ---- pass 1: absmax of the updated moments over the block
+  float mx_m = 0.f;
+  uint32_t mx_vb = 0u;          // v >= 0: bit order is value order; a NaN or an infinity ends up on top
+#pragma unroll
+  for (int c = 0; c < 128; c += 32) {
+    uint32_t acc[32];
+    tmem_ld_32x32(t_addr + (uint32_t)c, acc);
+    tmem_ld_wait();
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const float r = __uint_as_float(acc[j]);
+      const uint32_t im = (cm[(c + j) >> 2] >> (8 * (j & 3))) & 0xffu, iv = (cv[(c + j) >> 2] >> (8 * (j & 3))) & 0xffu;
+      const float m = adam_m(__fmul_rn(t.code_s[im], am_m), r, ap);
+      const float v = adam_v(__fmul_rn(t.code_u[iv], am_v), r, ap);
+      mx_m = fmaxf(mx_m, fabsf(m));
+      mx_vb = max(mx_vb, __float_as_uint(v));
+    }
+  }
+  for (int o = 1; o < p.q_rows; o <<= 1) {      // the q_rows lanes of the block (a power of two up to 32)
+    mx_m = fmaxf(mx_m, __shfl_xor_sync(0xffffffffu, mx_m, o));
+    mx_vb = max(mx_vb, __shfl_xor_sync(0xffffffffu, mx_vb, o));
+  }
+  const bool bad = mx_vb >= 0x7f800000u;
+  const float mx_v = __uint_as_float(mx_vb);
+  // an all-zero block: with 0 in place of the reciprocal every y' is 0 and takes the code of zero
+  const float inv_m = mx_m != 0.f ? 1.0f / mx_m : 0.f, inv_v = mx_v != 0.f ? 1.0f / mx_v : 0.f;
+
+  // ---- pass 2: N and the new codes
+#pragma unroll
+  for (int c = 0; c < 128; c += 32) {
+    uint32_t acc[32];
+    if (!__any_sync(0xffffffffu, ncols - c > 0)) break;  // the whole warp is past the last column
+    tmem_ld_32x32(t_addr + (uint32_t)c, acc);
+    tmem_ld_wait();
+    float n[32];
+    uint32_t pm[8], pv[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      float xm[4], xv[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int j = 4 * q + k;
+        const float r = __uint_as_float(acc[j]);
+        const uint32_t im = (cm[(c + j) >> 2] >> (8 * k)) & 0xffu, iv = (cv[(c + j) >> 2] >> (8 * k)) & 0xffu;
+        xm[k] = adam_m(__fmul_rn(t.code_s[im], am_m), r, ap);
+        xv[k] = adam_v(__fmul_rn(t.code_u[iv], am_v), r, ap);
+        n[j] = adam_normalised(xm[k], xv[k], ap);
+      }
+      pm[q] = q8_encode4<true>(xm, mx_m, inv_m, t.enc_s, t.mid_s);
+      pv[q] = q8_encode4<false>(xv, mx_v, inv_v, t.enc_u, t.mid_u);
+    }
+    if (vec) {
+      st_global_32B(Mrow + c, make_uint4(pm[0], pm[1], pm[2], pm[3]), make_uint4(pm[4], pm[5], pm[6], pm[7]));
+      st_global_32B(Vrow + c, make_uint4(pv[0], pv[1], pv[2], pv[3]), make_uint4(pv[4], pv[5], pv[6], pv[7]));
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (c + j < ncols) {
+          Mrow[c + j] = (uint8_t)(pm[j >> 2] >> (8 * (j & 3)));
+          Vrow[c + j] = (uint8_t)(pv[j >> 2] >> (8 * (j & 3)));
+        }
+    }
+    st_n32(Nrow + c, n, vec, ncols - c);
+  }
+  if (ncols > 0 && (row % p.q_rows) == 0) {     // the first lane of each block stores its absmax
+    p.Mam[tile] = mx_m;
+    p.Vam[tile] = mx_v;
+  }
+  return bad;
+}
+
 // ---- the kernel -------------------------------------------------------------------------------
 
 template <int EPI, typename TW, int CTAS>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(epi_threads(EPI), 1)
 gemm_tc_kernel(const __grid_constant__ TcGroup g) {
   using G = Geo<CTAS>;
+  constexpr int kEpiWarps = epi_warps(EPI);
   constexpr int kStages = G::kStages;
   constexpr int kStageBytes = G::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
@@ -392,7 +634,7 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(accf_bar(a), 1);
-      mbar_init(acce_bar(a), 4 * CTAS);             // one arrival per epilogue warp of the group, from every CTA
+      mbar_init(acce_bar(a), kEpiWarps * CTAS);     // one arrival per epilogue warp of the group, from every CTA
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -407,6 +649,9 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
       tmem_relinquish();
     }
   }
+  // the 8-bit code tables follow the barriers (256 bytes after the ring)
+  Q8Tables* q8t = reinterpret_cast<Q8Tables*>(ring_ptr + kStages * kStageBytes + 256);
+  if constexpr (EPI == EPI_ADAM_Q8) q8_tables_fill(*q8t, g.q8, (int)threadIdx.x, epi_threads(EPI));
   tc_fence_before();
   __syncthreads();
   if (CTAS == 2) cluster_sync_all();                // the peer's barriers exist before anyone signals them
@@ -523,7 +768,18 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
       const TcParams& p = g.p[pi];
       const int row = w.m0 + (int)rank * kBM + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kBN);
-      if (EPI != EPI_PARTIAL && w.n0 + kBN <= p.N) {
+      if constexpr (epi_is_adam(EPI)) {
+        // warps 2..5 take the first 128 columns of the tile, warps 6..9 the other 128
+        const int half = (warp - 2) >> 2;
+        const int col0 = w.n0 + half * 128;
+        bool bad;
+        if constexpr (EPI == EPI_ADAM_F32)
+          bad = epi_adam_f32(p, row, col0, t_row + (uint32_t)(half * 128), accf_bar(acc), acc_phase, abort_flag, ok);
+        else
+          bad = epi_adam_q8(p, row, col0, t_row + (uint32_t)(half * 128), accf_bar(acc), acc_phase, abort_flag, *q8t, ok);
+        if (!ok) break;
+        if (bad) atomicOr(p.status, GALORE_DEV_NONFINITE);
+      } else if (EPI != EPI_PARTIAL && w.n0 + kBN <= p.N) {
         // Interior tile of the weight update.  The thread's stretch of its W row is fetched into
         // registers BEFORE waiting for the accumulator: the loads do not depend on the MMAs, so the
         // whole W tile streams in from HBM while the tensor cores are still working on it.
@@ -653,7 +909,8 @@ int sm_count() {
 template <int EPI, typename TW, int CTAS>
 galore_status_t launch_tc_variant(const TcGroup& g, cudaStream_t st) {
   auto kern = gemm_tc_kernel<EPI, TW, CTAS>;
-  constexpr int smem = Geo<CTAS>::kSmemBytes;
+  constexpr int smem = Geo<CTAS>::kSmemBytes + epi_smem(EPI);
+  static_assert(smem <= 227 * 1024, "shared memory of one CTA");
   static bool configured = false;
   if (!configured) {
     GALORE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -664,7 +921,7 @@ galore_status_t launch_tc_variant(const TcGroup& g, cudaStream_t st) {
   const int teams = std::min(units, sm_count() / CTAS);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(teams * CTAS));
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(epi_threads(EPI));
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -812,6 +1069,30 @@ static galore_status_t project_problem(const TensorPlan* plan, const galore_conf
   return make_map(ma, G, c.m, c.n, ldg, kBM);
 }
 
+// the Adam part of a projection problem
+static galore_status_t set_adam(TcParams* p, const TcAdamArgs& a) {
+  if (a.state_fmt == GALORE_STATE_Q8_BLOCK &&
+      (a.q_block < 256 || a.q_block > 4096 || (a.q_block & (a.q_block - 1)) != 0)) return GALORE_ERR_INVALID_ARG;
+  p->Ms = a.M; p->Vs = a.V; p->Mc = a.Mc; p->Vc = a.Vc; p->Mam = a.Mam; p->Vam = a.Vam;
+  p->ld_s = a.ld_s;
+  p->q_rows = a.q_block / kStateTileCols;
+  p->q_tiles_c = (int)ceil_div(p->N, kStateTileCols);
+  p->Nout = (__nv_bfloat16*)a.Nout;
+  p->ld_n = a.ld_n;
+  p->ap = a.ap;
+  // 32-byte accesses: per thread 128 bytes of codes or 128-byte runs of fp32 moments and 64-byte runs of N,
+  // all starting at multiples of 128 columns
+  const uintptr_t bases = (uintptr_t)a.Nout | (uintptr_t)a.M | (uintptr_t)a.V | (uintptr_t)a.Mc | (uintptr_t)a.Vc;
+  const int64_t s_bytes = a.ld_s * (a.state_fmt == GALORE_STATE_F32 ? 4 : 1);
+  p->adam_vec = ((bases & 31) == 0 && (s_bytes % 32) == 0 && (a.ld_n % 16) == 0) ? 1 : 0;
+  return GALORE_OK;
+}
+
+static galore_status_t launch_project_adam(const TcGroup& g, int32_t state_fmt, cudaStream_t st) {
+  if (state_fmt == GALORE_STATE_F32) return launch_tc<EPI_ADAM_F32, float>(g, st);
+  return launch_tc<EPI_ADAM_Q8, float>(g, st);
+}
+
 // the weight update of a group: with the decay multiply only if some problem of the group decays
 static galore_status_t launch_apply(const TcGroup& g, int32_t w_dtype, cudaStream_t st) {
   bool decay = false;
@@ -860,6 +1141,19 @@ galore_status_t tensor_project(TensorPlan* plan, const galore_config_t& c, bool 
   return launch_tc<EPI_PARTIAL, float>(*g, st);
 }
 
+galore_status_t tensor_project_adam(TensorPlan* plan, const galore_config_t& c, bool left, const void* G, int64_t ldg,
+                                    const TcAdamArgs& adam, int32_t* status, cudaStream_t st) {
+  TcParams p;
+  CUtensorMap ma, mb;
+  GALORE_TRY(project_problem(plan, c, left, G, ldg, nullptr, 0, 1, status, &p, &ma, &mb));
+  GALORE_TRY(set_adam(&p, adam));
+  std::unique_ptr<TcGroup> g(new TcGroup);
+  g->count = 0;
+  if (adam.state_fmt == GALORE_STATE_Q8_BLOCK) GALORE_TRY(q8_table_ptrs(&g->q8));
+  group_add(*g, ma, mb, p);
+  return launch_project_adam(*g, adam.state_fmt, st);
+}
+
 galore_status_t tensor_back_project(TensorPlan* plan, const galore_config_t& c, bool left, void* W, int64_t ldw,
                                     float scale, float keep, int32_t* status, cudaStream_t st) {
   TcParams p;
@@ -896,6 +1190,23 @@ galore_status_t tensor_group_add_project(TensorGroup* t, const TensorPlan* plan,
   GALORE_TRY(project_problem(plan, c, left, G, ldg, part, ld_part, splits, status, &p, &ma, &mb));
   group_add(t->g, ma, mb, p);
   return GALORE_OK;
+}
+
+galore_status_t tensor_group_add_project_adam(TensorGroup* t, const TensorPlan* plan, const galore_config_t& c, bool left,
+                                              const void* G, int64_t ldg, const TcAdamArgs& adam, int32_t* status) {
+  if (t->g.count >= kMaxGroup) return GALORE_ERR_BUFFER_TOO_SMALL;
+  TcParams p;
+  CUtensorMap ma, mb;
+  GALORE_TRY(project_problem(plan, c, left, G, ldg, nullptr, 0, 1, status, &p, &ma, &mb));
+  GALORE_TRY(set_adam(&p, adam));
+  group_add(t->g, ma, mb, p);
+  return GALORE_OK;
+}
+
+galore_status_t tensor_group_launch_project_adam(TensorGroup* t, int32_t state_fmt, cudaStream_t st) {
+  if (t->g.count == 0) return GALORE_OK;
+  if (state_fmt == GALORE_STATE_Q8_BLOCK) GALORE_TRY(q8_table_ptrs(&t->g.q8));
+  return launch_project_adam(t->g, state_fmt, st);
 }
 
 galore_status_t tensor_group_add_back(TensorGroup* t, const TensorPlan* plan, const galore_config_t& c, bool left,

@@ -4,8 +4,23 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "q8_code.cuh"
 
 namespace galore {
+
+// What the projection needs to run Adam on its output (Algorithm 1's update block and Eq. 15 in the
+// epilogue): the layer's moments and where the normalised update goes.
+struct TcAdamArgs {
+  int32_t state_fmt;          // galore_state_fmt_t
+  float *M, *V;               // fp32 moments (rows of ld_s floats), or
+  uint8_t *Mc, *Vc;           // 8-bit codes (rows of ld_s bytes) with
+  float *Mam, *Vam;           // one absmax per tile of q_block / 128 rows x 128 columns
+  int64_t ld_s;
+  int q_block;
+  void* Nout;                 // bf16, leading dimension ld_n
+  int64_t ld_n;
+  AdamParams ap;
+};
 
 // Per-layer launch state of the tensor-core path: tensor maps of the operands the library owns
 // (projector, normalised update).  The map of G is encoded per call; W is accessed without TMA.
@@ -33,6 +48,9 @@ bool tensor_operands_aligned(const galore_config_t& cfg, const void* W, int64_t 
 // R partials <- P^T G (left) / G Q (right)
 galore_status_t tensor_project(TensorPlan* plan, const galore_config_t& cfg, bool left, const void* G, int64_t ldg,
                                int32_t* status, cudaStream_t st);
+// the same projection with Adam in its epilogue (one K slice): updates the moments, writes N, no R in memory
+galore_status_t tensor_project_adam(TensorPlan* plan, const galore_config_t& cfg, bool left, const void* G, int64_t ldg,
+                                    const TcAdamArgs& adam, int32_t* status, cudaStream_t st);
 // W <- W - scale * P N (left) / N Q^T (right), N read from plan->Nbuf
 galore_status_t tensor_back_project(TensorPlan* plan, const galore_config_t& cfg, bool left, void* W, int64_t ldw,
                                     float scale, float keep, int32_t* status, cudaStream_t st);
@@ -49,6 +67,11 @@ int tensor_group_capacity();
 galore_status_t tensor_group_add_project(TensorGroup* t, const TensorPlan* plan, const galore_config_t& cfg, bool left,
                                          const void* G, int64_t ldg, float* part, int64_t ld_part, int splits,
                                          int32_t* status);
+// the layer's projection with Adam in its epilogue; launch with tensor_group_launch_project_adam
+// (all layers of the group have the same state format)
+galore_status_t tensor_group_add_project_adam(TensorGroup* t, const TensorPlan* plan, const galore_config_t& cfg, bool left,
+                                              const void* G, int64_t ldg, const TcAdamArgs& adam, int32_t* status);
+galore_status_t tensor_group_launch_project_adam(TensorGroup* t, int32_t state_fmt, cudaStream_t st);
 // the layer's back-projection reading its normalised update from Nbuf (bf16, leading dimension ld_n)
 galore_status_t tensor_group_add_back(TensorGroup* t, const TensorPlan* plan, const galore_config_t& cfg, bool left,
                                       const void* Nbuf, int64_t ld_n, void* W, int64_t ldw, float scale, float keep,

@@ -101,7 +101,13 @@ extern "C" galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank
   ap.eps = (float)eps;
   ap.inv_bc1 = (float)(1.0 / (1.0 - pow(beta1, t)));
   ap.inv_bc2 = (float)(1.0 / (1.0 - pow(beta2, t)));
-  GALORE_TRY(launch_adam_f32(Rpart, splits, nel, nel, M, V, Nbuf, GALORE_F32, ap, status, st));
+  AdamItem item = {};
+  item.Rpart = Rpart; item.splits = splits; item.split_stride = nel;
+  item.rows = (int)srows; item.cols = (int)scols;
+  item.r_ld = item.n_ld = item.s_ld = scols;       // everything packed
+  item.M = M; item.V = V; item.Nout = Nbuf;
+  item.p = ap; item.status = status;
+  GALORE_TRY(launch_adam(item, GALORE_STATE_F32, 2048, GALORE_F32, st));
 
   EpiApplyW<float> apply{W, ldw, lr * alpha};
   if (left)

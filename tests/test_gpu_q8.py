@@ -70,6 +70,20 @@ def test_quotients_next_to_thresholds_any_absmax(signed):
     assert np.array_equal(codes_g.cpu().numpy(), codes_o)
 
 
+@pytest.mark.parametrize("signed", [True, False])
+@pytest.mark.parametrize("rows,cols,tile", [(37, 300, (16, 128)), (64, 256, (16, 128)), (5, 128, (2, 128)),
+                                            (33, 129, (32, 128)), (40, 90, (8, 32))])
+def test_tiled_blocks_bit_exact(signed, rows, cols, tile):
+    """Quantisation blocks as tiles of a matrix (the layout of a layer's 8-bit moments), ragged edges included."""
+    x = _inputs(rows * cols, signed, seed=rows + cols).reshape(rows, cols)
+    codes_o, am_o = go.quantize_tiles(x, signed, *tile)
+    codes_g, am_g = gb.galore_q8_quantize(torch.from_numpy(x).cuda(), signed, tile=tile)
+    assert np.array_equal(codes_g.cpu().numpy(), codes_o)
+    assert np.array_equal(am_g.cpu().numpy(), am_o)
+    back_g = gb.galore_q8_dequantize(codes_g, am_g, signed, tile=tile)
+    assert np.array_equal(back_g.cpu().numpy(), go.dequantize_tiles(codes_o, am_o, signed, *tile))
+
+
 def test_empty_input():
     codes, am = gb.galore_q8_quantize(torch.zeros(0, device="cuda"), True, 2048)
     assert codes.numel() == 0 and am.numel() == 0

@@ -73,8 +73,8 @@ def test_tensor_path_q8_states(m, n, r, qb):
 
 @pytest.mark.parametrize("m,n,r,qb", [(256, 1100, 64, 2048), (1100, 256, 64, 1024), (200, 2741, 72, 4096)])
 def test_tensor_path_q8_states_with_padded_rows(m, n, r, qb):
-    """Row lengths that are no multiple of 8: R and N have padded rows while the state stays packed, so
-    the full blocks go to the padded-row kernel and the tail block to the general one."""
+    """Row lengths that are no multiple of 8 or of the tile width: R, N and the codes have padded rows and the
+    last tile column (and, on the right side, the last tile row) is cut off at the border of the state."""
     ld = (n + 7) // 8 * 8
     layer, orc, errs = _run(m, n, r, "bf16", "q8", steps=4, q_block=qb, ldw=ld, ldg=ld)
     assert layer.uses_tensor_path and layer.device_status() == 0
