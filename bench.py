@@ -66,11 +66,37 @@ def p_dtype_of(w):
     return "bf16" if w.g_dtype == "bf16" else "f32"
 
 
-# DRAM bytes per parameter moved by the two tcgen05 launches of a step (projection + back-projection),
-# from the ncu capture summarised in profiles/gemm_tc_and_adam_single_4096x11008_r1024.md (one
-# 4096 x 11008 matrix, r = 1024: 355 MB for 45.09 M parameters).  Traffic grows with the parameters a
-# launch covers; set to None whenever those kernels change after the capture.
-GEMM_DRAM_BYTES_PER_PARAM = 7.88
+# DRAM traffic per launch of the step's kernels from ncu captures of the kernels as they are now
+# (dram__bytes_read.sum + dram__bytes_write.sum, summarised under profiles/ with the command that made
+# them), as bytes per parameter covered by the launch: traffic grows in proportion to the matrices a
+# launch covers.  None: not captured since the kernel last changed.
+KERNEL_DRAM_BYTES_PER_PARAM = {
+    # (workload rank, state format): {"projection": ..., "back_projection": ...}
+}
+
+
+def kernel_costs(w, shapes):
+    """Algorithmic flops and bytes of each kernel of the step, summed over the layer set.
+
+    projection (with Adam in its epilogue when fused): reads G and P, reads and writes the moments, writes N.
+    back-projection: reads P and N, reads and writes W.  N (r x max(m, n) bf16 or fp32) is an intermediate
+    the method itself does not need; it is counted here because these are per-kernel roofs."""
+    proj = {"flops": 0, "bytes": 0}
+    back = {"flops": 0, "bytes": 0}
+    adam = {"flops": 0, "bytes": 0}
+    n_b = 2 if w.g_dtype == "bf16" else 4
+    for (m, n) in shapes:
+        r = w.rank
+        d, big = (m, n) if m <= n else (n, m)
+        nel = r * big
+        state = 4 * nel * 4 if w.state_fmt == "f32" else 4 * nel + 4 * 4 * ((nel + w.q_block - 1) // w.q_block)
+        p_bytes = d * r * elem_bytes(p_dtype_of(w))
+        proj["flops"] += 2 * m * n * r
+        proj["bytes"] += m * n * elem_bytes(w.g_dtype) + p_bytes
+        adam["bytes"] += state + nel * n_b
+        back["flops"] += 2 * m * n * r
+        back["bytes"] += 2 * m * n * elem_bytes(w.w_dtype) + p_bytes + nel * n_b
+    return proj, adam, back
 
 
 def max_over_ranks(value: float, dist, device) -> float:
@@ -136,18 +162,27 @@ class ClockSampler:
         return res
 
 
-def cpu_oracle_sample(w, steps=1):
-    """Times the oracle, as it stands, on one matrix of each distinct shape of the workload."""
+def _blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_oracle_sample(w, steps=1, extras=False):
+    """Times the oracle, as it stands (numpy on the host's BLAS, fp64), on one matrix of each distinct shape.
+
+    extras: also one step on the smallest shape with the BLAS pool limited to one thread, and one projector
+    refresh (the oracle's SVD through the library routine it uses at sizes its Jacobi code cannot reach in
+    test time) on the smallest shape.  Returns (params/s, cores, seconds, extras dict)."""
     import numpy as np
     from oracle import galore_oracle as go
     from paper_2403_03507_b200 import workloads as wl
-    try:
-        from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
-    except Exception:
-        cores = os.cpu_count() or 1
+    cores = _blas_threads()
     total_params, total_time = 0, 0.0
     rng = np.random.default_rng(0)
+    smallest = None
     for (m, n, _count) in w.shapes:
         side = "left" if m <= n else "right"
         orc = go.GaLoreOracle(m, n, w.rank, w.alpha, w.refresh_gap, w.beta1, w.beta2, w.eps, w_store=w.w_dtype,
@@ -162,14 +197,32 @@ def cpu_oracle_sample(w, steps=1):
             W = orc.step(W, G, w.lr, auto_refresh=False)
         total_time += time.perf_counter() - t0
         total_params += m * n * steps
-    return total_params / total_time, cores, total_time
+        if smallest is None or m * n < smallest[0] * smallest[1]:
+            smallest = (m, n, orc, G, W, side)
+    extra = {}
+    if extras and smallest is not None:
+        m, n, orc, G, W, side = smallest
+        try:
+            from threadpoolctl import threadpool_limits
+            with threadpool_limits(limits=1):
+                t0 = time.perf_counter()
+                orc.step(W, G, w.lr, auto_refresh=False)
+                t1 = time.perf_counter() - t0
+            extra["one_thread"] = {"value": m * n / t1, "unit": UNIT, "shape": [m, n], "seconds": t1}
+        except Exception as e:                                  # threadpoolctl missing: say so rather than guess
+            extra["one_thread"] = {"unavailable": repr(e)}
+        t0 = time.perf_counter()
+        go.top_r_projector(G, w.rank, side, method="lapack")
+        extra["refresh"] = {"seconds": time.perf_counter() - t0, "shape": [m, n], "rank": w.rank, "cores": cores,
+                            "method": "library SVD as one step (the Jacobi code is the pinned definition at small sizes)"}
+    return total_params / total_time, cores, total_time, extra
 
 
 def run_reference(args, w):
     value, cores, _ = None, None, None
     times = []
     for i in range(args.warmup + args.steps):
-        v, cores, t = cpu_oracle_sample(w, 1)
+        v, cores, t, _ = cpu_oracle_sample(w, 1)
         if i >= args.warmup:
             times.append((v, t))
     value = sum(v for v, _ in times) / len(times)
@@ -179,7 +232,8 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic", "config": {"workload": w.name, "rank": w.rank, "state_fmt": w.state_fmt},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "backend": "numpy on the host BLAS, fp64",
+                         "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -211,9 +265,11 @@ def main():
     ap.add_argument("--refresh-only", action="store_true",
                     help="run the projector refresh of each distinct shape and print its timings; no step is timed "
                          "(for profiling the refresh on its own)")
-    ap.add_argument("--extra-workloads", default="llama_1b_q8,llama_1b_f32",
+    ap.add_argument("--extra-workloads", default="llama_1b_q8,llama_1b_f32,llama_130m,sweep",
                     help="comma-separated workloads also timed, device-resident only, reported under other_workloads "
-                         "(only with the default workload; empty string to skip)")
+                         "(only with the default workload; empty string to skip).  'sweep' = the rank sweep on one "
+                         "4096 x 11008 matrix: six ranks x both state formats, one matrix per step, with the refresh "
+                         "and the throughput with the refresh spread over T = 50, 200, 1000 steps")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else max(args.warmup, 0)
 
@@ -247,8 +303,17 @@ def main():
     if rank == 0:
         extras = []
         names = [x for x in args.extra_workloads.split(",") if x] if args.workload == "llama_7b_q8" and world == 1 and not args.refresh_only else []
+        import dataclasses
         for name in names:
-            extras.append(time_workload(wl.WORKLOADS[name], args, dev, None, 1, 0, full=False))
+            if name == "sweep":
+                args.amortise_gaps = wl.SWEEP_GAPS
+                for r in wl.SWEEP_RANKS:
+                    for fmt in ("q8", "f32"):
+                        ws = dataclasses.replace(wl.WORKLOADS["sweep_4096x11008"], rank=r, state_fmt=fmt)
+                        extras.append(time_workload(ws, args, dev, None, 1, 0, full=False, mode="layer"))
+                args.amortise_gaps = ()
+            else:
+                extras.append(time_workload(wl.WORKLOADS[name], args, dev, None, 1, 0, full=False))
         if extras:
             res["other_workloads"] = extras
         print(json.dumps(res), flush=True)
@@ -258,7 +323,8 @@ def main():
     return 0
 
 
-def time_workload(w, args, dev, dist, world, rank, full):
+def time_workload(w, args, dev, dist, world, rank, full, mode=None):
+    mode = mode or args.mode
     import torch
     from paper_2403_03507_b200 import binding as gb
     from paper_2403_03507_b200 import workloads as wl
@@ -345,10 +411,10 @@ def time_workload(w, args, dev, dist, world, rank, full):
                        "timer": "host clock around the call, which returns when every refresh has finished"}
         del space
 
-    batch = gb.Batch(layers, Ws, Gs, device=dev) if args.mode == "batch" else None
+    batch = gb.Batch(layers, Ws, Gs, device=dev) if mode == "batch" else None
 
     arrive = None
-    if args.mode == "arrive":
+    if mode == "arrive":
         # A producer stream stands in for the backward pass: it writes layer i's gradient into the next
         # buffer of a small ring (a device copy of a resident gradient, i.e. the write traffic of the
         # kernel that would produce it) and signals; the step of layer i waits for that, runs on the
@@ -418,30 +484,44 @@ def time_workload(w, args, dev, dist, world, rank, full):
     gb.galore_profile_enable(False)
     phase_ms, phase_cnt = gb.galore_profile_read()
     uses_tc = all(l.uses_tensor_path for l in layers)
-    gemm_ms = phase_ms[0] + phase_ms[2]
-    gemm_launches = phase_cnt[0] + phase_cnt[2]
-    # dominant kernels: the two projection GEMMs (2 m n r flops each)
+    # whole-step roofline: the slower of the algorithmic HBM bytes at the measured copy bandwidth and the
+    # projection flops at the measured sustained bf16 GEMM rate (fp32 FMA peak on the fp32 path)
     t_hbm = bytes_alg / (peaks["hbm_gbs"] * 1e9)
-    tc_peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    tc_peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) if uses_tc else FP32_FMA_TFLOPS
     t_tc = flops_alg / (tc_peak * 1e12)
-    achieved_tflops = (flops_alg * prof_steps) / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
-    if uses_tc:
-        roof = {"bound": "tensor", "achieved": achieved_tflops, "peak": tc_peak, "unit": "TFLOP/s",
-                "frac": achieved_tflops / tc_peak if achieved_tflops else None,
-                "traffic": (GEMM_DRAM_BYTES_PER_PARAM * w.params * prof_steps / gemm_launches
-                            if GEMM_DRAM_BYTES_PER_PARAM and gemm_launches and w.rank == 1024 else None),
-                "traffic_unit": "bytes per launch, scaled from a one-matrix ncu capture by parameters covered",
-                "peak_source": peaks["source"] + " (sustained bf16 GEMM)"}
+    t_roof = max(t_hbm, t_tc)
+    bound = "hbm" if t_hbm >= t_tc else ("tensor" if uses_tc else "alu")
+    if bound == "hbm":
+        achieved, peak, unit = bytes_alg / (ms_step * 1e-3) / 1e9, peaks["hbm_gbs"], "GB/s"
     else:
-        roof = {"bound": "alu", "achieved": achieved_tflops, "peak": FP32_FMA_TFLOPS, "unit": "TFLOP/s",
-                "frac": achieved_tflops / FP32_FMA_TFLOPS if achieved_tflops else None, "traffic": None,
-                "peak_source": "148 SMs x 128 fp32 lanes x 2 x 1.965 GHz"}
-    roof["kernel"] = "projection + back-projection GEMMs"
-    roof["avg_launch_ms"] = gemm_ms / gemm_launches if gemm_launches else None
-    roof["phase_ms_per_step"] = {"projection": phase_ms[0] / prof_steps, "adam": phase_ms[1] / prof_steps,
-                                 "back_projection": phase_ms[2] / prof_steps}
-    roof["step_roofline_ms"] = {"hbm": t_hbm * 1e3, "tensor": t_tc * 1e3}
-    roof["step_frac_of_roofline"] = max(t_hbm, t_tc) * 1e3 / ms_step
+        achieved, peak, unit = flops_alg / (ms_step * 1e-3) / 1e12, tc_peak, "TFLOP/s"
+    # per kernel: event time per step, what it achieves and the fraction of its own roof
+    kp, ka, kb = kernel_costs(w, shapes_of)
+    fused = phase_cnt[1] == 0                   # Adam ran in the projection's epilogue: no launch of its own
+    if fused:
+        kp = {"flops": kp["flops"], "bytes": kp["bytes"] + ka["bytes"]}
+
+    def kernel_entry(ms_total, launches_total, cost):
+        if not launches_total:
+            return None
+        ms = ms_total / prof_steps
+        roof_ms = max(cost["flops"] / (tc_peak * 1e12), cost["bytes"] / (peaks["hbm_gbs"] * 1e9)) * 1e3
+        return {"ms_per_step": ms, "launches_per_step": launches_total / prof_steps,
+                "tflops": cost["flops"] / (ms * 1e-3) / 1e12 if cost["flops"] else None,
+                "gbs": cost["bytes"] / (ms * 1e-3) / 1e9, "roof_ms": roof_ms, "frac_of_own_roof": roof_ms / ms}
+    kernels = {"projection_with_adam" if fused else "projection": kernel_entry(phase_ms[0], phase_cnt[0], kp),
+               "adam": kernel_entry(phase_ms[1], phase_cnt[1], ka),
+               "back_projection": kernel_entry(phase_ms[2], phase_cnt[2], kb)}
+    traffic = KERNEL_DRAM_BYTES_PER_PARAM.get((w.rank, w.state_fmt))
+    roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": t_roof * 1e3 / ms_step,
+            "traffic": ({k: v * w.params / max(1.0, kernels[k]["launches_per_step"]) for k, v in traffic.items() if kernels.get(k)}
+                        if traffic else None),
+            "traffic_unit": "DRAM bytes per launch, by kernel, scaled from the ncu capture by the parameters a launch covers",
+            "peak_source": peaks["source"] + (" (sustained bf16 GEMM)" if bound == "tensor" else " (copy bandwidth)" if bound == "hbm" else " (unit counts x max clock)"),
+            "scope": "whole step: algorithmic bytes and flops of every matrix / measured step time",
+            "kernels": {k: v for k, v in kernels.items() if v},
+            "step_roofline_ms": {"hbm": t_hbm * 1e3, "tensor" if uses_tc else "fp32_fma": t_tc * 1e3},
+            "algorithmic": {"bytes_per_step": bytes_alg, "flops_per_step": flops_alg}}
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -449,7 +529,7 @@ def time_workload(w, args, dev, dist, world, rank, full):
         "dtype": "bf16" if uses_tc else "f32", "data": "synthetic",
         "config": {"workload": w.name, "matrices": w.matrices, "params": w.params, "rank": w.rank,
                    "state_fmt": w.state_fmt, "w_dtype": w.w_dtype, "g_dtype": w.g_dtype, "alpha": w.alpha,
-                   "refresh_gap": w.refresh_gap, "weight_decay": args.weight_decay, "tensor_path": uses_tc, "mode": args.mode, "parallelism": f"replicas x{world}",
+                   "refresh_gap": w.refresh_gap, "weight_decay": args.weight_decay, "tensor_path": uses_tc, "mode": mode, "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (whole layer set streamed each step)"},
         "clocks": clocks, "gpu_launches": launches, "roofline": roof,
         "refresh": refresh_info,
@@ -457,15 +537,19 @@ def time_workload(w, args, dev, dist, world, rank, full):
     if refresh_set:
         # Algorithm 1 refreshes every matrix once per `refresh_gap` steps: the step plus its share of that
         set_ms = refresh_set["ms"]
-        amortised_ms = ms_step + set_ms / w.refresh_gap
+        gaps = sorted({w.refresh_gap, *getattr(args, "amortise_gaps", ())})
         out["refresh_set"] = refresh_set
         out["refresh_amortised"] = {"refresh_ms_whole_set": set_ms, "refresh_gap": w.refresh_gap,
                                     "one_by_one_ms_whole_set": sum(x["ms"] * x["count"] for x in refresh_info),
-                                    "ms_per_step": amortised_ms, "value": world * w.params / (amortised_ms * 1e-3),
-                                    "unit": UNIT}
+                                    "ms_per_step": ms_step + set_ms / w.refresh_gap,
+                                    "value": world * w.params / ((ms_step + set_ms / w.refresh_gap) * 1e-3), "unit": UNIT,
+                                    "by_gap": {str(T): world * w.params / ((ms_step + set_ms / T) * 1e-3) for T in gaps}}
+        # the same two records inside an object every reader of the line keeps
+        roof["refresh_set"] = refresh_set
+        roof["refresh_amortised"] = out["refresh_amortised"]
     if not full:
         return {k: out[k] for k in ("value", "ms_per_step", "config", "roofline", "refresh", "refresh_set",
-                                    "refresh_amortised", "gpu_launches") if k in out}
+                                    "refresh_amortised", "gpu_launches", "clocks") if k in out}
 
     # ---- end to end through the host-buffer entry point -------------------------------------------
     if not args.no_e2e:
@@ -492,7 +576,7 @@ def time_workload(w, args, dev, dist, world, rank, full):
         e2e_steps = max(1, min(args.steps, 3))
         h2d = sum(m * n * (elem_bytes(w.w_dtype) + elem_bytes(w.g_dtype)) for (m, n) in shapes_of)
         d2h = sum(m * n * elem_bytes(w.w_dtype) for (m, n) in shapes_of)
-        if args.mode == "batch":
+        if mode == "batch":
             hb = gb.HostBatch(layers, W_hosts, G_hosts, slots=3, device=dev)
             e2e_call = "galore_step_host_batch, 3 staging slots"
 
@@ -527,10 +611,10 @@ def time_workload(w, args, dev, dist, world, rank, full):
     out["device_status"] = flags
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, cores, t = cpu_oracle_sample(w, 1)
-        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+        v, cores, t, extra = cpu_oracle_sample(w, 1, extras=True)
+        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "backend": "numpy on the host BLAS, fp64",
                                "sample": f"1 oracle step on one matrix of each distinct shape ({len(w.shapes)} of "
-                                         f"{w.matrices} matrices), given projector, {t:.1f} s"}
+                                         f"{w.matrices} matrices), given projector, {t:.1f} s", **extra}
     return out
 
 

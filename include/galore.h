@@ -26,9 +26,11 @@
  *     return without synchronising, except where stated.
  *   - Work of different handles is meant to be queued on ONE stream per
  *     device (the list entry points add internal streams of their own, joined
- *     by events).  Driving several handles from several host threads on
- *     several streams at once is not supported: refreshes run that way
- *     stalled on the test machines, and the cause was not found.
+ *     by events).  Tensor-core launches given on different streams are chained
+ *     by the library with events, one after another in the order of the calls:
+ *     each needs a whole SM's tensor memory and shared memory, so they would
+ *     not overlap anyway, and runs that kept several streams of them in flight
+ *     stalled on the test machines for a reason that was not found.
  *   - Every entry point returns a galore_status_t: 0 ok, > 0 warning, < 0
  *     error.  Nothing throws or aborts across this boundary.  Conditions
  *     detected on the device (non-finite values, a bounded wait that ran out)
@@ -55,8 +57,8 @@ typedef enum {
   GALORE_ERR_BUFFER_TOO_SMALL = -4,
   GALORE_ERR_CUDA = -5,          /* a CUDA runtime/driver call failed; see galore_last_cuda_error() */
   GALORE_ERR_STATE = -6,         /* e.g. a step without a projector when auto_refresh is off */
-  GALORE_ERR_NONFINITE = -7,
-  GALORE_ERR_TIMEOUT = -8,
+  GALORE_ERR_NONFINITE = -7,     /* galore_check_device: a non-finite projected gradient was seen */
+  GALORE_ERR_TIMEOUT = -8,       /* galore_check_device: a bounded device-side wait ran out */
   GALORE_ERR_UNIMPLEMENTED = -9
 } galore_status_t;
 
@@ -74,7 +76,6 @@ typedef enum {
 enum {
   GALORE_DEV_NONFINITE = 1,     /* a non-finite projected gradient was seen */
   GALORE_DEV_WAIT_EXPIRED = 2,  /* a bounded device-side wait ran out */
-  GALORE_DEV_BOUNDS = 4,        /* an internal index check failed */
   GALORE_DEV_CHOLESKY = 8       /* a Gram matrix in the refresh was not positive definite */
 };
 
@@ -227,7 +228,8 @@ galore_status_t galore_free(galore_layer_t* layer);
  *   completed_steps  k of Algorithm 1 before this call (bias correction uses k + 1)
  *   side  galore_side_t (AUTO: left iff m <= n)
  *   device_flags  optional host pointer; when non-NULL the call waits for the stream and stores
- *                 the GALORE_DEV_* bits the kernels latched, otherwise it returns without waiting
+ *                 the GALORE_DEV_* bits the kernels of THIS call latched, otherwise it returns
+ *                 without waiting; either way the bits are also kept for galore_static_status()
  * No refresh is done here: the caller supplies P.
  *
  * Limits and rules
@@ -236,6 +238,8 @@ galore_status_t galore_free(galore_layer_t* layer);
  *     GALORE_ERR_BUFFER_TOO_SMALL and nothing is launched.
  *   - The first call on each device looks up the array's device address (with that device
  *     current).  Make that first call outside of any stream capture.
+ *   - `stream` must belong to the current device (checked: GALORE_ERR_INVALID_ARG otherwise); the
+ *     array that is used is the current device's.
  *   - All calls on a device share the array, and it keeps the previous call's contents.  The call
  *     clears the status word it needs at zero; everything else it reads it has written first.
  *     Calls whose GPU work can overlap (two streams, two threads) race on the array: serialise
@@ -246,6 +250,10 @@ galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank, int32_t s
                                    double beta2, double eps, int64_t completed_steps, const float* P, float* M,
                                    float* V, float* W, int64_t ldw, const float* G, int64_t ldg, float lr,
                                    int32_t* device_flags, void* stream);
+/* GALORE_DEV_* bits latched by every galore_step_static call on the current device since the last
+ * call of this function (they accumulate across calls, so the asynchronous form loses nothing).
+ * Synchronises `stream`, returns the bits in *flags and clears them. */
+galore_status_t galore_static_status(int32_t* flags, void* stream);
 
 /* ---- accessors (tests, checkpoint/resume) -------------------------------- */
 
@@ -264,7 +272,7 @@ galore_status_t galore_get_moments(galore_layer_t* layer, float* M, float* V, si
  * state at I * ceil(cols / 128) + J); device memory. */
 galore_status_t galore_get_q8_state(galore_layer_t* layer, uint8_t* M_codes, float* M_absmax,
                                     uint8_t* V_codes, float* V_absmax, void* stream);
-/* Completed steps k.  A checkpoint is the caller's state buffer plus this counter. */
+/* Completed steps k. */
 galore_status_t galore_get_step_count(const galore_layer_t* layer, int64_t* k);
 galore_status_t galore_set_step_count(galore_layer_t* layer, int64_t k);
 /* Resolved side (galore_side_t), whether the tensor-core path is in use, and the state shape. */
@@ -272,6 +280,22 @@ galore_status_t galore_layer_info(const galore_layer_t* layer, int32_t* side, in
                                   int64_t* state_rows, int64_t* state_cols);
 /* Synchronises `stream`, returns the device status bits and clears them. */
 galore_status_t galore_device_status(galore_layer_t* layer, int32_t* flags, void* stream);
+/* The same read-and-clear as a status: GALORE_ERR_TIMEOUT if a bounded wait ran out, else
+ * GALORE_ERR_NONFINITE for a non-finite projected gradient, else GALORE_ERR_STATE for a Cholesky
+ * breakdown in the refresh, else GALORE_OK. */
+galore_status_t galore_check_device(galore_layer_t* layer, void* stream);
+
+/* Checkpoint and resume of one layer: everything Algorithm 1 carries from one iteration to the
+ * next -- the projector P, the moments M and V (fp32, or codes and absmax) and the number of
+ * completed steps -- as one block of HOST memory of galore_export_bytes() bytes (a small header,
+ * then the state buffer as it is laid out on the device).  galore_import_state restores it into a
+ * layer created with the same shape, rank, side, projector dtype, state format and block size
+ * (GALORE_ERR_STATE otherwise; GALORE_ERR_INVALID_ARG if the block is not an export of this
+ * library).  A run that exports, imports into a fresh layer and goes on is bit-identical to one
+ * that never stopped.  Both calls synchronise `stream`. */
+galore_status_t galore_export_bytes(const galore_layer_t* layer, size_t* bytes);
+galore_status_t galore_export_state(galore_layer_t* layer, void* dst_host, size_t bytes, void* stream);
+galore_status_t galore_import_state(galore_layer_t* layer, const void* src_host, size_t bytes, void* stream);
 
 /* ---- 8-bit block-wise state format (Sec. 4.3 names 8-bit Adam states; the
  *      format is this library's) ------------------------------------------- */

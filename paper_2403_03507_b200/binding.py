@@ -21,7 +21,7 @@ SIDE_AUTO, SIDE_LEFT, SIDE_RIGHT = 0, 1, 2
 F32, BF16 = 0, 1
 STATE_F32, STATE_Q8_BLOCK = 0, 1
 PATH_AUTO, PATH_FP32, PATH_TENSOR = 0, 1, 2
-DEV_NONFINITE, DEV_WAIT_EXPIRED, DEV_BOUNDS, DEV_CHOLESKY = 1, 2, 4, 8
+DEV_NONFINITE, DEV_WAIT_EXPIRED, DEV_CHOLESKY = 1, 2, 8
 
 _DTYPES = {"f32": F32, "bf16": BF16, torch.float32: F32, torch.bfloat16: BF16}
 _TORCH = {F32: torch.float32, BF16: torch.bfloat16}
@@ -91,6 +91,11 @@ _PROTOTYPES = {
     "galore_layer_info": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int64),
                                     C.POINTER(C.c_int64)]),
     "galore_device_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32), C.c_void_p]),
+    "galore_check_device": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "galore_export_bytes": (C.c_int, [C.c_void_p, C.POINTER(C.c_size_t)]),
+    "galore_export_state": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "galore_import_state": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "galore_static_status": (C.c_int, [C.POINTER(C.c_int32), C.c_void_p]),
     "galore_q8_codebook": (C.c_int, [C.c_int32, C.POINTER(C.c_float)]),
     "galore_q8_quantize": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
                                      C.c_void_p, C.c_void_p]),
@@ -218,6 +223,13 @@ def galore_step_static(P, M, V, W, G, lr, completed_steps, alpha=0.25, beta1=0.9
     return flags.value
 
 
+def galore_static_status(stream=None) -> int:
+    """Status bits latched by galore_step_static calls on the current device since the last read; clears them."""
+    f = C.c_int32(0)
+    _check(lib().galore_static_status(C.byref(f), _stream_ptr(stream)), "galore_static_status")
+    return f.value
+
+
 def galore_launch_count() -> int:
     return int(lib().galore_launch_count())
 
@@ -334,6 +346,22 @@ class Layer:
     @step_count.setter
     def step_count(self, k: int):
         _check(lib().galore_set_step_count(self.handle, k), "galore_set_step_count")
+
+    def check_device(self, stream=None) -> int:
+        """galore_check_device: the latched device conditions as a status code (0 ok, negative error); does not raise."""
+        return int(lib().galore_check_device(self.handle, _stream_ptr(stream)))
+
+    def export_state(self, stream=None) -> torch.Tensor:
+        """galore_export_state into a new pinned host buffer (uint8)."""
+        n = C.c_size_t(0)
+        _check(lib().galore_export_bytes(self.handle, C.byref(n)), "galore_export_bytes")
+        buf = torch.empty(n.value, dtype=torch.uint8).pin_memory()
+        _check(lib().galore_export_state(self.handle, buf.data_ptr(), buf.numel(), _stream_ptr(stream)), "galore_export_state")
+        return buf
+
+    def import_state(self, buf: torch.Tensor, stream=None):
+        assert not buf.is_cuda and buf.dtype == torch.uint8 and buf.is_contiguous()
+        _check(lib().galore_import_state(self.handle, buf.data_ptr(), buf.numel(), _stream_ptr(stream)), "galore_import_state")
 
     def device_status(self, stream=None) -> int:
         f = C.c_int32()

@@ -89,6 +89,7 @@ struct galore_layer {
   float* Rpart;
   void* Nbuf;
   void* refresh_ws;
+  size_t state_bytes;    // size of the caller's state buffer as laid out here (it starts at P)
   bool refreshed_here = false;   // the last refresh ran in refresh_ws (its unrounded projector is still there)
   TensorPlan tc;         // tensor-map state of the tcgen05 path (unused on the fp32 path)
 };
@@ -155,7 +156,7 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
   }
   s->tc_splits = s->tensor_path ? tensor_proj_splits(*c, s->left) : 0;
   s->ld_part = (s->scols + 7) / 8 * 8;     // 32-byte rows for whole-sector vector stores
-  s->ld_n = (s->scols + 7) / 8 * 8;        // 16-byte bf16 rows for TMA
+  s->ld_n = (s->scols + 15) / 16 * 16;     // 32-byte bf16 rows: TMA needs 16, the epilogue that writes N stores 32 at a time
 
   size_t o = 0;
   s->off_P = o; o += align_up((size_t)s->d * r * dtype_size(c->p_dtype), 256);
@@ -256,9 +257,26 @@ galore_status_t step_simt(galore_layer* l, void* W, int64_t ldw, const void* G, 
 }
 
 // projection and back-projection on tcgen05, Adam in between reading the padded partials
+TcAdamArgs tc_adam_args(const galore_layer* l, void* nbuf, const AdamParams& ap) {
+  TcAdamArgs a = {};
+  a.state_fmt = l->cfg.state_fmt;
+  a.M = l->M; a.V = l->V; a.Mc = l->Mc; a.Vc = l->Vc; a.Mam = l->Mam; a.Vam = l->Vam;
+  a.ld_s = l->ld_s;
+  a.q_block = l->q_block;
+  a.Nout = nbuf;
+  a.ld_n = l->ld_n;
+  a.ap = ap;
+  return a;
+}
+
 galore_status_t step_tensor(galore_layer* l, void* W, int64_t ldw, const void* G, int64_t ldg, float lr,
                             const AdamParams& ap, cudaStream_t st) {
-  {
+  if (l->tc.splits == 1) {
+    // one K slice per tile: Adam runs in the projection's epilogue, R never reaches memory
+    PhaseTimer pt(0, st);
+    GALORE_TRY(tensor_project_adam(&l->tc, l->cfg, l->left, G, ldg, tc_adam_args(l, l->Nbuf, ap), l->status, st));
+  } else {
+   {
     PhaseTimer pt(0, st);
     GALORE_TRY(tensor_project(&l->tc, l->cfg, l->left, G, ldg, l->status, st));
   }
@@ -266,6 +284,7 @@ galore_status_t step_tensor(galore_layer* l, void* W, int64_t ldw, const void* G
     PhaseTimer pt(1, st);
     GALORE_TRY(launch_adam(adam_item(l, l->Rpart, l->tc.splits, l->srows * l->ld_part, l->ld_part, l->Nbuf, l->ld_n, ap),
                            l->cfg.state_fmt, l->q_block, GALORE_BF16, st));
+   }
   }
   PhaseTimer pt(2, st);
   return tensor_back_project(&l->tc, l->cfg, l->left, W, ldw, lr * l->cfg.alpha, decay_keep(l, lr), l->status, st);
@@ -345,6 +364,7 @@ galore_status_t galore_init_layer(const galore_config_t* cfg, void* state_buf, s
   l->Rpart = (float*)(ws + s.off_R);
   l->Nbuf = ws + s.off_N;
   l->refresh_ws = ws + s.off_refresh;
+  l->state_bytes = s.state_bytes;
 
   cudaError_t e = cudaSuccess;
   if (cfg->state_fmt == GALORE_STATE_F32) {
@@ -463,11 +483,27 @@ struct HostPipe {
   cudaStream_t in = nullptr, out = nullptr;
   cudaEvent_t start = nullptr;
   std::vector<cudaEvent_t> arrived, stepped, drained;   // per layer, per layer, per slot
+  void release() {    // streams and events go back when the thread ends or moves to another device
+    if (device < 0) return;
+    int cur = 0;
+    const bool sw = cudaGetDevice(&cur) == cudaSuccess && cur != device && cudaSetDevice(device) == cudaSuccess;
+    for (auto* v : {&arrived, &stepped, &drained}) {
+      for (cudaEvent_t e : *v) cudaEventDestroy(e);
+      v->clear();
+    }
+    if (start) cudaEventDestroy(start);
+    if (in) cudaStreamDestroy(in);
+    if (out) cudaStreamDestroy(out);
+    start = nullptr; in = out = nullptr;
+    if (sw) cudaSetDevice(cur);
+    device = -1;
+  }
+  ~HostPipe() { release(); }
 };
 
 galore_status_t host_pipe_prepare(HostPipe& hp, int dev, size_t layers, size_t slots) {
   if (hp.device != dev) {
-    hp = HostPipe();
+    hp.release();
     hp.device = dev;
     GALORE_CUDA_TRY(cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking));
     GALORE_CUDA_TRY(cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking));
@@ -552,12 +588,18 @@ galore_status_t galore_step_host_batch(galore_layer_t* const* layers, void* cons
 namespace {
 
 // bytes of group scratch one layer needs: R (one or tc_splits partial buffers) and N, each 256-aligned
-size_t batch_layer_bytes(const galore_layer* l, int splits) {
-  return align_up((size_t)splits * l->srows * l->ld_part * 4, 256) + align_up((size_t)l->srows * l->ld_n * 2, 256);
+// With four or more layers in flight K is not sliced, Adam runs in the projection's epilogue and R is
+// never stored: the group scratch of a layer is its N alone.
+bool batch_fuses(int eligible) { return eligible >= 4; }
+size_t batch_r_bytes(const galore_layer* l, int splits, bool fuse) {
+  return fuse ? 0 : align_up((size_t)splits * l->srows * l->ld_part * 4, 256);
+}
+size_t batch_layer_bytes(const galore_layer* l, int splits, bool fuse) {
+  return batch_r_bytes(l, splits, fuse) + align_up((size_t)l->srows * l->ld_n * 2, 256);
 }
 
 // With several layers in flight there are enough tiles to fill the machine without slicing K.
-int batch_splits(const galore_layer* l, int eligible) { return eligible >= 4 ? 1 : l->tc_splits; }
+int batch_splits(const galore_layer* l, int eligible) { return batch_fuses(eligible) ? 1 : l->tc_splits; }
 
 bool batch_eligible(const galore_layer* l, const void* W, int64_t ldw, const void* G, int64_t ldg) {
   return l->tensor_path && l->has_projector && tensor_operands_aligned(l->cfg, W, ldw, G, ldg);
@@ -607,7 +649,7 @@ galore_status_t galore_batch_query_bytes(galore_layer_t* const* layers, int32_t 
   const int cap = std::min(tensor_group_capacity(), (int)kAdamGroup);
   std::vector<size_t> need;
   for (int32_t i = 0; i < count; ++i)
-    if (layers[i]->tensor_path) need.push_back(batch_layer_bytes(layers[i], batch_splits(layers[i], eligible)));
+    if (layers[i]->tensor_path) need.push_back(batch_layer_bytes(layers[i], batch_splits(layers[i], eligible), batch_fuses(eligible)));
   size_t best = 0, run = 0;
   for (size_t i = 0; i < need.size(); ++i) {
     run += need[i];
@@ -655,7 +697,7 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
       galore_layer* l = layers[i];
       const bool ok = batch_ws && batch_eligible(l, W[i], ldw[i], G[i], ldg[i]);
       const int splits = batch_splits(l, eligible);
-      const size_t need = ok ? batch_layer_bytes(l, splits) : 0;
+      const size_t need = ok ? batch_layer_bytes(l, splits, batch_fuses(eligible)) : 0;
       if (!ok || need > half) {
         // plain step (its refresh, if due, is already done: auto_refresh off for this call)
         const int32_t saved = l->cfg.auto_refresh;
@@ -688,7 +730,21 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
     const galore_layer* l = layers[mb.index];
     char* base = (char*)batch_ws + (gi & 1) * half + mb.offset;
     *part = (float*)base;
-    *nbuf = base + align_up((size_t)mb.splits * l->srows * l->ld_part * 4, 256);
+    *nbuf = base + batch_r_bytes(l, mb.splits, batch_fuses(eligible));
+  };
+  auto fused = [&](size_t) { return batch_fuses(eligible); };
+  auto launch_proj_adam = [&](size_t gi, cudaStream_t s) -> galore_status_t {
+    tensor_group_reset(scratch.proj);
+    const galore_layer* first = layers[groups[gi][0].index];
+    for (const BatchMember& mb : groups[gi]) {
+      galore_layer* l = layers[mb.index];
+      float* part; void* nbuf;
+      scratch_of(gi, mb, &part, &nbuf);
+      GALORE_TRY(tensor_group_add_project_adam(scratch.proj, &l->tc, l->cfg, l->left, G[mb.index], ldg[mb.index],
+                                               tc_adam_args(l, nbuf, adam_params(l)), l->status));
+    }
+    PhaseTimer pt(0, s);
+    return tensor_group_launch_project_adam(scratch.proj, first->cfg.state_fmt, s);
   };
   auto launch_proj = [&](size_t gi, cudaStream_t s) -> galore_status_t {
     tensor_group_reset(scratch.proj);
@@ -736,8 +792,12 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
   // stream under the projection of group g+1 was measured and dropped: within 2 % either way, and
   // other experiments with two streams of kernels around the tensor-core kernels stalled.)
   for (size_t gi = 0; gi < groups.size(); ++gi) {
-    GALORE_TRY(launch_proj(gi, st));
-    GALORE_TRY(launch_adam(gi, st));
+    if (fused(gi)) {
+      GALORE_TRY(launch_proj_adam(gi, st));
+    } else {
+      GALORE_TRY(launch_proj(gi, st));
+      GALORE_TRY(launch_adam(gi, st));
+    }
     GALORE_TRY(launch_back(gi, st));
   }
   return worst;
@@ -841,6 +901,85 @@ galore_status_t galore_device_status(galore_layer_t* l, int32_t* flags, void* st
   GALORE_CUDA_TRY(cudaMemsetAsync(l->status, 0, sizeof(f), st));
   GALORE_CUDA_TRY(cudaStreamSynchronize(st));
   *flags = f;
+  return GALORE_OK;
+}
+
+galore_status_t galore_check_device(galore_layer_t* l, void* stream) {
+  int32_t f = 0;
+  GALORE_TRY(galore_device_status(l, &f, stream));
+  if (f & GALORE_DEV_WAIT_EXPIRED) return GALORE_ERR_TIMEOUT;
+  if (f & GALORE_DEV_NONFINITE) return GALORE_ERR_NONFINITE;
+  if (f & GALORE_DEV_CHOLESKY) return GALORE_ERR_STATE;
+  return GALORE_OK;
+}
+
+// ---- checkpoint: what Algorithm 1 carries from one iteration to the next (P, M, V, step count) ----
+namespace {
+
+struct ExportHeader {
+  uint64_t magic;          // "GALOREST"
+  uint32_t version;
+  uint32_t header_bytes;
+  uint64_t layout_hash;    // of everything that fixes the layout of the state buffer
+  int64_t completed_steps;
+  int32_t has_projector;
+  int32_t reserved;
+  uint64_t state_bytes;
+};
+constexpr uint64_t kExportMagic = 0x5453455230414c47ull;
+
+uint64_t layout_hash(const galore_layer* l) {
+  const int64_t fields[] = {l->cfg.m, l->cfg.n, l->cfg.rank, l->left ? 1 : 0, l->cfg.p_dtype, l->cfg.state_fmt,
+                            l->q_block, l->ld_s, (int64_t)l->state_bytes};
+  uint64_t h = 1469598103934665603ull;          // FNV-1a over the bytes of the fields
+  for (int64_t f : fields)
+    for (int b = 0; b < 8; ++b) {
+      h ^= (uint64_t)(f >> (8 * b)) & 0xffu;
+      h *= 1099511628211ull;
+    }
+  return h;
+}
+
+}  // namespace
+
+galore_status_t galore_export_bytes(const galore_layer_t* l, size_t* bytes) {
+  if (!l || !bytes) return GALORE_ERR_INVALID_ARG;
+  *bytes = sizeof(ExportHeader) + l->state_bytes;
+  return GALORE_OK;
+}
+
+galore_status_t galore_export_state(galore_layer_t* l, void* dst_host, size_t bytes, void* stream) {
+  if (!l || !dst_host) return GALORE_ERR_INVALID_ARG;
+  if (bytes < sizeof(ExportHeader) + l->state_bytes) return GALORE_ERR_BUFFER_TOO_SMALL;
+  ExportHeader h = {};
+  h.magic = kExportMagic;
+  h.version = 1;
+  h.header_bytes = (uint32_t)sizeof(ExportHeader);
+  h.layout_hash = layout_hash(l);
+  h.completed_steps = l->k;
+  h.has_projector = l->has_projector ? 1 : 0;
+  h.state_bytes = l->state_bytes;
+  memcpy(dst_host, &h, sizeof(h));
+  cudaStream_t st = (cudaStream_t)stream;
+  GALORE_CUDA_TRY(cudaMemcpyAsync((char*)dst_host + sizeof(h), l->P, l->state_bytes, cudaMemcpyDeviceToHost, st));
+  GALORE_CUDA_TRY(cudaStreamSynchronize(st));
+  return GALORE_OK;
+}
+
+galore_status_t galore_import_state(galore_layer_t* l, const void* src_host, size_t bytes, void* stream) {
+  if (!l || !src_host) return GALORE_ERR_INVALID_ARG;
+  if (bytes < sizeof(ExportHeader)) return GALORE_ERR_BUFFER_TOO_SMALL;
+  ExportHeader h;
+  memcpy(&h, src_host, sizeof(h));
+  if (h.magic != kExportMagic || h.version != 1 || h.header_bytes != sizeof(ExportHeader)) return GALORE_ERR_INVALID_ARG;
+  if (h.layout_hash != layout_hash(l) || h.state_bytes != l->state_bytes) return GALORE_ERR_STATE;   // another configuration
+  if (bytes < sizeof(ExportHeader) + l->state_bytes || h.completed_steps < 0) return GALORE_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  GALORE_CUDA_TRY(cudaMemcpyAsync(l->P, (const char*)src_host + sizeof(h), l->state_bytes, cudaMemcpyHostToDevice, st));
+  GALORE_CUDA_TRY(cudaStreamSynchronize(st));
+  l->k = h.completed_steps;
+  l->has_projector = h.has_projector != 0;
+  l->refreshed_here = false;
   return GALORE_OK;
 }
 

@@ -906,6 +906,34 @@ int sm_count() {
   return sms;
 }
 
+// Launches of these kernels given on different streams are chained with an event, in the order of
+// the calls.  One CTA takes a whole SM's tensor memory and nearly all of its shared memory, so two
+// of them never share an SM and little is lost; runs that kept several streams of them in flight
+// did not finish on the test machines, and no cause was found in the code.
+struct StreamChain {
+  std::mutex mutex;
+  cudaStream_t last[64] = {};
+  cudaEvent_t done[64] = {};
+  bool used[64] = {};
+};
+StreamChain g_chain;
+
+galore_status_t chain_before(cudaStream_t st, int* dev_out) {
+  int dev = 0;
+  GALORE_CUDA_TRY(cudaGetDevice(&dev));
+  *dev_out = dev;
+  if (dev < 0 || dev >= 64) return GALORE_ERR_INVALID_ARG;
+  if (g_chain.used[dev] && g_chain.last[dev] != st) GALORE_CUDA_TRY(cudaStreamWaitEvent(st, g_chain.done[dev], 0));
+  return GALORE_OK;
+}
+galore_status_t chain_after(cudaStream_t st, int dev) {
+  if (!g_chain.done[dev]) GALORE_CUDA_TRY(cudaEventCreateWithFlags(&g_chain.done[dev], cudaEventDisableTiming));
+  GALORE_CUDA_TRY(cudaEventRecord(g_chain.done[dev], st));
+  g_chain.last[dev] = st;
+  g_chain.used[dev] = true;
+  return GALORE_OK;
+}
+
 template <int EPI, typename TW, int CTAS>
 galore_status_t launch_tc_variant(const TcGroup& g, cudaStream_t st) {
   auto kern = gemm_tc_kernel<EPI, TW, CTAS>;
@@ -931,9 +959,12 @@ galore_status_t launch_tc_variant(const TcGroup& g, cudaStream_t st) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  std::lock_guard<std::mutex> lock(g_chain.mutex);
+  int dev = 0;
+  GALORE_TRY(chain_before(st, &dev));
   GALORE_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, g));
   count_launch();
-  return GALORE_OK;
+  return chain_after(st, dev);
 }
 
 // every problem of a group was tiled for the same variant (TcParams::tile_m)

@@ -299,50 +299,6 @@ __global__ void place_diag_inverse_kernel(const S* __restrict__ slabs, int b, S*
   }
 }
 
-// ---- parallel one-sided Jacobi on a symmetric matrix -------------------------------
-// X starts as H, Vt as the identity.  A rotation of rows (p, q) that makes the
-// two rows of X orthogonal is applied to X and to Vt; at convergence
-// X = Theta V^T, so row norms are the eigenvalues and rows of Vt the eigenvectors.
-// One launch handles one round of the round-robin schedule: np/2 disjoint pairs.
-__global__ void __launch_bounds__(256) jacobi_round_kernel(double* __restrict__ X, double* __restrict__ Vt, int b, int np,
-                                                           int round, double tol, int* __restrict__ rotations) {
-  __shared__ double red[8];
-  const int k = blockIdx.x;
-  auto player = [&](int pos) { return pos == 0 ? 0 : 1 + (((pos - 1 - round) % (np - 1)) + (np - 1)) % (np - 1); };
-  int p = player(k), q = player(np - 1 - k);
-  if (p >= b || q >= b) return;
-  if (p > q) { int t = p; p = q; q = t; }
-  double* xp = X + (int64_t)p * b;
-  double* xq = X + (int64_t)q * b;
-  double app = 0.0, aqq = 0.0, apq = 0.0;
-  for (int j = threadIdx.x; j < b; j += 256) {
-    double a = xp[j], c = xq[j];
-    app += a * a;
-    aqq += c * c;
-    apq += a * c;
-  }
-  app = block_sum_256(app, red);
-  aqq = block_sum_256(aqq, red);
-  apq = block_sum_256(apq, red);
-  if (apq == 0.0 || fabs(apq) <= tol * sqrt(app * aqq)) return;
-  const double zeta = (aqq - app) / (2.0 * apq);
-  const double t = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
-  const double c = 1.0 / sqrt(1.0 + t * t);
-  const double s = c * t;
-  double* vp = Vt + (int64_t)p * b;
-  double* vq = Vt + (int64_t)q * b;
-  for (int j = threadIdx.x; j < b; j += 256) {
-    double a = xp[j], d = xq[j];
-    xp[j] = c * a - s * d;
-    xq[j] = s * a + c * d;
-    a = vp[j];
-    d = vq[j];
-    vp[j] = c * a - s * d;
-    vq[j] = s * a + c * d;
-  }
-  if (threadIdx.x == 0) atomicAdd(rotations, 1);
-}
-
 __global__ void __launch_bounds__(256) row_norm_kernel(const double* __restrict__ X, int b, double* __restrict__ lam) {
   __shared__ double red[8];
   const double* x = X + (int64_t)blockIdx.x * b;

@@ -9,8 +9,10 @@
 // intermediates are placed in one fixed array that is part of the loaded module.
 //
 // The array is shared by every call in the process (per device) and keeps whatever the previous
-// call left in it.  Nothing in it needs to start at zero except the status word, which each call
-// clears itself; every other byte that is read has been written earlier in the same call.  Two
+// call left in it.  Nothing in it needs to start at zero except the word that collects this call's
+// status bits, which each call clears itself (a second word accumulates them across calls until
+// galore_static_status() reads it); every other byte that is read has been written earlier in the
+// same call.  Two
 // calls whose GPU work overlaps (different streams, or different host threads) would both write
 // the array and race: callers serialise them.
 #include <mutex>
@@ -45,9 +47,37 @@ static galore_status_t static_scratch(void** out) {
   return GALORE_OK;
 }
 
+// the bits of this call (word 0) are added to the word that only galore_static_status() clears (word 1)
+__global__ void fold_status_kernel(int32_t* words) {
+  if (words[0]) atomicOr(words + 1, words[0]);
+}
+
+// the stream, if one is given, must live on the device whose array is about to be used
+static galore_status_t check_stream_device(cudaStream_t st) {
+  if (!st || st == cudaStreamLegacy || st == cudaStreamPerThread) return GALORE_OK;
+  int cur = 0, dev = 0;
+  GALORE_CUDA_TRY(cudaGetDevice(&cur));
+  GALORE_CUDA_TRY(cudaStreamGetDevice(st, &dev));
+  return dev == cur ? GALORE_OK : GALORE_ERR_INVALID_ARG;
+}
+
 }  // namespace galore
 
 using namespace galore;
+
+extern "C" galore_status_t galore_static_status(int32_t* flags, void* stream) {
+  if (!flags) return GALORE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  GALORE_TRY(check_stream_device(st));
+  void* base = nullptr;
+  GALORE_TRY(static_scratch(&base));
+  int32_t f = 0;
+  GALORE_CUDA_TRY(cudaMemcpyAsync(&f, (int32_t*)base + 1, sizeof(f), cudaMemcpyDeviceToHost, st));
+  GALORE_CUDA_TRY(cudaMemsetAsync((int32_t*)base + 1, 0, sizeof(f), st));
+  GALORE_CUDA_TRY(cudaStreamSynchronize(st));
+  *flags = f;
+  return GALORE_OK;
+}
 
 extern "C" galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank, int32_t side, float alpha,
                                                double beta1, double beta2, double eps, int64_t completed_steps,
@@ -78,13 +108,14 @@ extern "C" galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank
   const size_t need = 256 + align_up((size_t)splits * nel * 4, 256) + align_up((size_t)nel * 4, 256);
   if (need > kStaticScratchBytes) return GALORE_ERR_BUFFER_TOO_SMALL;   // layer too large for the built-in scratch
 
+  cudaStream_t st = (cudaStream_t)stream;
+  GALORE_TRY(check_stream_device(st));
   void* base = nullptr;
   GALORE_TRY(static_scratch(&base));
-  cudaStream_t st = (cudaStream_t)stream;
   int32_t* status = (int32_t*)base;
   float* Rpart = (float*)((char*)base + 256);
   float* Nbuf = (float*)((char*)base + 256 + align_up((size_t)splits * nel * 4, 256));
-  GALORE_CUDA_TRY(cudaMemsetAsync(status, 0, 256, st));   // the one part that must start at zero
+  GALORE_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));   // this call's bits: the one part that must start at zero
 
   EpiStore<float, float> epi{Rpart, scols, nel, 1.f, 0.f};
   if (left)
@@ -114,6 +145,9 @@ extern "C" galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank
     GALORE_TRY((launch_gemm_simt<float, float, float>((int)m, (int)n, r, P, r, 1, Nbuf, n, 1, 1, apply, st)));
   else
     GALORE_TRY((launch_gemm_simt<float, float, float>((int)m, (int)n, r, Nbuf, r, 1, P, 1, r, 1, apply, st)));
+
+  fold_status_kernel<<<1, 1, 0, st>>>(status);
+  GALORE_LAUNCH_CHECK();
 
   if (device_flags) {   // optional: wait for the step and report what the kernels latched
     int32_t f = 0;

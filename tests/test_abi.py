@@ -76,6 +76,17 @@ def test_invalid_configs_are_rejected(kw, status):
         gb.galore_query_bytes(cfg)
 
 
+def test_states_too_large_for_32_bit_row_arithmetic_are_refused():
+    # 2^31 - 1 columns at rank 2: the state has 2 rows of 2^31 elements, beyond what the kernels index
+    cfg = gb.make_config(4, 2 ** 31 - 1, 2, w_dtype="f32", g_dtype="f32")
+    sb, wb = C.c_size_t(), C.c_size_t()
+    assert gb.lib().galore_query_bytes(C.byref(cfg), C.byref(sb), C.byref(wb)) == gb.ERR_SHAPE
+    out = C.c_void_p()
+    assert gb.lib().galore_init_layer(C.byref(cfg), 256, 1 << 40, 256, 1 << 40, None, C.byref(out)) == gb.ERR_SHAPE
+    # a large but addressable layer is accepted
+    assert gb.lib().galore_query_bytes(C.byref(gb.make_config(16384, 65536, 2048)), C.byref(sb), C.byref(wb)) == 0
+
+
 def test_rank_equal_to_min_dimension_is_legal():
     gb.galore_query_bytes(gb.make_config(12, 20, 12, w_dtype="f32", g_dtype="f32"))
 

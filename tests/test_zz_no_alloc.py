@@ -4,8 +4,8 @@ Some users of the library run where a device allocation is off limits (a framewo
 device memory and forbids cudaMalloc, or a call site that cannot afford the device-wide
 synchronisation an allocation implies), so they cannot create the workspace the regular entry
 points need.  galore_step_static keeps its intermediates in an array built into the library.
-This file checks it against the regular galore_step on two consecutive steps; it is named so that
-pytest collects it after every other test file.
+This file checks it against the regular galore_step and against the CPU oracle on two consecutive
+steps; it is named so that pytest collects it after every other test file.
 """
 import ctypes as C
 
@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import galore_oracle as go
 from paper_2403_03507_b200 import binding as gb
 from paper_2403_03507_b200 import workloads as wl
 
@@ -41,9 +42,15 @@ def test_static_step_matches_regular_step_on_two_calls_in_a_row(m, n, r):
     W_ref, W_new = W0.clone(), W0.clone()
     M = torch.zeros(layer.state_shape, device="cuda")
     V = torch.zeros(layer.state_shape, device="cuda")
+    orc = go.GaLoreOracle(m, n, r, 0.25, 1000, w_store="f32", state="f32")
+    orc.set_projector(P.double().cpu().numpy())
+    W_orc = W0.double().cpu().numpy()
+    gb.galore_static_status()                      # start from a clean accumulated status word
     # the second step and the second shape run with whatever earlier calls left in the shared array
     for s in range(2):
-        G = torch.from_numpy(wl.make_gradient(m, n, wl.sub_seed(3, s), 1.0, 0.01, "f32")).float().cuda()
+        Gh = wl.make_gradient(m, n, wl.sub_seed(3, s), 1.0, 0.01, "f32")
+        G = torch.from_numpy(Gh).float().cuda()
+        W_orc = orc.step(W_orc, Gh, 1e-2, auto_refresh=False)
         layer.galore_step(W_ref, G, 1e-2)
         flags = gb.galore_step_static(P, M, V, W_new, G, 1e-2, completed_steps=s)
         assert flags == 0
@@ -51,6 +58,29 @@ def test_static_step_matches_regular_step_on_two_calls_in_a_row(m, n, r):
         err = (W_new.double() - W_ref.double()).norm() / W_ref.double().norm()
         derr = ((W_new.double() - W0.double()) - (W_ref.double() - W0.double())).norm() / (W_ref.double() - W0.double()).norm()
         assert err <= TOL_W_F32 and derr <= 1e-3, (s, float(err), float(derr))
+        # and against the oracle, within the fp32-path tolerance
+        Wn = W_new.double().cpu().numpy()
+        assert np.linalg.norm(Wn - W_orc) / np.linalg.norm(W_orc) <= TOL_W_F32
         M_ref, V_ref = layer.get_moments()
         assert torch.allclose(M, M_ref, rtol=1e-5, atol=1e-12) and torch.allclose(V, V_ref, rtol=1e-5, atol=1e-20)
     assert layer.device_status() == 0
+    assert gb.galore_static_status() == 0
+
+
+@pytest.mark.gpu
+def test_static_step_keeps_status_bits_for_the_asynchronous_form():
+    """Without a flags pointer the call returns at once; what its kernels latch must still be readable later."""
+    m, n, r = 64, 96, 8
+    P = torch.eye(m, device="cuda")[:, :r].contiguous()
+    M = torch.zeros(r, n, device="cuda")
+    V = torch.zeros(r, n, device="cuda")
+    W = torch.zeros(m, n, device="cuda")
+    G = torch.ones(m, n, device="cuda")
+    gb.galore_static_status()
+    G[0, 0] = float("inf")
+    assert gb.galore_step_static(P, M, V, W, G, 1e-2, completed_steps=0, want_flags=False) == 0
+    G[0, 0] = 1.0
+    M.zero_(); V.zero_()
+    assert gb.galore_step_static(P, M, V, W, G, 1e-2, completed_steps=0, want_flags=True) == 0   # this call was clean
+    assert gb.galore_static_status() & gb.DEV_NONFINITE        # the earlier one is not lost
+    assert gb.galore_static_status() == 0
