@@ -24,7 +24,7 @@ What it follows (GaLore, arXiv 2403.03507):
   * Sec. 4.3 ("8-bit optimizers") names block-wise 8-bit Adam states without
     giving a format.  The format used here is this project's own and is
     spelled out at `dynamic_code` (the code values) and `state_tile` (which
-    elements share an absmax: tiles of q_block / 128 rows x 128 columns of the
+    elements share an absmax: tiles of q_block / 64 rows x 64 columns of the
     state matrix); it is PARITY UNPINNED against the paper
     (the paper fixes nothing to pin it to) and pinned only by its own
     invariants in the tests.
@@ -261,14 +261,14 @@ def dequantize_blockwise(codes, absmax, signed: bool, block: int = 2048):
     return dequantize_tiles(codes, am, signed, 1, block).reshape(-1)
 
 
-STATE_TILE_COLS = 128
+STATE_TILE_COLS = 64
 
 
 def state_tile(q_block: int):
     """Shape of the quantisation blocks of the 8-bit moments: q_block elements as a tile of
-    q_block / 128 consecutive rows x 128 consecutive columns of the state matrix (2048 -> 16 x 128)."""
+    q_block / 64 consecutive rows x 64 consecutive columns of the state matrix (2048 -> 32 x 64)."""
     if q_block % STATE_TILE_COLS:
-        raise ValueError("q_block must be a multiple of 128")
+        raise ValueError("q_block must be a multiple of 64")
     return q_block // STATE_TILE_COLS, STATE_TILE_COLS
 
 

@@ -115,7 +115,7 @@ def test_q8_states_track_fp32_states():
         Wa, Wb = a.step(Wa, g, 1e-2), b.step(Wb, g, 1e-2)
     Ma, Va = a.moments()
     Mb, Vb = b.moments()
-    assert b.M_absmax.shape == ((r + 1) // 2, (n + 127) // 128)        # q_block 256 = tiles of 2 x 128
+    assert b.M_absmax.shape == ((r + 3) // 4, (n + 63) // 64)          # q_block 256 = tiles of 4 x 64
     assert np.linalg.norm(Mb - Ma) / np.linalg.norm(Ma) < 0.05
     assert np.linalg.norm((Wb - W0) - (Wa - W0)) / np.linalg.norm(Wa - W0) < 0.1
     # first step does not depend on the state format at all (states start at zero)
@@ -126,7 +126,7 @@ def test_q8_states_track_fp32_states():
 
 
 @pytest.mark.parametrize("signed", [True, False])
-@pytest.mark.parametrize("rows,cols,tr,tc", [(37, 300, 16, 128), (5, 128, 2, 128), (16, 129, 16, 128), (40, 90, 8, 32)])
+@pytest.mark.parametrize("rows,cols,tr,tc", [(37, 300, 32, 64), (5, 128, 4, 64), (33, 65, 32, 64), (40, 90, 8, 32)])
 def test_tiles_brute_force_geometry_and_codes(signed, rows, cols, tr, tc):
     """Which elements share an absmax, written out with explicit index arithmetic, and the nearest code by
     exhaustive search over the 256 values."""
@@ -175,10 +175,10 @@ def test_flat_blocks_are_tiles_of_a_one_row_matrix():
 
 
 def test_state_tile_shapes():
-    assert go.state_tile(2048) == (16, 128) and go.state_tile(256) == (2, 128) and go.state_tile(4096) == (32, 128)
+    assert go.state_tile(2048) == (32, 64) and go.state_tile(256) == (4, 64) and go.state_tile(1024) == (16, 64)
     with pytest.raises(ValueError):
         go.state_tile(1000)
-    o = go.GaLoreOracle(40, 300, 24, 0.25, 10, state="q8", q_block=2048)
-    assert o.M_codes.shape == (24, 300) and o.M_absmax.shape == (2, 3)
+    o = go.GaLoreOracle(40, 300, 40, 0.25, 10, state="q8", q_block=2048)
+    assert o.M_codes.shape == (40, 300) and o.M_absmax.shape == (2, 5)
     o = go.GaLoreOracle(300, 40, 24, 0.25, 10, state="q8", q_block=512)          # right side: state is m x r
-    assert o.V_codes.shape == (300, 24) and o.V_absmax.shape == (75, 1)
+    assert o.V_codes.shape == (300, 24) and o.V_absmax.shape == (38, 1)
