@@ -260,6 +260,11 @@ def main():
                          "projector (step timing does not depend on P's values; for short profiling runs)")
     ap.add_argument("--weight-decay", type=float, default=0.0,
                     help="GaLore-AdamW: decoupled weight decay folded into the weight update (0 = plain Adam)")
+    ap.add_argument("--adam-place", default="auto", choices=["auto", "projection", "own"],
+                    help="where Adam on R runs when K is not sliced: in the projection kernel's epilogue or in its own kernel")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="keep only this many transformer layers of the workload's layer set (0 = all): a small case "
+                         "of the same kernels for profiler captures")
     ap.add_argument("--rank", type=int, default=0, help="override the workload's rank (rank sweep on one shape)")
     ap.add_argument("--state-fmt", default="", choices=["", "f32", "q8"], help="override the workload's state format")
     ap.add_argument("--refresh-only", action="store_true",
@@ -278,6 +283,11 @@ def main():
     if args.rank or args.state_fmt:
         import dataclasses
         w = dataclasses.replace(w, rank=args.rank or w.rank, state_fmt=args.state_fmt or w.state_fmt)
+    if args.layers > 0 and len(w.shapes) == 3:
+        import dataclasses
+        (a, b, c4), (d, e, c2), (f, g, c1) = w.shapes
+        keep = min(args.layers, c1)
+        w = dataclasses.replace(w, shapes=((a, b, 4 * keep), (d, e, 2 * keep), (f, g, keep)))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -346,7 +356,8 @@ def time_workload(w, args, dev, dist, world, rank, full, mode=None):
     for (m, n, count) in w.shapes:
         cfg = gb.make_config(m, n, w.rank, alpha=w.alpha, refresh_gap=w.refresh_gap, beta1=w.beta1, beta2=w.beta2,
                              eps=w.eps, w_dtype=w.w_dtype, g_dtype=w.g_dtype, state_fmt=w.state_fmt,
-                             q_block=w.q_block, auto_refresh=False, seed=w.seed, weight_decay=args.weight_decay)
+                             q_block=w.q_block, auto_refresh=False, seed=w.seed, weight_decay=args.weight_decay,
+                             adam_place={"auto": gb.ADAM_AUTO, "projection": gb.ADAM_IN_PROJECTION, "own": gb.ADAM_OWN_KERNEL}[args.adam_place])
         cfgs[(m, n)] = cfg
         max_ws = max(max_ws, gb.galore_query_bytes(cfg)[1])
     workspace = torch.empty(max_ws, dtype=torch.uint8, device=dev)      # shared: layers step one after another

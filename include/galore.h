@@ -72,6 +72,8 @@ typedef enum {
   GALORE_PATH_TENSOR = 2  /* tcgen05 kernels; init fails with GALORE_ERR_ALIGNMENT/UNIMPLEMENTED if not eligible */
 } galore_path_t;
 
+typedef enum { GALORE_ADAM_AUTO = 0, GALORE_ADAM_IN_PROJECTION = 1, GALORE_ADAM_OWN_KERNEL = 2 } galore_adam_place_t;
+
 /* Bits of the device status word. */
 enum {
   GALORE_DEV_NONFINITE = 1,     /* a non-finite projected gradient was seen */
@@ -93,8 +95,8 @@ typedef struct {
   int32_t g_dtype;         /* galore_dtype_t of G */
   int32_t p_dtype;         /* galore_dtype_t the projector is stored in */
   int32_t state_fmt;       /* galore_state_fmt_t of M, V */
-  int32_t q_block;         /* elements per quantisation block: 256, 512, 1024, 2048 or 4096 (0 = 2048); a block is a
-                              tile of q_block / 128 consecutive rows x 128 consecutive columns of the state matrix */
+  int32_t q_block;         /* elements per quantisation block: 256, 512, 1024 or 2048 (0 = 2048); a block is a
+                              tile of q_block / 64 consecutive rows x 64 consecutive columns of the state matrix */
   int32_t auto_refresh;    /* 1: galore_step refreshes P when (completed steps) mod T == 0 */
   int32_t path;            /* galore_path_t */
   /* refresh: block subspace iteration on a block of rank + refresh_oversample
@@ -111,7 +113,11 @@ typedef struct {
    * supported optimizer without equations; the reading taken is Loshchilov & Hutter's:
    * W <- W (1 - lr lambda) - lr alpha P N, the decay on the full-rank weight with the plain lr. */
   float weight_decay;
-  int32_t reserved[7];
+  /* Where Adam on R runs when the projection's K is not sliced (galore_adam_place_t): AUTO lets the
+   * library choose per state format; IN_PROJECTION runs it in the projection kernel's epilogue (R is
+   * never stored); OWN_KERNEL always uses the stand-alone Adam kernel after the projection. */
+  int32_t adam_place;
+  int32_t reserved[6];
 } galore_config_t;
 
 /* Result of one refresh (host struct, filled after the refresh's stream work has completed). */
@@ -197,12 +203,17 @@ galore_status_t galore_step_host_batch(galore_layer_t* const* layers, void* cons
 galore_status_t galore_refresh_projector(galore_layer_t* layer, const void* G, int64_t ldg, void* stream,
                                          galore_refresh_info_t* info);
 
-/* The same refresh for `count` layers, one after another on `stream` (Algorithm 1 refreshes
- * every layer at the same steps), with `workspace` (device memory, 256-byte aligned, at least
- * galore_refresh_query_bytes() of every layer) in place of each layer's own refresh workspace,
- * so that layers which share their workspace can be refreshed through one call.
- * infos: NULL or `count` records.  Stops at the first error; otherwise returns
- * GALORE_WARN_NOT_CONVERGED if any layer reached its iteration cap. */
+/* The same refresh for `count` layers on `stream` (Algorithm 1 refreshes every layer at the same
+ * steps), with `workspace` (device memory, 256-byte aligned, at least galore_refresh_query_bytes()
+ * of every layer) in place of each layer's own refresh workspace, so that layers which share their
+ * workspace can be refreshed through one call.  Neighbours in the list that have the same shape,
+ * rank and dtypes are refreshed together, as many at a time (up to 8) as `workspace` holds copies
+ * of galore_refresh_query_bytes(): the serial parts of the method (Cholesky panels, the dense
+ * eigen-solver) then run for all of them at once.  Every layer receives the projector it would
+ * receive from galore_refresh_projector alone.
+ * infos: NULL or `count` records (phase times of layers refreshed together are the group's divided
+ * by its size).  Stops at the first error; otherwise returns GALORE_WARN_NOT_CONVERGED if any layer
+ * reached its iteration cap. */
 galore_status_t galore_refresh_query_bytes(const galore_layer_t* layer, size_t* bytes);
 galore_status_t galore_refresh_batch(galore_layer_t* const* layers, const void* const* G, const int64_t* ldg,
                                      int32_t count, void* workspace, size_t workspace_bytes, void* stream,
@@ -269,7 +280,7 @@ galore_status_t galore_set_projector(galore_layer_t* layer, const float* src, si
 /* Stored (uncorrected) moments as fp32, shape of R row-major packed, device memory (8-bit states are dequantised). */
 galore_status_t galore_get_moments(galore_layer_t* layer, float* M, float* V, size_t bytes_each, void* stream);
 /* Raw 8-bit state: codes (uint8, shape of R, packed) and per-block absmax (fp32, tile (I, J) of the
- * state at I * ceil(cols / 128) + J); device memory. */
+ * state at I * ceil(cols / 64) + J); device memory. */
 galore_status_t galore_get_q8_state(galore_layer_t* layer, uint8_t* M_codes, float* M_absmax,
                                     uint8_t* V_codes, float* V_absmax, void* stream);
 /* Completed steps k. */
@@ -308,7 +319,7 @@ galore_status_t galore_q8_codebook(int32_t is_signed, float* out256_host);
  * (I, J) at absmax[I * ceil(cols / tile_cols) + J]; tiles on the lower and right edges are cut off
  * at the border.  A flat array with blocks of b consecutive elements is rows = 1, tile 1 x b.
  * code = nearest code value to fp32(x / absmax), ties to the larger index; absmax = 0 stores the
- * code of 0.  The moments of a layer use tiles of (q_block / 128) x 128 of the state matrix. */
+ * code of 0.  The moments of a layer use tiles of (q_block / 64) x 64 of the state matrix. */
 galore_status_t galore_q8_quantize(const float* x, int64_t rows, int64_t cols, int32_t is_signed, int32_t tile_rows,
                                    int32_t tile_cols, uint8_t* codes, float* absmax, void* stream);
 galore_status_t galore_q8_dequantize(const uint8_t* codes, const float* absmax, int64_t rows, int64_t cols,

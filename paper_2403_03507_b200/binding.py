@@ -21,6 +21,7 @@ SIDE_AUTO, SIDE_LEFT, SIDE_RIGHT = 0, 1, 2
 F32, BF16 = 0, 1
 STATE_F32, STATE_Q8_BLOCK = 0, 1
 PATH_AUTO, PATH_FP32, PATH_TENSOR = 0, 1, 2
+ADAM_AUTO, ADAM_IN_PROJECTION, ADAM_OWN_KERNEL = 0, 1, 2
 DEV_NONFINITE, DEV_WAIT_EXPIRED, DEV_CHOLESKY = 1, 2, 8
 
 _DTYPES = {"f32": F32, "bf16": BF16, torch.float32: F32, torch.bfloat16: BF16}
@@ -34,7 +35,7 @@ class Config(C.Structure):
         ("side", C.c_int32), ("w_dtype", C.c_int32), ("g_dtype", C.c_int32), ("p_dtype", C.c_int32),
         ("state_fmt", C.c_int32), ("q_block", C.c_int32), ("auto_refresh", C.c_int32), ("path", C.c_int32),
         ("refresh_tol", C.c_float), ("refresh_max_iters", C.c_int32), ("refresh_oversample", C.c_int32),
-        ("seed", C.c_uint64), ("weight_decay", C.c_float), ("reserved", C.c_int32 * 7),
+        ("seed", C.c_uint64), ("weight_decay", C.c_float), ("adam_place", C.c_int32), ("reserved", C.c_int32 * 6),
     ]
 
 
@@ -142,7 +143,7 @@ def _stream_ptr(stream=None):
 def make_config(m, n, rank, alpha=0.25, refresh_gap=200, beta1=0.9, beta2=0.999, eps=1e-8, side=SIDE_AUTO,
                 w_dtype="bf16", g_dtype="bf16", p_dtype=None, state_fmt="f32", q_block=2048, auto_refresh=True,
                 path=PATH_AUTO, refresh_tol=0.0, refresh_max_iters=0, refresh_oversample=0, seed=0,
-                weight_decay=0.0) -> Config:
+                weight_decay=0.0, adam_place=ADAM_AUTO) -> Config:
     c = Config()
     c.m, c.n, c.rank, c.alpha, c.refresh_gap = m, n, rank, alpha, refresh_gap
     c.beta1, c.beta2, c.eps = beta1, beta2, eps
@@ -155,6 +156,7 @@ def make_config(m, n, rank, alpha=0.25, refresh_gap=200, beta1=0.9, beta2=0.999,
     c.q_block, c.auto_refresh, c.path = q_block, int(bool(auto_refresh)), path
     c.refresh_tol, c.refresh_max_iters, c.refresh_oversample, c.seed = refresh_tol, refresh_max_iters, refresh_oversample, seed
     c.weight_decay = weight_decay
+    c.adam_place = adam_place
     return c
 
 
@@ -170,7 +172,7 @@ def galore_q8_codebook(is_signed: bool):
     return list(out)
 
 
-STATE_TILE_COLS = 128
+STATE_TILE_COLS = 64
 
 
 def _tile_of(x, block, tile):

@@ -6,7 +6,7 @@
 // sliced over CTAs): they sum the split-K partials of R in a fixed order,
 // update the stored (uncorrected) moments, and emit the normalised update N
 // in the dtype the back-projection consumes.  A CTA handles one tile of
-// tile_rows x 128 state elements at a time; for 8-bit moments that tile is
+// tile_rows x 64 state elements at a time; for 8-bit moments that tile is
 // the quantisation block, so the block's absmax is a warp-shuffle +
 // shared-memory reduction and the state makes one round trip through HBM.
 #include "adam.cuh"
@@ -190,11 +190,11 @@ __device__ __forceinline__ void find_item(const AdamGroup& g, int gb, int& it, i
   local = gb - (it > 0 ? g.block_end[it - 1] : 0);
 }
 
-// Where a thread works inside a tile of 2 E rows x 128 columns: E consecutive elements of one row.
+// Where a thread works inside a tile of 4 E rows x 64 columns: E consecutive elements of one row.
 template <int E>
 struct TileThread {
   static constexpr int kPerRow = kStateTileCols / E;      // threads per tile row
-  static constexpr int kRows = 256 / kPerRow;             // = 2 E
+  static constexpr int kRows = 256 / kPerRow;             // = 4 E
   int row, col;
   __device__ __forceinline__ TileThread(int tile_r, int tile_c)
       : row(tile_r * kRows + (int)threadIdx.x / kPerRow), col(tile_c * kStateTileCols + ((int)threadIdx.x % kPerRow) * E) {}
@@ -299,7 +299,7 @@ __global__ void __launch_bounds__(256, GALORE_F32_CTAS) adam_f32_kernel(const __
 }
 
 // ---- 8-bit block-wise moments ---------------------------------------------------
-// One tile = one quantisation block of 256 E elements (2 E rows x 128 columns).  Elements outside
+// One tile = one quantisation block of 256 E elements (4 E rows x 64 columns).  Elements outside
 // the matrix (edge tiles) enter as zeros with the codes of zero, so they change no absmax.
 #ifndef GALORE_Q8_CTAS
 #define GALORE_Q8_CTAS 4          // resident CTAs per SM the kernel is compiled for (register budget)
@@ -451,7 +451,7 @@ q8_dequantize_kernel(const uint8_t* __restrict__ codes, int64_t ldc, const float
 
 // ---- launchers --------------------------------------------------------------------
 static bool valid_block(int block) {
-  return block == 256 || block == 512 || block == 1024 || block == 2048 || block == 4096;
+  return block == 256 || block == 512 || block == 1024 || block == 2048;
 }
 
 galore_status_t launch_adam_group(const AdamGroup& g, int32_t state_fmt, int q_block, int32_t n_dtype, cudaStream_t st) {
@@ -484,7 +484,7 @@ galore_status_t launch_adam_group(const AdamGroup& g, int32_t state_fmt, int q_b
     else GALORE_Q8_LAUNCH(float, E);                      \
     break;
   switch (q_block) {
-    GALORE_Q8_CASE(1) GALORE_Q8_CASE(2) GALORE_Q8_CASE(4) GALORE_Q8_CASE(8) GALORE_Q8_CASE(16)
+    GALORE_Q8_CASE(1) GALORE_Q8_CASE(2) GALORE_Q8_CASE(4) GALORE_Q8_CASE(8)
     default: return GALORE_ERR_INVALID_ARG;
   }
 #undef GALORE_Q8_CASE
@@ -496,7 +496,7 @@ galore_status_t adam_group_add(AdamGroup& g, const AdamItem& item, int32_t state
   if (g.count >= kAdamGroup) return GALORE_ERR_BUFFER_TOO_SMALL;
   if (item.rows <= 0 || item.cols <= 0) return GALORE_ERR_SHAPE;
   AdamItem a = item;
-  const int tile_rows = state_fmt == GALORE_STATE_F32 ? 16 : q_block / kStateTileCols;
+  const int tile_rows = state_fmt == GALORE_STATE_F32 ? 32 : q_block / kStateTileCols;
   a.tiles_c = (int)ceil_div(a.cols, kStateTileCols);
   const int64_t tiles = ceil_div(a.rows, tile_rows) * a.tiles_c;
   const int64_t before = g.count > 0 ? g.block_end[g.count - 1] : 0;

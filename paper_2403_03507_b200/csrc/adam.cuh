@@ -6,10 +6,10 @@
 
 namespace galore {
 
-constexpr int kStateTileCols = 128;   // a quantisation block is a tile of q_block / 128 rows x 128 columns of the state
+constexpr int kStateTileCols = 64;    // a quantisation block is a tile of q_block / 64 rows x 64 columns of the state
 
 // One layer's share of a grouped Adam launch.  The state (shape of R: rows x cols) is walked in tiles
-// of tile_rows x 128; R partials, N and the state arrays are row-major with their own row pitches.
+// of tile_rows x 64; R partials, N and the state arrays are row-major with their own row pitches.
 struct AdamItem {
   const float* Rpart;      // split-K partials of R
   int splits;
@@ -20,7 +20,7 @@ struct AdamItem {
   uint8_t *Mc, *Vc;        // 8-bit codes with
   float *Mam, *Vam;        // one absmax per tile, tile (I, J) at I * tiles_c + J
   void* Nout;              // normalised update (fp32 or bf16)
-  int tiles_c;             // set by adam_group_add: ceil(cols / 128)
+  int tiles_c;             // set by adam_group_add: ceil(cols / 64)
   int vec;                 // set by adam_group_add: bases and pitches allow the vector accesses of an interior tile
   AdamParams p;
   int32_t* status;
@@ -38,7 +38,7 @@ galore_status_t launch_adam_group(const AdamGroup& g, int32_t state_fmt, int q_b
 galore_status_t launch_adam(const AdamItem& item, int32_t state_fmt, int q_block, int32_t n_dtype, cudaStream_t st);
 
 // Pitches and sizes of a layer's state arrays.  fp32 moments: rows of ceil8(cols) floats; 8-bit codes:
-// rows of ceil32(cols) bytes, plus ceil(rows / (q_block / 128)) * ceil(cols / 128) absmax values.
+// rows of ceil32(cols) bytes, plus ceil(rows / (q_block / 64)) * ceil(cols / 64) absmax values.
 inline int64_t state_pitch(int32_t state_fmt, int64_t cols) {
   return state_fmt == GALORE_STATE_F32 ? (cols + 7) / 8 * 8 : (cols + 31) / 32 * 32;
 }

@@ -119,8 +119,9 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
     if (dt != GALORE_F32 && dt != GALORE_BF16) return GALORE_ERR_INVALID_ARG;
   if (c->state_fmt != GALORE_STATE_F32 && c->state_fmt != GALORE_STATE_Q8_BLOCK) return GALORE_ERR_INVALID_ARG;
   if (c->path < GALORE_PATH_AUTO || c->path > GALORE_PATH_TENSOR) return GALORE_ERR_INVALID_ARG;
+  if (c->adam_place < GALORE_ADAM_AUTO || c->adam_place > GALORE_ADAM_OWN_KERNEL) return GALORE_ERR_INVALID_ARG;
   s->q_block = c->q_block == 0 ? 2048 : c->q_block;
-  if (s->q_block != 256 && s->q_block != 512 && s->q_block != 1024 && s->q_block != 2048 && s->q_block != 4096)
+  if (s->q_block != 256 && s->q_block != 512 && s->q_block != 1024 && s->q_block != 2048)
     return GALORE_ERR_INVALID_ARG;
   s->left = c->side == GALORE_SIDE_AUTO ? (c->m <= c->n) : (c->side == GALORE_SIDE_LEFT);
   const int r = c->rank;
@@ -257,6 +258,15 @@ galore_status_t step_simt(galore_layer* l, void* W, int64_t ldw, const void* G, 
 }
 
 // projection and back-projection on tcgen05, Adam in between reading the padded partials
+// GALORE_ADAM_AUTO, by state format {fp32, 8-bit}.  fp32 moments: the epilogue's work is loads, five
+// multiply-adds and stores per element and hides under the MMAs of the next tile (LLaMA-1B set: 1.86 ms
+// against 1.01 + 1.14 ms for projection and Adam apart).  8-bit moments: about a hundred dependent
+// instructions per element with table lookups in between; the 16 epilogue warps that fit beside the
+// tensor-core pipeline issue 0.3 instructions per cycle and scheduler, the stand-alone kernel with 40
+// warps per SM 0.7, and the tile's epilogue then takes twice as long as its MMAs (LLaMA-7B set: 21.1 ms
+// against 10.3 + 8.0 ms apart).  So 8-bit moments keep the stand-alone kernel unless asked otherwise.
+constexpr bool kAutoFuses[2] = {true, false};
+
 TcAdamArgs tc_adam_args(const galore_layer* l, void* nbuf, const AdamParams& ap) {
   TcAdamArgs a = {};
   a.state_fmt = l->cfg.state_fmt;
@@ -269,9 +279,16 @@ TcAdamArgs tc_adam_args(const galore_layer* l, void* nbuf, const AdamParams& ap)
   return a;
 }
 
+// Adam in the projection's epilogue?  Only when K is not sliced; AUTO: see the note at its definition.
+bool adam_in_projection(const galore_layer* l, int splits) {
+  if (splits != 1 || l->cfg.adam_place == GALORE_ADAM_OWN_KERNEL) return false;
+  if (l->cfg.adam_place == GALORE_ADAM_IN_PROJECTION) return true;
+  return kAutoFuses[l->cfg.state_fmt == GALORE_STATE_F32 ? 0 : 1];
+}
+
 galore_status_t step_tensor(galore_layer* l, void* W, int64_t ldw, const void* G, int64_t ldg, float lr,
                             const AdamParams& ap, cudaStream_t st) {
-  if (l->tc.splits == 1) {
+  if (adam_in_projection(l, l->tc.splits)) {
     // one K slice per tile: Adam runs in the projection's epilogue, R never reaches memory
     PhaseTimer pt(0, st);
     GALORE_TRY(tensor_project_adam(&l->tc, l->cfg, l->left, G, ldg, tc_adam_args(l, l->Nbuf, ap), l->status, st));
@@ -290,8 +307,7 @@ galore_status_t step_tensor(galore_layer* l, void* W, int64_t ldw, const void* G
   return tensor_back_project(&l->tc, l->cfg, l->left, W, ldw, lr * l->cfg.alpha, decay_keep(l, lr), l->status, st);
 }
 
-galore_status_t do_refresh(galore_layer* l, const void* G, int64_t ldg, cudaStream_t st, galore_refresh_info_t* info,
-                           void* workspace = nullptr) {
+RefreshProblem refresh_problem(const galore_layer* l, const void* G, int64_t ldg) {
   RefreshProblem pr;
   pr.G = G;
   pr.g_dtype = l->cfg.g_dtype;
@@ -308,10 +324,23 @@ galore_status_t do_refresh(galore_layer* l, const void* G, int64_t ldg, cudaStre
   pr.max_iters = l->cfg.refresh_max_iters > 0 ? l->cfg.refresh_max_iters : 96;
   pr.first_iters = 6;
   pr.use_tensor = l->tensor_path;
+  return pr;
+}
+
+galore_status_t do_refresh(galore_layer* l, const void* G, int64_t ldg, cudaStream_t st, galore_refresh_info_t* info,
+                           void* workspace = nullptr) {
+  const RefreshProblem pr = refresh_problem(l, G, ldg);
   galore_status_t s = refresh_projector(pr, workspace ? workspace : l->refresh_ws, l->status, info, st);
   if (s >= 0) l->has_projector = true;
   l->refreshed_here = (s >= 0 && workspace == nullptr);
   return s;
+}
+
+// layers that can be refreshed in one group: same problem geometry and the same iteration limits
+bool same_refresh_shape(const galore_layer* a, const galore_layer* b) {
+  return a->cfg.m == b->cfg.m && a->cfg.n == b->cfg.n && a->left == b->left && a->cfg.rank == b->cfg.rank &&
+         a->block == b->block && a->cfg.g_dtype == b->cfg.g_dtype && a->tensor_path == b->tensor_path &&
+         a->cfg.refresh_max_iters == b->cfg.refresh_max_iters;
 }
 
 }  // namespace
@@ -415,11 +444,31 @@ galore_status_t galore_refresh_batch(galore_layer_t* const* layers, const void* 
     if (refresh_workspace_bytes(layers[i]->d, layers[i]->L, layers[i]->cfg.rank, layers[i]->block) > workspace_bytes)
       return GALORE_ERR_BUFFER_TOO_SMALL;
   }
+  // Layers of one shape that follow each other in the list are refreshed together, as many at a time
+  // as the workspace has room for (at most kMaxSlots): the serial parts of the method then run for
+  // all of them in one launch per kernel.
   galore_status_t warn = GALORE_OK;
-  for (int i = 0; i < count; ++i) {
-    const galore_status_t s = do_refresh(layers[i], G[i], ldg[i], (cudaStream_t)stream, infos ? &infos[i] : nullptr, workspace);
+  int i = 0;
+  while (i < count) {
+    const size_t slot = refresh_workspace_bytes(layers[i]->d, layers[i]->L, layers[i]->cfg.rank, layers[i]->block);
+    const int room = (int)std::min<size_t>(kMaxSlots, workspace_bytes / slot);
+    int n = 1;
+    while (n < room && i + n < count && same_refresh_shape(layers[i], layers[i + n])) ++n;
+    RefreshProblem prs[kMaxSlots];
+    int32_t* status[kMaxSlots];
+    for (int j = 0; j < n; ++j) {
+      prs[j] = refresh_problem(layers[i + j], G[i + j], ldg[i + j]);
+      status[j] = layers[i + j]->status;
+    }
+    const galore_status_t s = refresh_projector_group(prs, n, workspace, slot, status, infos ? &infos[i] : nullptr,
+                                                      (cudaStream_t)stream);
     if (s < 0) return s;
+    for (int j = 0; j < n; ++j) {
+      layers[i + j]->has_projector = true;
+      layers[i + j]->refreshed_here = false;
+    }
     if (s > warn) warn = s;
+    i += n;
   }
   return warn;
 }
@@ -590,16 +639,16 @@ namespace {
 // bytes of group scratch one layer needs: R (one or tc_splits partial buffers) and N, each 256-aligned
 // With four or more layers in flight K is not sliced, Adam runs in the projection's epilogue and R is
 // never stored: the group scratch of a layer is its N alone.
-bool batch_fuses(int eligible) { return eligible >= 4; }
-size_t batch_r_bytes(const galore_layer* l, int splits, bool fuse) {
-  return fuse ? 0 : align_up((size_t)splits * l->srows * l->ld_part * 4, 256);
+bool batch_unsliced(int eligible) { return eligible >= 4; }
+size_t batch_r_bytes(const galore_layer* l, int splits) {
+  return adam_in_projection(l, splits) ? 0 : align_up((size_t)splits * l->srows * l->ld_part * 4, 256);
 }
-size_t batch_layer_bytes(const galore_layer* l, int splits, bool fuse) {
-  return batch_r_bytes(l, splits, fuse) + align_up((size_t)l->srows * l->ld_n * 2, 256);
+size_t batch_layer_bytes(const galore_layer* l, int splits) {
+  return batch_r_bytes(l, splits) + align_up((size_t)l->srows * l->ld_n * 2, 256);
 }
 
 // With several layers in flight there are enough tiles to fill the machine without slicing K.
-int batch_splits(const galore_layer* l, int eligible) { return batch_fuses(eligible) ? 1 : l->tc_splits; }
+int batch_splits(const galore_layer* l, int eligible) { return batch_unsliced(eligible) ? 1 : l->tc_splits; }
 
 bool batch_eligible(const galore_layer* l, const void* W, int64_t ldw, const void* G, int64_t ldg) {
   return l->tensor_path && l->has_projector && tensor_operands_aligned(l->cfg, W, ldw, G, ldg);
@@ -649,7 +698,7 @@ galore_status_t galore_batch_query_bytes(galore_layer_t* const* layers, int32_t 
   const int cap = std::min(tensor_group_capacity(), (int)kAdamGroup);
   std::vector<size_t> need;
   for (int32_t i = 0; i < count; ++i)
-    if (layers[i]->tensor_path) need.push_back(batch_layer_bytes(layers[i], batch_splits(layers[i], eligible), batch_fuses(eligible)));
+    if (layers[i]->tensor_path) need.push_back(batch_layer_bytes(layers[i], batch_splits(layers[i], eligible)));
   size_t best = 0, run = 0;
   for (size_t i = 0; i < need.size(); ++i) {
     run += need[i];
@@ -697,7 +746,7 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
       galore_layer* l = layers[i];
       const bool ok = batch_ws && batch_eligible(l, W[i], ldw[i], G[i], ldg[i]);
       const int splits = batch_splits(l, eligible);
-      const size_t need = ok ? batch_layer_bytes(l, splits, batch_fuses(eligible)) : 0;
+      const size_t need = ok ? batch_layer_bytes(l, splits) : 0;
       if (!ok || need > half) {
         // plain step (its refresh, if due, is already done: auto_refresh off for this call)
         const int32_t saved = l->cfg.auto_refresh;
@@ -712,7 +761,8 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
       if (!fresh) {
         const galore_layer* first = layers[groups.back()[0].index];
         const bool same = first->cfg.w_dtype == l->cfg.w_dtype && first->cfg.state_fmt == l->cfg.state_fmt &&
-                          first->q_block == l->q_block && first->tc.ctas == l->tc.ctas;
+                          first->q_block == l->q_block && first->tc.ctas == l->tc.ctas &&
+                          adam_in_projection(first, groups.back()[0].splits) == adam_in_projection(l, splits);
         fresh = !same || (int)groups.back().size() >= cap || used + need > half;
       }
       if (fresh) {
@@ -730,9 +780,9 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
     const galore_layer* l = layers[mb.index];
     char* base = (char*)batch_ws + (gi & 1) * half + mb.offset;
     *part = (float*)base;
-    *nbuf = base + batch_r_bytes(l, mb.splits, batch_fuses(eligible));
+    *nbuf = base + batch_r_bytes(l, mb.splits);
   };
-  auto fused = [&](size_t) { return batch_fuses(eligible); };
+  auto fused = [&](size_t gi) { return adam_in_projection(layers[groups[gi][0].index], groups[gi][0].splits); };
   auto launch_proj_adam = [&](size_t gi, cudaStream_t s) -> galore_status_t {
     tensor_group_reset(scratch.proj);
     const galore_layer* first = layers[groups[gi][0].index];

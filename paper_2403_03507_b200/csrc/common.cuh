@@ -65,6 +65,26 @@ __device__ __forceinline__ double rsqrt_newton(double x) {
   return y * __hiloint2double((1023 - ex / 2) << 20, 0);
 }
 
+// Several copies ("slots") of one workspace layout, `bytes` apart: a launch that carries a slot list
+// runs the same problem in every listed slot, all of its workspace pointers shifted by
+// id[i] * bytes for the i-th part of the grid.  Used to run the latency-bound small kernels of the
+// projector refresh for several layers of the same shape at once.
+constexpr int kMaxSlots = 8;
+struct SlotList {
+  int n;
+  int id[kMaxSlots];
+  int64_t bytes;
+};
+inline SlotList single_slot() {
+  SlotList s = {};
+  s.n = 1;
+  return s;
+}
+template <typename T>
+__host__ __device__ __forceinline__ T* slot_ptr(T* p, int64_t shift) {
+  return (T*)((char*)p + shift);
+}
+
 // Status word in the workspace (first 256 bytes).
 struct DeviceStatus {
   int32_t flags;

@@ -55,9 +55,14 @@ __device__ __forceinline__ BlockPair block_pair(int pair, int round, int nblk) {
 
 // part[(pair * chunks + chunk)] (64 x 64) = rows(pair)[:, chunk] rows(pair)[:, chunk]^T
 __global__ void __launch_bounds__(128) jb_gram_kernel(const double* __restrict__ X, int b, int nblk, int round, int chunks,
-                                                      double* __restrict__ part) {
+                                                      double* __restrict__ part, const SlotList slots) {
   __shared__ __align__(16) double Xs[2][kPairRows][kGramLd];
   const int pair = blockIdx.x, chunk = blockIdx.y;
+  {
+    const int64_t shift = (int64_t)slots.id[blockIdx.z] * slots.bytes;     // blockIdx.z: workspace slot
+    X = slot_ptr(X, shift);
+    part = slot_ptr(part, shift);
+  }
   const BlockPair bp = block_pair(pair, round, nblk);
   if (bp.I * kBlockRows >= b) return;                 // both blocks are padding
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -200,8 +205,16 @@ __device__ __forceinline__ void block_update(const BlockTask& t, const double2* 
 
 __global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* __restrict__ part, int chunks, int b, int nblk,
                                                                  int round, double tol, double* __restrict__ rot_out,
-                                                                 int* __restrict__ flags, int* __restrict__ rotations) {
+                                                                 int* __restrict__ flags, int* __restrict__ rotations,
+                                                                 const SlotList slots) {
   extern __shared__ __align__(16) double jb_smem[];
+  {
+    const int64_t shift = (int64_t)slots.id[blockIdx.y] * slots.bytes;     // blockIdx.y: workspace slot
+    part = slot_ptr(part, shift);
+    rot_out = slot_ptr(rot_out, shift);
+    flags = slot_ptr(flags, shift);
+    rotations = slot_ptr(rotations, shift);
+  }
   // the two copies of A, then the two copies of Rot (addresses computed, not looked up: an array of
   // pointers indexed by the round would live in local memory)
   auto Abuf = [&](int which) { return jb_smem + which * (kPairRows * kALd); };
@@ -315,14 +328,23 @@ __global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* _
 
 // rows(pair)[:, cols] <- Rot rows(pair)[:, cols]  for X (blockIdx.z = 0) and, if present, Vt (blockIdx.z = 1)
 __global__ void __launch_bounds__(256) jb_apply_kernel(double* __restrict__ X, double* __restrict__ Vt, int b, int nblk, int round,
-                                                       const double* __restrict__ rot, const int* __restrict__ flags) {
+                                                       const double* __restrict__ rot, const int* __restrict__ flags,
+                                                       const SlotList slots, int matrices) {
   extern __shared__ __align__(16) double jb_smem[];
   double(*Rs)[kRotLd] = reinterpret_cast<double(*)[kRotLd]>(jb_smem);
   double(*Xs)[kTileLd] = reinterpret_cast<double(*)[kTileLd]>(jb_smem + kPairRows * kRotLd);
   const int pair = blockIdx.x;
+  const int which = blockIdx.z % matrices;                                  // 0: X, 1: Vt
+  {
+    const int64_t shift = (int64_t)slots.id[blockIdx.z / matrices] * slots.bytes;
+    X = slot_ptr(X, shift);
+    Vt = Vt ? slot_ptr(Vt, shift) : Vt;
+    rot = slot_ptr(rot, shift);
+    flags = slot_ptr(flags, shift);
+  }
   if (flags[pair] == 0) return;
   const BlockPair bp = block_pair(pair, round, nblk);
-  double* M = blockIdx.z ? Vt : X;
+  double* M = which ? Vt : X;
   const int c0 = blockIdx.y * kApplyCols;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
@@ -413,8 +435,10 @@ size_t jacobi_scratch_bytes(int b) {
 }
 
 galore_status_t jacobi_eigh(double* X, double* Vt, int b, void* scratch, int* counter, double tol, int max_sweeps,
-                            int* sweeps_out, cudaStream_t st) {
-  if (sweeps_out) *sweeps_out = 0;
+                            int* sweeps_out, cudaStream_t st, const SlotList* slot_list) {
+  const SlotList all = slot_list ? *slot_list : single_slot();
+  for (int i = 0; i < all.n; ++i)
+    if (sweeps_out) sweeps_out[i] = 0;
   if (b < 2) return GALORE_OK;
   const JacobiGeometry g = jacobi_geometry(b);
   const size_t tile = (size_t)kPairRows * kPairRows * sizeof(double);
@@ -429,24 +453,43 @@ galore_status_t jacobi_eigh(double* X, double* Vt, int b, void* scratch, int* co
   GALORE_CUDA_TRY(cudaFuncSetAttribute(jb_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSweepSmem));
   GALORE_CUDA_TRY(cudaFuncSetAttribute(jb_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kApplySmem));
 
+  // Slots leave the list as they converge (a sweep without a rotation), so every problem sees exactly
+  // the sweeps it would see on its own.
+  SlotList live = all;
+  int where[kMaxSlots];                       // position of live.id[i] in the caller's list
+  for (int i = 0; i < all.n; ++i) where[i] = i;
+  const int matrices = Vt ? 2 : 1;
   int sweeps = 0;
-  while (sweeps < max_sweeps) {
-    GALORE_CUDA_TRY(cudaMemsetAsync(counter, 0, sizeof(int), st));
+  while (sweeps < max_sweeps && live.n > 0) {
+    for (int i = 0; i < live.n; ++i)
+      GALORE_CUDA_TRY(cudaMemsetAsync(slot_ptr(counter, (int64_t)live.id[i] * live.bytes), 0, sizeof(int), st));
     for (int round = 0; round < g.nblk - 1; ++round) {
-      jb_gram_kernel<<<dim3(g.pairs, g.chunks), 128, 0, st>>>(X, b, g.nblk, round, g.chunks, part);
+      jb_gram_kernel<<<dim3(g.pairs, g.chunks, live.n), 128, 0, st>>>(X, b, g.nblk, round, g.chunks, part, live);
       GALORE_LAUNCH_CHECK();
-      jb_sweep_kernel<<<g.pairs, kSweepThreads, kSweepSmem, st>>>(part, g.chunks, b, g.nblk, round, tol, rot, flags, counter);
+      jb_sweep_kernel<<<dim3(g.pairs, live.n), kSweepThreads, kSweepSmem, st>>>(part, g.chunks, b, g.nblk, round, tol, rot, flags,
+                                                                              counter, live);
       GALORE_LAUNCH_CHECK();
-      jb_apply_kernel<<<dim3(g.pairs, g.col_tiles, Vt ? 2 : 1), 256, kApplySmem, st>>>(X, Vt, b, g.nblk, round, rot, flags);
+      jb_apply_kernel<<<dim3(g.pairs, g.col_tiles, matrices * live.n), 256, kApplySmem, st>>>(X, Vt, b, g.nblk, round, rot, flags,
+                                                                                            live, matrices);
       GALORE_LAUNCH_CHECK();
     }
     ++sweeps;
-    int rot_count = 0;
-    GALORE_CUDA_TRY(cudaMemcpyAsync(&rot_count, counter, sizeof(int), cudaMemcpyDeviceToHost, st));
+    int rot_count[kMaxSlots] = {};
+    for (int i = 0; i < live.n; ++i)
+      GALORE_CUDA_TRY(cudaMemcpyAsync(&rot_count[i], slot_ptr(counter, (int64_t)live.id[i] * live.bytes), sizeof(int),
+                                      cudaMemcpyDeviceToHost, st));
     GALORE_CUDA_TRY(cudaStreamSynchronize(st));
-    if (rot_count == 0) break;
+    int kept = 0;
+    for (int i = 0; i < live.n; ++i) {
+      if (sweeps_out) sweeps_out[where[i]] = sweeps;
+      if (rot_count[i] != 0) {
+        live.id[kept] = live.id[i];
+        where[kept] = where[i];
+        ++kept;
+      }
+    }
+    live.n = kept;
   }
-  if (sweeps_out) *sweeps_out = sweeps;
   return GALORE_OK;
 }
 

@@ -15,7 +15,10 @@ size_t jacobi_scratch_bytes(int b);
 //    the eigenvectors as its rows; needed only when eigenvalues near zero matter).
 // counter: one device int used to count rotations per sweep.
 // Synchronises the stream once per sweep.  sweeps_out receives the number of sweeps run.
+// slots: optional list of workspace slots; every pointer argument then names slot 0's copy and the
+// same problem is solved in each listed slot, all slots in one launch per kernel (a slot drops out
+// once it has converged); sweeps_out then has one entry per listed slot.
 galore_status_t jacobi_eigh(double* X, double* Vt, int b, void* scratch, int* counter, double tol, int max_sweeps,
-                            int* sweeps_out, cudaStream_t st);
+                            int* sweeps_out, cudaStream_t st, const SlotList* slots = nullptr);
 
 }  // namespace galore

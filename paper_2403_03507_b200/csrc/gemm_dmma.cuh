@@ -5,7 +5,8 @@
 // Same contract as the FMA kernel of gemm_simt.cuh with a double accumulator: any operand dtype
 // (converted to double while staging), any leading dimension, both transpositions, and every
 // finished element handed to epi(i, j, acc, z).  blockIdx.z selects one problem of a batch whose
-// operands lie `batchA` / `batchB` elements apart.  It carries the fp64 products of the projector
+// operands lie `batchA` / `batchB` elements apart; with a slot list of n entries the grid holds n
+// such batches, batch i with A, B and the epilogue's output shifted by id[i] * bytes.  It carries the fp64 products of the projector
 // refresh (Gram matrices, triangular inverses, Rayleigh-Ritz).
 #pragma once
 
@@ -24,7 +25,7 @@ __device__ __forceinline__ void dmma_m8n8k4(double (&d)[2], double a, double b) 
 template <typename TA, typename TB, int BM, int BN, int WM, int WN, class Epi>
 __global__ void __launch_bounds__((BM / WM) * (BN / WN) * 32)
 gemm_dmma_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int64_t sAk, int64_t batchA,
-                 const TB* __restrict__ B, int64_t sBk, int64_t sBj, int64_t batchB, Epi epi) {
+                 const TB* __restrict__ B, int64_t sBk, int64_t sBj, int64_t batchB, Epi epi_in, const SlotList slots) {
   constexpr int BK = 16;
   constexpr int NT = (BM / WM) * (BN / WN) * 32;
   constexpr int LA = BM * BK / NT, LB = BN * BK / NT;
@@ -39,8 +40,17 @@ gemm_dmma_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int
   const int g = lane >> 2, t = lane & 3;
   const int wm0 = (warp / (BN / WN)) * WM, wn0 = (warp % (BN / WN)) * WN;
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-  A += (int64_t)blockIdx.z * batchA;
-  B += (int64_t)blockIdx.z * batchB;
+  const int inner = gridDim.z / slots.n;
+  const int zi = blockIdx.z % inner;
+  const int64_t shift = (int64_t)slots.id[blockIdx.z / inner] * slots.bytes;
+  Epi epi = epi_in;
+  if (shift) {
+    A = slot_ptr(A, shift);
+    B = slot_ptr(B, shift);
+    epi.shift(shift);
+  }
+  A += (int64_t)zi * batchA;
+  B += (int64_t)zi * batchB;
   const bool a_kfast = (sAk == 1);
   const bool b_kfast = (sBk == 1);
 
@@ -112,8 +122,8 @@ gemm_dmma_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int
 #pragma unroll
     for (int j = 0; j < WN / 8; ++j) {
       const int gj = n0 + wn0 + j * 8 + 2 * t;
-      if (gj < N) epi(gi, gj, acc[i][j][0], (int)blockIdx.z);
-      if (gj + 1 < N) epi(gi, gj + 1, acc[i][j][1], (int)blockIdx.z);
+      if (gj < N) epi(gi, gj, acc[i][j][0], zi);
+      if (gj + 1 < N) epi(gi, gj + 1, acc[i][j][1], zi);
     }
   }
 }
@@ -121,17 +131,19 @@ gemm_dmma_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int
 template <typename TA, typename TB, class Epi>
 galore_status_t launch_gemm_dmma(int M, int N, int K, const TA* A, int64_t sAi, int64_t sAk, const TB* B, int64_t sBk,
                                  int64_t sBj, Epi epi, cudaStream_t stream, int batch = 1, int64_t batchA = 0,
-                                 int64_t batchB = 0) {
+                                 int64_t batchB = 0, const SlotList* slot_list = nullptr) {
   if (M <= 0 || N <= 0 || batch <= 0) return GALORE_OK;
+  const SlotList slots = slot_list ? *slot_list : single_slot();
+  batch *= slots.n;
   const bool small = (int64_t)M * N * batch < (int64_t)128 * 128 * 96;
   if (small) {
     dim3 grid((unsigned)ceil_div(N, 64), (unsigned)ceil_div(M, 64), (unsigned)batch);
     gemm_dmma_kernel<TA, TB, 64, 64, 32, 32, Epi><<<grid, 128, 0, stream>>>(M, N, K, A, sAi, sAk, batchA, B, sBk, sBj,
-                                                                           batchB, epi);
+                                                                           batchB, epi, slots);
   } else {
     dim3 grid((unsigned)ceil_div(N, 128), (unsigned)ceil_div(M, 128), (unsigned)batch);
     gemm_dmma_kernel<TA, TB, 128, 128, 32, 64, Epi><<<grid, 256, 0, stream>>>(M, N, K, A, sAi, sAk, batchA, B, sBk, sBj,
-                                                                             batchB, epi);
+                                                                             batchB, epi, slots);
   }
   GALORE_LAUNCH_CHECK();
   return GALORE_OK;

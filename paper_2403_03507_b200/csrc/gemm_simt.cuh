@@ -9,7 +9,8 @@
 // (where bf16 tensor-core inputs would break the fp32 tolerance) or not
 // TMA-aligned, and all fp64 work of the projector refresh.
 // blockIdx.z selects a K slice of `kchunk` elements (split-K) or, when `batched`, one problem of
-// a batch whose operands lie batchA / batchB elements apart.
+// a batch whose operands lie batchA / batchB elements apart; with a slot list of n entries the grid
+// holds n such groups, group i with A, B and the epilogue's output shifted by id[i] * bytes.
 #pragma once
 
 #include "common.cuh"
@@ -19,8 +20,8 @@ namespace galore {
 template <typename TA, typename TB, typename TAcc, int BM, int BN, int BK, int TM, int TN, class Epi>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN))
 gemm_simt_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int64_t sAk,
-                 const TB* __restrict__ B, int64_t sBk, int64_t sBj, int kchunk, Epi epi, int batched = 0,
-                 int64_t batchA = 0, int64_t batchB = 0) {
+                 const TB* __restrict__ B, int64_t sBk, int64_t sBj, int kchunk, Epi epi_in, int batched,
+                 int64_t batchA, int64_t batchB, const SlotList slots) {
   constexpr int NT = (BM / TM) * (BN / TN);
   constexpr int LA = BM * BK / NT;   // elements of the A tile each thread fetches
   constexpr int LB = BN * BK / NT;
@@ -32,11 +33,20 @@ gemm_simt_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int
   const int tid = threadIdx.x;
   const int tx = tid % (BN / TN), ty = tid / (BN / TN);
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-  const int k_begin = batched ? 0 : blockIdx.z * kchunk;
+  const int inner = gridDim.z / slots.n;
+  const int zi = blockIdx.z % inner;
+  const int64_t shift = (int64_t)slots.id[blockIdx.z / inner] * slots.bytes;
+  Epi epi = epi_in;
+  if (shift) {
+    A = slot_ptr(A, shift);
+    B = slot_ptr(B, shift);
+    epi.shift(shift);
+  }
+  const int k_begin = batched ? 0 : zi * kchunk;
   const int k_end = batched ? K : min(K, k_begin + kchunk);
   if (batched) {
-    A += (int64_t)blockIdx.z * batchA;
-    B += (int64_t)blockIdx.z * batchB;
+    A += (int64_t)zi * batchA;
+    B += (int64_t)zi * batchB;
   }
   const bool a_kfast = (sAk == 1);   // consecutive threads walk the contiguous direction
   const bool b_kfast = (sBk == 1);
@@ -109,7 +119,7 @@ gemm_simt_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int
 #pragma unroll
     for (int v = 0; v < TN; ++v) {
       int j = n0 + (v / 4) * (BN / (TN / 4)) + tx * 4 + (v % 4);
-      if (j < N) epi(i, j, acc[u][v], (int)blockIdx.z);
+      if (j < N) epi(i, j, acc[u][v], zi);
     }
   }
 }
@@ -123,6 +133,7 @@ struct EpiStore {
   int64_t ldc;
   int64_t split_stride;
   TAcc alpha, beta;
+  __device__ __forceinline__ void shift(int64_t bytes) { C = slot_ptr(C, bytes); }
   __device__ __forceinline__ void operator()(int i, int j, TAcc acc, int z) const {
     TC* p = C + (int64_t)z * split_stride + (int64_t)i * ldc + j;
     TAcc v = alpha * acc;
@@ -139,6 +150,7 @@ struct EpiApplyW {
   int64_t ldw;
   float scale;
   float keep = 1.0f;
+  __device__ __forceinline__ void shift(int64_t bytes) { W = slot_ptr(W, bytes); }
   __device__ __forceinline__ void operator()(int i, int j, float acc, int) const {
     TW* p = W + (int64_t)i * ldw + j;
     *p = cvt<TW>(fmaf(-scale, acc, keep * cvt<float>(*p)));
@@ -148,23 +160,24 @@ struct EpiApplyW {
 template <typename TA, typename TB, typename TAcc, class Epi>
 galore_status_t launch_gemm_simt(int M, int N, int K, const TA* A, int64_t sAi, int64_t sAk, const TB* B,
                                  int64_t sBk, int64_t sBj, int splits, Epi epi, cudaStream_t stream, int batch = 0,
-                                 int64_t batchA = 0, int64_t batchB = 0) {
+                                 int64_t batchA = 0, int64_t batchB = 0, const SlotList* slot_list = nullptr) {
   if (M <= 0 || N <= 0) return GALORE_OK;
   if (batch > 0) splits = 1;       // a batch uses blockIdx.z for the problem index
   if (splits < 1) splits = 1;
   int kchunk = (int)ceil_div(ceil_div(K, splits), 16) * 16;
   if (kchunk < 16) kchunk = 16;
   splits = (int)ceil_div(K > 0 ? K : 1, kchunk);
-  const unsigned gz = batch > 0 ? (unsigned)batch : (unsigned)splits;
-  const bool small = (int64_t)M * N * (batch > 0 ? batch : 1) < (int64_t)128 * 128 * 96;
+  const SlotList slots = slot_list ? *slot_list : single_slot();
+  const unsigned gz = (batch > 0 ? (unsigned)batch : (unsigned)splits) * (unsigned)slots.n;
+  const bool small = (int64_t)M * N * (batch > 0 ? batch : 1) * slots.n < (int64_t)128 * 128 * 96;
   if (small) {
     dim3 grid((unsigned)ceil_div(N, 64), (unsigned)ceil_div(M, 64), gz);
     gemm_simt_kernel<TA, TB, TAcc, 64, 64, 16, 4, 4, Epi><<<grid, 256, 0, stream>>>(
-        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi, batch > 0 ? 1 : 0, batchA, batchB);
+        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi, batch > 0 ? 1 : 0, batchA, batchB, slots);
   } else {
     dim3 grid((unsigned)ceil_div(N, 128), (unsigned)ceil_div(M, 128), gz);
     gemm_simt_kernel<TA, TB, TAcc, 128, 128, 16, 8, 8, Epi><<<grid, 256, 0, stream>>>(
-        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi, batch > 0 ? 1 : 0, batchA, batchB);
+        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi, batch > 0 ? 1 : 0, batchA, batchB, slots);
   }
   GALORE_LAUNCH_CHECK();
   return GALORE_OK;

@@ -63,10 +63,12 @@ constexpr long long kWaitLimitCycles = 4000000000LL;   // about two seconds
 // EPI_ADAM_F32 / EPI_ADAM_Q8: the projection with Adam on its output tile (fp32 / 8-bit moments).
 enum { EPI_PARTIAL = 0, EPI_APPLY = 1, EPI_APPLY_DECAY = 2, EPI_ADAM_F32 = 3, EPI_ADAM_Q8 = 4 };
 constexpr bool epi_is_adam(int epi) { return epi == EPI_ADAM_F32 || epi == EPI_ADAM_Q8; }
-// Adam is instruction-heavy (about 70 per element with 8-bit moments): eight epilogue warps, two
-// per quarter of the accumulator's lanes with 128 columns each, keep every scheduler of the SM busy
-// while the tensor cores work on the next tile.
-constexpr int epi_warps(int epi) { return epi_is_adam(epi) ? 8 : 4; }
+// Adam is instruction-heavy (about 70 per element with 8-bit moments) and every element is a chain
+// of dependent lookups and arithmetic: sixteen epilogue warps, four per quarter of the accumulator's
+// lanes with 64 columns each, give every scheduler of the SM four warps to switch between while the
+// tensor cores work on the next tile (eight warps of 128 columns each ran three times longer than
+// the MMAs of a tile).
+constexpr int epi_warps(int epi) { return epi_is_adam(epi) ? 16 : 4; }
 constexpr int epi_threads(int epi) { return 64 + 32 * epi_warps(epi); }     // + producer warp and MMA warp
 constexpr int epi_smem(int epi) { return epi == EPI_ADAM_Q8 ? (int)sizeof(Q8Tables) : 0; }
 
@@ -92,7 +94,7 @@ struct TcParams {
   // EPI_ADAM_*: the state of the layer (rows x cols of the output, row pitch ld_s) and where N goes
   float *Ms, *Vs;             // fp32 moments, or
   uint8_t *Mc, *Vc;           // 8-bit codes with
-  float *Mam, *Vam;           // one absmax per tile of q_rows x 128 state elements, tile (I, J) at I * q_tiles_c + J
+  float *Mam, *Vam;           // one absmax per tile of q_rows x 64 state elements, tile (I, J) at I * q_tiles_c + J
   int64_t ld_s;
   int q_rows, q_tiles_c;
   __nv_bfloat16* Nout;
@@ -380,55 +382,77 @@ __device__ __forceinline__ void epi_apply(const TcParams& p, int row, int col0, 
 
 
 // ---- Adam in the projection's epilogue ----------------------------------------------------------
-// The thread owns row `row` of R and the 128 columns from col0 on (Algorithm 1, the update block on
-// its part of R; Eq. 15 for N).  Rows and columns outside the matrix hold exact zeros in the
-// accumulator (TMA fills out-of-range operand elements with zeros).
+// The thread owns row `row` of R and the kAdamCols columns from col0 on (Algorithm 1, the update
+// block on its part of R; Eq. 15 for N), and walks them kAdamChunk at a time.  Rows and columns
+// outside the matrix hold exact zeros in the accumulator (TMA fills out-of-range operand elements
+// with zeros).
+constexpr int kAdamCols = kStateTileCols;    // 64: columns per epilogue warp = width of a quantisation block
+constexpr int kAdamChunk = 16;
 
-__device__ __forceinline__ void st_n32(__nv_bfloat16* dst, const float (&n)[32], bool vec, int valid) {
+// 32 lanes x 16 consecutive fp32 columns
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+
+// 16 values of N as bf16: one 32-byte store when the row allows it
+__device__ __forceinline__ void st_n16(__nv_bfloat16* dst, const float (&n)[16], bool vec, int valid) {
   if (vec) {
-    uint32_t w[16];
+    uint32_t w[8];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
+    for (int j = 0; j < 8; ++j) {
       const __nv_bfloat162 h = __floats2bfloat162_rn(n[2 * j], n[2 * j + 1]);
       w[j] = *reinterpret_cast<const uint32_t*>(&h);
     }
     st_global_32B(dst, make_uint4(w[0], w[1], w[2], w[3]), make_uint4(w[4], w[5], w[6], w[7]));
-    st_global_32B(dst + 16, make_uint4(w[8], w[9], w[10], w[11]), make_uint4(w[12], w[13], w[14], w[15]));
   } else {
 #pragma unroll
-    for (int j = 0; j < 32; ++j)
+    for (int j = 0; j < 16; ++j)
       if (j < valid) dst[j] = __float2bfloat16_rn(n[j]);
   }
 }
 
-// fp32 moments: one pass, 32 columns at a time
+__device__ __forceinline__ void ld16f(const float* src, float (&x)[16]) {
+#pragma unroll
+  for (int j = 0; j < 16; j += 8) {
+    uint4 a, b;
+    ld_global_32B(src + j, a, b);
+    x[j] = __uint_as_float(a.x); x[j + 1] = __uint_as_float(a.y); x[j + 2] = __uint_as_float(a.z); x[j + 3] = __uint_as_float(a.w);
+    x[j + 4] = __uint_as_float(b.x); x[j + 5] = __uint_as_float(b.y); x[j + 6] = __uint_as_float(b.z); x[j + 7] = __uint_as_float(b.w);
+  }
+}
+__device__ __forceinline__ void st16f(float* dst, const float (&x)[16]) {
+#pragma unroll
+  for (int j = 0; j < 16; j += 8)
+    st_global_32B(dst + j, make_uint4(__float_as_uint(x[j]), __float_as_uint(x[j + 1]), __float_as_uint(x[j + 2]), __float_as_uint(x[j + 3])),
+                  make_uint4(__float_as_uint(x[j + 4]), __float_as_uint(x[j + 5]), __float_as_uint(x[j + 6]), __float_as_uint(x[j + 7])));
+}
+
+// fp32 moments: one pass
 __device__ __forceinline__ bool epi_adam_f32(const TcParams& p, int row, int col0, uint32_t t_addr, uint32_t accf,
                                              uint32_t acc_phase, volatile int* abort_flag, bool& ok) {
   const bool row_ok = row < p.M;
-  const int ncols = row_ok ? max(0, min(128, p.N - col0)) : 0;       // columns of this thread inside the matrix
+  const int ncols = row_ok ? max(0, min(kAdamCols, p.N - col0)) : 0;       // columns of this thread inside the matrix
   const bool vec = p.adam_vec != 0;
   const AdamParams ap = p.ap;
   const int64_t so = (int64_t)row * p.ld_s + col0;
   float* __restrict__ Mrow = p.Ms + so;
   float* __restrict__ Vrow = p.Vs + so;
   __nv_bfloat16* __restrict__ Nrow = p.Nout + (int64_t)row * p.ld_n + col0;
-  float m[32], v[32];
+  float m[kAdamChunk], v[kAdamChunk];
   auto fetch = [&](int c) {
     const int valid = ncols - c;
-    if (valid >= 32 && vec) {
-#pragma unroll
-      for (int j = 0; j < 32; j += 8) {
-        uint4 a, b;
-        ld_global_32B(Mrow + c + j, a, b);
-        m[j] = __uint_as_float(a.x); m[j + 1] = __uint_as_float(a.y); m[j + 2] = __uint_as_float(a.z); m[j + 3] = __uint_as_float(a.w);
-        m[j + 4] = __uint_as_float(b.x); m[j + 5] = __uint_as_float(b.y); m[j + 6] = __uint_as_float(b.z); m[j + 7] = __uint_as_float(b.w);
-        ld_global_32B(Vrow + c + j, a, b);
-        v[j] = __uint_as_float(a.x); v[j + 1] = __uint_as_float(a.y); v[j + 2] = __uint_as_float(a.z); v[j + 3] = __uint_as_float(a.w);
-        v[j + 4] = __uint_as_float(b.x); v[j + 5] = __uint_as_float(b.y); v[j + 6] = __uint_as_float(b.z); v[j + 7] = __uint_as_float(b.w);
-      }
+    if (valid >= kAdamChunk && vec) {
+      ld16f(Mrow + c, m);
+      ld16f(Vrow + c, v);
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
+      for (int j = 0; j < kAdamChunk; ++j) {
         m[j] = j < valid ? Mrow[c + j] : 0.f;
         v[j] = j < valid ? Vrow[c + j] : 0.f;
       }
@@ -440,106 +464,121 @@ __device__ __forceinline__ bool epi_adam_f32(const TcParams& p, int row, int col
   tc_fence_after();
   uint32_t top = 0u;      // largest bit pattern among the new second moments (all >= 0): a non-finite r shows here
 #pragma unroll 1
-  for (int c = 0; c < 128; c += 32) {
+  for (int c = 0; c < kAdamCols; c += kAdamChunk) {
     const int valid = ncols - c;
     if (!__any_sync(0xffffffffu, valid > 0)) break;      // the whole warp is past the last column
     if (c > 0) fetch(c);
-    uint32_t acc[32];
-    tmem_ld_32x32(t_addr + (uint32_t)c, acc);
+    uint32_t acc[kAdamChunk];
+    tmem_ld_32x16(t_addr + (uint32_t)c, acc);
     tmem_ld_wait();
-    float n[32];
+    float n[kAdamChunk];
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
+    for (int j = 0; j < kAdamChunk; ++j) {
       const float r = __uint_as_float(acc[j]);
       m[j] = adam_m(m[j], r, ap);
       v[j] = adam_v(v[j], r, ap);
       n[j] = adam_normalised(m[j], v[j], ap);
       top = max(top, __float_as_uint(v[j]));
     }
-    if (valid >= 32 && vec) {
-#pragma unroll
-      for (int j = 0; j < 32; j += 8) {
-        st_global_32B(Mrow + c + j, make_uint4(__float_as_uint(m[j]), __float_as_uint(m[j + 1]), __float_as_uint(m[j + 2]), __float_as_uint(m[j + 3])),
-                      make_uint4(__float_as_uint(m[j + 4]), __float_as_uint(m[j + 5]), __float_as_uint(m[j + 6]), __float_as_uint(m[j + 7])));
-        st_global_32B(Vrow + c + j, make_uint4(__float_as_uint(v[j]), __float_as_uint(v[j + 1]), __float_as_uint(v[j + 2]), __float_as_uint(v[j + 3])),
-                      make_uint4(__float_as_uint(v[j + 4]), __float_as_uint(v[j + 5]), __float_as_uint(v[j + 6]), __float_as_uint(v[j + 7])));
-      }
+    if (valid >= kAdamChunk && vec) {
+      st16f(Mrow + c, m);
+      st16f(Vrow + c, v);
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
+      for (int j = 0; j < kAdamChunk; ++j)
         if (j < valid) {
           Mrow[c + j] = m[j];
           Vrow[c + j] = v[j];
         }
     }
-    st_n32(Nrow + c, n, valid >= 32 && vec, valid);
+    st_n16(Nrow + c, n, valid >= kAdamChunk && vec, valid);
   }
   return top >= 0x7f800000u;
 }
 
-// 8-bit moments.  A quantisation block is a tile of q_rows x 128 state elements: q_rows lanes of this
+// 32 lanes x 8 consecutive fp32 columns
+__device__ __forceinline__ void tmem_ld_32x8(uint32_t taddr, uint32_t (&v)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(taddr)
+               : "memory");
+}
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// eight old codes of one moment, columns [c, c + 8) of the thread's stretch: one 8-byte load, or byte by
+// byte with the code of zero outside the matrix
+__device__ __forceinline__ uint2 ld_codes8(const uint8_t* row, int c, int ncols, bool vec, uint32_t zero_code) {
+  if (vec) return *reinterpret_cast<const uint2*>(row + c);
+  uint32_t w[2] = {0u, 0u};
+#pragma unroll
+  for (int k = 0; k < 8; ++k) w[k >> 2] |= (c + k < ncols ? (uint32_t)row[c + k] : zero_code) << (8 * (k & 3));
+  return make_uint2(w[0], w[1]);
+}
+
+// 8-bit moments.  A quantisation block is a tile of q_rows x 64 state elements: q_rows lanes of this
 // warp hold all of it, so its absmax is a warp-shuffle reduction.  Two passes over the accumulator:
 // the first finds the block's absmax of the updated moments, the second recomputes them (the same
-// instructions, hence the same bits), writes N and the new codes.
+// instructions, hence the same bits), writes N and the new codes.  Both walk the thread's 64
+// columns eight at a time in loops that are NOT unrolled: sixteen warps at different points of a
+// fully unrolled body (about 5000 instructions) spent most of their time waiting for instruction
+// fetch, and the old codes kept in registers across both passes spilled.  The codes are read once
+// per pass instead, the second time from L2.
 __device__ __forceinline__ bool epi_adam_q8(const TcParams& p, int row, int col0, uint32_t t_addr, uint32_t accf,
                                             uint32_t acc_phase, volatile int* abort_flag, const Q8Tables& t, bool& ok) {
+  constexpr int CH = 8;
   const bool row_ok = row < p.M;
-  const int ncols = row_ok ? max(0, min(128, p.N - col0)) : 0;
-  const bool vec = p.adam_vec != 0 && ncols == 128;
+  const int ncols = row_ok ? max(0, min(kAdamCols, p.N - col0)) : 0;
+  const bool vec = p.adam_vec != 0 && ncols == kAdamCols;
   const AdamParams ap = p.ap;
   const int64_t so = (int64_t)row * p.ld_s + col0;
   uint8_t* __restrict__ Mrow = p.Mc + so;
   uint8_t* __restrict__ Vrow = p.Vc + so;
   __nv_bfloat16* __restrict__ Nrow = p.Nout + (int64_t)row * p.ld_n + col0;
-  const int tile = ncols > 0 ? (row / p.q_rows) * p.q_tiles_c + (col0 >> 7) : 0;
-  // old codes of the thread's 128 elements (zero codes outside the matrix) and the block's old absmax:
-  // none of it depends on the MMAs, so it is in flight while the tile is computed
-  uint32_t cm[32], cv[32];
-  if (vec) {
-#pragma unroll
-    for (int j = 0; j < 32; j += 8) {
-      uint4 a, b;
-      ld_global_32B(Mrow + 4 * j, a, b);
-      cm[j] = a.x; cm[j + 1] = a.y; cm[j + 2] = a.z; cm[j + 3] = a.w; cm[j + 4] = b.x; cm[j + 5] = b.y; cm[j + 6] = b.z; cm[j + 7] = b.w;
-      ld_global_32B(Vrow + 4 * j, a, b);
-      cv[j] = a.x; cv[j + 1] = a.y; cv[j + 2] = a.z; cv[j + 3] = a.w; cv[j + 4] = b.x; cv[j + 5] = b.y; cv[j + 6] = b.z; cv[j + 7] = b.w;
-    }
-  } else {
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-      uint32_t wm = 0u, wv = 0u;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const bool in = 4 * j + k < ncols;
-        wm |= (in ? (uint32_t)Mrow[4 * j + k] : 127u) << (8 * k);
-        wv |= (in ? (uint32_t)Vrow[4 * j + k] : 0u) << (8 * k);
-      }
-      cm[j] = wm;
-      cv[j] = wv;
-    }
+  const int tile = ncols > 0 ? (row / p.q_rows) * p.q_tiles_c + col0 / kAdamCols : 0;
+  // the old codes and the block's old absmax do not depend on the MMAs: asked for now, they arrive
+  // while the tile is computed
+  if (ncols > 0) {
+    prefetch_l2(Mrow);
+    prefetch_l2(Vrow);
   }
   const float am_m = ncols > 0 ? p.Mam[tile] : 0.f, am_v = ncols > 0 ? p.Vam[tile] : 0.f;
   // the decision is taken by the warp as a whole: what follows is warp-synchronous
   if (!__all_sync(0xffffffffu, mbar_wait(accf, acc_phase, abort_flag))) { ok = false; return false; }
   tc_fence_after();
-  if (!__any_sync(0xffffffffu, ncols > 0)) return false;   // the warp's part of the tile lies outside the matrix
+  const int wcols = __reduce_max_sync(0xffffffffu, ncols);       // columns any lane of the warp has
+  if (wcols == 0) return false;                                  // the warp's part of the tile lies outside the matrix
 
+  // Both passes are software-pipelined by one chunk: the next chunk's accumulator columns and old
+  // codes are asked for before the current chunk's arithmetic, which is a chain of dependent
+  // shared-memory lookups per element.
   // ---- pass 1: absmax of the updated moments over the block
   float mx_m = 0.f;
   uint32_t mx_vb = 0u;          // v >= 0: bit order is value order; a NaN or an infinity ends up on top
+  {
+    uint2 nm = ld_codes8(Mrow, 0, ncols, vec, 127u), nv = ld_codes8(Vrow, 0, ncols, vec, 0u);
+    uint32_t nacc[CH];
+    tmem_ld_32x8(t_addr, nacc);
+#pragma unroll 1
+    for (int c = 0; c < wcols; c += CH) {
+      const uint2 cm = nm, cv = nv;
+      uint32_t acc[CH];
+      tmem_ld_wait();
 #pragma unroll
-  for (int c = 0; c < 128; c += 32) {
-    uint32_t acc[32];
-    tmem_ld_32x32(t_addr + (uint32_t)c, acc);
-    tmem_ld_wait();
+      for (int j = 0; j < CH; ++j) acc[j] = nacc[j];
+      if (c + CH < wcols) {
+        tmem_ld_32x8(t_addr + (uint32_t)(c + CH), nacc);
+        nm = ld_codes8(Mrow, c + CH, ncols, vec, 127u);
+        nv = ld_codes8(Vrow, c + CH, ncols, vec, 0u);
+      }
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
-      const float r = __uint_as_float(acc[j]);
-      const uint32_t im = (cm[(c + j) >> 2] >> (8 * (j & 3))) & 0xffu, iv = (cv[(c + j) >> 2] >> (8 * (j & 3))) & 0xffu;
-      const float m = adam_m(__fmul_rn(t.code_s[im], am_m), r, ap);
-      const float v = adam_v(__fmul_rn(t.code_u[iv], am_v), r, ap);
-      mx_m = fmaxf(mx_m, fabsf(m));
-      mx_vb = max(mx_vb, __float_as_uint(v));
+      for (int j = 0; j < CH; ++j) {
+        const float r = __uint_as_float(acc[j]);
+        const uint32_t im = ((j < 4 ? cm.x : cm.y) >> (8 * (j & 3))) & 0xffu, iv = ((j < 4 ? cv.x : cv.y) >> (8 * (j & 3))) & 0xffu;
+        const float m = adam_m(__fmul_rn(t.code_s[im], am_m), r, ap);
+        const float v = adam_v(__fmul_rn(t.code_u[iv], am_v), r, ap);
+        mx_m = fmaxf(mx_m, fabsf(m));
+        mx_vb = max(mx_vb, __float_as_uint(v));
+      }
     }
   }
   for (int o = 1; o < p.q_rows; o <<= 1) {      // the q_rows lanes of the block (a power of two up to 32)
@@ -551,42 +590,77 @@ __device__ __forceinline__ bool epi_adam_q8(const TcParams& p, int row, int col0
   // an all-zero block: with 0 in place of the reciprocal every y' is 0 and takes the code of zero
   const float inv_m = mx_m != 0.f ? 1.0f / mx_m : 0.f, inv_v = mx_v != 0.f ? 1.0f / mx_v : 0.f;
 
-  // ---- pass 2: N and the new codes
+  // ---- pass 2: N and the new codes, eight elements at a time with one (rare) branch to the exact search
+  {
+    uint2 nm = ld_codes8(Mrow, 0, ncols, vec, 127u), nv = ld_codes8(Vrow, 0, ncols, vec, 0u);
+    uint32_t nacc[CH];
+    tmem_ld_32x8(t_addr, nacc);
+#pragma unroll 1
+    for (int c = 0; c < wcols; c += CH) {
+      const uint2 cm = nm, cv = nv;
+      uint32_t acc[CH];
+      tmem_ld_wait();
 #pragma unroll
-  for (int c = 0; c < 128; c += 32) {
-    uint32_t acc[32];
-    if (!__any_sync(0xffffffffu, ncols - c > 0)) break;  // the whole warp is past the last column
-    tmem_ld_32x32(t_addr + (uint32_t)c, acc);
-    tmem_ld_wait();
-    float n[32];
-    uint32_t pm[8], pv[8];
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      float xm[4], xv[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int j = 4 * q + k;
-        const float r = __uint_as_float(acc[j]);
-        const uint32_t im = (cm[(c + j) >> 2] >> (8 * k)) & 0xffu, iv = (cv[(c + j) >> 2] >> (8 * k)) & 0xffu;
-        xm[k] = adam_m(__fmul_rn(t.code_s[im], am_m), r, ap);
-        xv[k] = adam_v(__fmul_rn(t.code_u[iv], am_v), r, ap);
-        n[j] = adam_normalised(xm[k], xv[k], ap);
+      for (int j = 0; j < CH; ++j) acc[j] = nacc[j];
+      if (c + CH < wcols) {
+        tmem_ld_32x8(t_addr + (uint32_t)(c + CH), nacc);
+        nm = ld_codes8(Mrow, c + CH, ncols, vec, 127u);
+        nv = ld_codes8(Vrow, c + CH, ncols, vec, 0u);
       }
-      pm[q] = q8_encode4<true>(xm, mx_m, inv_m, t.enc_s, t.mid_s);
-      pv[q] = q8_encode4<false>(xv, mx_v, inv_v, t.enc_u, t.mid_u);
-    }
-    if (vec) {
-      st_global_32B(Mrow + c, make_uint4(pm[0], pm[1], pm[2], pm[3]), make_uint4(pm[4], pm[5], pm[6], pm[7]));
-      st_global_32B(Vrow + c, make_uint4(pv[0], pv[1], pv[2], pv[3]), make_uint4(pv[4], pv[5], pv[6], pv[7]));
-    } else {
+      float xm[CH], xv[CH];
+      uint32_t nw[CH / 2];
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (c + j < ncols) {
-          Mrow[c + j] = (uint8_t)(pm[j >> 2] >> (8 * (j & 3)));
-          Vrow[c + j] = (uint8_t)(pv[j >> 2] >> (8 * (j & 3)));
+      for (int j = 0; j < CH; j += 2) {
+        float n[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          const int e = j + k;
+          const float r = __uint_as_float(acc[e]);
+          const uint32_t im = ((e < 4 ? cm.x : cm.y) >> (8 * (e & 3))) & 0xffu, iv = ((e < 4 ? cv.x : cv.y) >> (8 * (e & 3))) & 0xffu;
+          xm[e] = adam_m(__fmul_rn(t.code_s[im], am_m), r, ap);
+          xv[e] = adam_v(__fmul_rn(t.code_u[iv], am_v), r, ap);
+          n[k] = adam_normalised(xm[e], xv[e], ap);
         }
+        const __nv_bfloat162 h = __floats2bfloat162_rn(n[0], n[1]);
+        nw[j >> 1] = *reinterpret_cast<const uint32_t*>(&h);
+      }
+      uint32_t pm[2] = {0u, 0u}, pv[2] = {0u, 0u}, need = 0u;     // need: bit e for M value e, bit 8 + e for V value e
+#pragma unroll
+      for (int e = 0; e < CH; ++e) {
+        bool ex_m, ex_v;
+        const uint32_t km = q8_encode_fast<true>(xm[e], inv_m, t.enc_s, ex_m) & 0xffu;
+        const uint32_t kv = q8_encode_fast<false>(xv[e], inv_v, t.enc_u, ex_v) & 0xffu;
+        pm[e >> 2] |= km << (8 * (e & 3));
+        pv[e >> 2] |= kv << (8 * (e & 3));
+        need |= ((ex_m ? 1u : 0u) << e) | ((ex_v ? 1u : 0u) << (8 + e));
+      }
+      if (need != 0u) {                         // about one value in 4000: the quotient by IEEE division, searched exactly
+#pragma unroll
+        for (int e = 0; e < CH; ++e) {
+          if (need & (1u << e)) {
+            const uint32_t k = (uint32_t)q8_encode(__fdiv_rn(xm[e], mx_m), t.mid_s) & 0xffu;
+            pm[e >> 2] = (pm[e >> 2] & ~(0xffu << (8 * (e & 3)))) | (k << (8 * (e & 3)));
+          }
+          if (need & (0x100u << e)) {
+            const uint32_t k = (uint32_t)q8_encode(__fdiv_rn(xv[e], mx_v), t.mid_u) & 0xffu;
+            pv[e >> 2] = (pv[e >> 2] & ~(0xffu << (8 * (e & 3)))) | (k << (8 * (e & 3)));
+          }
+        }
+      }
+      if (vec) {
+        *reinterpret_cast<uint2*>(Mrow + c) = make_uint2(pm[0], pm[1]);
+        *reinterpret_cast<uint2*>(Vrow + c) = make_uint2(pv[0], pv[1]);
+        *reinterpret_cast<uint4*>(Nrow + c) = make_uint4(nw[0], nw[1], nw[2], nw[3]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < CH; ++j)
+          if (c + j < ncols) {
+            Mrow[c + j] = (uint8_t)(pm[j >> 2] >> (8 * (j & 3)));
+            Vrow[c + j] = (uint8_t)(pv[j >> 2] >> (8 * (j & 3)));
+            reinterpret_cast<uint16_t*>(Nrow)[c + j] = (uint16_t)(nw[j >> 1] >> (16 * (j & 1)));
+          }
+      }
     }
-    st_n32(Nrow + c, n, vec, ncols - c);
   }
   if (ncols > 0 && (row % p.q_rows) == 0) {     // the first lane of each block stores its absmax
     p.Mam[tile] = mx_m;
@@ -769,14 +843,14 @@ gemm_tc_kernel(const __grid_constant__ TcGroup g) {
       const int row = w.m0 + (int)rank * kBM + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kBN);
       if constexpr (epi_is_adam(EPI)) {
-        // warps 2..5 take the first 128 columns of the tile, warps 6..9 the other 128
-        const int half = (warp - 2) >> 2;
-        const int col0 = w.n0 + half * 128;
+        // warps 2..5 take the first 64 columns of the tile, warps 6..9 the next 64, and so on
+        const int part = (warp - 2) >> 2;
+        const int col0 = w.n0 + part * kAdamCols;
         bool bad;
         if constexpr (EPI == EPI_ADAM_F32)
-          bad = epi_adam_f32(p, row, col0, t_row + (uint32_t)(half * 128), accf_bar(acc), acc_phase, abort_flag, ok);
+          bad = epi_adam_f32(p, row, col0, t_row + (uint32_t)(part * kAdamCols), accf_bar(acc), acc_phase, abort_flag, ok);
         else
-          bad = epi_adam_q8(p, row, col0, t_row + (uint32_t)(half * 128), accf_bar(acc), acc_phase, abort_flag, *q8t, ok);
+          bad = epi_adam_q8(p, row, col0, t_row + (uint32_t)(part * kAdamCols), accf_bar(acc), acc_phase, abort_flag, *q8t, ok);
         if (!ok) break;
         if (bad) atomicOr(p.status, GALORE_DEV_NONFINITE);
       } else if (EPI != EPI_PARTIAL && w.n0 + kBN <= p.N) {
@@ -1103,7 +1177,7 @@ static galore_status_t project_problem(const TensorPlan* plan, const galore_conf
 // the Adam part of a projection problem
 static galore_status_t set_adam(TcParams* p, const TcAdamArgs& a) {
   if (a.state_fmt == GALORE_STATE_Q8_BLOCK &&
-      (a.q_block < 256 || a.q_block > 4096 || (a.q_block & (a.q_block - 1)) != 0)) return GALORE_ERR_INVALID_ARG;
+      (a.q_block < 256 || a.q_block > 2048 || (a.q_block & (a.q_block - 1)) != 0)) return GALORE_ERR_INVALID_ARG;
   p->Ms = a.M; p->Vs = a.V; p->Mc = a.Mc; p->Vc = a.Vc; p->Mam = a.Mam; p->Vam = a.Vam;
   p->ld_s = a.ld_s;
   p->q_rows = a.q_block / kStateTileCols;
@@ -1111,8 +1185,8 @@ static galore_status_t set_adam(TcParams* p, const TcAdamArgs& a) {
   p->Nout = (__nv_bfloat16*)a.Nout;
   p->ld_n = a.ld_n;
   p->ap = a.ap;
-  // 32-byte accesses: per thread 128 bytes of codes or 128-byte runs of fp32 moments and 64-byte runs of N,
-  // all starting at multiples of 128 columns
+  // 32-byte accesses (16 for the code stores): per thread 64 bytes of codes, 64-byte runs of fp32 moments and
+  // 32-byte runs of N, all starting at multiples of 16 columns
   const uintptr_t bases = (uintptr_t)a.Nout | (uintptr_t)a.M | (uintptr_t)a.V | (uintptr_t)a.Mc | (uintptr_t)a.Vc;
   const int64_t s_bytes = a.ld_s * (a.state_fmt == GALORE_STATE_F32 ? 4 : 1);
   p->adam_vec = ((bases & 31) == 0 && (s_bytes % 32) == 0 && (a.ld_n % 16) == 0) ? 1 : 0;

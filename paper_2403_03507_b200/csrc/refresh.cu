@@ -218,9 +218,16 @@ __global__ void split_kernel(const float* __restrict__ x, __nv_bfloat16* __restr
 __device__ __forceinline__ double pivot_rsqrt(double x) { return rsqrt_newton(x); }
 __device__ __forceinline__ float pivot_rsqrt(float x) { return rsqrtf(x); }
 
+// blockIdx.x: position in the slot list (one CTA per workspace slot)
 template <typename T>
 __global__ void __launch_bounds__(256) potf2_inv_kernel(T* __restrict__ C, int ld, int nb, T* __restrict__ Linv,
-                                                        int32_t* __restrict__ status) {
+                                                        int32_t* __restrict__ status, const SlotList slots) {
+  {
+    const int64_t shift = (int64_t)slots.id[blockIdx.x] * slots.bytes;
+    C = slot_ptr(C, shift);
+    Linv = slot_ptr(Linv, shift);
+    status = slot_ptr(status, shift);
+  }
   __shared__ T Ls[64][65];       // the factor: needed again for the inverse and for the write-back
   __shared__ T col[64];
   __shared__ T rdiag[64];
@@ -290,7 +297,12 @@ __global__ void __launch_bounds__(256) potf2_inv_kernel(T* __restrict__ C, int l
 
 // diagonal 64 x 64 blocks of T <- the inverses of the diagonal blocks of L (slab p = block p)
 template <typename S>
-__global__ void place_diag_inverse_kernel(const S* __restrict__ slabs, int b, S* __restrict__ T) {
+__global__ void place_diag_inverse_kernel(const S* __restrict__ slabs, int b, S* __restrict__ T, const SlotList slots) {
+  {
+    const int64_t shift = (int64_t)slots.id[blockIdx.y] * slots.bytes;     // blockIdx.y: workspace slot
+    slabs = slot_ptr(slabs, shift);
+    T = slot_ptr(T, shift);
+  }
   const int p = blockIdx.x, j0 = p * 64;
   const int nb = min(64, b - j0);
   for (int idx = threadIdx.x; idx < 64 * 64; idx += blockDim.x) {
@@ -371,10 +383,20 @@ __global__ void __launch_bounds__(256) residual_pair_kernel(const float* __restr
 struct EpiSplitPair {
   __nv_bfloat16 *hi, *lo;
   int64_t ld;
+  __device__ __forceinline__ void shift(int64_t bytes) {
+    hi = slot_ptr(hi, bytes);
+    lo = slot_ptr(lo, bytes);
+  }
   __device__ __forceinline__ void operator()(int i, int j, double acc, int) const {
     split_bf16((float)acc, hi[(int64_t)i * ld + j], lo[(int64_t)i * ld + j]);
   }
 };
+
+// status |= flags; flags = 0  (what the slot-wise kernels latched goes to the layer's own status word)
+__global__ void merge_flags_kernel(int32_t* __restrict__ status, int32_t* __restrict__ flags) {
+  if (*flags) atomicOr(status, *flags);
+  *flags = 0;
+}
 
 static inline unsigned grid_for(int64_t count) { return (unsigned)std::min<int64_t>(ceil_div(count, 256), 148 * 8); }
 
@@ -400,6 +422,7 @@ struct RefreshBuffers {
   double* scal;   // 4 scalars
   double* part;   // kSumsqBlocks partial sums
   int* counter;   // 1
+  int32_t* flags; // device status bits latched by kernels that run for several slots at once
   void* jac;      // scratch of the Jacobi eigensolver
   double* slabs;  // ceil(b / 64) inverses of 64 x 64 diagonal blocks
   // tensor-core power steps
@@ -454,7 +477,7 @@ static RefreshBuffers layout(void* base, int64_t d, int64_t L, int r, int b) {
   w.order = (int*)p; carve(p, (size_t)b * 4);
   w.scal = (double*)p; carve(p, 256);
   w.part = (double*)p; carve(p, 8 * 1024);
-  w.counter = (int*)p; carve(p, 256);
+  w.counter = (int*)p; w.flags = (int32_t*)(p + 64); carve(p, 256);
   w.jac = (void*)p; carve(p, jacobi_scratch_bytes(b));
   w.slabs = (double*)p; carve(p, (size_t)ceil_div(b, 64) * 4096 * 8);
   w.Yc = (float*)p; carve(p, (size_t)d * b * 4);
@@ -472,57 +495,136 @@ const double* refresh_unrounded_projector(void* workspace, int64_t d, int64_t L,
 }
 
 // ---------------------------------------------------------------------------
-// building blocks
+// A group of layers of one shape refreshed together
 // ---------------------------------------------------------------------------
+// Each layer ("lane") owns one slot of the workspace, all slots laid out alike.  The tensor-core
+// products take the lanes' problems in one grouped launch; the latency-bound small kernels
+// (Cholesky panels, triangular inverses, the Jacobi eigen-solver) run for all lanes in one launch
+// per kernel, their workspace pointers shifted per slot; element-wise kernels and everything that
+// touches a layer's own G or P are launched lane by lane.  Every lane makes exactly the steps it
+// would make on its own (its own iteration count and orthonormalisation schedule), so a layer's
+// projector does not depend on what it was grouped with.
 
-// C (b x b, fp64) = Y^T Y
-template <typename TY>
-static galore_status_t gram(const TY* Y, int64_t d, int b, double* C, cudaStream_t st) {
-  EpiStore<double, double> epi{C, b, 0, 1.0, 0.0};
-  return launch_gemm_dmma<TY, TY>(b, b, (int)d, Y, 1, b, Y, b, 1, epi, st);
+struct TensorRefresh {
+  float* F[3];          // fp32 d x b buffers; F[master] holds Y
+  int master;
+};
+
+struct Lane {
+  RefreshProblem pr;
+  int slot;
+  char* base;                 // start of the lane's slot
+  RefreshBuffers w;
+  int32_t* status;            // the layer's own status word
+  float *Y, *Yn;              // current block and the other buffer (FMA path)
+  TensorRefresh tr;
+  int q_done = 0, q_target = 0, orth_every = 1;
+  std::vector<double> theta;
+  double predicted = 0.0;
+  bool converged = false, with_vt = false, iterating = true;
+  galore_refresh_info_t info = {};
+};
+
+struct Ctx {
+  char* base0;                // slot 0 of the workspace
+  int64_t slot_bytes;
+  int64_t d, L;
+  int r, b;
+  bool left, tensor;
+  RefreshBuffers w0;          // slot 0's buffers: what a launch over a slot list is given
+  TensorGroup* tg;
+  cudaStream_t st;
+};
+
+// lanes whose pointers sit at the same place inside their slots can share a launch
+struct LaneSet {
+  int64_t off_a, off_b;
+  SlotList list;
+  std::vector<Lane*> lanes;
+};
+template <class KeyA, class KeyB>
+static std::vector<LaneSet> sets_of(const Ctx& c, const std::vector<Lane*>& lanes, KeyA a_of, KeyB b_of) {
+  std::vector<LaneSet> out;
+  for (Lane* l : lanes) {
+    const int64_t oa = (const char*)a_of(l) - l->base, ob = (const char*)b_of(l) - l->base;
+    LaneSet* g = nullptr;
+    for (LaneSet& x : out)
+      if (x.off_a == oa && x.off_b == ob) g = &x;
+    if (!g) {
+      out.push_back(LaneSet{});
+      g = &out.back();
+      g->off_a = oa;
+      g->off_b = ob;
+      g->list = SlotList{};
+      g->list.bytes = c.slot_bytes;
+    }
+    g->list.id[g->list.n++] = l->slot;
+    g->lanes.push_back(l);
+  }
+  return out;
+}
+static SlotList slots_of(const Ctx& c, const std::vector<Lane*>& lanes) {
+  SlotList s = {};
+  s.bytes = c.slot_bytes;
+  for (Lane* l : lanes) s.id[s.n++] = l->slot;
+  return s;
+}
+
+// C (b x b, fp64, at `dst` of slot 0) = Y^T Y, Y (rows x b) at src(lane)
+template <typename TY, class Src>
+static galore_status_t gram(const Ctx& c, const std::vector<Lane*>& lanes, Src src, int64_t rows, double* dst0) {
+  for (const LaneSet& g : sets_of(c, lanes, src, src)) {
+    const TY* Y0 = (const TY*)(c.base0 + g.off_a);
+    EpiStore<double, double> epi{dst0, c.b, 0, 1.0, 0.0};
+    GALORE_TRY((launch_gemm_dmma<TY, TY>(c.b, c.b, (int)rows, Y0, 1, c.b, Y0, c.b, 1, epi, c.st, 1, 0, 0, &g.list)));
+  }
+  return GALORE_OK;
 }
 
 // Blocked Cholesky of the b x b matrix C (lower triangle, in place), then T = L^-1 (b x b, lower,
-// zero above the diagonal).
+// zero above the diagonal), in every listed slot; pointers name slot 0's copies.
 //   factor : per 64-wide panel the diagonal block (with its inverse, kept in w.slabs), the panel
 //            below it and the trailing update;
 //   invert : the inverses of the diagonal blocks are merged pairwise, level by level,
 //            [T11 0; T21 T22] with T21 = -T22 L21 T11, every level two batched products.
-// scratch: b*b/4 doubles.
+// scratch: b*b/4 elements.
 // (S = double: products on the fp64 MMA unit; S = float, used between the tensor-core power steps
 // whose Gram matrices carry about 16 bits anyway: FMA products and a ten times shorter pivot chain.)
 template <typename TA, typename TB, typename S, class Epi>
 static galore_status_t gemm_scalar(int M, int N, int K, const TA* A, int64_t sAi, int64_t sAk, const TB* B, int64_t sBk,
-                                   int64_t sBj, Epi epi, cudaStream_t st, int batch = 1, int64_t bA = 0, int64_t bB = 0) {
+                                   int64_t sBj, Epi epi, cudaStream_t st, const SlotList& sl, int batch = 1, int64_t bA = 0,
+                                   int64_t bB = 0) {
   if constexpr (std::is_same<S, double>::value)
-    return launch_gemm_dmma<TA, TB>(M, N, K, A, sAi, sAk, B, sBk, sBj, epi, st, batch, bA, bB);
+    return launch_gemm_dmma<TA, TB>(M, N, K, A, sAi, sAk, B, sBk, sBj, epi, st, batch, bA, bB, &sl);
   else
-    return launch_gemm_simt<TA, TB, float>(M, N, K, A, sAi, sAk, B, sBk, sBj, 1, epi, st, batch, bA, bB);
+    return launch_gemm_simt<TA, TB, float>(M, N, K, A, sAi, sAk, B, sBk, sBj, 1, epi, st, batch, bA, bB, &sl);
 }
 
 template <typename S>
-static galore_status_t cholesky_inverse(S* C, int b, S* T, S* scratch, const RefreshBuffers& w, int32_t* status,
-                                        cudaStream_t st) {
+static galore_status_t cholesky_inverse(const Ctx& c, const SlotList& sl, S* C, S* T, S* scratch) {
+  const int b = c.b;
+  cudaStream_t st = c.st;
   const int nblk = (int)ceil_div(b, 64);
-  S* slabs = (S*)w.slabs;
+  S* slabs = (S*)c.w0.slabs;
   for (int p = 0; p < nblk; ++p) {
     const int j0 = p * 64, nb = std::min(64, b - j0), j1 = j0 + nb;
     S* slab = slabs + (int64_t)p * 4096;
-    potf2_inv_kernel<S><<<1, 256, 0, st>>>(C + (int64_t)j0 * b + j0, b, nb, slab, status);
+    potf2_inv_kernel<S><<<sl.n, 256, 0, st>>>(C + (int64_t)j0 * b + j0, b, nb, slab, c.w0.flags, sl);
     GALORE_LAUNCH_CHECK();
     if (j1 < b) {
       const int rem = b - j1;
       S* panel = C + (int64_t)j1 * b + j0;
       // L[rest, J] = C[rest, J] Linv^T   (in place: one CTA column covers all nb columns)
       EpiStore<S, S> epi{panel, b, 0, S(1), S(0)};
-      GALORE_TRY((gemm_scalar<S, S, S>(rem, nb, nb, panel, b, 1, slab, 1, 64, epi, st)));
+      GALORE_TRY((gemm_scalar<S, S, S>(rem, nb, nb, panel, b, 1, slab, 1, 64, epi, st, sl)));
       // C[rest, rest] -= L[rest, J] L[rest, J]^T
       EpiStore<S, S> upd{C + (int64_t)j1 * b + j1, b, 0, S(-1), S(1)};
-      GALORE_TRY((gemm_scalar<S, S, S>(rem, rem, nb, panel, b, 1, panel, 1, b, upd, st)));
+      GALORE_TRY((gemm_scalar<S, S, S>(rem, rem, nb, panel, b, 1, panel, 1, b, upd, st, sl)));
     }
   }
-  GALORE_CUDA_TRY(cudaMemsetAsync(T, 0, sizeof(S) * b * b, st));
-  place_diag_inverse_kernel<S><<<nblk, 256, 0, st>>>(slabs, b, T);
+  for (int i = 0; i < sl.n; ++i)
+    GALORE_CUDA_TRY(cudaMemsetAsync(slot_ptr(T, (int64_t)sl.id[i] * sl.bytes), 0, sizeof(S) * b * b, st));
+  place_diag_inverse_kernel<S><<<dim3(nblk, sl.n), 256, 0, st>>>(slabs, b, T, sl);
   GALORE_LAUNCH_CHECK();
   for (int64_t s = 64; s < b; s *= 2) {
     const int64_t step = 2 * s * b + 2 * s;            // from one merged block to the next, in elements
@@ -539,339 +641,478 @@ static galore_status_t cholesky_inverse(S* C, int b, S* T, S* scratch, const Ref
       S* T21 = T + (o + s) * b + o;
       // W = L21 T11
       EpiStore<S, S> ew{scratch, s, s * s, S(1), S(0)};
-      GALORE_TRY((gemm_scalar<S, S, S>(s2, (int)s, (int)s, L21, b, 1, T11, b, 1, ew, st, count, step, step)));
+      GALORE_TRY((gemm_scalar<S, S, S>(s2, (int)s, (int)s, L21, b, 1, T11, b, 1, ew, st, sl, count, step, step)));
       // T21 = -T22 W
       EpiStore<S, S> et{T21, b, step, S(-1), S(0)};
-      GALORE_TRY((gemm_scalar<S, S, S>(s2, (int)s, s2, T22, b, 1, scratch, s, 1, et, st, count, step, s * s)));
+      GALORE_TRY((gemm_scalar<S, S, S>(s2, (int)s, s2, T22, b, 1, scratch, s, 1, et, st, sl, count, step, s * s)));
     }
   }
   return GALORE_OK;
 }
 
-// out = Y L^-T with L L^T = Y^T Y (CholeskyQR); out must not alias Y.  Uses w.C, w.Vt, w.H.
-template <typename TY, typename TO>
-static galore_status_t orthonormalise(const TY* Y, TO* out, int64_t d, int b, const RefreshBuffers& w, int32_t* status,
-                                      cudaStream_t st) {
-  GALORE_TRY(gram(Y, d, b, w.C, st));
-  GALORE_TRY(cholesky_inverse<double>(w.C, b, w.Vt, w.H, w, status, st));
-  EpiStore<TO, double> epi{out, b, 0, 1.0, 0.0};
-  return launch_gemm_dmma<TY, double>((int)d, b, b, Y, b, 1, w.Vt, 1, b, epi, st);
+// out = Y L^-T with L L^T = Y^T Y (CholeskyQR), Y at src(lane), out at dst(lane); out must not alias Y.
+// Uses C, Vt, H of every lane.
+template <typename TY, typename TO, class Src, class Dst>
+static galore_status_t orthonormalise(const Ctx& c, const std::vector<Lane*>& lanes, Src src, Dst dst) {
+  GALORE_TRY((gram<TY>(c, lanes, src, c.d, c.w0.C)));
+  GALORE_TRY(cholesky_inverse<double>(c, slots_of(c, lanes), c.w0.C, c.w0.Vt, c.w0.H));
+  for (const LaneSet& g : sets_of(c, lanes, src, dst)) {
+    EpiStore<TO, double> epi{(TO*)(c.base0 + g.off_b), c.b, 0, 1.0, 0.0};
+    GALORE_TRY((launch_gemm_dmma<TY, double>((int)c.d, c.b, c.b, (const TY*)(c.base0 + g.off_a), c.b, 1, c.w0.Vt, 1, c.b, epi,
+                                             c.st, 1, 0, 0, &g.list)));
+  }
+  return GALORE_OK;
 }
 
 // ---- power step on the tensor cores -------------------------------------------------------------
 // The block Y lives as an fp32 master (one of three d x b buffers) plus its bf16 hi/lo pair.  Every
 // product below is a tcgen05 GEMM on bf16 operands with fp32 output; a product with a hi/lo operand
-// is two (or three) problems of one grouped launch whose outputs are added afterwards.
-
-struct TensorRefresh {
-  TensorGroup* tg;
-  float* F[3];          // fp32 d x b buffers; F[master] holds Y
-  int master;
-  int32_t* status;
-};
+// is two (or three) problems of one grouped launch whose outputs are added afterwards.  The
+// problems of all lanes travel in the same grouped launches.
 
 // Y <- Y L^-T with L L^T = Y^T Y: CholeskyQR whose two big products run on the tensor cores.
 // In: hi/lo pair of Y valid (the fp32 master itself is not read).  Out: master and pair updated.
-static galore_status_t orth_tensor(TensorRefresh& t, const RefreshBuffers& w, int64_t d, int b, cudaStream_t st) {
-  const int64_t bb = (int64_t)b * b, yb = d * b;
-  float* g0 = (float*)w.H;
-  float* g1 = g0 + bb;
-  float* g2 = (float*)w.Y64;
-  tensor_group_reset(t.tg);   // Gram = (hi + lo)^T (hi + lo) without the lo^T lo term
-  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 1, w.Yhi, b, 1, b, b, (int)d, g0, b, t.status));
-  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 1, w.Ylo, b, 1, b, b, (int)d, g1, b, t.status));
-  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Ylo, b, 1, w.Yhi, b, 1, b, b, (int)d, g2, b, t.status));
-  GALORE_TRY(tensor_group_launch_project(t.tg, st));
-  gram_sum_kernel<<<grid_for(bb), 256, 0, st>>>(g0, g1, g2, (float*)w.C, bb);
-  GALORE_LAUNCH_CHECK();
+static galore_status_t orth_tensor(const Ctx& c, const std::vector<Lane*>& lanes) {
+  if (lanes.empty()) return GALORE_OK;
+  const int b = c.b;
+  const int64_t d = c.d, bb = (int64_t)b * b, yb = d * b;
+  cudaStream_t st = c.st;
+  tensor_group_reset(c.tg);   // Gram = (hi + lo)^T (hi + lo) without the lo^T lo term
+  for (Lane* l : lanes) {
+    const RefreshBuffers& w = l->w;
+    float* g0 = (float*)w.H;
+    float* g1 = g0 + bb;
+    float* g2 = (float*)w.Y64;
+    GALORE_TRY(tensor_group_add_gemm(c.tg, w.Yhi, b, 1, w.Yhi, b, 1, b, b, (int)d, g0, b, l->status));
+    GALORE_TRY(tensor_group_add_gemm(c.tg, w.Yhi, b, 1, w.Ylo, b, 1, b, b, (int)d, g1, b, l->status));
+    GALORE_TRY(tensor_group_add_gemm(c.tg, w.Ylo, b, 1, w.Yhi, b, 1, b, b, (int)d, g2, b, l->status));
+  }
+  GALORE_TRY(tensor_group_launch_project(c.tg, st));
+  for (Lane* l : lanes) {
+    const RefreshBuffers& w = l->w;
+    gram_sum_kernel<<<grid_for(bb), 256, 0, st>>>((float*)w.H, (float*)w.H + bb, (float*)w.Y64, (float*)w.C, bb);
+    GALORE_LAUNCH_CHECK();
+  }
   // T = L^-1, split into a bf16 pair; as the second operand of Y L^-T it is read K-contiguous
-  GALORE_TRY(cholesky_inverse<float>((float*)w.C, b, (float*)w.Vt, (float*)w.H, w, t.status, st));
-  split_kernel<<<grid_for(bb), 256, 0, st>>>((const float*)w.Vt, w.Thi, w.Tlo, bb);
-  GALORE_LAUNCH_CHECK();
-  const int m = t.master, s1 = (m + 1) % 3, s2 = (m + 2) % 3;
-  tensor_group_reset(t.tg);   // Y T = hi Thi + hi Tlo + lo Thi
-  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 0, w.Thi, b, 0, (int)d, b, b, t.F[m], b, t.status));
-  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Yhi, b, 0, w.Tlo, b, 0, (int)d, b, b, t.F[s1], b, t.status));
-  GALORE_TRY(tensor_group_add_gemm(t.tg, w.Ylo, b, 0, w.Thi, b, 0, (int)d, b, b, t.F[s2], b, t.status));
-  GALORE_TRY(tensor_group_launch_project(t.tg, st));
-  sum_split_kernel<<<grid_for(yb), 256, 0, st>>>(t.F[m], t.F[s1], t.F[s2], t.F[m], w.Yhi, w.Ylo, yb);
-  GALORE_LAUNCH_CHECK();
+  GALORE_TRY(cholesky_inverse<float>(c, slots_of(c, lanes), (float*)c.w0.C, (float*)c.w0.Vt, (float*)c.w0.H));
+  for (Lane* l : lanes) {
+    split_kernel<<<grid_for(bb), 256, 0, st>>>((const float*)l->w.Vt, l->w.Thi, l->w.Tlo, bb);
+    GALORE_LAUNCH_CHECK();
+  }
+  tensor_group_reset(c.tg);   // Y T = hi Thi + hi Tlo + lo Thi
+  for (Lane* l : lanes) {
+    const RefreshBuffers& w = l->w;
+    TensorRefresh& t = l->tr;
+    const int m = t.master, s1 = (m + 1) % 3, s2 = (m + 2) % 3;
+    GALORE_TRY(tensor_group_add_gemm(c.tg, w.Yhi, b, 0, w.Thi, b, 0, (int)d, b, b, t.F[m], b, l->status));
+    GALORE_TRY(tensor_group_add_gemm(c.tg, w.Yhi, b, 0, w.Tlo, b, 0, (int)d, b, b, t.F[s1], b, l->status));
+    GALORE_TRY(tensor_group_add_gemm(c.tg, w.Ylo, b, 0, w.Thi, b, 0, (int)d, b, b, t.F[s2], b, l->status));
+  }
+  GALORE_TRY(tensor_group_launch_project(c.tg, st));
+  for (Lane* l : lanes) {
+    TensorRefresh& t = l->tr;
+    const int m = t.master, s1 = (m + 1) % 3, s2 = (m + 2) % 3;
+    sum_split_kernel<<<grid_for(yb), 256, 0, st>>>(t.F[m], t.F[s1], t.F[s2], t.F[m], l->w.Yhi, l->w.Ylo, yb);
+    GALORE_LAUNCH_CHECK();
+  }
   return GALORE_OK;
 }
 
-// Z = A^T Y ; Y' = A Z + delta Y ; Y = orth(Y')
-static galore_status_t power_step_tensor(TensorRefresh& t, const RefreshProblem& pr, const RefreshBuffers& w, int64_t d,
-                                         int64_t L, int b, bool orth, cudaStream_t st) {
-  const int64_t zb = L * b, yb = d * b;
-  float* z0 = (float*)w.Zu;
-  float* z1 = z0 + zb;
-  const int at_mn = pr.left ? 1 : 0;   // A^T as the first operand: G^T (left) is M-contiguous in G, G (right) is K-contiguous
-  const int a_mn = pr.left ? 0 : 1;    // A as the first operand
-  tensor_group_reset(t.tg);
-  GALORE_TRY(tensor_group_add_gemm(t.tg, pr.G, pr.ldg, at_mn, w.Yhi, b, 1, (int)L, b, (int)d, z0, b, t.status));
-  GALORE_TRY(tensor_group_add_gemm(t.tg, pr.G, pr.ldg, at_mn, w.Ylo, b, 1, (int)L, b, (int)d, z1, b, t.status));
-  GALORE_TRY(tensor_group_launch_project(t.tg, st));
-  sum_split_kernel<<<grid_for(zb), 256, 0, st>>>(z0, z1, nullptr, nullptr, w.Zhi, w.Zlo, zb);
-  GALORE_LAUNCH_CHECK();
-  const int m = t.master, s1 = (m + 1) % 3, s2 = (m + 2) % 3;
-  tensor_group_reset(t.tg);
-  GALORE_TRY(tensor_group_add_gemm(t.tg, pr.G, pr.ldg, a_mn, w.Zhi, b, 1, (int)d, b, (int)L, t.F[s1], b, t.status));
-  GALORE_TRY(tensor_group_add_gemm(t.tg, pr.G, pr.ldg, a_mn, w.Zlo, b, 1, (int)d, b, (int)L, t.F[s2], b, t.status));
-  GALORE_TRY(tensor_group_launch_project(t.tg, st));
-  add_sumsq_kernel<<<kSumsqBlocks, 256, 0, st>>>(t.F[s1], t.F[s2], yb, w.part);
-  GALORE_LAUNCH_CHECK();
-  shift_split_kernel<<<grid_for(yb), 256, 0, st>>>(t.F[s1], t.F[m], yb, b, w.part, w.Yhi, w.Ylo);
-  GALORE_LAUNCH_CHECK();
-  t.master = s1;
-  return orth ? orth_tensor(t, w, d, b, st) : GALORE_OK;
+// Z = A^T Y ; Y' = A Z + delta Y for every lane; then Y = orth(Y') for the lanes in `orth`
+static galore_status_t power_step_tensor(const Ctx& c, const std::vector<Lane*>& lanes, const std::vector<Lane*>& orth) {
+  if (lanes.empty()) return GALORE_OK;
+  const int b = c.b;
+  const int64_t d = c.d, L = c.L, zb = L * b, yb = d * b;
+  cudaStream_t st = c.st;
+  const int at_mn = c.left ? 1 : 0;   // A^T as the first operand: G^T (left) is M-contiguous in G, G (right) is K-contiguous
+  const int a_mn = c.left ? 0 : 1;    // A as the first operand
+  tensor_group_reset(c.tg);
+  for (Lane* l : lanes) {
+    float* z0 = (float*)l->w.Zu;
+    GALORE_TRY(tensor_group_add_gemm(c.tg, l->pr.G, l->pr.ldg, at_mn, l->w.Yhi, b, 1, (int)L, b, (int)d, z0, b, l->status));
+    GALORE_TRY(tensor_group_add_gemm(c.tg, l->pr.G, l->pr.ldg, at_mn, l->w.Ylo, b, 1, (int)L, b, (int)d, z0 + zb, b, l->status));
+  }
+  GALORE_TRY(tensor_group_launch_project(c.tg, st));
+  for (Lane* l : lanes) {
+    float* z0 = (float*)l->w.Zu;
+    sum_split_kernel<<<grid_for(zb), 256, 0, st>>>(z0, z0 + zb, nullptr, nullptr, l->w.Zhi, l->w.Zlo, zb);
+    GALORE_LAUNCH_CHECK();
+  }
+  tensor_group_reset(c.tg);
+  for (Lane* l : lanes) {
+    TensorRefresh& t = l->tr;
+    const int m = t.master, s1 = (m + 1) % 3, s2 = (m + 2) % 3;
+    GALORE_TRY(tensor_group_add_gemm(c.tg, l->pr.G, l->pr.ldg, a_mn, l->w.Zhi, b, 1, (int)d, b, (int)L, t.F[s1], b, l->status));
+    GALORE_TRY(tensor_group_add_gemm(c.tg, l->pr.G, l->pr.ldg, a_mn, l->w.Zlo, b, 1, (int)d, b, (int)L, t.F[s2], b, l->status));
+  }
+  GALORE_TRY(tensor_group_launch_project(c.tg, st));
+  for (Lane* l : lanes) {
+    TensorRefresh& t = l->tr;
+    const int m = t.master, s1 = (m + 1) % 3, s2 = (m + 2) % 3;
+    add_sumsq_kernel<<<kSumsqBlocks, 256, 0, st>>>(t.F[s1], t.F[s2], yb, l->w.part);
+    GALORE_LAUNCH_CHECK();
+    shift_split_kernel<<<grid_for(yb), 256, 0, st>>>(t.F[s1], t.F[m], yb, b, l->w.part, l->w.Yhi, l->w.Ylo);
+    GALORE_LAUNCH_CHECK();
+    t.master = s1;
+    l->Y = t.F[t.master];
+  }
+  return orth_tensor(c, orth);
+}
+
+// the same step with FMA products (any dtype, any leading dimension); always ends orthonormal
+template <typename TG>
+static galore_status_t power_step_fma(const Ctx& c, const std::vector<Lane*>& lanes) {
+  if (lanes.empty()) return GALORE_OK;
+  const int b = c.b;
+  const int64_t d = c.d, L = c.L, yb = d * b;
+  cudaStream_t st = c.st;
+  for (Lane* l : lanes) {
+    const TG* G = (const TG*)l->pr.G;
+    const int64_t sAi = c.left ? l->pr.ldg : 1;    // A(i, l) = G[i*sAi + l*sAl]
+    const int64_t sAl = c.left ? 1 : l->pr.ldg;
+    float* Z = (float*)l->w.Zu;
+    {  // Z = A^T Y   (L x b)
+      EpiStore<float, float> epi{Z, b, 0, 1.f, 0.f};
+      GALORE_TRY((launch_gemm_simt<TG, float, float>((int)L, b, (int)d, G, sAl, sAi, l->Y, b, 1, 1, epi, st)));
+    }
+    {  // Y' = A Z     (d x b)
+      EpiStore<float, float> epi{l->Yn, b, 0, 1.f, 0.f};
+      GALORE_TRY((launch_gemm_simt<TG, float, float>((int)d, b, (int)L, G, sAi, sAl, Z, b, 1, 1, epi, st)));
+    }
+    sumsq_kernel<<<kSumsqBlocks, 256, 0, st>>>(l->Yn, yb, l->w.part);
+    GALORE_LAUNCH_CHECK();
+    shift_kernel<<<grid_for(yb), 256, 0, st>>>(l->Yn, l->Y, yb, b, l->w.part);
+    GALORE_LAUNCH_CHECK();
+  }
+  // the old block is no longer needed: it receives the result
+  return orthonormalise<float, float>(c, lanes, [](Lane* l) { return l->Yn; }, [](Lane* l) { return l->Y; });
 }
 
 template <typename TG>
-static galore_status_t refresh_typed(const RefreshProblem& pr, void* workspace, int32_t* status,
-                                     galore_refresh_info_t* info, cudaStream_t st) {
-  const TG* G = (const TG*)pr.G;
-  const int64_t d = pr.left ? pr.m : pr.n;
-  const int64_t L = pr.left ? pr.n : pr.m;
-  const int64_t sAi = pr.left ? pr.ldg : 1;    // A(i, l) = G[i*sAi + l*sAl]
-  const int64_t sAl = pr.left ? 1 : pr.ldg;
-  const int r = pr.rank, b = pr.block;
-  RefreshBuffers w = layout(workspace, d, L, r, b);
-  galore_refresh_info_t local = {};
-  local.block = b;
-  // phase clock: host time at points where the stream is synchronised anyway
-  using clk = std::chrono::steady_clock;
-  auto now_synced = [&]() {
-    cudaStreamSynchronize(st);
-    return clk::now();
-  };
-  auto ms_between = [](clk::time_point a, clk::time_point b2) { return std::chrono::duration<double, std::milli>(b2 - a).count(); };
-  const clk::time_point t_begin = now_synced();
-
-  float* Y = w.Ya;
-  float* Yn = w.Yb;
-  const int64_t yb = d * b;
-  int q_done = 0;
-  std::vector<double> theta(b);
+static galore_status_t refresh_group(const RefreshProblem* prs, int count, void* workspace, size_t slot_bytes,
+                                     int32_t* const* status, galore_refresh_info_t* infos, cudaStream_t st) {
+  if (count < 1 || count > kMaxSlots) return GALORE_ERR_INVALID_ARG;
+  const RefreshProblem& p0 = prs[0];
+  Ctx c = {};
+  c.base0 = (char*)workspace;
+  c.slot_bytes = (int64_t)slot_bytes;
+  c.left = p0.left;
+  c.d = p0.left ? p0.m : p0.n;
+  c.L = p0.left ? p0.n : p0.m;
+  c.r = p0.rank;
+  c.b = p0.block;
+  c.st = st;
+  const int64_t d = c.d, L = c.L;
+  const int r = c.r, b = c.b;
+  c.w0 = layout(workspace, d, L, r, b);
   const bool full_space = (b == d);
-
-  // tensor cores carry the power steps when the gradient is bf16 and everything is TMA-addressable
-  const bool tensor = pr.use_tensor && !full_space && sizeof(TG) == 2 && (b % 8) == 0 && (pr.ldg % 8) == 0 &&
-                      (((uintptr_t)pr.G) & 15) == 0;
-  TensorRefresh tr = {};
+  // tensor cores carry the power steps when the gradients are bf16 and everything is TMA-addressable
+  bool tensor = p0.use_tensor && !full_space && sizeof(TG) == 2 && (b % 8) == 0;
+  for (int i = 0; i < count; ++i) tensor = tensor && (prs[i].ldg % 8) == 0 && (((uintptr_t)prs[i].G) & 15) == 0;
+  c.tensor = tensor;
   struct GroupGuard {
     TensorGroup* g;
     ~GroupGuard() { tensor_group_free(g); }
   } guard{nullptr};
-  if (!full_space) {
-    fill_normal_kernel<<<grid_for(yb), 256, 0, st>>>(Y, yb, pr.seed);
-    GALORE_LAUNCH_CHECK();
-    if (tensor) {
-      guard.g = tr.tg = tensor_group_new();
-      if (!tr.tg) return GALORE_ERR_INVALID_ARG;
-      tr.F[0] = w.Ya; tr.F[1] = w.Yb; tr.F[2] = w.Yc;
-      tr.master = 0;
-      tr.status = status;
-      split_kernel<<<grid_for(yb), 256, 0, st>>>(Y, w.Yhi, w.Ylo, yb);
-      GALORE_LAUNCH_CHECK();
-      GALORE_TRY(orth_tensor(tr, w, d, b, st));
-    } else {
-      GALORE_TRY(orthonormalise(Y, Yn, d, b, w, status, st));
-      std::swap(Y, Yn);
-    }
+  if (tensor) {
+    guard.g = c.tg = tensor_group_new();
+    if (!c.tg) return GALORE_ERR_INVALID_ARG;
   }
-  double predicted = 0.0;
-  bool converged = full_space;
 
-  // one power step, Z = A^T Y ; Y' = A Z + delta Y ; optionally Y = orth(Y')
-  auto one_step = [&](bool orth) -> galore_status_t {
-    if (tensor) {
-      GALORE_TRY(power_step_tensor(tr, pr, w, d, L, b, orth, st));
-      Y = tr.F[tr.master];
-      return GALORE_OK;
-    }
-    float* Z = (float*)w.Zu;
-    {  // Z = A^T Y   (L x b)
-      EpiStore<float, float> epi{Z, b, 0, 1.f, 0.f};
-      GALORE_TRY((launch_gemm_simt<TG, float, float>((int)L, b, (int)d, G, sAl, sAi, Y, b, 1, 1, epi, st)));
-    }
-    {  // Y' = A Z     (d x b)
-      EpiStore<float, float> epi{Yn, b, 0, 1.f, 0.f};
-      GALORE_TRY((launch_gemm_simt<TG, float, float>((int)d, b, (int)L, G, sAi, sAl, Z, b, 1, 1, epi, st)));
-    }
-    sumsq_kernel<<<kSumsqBlocks, 256, 0, st>>>(Yn, yb, w.part);
-    GALORE_LAUNCH_CHECK();
-    shift_kernel<<<grid_for(yb), 256, 0, st>>>(Yn, Y, yb, b, w.part);
-    GALORE_LAUNCH_CHECK();
-    return orthonormalise(Yn, Y, d, b, w, status, st);    // the old block is no longer needed: reuse it for the result
+  std::vector<Lane> store(count);
+  std::vector<Lane*> all;
+  const int64_t yb = d * b;
+  for (int i = 0; i < count; ++i) {
+    Lane& l = store[i];
+    l.pr = prs[i];
+    l.slot = i;
+    l.base = c.base0 + (int64_t)i * c.slot_bytes;
+    l.w = layout(l.base, d, L, r, b);
+    l.status = status[i];
+    l.Y = l.w.Ya;
+    l.Yn = l.w.Yb;
+    l.tr.F[0] = l.w.Ya; l.tr.F[1] = l.w.Yb; l.tr.F[2] = l.w.Yc;
+    l.tr.master = 0;
+    l.theta.assign(b, 0.0);
+    l.info.block = b;
+    l.converged = full_space;
+    all.push_back(&l);
+    GALORE_CUDA_TRY(cudaMemsetAsync(l.w.flags, 0, sizeof(int32_t), st));
+  }
+
+  // phase clock (only when the caller wants the record): host time at points where the stream is idle
+  using clk = std::chrono::steady_clock;
+  const bool timed = infos != nullptr;
+  auto now_synced = [&]() {
+    if (timed) cudaStreamSynchronize(st);
+    return clk::now();
+  };
+  auto ms_between = [](clk::time_point a, clk::time_point b2) { return std::chrono::duration<double, std::milli>(b2 - a).count(); };
+  double ms_ritz = 0.0, ms_jacobi = 0.0, ms_power = 0.0;
+  const clk::time_point t_begin = now_synced();
+
+  auto step = [&](const std::vector<Lane*>& lanes, const std::vector<Lane*>& orth) -> galore_status_t {
+    if (tensor) return power_step_tensor(c, lanes, orth);
+    return power_step_fma<TG>(c, lanes);
+  };
+  auto read_theta = [&](const std::vector<Lane*>& lanes) -> galore_status_t {
+    for (Lane* l : lanes)
+      GALORE_CUDA_TRY(cudaMemcpyAsync(l->theta.data(), l->w.theta, sizeof(double) * b, cudaMemcpyDeviceToHost, st));
+    GALORE_CUDA_TRY(cudaStreamSynchronize(st));
+    return GALORE_OK;
   };
 
-  // ---- first steps, then a cheap look at the spectrum ------------------------------------------
-  // After a step from an orthonormal Y, ||z_i||^2 (Z = A^T Y) are the Rayleigh quotients of the
-  // block's columns.  Sorted, they stand in for the Ritz values: enough to size the iteration
-  // (their spread is narrower than the spectrum's, which errs towards more steps) and to decide
-  // how many steps may be chained before the block has to be orthonormalised again.
-  int q_target = 0;
-  int orth_every = 1;
   if (!full_space) {
-    const int q0 = std::min(pr.max_iters, std::max(1, pr.first_iters));
-    for (; q_done < q0; ++q_done) GALORE_TRY(one_step(true));
-    q_target = q_done;
-    if (b > r && q_done < pr.max_iters) {
-      double* slices = (double*)w.Y64;                      // kColSlices x b doubles, Y64 is idle here
-      const float* z0 = (const float*)w.Zu;
-      const float* z1 = tensor ? z0 + L * b : nullptr;
-      colsumsq_partial_kernel<<<dim3((unsigned)ceil_div(b, 128), kColSlices), 128, 0, st>>>(z0, z1, L, b, slices);
+    for (Lane* l : all) {
+      fill_normal_kernel<<<grid_for(yb), 256, 0, st>>>(l->Y, yb, l->pr.seed);
       GALORE_LAUNCH_CHECK();
-      colsumsq_final_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(slices, b, w.lam);
-      GALORE_LAUNCH_CHECK();
-      rank_desc_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(w.lam, b, w.theta, w.order);
-      GALORE_LAUNCH_CHECK();
-      GALORE_CUDA_TRY(cudaMemcpyAsync(theta.data(), w.theta, sizeof(double) * b, cudaMemcpyDeviceToHost, st));
-      GALORE_CUDA_TRY(cudaStreamSynchronize(st));
-      const double ratio = theta[r - 1] > 0.0 ? theta[b - 1] / theta[r - 1] : 1.0;
-      if (ratio > 0.0 && ratio < 1.0) {
-        const int need = (int)ceil(log(pr.tol) / log(ratio)) + 1;
-        q_target = std::min(pr.max_iters, std::max(need, q_done));
-      } else if (ratio >= 1.0) {
-        q_target = pr.max_iters;
+      if (tensor) {
+        split_kernel<<<grid_for(yb), 256, 0, st>>>(l->Y, l->w.Yhi, l->w.Ylo, yb);
+        GALORE_LAUNCH_CHECK();
       }
-      if (tensor && theta[b - 1] > 0.0) {
-        // chained steps multiply the block's condition number by theta_1/theta_b each; the bf16 pair
-        // carries 16 bits and the Gram matrix squares the product, so keep it below about 100
-        const double spread = theta[0] / theta[b - 1];
-        orth_every = spread > 1.0 ? (int)floor(log(100.0) / log(spread)) : 8;
-        orth_every = std::max(1, std::min(orth_every, 8));
+    }
+    if (tensor) {
+      GALORE_TRY(orth_tensor(c, all));
+    } else {
+      GALORE_TRY((orthonormalise<float, float>(c, all, [](Lane* l) { return l->Y; }, [](Lane* l) { return l->Yn; })));
+      for (Lane* l : all) std::swap(l->Y, l->Yn);
+    }
+
+    // ---- first steps, then a cheap look at the spectrum ------------------------------------------
+    // After a step from an orthonormal Y, ||z_i||^2 (Z = A^T Y) are the Rayleigh quotients of the
+    // block's columns.  Sorted, they stand in for the Ritz values: enough to size the iteration
+    // (their spread is narrower than the spectrum's, which errs towards more steps) and to decide
+    // how many steps may be chained before the block has to be orthonormalised again.
+    const int q0 = std::min(p0.max_iters, std::max(1, p0.first_iters));
+    for (int q = 0; q < q0; ++q) GALORE_TRY(step(all, all));
+    for (Lane* l : all) l->q_done = l->q_target = q0;
+    if (b > r && q0 < p0.max_iters) {
+      for (Lane* l : all) {
+        double* slices = (double*)l->w.Y64;                      // kColSlices x b doubles, Y64 is idle here
+        const float* z0 = (const float*)l->w.Zu;
+        const float* z1 = tensor ? z0 + L * b : nullptr;
+        colsumsq_partial_kernel<<<dim3((unsigned)ceil_div(b, 128), kColSlices), 128, 0, st>>>(z0, z1, L, b, slices);
+        GALORE_LAUNCH_CHECK();
+        colsumsq_final_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(slices, b, l->w.lam);
+        GALORE_LAUNCH_CHECK();
+        rank_desc_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(l->w.lam, b, l->w.theta, l->w.order);
+        GALORE_LAUNCH_CHECK();
+      }
+      GALORE_TRY(read_theta(all));
+      for (Lane* l : all) {
+        const std::vector<double>& theta = l->theta;
+        const double ratio = theta[r - 1] > 0.0 ? theta[b - 1] / theta[r - 1] : 1.0;
+        if (ratio > 0.0 && ratio < 1.0) {
+          const int need = (int)ceil(log(l->pr.tol) / log(ratio)) + 1;
+          l->q_target = std::min(l->pr.max_iters, std::max(need, l->q_done));
+        } else if (ratio >= 1.0) {
+          l->q_target = l->pr.max_iters;
+        }
+        if (tensor && theta[b - 1] > 0.0) {
+          // chained steps multiply the block's condition number by theta_1/theta_b each; the bf16 pair
+          // carries 16 bits and the Gram matrix squares the product, so keep it below about 100
+          const double spread = theta[0] / theta[b - 1];
+          l->orth_every = spread > 1.0 ? (int)floor(log(100.0) / log(spread)) : 8;
+          l->orth_every = std::max(1, std::min(l->orth_every, 8));
+        }
       }
     }
   }
-  bool with_vt = false;
 
-  for (;;) {
-    // ---- power steps ---------------------------------------------------------
-    for (; q_done < q_target; ++q_done) {
-      const bool orth = ((q_target - 1 - q_done) % orth_every) == 0;      // the last step always ends orthonormal
-      GALORE_TRY(one_step(orth));
+  std::vector<Lane*> live = all;            // lanes that still iterate
+  while (!live.empty()) {
+    // ---- power steps: every lane up to its own target, on its own orthonormalisation schedule ----
+    for (;;) {
+      std::vector<Lane*> stepping, orth;
+      for (Lane* l : live)
+        if (l->q_done < l->q_target) {
+          stepping.push_back(l);
+          if (((l->q_target - 1 - l->q_done) % l->orth_every) == 0) orth.push_back(l);   // the last step always ends orthonormal
+        }
+      if (stepping.empty()) break;
+      GALORE_TRY(step(stepping, orth));
+      for (Lane* l : stepping) l->q_done += 1;
     }
     // ---- Rayleigh-Ritz in fp64 --------------------------------------------------
     const clk::time_point t_rr = now_synced();
-    local.ms_power = ms_between(t_begin, t_rr) - local.ms_ritz - local.ms_jacobi;
+    ms_power = ms_between(t_begin, t_rr) - ms_ritz - ms_jacobi;
     if (full_space) {
-      set_identity_kernel<<<grid_for(yb), 256, 0, st>>>(w.Y64, (int)d);
-      GALORE_LAUNCH_CHECK();
+      for (Lane* l : live) {
+        set_identity_kernel<<<grid_for(yb), 256, 0, st>>>(l->w.Y64, (int)d);
+        GALORE_LAUNCH_CHECK();
+      }
     } else {
       // Y left the last power step orthonormal to working precision (1e-7 on the FMA path, about 1e-4 from the
       // bf16 pairs); one CholeskyQR pass in fp64 from there is orthonormal to double rounding
-      GALORE_TRY(orthonormalise(Y, w.Y64, d, b, w, status, st));
+      GALORE_TRY((orthonormalise<float, double>(c, live, [](Lane* l) { return l->Y; }, [](Lane* l) { return l->w.Y64; })));
     }
-    double* Z64 = (double*)w.Zu;
-    {  // Z = A^T Y   (L x b), fp64
-      EpiStore<double, double> epi{Z64, b, 0, 1.0, 0.0};
-      GALORE_TRY((launch_gemm_dmma<TG, double>((int)L, b, (int)d, G, sAl, sAi, w.Y64, b, 1, epi, st)));
+    for (Lane* l : live) {   // Z = A^T Y   (L x b), fp64
+      const TG* G = (const TG*)l->pr.G;
+      const int64_t sAi = c.left ? l->pr.ldg : 1, sAl = c.left ? 1 : l->pr.ldg;
+      EpiStore<double, double> epi{(double*)l->w.Zu, b, 0, 1.0, 0.0};
+      GALORE_TRY((launch_gemm_dmma<TG, double>((int)L, b, (int)d, G, sAl, sAi, l->w.Y64, b, 1, epi, st)));
     }
     const clk::time_point t_jac = now_synced();
-    local.ms_ritz += ms_between(t_rr, t_jac);
+    ms_ritz += ms_between(t_rr, t_jac);
     // Eigenvectors are read off the rotated rows Theta V^T; only when wanted eigenvalues are tiny
     // against the largest (a gradient of rank below r) are the rotations accumulated separately.
-    for (;;) {
-      GALORE_TRY(gram(Z64, L, b, w.H, st));                   // H = Z^T Z
-      if (with_vt) {
-        set_identity_kernel<<<grid_for((int64_t)b * b), 256, 0, st>>>(w.Vt, b);
+    std::vector<Lane*> solving = live;
+    while (!solving.empty()) {
+      GALORE_TRY((gram<double>(c, solving, [](Lane* l) { return (double*)l->w.Zu; }, L, c.w0.H)));     // H = Z^T Z
+      std::vector<Lane*> plain, with_vt;
+      for (Lane* l : solving) (l->with_vt ? with_vt : plain).push_back(l);
+      for (Lane* l : with_vt) {
+        set_identity_kernel<<<grid_for((int64_t)b * b), 256, 0, st>>>(l->w.Vt, b);
         GALORE_LAUNCH_CHECK();
       }
-      int sweeps = 0;
-      GALORE_TRY(jacobi_eigh(w.H, with_vt ? w.Vt : nullptr, b, w.jac, w.counter, 1e-11, 40, &sweeps, st));
-      local.jacobi_sweeps = sweeps;
-      row_norm_kernel<<<b, 256, 0, st>>>(w.H, b, w.lam);
-      GALORE_LAUNCH_CHECK();
-      rank_desc_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(w.lam, b, w.theta, w.order);
-      GALORE_LAUNCH_CHECK();
-      GALORE_CUDA_TRY(cudaMemcpyAsync(theta.data(), w.theta, sizeof(double) * b, cudaMemcpyDeviceToHost, st));
-      GALORE_CUDA_TRY(cudaStreamSynchronize(st));
-      if (with_vt || theta[r - 1] > 1e-8 * theta[0]) break;
-      with_vt = true;
+      for (int pass = 0; pass < 2; ++pass) {
+        const std::vector<Lane*>& set = pass == 0 ? plain : with_vt;
+        if (set.empty()) continue;
+        const SlotList sl = slots_of(c, set);
+        int sweeps[kMaxSlots] = {};
+        GALORE_TRY(jacobi_eigh(c.w0.H, pass == 0 ? nullptr : c.w0.Vt, b, c.w0.jac, c.w0.counter, 1e-11, 40, sweeps, st, &sl));
+        for (size_t i = 0; i < set.size(); ++i) set[i]->info.jacobi_sweeps = sweeps[i];
+      }
+      for (Lane* l : solving) {
+        row_norm_kernel<<<b, 256, 0, st>>>(l->w.H, b, l->w.lam);
+        GALORE_LAUNCH_CHECK();
+        rank_desc_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(l->w.lam, b, l->w.theta, l->w.order);
+        GALORE_LAUNCH_CHECK();
+      }
+      GALORE_TRY(read_theta(solving));
+      std::vector<Lane*> again;
+      for (Lane* l : solving)
+        if (!l->with_vt && !(l->theta[r - 1] > 1e-8 * l->theta[0])) {
+          l->with_vt = true;
+          again.push_back(l);
+        }
+      solving = again;
     }
-    local.ms_jacobi += ms_between(t_jac, now_synced());
+    ms_jacobi += ms_between(t_jac, now_synced());
 
+    std::vector<Lane*> more;
     if (!full_space) {
-      const double th_r = theta[r - 1], th_b = theta[b - 1];
-      const double ratio = (b > r && th_r > 0.0) ? th_b / th_r : 1.0;
-      predicted = (ratio < 1.0) ? pow(ratio, (double)q_done) : 1.0;
-      converged = predicted <= pr.tol;
-      if (!converged && q_done < pr.max_iters && ratio < 1.0 && ratio > 0.0) {
-        int need = (int)ceil(log(pr.tol) / log(ratio)) + 2;
-        q_target = std::min(pr.max_iters, std::max(need, q_done + 1));
-        continue;                                              // more power steps, then Rayleigh-Ritz again
+      for (Lane* l : live) {
+        const double th_r = l->theta[r - 1], th_b = l->theta[b - 1];
+        const double ratio = (b > r && th_r > 0.0) ? th_b / th_r : 1.0;
+        l->predicted = (ratio < 1.0) ? pow(ratio, (double)l->q_done) : 1.0;
+        l->converged = l->predicted <= l->pr.tol;
+        if (!l->converged && l->q_done < l->pr.max_iters && ratio < 1.0 && ratio > 0.0) {
+          const int need = (int)ceil(log(l->pr.tol) / log(ratio)) + 2;
+          l->q_target = std::min(l->pr.max_iters, std::max(need, l->q_done + 1));
+          more.push_back(l);                                       // more power steps, then Rayleigh-Ritz again
+        }
       }
     }
-    break;
+    live = more;
   }
 
   // ---- P = Y S[:, top r] ------------------------------------------------------------
-  if (with_vt)
-    gather_rows_kernel<<<r, 256, 0, st>>>(w.Vt, w.order, b, w.Vsel);
-  else
-    gather_rows_scaled_kernel<<<r, 256, 0, st>>>(w.H, w.lam, w.order, b, w.Vsel);
-  GALORE_LAUNCH_CHECK();
-  {
-    EpiStore<double, double> epi{w.P64, r, 0, 1.0, 0.0};
-    GALORE_TRY((launch_gemm_dmma<double, double>((int)d, r, b, w.Y64, b, 1, w.Vsel, 1, b, epi, st)));
-  }
   const int64_t pc = d * r;
-  if (pr.p_dtype == GALORE_BF16)
-    convert_kernel<double, __nv_bfloat16><<<grid_for(pc), 256, 0, st>>>(w.P64, (__nv_bfloat16*)pr.P, pc);
-  else
-    convert_kernel<double, float><<<grid_for(pc), 256, 0, st>>>(w.P64, (float*)pr.P, pc);
-  GALORE_LAUNCH_CHECK();
-
-  // ---- a-posteriori residual of the kept Ritz pairs -----------------------------------
-  // || A A^T P - P Theta ||.  It is a diagnostic: on the tensor path A^T P = Z S is formed from the
-  // products already at hand and A (A^T P) runs on the tensor cores in bf16 pairs.
-  const bool tensor_residual = tensor && (r % 8) == 0;
-  if (tensor_residual) {
-    EpiSplitPair e1{w.Zhi, w.Zlo, r};
-    GALORE_TRY((launch_gemm_dmma<double, double>((int)L, r, b, (const double*)w.Zu, b, 1, w.Vsel, 1, b, e1, st)));
-    const int a_mn = pr.left ? 0 : 1;
-    const int s1 = (tr.master + 1) % 3, s2 = (tr.master + 2) % 3;
-    tensor_group_reset(tr.tg);
-    GALORE_TRY(tensor_group_add_gemm(tr.tg, pr.G, pr.ldg, a_mn, w.Zhi, r, 1, (int)d, r, (int)L, tr.F[s1], r, status));
-    GALORE_TRY(tensor_group_add_gemm(tr.tg, pr.G, pr.ldg, a_mn, w.Zlo, r, 1, (int)d, r, (int)L, tr.F[s2], r, status));
-    GALORE_TRY(tensor_group_launch_project(tr.tg, st));
-    GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
-    residual_pair_kernel<<<grid_for(d * r), 256, 0, st>>>(tr.F[s1], tr.F[s2], w.P64, w.theta, d, r, w.scal);
-    GALORE_LAUNCH_CHECK();
-  } else {
-    double* T1 = (double*)w.Zu;   // L x r
-    double* T2 = w.Y64;           // d x r (Y64 is no longer needed)
-    EpiStore<double, double> e1{T1, r, 0, 1.0, 0.0};
-    GALORE_TRY((launch_gemm_dmma<TG, double>((int)L, r, (int)d, G, sAl, sAi, w.P64, r, 1, e1, st)));
-    EpiStore<double, double> e2{T2, r, 0, 1.0, 0.0};
-    GALORE_TRY((launch_gemm_dmma<TG, double>((int)d, r, (int)L, G, sAi, sAl, T1, r, 1, e2, st)));
-    GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
-    residual_kernel<<<grid_for(pc), 256, 0, st>>>(T2, w.P64, w.theta, d, r, w.scal);
+  for (Lane* l : all) {
+    const RefreshBuffers& w = l->w;
+    if (l->with_vt)
+      gather_rows_kernel<<<r, 256, 0, st>>>(w.Vt, w.order, b, w.Vsel);
+    else
+      gather_rows_scaled_kernel<<<r, 256, 0, st>>>(w.H, w.lam, w.order, b, w.Vsel);
     GALORE_LAUNCH_CHECK();
   }
   {
-    double sc[2] = {0, 0};
-    GALORE_CUDA_TRY(cudaMemcpyAsync(sc, w.scal, sizeof(sc), cudaMemcpyDeviceToHost, st));
-    GALORE_CUDA_TRY(cudaStreamSynchronize(st));
-    local.residual = theta[0] > 0.0 ? sqrt(sc[1]) / (theta[0] * sqrt((double)r)) : 0.0;
+    EpiStore<double, double> epi{c.w0.P64, r, 0, 1.0, 0.0};
+    const SlotList sl = slots_of(c, all);
+    GALORE_TRY((launch_gemm_dmma<double, double>((int)d, r, b, c.w0.Y64, b, 1, c.w0.Vsel, 1, b, epi, st, 1, 0, 0, &sl)));
   }
-  local.ms_total = ms_between(t_begin, now_synced());
-  local.ms_ritz = local.ms_total - local.ms_power - local.ms_jacobi;
-  local.iterations = q_done;
-  local.converged = converged ? 1 : 0;
-  local.predicted_error = predicted;
-  local.sigma_1 = sqrt(theta[0]);
-  local.sigma_r = sqrt(theta[r - 1]);
-  local.sigma_next = (b > r) ? sqrt(theta[r]) : 0.0;
-  if (info) *info = local;
-  return converged ? GALORE_OK : GALORE_WARN_NOT_CONVERGED;
+  for (Lane* l : all) {
+    if (l->pr.p_dtype == GALORE_BF16)
+      convert_kernel<double, __nv_bfloat16><<<grid_for(pc), 256, 0, st>>>(l->w.P64, (__nv_bfloat16*)l->pr.P, pc);
+    else
+      convert_kernel<double, float><<<grid_for(pc), 256, 0, st>>>(l->w.P64, (float*)l->pr.P, pc);
+    GALORE_LAUNCH_CHECK();
+    merge_flags_kernel<<<1, 1, 0, st>>>(l->status, l->w.flags);
+    GALORE_LAUNCH_CHECK();
+  }
+
+  // ---- a-posteriori residual of the kept Ritz pairs (a diagnostic: only when the record is wanted) ----
+  // || A A^T P - P Theta ||.  On the tensor path A^T P = Z S is formed from the products already at
+  // hand and A (A^T P) runs on the tensor cores in bf16 pairs.
+  if (infos) {
+    const bool tensor_residual = tensor && (r % 8) == 0;
+    for (Lane* l : all) {
+      const RefreshBuffers& w = l->w;
+      const TG* G = (const TG*)l->pr.G;
+      const int64_t sAi = c.left ? l->pr.ldg : 1, sAl = c.left ? 1 : l->pr.ldg;
+      if (tensor_residual) {
+        EpiSplitPair e1{w.Zhi, w.Zlo, r};
+        GALORE_TRY((launch_gemm_dmma<double, double>((int)L, r, b, (const double*)w.Zu, b, 1, w.Vsel, 1, b, e1, st)));
+        const int a_mn = c.left ? 0 : 1;
+        const int s1 = (l->tr.master + 1) % 3, s2 = (l->tr.master + 2) % 3;
+        tensor_group_reset(c.tg);
+        GALORE_TRY(tensor_group_add_gemm(c.tg, l->pr.G, l->pr.ldg, a_mn, w.Zhi, r, 1, (int)d, r, (int)L, l->tr.F[s1], r, l->status));
+        GALORE_TRY(tensor_group_add_gemm(c.tg, l->pr.G, l->pr.ldg, a_mn, w.Zlo, r, 1, (int)d, r, (int)L, l->tr.F[s2], r, l->status));
+        GALORE_TRY(tensor_group_launch_project(c.tg, st));
+        GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
+        residual_pair_kernel<<<grid_for(d * r), 256, 0, st>>>(l->tr.F[s1], l->tr.F[s2], w.P64, w.theta, d, r, w.scal);
+        GALORE_LAUNCH_CHECK();
+      } else {
+        double* T1 = (double*)w.Zu;   // L x r
+        double* T2 = w.Y64;           // d x r (Y64 is no longer needed)
+        EpiStore<double, double> e1{T1, r, 0, 1.0, 0.0};
+        GALORE_TRY((launch_gemm_dmma<TG, double>((int)L, r, (int)d, G, sAl, sAi, w.P64, r, 1, e1, st)));
+        EpiStore<double, double> e2{T2, r, 0, 1.0, 0.0};
+        GALORE_TRY((launch_gemm_dmma<TG, double>((int)d, r, (int)L, G, sAi, sAl, T1, r, 1, e2, st)));
+        GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
+        residual_kernel<<<grid_for(pc), 256, 0, st>>>(T2, w.P64, w.theta, d, r, w.scal);
+        GALORE_LAUNCH_CHECK();
+      }
+    }
+    std::vector<double> sc(2 * (size_t)count, 0.0);
+    for (int i = 0; i < count; ++i)
+      GALORE_CUDA_TRY(cudaMemcpyAsync(&sc[2 * i], store[i].w.scal, 2 * sizeof(double), cudaMemcpyDeviceToHost, st));
+    GALORE_CUDA_TRY(cudaStreamSynchronize(st));
+    for (int i = 0; i < count; ++i) {
+      const Lane& l = store[i];
+      store[i].info.residual = l.theta[0] > 0.0 ? sqrt(sc[2 * i + 1]) / (l.theta[0] * sqrt((double)r)) : 0.0;
+    }
+  }
+  GALORE_CUDA_TRY(cudaStreamSynchronize(st));      // the refresh is complete when the call returns
+  const double ms_total = ms_between(t_begin, clk::now());
+  galore_status_t worst = GALORE_OK;
+  for (int i = 0; i < count; ++i) {
+    Lane& l = store[i];
+    // times of the group as a whole, divided evenly among its layers
+    l.info.ms_total = ms_total / count;
+    l.info.ms_power = ms_power / count;
+    l.info.ms_jacobi = ms_jacobi / count;
+    l.info.ms_ritz = (ms_total - ms_power - ms_jacobi) / count;
+    l.info.iterations = l.q_done;
+    l.info.converged = l.converged ? 1 : 0;
+    l.info.predicted_error = l.predicted;
+    l.info.sigma_1 = sqrt(l.theta[0]);
+    l.info.sigma_r = sqrt(l.theta[r - 1]);
+    l.info.sigma_next = (b > r) ? sqrt(l.theta[r]) : 0.0;
+    if (infos) infos[i] = l.info;
+    if (!l.converged) worst = GALORE_WARN_NOT_CONVERGED;
+  }
+  return worst;
+}
+
+galore_status_t refresh_projector_group(const RefreshProblem* prs, int count, void* workspace, size_t slot_bytes,
+                                        int32_t* const* status, galore_refresh_info_t* infos, cudaStream_t st) {
+  if (!prs || count < 1) return GALORE_ERR_INVALID_ARG;
+  for (int i = 1; i < count; ++i) {
+    const RefreshProblem &a = prs[0], &b = prs[i];
+    if (a.m != b.m || a.n != b.n || a.left != b.left || a.rank != b.rank || a.block != b.block || a.g_dtype != b.g_dtype ||
+        a.use_tensor != b.use_tensor || a.max_iters != b.max_iters || a.first_iters != b.first_iters)
+      return GALORE_ERR_INVALID_ARG;
+  }
+  if (prs[0].g_dtype == GALORE_BF16) return refresh_group<__nv_bfloat16>(prs, count, workspace, slot_bytes, status, infos, st);
+  return refresh_group<float>(prs, count, workspace, slot_bytes, status, infos, st);
 }
 
 galore_status_t refresh_projector(const RefreshProblem& pr, void* workspace, int32_t* status,
                                   galore_refresh_info_t* info, cudaStream_t st) {
-  if (pr.g_dtype == GALORE_BF16) return refresh_typed<__nv_bfloat16>(pr, workspace, status, info, st);
-  return refresh_typed<float>(pr, workspace, status, info, st);
+  const int64_t d = pr.left ? pr.m : pr.n, L = pr.left ? pr.n : pr.m;
+  return refresh_projector_group(&pr, 1, workspace, refresh_workspace_bytes(d, L, pr.rank, pr.block), &status, info, st);
 }
 
 }  // namespace galore

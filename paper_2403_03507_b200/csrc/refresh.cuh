@@ -33,4 +33,13 @@ const double* refresh_unrounded_projector(void* workspace, int64_t d, int64_t L,
 galore_status_t refresh_projector(const RefreshProblem& pr, void* workspace, int32_t* status,
                                   galore_refresh_info_t* info, cudaStream_t st);
 
+// The same refresh for `count` (<= kMaxSlots) problems of one shape, rank, block and dtype at once:
+// problem i works in the i-th slot of `workspace` (slots of slot_bytes = refresh_workspace_bytes()
+// each) and latches device conditions in status[i].  Each projector is what refresh_projector
+// would produce for that problem alone; the serial parts of the method run for all problems in one
+// launch per kernel.  infos: nullptr or `count` records (phase times are the group's, divided by
+// count; the a-posteriori residual is computed only when the record is wanted).
+galore_status_t refresh_projector_group(const RefreshProblem* prs, int count, void* workspace, size_t slot_bytes,
+                                        int32_t* const* status, galore_refresh_info_t* infos, cudaStream_t st);
+
 }  // namespace galore

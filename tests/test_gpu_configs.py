@@ -145,8 +145,8 @@ def test_rank_sweep_matrix_refresh_and_steps():
                 rep = assert_elementwise(Wg, Wo, W0, "bf16", 2, watch=wt)
             else:
                 Mc, _Ma, Vc, _Va = [t.cpu().numpy() for t in step_layer.get_q8_state()]
-                assert np.mean(Mc != o.M_codes) < 5e-3 and np.max(np.abs(cs[Mc] - cs[o.M_codes])) <= 0.9 / 64 + 1e-6
-                assert np.mean(Vc != o.V_codes) < 5e-3 and np.max(np.abs(cu[Vc] - cu[o.V_codes])) <= 0.9 / 128 + 1e-6
+                assert np.mean(Mc != o.M_codes) < 5e-3 and np.max(np.abs(cs[Mc] - cs[o.M_codes])) <= 2 * 0.9 / 64 + 1e-6
+                assert np.mean(Vc != o.V_codes) < 5e-3 and np.max(np.abs(cu[Vc] - cu[o.V_codes])) <= 2 * 0.9 / 128 + 1e-6
                 rep = elementwise_report(Wg, Wo, W0, "bf16", wt.peak)
                 # one differing code changes one N element by O(1) and with it a column of W by lr alpha |P|:
                 # a small share of the largest update, on a small share of the elements

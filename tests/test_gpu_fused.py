@@ -23,11 +23,11 @@ def _ld(n):
     return (n + 15) // 16 * 16
 
 
-def _build(state_fmt, w_dtype, q_block, shapes=SHAPES, weight_decay=0.0):
+def _build(state_fmt, w_dtype, q_block, shapes=SHAPES, weight_decay=0.0, adam_place=gb.ADAM_IN_PROJECTION):
     layers, orcs, Wd, W0s = [], [], [], []
     for i, (m, n, r) in enumerate(shapes):
         cfg = gb.make_config(m, n, r, refresh_gap=1000, w_dtype=w_dtype, g_dtype="bf16", state_fmt=state_fmt,
-                             auto_refresh=False, q_block=q_block, weight_decay=weight_decay)
+                             auto_refresh=False, q_block=q_block, weight_decay=weight_decay, adam_place=adam_place)
         layer = gb.Layer(cfg)
         assert layer.uses_tensor_path
         d = m if layer.side == gb.SIDE_LEFT else n
@@ -42,7 +42,7 @@ def _build(state_fmt, w_dtype, q_block, shapes=SHAPES, weight_decay=0.0):
 
 
 @pytest.mark.parametrize("state_fmt,w_dtype,q_block", [("f32", "bf16", 2048), ("f32", "f32", 2048), ("q8", "bf16", 2048),
-                                                       ("q8", "bf16", 256), ("q8", "f32", 4096), ("q8", "bf16", 1024)])
+                                                       ("q8", "bf16", 256), ("q8", "f32", 512), ("q8", "bf16", 1024)])
 def test_fused_batch_matches_the_oracle_element_by_element(state_fmt, w_dtype, q_block):
     layers, orcs, Wd, W0s = _build(state_fmt, w_dtype, q_block)
     launches0 = gb.galore_launch_count()
@@ -79,15 +79,16 @@ def test_fused_batch_matches_the_oracle_element_by_element(state_fmt, w_dtype, q
         else:
             Mc, Ma, Vc, Va = [t.cpu().numpy() for t in layer.get_q8_state()]
             assert np.allclose(Ma, o.M_absmax, rtol=1e-5, atol=0) and np.allclose(Va, o.V_absmax, rtol=1e-5, atol=0)
-            # fp32 against fp64 arithmetic may move a value on a threshold to the neighbouring code, never further
-            assert np.mean(Mc != o.M_codes) < 5e-3 and np.max(np.abs(cs[Mc] - cs[o.M_codes])) <= 0.9 / 64 + 1e-6
-            assert np.mean(Vc != o.V_codes) < 5e-3 and np.max(np.abs(cu[Vc] - cu[o.V_codes])) <= 0.9 / 128 + 1e-6
+            # fp32 against fp64 arithmetic may move a value on a threshold to the neighbouring code; such a code is an
+            # input difference of the next step, so over a few steps two coarse steps bound the distance
+            assert np.mean(Mc != o.M_codes) < 5e-3 and np.max(np.abs(cs[Mc] - cs[o.M_codes])) <= 2 * 0.9 / 64 + 1e-6
+            assert np.mean(Vc != o.V_codes) < 5e-3 and np.max(np.abs(cu[Vc] - cu[o.V_codes])) <= 2 * 0.9 / 128 + 1e-6
 
 
 def test_single_layer_step_without_k_slices_runs_adam_in_the_projection():
     # 1024 x 8192, r = 512: 2 x 32 tiles of 256 x 256 fill the machine without slicing K: two launches per step
     m, n, r = 1024, 8192, 512
-    cfg = gb.make_config(m, n, r, state_fmt="q8", auto_refresh=False)
+    cfg = gb.make_config(m, n, r, state_fmt="q8", auto_refresh=False, adam_place=gb.ADAM_IN_PROJECTION)
     layer = gb.Layer(cfg)
     P = wl.round_to(wl.random_orthonormal(m, r, np.random.default_rng(0)), "bf16")
     layer.set_projector(torch.from_numpy(P))
@@ -117,24 +118,25 @@ def _signed_permutation(d, r, rng):
     return P
 
 
-@pytest.mark.parametrize("mode", ["fused", "tensor_standalone", "fp32_path"])
-@pytest.mark.parametrize("q_block", [256, 2048, 4096])
+@pytest.mark.parametrize("mode", ["fused", "tensor_standalone", "tensor_standalone_batch", "fp32_path"])
+@pytest.mark.parametrize("q_block", [256, 1024, 2048])
 def test_codes_are_bit_exact_when_fp32_arithmetic_is_exact(mode, q_block):
     """beta1 = 0.5, beta2 = 0.75, P = columns of a signed permutation matrix and bf16 gradients: R is a signed
     copy of rows of G, the moment updates are exact in fp32 (products of at most 8 x 8 or 2 x 24 bits, one
     rounding in the final sum on both sides), so the stored codes and absmax must equal the oracle's bit for
     bit, on every kernel that writes them: the projection epilogue, the stand-alone tile kernel on the
-    tensor path (a batch of fewer than four layers) and on the fp32 path (interior and edge tiles)."""
+    tensor path (batches of fewer and of more than four layers) and on the fp32 path (interior and edge tiles)."""
     shapes = [(256, 512, 64), (512, 256, 64), (200, 304, 16), (300, 1365, 264), (1365, 300, 264)]
     if mode == "tensor_standalone":
-        shapes = shapes[:3]                      # fewer than four layers per batch: no fusion
+        shapes = shapes[:3]                      # fewer than four layers per batch: K may be sliced, Adam in its own kernel
     rng = np.random.default_rng(q_block)
     layers, orcs, Wd = [], [], []
     for i, (m, n, r) in enumerate(shapes):
         g_dtype = "f32" if mode == "fp32_path" else "bf16"
         cfg = gb.make_config(m, n, r, refresh_gap=1000, beta1=0.5, beta2=0.75, w_dtype="bf16", g_dtype=g_dtype,
                              state_fmt="q8", auto_refresh=False, q_block=q_block,
-                             path=gb.PATH_FP32 if mode == "fp32_path" else gb.PATH_TENSOR)
+                             path=gb.PATH_FP32 if mode == "fp32_path" else gb.PATH_TENSOR,
+                             adam_place=gb.ADAM_IN_PROJECTION if mode == "fused" else gb.ADAM_OWN_KERNEL)
         layer = gb.Layer(cfg)
         d = m if layer.side == gb.SIDE_LEFT else n
         P = _signed_permutation(d, r, rng)

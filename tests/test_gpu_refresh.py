@@ -166,3 +166,56 @@ def test_full_size_7b_refresh_meets_the_angle_bound_before_rounding():
     off = D - np.diag(np.diag(D))
     assert np.linalg.norm(off) < 1e-3 * np.linalg.norm(D)
     assert np.all(np.diff(np.diag(D)) <= 1e-6 * D[0, 0])
+
+
+@pytest.mark.parametrize("g_dtype,m,n,r", [("bf16", 512, 1376, 128), ("bf16", 1376, 512, 128), ("f32", 256, 640, 32)])
+def test_layers_refreshed_as_a_group_get_the_projectors_of_single_refreshes(g_dtype, m, n, r):
+    """galore_refresh_batch runs neighbours of one shape together (one launch per serial kernel for the whole
+    group, grouped tensor-core products).  Every layer keeps its own iteration count and schedule, so the
+    stored projector must equal, bit for bit, the one galore_refresh_projector computes for it alone.  The
+    gradients differ in spectrum (noise-dominated, gapped, low rank), hence in iterations and Jacobi sweeps;
+    a layer of another shape in the middle of the list splits the groups."""
+    k = min(m, n)
+    grads = [wl.make_gradient(m, n, wl.sub_seed(71, 0), 1.0, 0.01, g_dtype),
+             wl.make_gradient(m, n, wl.sub_seed(71, 1), 0.8, 0.05, g_dtype),
+             wl.make_planted(m, n, 72, np.concatenate([np.linspace(3, 2, r), 0.3 * np.arange(1, k - r + 1) ** -0.5]), g_dtype)[0],
+             wl.make_gradient(m, n, wl.sub_seed(71, 3), 1.0, 0.01, g_dtype),
+             wl.make_planted(m, n, 73, np.linspace(4, 1, r), g_dtype)[0],          # rank r: the block is rank-deficient
+             wl.make_gradient(m, n, wl.sub_seed(71, 5), 1.0, 0.02, g_dtype)]
+    other = wl.make_gradient(m // 2, n, wl.sub_seed(71, 9), 1.0, 0.01, g_dtype)
+    ld = (n + 15) // 16 * 16
+    Gd = [to_dev(g, g_dtype, ld) for g in grads]
+    Gd.insert(3, to_dev(other, g_dtype, ld))
+
+    def layers():
+        out = []
+        for i, g in enumerate(Gd):
+            mm = g.shape[0]
+            out.append(gb.Layer(gb.make_config(mm, n, min(r, mm, n), w_dtype="bf16", g_dtype=g_dtype, p_dtype="f32",
+                                               auto_refresh=False, seed=100 + i)))
+        return out
+    single, grouped = layers(), layers()
+    infos_single = []
+    for layer, g in zip(single, Gd):
+        st, info = layer.galore_refresh_projector(g)
+        assert st in (gb.OK, gb.WARN_NOT_CONVERGED)
+        infos_single.append(info.as_dict())
+    need = max(gb.galore_refresh_query_bytes(l) for l in grouped)
+    ws = torch.empty(4 * need, dtype=torch.uint8, device="cuda")          # room for groups of four
+    st, infos = gb.galore_refresh_batch(grouped, Gd, workspace=ws)
+    assert st in (gb.OK, gb.WARN_NOT_CONVERGED)
+    for a, b_, ia, ib in zip(single, grouped, infos_single, infos):
+        assert a.device_status() == b_.device_status()
+        assert torch.equal(a.get_projector(), b_.get_projector())
+        assert ia["iterations"] == ib.iterations and ia["jacobi_sweeps"] == ib.jacobi_sweeps
+        assert ia["converged"] == ib.converged and ia["sigma_r"] == ib.sigma_r
+    # and without a record (no phase clock, no residual) the projectors are the same again
+    again = layers()
+    lib_st = gb.lib().galore_refresh_batch((gb.C.c_void_p * len(again))(*[l.handle.value for l in again]),
+                                           (gb.C.c_void_p * len(again))(*[g.data_ptr() for g in Gd]),
+                                           (gb.C.c_int64 * len(again))(*[g.stride(0) for g in Gd]), len(again),
+                                           ws.data_ptr(), ws.numel(), None, None)
+    assert lib_st in (gb.OK, gb.WARN_NOT_CONVERGED)
+    torch.cuda.synchronize()
+    for a, c in zip(single, again):
+        assert torch.equal(a.get_projector(), c.get_projector())
