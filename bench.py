@@ -262,6 +262,8 @@ def main():
                     help="GaLore-AdamW: decoupled weight decay folded into the weight update (0 = plain Adam)")
     ap.add_argument("--adam-place", default="auto", choices=["auto", "projection", "own"],
                     help="where Adam on R runs when K is not sliced: in the projection kernel's epilogue or in its own kernel")
+    ap.add_argument("--refresh-slots", type=int, default=8,
+                    help="layers of one shape refreshed together by galore_refresh_batch (workspace copies; 1 = one by one)")
     ap.add_argument("--layers", type=int, default=0,
                     help="keep only this many transformer layers of the workload's layer set (0 = all): a small case "
                          "of the same kernels for profiler captures")
@@ -410,8 +412,10 @@ def time_workload(w, args, dev, dist, world, rank, full, mode=None):
     refresh_set = None
     if args.projector == "refresh":
         import time
+        # room for eight layers of one shape at a time: the library then refreshes them as a group
         need = max(gb.galore_refresh_query_bytes(l) for l in layers)
-        space = torch.empty(need, dtype=torch.uint8, device=dev)
+        slots = max(1, min(8, int(args.refresh_slots)))
+        space = torch.empty(slots * need, dtype=torch.uint8, device=dev)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         st, infos = gb.galore_refresh_batch(layers, Gs, stream=stream, workspace=space)
@@ -419,6 +423,7 @@ def time_workload(w, args, dev, dist, world, rank, full, mode=None):
         refresh_set = {"ms": (time.perf_counter() - t0) * 1e3, "matrices": len(layers), "status": st,
                        "not_converged": sum(1 for x in infos if not x.converged),
                        "iterations_max": max(x.iterations for x in infos),
+                       "slots": slots,
                        "timer": "host clock around the call, which returns when every refresh has finished"}
         del space
 

@@ -405,10 +405,12 @@ def galore_refresh_query_bytes(layer) -> int:
     return out.value
 
 
-def galore_refresh_batch(layers, Gs, stream=None, workspace=None):
-    """Refreshes the projectors of `layers` from `Gs`, one after another, through one shared workspace.
+def galore_refresh_batch(layers, Gs, stream=None, workspace=None, want_infos=True):
+    """Refreshes the projectors of `layers` from `Gs` through one shared workspace; neighbours of one shape are
+    refreshed together, as many at a time as the workspace holds copies of one layer's refresh workspace.
 
-    workspace: a uint8 CUDA tensor (allocated here when None).  Returns (status, infos).
+    workspace: a uint8 CUDA tensor (allocated here, for one layer at a time, when None).  Returns (status, infos);
+    without want_infos the library skips its phase clock and the residual diagnostic, and infos is [].
     """
     n = len(layers)
     need = max(galore_refresh_query_bytes(l) for l in layers)
@@ -417,10 +419,10 @@ def galore_refresh_batch(layers, Gs, stream=None, workspace=None):
     hs = (C.c_void_p * n)(*[l.handle.value for l in layers])
     gp = (C.c_void_p * n)(*[g.data_ptr() for g in Gs])
     lg = (C.c_int64 * n)(*[g.stride(0) for g in Gs])
-    infos = (RefreshInfo * n)()
+    infos = (RefreshInfo * n)() if want_infos else None
     st = _check(lib().galore_refresh_batch(hs, gp, lg, n, workspace.data_ptr(), workspace.numel(), _stream_ptr(stream),
                                            infos), "galore_refresh_batch")
-    return st, list(infos)
+    return st, (list(infos) if want_infos else [])
 
 
 def galore_batch_query_bytes(layers) -> int:

@@ -205,7 +205,12 @@ def test_export_import_resume_is_bit_identical(state_fmt, g_dtype, w_dtype):
         c.galore_step(Wc, g, 1e-2)
     torch.cuda.synchronize()
     assert torch.equal(Wc, Wa)
-    assert torch.equal(c.state, a.state)
+    # the states themselves (the raw buffers also hold alignment padding that nothing writes)
+    assert torch.equal(c.get_projector(), a.get_projector())
+    if state_fmt == "q8":
+        assert all(torch.equal(x, y) for x, y in zip(c.get_q8_state(), a.get_q8_state()))
+    else:
+        assert all(torch.equal(x, y) for x, y in zip(c.get_moments(), a.get_moments()))
     # a blob of another configuration is refused, a truncated or foreign one too
     other = gb.Layer(gb.make_config(m, n, r + 8, refresh_gap=T, w_dtype=w_dtype, g_dtype=g_dtype, state_fmt=state_fmt))
     with pytest.raises(gb.GaloreError) as e:
