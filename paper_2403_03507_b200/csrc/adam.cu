@@ -239,9 +239,9 @@ __device__ __forceinline__ void load_r(const AdamItem& a, int64_t off, bool fast
 
 // ---- fp32 moments -------------------------------------------------------------
 template <typename TN>
-__device__ __forceinline__ bool adam_f32_tile(const AdamItem& a, int tile) {
+__device__ __forceinline__ bool adam_f32_tile(const AdamItem& a, int b) {
   constexpr int E = 8;
-  const TileThread<E> tt(tile / a.tiles_c, tile % a.tiles_c);
+  const TileThread<E> tt(a.sub_r0 + b / a.sub_nc, a.sub_c0 + b % a.sub_nc);
   const int valid = tt.row < a.rows ? min(E, a.cols - tt.col) : 0;     // elements of the run inside the matrix
   if (valid <= 0) return false;
   const bool fast = a.vec && valid == E;
@@ -305,11 +305,15 @@ __global__ void __launch_bounds__(256, GALORE_F32_CTAS) adam_f32_kernel(const __
 #define GALORE_Q8_CTAS 4          // resident CTAs per SM the kernel is compiled for (register budget)
 #endif
 
-template <typename TN, int E>
-__device__ __forceinline__ bool adam_q8_tile(const AdamItem& a, int tile, Q8Tables& t, int parity) {
-  const TileThread<E> tt(tile / a.tiles_c, tile % a.tiles_c);
-  const int valid = tt.row < a.rows ? max(0, min(E, a.cols - tt.col)) : 0;
-  const bool fast = a.vec && valid == E;
+// FAST: the launch holds interior tiles of layers whose arrays allow vector accesses only, so nothing
+// is predicated (fewer registers: one more resident CTA per SM).
+template <typename TN, int E, bool FAST>
+__device__ __forceinline__ bool adam_q8_tile(const AdamItem& a, int b, Q8Tables& t, int parity) {
+  const int tile_r = a.sub_r0 + b / a.sub_nc, tile_c = a.sub_c0 + b % a.sub_nc;
+  const int tile = tile_r * a.tiles_c + tile_c;
+  const TileThread<E> tt(tile_r, tile_c);
+  const int valid = FAST ? E : (tt.row < a.rows ? max(0, min(E, a.cols - tt.col)) : 0);
+  const bool fast = FAST || (a.vec && valid == E);
   const AdamParams p = a.p;
   const int64_t so = (int64_t)tt.row * a.s_ld + tt.col;
   const float am_m = a.Mam[tile], am_v = a.Vam[tile];
@@ -380,8 +384,13 @@ __device__ __forceinline__ bool adam_q8_tile(const AdamItem& a, int tile, Q8Tabl
   return bad;
 }
 
-template <typename TN, int E>
-__global__ void __launch_bounds__(256, GALORE_Q8_CTAS) adam_q8_kernel(const __grid_constant__ AdamGroup g, const Q8TablePtrs tp) {
+#ifndef GALORE_Q8_FAST_CTAS
+#define GALORE_Q8_FAST_CTAS 6       // 40 registers with a few spills: 7.0 ms for the LLaMA-7B set against 7.5 ms at 5 or 4 (32 KiB of tables per CTA: 6 is what fits)
+#endif
+constexpr int q8_ctas(bool fast) { return fast ? GALORE_Q8_FAST_CTAS : GALORE_Q8_CTAS; }
+
+template <typename TN, int E, bool FAST>
+__global__ void __launch_bounds__(256, q8_ctas(FAST)) adam_q8_kernel(const __grid_constant__ AdamGroup g, const Q8TablePtrs tp) {
   __shared__ Q8Tables t;
   q8_tables_fill(t, tp, threadIdx.x, 256);
   __syncthreads();
@@ -391,7 +400,7 @@ __global__ void __launch_bounds__(256, GALORE_Q8_CTAS) adam_q8_kernel(const __gr
   for (int gb = blockIdx.x; gb < total; gb += gridDim.x, parity ^= 1) {
     int tile;
     find_item(g, gb, it, tile);
-    if (adam_q8_tile<TN, E>(g.item[it], tile, t, parity)) bad_item = it;   // per thread: a non-finite input is reported by the threads that met it
+    if (adam_q8_tile<TN, E, FAST>(g.item[it], tile, t, parity)) bad_item = it;   // per thread: a non-finite input is reported by the threads that met it
   }
   if (bad_item >= 0) atomicOr(g.item[bad_item].status, GALORE_DEV_NONFINITE);
 }
@@ -469,27 +478,66 @@ galore_status_t launch_adam_group(const AdamGroup& g, int32_t state_fmt, int q_b
   if (!valid_block(q_block)) return GALORE_ERR_INVALID_ARG;
   Q8TablePtrs tp;
   GALORE_TRY(q8_table_ptrs(&tp));
-  // one resident wave: the 32 KiB of tables are set up once per SM slot
-  const unsigned grid = (unsigned)std::min(total, 148 * GALORE_Q8_CTAS);
-#define GALORE_Q8_LAUNCH(TN, E)                                                                              \
-  do {                                                                                                       \
-    GALORE_CUDA_TRY(cudaFuncSetAttribute(adam_q8_kernel<TN, E>, cudaFuncAttributePreferredSharedMemoryCarveout, \
-                                         cudaSharedmemCarveoutMaxShared));                                   \
-    adam_q8_kernel<TN, E><<<grid, 256, 0, st>>>(g, tp);                                                      \
-    GALORE_LAUNCH_CHECK();                                                                                   \
+  // The interior tiles of layers whose arrays allow vector accesses go to the kernel that holds the
+  // unpredicated code alone; the ragged right and bottom strips and everything else to the general one.
+  const int tile_rows = q_block / kStateTileCols;
+  std::unique_ptr<AdamGroup> fast(new AdamGroup), rest(new AdamGroup);
+  fast->count = rest->count = 0;
+  auto launch = [&](const AdamGroup& grp, bool is_fast) -> galore_status_t {
+    if (grp.count == 0) return GALORE_OK;
+    const int blocks = grp.block_end[grp.count - 1];
+    // one resident wave: the 32 KiB of tables are set up once per SM slot
+    const unsigned grid = (unsigned)std::min(blocks, 148 * q8_ctas(is_fast));
+#define GALORE_Q8_LAUNCH(TN, E, F)                                                                              \
+  do {                                                                                                          \
+    GALORE_CUDA_TRY(cudaFuncSetAttribute(adam_q8_kernel<TN, E, F>, cudaFuncAttributePreferredSharedMemoryCarveout, \
+                                         cudaSharedmemCarveoutMaxShared));                                      \
+    adam_q8_kernel<TN, E, F><<<grid, 256, 0, st>>>(grp, tp);                                                    \
+    GALORE_LAUNCH_CHECK();                                                                                      \
   } while (0)
-#define GALORE_Q8_CASE(E)                                 \
-  case E * 256:                                           \
-    if (nb) GALORE_Q8_LAUNCH(__nv_bfloat16, E);           \
-    else GALORE_Q8_LAUNCH(float, E);                      \
+#define GALORE_Q8_CASE(E)                                        \
+  case E * 256:                                                  \
+    if (nb && is_fast) GALORE_Q8_LAUNCH(__nv_bfloat16, E, true); \
+    else if (nb) GALORE_Q8_LAUNCH(__nv_bfloat16, E, false);      \
+    else if (is_fast) GALORE_Q8_LAUNCH(float, E, true);          \
+    else GALORE_Q8_LAUNCH(float, E, false);                      \
     break;
-  switch (q_block) {
-    GALORE_Q8_CASE(1) GALORE_Q8_CASE(2) GALORE_Q8_CASE(4) GALORE_Q8_CASE(8)
-    default: return GALORE_ERR_INVALID_ARG;
-  }
+    switch (q_block) {
+      GALORE_Q8_CASE(1) GALORE_Q8_CASE(2) GALORE_Q8_CASE(4) GALORE_Q8_CASE(8)
+      default: return GALORE_ERR_INVALID_ARG;
+    }
 #undef GALORE_Q8_CASE
 #undef GALORE_Q8_LAUNCH
-  return GALORE_OK;
+    return GALORE_OK;
+  };
+  auto append = [&](AdamGroup& dst, bool is_fast, const AdamItem& a, int r0, int c0, int nr, int nc) -> galore_status_t {
+    if (nr <= 0 || nc <= 0) return GALORE_OK;
+    if (dst.count == kAdamGroup) {            // full: send what has been collected and start again
+      GALORE_TRY(launch(dst, is_fast));
+      dst.count = 0;
+    }
+    const int j = dst.count++;
+    dst.item[j] = a;
+    dst.item[j].sub_r0 = r0;
+    dst.item[j].sub_c0 = c0;
+    dst.item[j].sub_nc = nc;
+    dst.block_end[j] = (j > 0 ? dst.block_end[j - 1] : 0) + nr * nc;
+    return GALORE_OK;
+  };
+  for (int i = 0; i < g.count; ++i) {
+    const AdamItem& a = g.item[i];
+    const int tr = (int)ceil_div(a.rows, tile_rows), tc = a.tiles_c;
+    const int full_r = a.rows / tile_rows, full_c = a.cols / kStateTileCols;
+    if (a.vec) {
+      GALORE_TRY(append(*fast, true, a, 0, 0, full_r, full_c));
+      GALORE_TRY(append(*rest, false, a, 0, full_c, tr, tc - full_c));            // ragged right strip
+      GALORE_TRY(append(*rest, false, a, full_r, 0, tr - full_r, full_c));        // ragged bottom strip
+    } else {
+      GALORE_TRY(append(*rest, false, a, 0, 0, tr, tc));
+    }
+  }
+  GALORE_TRY(launch(*fast, true));
+  return launch(*rest, false);
 }
 
 galore_status_t adam_group_add(AdamGroup& g, const AdamItem& item, int32_t state_fmt, int q_block) {
@@ -508,6 +556,8 @@ galore_status_t adam_group_add(AdamGroup& g, const AdamItem& item, int32_t state
   const bool pitches = (a.r_ld % 4) == 0 && (a.n_ld % 8) == 0 && (a.split_stride % 4) == 0 &&
                        (a.s_ld % (state_fmt == GALORE_STATE_F32 ? 4 : 16)) == 0;
   a.vec = ((bases & 15) == 0 && pitches) ? 1 : 0;
+  a.sub_r0 = a.sub_c0 = 0;
+  a.sub_nc = a.tiles_c;
   const int i = g.count++;
   g.item[i] = a;
   g.block_end[i] = (int)(before + tiles);

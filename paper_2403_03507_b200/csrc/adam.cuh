@@ -22,6 +22,7 @@ struct AdamItem {
   void* Nout;              // normalised update (fp32 or bf16)
   int tiles_c;             // set by adam_group_add: ceil(cols / 64)
   int vec;                 // set by adam_group_add: bases and pitches allow the vector accesses of an interior tile
+  int sub_r0, sub_c0, sub_nc;  // the item covers the tiles (sub_r0 + b / sub_nc, sub_c0 + b % sub_nc), b = 0, 1, ...
   AdamParams p;
   int32_t* status;
 };

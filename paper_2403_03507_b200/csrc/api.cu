@@ -484,15 +484,7 @@ galore_status_t galore_step(galore_layer_t* l, void* W, int64_t ldw, const void*
     warn = s;
   }
   if (!l->has_projector) return GALORE_ERR_STATE;
-  const double t = (double)(l->k + 1);
-  AdamParams ap;
-  ap.b1 = (float)l->cfg.beta1;
-  ap.b2 = (float)l->cfg.beta2;
-  ap.omb1 = (float)(1.0 - l->cfg.beta1);
-  ap.omb2 = (float)(1.0 - l->cfg.beta2);
-  ap.eps = (float)l->cfg.eps;
-  ap.inv_bc1 = (float)(1.0 / (1.0 - pow(l->cfg.beta1, t)));
-  ap.inv_bc2 = (float)(1.0 / (1.0 - pow(l->cfg.beta2, t)));
+  const AdamParams ap = make_adam_params(l->cfg.beta1, l->cfg.beta2, l->cfg.eps, (double)(l->k + 1));
   galore_status_t s;
   if (l->tensor_path && tensor_operands_aligned(l->cfg, W, ldw, G, ldg)) {
     s = step_tensor(l, W, ldw, G, ldg, lr, ap, st);
@@ -655,16 +647,7 @@ bool batch_eligible(const galore_layer* l, const void* W, int64_t ldw, const voi
 }
 
 AdamParams adam_params(const galore_layer* l) {
-  const double t = (double)(l->k + 1);
-  AdamParams ap;
-  ap.b1 = (float)l->cfg.beta1;
-  ap.b2 = (float)l->cfg.beta2;
-  ap.omb1 = (float)(1.0 - l->cfg.beta1);
-  ap.omb2 = (float)(1.0 - l->cfg.beta2);
-  ap.eps = (float)l->cfg.eps;
-  ap.inv_bc1 = (float)(1.0 / (1.0 - pow(l->cfg.beta1, t)));
-  ap.inv_bc2 = (float)(1.0 / (1.0 - pow(l->cfg.beta2, t)));
-  return ap;
+  return make_adam_params(l->cfg.beta1, l->cfg.beta2, l->cfg.eps, (double)(l->k + 1));
 }
 
 struct BatchScratch {   // host-side objects reused across calls on this thread

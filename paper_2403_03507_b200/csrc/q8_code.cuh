@@ -3,6 +3,8 @@
 // states; the format is this library's).
 #pragma once
 
+#include <math.h>
+
 #include "common.cuh"
 
 namespace galore {
@@ -117,13 +119,31 @@ struct AdamParams {
   float omb1, omb2;      // 1 - beta1, 1 - beta2
   float eps;
   float inv_bc1, inv_bc2;  // 1 / (1 - beta^t), t = completed steps + 1
+  float nrm_a, nrm_b;      // Eq. 15 as m / (nrm_a sqrt(v) + nrm_b): sqrt(inv_bc2) / inv_bc1 and eps / inv_bc1
 };
+// fills the derived fields; beta1, beta2, eps as given by the caller, t = completed steps + 1
+inline AdamParams make_adam_params(double beta1, double beta2, double eps, double t) {
+  AdamParams ap;
+  ap.b1 = (float)beta1;
+  ap.b2 = (float)beta2;
+  ap.omb1 = (float)(1.0 - beta1);
+  ap.omb2 = (float)(1.0 - beta2);
+  ap.eps = (float)eps;
+  const double ibc1 = 1.0 / (1.0 - pow(beta1, t)), ibc2 = 1.0 / (1.0 - pow(beta2, t));
+  ap.inv_bc1 = (float)ibc1;
+  ap.inv_bc2 = (float)ibc2;
+  ap.nrm_a = (float)(sqrt(ibc2) / ibc1);
+  ap.nrm_b = (float)(eps / ibc1);
+  return ap;
+}
 
+// N = [m / (1 - b1^t)] / (sqrt(v / (1 - b2^t)) + eps), with the two corrections folded into the
+// constants of one multiply-add: m / (nrm_a sqrt(v) + nrm_b).
 __device__ __forceinline__ float adam_normalised(float m, float v, const AdamParams& p) {
   float root, inv;
-  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(root) : "f"(v * p.inv_bc2));
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(root + p.eps));
-  return (m * p.inv_bc1) * inv;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(root) : "f"(v));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(fmaf(root, p.nrm_a, p.nrm_b)));
+  return m * inv;
 }
 
 // The moment updates of Algorithm 1 with the rounding order fixed (no contraction left to the

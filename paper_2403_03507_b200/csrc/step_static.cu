@@ -123,15 +123,7 @@ extern "C" galore_status_t galore_step_static(int64_t m, int64_t n, int32_t rank
   else
     GALORE_TRY((launch_gemm_simt<float, float, float>((int)m, r, (int)n, G, ldg, 1, P, r, 1, splits, epi, st)));
 
-  const double t = (double)(completed_steps + 1);
-  AdamParams ap;
-  ap.b1 = (float)beta1;
-  ap.b2 = (float)beta2;
-  ap.omb1 = (float)(1.0 - beta1);
-  ap.omb2 = (float)(1.0 - beta2);
-  ap.eps = (float)eps;
-  ap.inv_bc1 = (float)(1.0 / (1.0 - pow(beta1, t)));
-  ap.inv_bc2 = (float)(1.0 / (1.0 - pow(beta2, t)));
+  const AdamParams ap = make_adam_params(beta1, beta2, eps, (double)(completed_steps + 1));
   AdamItem item = {};
   item.Rpart = Rpart; item.splits = splits; item.split_stride = nel;
   item.rows = (int)srows; item.cols = (int)scols;
