@@ -269,6 +269,9 @@ def main():
                          "of the same kernels for profiler captures")
     ap.add_argument("--rank", type=int, default=0, help="override the workload's rank (rank sweep on one shape)")
     ap.add_argument("--state-fmt", default="", choices=["", "f32", "q8"], help="override the workload's state format")
+    ap.add_argument("--refresh-warm", type=int, default=0,
+                    help="power steps of a refresh started from the stored projector (0: every refresh starts cold); "
+                         "with N > 0 the whole set is also refreshed a second time from slightly moved gradients")
     ap.add_argument("--refresh-only", action="store_true",
                     help="run the projector refresh of each distinct shape and print its timings; no step is timed "
                          "(for profiling the refresh on its own)")
@@ -359,6 +362,7 @@ def time_workload(w, args, dev, dist, world, rank, full, mode=None):
         cfg = gb.make_config(m, n, w.rank, alpha=w.alpha, refresh_gap=w.refresh_gap, beta1=w.beta1, beta2=w.beta2,
                              eps=w.eps, w_dtype=w.w_dtype, g_dtype=w.g_dtype, state_fmt=w.state_fmt,
                              q_block=w.q_block, auto_refresh=False, seed=w.seed, weight_decay=args.weight_decay,
+                             refresh_warm_iters=args.refresh_warm,
                              adam_place={"auto": gb.ADAM_AUTO, "projection": gb.ADAM_IN_PROJECTION, "own": gb.ADAM_OWN_KERNEL}[args.adam_place])
         cfgs[(m, n)] = cfg
         max_ws = max(max_ws, gb.galore_query_bytes(cfg)[1])
@@ -393,7 +397,7 @@ def time_workload(w, args, dev, dist, world, rank, full, mode=None):
                 first = layer.get_projector()
                 if args.refresh_only:
                     break
-            else:
+            elif args.projector == "random":
                 layer.set_projector(first)                              # timing does not depend on P's values
             Wt = padded(m, n, tdt[w.w_dtype])
             Wt.copy_(torch.randn(m, n, device=dev) * 0.02)
@@ -425,6 +429,23 @@ def time_workload(w, args, dev, dist, world, rank, full, mode=None):
                        "iterations_max": max(x.iterations for x in infos),
                        "slots": slots,
                        "timer": "host clock around the call, which returns when every refresh has finished"}
+        if args.refresh_warm > 0:
+            # The next refresh of training sees gradients whose subspace has moved a little (Sec. 4.1): every
+            # gradient gets 2 % of its rms as fresh noise, then the set is refreshed again from its projectors.
+            gen = torch.Generator(device=dev)
+            gen.manual_seed(w.seed + 17)
+            for g in {x.data_ptr(): x for x in Gs}.values():
+                rms = g.float().pow(2).mean().sqrt().item()
+                g.add_((torch.randn(g.shape, device=dev, generator=gen) * (0.02 * rms)).to(g.dtype))
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            st, infos = gb.galore_refresh_batch(layers, Gs, stream=stream, workspace=space)
+            torch.cuda.synchronize()
+            refresh_set["warm_start"] = {"ms": (time.perf_counter() - t0) * 1e3, "status": st, "first_steps": args.refresh_warm,
+                                         "not_converged": sum(1 for x in infos if not x.converged),
+                                         "iterations_max": max(x.iterations for x in infos),
+                                         "iterations_mean": sum(x.iterations for x in infos) / len(infos),
+                                         "gradients": "the cold refresh's plus 2 % of their rms as fresh noise"}
         del space
 
     batch = gb.Batch(layers, Ws, Gs, device=dev) if mode == "batch" else None

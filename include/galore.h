@@ -117,7 +117,14 @@ typedef struct {
    * library choose per state format; IN_PROJECTION runs it in the projection kernel's epilogue (R is
    * never stored); OWN_KERNEL always uses the stand-alone Adam kernel after the projection. */
   int32_t adam_place;
-  int32_t reserved[6];
+  /* Warm-started refresh (the subspace of consecutive gradients changes slowly, Sec. 4.1): > 0 makes
+   * every refresh of a layer that already has a projector start from that projector (plus random
+   * columns for the oversampling) and run this many power steps before its Rayleigh-Ritz pass.  The
+   * result is then judged by its own residual: residual over spectral gap bounds the angle to the
+   * exact subspace; within 10 x refresh_tol the refresh ends there, otherwise it continues like a
+   * cold one.  0 = always start from a random block. */
+  int32_t refresh_warm_iters;
+  int32_t reserved[5];
 } galore_config_t;
 
 /* Result of one refresh (host struct, filled after the refresh's stream work has completed). */

@@ -35,7 +35,7 @@ class Config(C.Structure):
         ("side", C.c_int32), ("w_dtype", C.c_int32), ("g_dtype", C.c_int32), ("p_dtype", C.c_int32),
         ("state_fmt", C.c_int32), ("q_block", C.c_int32), ("auto_refresh", C.c_int32), ("path", C.c_int32),
         ("refresh_tol", C.c_float), ("refresh_max_iters", C.c_int32), ("refresh_oversample", C.c_int32),
-        ("seed", C.c_uint64), ("weight_decay", C.c_float), ("adam_place", C.c_int32), ("reserved", C.c_int32 * 6),
+        ("seed", C.c_uint64), ("weight_decay", C.c_float), ("adam_place", C.c_int32), ("refresh_warm_iters", C.c_int32), ("reserved", C.c_int32 * 5),
     ]
 
 
@@ -143,7 +143,7 @@ def _stream_ptr(stream=None):
 def make_config(m, n, rank, alpha=0.25, refresh_gap=200, beta1=0.9, beta2=0.999, eps=1e-8, side=SIDE_AUTO,
                 w_dtype="bf16", g_dtype="bf16", p_dtype=None, state_fmt="f32", q_block=2048, auto_refresh=True,
                 path=PATH_AUTO, refresh_tol=0.0, refresh_max_iters=0, refresh_oversample=0, seed=0,
-                weight_decay=0.0, adam_place=ADAM_AUTO) -> Config:
+                weight_decay=0.0, adam_place=ADAM_AUTO, refresh_warm_iters=0) -> Config:
     c = Config()
     c.m, c.n, c.rank, c.alpha, c.refresh_gap = m, n, rank, alpha, refresh_gap
     c.beta1, c.beta2, c.eps = beta1, beta2, eps
@@ -157,6 +157,7 @@ def make_config(m, n, rank, alpha=0.25, refresh_gap=200, beta1=0.9, beta2=0.999,
     c.refresh_tol, c.refresh_max_iters, c.refresh_oversample, c.seed = refresh_tol, refresh_max_iters, refresh_oversample, seed
     c.weight_decay = weight_decay
     c.adam_place = adam_place
+    c.refresh_warm_iters = refresh_warm_iters
     return c
 
 

@@ -120,6 +120,7 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
   if (c->state_fmt != GALORE_STATE_F32 && c->state_fmt != GALORE_STATE_Q8_BLOCK) return GALORE_ERR_INVALID_ARG;
   if (c->path < GALORE_PATH_AUTO || c->path > GALORE_PATH_TENSOR) return GALORE_ERR_INVALID_ARG;
   if (c->adam_place < GALORE_ADAM_AUTO || c->adam_place > GALORE_ADAM_OWN_KERNEL) return GALORE_ERR_INVALID_ARG;
+  if (c->refresh_warm_iters < 0) return GALORE_ERR_INVALID_ARG;
   s->q_block = c->q_block == 0 ? 2048 : c->q_block;
   if (s->q_block != 256 && s->q_block != 512 && s->q_block != 1024 && s->q_block != 2048)
     return GALORE_ERR_INVALID_ARG;
@@ -324,6 +325,7 @@ RefreshProblem refresh_problem(const galore_layer* l, const void* G, int64_t ldg
   pr.max_iters = l->cfg.refresh_max_iters > 0 ? l->cfg.refresh_max_iters : 96;
   pr.first_iters = 6;
   pr.use_tensor = l->tensor_path;
+  pr.warm_iters = (l->cfg.refresh_warm_iters > 0 && l->has_projector) ? l->cfg.refresh_warm_iters : 0;
   return pr;
 }
 

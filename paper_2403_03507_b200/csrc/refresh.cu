@@ -57,6 +57,13 @@ __global__ void fill_normal_kernel(float* __restrict__ Y, int64_t count, uint64_
   }
 }
 
+// first r columns of the start block <- the projector of the previous refresh (rows x r, packed)
+template <typename TP>
+__global__ void place_previous_kernel(float* __restrict__ Y, const TP* __restrict__ P, int64_t rows, int r, int b) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < rows * r; i += (int64_t)gridDim.x * blockDim.x)
+    Y[(i / r) * b + (i % r)] = cvt<float>(P[i]);
+}
+
 __global__ void set_identity_kernel(double* __restrict__ A, int n) {
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < (int64_t)n * n; i += (int64_t)gridDim.x * blockDim.x)
     A[i] = (i / n == i % n) ? 1.0 : 0.0;
@@ -520,8 +527,12 @@ struct Lane {
   TensorRefresh tr;
   int q_done = 0, q_target = 0, orth_every = 1;
   std::vector<double> theta;
-  double predicted = 0.0;
+  double predicted = 0.0, res_abs = 0.0;
   bool converged = false, with_vt = false, iterating = true;
+  bool p64_current = false;   // P64 holds the Ritz vectors of the lane's last Rayleigh-Ritz pass
+  bool warm_check = false;    // started from the previous projector: the first Rayleigh-Ritz pass is judged by its residual
+  int warm_from = 0;          // steps done when the warm start was judged, and the error bound found there
+  double warm_bound = 1.0;    // (a cold start: 0 steps, error 1)
   galore_refresh_info_t info = {};
 };
 
@@ -862,10 +873,35 @@ static galore_status_t refresh_group(const RefreshProblem* prs, int count, void*
     return GALORE_OK;
   };
 
+  // power steps for the given lanes, every lane up to its own target on its own orthonormalisation schedule
+  auto run_steps = [&](const std::vector<Lane*>& lanes) -> galore_status_t {
+    for (;;) {
+      std::vector<Lane*> stepping, orth;
+      for (Lane* l : lanes)
+        if (l->q_done < l->q_target) {
+          stepping.push_back(l);
+          if (((l->q_target - 1 - l->q_done) % l->orth_every) == 0) orth.push_back(l);   // the last step always ends orthonormal
+        }
+      if (stepping.empty()) return GALORE_OK;
+      GALORE_TRY(step(stepping, orth));
+      for (Lane* l : stepping) l->q_done += 1;
+    }
+  };
+
   if (!full_space) {
     for (Lane* l : all) {
       fill_normal_kernel<<<grid_for(yb), 256, 0, st>>>(l->Y, yb, l->pr.seed);
       GALORE_LAUNCH_CHECK();
+      if (l->pr.warm_iters > 0) {
+        // Warm start (the subspace of consecutive gradients changes slowly, Sec. 4.1): the stored
+        // projector spans most of what is wanted already, the random columns carry the oversampling.
+        l->warm_check = true;
+        if (l->pr.p_dtype == GALORE_BF16)
+          place_previous_kernel<__nv_bfloat16><<<grid_for(d * r), 256, 0, st>>>(l->Y, (const __nv_bfloat16*)l->pr.P, d, r, b);
+        else
+          place_previous_kernel<float><<<grid_for(d * r), 256, 0, st>>>(l->Y, (const float*)l->pr.P, d, r, b);
+        GALORE_LAUNCH_CHECK();
+      }
       if (tensor) {
         split_kernel<<<grid_for(yb), 256, 0, st>>>(l->Y, l->w.Yhi, l->w.Ylo, yb);
         GALORE_LAUNCH_CHECK();
@@ -883,11 +919,19 @@ static galore_status_t refresh_group(const RefreshProblem* prs, int count, void*
     // block's columns.  Sorted, they stand in for the Ritz values: enough to size the iteration
     // (their spread is narrower than the spectrum's, which errs towards more steps) and to decide
     // how many steps may be chained before the block has to be orthonormalised again.
-    const int q0 = std::min(p0.max_iters, std::max(1, p0.first_iters));
-    for (int q = 0; q < q0; ++q) GALORE_TRY(step(all, all));
-    for (Lane* l : all) l->q_done = l->q_target = q0;
-    if (b > r && q0 < p0.max_iters) {
-      for (Lane* l : all) {
+    // A warm-started lane runs its given number of steps first.  If the look says that a cold start
+    // would need no more than twice that, the lane goes to Rayleigh-Ritz and is judged by its residual;
+    // otherwise (no gap behind the block: the gradient is dominated by noise) it carries on as a cold
+    // one, which costs it nothing but keeps what its start already spans.
+    for (Lane* l : all)
+      l->q_target = l->warm_check ? std::min(l->pr.max_iters, l->pr.warm_iters)
+                                  : std::min(l->pr.max_iters, std::max(1, l->pr.first_iters));
+    GALORE_TRY(run_steps(all));
+    if (b > r) {
+      std::vector<Lane*> sized;
+      for (Lane* l : all)
+        if (l->q_done < l->pr.max_iters) sized.push_back(l);
+      for (Lane* l : sized) {
         double* slices = (double*)l->w.Y64;                      // kColSlices x b doubles, Y64 is idle here
         const float* z0 = (const float*)l->w.Zu;
         const float* z1 = tensor ? z0 + L * b : nullptr;
@@ -898,16 +942,14 @@ static galore_status_t refresh_group(const RefreshProblem* prs, int count, void*
         rank_desc_kernel<<<(unsigned)ceil_div(b, 128), 128, 0, st>>>(l->w.lam, b, l->w.theta, l->w.order);
         GALORE_LAUNCH_CHECK();
       }
-      GALORE_TRY(read_theta(all));
-      for (Lane* l : all) {
+      if (!sized.empty()) GALORE_TRY(read_theta(sized));
+      for (Lane* l : sized) {
         const std::vector<double>& theta = l->theta;
         const double ratio = theta[r - 1] > 0.0 ? theta[b - 1] / theta[r - 1] : 1.0;
-        if (ratio > 0.0 && ratio < 1.0) {
-          const int need = (int)ceil(log(l->pr.tol) / log(ratio)) + 1;
-          l->q_target = std::min(l->pr.max_iters, std::max(need, l->q_done));
-        } else if (ratio >= 1.0) {
-          l->q_target = l->pr.max_iters;
-        }
+        const int need = (ratio > 0.0 && ratio < 1.0) ? (int)ceil(log(l->pr.tol) / log(ratio)) + 1
+                                                      : (ratio >= 1.0 ? l->pr.max_iters : l->q_done);
+        if (l->warm_check && need > 2 * l->q_done) l->warm_check = false;
+        if (!l->warm_check) l->q_target = std::min(l->pr.max_iters, std::max(need, l->q_done));
         if (tensor && theta[b - 1] > 0.0) {
           // chained steps multiply the block's condition number by theta_1/theta_b each; the bf16 pair
           // carries 16 bits and the Gram matrix squares the product, so keep it below about 100
@@ -919,20 +961,70 @@ static galore_status_t refresh_group(const RefreshProblem* prs, int count, void*
     }
   }
 
+  // P64 = Y64 S[:, top r] from the last Rayleigh-Ritz pass of the given lanes
+  const int64_t pc = d * r;
+  auto make_p64 = [&](const std::vector<Lane*>& lanes) -> galore_status_t {
+    if (lanes.empty()) return GALORE_OK;
+    for (Lane* l : lanes) {
+      const RefreshBuffers& w = l->w;
+      l->p64_current = true;
+      if (l->with_vt)
+        gather_rows_kernel<<<r, 256, 0, st>>>(w.Vt, w.order, b, w.Vsel);
+      else
+        gather_rows_scaled_kernel<<<r, 256, 0, st>>>(w.H, w.lam, w.order, b, w.Vsel);
+      GALORE_LAUNCH_CHECK();
+    }
+    EpiStore<double, double> epi{c.w0.P64, r, 0, 1.0, 0.0};
+    const SlotList sl = slots_of(c, lanes);
+    return launch_gemm_dmma<double, double>((int)d, r, b, c.w0.Y64, b, 1, c.w0.Vsel, 1, b, epi, st, 1, 0, 0, &sl);
+  };
+  // res_abs = || A A^T P - P Theta ||_F of the given lanes (after make_p64; synchronises the stream).
+  // On the tensor path A^T P = Z S is formed from the products already at hand and A (A^T P) runs on
+  // the tensor cores in bf16 pairs.  Leaves the iteration's block Y untouched.
+  auto residuals = [&](const std::vector<Lane*>& lanes) -> galore_status_t {
+    if (lanes.empty()) return GALORE_OK;
+    const bool tensor_residual = tensor && (r % 8) == 0;
+    for (Lane* l : lanes) {
+      const RefreshBuffers& w = l->w;
+      const TG* G = (const TG*)l->pr.G;
+      const int64_t sAi = c.left ? l->pr.ldg : 1, sAl = c.left ? 1 : l->pr.ldg;
+      if (tensor_residual) {
+        EpiSplitPair e1{w.Zhi, w.Zlo, r};
+        GALORE_TRY((launch_gemm_dmma<double, double>((int)L, r, b, (const double*)w.Zu, b, 1, w.Vsel, 1, b, e1, st)));
+        const int a_mn = c.left ? 0 : 1;
+        const int s1 = (l->tr.master + 1) % 3, s2 = (l->tr.master + 2) % 3;
+        tensor_group_reset(c.tg);
+        GALORE_TRY(tensor_group_add_gemm(c.tg, l->pr.G, l->pr.ldg, a_mn, w.Zhi, r, 1, (int)d, r, (int)L, l->tr.F[s1], r, l->status));
+        GALORE_TRY(tensor_group_add_gemm(c.tg, l->pr.G, l->pr.ldg, a_mn, w.Zlo, r, 1, (int)d, r, (int)L, l->tr.F[s2], r, l->status));
+        GALORE_TRY(tensor_group_launch_project(c.tg, st));
+        GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
+        residual_pair_kernel<<<grid_for(d * r), 256, 0, st>>>(l->tr.F[s1], l->tr.F[s2], w.P64, w.theta, d, r, w.scal);
+        GALORE_LAUNCH_CHECK();
+      } else {
+        double* T1 = (double*)w.Zu;   // L x r
+        double* T2 = w.Y64;           // d x r (Y64 is no longer needed once P64 exists)
+        EpiStore<double, double> e1{T1, r, 0, 1.0, 0.0};
+        GALORE_TRY((launch_gemm_dmma<TG, double>((int)L, r, (int)d, G, sAl, sAi, w.P64, r, 1, e1, st)));
+        EpiStore<double, double> e2{T2, r, 0, 1.0, 0.0};
+        GALORE_TRY((launch_gemm_dmma<TG, double>((int)d, r, (int)L, G, sAi, sAl, T1, r, 1, e2, st)));
+        GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
+        residual_kernel<<<grid_for(pc), 256, 0, st>>>(T2, w.P64, w.theta, d, r, w.scal);
+        GALORE_LAUNCH_CHECK();
+      }
+    }
+    std::vector<double> sc(2 * lanes.size(), 0.0);
+    for (size_t i = 0; i < lanes.size(); ++i)
+      GALORE_CUDA_TRY(cudaMemcpyAsync(&sc[2 * i], lanes[i]->w.scal, 2 * sizeof(double), cudaMemcpyDeviceToHost, st));
+    GALORE_CUDA_TRY(cudaStreamSynchronize(st));
+    for (size_t i = 0; i < lanes.size(); ++i) lanes[i]->res_abs = sqrt(sc[2 * i + 1]);
+    return GALORE_OK;
+  };
+
   std::vector<Lane*> live = all;            // lanes that still iterate
   while (!live.empty()) {
     // ---- power steps: every lane up to its own target, on its own orthonormalisation schedule ----
-    for (;;) {
-      std::vector<Lane*> stepping, orth;
-      for (Lane* l : live)
-        if (l->q_done < l->q_target) {
-          stepping.push_back(l);
-          if (((l->q_target - 1 - l->q_done) % l->orth_every) == 0) orth.push_back(l);   // the last step always ends orthonormal
-        }
-      if (stepping.empty()) break;
-      GALORE_TRY(step(stepping, orth));
-      for (Lane* l : stepping) l->q_done += 1;
-    }
+    GALORE_TRY(run_steps(live));
+    for (Lane* l : live) l->p64_current = false;
     // ---- Rayleigh-Ritz in fp64 --------------------------------------------------
     const clk::time_point t_rr = now_synced();
     ms_power = ms_between(t_begin, t_rr) - ms_ritz - ms_jacobi;
@@ -992,10 +1084,42 @@ static galore_status_t refresh_group(const RefreshProblem* prs, int count, void*
 
     std::vector<Lane*> more;
     if (!full_space) {
+      // A warm-started lane is judged by what it reached, not by a prediction from a random start:
+      // the residual of its Ritz pairs over the gap behind the r-th Ritz value bounds the sine of the
+      // largest angle to the exact invariant subspace (Davis-Kahan, with Frobenius for spectral norm:
+      // on the safe side).  If that is not within the tolerance the lane goes on like a cold one, its
+      // remaining steps sized from the bound instead of from 1.
+      std::vector<Lane*> judged;
+      for (Lane* l : live)
+        if (l->warm_check) judged.push_back(l);
+      if (!judged.empty()) {
+        GALORE_TRY(make_p64(judged));
+        GALORE_TRY(residuals(judged));
+      }
+      for (Lane* l : judged) {
+        l->warm_check = false;
+        const double th_r = l->theta[r - 1], th_b = l->theta[b - 1];
+        const double gap = b > r ? th_r - l->theta[r] : 0.0;
+        const double bound = gap > 0.0 ? l->res_abs / gap : 1.0;
+        l->predicted = std::min(1.0, bound);
+        // a prediction from a random start is held to the tolerance itself, which leaves a margin of ten to
+        // the 1e-3 rad the projector has to meet; a bound on what was reached needs no such margin
+        l->converged = bound <= 10.0 * l->pr.tol;
+        const double ratio = (b > r && th_r > 0.0) ? th_b / th_r : 1.0;
+        if (!l->converged && l->q_done < l->pr.max_iters && ratio < 1.0 && ratio > 0.0) {
+          const int need = (int)ceil(log(l->pr.tol / l->predicted) / log(ratio)) + 1;
+          l->q_target = std::min(l->pr.max_iters, l->q_done + std::max(1, need));
+          l->warm_from = l->q_done;
+          l->warm_bound = l->predicted;
+          more.push_back(l);
+        }
+      }
       for (Lane* l : live) {
+        if (std::find(judged.begin(), judged.end(), l) != judged.end()) continue;
         const double th_r = l->theta[r - 1], th_b = l->theta[b - 1];
         const double ratio = (b > r && th_r > 0.0) ? th_b / th_r : 1.0;
-        l->predicted = (ratio < 1.0) ? pow(ratio, (double)l->q_done) : 1.0;
+        // from a random start the error begins at 1; after a warm start at the bound found above
+        l->predicted = (ratio < 1.0) ? l->warm_bound * pow(ratio, (double)(l->q_done - l->warm_from)) : 1.0;
         l->converged = l->predicted <= l->pr.tol;
         if (!l->converged && l->q_done < l->pr.max_iters && ratio < 1.0 && ratio > 0.0) {
           const int need = (int)ceil(log(l->pr.tol) / log(ratio)) + 2;
@@ -1007,21 +1131,12 @@ static galore_status_t refresh_group(const RefreshProblem* prs, int count, void*
     live = more;
   }
 
-  // ---- P = Y S[:, top r] ------------------------------------------------------------
-  const int64_t pc = d * r;
-  for (Lane* l : all) {
-    const RefreshBuffers& w = l->w;
-    if (l->with_vt)
-      gather_rows_kernel<<<r, 256, 0, st>>>(w.Vt, w.order, b, w.Vsel);
-    else
-      gather_rows_scaled_kernel<<<r, 256, 0, st>>>(w.H, w.lam, w.order, b, w.Vsel);
-    GALORE_LAUNCH_CHECK();
-  }
-  {
-    EpiStore<double, double> epi{c.w0.P64, r, 0, 1.0, 0.0};
-    const SlotList sl = slots_of(c, all);
-    GALORE_TRY((launch_gemm_dmma<double, double>((int)d, r, b, c.w0.Y64, b, 1, c.w0.Vsel, 1, b, epi, st, 1, 0, 0, &sl)));
-  }
+  // ---- P = Y S[:, top r], rounded to the stored dtype ------------------------------------------
+  // (a lane judged by its residual and found converged has its P64 already, and the residual used Y64 as scratch)
+  std::vector<Lane*> unmade;
+  for (Lane* l : all)
+    if (!l->p64_current) unmade.push_back(l);
+  GALORE_TRY(make_p64(unmade));
   for (Lane* l : all) {
     if (l->pr.p_dtype == GALORE_BF16)
       convert_kernel<double, __nv_bfloat16><<<grid_for(pc), 256, 0, st>>>(l->w.P64, (__nv_bfloat16*)l->pr.P, pc);
@@ -1031,48 +1146,10 @@ static galore_status_t refresh_group(const RefreshProblem* prs, int count, void*
     merge_flags_kernel<<<1, 1, 0, st>>>(l->status, l->w.flags);
     GALORE_LAUNCH_CHECK();
   }
-
-  // ---- a-posteriori residual of the kept Ritz pairs (a diagnostic: only when the record is wanted) ----
-  // || A A^T P - P Theta ||.  On the tensor path A^T P = Z S is formed from the products already at
-  // hand and A (A^T P) runs on the tensor cores in bf16 pairs.
+  // the a-posteriori residual of the kept Ritz pairs is a diagnostic: only when the record is wanted
   if (infos) {
-    const bool tensor_residual = tensor && (r % 8) == 0;
-    for (Lane* l : all) {
-      const RefreshBuffers& w = l->w;
-      const TG* G = (const TG*)l->pr.G;
-      const int64_t sAi = c.left ? l->pr.ldg : 1, sAl = c.left ? 1 : l->pr.ldg;
-      if (tensor_residual) {
-        EpiSplitPair e1{w.Zhi, w.Zlo, r};
-        GALORE_TRY((launch_gemm_dmma<double, double>((int)L, r, b, (const double*)w.Zu, b, 1, w.Vsel, 1, b, e1, st)));
-        const int a_mn = c.left ? 0 : 1;
-        const int s1 = (l->tr.master + 1) % 3, s2 = (l->tr.master + 2) % 3;
-        tensor_group_reset(c.tg);
-        GALORE_TRY(tensor_group_add_gemm(c.tg, l->pr.G, l->pr.ldg, a_mn, w.Zhi, r, 1, (int)d, r, (int)L, l->tr.F[s1], r, l->status));
-        GALORE_TRY(tensor_group_add_gemm(c.tg, l->pr.G, l->pr.ldg, a_mn, w.Zlo, r, 1, (int)d, r, (int)L, l->tr.F[s2], r, l->status));
-        GALORE_TRY(tensor_group_launch_project(c.tg, st));
-        GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
-        residual_pair_kernel<<<grid_for(d * r), 256, 0, st>>>(l->tr.F[s1], l->tr.F[s2], w.P64, w.theta, d, r, w.scal);
-        GALORE_LAUNCH_CHECK();
-      } else {
-        double* T1 = (double*)w.Zu;   // L x r
-        double* T2 = w.Y64;           // d x r (Y64 is no longer needed)
-        EpiStore<double, double> e1{T1, r, 0, 1.0, 0.0};
-        GALORE_TRY((launch_gemm_dmma<TG, double>((int)L, r, (int)d, G, sAl, sAi, w.P64, r, 1, e1, st)));
-        EpiStore<double, double> e2{T2, r, 0, 1.0, 0.0};
-        GALORE_TRY((launch_gemm_dmma<TG, double>((int)d, r, (int)L, G, sAi, sAl, T1, r, 1, e2, st)));
-        GALORE_CUDA_TRY(cudaMemsetAsync(w.scal, 0, 32, st));
-        residual_kernel<<<grid_for(pc), 256, 0, st>>>(T2, w.P64, w.theta, d, r, w.scal);
-        GALORE_LAUNCH_CHECK();
-      }
-    }
-    std::vector<double> sc(2 * (size_t)count, 0.0);
-    for (int i = 0; i < count; ++i)
-      GALORE_CUDA_TRY(cudaMemcpyAsync(&sc[2 * i], store[i].w.scal, 2 * sizeof(double), cudaMemcpyDeviceToHost, st));
-    GALORE_CUDA_TRY(cudaStreamSynchronize(st));
-    for (int i = 0; i < count; ++i) {
-      const Lane& l = store[i];
-      store[i].info.residual = l.theta[0] > 0.0 ? sqrt(sc[2 * i + 1]) / (l.theta[0] * sqrt((double)r)) : 0.0;
-    }
+    GALORE_TRY(residuals(all));
+    for (Lane* l : all) l->info.residual = l->theta[0] > 0.0 ? l->res_abs / (l->theta[0] * sqrt((double)r)) : 0.0;
   }
   GALORE_CUDA_TRY(cudaStreamSynchronize(st));      // the refresh is complete when the call returns
   const double ms_total = ms_between(t_begin, clk::now());

@@ -20,6 +20,8 @@ struct RefreshProblem {
   int max_iters;
   int first_iters;      // power steps before the first Rayleigh-Ritz
   bool use_tensor;      // power steps on the tensor cores when G is bf16 and TMA-addressable
+  int warm_iters;       // > 0: start from the projector already stored in P (its r columns plus random ones)
+                        // and run this many power steps before the first Rayleigh-Ritz pass; 0: random start
 };
 
 // d = rows of the projector, L = the other dimension of G

@@ -125,6 +125,22 @@ def make_planted(m: int, n: int, seed: int, spectrum, dtype: str = "f64"):
     return round_to(G, dtype), U, V
 
 
+def make_rotating(m: int, n: int, seed: int, spectrum, drift: float, t: int, noise: float = 0.0, dtype: str = "f64"):
+    """Gradient t of a sequence whose singular subspaces turn slowly (what makes a warm-started refresh pay):
+    G_t = U_t diag(spectrum) V_t^T + noise, with U_t = orth(U_0 + t drift E_u), V_t likewise, E fixed Gaussian
+    matrices: consecutive left (right) subspaces are about `drift` * sqrt(m) (sqrt(n)) radians apart."""
+    rng = np.random.default_rng(seed)
+    k = len(spectrum)
+    U0, V0 = random_orthonormal(m, k, rng), random_orthonormal(n, k, rng)
+    Eu, Ev = rng.standard_normal((m, k)), rng.standard_normal((n, k))
+    U, _ = np.linalg.qr(U0 + t * drift * Eu)
+    V, _ = np.linalg.qr(V0 + t * drift * Ev)
+    G = (U * np.asarray(spectrum, np.float64)) @ V.T
+    if noise:
+        G = G + noise * np.random.default_rng(seed + 1 + t).standard_normal((m, n))
+    return round_to(G, dtype)
+
+
 def make_weight(m: int, n: int, seed: int, dtype: str = "f32", std: float = 0.02) -> np.ndarray:
     rng = np.random.default_rng(seed)
     return round_to(std * rng.standard_normal((m, n)), dtype)

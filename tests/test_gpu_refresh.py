@@ -219,3 +219,50 @@ def test_layers_refreshed_as_a_group_get_the_projectors_of_single_refreshes(g_dt
     torch.cuda.synchronize()
     for a, c in zip(single, again):
         assert torch.equal(a.get_projector(), c.get_projector())
+
+
+@pytest.mark.parametrize("g_dtype,m,n,r", [("bf16", 512, 1376, 64), ("bf16", 1376, 512, 64), ("f32", 256, 640, 32)])
+def test_warm_started_refresh_reaches_the_cold_subspace_in_fewer_steps(g_dtype, m, n, r):
+    """Gradients whose singular subspaces turn slowly (a gapped spectrum, 0.02 rad between consecutive steps):
+    a refresh that starts from the stored projector and runs three power steps is accepted by its own
+    residual-over-gap bound, lands in the oracle's subspace, and needs a fraction of the cold refresh's steps.
+    On the workloads' noise-dominated spectrum (no gap behind the block) the look at the Rayleigh quotients
+    after those three steps sends the refresh on to the full iteration of a cold one, from its warm block."""
+    k = min(m, n)
+    spectrum = np.concatenate([np.linspace(3.0, 2.0, r), 0.3 * np.arange(1, k - r + 1, dtype=np.float64) ** -0.5])
+    side = "left" if m <= n else "right"
+    drift = 0.02 / np.sqrt(max(m, n))
+    G0 = wl.make_rotating(m, n, 91, spectrum, drift, 0, dtype=g_dtype)
+    G1 = wl.make_rotating(m, n, 91, spectrum, drift, 1, dtype=g_dtype)
+    ld = (n + 15) // 16 * 16
+    P0_orc, _ = go.top_r_projector(G0, r, side, method="lapack")
+    P1_orc, _ = go.top_r_projector(G1, r, side, method="lapack")
+    moved = go.largest_principal_angle(P0_orc, P1_orc)
+    assert 5e-3 < moved < 0.2                                  # the subspace did move, by a small angle
+
+    def layer(warm):
+        return gb.Layer(gb.make_config(m, n, r, w_dtype="bf16", g_dtype=g_dtype, p_dtype="f32", auto_refresh=False, seed=3,
+                                       refresh_warm_iters=warm))
+    cold, warm = layer(0), layer(3)
+    for l in (cold, warm):                                     # the first refresh of a layer has nothing to start from
+        st, info0 = l.galore_refresh_projector(to_dev(G0, g_dtype, ld))
+        assert st == gb.OK and go.largest_principal_angle(P0_orc, to_host(l.get_projector())) < 1e-3
+    st_c, info_c = cold.galore_refresh_projector(to_dev(G1, g_dtype, ld))
+    st_w, info_w = warm.galore_refresh_projector(to_dev(G1, g_dtype, ld))
+    Pc, Pw = to_host(cold.get_projector()), to_host(warm.get_projector())
+    print(f"{g_dtype} {m}x{n} r={r}: subspace moved {moved:.3f} rad; cold {info_c.iterations} steps, warm {info_w.iterations} steps, "
+          f"bound {info_w.predicted_error:.2e}, angles cold {go.largest_principal_angle(P1_orc, Pc):.2e} warm {go.largest_principal_angle(P1_orc, Pw):.2e}")
+    assert st_c == gb.OK and st_w == gb.OK and info_w.converged == 1
+    assert go.largest_principal_angle(P1_orc, Pw) < 1e-3
+    assert go.largest_principal_angle(Pc, Pw) < 1e-3           # the same subspace as the cold refresh
+    assert info_w.iterations <= 6 and info_w.iterations < info_c.iterations
+    assert np.abs(Pw.T @ Pw - np.eye(r)).max() < 1e-5
+    # noise-dominated spectrum: the warm start falls back to the full iteration and still converges
+    N0 = wl.make_gradient(m, n, wl.sub_seed(92, 0), 1.0, 0.01, g_dtype)
+    N1 = wl.make_gradient(m, n, wl.sub_seed(92, 1), 1.0, 0.01, g_dtype)
+    hard = layer(3)
+    hard.galore_refresh_projector(to_dev(N0, g_dtype, ld))
+    st_h, info_h = hard.galore_refresh_projector(to_dev(N1, g_dtype, ld))
+    Ph_orc, _ = go.top_r_projector(N1, r, side, method="lapack")
+    assert st_h == gb.OK and info_h.converged == 1 and info_h.iterations > 6
+    assert go.largest_principal_angle(Ph_orc, to_host(hard.get_projector())) < 1e-3
