@@ -142,6 +142,8 @@ typedef struct {
   double ms_power;           /* power steps and their orthonormalisations */
   double ms_ritz;            /* final orthonormalisation, fp64 products, sorting, P = Y S (without the eigen-solve) */
   double ms_jacobi;          /* Jacobi eigen-solves */
+  int32_t ritz_passes;       /* Rayleigh-Ritz passes (each ends a run of power steps) */
+  int32_t reserved;
 } galore_refresh_info_t;
 
 /* Sizes of the two caller-allocated device buffers for one layer.

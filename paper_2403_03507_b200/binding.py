@@ -45,6 +45,7 @@ class RefreshInfo(C.Structure):
         ("predicted_error", C.c_double), ("residual", C.c_double), ("sigma_r", C.c_double),
         ("sigma_next", C.c_double), ("sigma_1", C.c_double),
         ("ms_total", C.c_double), ("ms_power", C.c_double), ("ms_ritz", C.c_double), ("ms_jacobi", C.c_double),
+        ("ritz_passes", C.c_int32), ("reserved", C.c_int32),
     ]
 
     def as_dict(self):

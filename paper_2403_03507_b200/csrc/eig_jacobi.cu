@@ -162,7 +162,7 @@ constexpr int kSlots = kPairRows / 2;
 constexpr int kBlockTasks = kSlots * (kSlots + 1) / 2;
 constexpr int kSweepThreads = 512;
 constexpr int kALd = kPairRows + 1;
-constexpr size_t kSweepSmem = 4 * (size_t)kPairRows * kALd * sizeof(double);
+constexpr size_t kSweepSmem = 2 * (size_t)kPairRows * kALd * sizeof(double);   // A and Rot: three CTAs fit on an SM
 
 __host__ __device__ __forceinline__ int next_position(int pos) { return pos == 0 ? 0 : (pos == kPairRows - 1 ? 1 : pos + 1); }
 __host__ __device__ __forceinline__ int upper_offset(int i, int j) { return i < j ? i * kALd + j : j * kALd + i; }
@@ -191,19 +191,26 @@ __device__ __forceinline__ BlockTask make_block_task(int task) {
   return t;
 }
 
-__device__ __forceinline__ void block_update(const BlockTask& t, const double2* cs, const double* cur, double* nxt) {
+// B <- R_u B R_v^T for one 2 x 2 block, in two halves with a barrier between them: the results go back
+// into the same copy of A, one position on, once every thread has read its entries.
+struct BlockValues {
+  double a0, a1, a2, a3;
+};
+__device__ __forceinline__ BlockValues block_read(const BlockTask& t, const double* A) {
+  return BlockValues{A[t.rd[0]], A[t.rd[1]], A[t.rd[2]], A[t.rd[3]]};
+}
+__device__ __forceinline__ void block_write(const BlockTask& t, const double2* cs, const BlockValues& b, double* A) {
   const double2 ru = cs[t.u], rv = cs[t.v];
-  const double a0 = cur[t.rd[0]], a1 = cur[t.rd[1]], a2 = cur[t.rd[2]], a3 = cur[t.rd[3]];
-  // B <- R_u B R_v^T.  For u == v the two off-diagonal entries are one stored value; both results agree.
-  const double r00 = ru.x * a0 - ru.y * a2, r01 = ru.x * a1 - ru.y * a3;
-  const double r10 = ru.y * a0 + ru.x * a2, r11 = ru.y * a1 + ru.x * a3;
-  nxt[t.wr[0]] = rv.x * r00 - rv.y * r01;
-  nxt[t.wr[1]] = rv.y * r00 + rv.x * r01;
-  nxt[t.wr[2]] = rv.x * r10 - rv.y * r11;
-  nxt[t.wr[3]] = rv.y * r10 + rv.x * r11;
+  // For u == v the two off-diagonal entries are one stored value; both results agree.
+  const double r00 = ru.x * b.a0 - ru.y * b.a2, r01 = ru.x * b.a1 - ru.y * b.a3;
+  const double r10 = ru.y * b.a0 + ru.x * b.a2, r11 = ru.y * b.a1 + ru.x * b.a3;
+  A[t.wr[0]] = rv.x * r00 - rv.y * r01;
+  A[t.wr[1]] = rv.y * r00 + rv.x * r01;
+  A[t.wr[2]] = rv.x * r10 - rv.y * r11;
+  A[t.wr[3]] = rv.y * r10 + rv.x * r11;
 }
 
-__global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* __restrict__ part, int chunks, int b, int nblk,
+__global__ void __launch_bounds__(kSweepThreads, 2) jb_sweep_kernel(const double* __restrict__ part, int chunks, int b, int nblk,
                                                                  int round, double tol, double* __restrict__ rot_out,
                                                                  int* __restrict__ flags, int* __restrict__ rotations,
                                                                  const SlotList slots) {
@@ -215,10 +222,8 @@ __global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* _
     flags = slot_ptr(flags, shift);
     rotations = slot_ptr(rotations, shift);
   }
-  // the two copies of A, then the two copies of Rot (addresses computed, not looked up: an array of
-  // pointers indexed by the round would live in local memory)
-  auto Abuf = [&](int which) { return jb_smem + which * (kPairRows * kALd); };
-  auto Rbuf = [&](int which) { return jb_smem + (2 + which) * (kPairRows * kALd); };
+  double* const As = jb_smem;                          // the Gram matrix (upper triangle used)
+  double* const Rs = jb_smem + kPairRows * kALd;       // the accumulated rotation
   __shared__ double2 cs[kSlots];
   const int pair = blockIdx.x, tid = threadIdx.x;
   const BlockPair bp = block_pair(pair, round, nblk);
@@ -247,8 +252,8 @@ __global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* _
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int idx = tid + kSweepThreads * i;
-      Abuf(0)[(idx >> 6) * kALd + (idx & 63)] = sum[i];
-      Rbuf(0)[(idx >> 6) * kALd + (idx & 63)] = ((idx >> 6) == (idx & 63)) ? 1.0 : 0.0;
+      As[(idx >> 6) * kALd + (idx & 63)] = sum[i];
+      Rs[(idx >> 6) * kALd + (idx & 63)] = ((idx >> 6) == (idx & 63)) ? 1.0 : 0.0;
     }
   }
   const BlockTask t0 = make_block_task(tid);                                   // tasks 0 .. 511
@@ -262,10 +267,7 @@ __global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* _
   int applied = 0;
   const double tol2 = tol * tol;
   for (int rr = 0; rr < kSweepRounds; ++rr) {
-    const double* Ac = Abuf(rr & 1);
-    double* An = Abuf((rr + 1) & 1);
-    const double* Rc = Rbuf(rr & 1);
-    double* Rn = Rbuf((rr + 1) & 1);
+    const double* Ac = As;
     if (tid < kSlots) {
       const int f = tid, g = kPairRows - 1 - tid;
       const double app = Ac[f * kALd + f], aqq = Ac[g * kALd + g], apq = Ac[f * kALd + g];
@@ -295,16 +297,25 @@ __global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* _
       }
       cs[tid] = make_double2(c, s);
     }
+    // every entry moves one position on (the round-robin order of the rows): read, barrier, write
+    const BlockValues v0 = block_read(t0, As);
+    BlockValues v1 = v0;
+    if (second) v1 = block_read(t1, As);
+    double rx[4], ry[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      rx[i] = Rs[rf + 16 * i];
+      ry[i] = Rs[rg + 16 * i];
+    }
     __syncthreads();
-    block_update(t0, cs, Ac, An);
-    if (second) block_update(t1, cs, Ac, An);
+    block_write(t0, cs, v0, As);
+    if (second) block_write(t1, cs, v1, As);
     {
       const double2 r = cs[rslot];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const double x = Rc[rf + 16 * i], y = Rc[rg + 16 * i];
-        Rn[wf + 16 * i] = r.x * x - r.y * y;
-        Rn[wg + 16 * i] = r.y * x + r.x * y;
+        Rs[wf + 16 * i] = r.x * rx[i] - r.y * ry[i];
+        Rs[wg + 16 * i] = r.y * rx[i] + r.x * ry[i];
       }
     }
     __syncthreads();
@@ -320,7 +331,7 @@ __global__ void __launch_bounds__(kSweepThreads) jb_sweep_kernel(const double* _
   }
   __syncthreads();
   if (cs[0].x != 0.0) {   // all rows are back at their own positions after the 63 rounds
-    const double* Rf = Rbuf(kSweepRounds & 1);
+    const double* Rf = Rs;
     double* out = rot_out + (int64_t)pair * (kPairRows * kPairRows);
     for (int idx = tid; idx < kPairRows * kPairRows; idx += kSweepThreads) out[idx] = Rf[(idx >> 6) * kALd + (idx & 63)];
   }

@@ -172,6 +172,22 @@ __global__ void __launch_bounds__(256) shift_split_kernel(float* __restrict__ Yn
   }
 }
 
+// One step of a degree-2 Chebyshev filter on B = A A^T over the damped interval [0, 2c] (half width c):
+// first step Y1 = (B Y0 - c Y0) / c, second step Y2 = 2 (B Y1 - c Y1) / c - Y0 = T_2((B - c) / c) Y0.
+// x0 + x1 is the hi/lo product B y; v = s (x0 + x1 - c y) - z (z: the block two steps back, or null),
+// stored in x0 and as a hi/lo pair.
+__global__ void __launch_bounds__(256) cheb_split_kernel(float* __restrict__ x0, const float* __restrict__ x1,
+                                                         const float* __restrict__ y, const float* __restrict__ z, float c,
+                                                         float s, int64_t count, __nv_bfloat16* __restrict__ hi,
+                                                         __nv_bfloat16* __restrict__ lo) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x) {
+    float v = s * fmaf(-c, y[i], x0[i] + x1[i]);
+    if (z) v -= z[i];
+    x0[i] = v;
+    split_bf16(v, hi[i], lo[i]);
+  }
+}
+
 // Rayleigh quotients of the block: ||z_i||^2 with Z = A^T Y (+ second partial of a hi/lo product).
 // Slice s of kColSlices sums rows s, s + kColSlices, ...; slices are added in order afterwards.
 constexpr int kColSlices = 64;
@@ -512,9 +528,22 @@ const double* refresh_unrounded_projector(void* workspace, int64_t d, int64_t L,
 // would make on its own (its own iteration count and orthonormalisation schedule), so a layer's
 // projector does not depend on what it was grouped with.
 
+// Chebyshev acceleration of slowly converging blocks: used when the look asks for more than this many
+// further plain steps, and only while T_2 at theta_1 (the growth of the block's condition number over a
+// pair, which the bf16 pairs and the squared Gram matrix have to carry) stays below the second constant.
+constexpr int kChebyshevFrom = 8;
+constexpr double kChebyshevSpread = 150.0;
+static inline double cheb_t2(double x) { return 2.0 * x * x - 1.0; }
+
 struct TensorRefresh {
-  float* F[3];          // fp32 d x b buffers; F[master] holds Y
-  int master;
+  float* F[4];          // fp32 d x b buffers; F[master] holds Y.  F[3] (the idle upper half of Y64) only ever
+  int master;           // receives the second partial product of the closing step of a Chebyshev pair
+  int prev = -1;        // buffer of the block one step back, between the two steps of a Chebyshev pair
+};
+// one run of Chebyshev pairs with a fixed interval
+struct ChebSegment {
+  double c;             // centre = half width of the damped interval [0, 2c]
+  int pairs;
 };
 
 struct Lane {
@@ -529,6 +558,9 @@ struct Lane {
   std::vector<double> theta;
   double predicted = 0.0, res_abs = 0.0;
   bool converged = false, with_vt = false, iterating = true;
+  bool cheb = false;          // power steps come in pairs that apply T_2 of the shifted operator
+  int q_plain = 0;            // plain power steps among q_done
+  std::vector<ChebSegment> segs;
   bool p64_current = false;   // P64 holds the Ritz vectors of the lane's last Rayleigh-Ritz pass
   bool warm_check = false;    // started from the previous projector: the first Rayleigh-Ritz pass is judged by its residual
   int warm_from = 0;          // steps done when the warm start was judged, and the error bound found there
@@ -749,21 +781,49 @@ static galore_status_t power_step_tensor(const Ctx& c, const std::vector<Lane*>&
     sum_split_kernel<<<grid_for(zb), 256, 0, st>>>(z0, z0 + zb, nullptr, nullptr, l->w.Zhi, l->w.Zlo, zb);
     GALORE_LAUNCH_CHECK();
   }
+  // outputs of the two partial products: two buffers that hold neither Y nor, inside a Chebyshev pair, the block before it
+  auto outputs = [](const TensorRefresh& t, int& o1, int& o2) {
+    if (t.prev < 0) {
+      o1 = (t.master + 1) % 3;
+      o2 = (t.master + 2) % 3;
+    } else {
+      o1 = 3 - t.master - t.prev;     // the third of the buffers 0, 1, 2
+      o2 = 3;
+    }
+  };
   tensor_group_reset(c.tg);
   for (Lane* l : lanes) {
     TensorRefresh& t = l->tr;
-    const int m = t.master, s1 = (m + 1) % 3, s2 = (m + 2) % 3;
+    int s1, s2;
+    outputs(t, s1, s2);
     GALORE_TRY(tensor_group_add_gemm(c.tg, l->pr.G, l->pr.ldg, a_mn, l->w.Zhi, b, 1, (int)d, b, (int)L, t.F[s1], b, l->status));
     GALORE_TRY(tensor_group_add_gemm(c.tg, l->pr.G, l->pr.ldg, a_mn, l->w.Zlo, b, 1, (int)d, b, (int)L, t.F[s2], b, l->status));
   }
   GALORE_TRY(tensor_group_launch_project(c.tg, st));
   for (Lane* l : lanes) {
     TensorRefresh& t = l->tr;
-    const int m = t.master, s1 = (m + 1) % 3, s2 = (m + 2) % 3;
-    add_sumsq_kernel<<<kSumsqBlocks, 256, 0, st>>>(t.F[s1], t.F[s2], yb, l->w.part);
-    GALORE_LAUNCH_CHECK();
-    shift_split_kernel<<<grid_for(yb), 256, 0, st>>>(t.F[s1], t.F[m], yb, b, l->w.part, l->w.Yhi, l->w.Ylo);
-    GALORE_LAUNCH_CHECK();
+    const int m = t.master;
+    int s1, s2;
+    outputs(t, s1, s2);
+    if (!l->cheb) {
+      add_sumsq_kernel<<<kSumsqBlocks, 256, 0, st>>>(t.F[s1], t.F[s2], yb, l->w.part);
+      GALORE_LAUNCH_CHECK();
+      shift_split_kernel<<<grid_for(yb), 256, 0, st>>>(t.F[s1], t.F[m], yb, b, l->w.part, l->w.Yhi, l->w.Ylo);
+      GALORE_LAUNCH_CHECK();
+      l->q_plain += 1;
+    } else {
+      const float cc = (float)l->segs.back().c, inv = (float)(1.0 / l->segs.back().c);
+      if (t.prev < 0) {       // opening step of a pair: the block it starts from is needed once more
+        cheb_split_kernel<<<grid_for(yb), 256, 0, st>>>(t.F[s1], t.F[s2], t.F[m], nullptr, cc, inv, yb, l->w.Yhi, l->w.Ylo);
+        t.prev = m;
+      } else {
+        cheb_split_kernel<<<grid_for(yb), 256, 0, st>>>(t.F[s1], t.F[s2], t.F[m], t.F[t.prev], cc, 2.0f * inv, yb, l->w.Yhi,
+                                                        l->w.Ylo);
+        t.prev = -1;
+        l->segs.back().pairs += 1;
+      }
+      GALORE_LAUNCH_CHECK();
+    }
     t.master = s1;
     l->Y = t.F[t.master];
   }
@@ -843,6 +903,7 @@ static galore_status_t refresh_group(const RefreshProblem* prs, int count, void*
     l.Y = l.w.Ya;
     l.Yn = l.w.Yb;
     l.tr.F[0] = l.w.Ya; l.tr.F[1] = l.w.Yb; l.tr.F[2] = l.w.Yc;
+    l.tr.F[3] = (float*)l.w.Y64 + yb;
     l.tr.master = 0;
     l.theta.assign(b, 0.0);
     l.info.block = b;
@@ -950,7 +1011,25 @@ static galore_status_t refresh_group(const RefreshProblem* prs, int count, void*
                                                       : (ratio >= 1.0 ? l->pr.max_iters : l->q_done);
         if (l->warm_check && need > 2 * l->q_done) l->warm_check = false;
         if (!l->warm_check) l->q_target = std::min(l->pr.max_iters, std::max(need, l->q_done));
-        if (tensor && theta[b - 1] > 0.0) {
+        if (tensor && !l->warm_check && need - l->q_done > kChebyshevFrom && ratio > 0.25 && ratio < 1.0) {
+          // A slowly converging block (no gap behind it): the remaining steps come in pairs that apply
+          // T_2 of the operator mapped so that [0, theta_b] falls on [-1, 1].  What lies in the interval stays
+          // bounded by 1 while theta_r grows by T_2(2 theta_r / theta_b - 1) per pair, against
+          // (theta_r / theta_b)^2 of two plain steps.  The look's theta_b is on the high side, which
+          // widens the interval: slower than it could be, never wrong.
+          const double beta = theta[b - 1];
+          const double gain = cheb_t2(2.0 * theta[r - 1] / beta - 1.0), spread = cheb_t2(2.0 * theta[0] / beta - 1.0);
+          if (gain > 1.0 && spread <= kChebyshevSpread) {
+            const double left = pow(ratio, (double)l->q_done);            // what the plain steps have achieved
+            const int pairs = std::max(1, (int)ceil(log(left / l->pr.tol) / log(gain)) + 1);
+            l->cheb = true;
+            l->segs.push_back(ChebSegment{0.5 * beta, 0});
+            l->q_target = std::min(l->q_done + 2 * pairs, l->q_done + (l->pr.max_iters - l->q_done) / 2 * 2);
+          }
+        }
+        if (l->cheb) {
+          l->orth_every = 2;           // the filter's own growth of the block's condition number was checked above
+        } else if (tensor && theta[b - 1] > 0.0) {
           // chained steps multiply the block's condition number by theta_1/theta_b each; the bf16 pair
           // carries 16 bits and the Gram matrix squares the product, so keep it below about 100
           const double spread = theta[0] / theta[b - 1];
@@ -1024,7 +1103,10 @@ static galore_status_t refresh_group(const RefreshProblem* prs, int count, void*
   while (!live.empty()) {
     // ---- power steps: every lane up to its own target, on its own orthonormalisation schedule ----
     GALORE_TRY(run_steps(live));
-    for (Lane* l : live) l->p64_current = false;
+    for (Lane* l : live) {
+      l->p64_current = false;
+      l->info.ritz_passes += 1;
+    }
     // ---- Rayleigh-Ritz in fp64 --------------------------------------------------
     const clk::time_point t_rr = now_synced();
     ms_power = ms_between(t_begin, t_rr) - ms_ritz - ms_jacobi;
@@ -1118,6 +1200,26 @@ static galore_status_t refresh_group(const RefreshProblem* prs, int count, void*
         if (std::find(judged.begin(), judged.end(), l) != judged.end()) continue;
         const double th_r = l->theta[r - 1], th_b = l->theta[b - 1];
         const double ratio = (b > r && th_r > 0.0) ? th_b / th_r : 1.0;
+        if (l->cheb) {
+          // plain steps as below; every Chebyshev pair divides the error by T_2 at theta_r over the largest
+          // value the filter takes on what is to be damped (1 inside its interval, T_2 at theta_b beyond it)
+          double log_err = (ratio < 1.0 && ratio > 0.0) ? l->q_plain * log(ratio) : 0.0;
+          for (const ChebSegment& sg : l->segs) {
+            const double num = std::max(1.0, fabs(cheb_t2(th_b / sg.c - 1.0))), den = cheb_t2(th_r / sg.c - 1.0);
+            if (den > num) log_err += sg.pairs * log(num / den);
+          }
+          l->predicted = ratio < 1.0 ? std::min(1.0, exp(log_err)) : 1.0;
+          l->converged = l->predicted <= l->pr.tol;
+          if (!l->converged && l->q_done + 1 < l->pr.max_iters && ratio < 1.0 && ratio > 0.0) {
+            const double c2 = 0.5 * 1.02 * th_b;                   // the interval now ends just above the b-th Ritz value
+            const double gain = cheb_t2(th_r / c2 - 1.0);
+            const int pairs = gain > 1.0 ? std::max(1, (int)ceil(log(l->predicted / l->pr.tol) / log(gain)) + 1) : 1;
+            l->segs.push_back(ChebSegment{c2, 0});
+            l->q_target = std::min(l->q_done + 2 * pairs, l->q_done + (l->pr.max_iters - l->q_done) / 2 * 2);
+            more.push_back(l);
+          }
+          continue;
+        }
         // from a random start the error begins at 1; after a warm start at the bound found above
         l->predicted = (ratio < 1.0) ? l->warm_bound * pow(ratio, (double)(l->q_done - l->warm_from)) : 1.0;
         l->converged = l->predicted <= l->pr.tol;
