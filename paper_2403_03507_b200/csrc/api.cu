@@ -323,7 +323,7 @@ RefreshProblem refresh_problem(const galore_layer* l, const void* G, int64_t ldg
   pr.seed = l->cfg.seed;
   pr.tol = l->cfg.refresh_tol > 0.f ? (double)l->cfg.refresh_tol : 1e-4;
   pr.max_iters = l->cfg.refresh_max_iters > 0 ? l->cfg.refresh_max_iters : 96;
-  pr.first_iters = 6;
+  pr.first_iters = 4;
   pr.use_tensor = l->tensor_path;
   pr.warm_iters = (l->cfg.refresh_warm_iters > 0 && l->has_projector) ? l->cfg.refresh_warm_iters : 0;
   return pr;
