@@ -28,6 +28,12 @@ What it follows (GaLore, arXiv 2403.03507):
     state matrix); it is PARITY UNPINNED against the paper
     (the paper fixes nothing to pin it to) and pinned only by its own
     invariants in the tests.
+  * Sec. "GaLore with memory-efficient optimizers" names Adafactor with
+    first-order statistics as another inner optimizer and prints no formulas.
+    `adafactor_update` is the published Adafactor update (Shazeer & Stern) on
+    the compact gradient, the reading of its options stated there; it is
+    PARITY UNPINNED against the paper and pinned against an independent
+    library implementation of that algorithm, a closed form and brute force.
 
 Storage emulation: arithmetic is always fp64; values are rounded when they are
 *stored* (weights to bf16 or fp32, moments to fp32 or to 8-bit codes), because
@@ -276,6 +282,37 @@ def state_tile(q_block: int):
 # Algorithm 1
 # --------------------------------------------------------------------------
 
+# ---------------------------------------------------------------------------
+# Adafactor as the inner regulariser (Sec. "GaLore with memory-efficient optimizers": Adafactor
+# "with first-order statistics"; the paper prints no formulas, so the update is the published one
+# of Shazeer & Stern, "Adafactor: Adaptive Learning Rates with Sublinear Memory Cost", Algorithm 4
+# with momentum, written for the compact gradient R).  Reading taken here: external learning rate
+# (no relative step size, no parameter scaling), decay beta2_t = 1 - t^-0.8, eps_1 = 1e-30, update
+# clipping at d = 1, momentum beta1 on the clipped update, and the learning rate applied where
+# Algorithm 1 applies it (W <- W - lr alpha P N), not inside the momentum.
+# ---------------------------------------------------------------------------
+ADAFACTOR_DECAY = 0.8
+ADAFACTOR_EPS1 = 1e-30
+ADAFACTOR_CLIP = 1.0
+
+
+def adafactor_update(R, M_prev, v_row, v_col, t, beta1):
+    """One Adafactor step on R (rows x cols).  v_row (rows) and v_col (cols) are the running means of
+    R^2 + eps_1 along each row and each column; their outer product over the mean of v_row is the
+    factored second moment.  Returns (N, v_row, v_col) with N = the new first moment."""
+    R = np.asarray(R, dtype=np.float64)
+    beta2t = 1.0 - float(t) ** (-ADAFACTOR_DECAY)
+    sq = R * R + ADAFACTOR_EPS1
+    v_row = beta2t * v_row + (1.0 - beta2t) * sq.mean(axis=1)
+    v_col = beta2t * v_col + (1.0 - beta2t) * sq.mean(axis=0)
+    V_hat = np.outer(v_row, v_col) / v_row.mean()
+    U = R / np.sqrt(V_hat)
+    rms = np.sqrt(np.mean(U * U))
+    U = U / max(1.0, rms / ADAFACTOR_CLIP)
+    N = beta1 * M_prev + (1.0 - beta1) * U
+    return N, v_row, v_col
+
+
 class GaLoreOracle:
     """One 2-D weight's GaLore-Adam state and step (Algorithm 1), in fp64.
 
@@ -284,8 +321,11 @@ class GaLoreOracle:
     n_store : 'f64' | 'f32' | 'bf16'   rounding applied to the normalised update
                                         before it is projected back (the CUDA
                                         path feeds its tensor cores bf16)
-    inner   : 'adam' | 'identity'      the regulariser rho_t; 'identity' is the
-                                        rho_t = 1 case of Sec. 3.3 used by one pin
+    inner   : 'adam' | 'identity' | 'adafactor'
+                                        the regulariser rho_t; 'identity' is the
+                                        rho_t = 1 case of Sec. 3.3 used by one pin;
+                                        'adafactor' is Adafactor with first-order
+                                        statistics (see adafactor_update)
     """
 
     def __init__(self, m, n, rank, alpha, refresh_gap, beta1=0.9, beta2=0.999, eps=1e-8,
@@ -321,6 +361,12 @@ class GaLoreOracle:
         else:
             self.M = np.zeros(shape, dtype=np.float64)
             self.V = np.zeros(shape, dtype=np.float64)
+        if inner == "adafactor":
+            if state == "q8":
+                raise ValueError("the factored second moment is kept in floating point")
+            self.V = None
+            self.v_row = np.zeros(shape[0], dtype=np.float64)
+            self.v_col = np.zeros(shape[1], dtype=np.float64)
         self.refreshes = 0
 
     # -- state accessors ----------------------------------------------------
@@ -335,6 +381,8 @@ class GaLoreOracle:
     def optimizer_state_elements(self) -> int:
         """Elements held besides W: projector plus two moments (Sec. 4.2: mr + 2nr for m <= n)."""
         proj = (self.m if self.side == "left" else self.n) * self.r
+        if self.inner == "adafactor":                   # first moment plus one row and one column vector
+            return proj + self.state_shape[0] * self.state_shape[1] + self.state_shape[0] + self.state_shape[1]
         return proj + 2 * self.state_shape[0] * self.state_shape[1]
 
     def set_projector(self, proj):
@@ -363,6 +411,10 @@ class GaLoreOracle:
         R = P.T @ G if self.side == "left" else G @ P
         if self.inner == "identity":
             N = R
+        elif self.inner == "adafactor":
+            N, self.v_row, self.v_col = adafactor_update(R, self.M, self.v_row, self.v_col, self.k + 1, self.beta1)
+            self.M = _store(N, self.state)
+            self.v_row, self.v_col = _store(self.v_row, self.state), _store(self.v_col, self.state)
         else:
             M_prev, V_prev = self.moments()
             M = self.beta1 * M_prev + (1.0 - self.beta1) * R
