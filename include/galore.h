@@ -64,7 +64,13 @@ typedef enum {
 
 typedef enum { GALORE_SIDE_AUTO = 0, GALORE_SIDE_LEFT = 1, GALORE_SIDE_RIGHT = 2 } galore_side_t;
 typedef enum { GALORE_F32 = 0, GALORE_BF16 = 1 } galore_dtype_t;
-typedef enum { GALORE_STATE_F32 = 0, GALORE_STATE_Q8_BLOCK = 1 } galore_state_fmt_t;
+/* How the inner optimizer's statistics are kept.  F32 and Q8_BLOCK are Adam's two moments (Algorithm 1;
+ * Sec. 4.3 for the 8-bit form).  ADAFACTOR swaps the inner optimizer (Sec. "GaLore with memory-efficient
+ * optimizers": Adafactor with first-order statistics; the paper prints no formulas, the update is Shazeer
+ * and Stern's): an fp32 first moment of R's shape plus one fp32 value per row and per column of R for the
+ * factored second moment, decay 1 - t^-0.8, eps_1 = 1e-30, update clipping at 1, beta1 as the momentum,
+ * the learning rate applied in the weight update as for Adam; beta2 and eps are not used. */
+typedef enum { GALORE_STATE_F32 = 0, GALORE_STATE_Q8_BLOCK = 1, GALORE_STATE_ADAFACTOR = 2 } galore_state_fmt_t;
 /* which kernels carry the two projections */
 typedef enum {
   GALORE_PATH_AUTO = 0,   /* tensor cores when dtypes/alignment allow, else the fp32 path */
@@ -286,8 +292,13 @@ galore_status_t galore_get_projector(galore_layer_t* layer, float* dst, size_t d
  * workspace.  The 1e-3 rad bound of the refresh is a statement about this matrix. */
 galore_status_t galore_get_unrounded_projector(galore_layer_t* layer, double* dst, size_t dst_bytes, void* stream);
 galore_status_t galore_set_projector(galore_layer_t* layer, const float* src, size_t src_bytes, void* stream);
-/* Stored (uncorrected) moments as fp32, shape of R row-major packed, device memory (8-bit states are dequantised). */
+/* Stored (uncorrected) Adam moments as fp32, shape of R row-major packed, device memory (8-bit states are
+ * dequantised; GALORE_ERR_STATE for Adafactor, whose second moment is factored). */
 galore_status_t galore_get_moments(galore_layer_t* layer, float* M, float* V, size_t bytes_each, void* stream);
+/* Adafactor state (GALORE_STATE_ADAFACTOR, else GALORE_ERR_STATE): the first moment (fp32, shape of R, row-major
+ * packed), the running row means (rows of R entries) and column means (columns of R entries) of R^2 + eps_1;
+ * device memory. */
+galore_status_t galore_get_adafactor_state(galore_layer_t* layer, float* M, float* v_row, float* v_col, void* stream);
 /* Raw 8-bit state: codes (uint8, shape of R, packed) and per-block absmax (fp32, tile (I, J) of the
  * state at I * ceil(cols / 64) + J); device memory. */
 galore_status_t galore_get_q8_state(galore_layer_t* layer, uint8_t* M_codes, float* M_absmax,

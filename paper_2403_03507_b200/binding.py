@@ -19,7 +19,7 @@ ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL = -1, -2, -3, -4
 ERR_CUDA, ERR_STATE, ERR_NONFINITE, ERR_TIMEOUT, ERR_UNIMPLEMENTED = -5, -6, -7, -8, -9
 SIDE_AUTO, SIDE_LEFT, SIDE_RIGHT = 0, 1, 2
 F32, BF16 = 0, 1
-STATE_F32, STATE_Q8_BLOCK = 0, 1
+STATE_F32, STATE_Q8_BLOCK, STATE_ADAFACTOR = 0, 1, 2
 PATH_AUTO, PATH_FP32, PATH_TENSOR = 0, 1, 2
 ADAM_AUTO, ADAM_IN_PROJECTION, ADAM_OWN_KERNEL = 0, 1, 2
 DEV_NONFINITE, DEV_WAIT_EXPIRED, DEV_CHOLESKY = 1, 2, 8
@@ -87,6 +87,7 @@ _PROTOTYPES = {
     "galore_get_unrounded_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "galore_set_projector": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "galore_get_moments": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "galore_get_adafactor_state": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "galore_get_q8_state": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "galore_get_step_count": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
     "galore_set_step_count": (C.c_int, [C.c_void_p, C.c_int64]),
@@ -153,7 +154,8 @@ def make_config(m, n, rank, alpha=0.25, refresh_gap=200, beta1=0.9, beta2=0.999,
     if p_dtype is None:   # bf16 projector only where the gradient is bf16 too (tensor-core operands)
         p_dtype = "bf16" if c.g_dtype == BF16 else "f32"
     c.p_dtype = _DTYPES[p_dtype]
-    c.state_fmt = {"f32": STATE_F32, "q8": STATE_Q8_BLOCK, STATE_F32: STATE_F32, STATE_Q8_BLOCK: STATE_Q8_BLOCK}[state_fmt]
+    c.state_fmt = {"f32": STATE_F32, "q8": STATE_Q8_BLOCK, "adafactor": STATE_ADAFACTOR, STATE_F32: STATE_F32,
+                   STATE_Q8_BLOCK: STATE_Q8_BLOCK, STATE_ADAFACTOR: STATE_ADAFACTOR}[state_fmt]
     c.q_block, c.auto_refresh, c.path = q_block, int(bool(auto_refresh)), path
     c.refresh_tol, c.refresh_max_iters, c.refresh_oversample, c.seed = refresh_tol, refresh_max_iters, refresh_oversample, seed
     c.weight_decay = weight_decay
@@ -328,6 +330,15 @@ class Layer:
         _check(lib().galore_get_moments(self.handle, M.data_ptr(), V.data_ptr(), M.numel() * 4, _stream_ptr(stream)),
                "galore_get_moments")
         return M, V
+
+    def get_adafactor_state(self, stream=None):
+        rows, cols = self.state_shape
+        M = torch.empty(rows, cols, dtype=torch.float32, device=self.device)
+        v_row = torch.empty(rows, dtype=torch.float32, device=self.device)
+        v_col = torch.empty(cols, dtype=torch.float32, device=self.device)
+        _check(lib().galore_get_adafactor_state(self.handle, M.data_ptr(), v_row.data_ptr(), v_col.data_ptr(),
+                                                _stream_ptr(stream)), "galore_get_adafactor_state")
+        return M, v_row, v_col
 
     def get_q8_state(self, stream=None):
         rows, cols = self.state_shape

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgalore.so")
-SOURCES = ["api.cu", "adam.cu", "refresh.cu", "eig_jacobi.cu", "gemm_tc.cu", "step_static.cu"]
+SOURCES = ["api.cu", "adam.cu", "adafactor.cu", "refresh.cu", "eig_jacobi.cu", "gemm_tc.cu", "step_static.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-shared"]
 

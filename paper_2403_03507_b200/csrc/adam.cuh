@@ -41,7 +41,7 @@ galore_status_t launch_adam(const AdamItem& item, int32_t state_fmt, int q_block
 // Pitches and sizes of a layer's state arrays.  fp32 moments: rows of ceil8(cols) floats; 8-bit codes:
 // rows of ceil32(cols) bytes, plus ceil(rows / (q_block / 64)) * ceil(cols / 64) absmax values.
 inline int64_t state_pitch(int32_t state_fmt, int64_t cols) {
-  return state_fmt == GALORE_STATE_F32 ? (cols + 7) / 8 * 8 : (cols + 31) / 32 * 32;
+  return state_fmt == GALORE_STATE_Q8_BLOCK ? (cols + 31) / 32 * 32 : (cols + 7) / 8 * 8;
 }
 inline int64_t state_tiles(int64_t rows, int64_t cols, int q_block) {
   return ceil_div(rows, q_block / kStateTileCols) * ceil_div(cols, kStateTileCols);

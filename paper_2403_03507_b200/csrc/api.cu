@@ -12,6 +12,7 @@
 #include <vector>
 #include <string>
 
+#include "adafactor.cuh"
 #include "adam.cuh"
 #include "common.cuh"
 #include "gemm_simt.cuh"
@@ -83,6 +84,8 @@ struct galore_layer {
   // device memory (all inside the caller's two buffers)
   void* P;
   float *M, *V;
+  float *v_row, *v_col;  // Adafactor: running means of R^2 along rows and columns (V is unused then)
+  float* af_scratch;
   uint8_t *Mc, *Vc;
   float *Mam, *Vam;
   int32_t* status;
@@ -103,7 +106,8 @@ struct Sizes {
   int64_t ld_part, ld_n, ld_s;
   bool tensor_path;
   size_t off_P, off_M, off_V, off_Mam, off_Vam, state_bytes;
-  size_t off_status, off_R, off_N, off_refresh, ws_bytes;
+  size_t off_vrow, off_vcol;
+  size_t off_status, off_R, off_N, off_af, off_refresh, ws_bytes;
 };
 
 galore_status_t resolve(const galore_config_t* c, Sizes* s) {
@@ -117,7 +121,7 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
   if (c->side < GALORE_SIDE_AUTO || c->side > GALORE_SIDE_RIGHT) return GALORE_ERR_INVALID_ARG;
   for (int32_t dt : {c->w_dtype, c->g_dtype, c->p_dtype})
     if (dt != GALORE_F32 && dt != GALORE_BF16) return GALORE_ERR_INVALID_ARG;
-  if (c->state_fmt != GALORE_STATE_F32 && c->state_fmt != GALORE_STATE_Q8_BLOCK) return GALORE_ERR_INVALID_ARG;
+  if (c->state_fmt < GALORE_STATE_F32 || c->state_fmt > GALORE_STATE_ADAFACTOR) return GALORE_ERR_INVALID_ARG;
   if (c->path < GALORE_PATH_AUTO || c->path > GALORE_PATH_TENSOR) return GALORE_ERR_INVALID_ARG;
   if (c->adam_place < GALORE_ADAM_AUTO || c->adam_place > GALORE_ADAM_OWN_KERNEL) return GALORE_ERR_INVALID_ARG;
   if (c->refresh_warm_iters < 0) return GALORE_ERR_INVALID_ARG;
@@ -162,10 +166,16 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
 
   size_t o = 0;
   s->off_P = o; o += align_up((size_t)s->d * r * dtype_size(c->p_dtype), 256);
+  s->off_vrow = s->off_vcol = 0;
   if (c->state_fmt == GALORE_STATE_F32) {
     s->off_M = o; o += align_up((size_t)s->srows * s->ld_s * 4, 256);
     s->off_V = o; o += align_up((size_t)s->srows * s->ld_s * 4, 256);
     s->off_Mam = s->off_Vam = o;
+  } else if (c->state_fmt == GALORE_STATE_ADAFACTOR) {
+    s->off_M = o; o += align_up((size_t)s->srows * s->ld_s * 4, 256);
+    s->off_vrow = o; o += align_up((size_t)s->srows * 4, 256);
+    s->off_vcol = o; o += align_up((size_t)s->scols * 4, 256);
+    s->off_V = s->off_Mam = s->off_Vam = o;
   } else {
     s->off_M = o; o += align_up((size_t)s->srows * s->ld_s, 256);
     s->off_V = o; o += align_up((size_t)s->srows * s->ld_s, 256);
@@ -178,6 +188,8 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
   s->off_status = o; o += 256;
   s->off_R = o; o += align_up(std::max((size_t)s->proj_splits * s->nel, (size_t)s->tc_splits * s->srows * s->ld_part) * 4, 256);
   s->off_N = o; o += align_up(std::max((size_t)s->nel * 4, (size_t)s->srows * s->ld_n * 2), 256);
+  s->off_af = o;
+  if (c->state_fmt == GALORE_STATE_ADAFACTOR) o += adafactor_scratch_bytes(s->srows, s->scols);
   s->off_refresh = o; o += refresh_workspace_bytes(s->d, s->L, r, s->block);
   s->ws_bytes = o;
   return GALORE_OK;
@@ -220,6 +232,21 @@ AdamItem adam_item(const galore_layer* l, const float* part, int splits, int64_t
   return a;
 }
 
+// the layer's Adafactor step on the same buffers
+galore_status_t launch_regulariser(const galore_layer* l, const AdamItem& a, int32_t n_dtype, cudaStream_t st) {
+  if (l->cfg.state_fmt != GALORE_STATE_ADAFACTOR) return launch_adam(a, l->cfg.state_fmt, l->q_block, n_dtype, st);
+  AdafactorItem f = {};
+  f.Rpart = const_cast<float*>(a.Rpart); f.splits = a.splits; f.split_stride = a.split_stride;
+  f.rows = a.rows; f.cols = a.cols;
+  f.r_ld = a.r_ld; f.n_ld = a.n_ld; f.s_ld = a.s_ld;
+  f.M = l->M; f.v_row = l->v_row; f.v_col = l->v_col;
+  f.Nout = a.Nout;
+  f.beta1 = (float)l->cfg.beta1;
+  f.t = (double)(l->k + 1);
+  f.scratch = l->af_scratch;
+  return launch_adafactor(f, n_dtype, st);
+}
+
 // GaLore-AdamW: W is multiplied by 1 - lr * lambda in the pass that subtracts the update (exactly 1 for lambda = 0)
 inline float decay_keep(const galore_layer* l, float lr) { return (float)(1.0 - (double)lr * (double)l->cfg.weight_decay); }
 
@@ -247,8 +274,7 @@ galore_status_t step_simt(galore_layer* l, void* W, int64_t ldw, const void* G, 
   }
   {
     PhaseTimer pt(1, st);
-    GALORE_TRY(launch_adam(adam_item(l, l->Rpart, l->proj_splits, l->nel, l->scols, l->Nbuf, l->scols, ap), l->cfg.state_fmt,
-                           l->q_block, GALORE_F32, st));
+    GALORE_TRY(launch_regulariser(l, adam_item(l, l->Rpart, l->proj_splits, l->nel, l->scols, l->Nbuf, l->scols, ap), GALORE_F32, st));
   }
   PhaseTimer pt(2, st);
   const float scale = lr * l->cfg.alpha, keep = decay_keep(l, lr);
@@ -282,7 +308,7 @@ TcAdamArgs tc_adam_args(const galore_layer* l, void* nbuf, const AdamParams& ap)
 
 // Adam in the projection's epilogue?  Only when K is not sliced; AUTO: see the note at its definition.
 bool adam_in_projection(const galore_layer* l, int splits) {
-  if (splits != 1 || l->cfg.adam_place == GALORE_ADAM_OWN_KERNEL) return false;
+  if (splits != 1 || l->cfg.adam_place == GALORE_ADAM_OWN_KERNEL || l->cfg.state_fmt == GALORE_STATE_ADAFACTOR) return false;
   if (l->cfg.adam_place == GALORE_ADAM_IN_PROJECTION) return true;
   return kAutoFuses[l->cfg.state_fmt == GALORE_STATE_F32 ? 0 : 1];
 }
@@ -300,8 +326,8 @@ galore_status_t step_tensor(galore_layer* l, void* W, int64_t ldw, const void* G
   }
   {
     PhaseTimer pt(1, st);
-    GALORE_TRY(launch_adam(adam_item(l, l->Rpart, l->tc.splits, l->srows * l->ld_part, l->ld_part, l->Nbuf, l->ld_n, ap),
-                           l->cfg.state_fmt, l->q_block, GALORE_BF16, st));
+    GALORE_TRY(launch_regulariser(l, adam_item(l, l->Rpart, l->tc.splits, l->srows * l->ld_part, l->ld_part, l->Nbuf, l->ld_n, ap),
+                                  GALORE_BF16, st));
    }
   }
   PhaseTimer pt(2, st);
@@ -382,9 +408,15 @@ galore_status_t galore_init_layer(const galore_config_t* cfg, void* state_buf, s
   char* ws = (char*)workspace;
   l->P = sb + s.off_P;
   l->M = l->V = nullptr; l->Mc = l->Vc = nullptr; l->Mam = l->Vam = nullptr;
+  l->v_row = l->v_col = nullptr; l->af_scratch = nullptr;
   if (cfg->state_fmt == GALORE_STATE_F32) {
     l->M = (float*)(sb + s.off_M);
     l->V = (float*)(sb + s.off_V);
+  } else if (cfg->state_fmt == GALORE_STATE_ADAFACTOR) {
+    l->M = (float*)(sb + s.off_M);
+    l->v_row = (float*)(sb + s.off_vrow);
+    l->v_col = (float*)(sb + s.off_vcol);
+    l->af_scratch = (float*)(ws + s.off_af);
   } else {
     l->Mc = (uint8_t*)(sb + s.off_M);
     l->Vc = (uint8_t*)(sb + s.off_V);
@@ -401,6 +433,10 @@ galore_status_t galore_init_layer(const galore_config_t* cfg, void* state_buf, s
   if (cfg->state_fmt == GALORE_STATE_F32) {
     e = cudaMemsetAsync(l->M, 0, (size_t)l->srows * l->ld_s * 4, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(l->V, 0, (size_t)l->srows * l->ld_s * 4, st);
+  } else if (cfg->state_fmt == GALORE_STATE_ADAFACTOR) {
+    e = cudaMemsetAsync(l->M, 0, (size_t)l->srows * l->ld_s * 4, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(l->v_row, 0, (size_t)l->srows * 4, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(l->v_col, 0, (size_t)l->scols * 4, st);
   } else {
     e = cudaMemsetAsync(l->Mc, 127, (size_t)l->srows * l->ld_s, st);   // 127 and 0 are the codes of the value 0
     if (e == cudaSuccess) e = cudaMemsetAsync(l->Vc, 0, (size_t)l->srows * l->ld_s, st);
@@ -645,7 +681,9 @@ size_t batch_layer_bytes(const galore_layer* l, int splits) {
 int batch_splits(const galore_layer* l, int eligible) { return batch_unsliced(eligible) ? 1 : l->tc_splits; }
 
 bool batch_eligible(const galore_layer* l, const void* W, int64_t ldw, const void* G, int64_t ldg) {
-  return l->tensor_path && l->has_projector && tensor_operands_aligned(l->cfg, W, ldw, G, ldg);
+  // (Adafactor's statistics span the whole of R: its layers step one by one)
+  return l->tensor_path && l->has_projector && l->cfg.state_fmt != GALORE_STATE_ADAFACTOR &&
+         tensor_operands_aligned(l->cfg, W, ldw, G, ldg);
 }
 
 AdamParams adam_params(const galore_layer* l) {
@@ -889,9 +927,21 @@ galore_status_t galore_get_moments(galore_layer_t* l, float* M, float* V, size_t
     GALORE_CUDA_TRY(cudaMemcpy2DAsync(V, row, l->V, (size_t)l->ld_s * 4, row, (size_t)l->srows, cudaMemcpyDeviceToDevice, st));
     return GALORE_OK;
   }
+  if (l->cfg.state_fmt != GALORE_STATE_Q8_BLOCK) return GALORE_ERR_STATE;   // Adafactor: galore_get_adafactor_state
   const int tr = l->q_block / kStateTileCols;
   GALORE_TRY(launch_q8_dequantize(l->Mc, l->ld_s, l->Mam, l->srows, l->scols, 1, tr, kStateTileCols, M, l->scols, st));
   return launch_q8_dequantize(l->Vc, l->ld_s, l->Vam, l->srows, l->scols, 0, tr, kStateTileCols, V, l->scols, st);
+}
+
+galore_status_t galore_get_adafactor_state(galore_layer_t* l, float* M, float* v_row, float* v_col, void* stream) {
+  if (!l || !M || !v_row || !v_col) return GALORE_ERR_INVALID_ARG;
+  if (l->cfg.state_fmt != GALORE_STATE_ADAFACTOR) return GALORE_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t row = (size_t)l->scols * 4;
+  GALORE_CUDA_TRY(cudaMemcpy2DAsync(M, row, l->M, (size_t)l->ld_s * 4, row, (size_t)l->srows, cudaMemcpyDeviceToDevice, st));
+  GALORE_CUDA_TRY(cudaMemcpyAsync(v_row, l->v_row, (size_t)l->srows * 4, cudaMemcpyDeviceToDevice, st));
+  GALORE_CUDA_TRY(cudaMemcpyAsync(v_col, l->v_col, (size_t)l->scols * 4, cudaMemcpyDeviceToDevice, st));
+  return GALORE_OK;
 }
 
 galore_status_t galore_get_q8_state(galore_layer_t* l, uint8_t* Mc, float* Mam, uint8_t* Vc, float* Vam, void* stream) {

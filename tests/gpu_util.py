@@ -132,8 +132,9 @@ def run_pair(m, n, r, steps, T, w_dtype="f32", g_dtype="f32", state_fmt="f32", p
     side_name = "left" if layer.side == gb.SIDE_LEFT else "right"
     n_store = "bf16" if layer.uses_tensor_path else "f64"
     orc = go.GaLoreOracle(m, n, r, 0.25, T, side=side_name, w_store=w_dtype, n_store=n_store,
-                          state={"f32": "f32", "q8": "q8"}[state_fmt], q_block=q_block, svd_method=svd_method,
-                          weight_decay=weight_decay)
+                          state={"f32": "f32", "q8": "q8", "adafactor": "f32"}[state_fmt], q_block=q_block,
+                          svd_method=svd_method, weight_decay=weight_decay,
+                          inner="adafactor" if state_fmt == "adafactor" else "adam")
     W0 = wl.make_weight(m, n, wl.sub_seed(seed, 999), w_dtype)
     W_orc = W0.copy()
     W_gpu = to_dev(W0, w_dtype, ldw)

@@ -36,7 +36,7 @@ def test_config_struct_layout_matches_header():
     assert gb.lib().galore_abi_sizes(C.byref(a), C.byref(b)) == 0
     assert (a.value, b.value) == (C.sizeof(gb.Config), C.sizeof(gb.RefreshInfo))
     assert gb.Config.seed.offset % 8 == 0
-    assert C.sizeof(gb.RefreshInfo) == 88
+    assert C.sizeof(gb.RefreshInfo) == 96
 
 
 def test_query_bytes_follows_memory_model():
