@@ -57,9 +57,19 @@ def algorithmic_cost(w, m, n):
     left = m <= n
     d, big = (m, n) if left else (n, m)
     nel = r * big
-    state = 4 * nel * 4 if w.state_fmt == "f32" else 4 * nel + 4 * 4 * ((nel + w.q_block - 1) // w.q_block)
+    state = state_bytes_per_step(w, nel, r, big)
     by = m * n * elem_bytes(w.g_dtype) + 2 * m * n * elem_bytes(w.w_dtype) + state + d * r * elem_bytes(p_dtype_of(w))
     return by, 4 * m * n * r
+
+
+def state_bytes_per_step(w, nel, r, big):
+    """Optimizer statistics read and written once per step: two fp32 moments, two 8-bit moments with their
+    absmax values, or Adafactor's fp32 first moment with one value per row and per column of R."""
+    if w.state_fmt == "f32":
+        return 4 * nel * 4
+    if w.state_fmt == "adafactor":
+        return 2 * nel * 4 + 2 * (r + big) * 4
+    return 4 * nel + 4 * 4 * ((nel + w.q_block - 1) // w.q_block)
 
 
 def p_dtype_of(w):
@@ -89,7 +99,7 @@ def kernel_costs(w, shapes):
         r = w.rank
         d, big = (m, n) if m <= n else (n, m)
         nel = r * big
-        state = 4 * nel * 4 if w.state_fmt == "f32" else 4 * nel + 4 * 4 * ((nel + w.q_block - 1) // w.q_block)
+        state = state_bytes_per_step(w, nel, r, big)
         p_bytes = d * r * elem_bytes(p_dtype_of(w))
         proj["flops"] += 2 * m * n * r
         proj["bytes"] += m * n * elem_bytes(w.g_dtype) + p_bytes
@@ -186,7 +196,8 @@ def cpu_oracle_sample(w, steps=1, extras=False):
     for (m, n, _count) in w.shapes:
         side = "left" if m <= n else "right"
         orc = go.GaLoreOracle(m, n, w.rank, w.alpha, w.refresh_gap, w.beta1, w.beta2, w.eps, w_store=w.w_dtype,
-                              state=w.state_fmt, q_block=w.q_block)
+                              state="f32" if w.state_fmt == "adafactor" else w.state_fmt, q_block=w.q_block,
+                              inner="adafactor" if w.state_fmt == "adafactor" else "adam")
         d = m if side == "left" else n
         P, _ = np.linalg.qr(rng.standard_normal((d, w.rank)))       # any orthonormal projector: timing only
         orc.set_projector(P)
@@ -268,14 +279,14 @@ def main():
                     help="keep only this many transformer layers of the workload's layer set (0 = all): a small case "
                          "of the same kernels for profiler captures")
     ap.add_argument("--rank", type=int, default=0, help="override the workload's rank (rank sweep on one shape)")
-    ap.add_argument("--state-fmt", default="", choices=["", "f32", "q8"], help="override the workload's state format")
+    ap.add_argument("--state-fmt", default="", choices=["", "f32", "q8", "adafactor"], help="override the workload's state format")
     ap.add_argument("--refresh-warm", type=int, default=0,
                     help="power steps of a refresh started from the stored projector (0: every refresh starts cold); "
                          "with N > 0 the whole set is also refreshed a second time from slightly moved gradients")
     ap.add_argument("--refresh-only", action="store_true",
                     help="run the projector refresh of each distinct shape and print its timings; no step is timed "
                          "(for profiling the refresh on its own)")
-    ap.add_argument("--extra-workloads", default="llama_1b_q8,llama_1b_f32,llama_130m,sweep",
+    ap.add_argument("--extra-workloads", default="llama_1b_q8,llama_1b_f32,llama_1b_adafactor,llama_130m,sweep",
                     help="comma-separated workloads also timed, device-resident only, reported under other_workloads "
                          "(only with the default workload; empty string to skip).  'sweep' = the rank sweep on one "
                          "4096 x 11008 matrix: six ranks x both state formats, one matrix per step, with the refresh "

@@ -30,4 +30,17 @@ struct AdafactorItem {
 size_t adafactor_scratch_bytes(int64_t rows, int64_t cols);
 galore_status_t launch_adafactor(const AdafactorItem& item, int32_t n_dtype, cudaStream_t st);
 
+// Several layers in the same launches (every reduction stays inside its layer and keeps its order: a
+// layer's result does not depend on what it is grouped with).  All items share the dtype of N.
+constexpr int kAdafactorGroup = 32;
+struct AdafactorGroup {
+  AdafactorItem item[kAdafactorGroup];
+  int tile_end[kAdafactorGroup];     // running totals of the statistics pass's tiles
+  int vec_end[kAdafactorGroup];      // running totals of the 256-entry blocks of v_row | v_col
+  float beta2t[kAdafactorGroup];
+  int count;
+};
+galore_status_t adafactor_group_add(AdafactorGroup& g, const AdafactorItem& item);
+galore_status_t launch_adafactor_group(const AdafactorGroup& g, int32_t n_dtype, cudaStream_t st);
+
 }  // namespace galore

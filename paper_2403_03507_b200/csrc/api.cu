@@ -233,8 +233,7 @@ AdamItem adam_item(const galore_layer* l, const float* part, int splits, int64_t
 }
 
 // the layer's Adafactor step on the same buffers
-galore_status_t launch_regulariser(const galore_layer* l, const AdamItem& a, int32_t n_dtype, cudaStream_t st) {
-  if (l->cfg.state_fmt != GALORE_STATE_ADAFACTOR) return launch_adam(a, l->cfg.state_fmt, l->q_block, n_dtype, st);
+AdafactorItem adafactor_item(const galore_layer* l, const AdamItem& a, float* scratch) {
   AdafactorItem f = {};
   f.Rpart = const_cast<float*>(a.Rpart); f.splits = a.splits; f.split_stride = a.split_stride;
   f.rows = a.rows; f.cols = a.cols;
@@ -243,8 +242,12 @@ galore_status_t launch_regulariser(const galore_layer* l, const AdamItem& a, int
   f.Nout = a.Nout;
   f.beta1 = (float)l->cfg.beta1;
   f.t = (double)(l->k + 1);
-  f.scratch = l->af_scratch;
-  return launch_adafactor(f, n_dtype, st);
+  f.scratch = scratch;
+  return f;
+}
+galore_status_t launch_regulariser(const galore_layer* l, const AdamItem& a, int32_t n_dtype, cudaStream_t st) {
+  if (l->cfg.state_fmt != GALORE_STATE_ADAFACTOR) return launch_adam(a, l->cfg.state_fmt, l->q_block, n_dtype, st);
+  return launch_adafactor(adafactor_item(l, a, l->af_scratch), n_dtype, st);
 }
 
 // GaLore-AdamW: W is multiplied by 1 - lr * lambda in the pass that subtracts the update (exactly 1 for lambda = 0)
@@ -673,17 +676,18 @@ bool batch_unsliced(int eligible) { return eligible >= 4; }
 size_t batch_r_bytes(const galore_layer* l, int splits) {
   return adam_in_projection(l, splits) ? 0 : align_up((size_t)splits * l->srows * l->ld_part * 4, 256);
 }
+size_t batch_n_bytes(const galore_layer* l) { return align_up((size_t)l->srows * l->ld_n * 2, 256); }
+// R partials, N and, for Adafactor, the scratch of its reductions (layers of a group run in the same launches)
 size_t batch_layer_bytes(const galore_layer* l, int splits) {
-  return batch_r_bytes(l, splits) + align_up((size_t)l->srows * l->ld_n * 2, 256);
+  return batch_r_bytes(l, splits) + batch_n_bytes(l) +
+         (l->cfg.state_fmt == GALORE_STATE_ADAFACTOR ? adafactor_scratch_bytes(l->srows, l->scols) : 0);
 }
 
 // With several layers in flight there are enough tiles to fill the machine without slicing K.
 int batch_splits(const galore_layer* l, int eligible) { return batch_unsliced(eligible) ? 1 : l->tc_splits; }
 
 bool batch_eligible(const galore_layer* l, const void* W, int64_t ldw, const void* G, int64_t ldg) {
-  // (Adafactor's statistics span the whole of R: its layers step one by one)
-  return l->tensor_path && l->has_projector && l->cfg.state_fmt != GALORE_STATE_ADAFACTOR &&
-         tensor_operands_aligned(l->cfg, W, ldw, G, ldg);
+  return l->tensor_path && l->has_projector && tensor_operands_aligned(l->cfg, W, ldw, G, ldg);
 }
 
 AdamParams adam_params(const galore_layer* l) {
@@ -694,10 +698,12 @@ struct BatchScratch {   // host-side objects reused across calls on this thread
   TensorGroup* proj = nullptr;
   TensorGroup* back = nullptr;
   AdamGroup* adam = nullptr;
+  AdafactorGroup* adafactor = nullptr;
   ~BatchScratch() {
     tensor_group_free(proj);
     tensor_group_free(back);
     delete adam;
+    delete adafactor;
   }
 };
 
@@ -756,8 +762,9 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
   if (!scratch.proj) scratch.proj = tensor_group_new();
   if (!scratch.back) scratch.back = tensor_group_new();
   if (!scratch.adam) scratch.adam = new (std::nothrow) AdamGroup;
-  if (!scratch.proj || !scratch.back || !scratch.adam) return GALORE_ERR_INVALID_ARG;
-  const int cap = std::min(tensor_group_capacity(), (int)kAdamGroup);
+  if (!scratch.adafactor) scratch.adafactor = new (std::nothrow) AdafactorGroup;
+  if (!scratch.proj || !scratch.back || !scratch.adam || !scratch.adafactor) return GALORE_ERR_INVALID_ARG;
+  const int cap = std::min(tensor_group_capacity(), std::min((int)kAdamGroup, (int)kAdafactorGroup));
 
   // ---- 1. partition: layers that cannot be grouped step on their own, the rest form groups ----------
   // Two groups are in flight at a time, each in its own half of the workspace.
@@ -833,15 +840,21 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
   };
   auto launch_adam = [&](size_t gi, cudaStream_t s) -> galore_status_t {
     scratch.adam->count = 0;
+    scratch.adafactor->count = 0;
     const galore_layer* first = layers[groups[gi][0].index];
+    const bool adafactor = first->cfg.state_fmt == GALORE_STATE_ADAFACTOR;
     for (const BatchMember& mb : groups[gi]) {
       galore_layer* l = layers[mb.index];
       float* part; void* nbuf;
       scratch_of(gi, mb, &part, &nbuf);
       const AdamItem a = adam_item(l, part, mb.splits, l->srows * l->ld_part, l->ld_part, nbuf, l->ld_n, adam_params(l));
-      GALORE_TRY(adam_group_add(*scratch.adam, a, l->cfg.state_fmt, l->q_block));
+      if (adafactor)
+        GALORE_TRY(adafactor_group_add(*scratch.adafactor, adafactor_item(l, a, (float*)((char*)nbuf + batch_n_bytes(l)))));
+      else
+        GALORE_TRY(adam_group_add(*scratch.adam, a, l->cfg.state_fmt, l->q_block));
     }
     PhaseTimer pt(1, s);
+    if (adafactor) return launch_adafactor_group(*scratch.adafactor, GALORE_BF16, s);
     return launch_adam_group(*scratch.adam, first->cfg.state_fmt, first->q_block, GALORE_BF16, s);
   };
   auto launch_back = [&](size_t gi, cudaStream_t s) -> galore_status_t {

@@ -32,7 +32,7 @@ class Workload:
     refresh_gap: int
     w_dtype: str             # 'f32' | 'bf16'
     g_dtype: str
-    state_fmt: str           # 'f32' | 'q8'
+    state_fmt: str           # 'f32' | 'q8' (Adam moments) | 'adafactor'
     spectrum_p: float
     noise: float
     lr: float = 1e-2
@@ -64,6 +64,8 @@ WORKLOADS = {
                              0.8, 0.05, seed=BASE_SEED + 2),
     "llama_1b_q8": Workload("llama_1b_q8", _llama(24, 2048, 5461), 512, 0.25, 200, "bf16", "bf16", "q8",
                             0.8, 0.05, seed=BASE_SEED + 2),
+    "llama_1b_adafactor": Workload("llama_1b_adafactor", _llama(24, 2048, 5461), 512, 0.25, 200, "bf16", "bf16",
+                                   "adafactor", 0.8, 0.05, seed=BASE_SEED + 2),
     "llama_7b_q8": Workload("llama_7b_q8", _llama(32, 4096, 11008), 1024, 0.25, 500, "bf16", "bf16", "q8",
                             0.8, 0.05, seed=BASE_SEED + 3),
     "sweep_4096x11008": Workload("sweep_4096x11008", ((4096, 11008, 1),), 1024, 0.25, 200, "bf16", "bf16", "q8",
