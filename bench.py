@@ -76,12 +76,16 @@ def p_dtype_of(w):
     return "bf16" if w.g_dtype == "bf16" else "f32"
 
 
-# DRAM traffic per launch of the step's kernels from ncu captures of the kernels as they are now
-# (dram__bytes_read.sum + dram__bytes_write.sum, summarised under profiles/ with the command that made
-# them), as bytes per parameter covered by the launch: traffic grows in proportion to the matrices a
-# launch covers.  None: not captured since the kernel last changed.
-KERNEL_DRAM_BYTES_PER_PARAM = {
-    # (workload rank, state format): {"projection": ..., "back_projection": ...}
+# DRAM traffic of the step's kernels from ncu captures of the kernels as they are now (dram__bytes_read.sum +
+# dram__bytes_write.sum of one launch over a group of attention-shaped matrices, summarised under profiles/
+# with the command that made them), as a multiple of the algorithmic bytes of that launch (kernel_costs
+# below).  Traffic grows in proportion to the matrices a launch covers, so a full-size launch is taken to
+# move the same multiple of its own algorithmic bytes.  Absent: not captured since the kernel last changed.
+KERNEL_DRAM_OVER_ALGORITHMIC = {
+    # (rank, state format): {kernel: measured / algorithmic}
+    # (the fp32 R the projection writes and the Adam kernel reads, 134.2 MB here, is traffic the method does not need)
+    (1024, "q8"): {"projection": 607.6 / 335.5, "adam": 405.3 / 201.3, "back_projection": 830.0 / 671.1},
+    (512, "f32"): {"projection_with_adam": 560.9 / 469.8, "back_projection": 438.1 / 335.5},
 }
 
 
@@ -560,11 +564,13 @@ def time_workload(w, args, dev, dist, world, rank, full, mode=None):
     kernels = {"projection_with_adam" if fused else "projection": kernel_entry(phase_ms[0], phase_cnt[0], kp),
                "adam": kernel_entry(phase_ms[1], phase_cnt[1], ka),
                "back_projection": kernel_entry(phase_ms[2], phase_cnt[2], kb)}
-    traffic = KERNEL_DRAM_BYTES_PER_PARAM.get((w.rank, w.state_fmt))
+    ratios = KERNEL_DRAM_OVER_ALGORITHMIC.get((w.rank, w.state_fmt))
+    alg_bytes = {"projection_with_adam": kp["bytes"], "projection": kp["bytes"], "adam": ka["bytes"], "back_projection": kb["bytes"]}
+    traffic = ({k: v * alg_bytes[k] / max(1.0, kernels[k]["launches_per_step"]) for k, v in ratios.items() if kernels.get(k)}
+               if ratios else None)
     roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": t_roof * 1e3 / ms_step,
-            "traffic": ({k: v * w.params / max(1.0, kernels[k]["launches_per_step"]) for k, v in traffic.items() if kernels.get(k)}
-                        if traffic else None),
-            "traffic_unit": "DRAM bytes per launch, by kernel, scaled from the ncu capture by the parameters a launch covers",
+            "traffic": traffic,
+            "traffic_unit": "DRAM bytes per launch, by kernel: the ncu capture's multiple of the algorithmic bytes times the algorithmic bytes of an average launch",
             "peak_source": peaks["source"] + (" (sustained bf16 GEMM)" if bound == "tensor" else " (copy bandwidth)" if bound == "hbm" else " (unit counts x max clock)"),
             "scope": "whole step: algorithmic bytes and flops of every matrix / measured step time",
             "kernels": {k: v for k, v in kernels.items() if v},

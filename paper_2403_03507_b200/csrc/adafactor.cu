@@ -76,10 +76,10 @@ __global__ void __launch_bounds__(kAfTileCols) af_stats_kernel(const __grid_cons
   const int r0 = tile_r * kAfTileRows, c0 = tile_c * kAfTileCols + 4 * lane;
   const bool vec = (it.r_ld % 4) == 0 && (it.split_stride % 4) == 0 && ((uintptr_t)it.Rpart & 15) == 0 && c0 + 3 < it.cols;
   float col[4] = {0.f, 0.f, 0.f, 0.f};
-  for (int i = warp; i < kAfTileRows; i += kAfTileCols / 32) {
-    const int row = r0 + i;
-    if (row >= it.rows) break;
-    float v[4] = {0.f, 0.f, 0.f, 0.f};
+  // the four columns of one row: the sum of the K slices, written back when there are several
+  auto load_row = [&](int row, float (&v)[4]) {
+    v[0] = v[1] = v[2] = v[3] = 0.f;
+    if (row >= it.rows) return;
     const int64_t at = (int64_t)row * it.r_ld + c0;
     if (vec) {
       float4 x = *reinterpret_cast<const float4*>(it.Rpart + at);
@@ -99,16 +99,26 @@ __global__ void __launch_bounds__(kAfTileCols) af_stats_kernel(const __grid_cons
           v[k] = x;
         }
     }
-    float row_sum = 0.f;
+  };
+  constexpr int kWarps = kAfTileCols / 32, kFlight = 4;      // four rows of a warp in flight
+  for (int i = warp; i < kAfTileRows; i += kWarps * kFlight) {
+    float v[kFlight][4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const float sq = v[k] * v[k];
-      col[k] += sq;
-      row_sum += sq;
+    for (int u = 0; u < kFlight; ++u) load_row(r0 + i + u * kWarps, v[u]);
+#pragma unroll
+    for (int u = 0; u < kFlight; ++u) {
+      const int row = r0 + i + u * kWarps;
+      float row_sum = 0.f;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float sq = v[u][k] * v[u][k];
+        col[k] += sq;
+        row_sum += sq;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) row_sum += __shfl_xor_sync(0xffffffffu, row_sum, o);
+      if (lane == 0 && row < it.rows) a.rowpart[(size_t)row * a.tiles_c + tile_c] = row_sum;
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) row_sum += __shfl_xor_sync(0xffffffffu, row_sum, o);
-    if (lane == 0) a.rowpart[(size_t)row * a.tiles_c + tile_c] = row_sum;
   }
 #pragma unroll
   for (int k = 0; k < 4; ++k) cs[warp][4 * lane + k] = col[k];
