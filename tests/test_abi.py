@@ -54,6 +54,12 @@ def test_query_bytes_follows_memory_model():
     nel = 1024 * 11008
     assert sb8 == 2 * 4096 * 1024 + 2 * nel + 2 * 4 * (nel // 2048)
     assert wb > 0
+    # Adafactor: first moment plus one value per row and per column of R (fp32 everywhere here), parts padded to 256 bytes
+    cfa = gb.make_config(m, n, r, w_dtype="f32", g_dtype="f32", state_fmt="adafactor")
+    sba, _ = gb.galore_query_bytes(cfa)
+    pad = lambda b: (b + 255) // 256 * 256
+    assert sba == pad(4 * m * r) + pad(4 * r * n) + pad(4 * r) + pad(4 * n)
+    assert 0 <= sba - 4 * go.GaLoreOracle(m, n, r, 0.25, 5, inner="adafactor").optimizer_state_elements() < 4 * 256
 
 
 @pytest.mark.parametrize("kw,status", [
