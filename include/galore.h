@@ -16,6 +16,8 @@
  *     leading dimension given in ELEMENTS, unless an argument says "host".
  *   - The caller passes the gradient (not its negative) and the update is
  *     subtracted.
+ *   - Timeline tools see NVTX ranges named galore.project, galore.adam, galore.back_project and
+ *     galore.refresh (with .steps and .rayleigh_ritz inside) on the calling thread.
  *   - The library allocates no device memory: the optimizer state and a
  *     scratch workspace are caller-allocated device buffers whose sizes come
  *     from galore_query_bytes() and which must outlive the handle.  A

@@ -45,7 +45,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if failed:
         raise RuntimeError("nvcc failed")
     subprocess.run(["nvcc", "-shared", "-o", LIB] + objs + ["-gencode", "arch=compute_100a,code=sm_100a",
-                                                             "-Xcompiler", "-fPIC", "-lcuda"], check=True)
+                                                             "-Xcompiler", "-fPIC", "-lcuda", "-ldl"], check=True)
     return LIB
 
 

@@ -35,11 +35,13 @@ static std::atomic<int> g_profile{0};
 static std::mutex g_profile_mutex;
 static std::vector<PhaseEvent> g_phase_events;
 
+static const char* const kPhaseNames[3] = {"galore.project", "galore.adam", "galore.back_project"};
 struct PhaseTimer {
+  NvtxRange range;      // the phase on the host timeline (launches are asynchronous: the kernels follow on the stream)
   bool on;
   PhaseEvent ev;
   cudaStream_t st;
-  PhaseTimer(int phase, cudaStream_t s) : on(g_profile.load(std::memory_order_relaxed) != 0), st(s) {
+  PhaseTimer(int phase, cudaStream_t s) : range(kPhaseNames[phase]), on(g_profile.load(std::memory_order_relaxed) != 0), st(s) {
     if (!on) return;
     ev.phase = phase;
     if (cudaEventCreate(&ev.a) != cudaSuccess || cudaEventCreate(&ev.b) != cudaSuccess) { on = false; return; }

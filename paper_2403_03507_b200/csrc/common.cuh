@@ -1,6 +1,8 @@
 // Shared host/device helpers of the GaLore CUDA library (sm_100a).
 #pragma once
 
+#include <nvtx3/nvToolsExt.h>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -89,6 +91,14 @@ __host__ __device__ __forceinline__ T* slot_ptr(T* p, int64_t shift) {
 struct DeviceStatus {
   int32_t flags;
   int32_t pad[63];
+};
+
+// A named range on the calling thread for timeline tools (NVTX; a few nanoseconds when no tool listens).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+  NvtxRange(const NvtxRange&) = delete;
+  NvtxRange& operator=(const NvtxRange&) = delete;
 };
 
 }  // namespace galore

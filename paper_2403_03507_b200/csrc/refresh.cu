@@ -863,6 +863,7 @@ template <typename TG>
 static galore_status_t refresh_group(const RefreshProblem* prs, int count, void* workspace, size_t slot_bytes,
                                      int32_t* const* status, galore_refresh_info_t* infos, cudaStream_t st) {
   if (count < 1 || count > kMaxSlots) return GALORE_ERR_INVALID_ARG;
+  NvtxRange whole("galore.refresh");
   const RefreshProblem& p0 = prs[0];
   Ctx c = {};
   c.base0 = (char*)workspace;
@@ -1102,7 +1103,11 @@ static galore_status_t refresh_group(const RefreshProblem* prs, int count, void*
   std::vector<Lane*> live = all;            // lanes that still iterate
   while (!live.empty()) {
     // ---- power steps: every lane up to its own target, on its own orthonormalisation schedule ----
-    GALORE_TRY(run_steps(live));
+    {
+      NvtxRange range("galore.refresh.steps");
+      GALORE_TRY(run_steps(live));
+    }
+    NvtxRange range("galore.refresh.rayleigh_ritz");
     for (Lane* l : live) {
       l->p64_current = false;
       l->info.ritz_passes += 1;

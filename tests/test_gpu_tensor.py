@@ -86,6 +86,34 @@ def test_tensor_path_q8_states_with_padded_rows(m, n, r, qb):
     assert np.mean(Vc != orc.V_codes) < 5e-3 and np.max(np.abs(cu[Vc] - cu[orc.V_codes])) <= 2 * 0.9 / 128 + 1e-6
 
 
+@pytest.mark.parametrize("m,n,r", [(512, 1024, 128), (1024, 512, 256)])
+def test_error_against_the_unrounded_normalised_update_is_reported(m, n, r):
+    """The tensor path feeds the back-projection a bf16 N; the oracle is normally run with the same rounding of
+    N (n_store="bf16").  Here the error against the oracle that keeps N in fp64 is measured beside it: it is
+    larger by the rounding of N (2^-9 relative per element) and still inside the bars."""
+    steps = 3
+    cfg = gb.make_config(m, n, r, refresh_gap=1000, w_dtype="f32", g_dtype="bf16", state_fmt="f32", auto_refresh=False)
+    layer = gb.Layer(cfg)
+    left = layer.side == gb.SIDE_LEFT
+    P = wl.round_to(wl.random_orthonormal(m if left else n, r, np.random.default_rng(2)), "bf16")
+    layer.set_projector(torch.from_numpy(P))
+    orcs = {ns: go.GaLoreOracle(m, n, r, 0.25, 1000, w_store="f32", state="f32", n_store=ns) for ns in ("bf16", "f64")}
+    for o in orcs.values():
+        o.set_projector(P)
+    W0 = wl.make_weight(m, n, 3, "f32")
+    Wg = to_dev(W0, "f32")
+    Wo = {ns: W0 for ns in orcs}
+    for s in range(steps):
+        G = wl.make_gradient(m, n, wl.sub_seed(6, s), 0.8, 0.05, "bf16")
+        layer.galore_step(Wg, to_dev(G, "bf16"), 1e-2)
+        for ns, o in orcs.items():
+            Wo[ns] = o.step(Wo[ns], G, 1e-2, auto_refresh=False)
+    err = {ns: rel_err(to_host(Wg) - W0, Wo[ns] - W0) for ns in orcs}
+    print(f"{m}x{n} r={r}: update error against the oracle with N rounded to bf16 {err['bf16']:.2e}, with N in fp64 {err['f64']:.2e}")
+    assert layer.uses_tensor_path
+    assert err["bf16"] < 2e-3 and err["f64"] < 5e-3 and err["bf16"] <= err["f64"]
+
+
 def test_unaligned_leading_dimension_falls_back_or_errors():
     # n = 5461 packed: rows are not 16-byte aligned, TMA cannot address them
     m, n, r = 256, 1001, 32

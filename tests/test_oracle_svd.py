@@ -75,6 +75,17 @@ def test_jacobi_agrees_with_library_svd_on_workload_spectrum():
         assert go.largest_principal_angle(Pj, Pl) < 1e-8
 
 
+def test_library_shortcut_agrees_with_jacobi_at_the_60m_mlp_shape():
+    """`method="lapack"` stands in for the Jacobi code at sizes it cannot reach in test time; here both run on
+    the full 512 x 1376 matrix of the smallest workload (rank 128, the workload's own noise-dominated recipe)."""
+    G = wl.make_gradient(512, 1376, seed=11, p=1.0, noise=0.01, dtype="f32")
+    Pj, Sj = go.top_r_projector(G, 128, "left", method="jacobi")
+    Pl, Sl = go.top_r_projector(G, 128, "left", method="lapack")
+    assert np.allclose(Sj, Sl, rtol=1e-11)
+    assert go.largest_principal_angle(Pj, Pl) < 1e-7
+    assert np.abs(Pj.T @ Pj - np.eye(128)).max() < 1e-12
+
+
 def test_principal_angle_of_known_rotation():
     # two planes in R^3 sharing e1, second axis tilted by 0.3 rad
     A = np.array([[1, 0], [0, 1], [0, 0]], float)
