@@ -148,18 +148,17 @@ __device__ __forceinline__ float warp_max(float v) {
 // max of two values over the CTA (256 threads) with a single barrier; every thread gets both.
 // `red` is one of two alternating 16-float buffers: a buffer is written again two calls later, and
 // the barrier of the call in between separates that from the last reads of this one.
-__device__ __forceinline__ void block_max2_256(float& x, float& y, float* red /* 16 floats */) {
-  x = warp_max(x);
-  y = warp_max(y);
-  if ((threadIdx.x & 31) == 0) {
-    red[threadIdx.x >> 5] = x;
-    red[8 + (threadIdx.x >> 5)] = y;
-  }
+// x and y are bit patterns of non-negative floats (their order is the order of the values): one
+// hardware warp reduction each, the eight warps' results through shared memory, one more reduction.
+__device__ __forceinline__ void block_max2_256(uint32_t& x, uint32_t& y, float* red /* 16 floats */) {
+  uint2* __restrict__ slots = reinterpret_cast<uint2*>(red);                 // 8-byte aligned (Q8Tables)
+  x = __reduce_max_sync(0xffffffffu, x);
+  y = __reduce_max_sync(0xffffffffu, y);
+  if ((threadIdx.x & 31) == 0) slots[threadIdx.x >> 5] = make_uint2(x, y);
   __syncthreads();
-  const float4* __restrict__ q = reinterpret_cast<const float4*>(red);      // 16-byte aligned (Q8Tables)
-  const float4 a = q[0], b = q[1], c = q[2], d = q[3];
-  x = fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w)));
-  y = fmaxf(fmaxf(fmaxf(c.x, c.y), fmaxf(c.z, c.w)), fmaxf(fmaxf(d.x, d.y), fmaxf(d.z, d.w)));
+  const uint2 v = slots[threadIdx.x & 7];
+  x = __reduce_max_sync(0xffffffffu, v.x);
+  y = __reduce_max_sync(0xffffffffu, v.y);
 }
 
 // BYTES (a power of two) from src to dst, both aligned to min(BYTES, 16): one access up to 16 bytes
@@ -188,6 +187,18 @@ __device__ __forceinline__ void copy_vec(void* dst, const void* src) {
 __device__ __forceinline__ void find_item(const AdamGroup& g, int gb, int& it, int& local) {
   while (it + 1 < g.count && gb >= g.block_end[it]) ++it;
   local = gb - (it > 0 ? g.block_end[it - 1] : 0);
+}
+
+// b -> (b / sub_nc, b % sub_nc) of an item's tile numbering, by multiply-high where the launcher found it exact
+__device__ __forceinline__ void tile_of(const AdamItem& a, int b, int& tile_r, int& tile_c) {
+  const int q = a.sub_magic ? (int)__umulhi((uint32_t)b, a.sub_magic) : b / a.sub_nc;
+  tile_r = a.sub_r0 + q;
+  tile_c = a.sub_c0 + (b - q * a.sub_nc);
+}
+inline uint32_t tile_magic(int64_t tiles, int nc) {
+  // mulhi(b, ceil(2^32 / nc)) = b / nc while b (ceil(2^32 / nc) nc - 2^32) < 2^32; the bracket is below nc
+  if (nc <= 1 || tiles * nc >= ((int64_t)1 << 32)) return 0u;
+  return (uint32_t)((((uint64_t)1 << 32) + (uint64_t)nc - 1) / (uint64_t)nc);
 }
 
 // Where a thread works inside a tile of 4 E rows x 64 columns: E consecutive elements of one row.
@@ -241,7 +252,9 @@ __device__ __forceinline__ void load_r(const AdamItem& a, int64_t off, bool fast
 template <typename TN>
 __device__ __forceinline__ bool adam_f32_tile(const AdamItem& a, int b) {
   constexpr int E = 8;
-  const TileThread<E> tt(a.sub_r0 + b / a.sub_nc, a.sub_c0 + b % a.sub_nc);
+  int tile_r, tile_c;
+  tile_of(a, b, tile_r, tile_c);
+  const TileThread<E> tt(tile_r, tile_c);
   const int valid = tt.row < a.rows ? min(E, a.cols - tt.col) : 0;     // elements of the run inside the matrix
   if (valid <= 0) return false;
   const bool fast = a.vec && valid == E;
@@ -309,7 +322,8 @@ __global__ void __launch_bounds__(256, GALORE_F32_CTAS) adam_f32_kernel(const __
 // is predicated (fewer registers: one more resident CTA per SM).
 template <typename TN, int E, bool FAST>
 __device__ __forceinline__ bool adam_q8_tile(const AdamItem& a, int b, Q8Tables& t, int parity) {
-  const int tile_r = a.sub_r0 + b / a.sub_nc, tile_c = a.sub_c0 + b % a.sub_nc;
+  int tile_r, tile_c;
+  tile_of(a, b, tile_r, tile_c);
   const int tile = tile_r * a.tiles_c + tile_c;
   const TileThread<E> tt(tile_r, tile_c);
   const int valid = FAST ? E : (tt.row < a.rows ? max(0, min(E, a.cols - tt.col)) : 0);
@@ -345,10 +359,13 @@ __device__ __forceinline__ bool adam_q8_tile(const AdamItem& a, int b, Q8Tables&
   }
   if (valid > 0) store_n<TN, E>((TN*)a.Nout + (int64_t)tt.row * a.n_ld + tt.col, n, fast, valid);
   const bool bad = mx_v_bits >= 0x7f800000u;
-  float mx_v = __uint_as_float(mx_v_bits);
-  block_max2_256(mx_m, mx_v, t.red + 16 + 16 * parity);
+  uint32_t mx_m_bits = __float_as_uint(mx_m);
+  block_max2_256(mx_m_bits, mx_v_bits, t.red + 16 + 16 * parity);
+  mx_m = __uint_as_float(mx_m_bits);
+  const float mx_v = __uint_as_float(mx_v_bits);
   // an all-zero block: with 0 in place of the reciprocal every y' is 0 and takes the code of zero
-  const float inv_m = mx_m != 0.f ? 1.0f / mx_m : 0.f, inv_v = mx_v != 0.f ? 1.0f / mx_v : 0.f;
+  // (the correctly rounded reciprocal, as 1 / x would give)
+  const float inv_m = mx_m != 0.f ? __frcp_rn(mx_m) : 0.f, inv_v = mx_v != 0.f ? __frcp_rn(mx_v) : 0.f;
   if constexpr (E % 4 == 0) {
     alignas(16) uint32_t pm[E / 4], pv[E / 4];
 #pragma unroll
@@ -521,6 +538,7 @@ galore_status_t launch_adam_group(const AdamGroup& g, int32_t state_fmt, int q_b
     dst.item[j].sub_r0 = r0;
     dst.item[j].sub_c0 = c0;
     dst.item[j].sub_nc = nc;
+    dst.item[j].sub_magic = tile_magic((int64_t)nr * nc, nc);
     dst.block_end[j] = (j > 0 ? dst.block_end[j - 1] : 0) + nr * nc;
     return GALORE_OK;
   };
@@ -558,6 +576,7 @@ galore_status_t adam_group_add(AdamGroup& g, const AdamItem& item, int32_t state
   a.vec = ((bases & 15) == 0 && pitches) ? 1 : 0;
   a.sub_r0 = a.sub_c0 = 0;
   a.sub_nc = a.tiles_c;
+  a.sub_magic = tile_magic(tiles, a.tiles_c);
   const int i = g.count++;
   g.item[i] = a;
   g.block_end[i] = (int)(before + tiles);

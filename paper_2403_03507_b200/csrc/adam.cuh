@@ -23,6 +23,7 @@ struct AdamItem {
   int tiles_c;             // set by adam_group_add: ceil(cols / 64)
   int vec;                 // set by adam_group_add: bases and pitches allow the vector accesses of an interior tile
   int sub_r0, sub_c0, sub_nc;  // the item covers the tiles (sub_r0 + b / sub_nc, sub_c0 + b % sub_nc), b = 0, 1, ...
+  uint32_t sub_magic;      // ceil(2^32 / sub_nc) when b / sub_nc = mulhi(b, sub_magic) for every b of the item, else 0
   AdamParams p;
   int32_t* status;
 };
