@@ -184,15 +184,18 @@ galore_status_t galore_step_host(galore_layer_t* layer, void* W_host, const void
                                  void* W_dev_staging, void* G_dev_staging, float lr, void* stream);
 
 /* Steps `count` layers on one stream, layer i with W[i], G[i] (device pointers; host arrays of
- * pointers and leading dimensions).  Same results as calling galore_step on each layer, but the
- * layers that run on the tensor-core path are stepped together: one grouped launch for all their
- * projections, one for Adam, one for all their back-projections, so that small matrices do not
- * each pay a kernel's ramp-up and the last wave of one matrix overlaps the first of the next.
- * batch_ws is a caller-allocated, 256-byte aligned device buffer that holds the intermediates
- * (R and N) of the layers of one group; galore_batch_query_bytes gives the size that lets the
- * groups be as large as the kernels allow.  A smaller buffer only makes the groups smaller; a
- * layer that does not fit at all, or is not on the tensor-core path, is stepped by galore_step
- * with its own workspace.  The layers' own workspaces may be shared with each other. */
+ * pointers and leading dimensions).  Same results as calling galore_step on each layer up to the
+ * order of floating-point sums (with several layers in flight the K dimension of the projection is
+ * not sliced), but the layers are stepped in groups of up to 32 of one kind (tensor-core path, or
+ * fp32 path with the same side and dtypes): one grouped launch for all their projections, one for
+ * the inner optimizer (none when Adam runs in the projection's epilogue), one for all their
+ * back-projections, so that small matrices do not each pay a kernel's ramp-up and the last wave of
+ * one matrix overlaps the first of the next.  batch_ws is a caller-allocated, 256-byte aligned
+ * device buffer that holds the intermediates (R and N) of the layers of one group; the groups run
+ * one after another on `stream` and use it in turn.  galore_batch_query_bytes gives the size that
+ * lets the groups be as large as the kernels allow.  A smaller buffer only makes the groups
+ * smaller; a layer that does not fit at all is stepped by galore_step with its own workspace.  The
+ * layers' own workspaces may be shared with each other. */
 galore_status_t galore_batch_query_bytes(galore_layer_t* const* layers, int32_t count, size_t* batch_ws_bytes);
 galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W, const int64_t* ldw,
                                   const void* const* G, const int64_t* ldg, int32_t count, float lr,

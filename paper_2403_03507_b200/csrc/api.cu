@@ -7,6 +7,7 @@
 
 #include <algorithm>
 #include <atomic>
+#include <memory>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -376,6 +377,72 @@ bool same_refresh_shape(const galore_layer* a, const galore_layer* b) {
          a->cfg.refresh_max_iters == b->cfg.refresh_max_iters;
 }
 
+// ---- layers on the fp32 path in a batch: the same three phases, each one grouped launch ----------------
+bool fma_groupable(const galore_layer* l) { return !l->tensor_path && l->has_projector; }
+bool fma_same_kind(const galore_layer* a, const galore_layer* b) {
+  return a->left == b->left && a->cfg.p_dtype == b->cfg.p_dtype && a->cfg.g_dtype == b->cfg.g_dtype &&
+         a->cfg.w_dtype == b->cfg.w_dtype && a->cfg.state_fmt == b->cfg.state_fmt && a->q_block == b->q_block;
+}
+// with eight or more such layers in flight the K dimension needs no slicing to fill the machine
+int fma_splits(const galore_layer* l, int groupable) {
+  return simt_effective_splits((int)l->d, groupable >= 8 ? 1 : l->proj_splits);
+}
+size_t fma_r_bytes(const galore_layer* l, int splits) { return align_up((size_t)splits * l->nel * 4, 256); }
+size_t fma_n_bytes(const galore_layer* l) { return align_up((size_t)l->nel * 4, 256); }
+size_t fma_layer_bytes(const galore_layer* l, int splits) {
+  return fma_r_bytes(l, splits) + fma_n_bytes(l) +
+         (l->cfg.state_fmt == GALORE_STATE_ADAFACTOR ? adafactor_scratch_bytes(l->srows, l->scols) : 0);
+}
+
+struct FmaProblem {       // one member of a group, with its operands of this call
+  galore_layer* l;
+  void* W;
+  int64_t ldw;
+  const void* G;
+  int64_t ldg;
+  float* part;            // R partials (fma_r_bytes), then N (fp32), then the Adafactor scratch
+  int splits;
+};
+
+template <typename TP, typename TG>
+galore_status_t fma_group_project(const std::vector<FmaProblem>& ps, cudaStream_t st) {
+  using Epi = EpiStore<float, float>;
+  std::unique_ptr<SimtGroup<Epi>> g(new SimtGroup<Epi>);
+  g->count = 0;
+  const bool left = ps[0].l->left;
+  for (const FmaProblem& q : ps) {
+    const galore_layer* l = q.l;
+    const int r = l->cfg.rank, m = (int)l->cfg.m, n = (int)l->cfg.n;
+    Epi epi{q.part, l->scols, l->nel, 1.f, 0.f};
+    if (left)    // R (r x n) = P^T G
+      GALORE_TRY(simt_group_add(*g, r, n, m, l->P, 1, r, q.G, q.ldg, 1, q.splits, epi));
+    else         // R (m x r) = G Q
+      GALORE_TRY(simt_group_add(*g, m, r, n, q.G, q.ldg, 1, l->P, r, 1, q.splits, epi));
+  }
+  if (left) return launch_gemm_simt_group<TP, TG, float>(*g, st);
+  return launch_gemm_simt_group<TG, TP, float>(*g, st);
+}
+
+template <typename TP, typename TW>
+galore_status_t fma_group_back(const std::vector<FmaProblem>& ps, float lr, cudaStream_t st) {
+  using Epi = EpiApplyW<TW>;
+  std::unique_ptr<SimtGroup<Epi>> g(new SimtGroup<Epi>);
+  g->count = 0;
+  const bool left = ps[0].l->left;
+  for (const FmaProblem& q : ps) {
+    const galore_layer* l = q.l;
+    const int r = l->cfg.rank, m = (int)l->cfg.m, n = (int)l->cfg.n;
+    const float* N = (const float*)((const char*)q.part + fma_r_bytes(l, q.splits));
+    Epi epi{(TW*)q.W, q.ldw, lr * l->cfg.alpha, decay_keep(l, lr)};
+    if (left)    // W -= scale * P N,  N is r x n
+      GALORE_TRY(simt_group_add(*g, m, n, r, l->P, r, 1, N, n, 1, 1, epi));
+    else         // W -= scale * N Q^T,  N is m x r
+      GALORE_TRY(simt_group_add(*g, m, n, r, N, r, 1, l->P, 1, r, 1, epi));
+  }
+  if (left) return launch_gemm_simt_group<TP, float, float>(*g, st);
+  return launch_gemm_simt_group<float, TP, float>(*g, st);
+}
+
 }  // namespace
 
 extern "C" {
@@ -724,8 +791,8 @@ galore_status_t galore_batch_query_bytes(galore_layer_t* const* layers, int32_t 
     if (!layers[i]) return GALORE_ERR_INVALID_ARG;
     eligible += layers[i]->tensor_path ? 1 : 0;
   }
-  // the largest sum over any run of `capacity` consecutive tensor-path layers, twice: two groups are in
-  // flight at a time (the Adam pass of one overlaps the GEMMs of the next)
+  // the largest sum over any run of `capacity` consecutive tensor-path layers: the groups run one after
+  // another on the caller's stream and use the same region in turn
   const int cap = std::min(tensor_group_capacity(), (int)kAdamGroup);
   std::vector<size_t> need;
   for (int32_t i = 0; i < count; ++i)
@@ -736,7 +803,21 @@ galore_status_t galore_batch_query_bytes(galore_layer_t* const* layers, int32_t 
     if (i >= (size_t)cap) run -= need[i - cap];
     best = std::max(best, run);
   }
-  *bytes = need.size() > (size_t)cap ? 2 * best : best;
+  *bytes = best;
+  // layers on the fp32 path are grouped the same way, after the others: the larger of the two needs
+  int groupable = 0;
+  for (int32_t i = 0; i < count; ++i) groupable += layers[i]->tensor_path ? 0 : 1;
+  std::vector<size_t> fneed;
+  for (int32_t i = 0; i < count; ++i)
+    if (!layers[i]->tensor_path) fneed.push_back(fma_layer_bytes(layers[i], fma_splits(layers[i], groupable)));
+  const int fcap = std::min((int)kSimtGroup, std::min((int)kAdamGroup, (int)kAdafactorGroup));
+  best = run = 0;
+  for (size_t i = 0; i < fneed.size(); ++i) {
+    run += fneed[i];
+    if (i >= (size_t)fcap) run -= fneed[i - fcap];
+    best = std::max(best, run);
+  }
+  *bytes = std::max(*bytes, best);
   return GALORE_OK;
 }
 
@@ -748,7 +829,7 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
   cudaStream_t st = (cudaStream_t)stream;
   galore_status_t worst = GALORE_OK;
   // refreshes that are due come first (each synchronises the stream and uses the layer's own workspace)
-  int eligible = 0;
+  int eligible = 0, groupable = 0;
   for (int32_t i = 0; i < count; ++i) {
     galore_layer* l = layers[i];
     if (!l || !W[i] || !G[i] || ldw[i] < l->cfg.n || ldg[i] < l->cfg.n) return GALORE_ERR_INVALID_ARG;
@@ -759,6 +840,7 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
     }
     if (!l->has_projector) return GALORE_ERR_STATE;
     eligible += batch_eligible(l, W[i], ldw[i], G[i], ldg[i]) ? 1 : 0;
+    groupable += fma_groupable(l) ? 1 : 0;
   }
   static thread_local BatchScratch scratch;
   if (!scratch.proj) scratch.proj = tensor_group_new();
@@ -769,17 +851,35 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
   const int cap = std::min(tensor_group_capacity(), std::min((int)kAdamGroup, (int)kAdafactorGroup));
 
   // ---- 1. partition: layers that cannot be grouped step on their own, the rest form groups ----------
-  // Two groups are in flight at a time, each in its own half of the workspace.
-  const size_t half = (batch_ws_bytes / 2) & ~(size_t)255;
-  std::vector<std::vector<BatchMember>> groups;
+  // The groups run one after another on the caller's stream, each in the whole batch workspace.
+  const size_t room = batch_ws_bytes & ~(size_t)255;
+  std::vector<std::vector<BatchMember>> groups, fgroups;
+  const int fcap = std::min((int)kSimtGroup, std::min((int)kAdamGroup, (int)kAdafactorGroup));
   {
-    size_t used = 0;
+    size_t used = 0, fused_bytes = 0;
     for (int32_t i = 0; i < count; ++i) {
       galore_layer* l = layers[i];
       const bool ok = batch_ws && batch_eligible(l, W[i], ldw[i], G[i], ldg[i]);
       const int splits = batch_splits(l, eligible);
       const size_t need = ok ? batch_layer_bytes(l, splits) : 0;
-      if (!ok || need > half) {
+      if (!ok && batch_ws && fma_groupable(l) && groupable >= 2) {
+        const int fs = fma_splits(l, groupable);
+        const size_t fneed = fma_layer_bytes(l, fs);
+        if (fneed <= room) {
+          bool fresh = fgroups.empty();
+          if (!fresh)
+            fresh = !fma_same_kind(layers[fgroups.back()[0].index], l) || (int)fgroups.back().size() >= fcap ||
+                    fused_bytes + fneed > room;
+          if (fresh) {
+            fgroups.emplace_back();
+            fused_bytes = 0;
+          }
+          fgroups.back().push_back(BatchMember{i, fused_bytes, fs});
+          fused_bytes += fneed;
+          continue;
+        }
+      }
+      if (!ok || need > room) {
         // plain step (its refresh, if due, is already done: auto_refresh off for this call)
         const int32_t saved = l->cfg.auto_refresh;
         l->cfg.auto_refresh = 0;
@@ -795,7 +895,7 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
         const bool same = first->cfg.w_dtype == l->cfg.w_dtype && first->cfg.state_fmt == l->cfg.state_fmt &&
                           first->q_block == l->q_block && first->tc.ctas == l->tc.ctas &&
                           adam_in_projection(first, groups.back()[0].splits) == adam_in_projection(l, splits);
-        fresh = !same || (int)groups.back().size() >= cap || used + need > half;
+        fresh = !same || (int)groups.back().size() >= cap || used + need > room;
       }
       if (fresh) {
         groups.emplace_back();
@@ -805,12 +905,13 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
       used += need;
     }
   }
-  if (groups.empty()) return worst;
+  if (groups.empty() && fgroups.empty()) return worst;
 
   // ---- 2. launch helpers -------------------------------------------------------------------------------
   auto scratch_of = [&](size_t gi, const BatchMember& mb, float** part, void** nbuf) {
     const galore_layer* l = layers[mb.index];
-    char* base = (char*)batch_ws + (gi & 1) * half + mb.offset;
+    (void)gi;
+    char* base = (char*)batch_ws + mb.offset;
     *part = (float*)base;
     *nbuf = base + batch_r_bytes(l, mb.splits);
   };
@@ -887,6 +988,50 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
       GALORE_TRY(launch_adam(gi, st));
     }
     GALORE_TRY(launch_back(gi, st));
+  }
+
+  // ---- 4. the groups of fp32-path layers -----------------------------------------------------------------
+  for (size_t gi = 0; gi < fgroups.size(); ++gi) {
+    std::vector<FmaProblem> ps;
+    for (const BatchMember& mb : fgroups[gi]) {
+      galore_layer* l = layers[mb.index];
+      ps.push_back(FmaProblem{l, W[mb.index], ldw[mb.index], G[mb.index], ldg[mb.index],
+                              (float*)((char*)batch_ws + mb.offset), mb.splits});
+    }
+    const galore_layer* first = ps[0].l;
+    const bool pb = first->cfg.p_dtype == GALORE_BF16, gb = first->cfg.g_dtype == GALORE_BF16, wb = first->cfg.w_dtype == GALORE_BF16;
+    {
+      PhaseTimer pt(0, st);
+      if (pb && gb) GALORE_TRY((fma_group_project<__nv_bfloat16, __nv_bfloat16>(ps, st)));
+      else if (pb) GALORE_TRY((fma_group_project<__nv_bfloat16, float>(ps, st)));
+      else if (gb) GALORE_TRY((fma_group_project<float, __nv_bfloat16>(ps, st)));
+      else GALORE_TRY((fma_group_project<float, float>(ps, st)));
+    }
+    {
+      scratch.adam->count = 0;
+      scratch.adafactor->count = 0;
+      const bool adafactor = first->cfg.state_fmt == GALORE_STATE_ADAFACTOR;
+      for (const FmaProblem& q : ps) {
+        galore_layer* l = q.l;
+        char* nbuf = (char*)q.part + fma_r_bytes(l, q.splits);
+        const AdamItem a = adam_item(l, q.part, q.splits, l->nel, l->scols, nbuf, l->scols, adam_params(l));
+        if (adafactor)
+          GALORE_TRY(adafactor_group_add(*scratch.adafactor, adafactor_item(l, a, (float*)(nbuf + fma_n_bytes(l)))));
+        else
+          GALORE_TRY(adam_group_add(*scratch.adam, a, l->cfg.state_fmt, l->q_block));
+      }
+      PhaseTimer pt(1, st);
+      if (adafactor) GALORE_TRY(launch_adafactor_group(*scratch.adafactor, GALORE_F32, st));
+      else GALORE_TRY(launch_adam_group(*scratch.adam, first->cfg.state_fmt, first->q_block, GALORE_F32, st));
+    }
+    {
+      PhaseTimer pt(2, st);
+      if (pb && wb) GALORE_TRY((fma_group_back<__nv_bfloat16, __nv_bfloat16>(ps, lr, st)));
+      else if (pb) GALORE_TRY((fma_group_back<__nv_bfloat16, float>(ps, lr, st)));
+      else if (wb) GALORE_TRY((fma_group_back<float, __nv_bfloat16>(ps, lr, st)));
+      else GALORE_TRY((fma_group_back<float, float>(ps, lr, st)));
+    }
+    for (const FmaProblem& q : ps) q.l->k += 1;
   }
   return worst;
 }

@@ -17,11 +17,11 @@
 
 namespace galore {
 
+// One BM x BN tile of C over the K range [k_begin, k_end): the main loop shared by the kernels below.
 template <typename TA, typename TB, typename TAcc, int BM, int BN, int BK, int TM, int TN, class Epi>
-__global__ void __launch_bounds__((BM / TM) * (BN / TN))
-gemm_simt_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int64_t sAk,
-                 const TB* __restrict__ B, int64_t sBk, int64_t sBj, int kchunk, Epi epi_in, int batched,
-                 int64_t batchA, int64_t batchB, const SlotList slots) {
+__device__ __forceinline__ void gemm_simt_tile(int M, int N, const TA* __restrict__ A, int64_t sAi, int64_t sAk,
+                                               const TB* __restrict__ B, int64_t sBk, int64_t sBj, int m0, int n0, int k_begin,
+                                               int k_end, int zi, const Epi& epi) {
   constexpr int NT = (BM / TM) * (BN / TN);
   constexpr int LA = BM * BK / NT;   // elements of the A tile each thread fetches
   constexpr int LB = BN * BK / NT;
@@ -32,22 +32,6 @@ gemm_simt_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int
 
   const int tid = threadIdx.x;
   const int tx = tid % (BN / TN), ty = tid / (BN / TN);
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
-  const int inner = gridDim.z / slots.n;
-  const int zi = blockIdx.z % inner;
-  const int64_t shift = (int64_t)slots.id[blockIdx.z / inner] * slots.bytes;
-  Epi epi = epi_in;
-  if (shift) {
-    A = slot_ptr(A, shift);
-    B = slot_ptr(B, shift);
-    epi.shift(shift);
-  }
-  const int k_begin = batched ? 0 : zi * kchunk;
-  const int k_end = batched ? K : min(K, k_begin + kchunk);
-  if (batched) {
-    A += (int64_t)zi * batchA;
-    B += (int64_t)zi * batchB;
-  }
   const bool a_kfast = (sAk == 1);   // consecutive threads walk the contiguous direction
   const bool b_kfast = (sBk == 1);
 
@@ -122,6 +106,97 @@ gemm_simt_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int
       if (j < N) epi(i, j, acc[u][v], zi);
     }
   }
+}
+
+template <typename TA, typename TB, typename TAcc, int BM, int BN, int BK, int TM, int TN, class Epi>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN))
+gemm_simt_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int64_t sAk,
+                 const TB* __restrict__ B, int64_t sBk, int64_t sBj, int kchunk, Epi epi_in, int batched,
+                 int64_t batchA, int64_t batchB, const SlotList slots) {
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int inner = gridDim.z / slots.n;
+  const int zi = blockIdx.z % inner;
+  const int64_t shift = (int64_t)slots.id[blockIdx.z / inner] * slots.bytes;
+  Epi epi = epi_in;
+  if (shift) {
+    A = slot_ptr(A, shift);
+    B = slot_ptr(B, shift);
+    epi.shift(shift);
+  }
+  const int k_begin = batched ? 0 : zi * kchunk;
+  const int k_end = batched ? K : min(K, k_begin + kchunk);
+  if (batched) {
+    A += (int64_t)zi * batchA;
+    B += (int64_t)zi * batchB;
+  }
+  gemm_simt_tile<TA, TB, TAcc, BM, BN, BK, TM, TN, Epi>(M, N, A, sAi, sAk, B, sBk, sBj, m0, n0, k_begin, k_end, zi, epi);
+}
+
+// ---- several problems of one operand-type combination in one launch ------------------------------
+// (the projections of a layer set on the fp32 path: one launch instead of one per layer)
+constexpr int kSimtGroup = 32;
+template <class Epi>
+struct SimtProblem {
+  int M, N, K;
+  const void* A;
+  int64_t sAi, sAk;
+  const void* B;
+  int64_t sBk, sBj;
+  int kchunk, splits;      // K slices of kchunk elements; slice z is handed to epi as its last argument
+  Epi epi;
+};
+template <class Epi>
+struct SimtGroup {
+  SimtProblem<Epi> p[kSimtGroup];
+  int cta_end[kSimtGroup];   // running totals of CTAs (tiles x K slices)
+  int count;
+};
+
+template <typename TA, typename TB, typename TAcc, int BM, int BN, int BK, int TM, int TN, class Epi>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN))
+gemm_simt_group_kernel(const __grid_constant__ SimtGroup<Epi> g) {
+  int it = 0;
+  while (it + 1 < g.count && (int)blockIdx.x >= g.cta_end[it]) ++it;
+  const SimtProblem<Epi>& p = g.p[it];
+  int local = (int)blockIdx.x - (it ? g.cta_end[it - 1] : 0);
+  const int tiles_n = (p.N + BN - 1) / BN, tiles_m = (p.M + BM - 1) / BM;
+  const int tn = local % tiles_n;
+  local /= tiles_n;
+  const int tm = local % tiles_m, zi = local / tiles_m;
+  const int k_begin = zi * p.kchunk, k_end = min(p.K, k_begin + p.kchunk);
+  gemm_simt_tile<TA, TB, TAcc, BM, BN, BK, TM, TN, Epi>(p.M, p.N, (const TA*)p.A, p.sAi, p.sAk, (const TB*)p.B, p.sBk, p.sBj,
+                                                        tm * BM, tn * BN, k_begin, k_end, zi, p.epi);
+}
+
+// adds one problem (128 x 128 tiles); `splits` as for launch_gemm_simt
+template <class Epi>
+galore_status_t simt_group_add(SimtGroup<Epi>& g, int M, int N, int K, const void* A, int64_t sAi, int64_t sAk, const void* B,
+                               int64_t sBk, int64_t sBj, int splits, const Epi& epi) {
+  if (g.count >= kSimtGroup) return GALORE_ERR_BUFFER_TOO_SMALL;
+  if (M <= 0 || N <= 0) return GALORE_ERR_SHAPE;
+  if (splits < 1) splits = 1;
+  int kchunk = (int)ceil_div(ceil_div(K, splits), 16) * 16;
+  if (kchunk < 16) kchunk = 16;
+  splits = (int)ceil_div(K > 0 ? K : 1, kchunk);
+  SimtProblem<Epi>& p = g.p[g.count];
+  p.M = M; p.N = N; p.K = K;
+  p.A = A; p.sAi = sAi; p.sAk = sAk;
+  p.B = B; p.sBk = sBk; p.sBj = sBj;
+  p.kchunk = kchunk; p.splits = splits;
+  p.epi = epi;
+  const int64_t ctas = ceil_div(M, 128) * ceil_div(N, 128) * splits;
+  const int64_t before = g.count ? g.cta_end[g.count - 1] : 0;
+  if (before + ctas >= ((int64_t)1 << 31)) return GALORE_ERR_SHAPE;
+  g.cta_end[g.count] = (int)(before + ctas);
+  g.count += 1;
+  return GALORE_OK;
+}
+template <typename TA, typename TB, typename TAcc, class Epi>
+galore_status_t launch_gemm_simt_group(const SimtGroup<Epi>& g, cudaStream_t stream) {
+  if (g.count <= 0) return GALORE_OK;
+  gemm_simt_group_kernel<TA, TB, TAcc, 128, 128, 16, 8, 8, Epi><<<(unsigned)g.cta_end[g.count - 1], 256, 0, stream>>>(g);
+  GALORE_LAUNCH_CHECK();
+  return GALORE_OK;
 }
 
 // ---- epilogues ----------------------------------------------------------------

@@ -113,3 +113,36 @@ def test_export_import_resumes_bit_identically():
     assert a.step_count == b.step_count == 6 and torch.equal(Wa, Wb)
     for x, y in zip(a.get_adafactor_state(), b.get_adafactor_state()):
         assert torch.equal(x, y)
+
+
+@pytest.mark.parametrize("state_fmt", ["adafactor", "f32"])
+def test_fp32_path_layers_in_a_batch_match_the_oracle(state_fmt):
+    """Nine fp32 layers (not on the tensor path) in one batched call: grouped launches of the FMA kernels for
+    the two projections, one grouped launch for the inner optimizer; K is not sliced with this many in flight."""
+    shapes = [(192, 640, 48), (192, 640, 48), (256, 333, 32), (130, 301, 17), (192, 640, 48), (256, 512, 64),
+              (200, 304, 16), (384, 1000, 128), (256, 333, 32)]
+    inner = "adafactor" if state_fmt == "adafactor" else "adam"
+    layers, orcs, Wg, Wo = [], [], [], []
+    for i, (m, n, r) in enumerate(shapes):
+        layer = gb.Layer(gb.make_config(m, n, r, w_dtype="f32", g_dtype="f32", state_fmt=state_fmt, auto_refresh=False))
+        P = wl.random_orthonormal(m, r, np.random.default_rng(i)).astype(np.float32)
+        layer.set_projector(torch.from_numpy(P))
+        o = go.GaLoreOracle(m, n, r, 0.25, 1000, w_store="f32", state="f32", inner=inner)
+        o.set_projector(P.astype(np.float64))
+        W0 = wl.make_weight(m, n, 50 + i, "f32")
+        layers.append(layer); orcs.append(o); Wg.append(to_dev(W0, "f32")); Wo.append(W0)
+    before = gb.galore_launch_count()
+    for s in range(3):
+        Gh = [wl.make_gradient(m, n, wl.sub_seed(21, i, s), 1.0, 0.05, "f32") for i, (m, n, r) in enumerate(shapes)]
+        Gd = [to_dev(g, "f32") for g in Gh]
+        gb.Batch(layers, Wg, Gd).galore_step_batch(1e-2)
+        Wo = [o.step(w, g, 1e-2, auto_refresh=False) for o, w, g in zip(orcs, Wo, Gh)]
+    torch.cuda.synchronize()
+    launches = gb.galore_launch_count() - before
+    assert launches <= 3 * (3 + (5 if state_fmt == "adafactor" else 2))          # one group per phase and step
+    for i, (wg, wo) in enumerate(zip(Wg, Wo)):
+        assert rel_err(to_host(wg), wo) < 1e-5, i
+    assert all(l.step_count == 3 and l.device_status() == 0 for l in layers)
+    if state_fmt == "adafactor":
+        for l, o in zip(layers, orcs):
+            _state_close(l, o, 1e-4)

@@ -100,15 +100,20 @@ def test_small_workspace_only_makes_groups_smaller_and_mixed_paths_work():
     gb.Batch(lb, Wb, G, workspace_bytes=full // 5).galore_step_batch(1e-2)      # several groups, maybe single steps
     for w1, w2 in zip(Wa, Wb):
         assert rel_err(to_host(w2), to_host(w1)) < 5e-4
-    # fp32 layers (not on the tensor path) inside a batch take the plain path
+    # fp32 layers (not on the tensor path) inside a batch run the same three phases as grouped launches of the
+    # FMA kernels; with many layers in flight K is not sliced, so sums differ from single steps in their order only
     lc, Wc, _, _ = _make("f32", "f32", path=gb.PATH_FP32, g_dtype="f32")
     ld_, Wd, _, _ = _make("f32", "f32", path=gb.PATH_FP32, g_dtype="f32")
     _, G32 = _grads(0, "f32")
+    before = gb.galore_launch_count()
     gb.Batch(lc, Wc, G32).galore_step_batch(1e-2)
+    grouped = gb.galore_launch_count() - before
     for l, w, g in zip(ld_, Wd, G32):
         l.galore_step(w, g, 1e-2)
+    assert grouped < gb.galore_launch_count() - before - grouped          # fewer launches than one step per layer
     for w1, w2 in zip(Wc, Wd):
-        assert torch.equal(w1, w2)
+        assert rel_err(to_host(w1), to_host(w2)) < 2e-5      # first step: N is close to sign(R), and R near zero may change sign with the order of the sum
+    assert all(l.step_count == 1 for l in lc)
 
 
 def test_auto_refresh_inside_a_batch():
