@@ -67,7 +67,12 @@ __global__ void __launch_bounds__(128) jb_gram_kernel(const double* __restrict__
   if (bp.I * kBlockRows >= b) return;                 // both blocks are padding
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int wy = warp >> 1, wx = warp & 1;
+  // The Gram matrix is symmetric and the sweep reads its upper triangle only: of the 8 x 8 grid of 8 x 8
+  // tiles the 36 with tile row <= tile column are formed.  Warps 0 and 3 take the upper halves of the two
+  // diagonal 32 x 32 quadrants (10 tiles each), warps 1 and 2 the two column halves of the off-diagonal one.
+  const int rb = warp == 3 ? 1 : 0, cb = warp == 0 ? 0 : 1;
+  constexpr uint32_t kUpper = 0x8cefu;                           // bit 4 i + j set for i <= j
+  const uint32_t mask = (warp == 0 || warp == 3) ? kUpper : (warp == 1 ? 0x3333u : 0xccccu);
   const int c_begin = chunk * kGramChunk;
   const int c_end = min(b, c_begin + kGramChunk);
   const int tiles = (c_end - c_begin + 31) / 32;
@@ -118,13 +123,14 @@ __global__ void __launch_bounds__(128) jb_gram_kernel(const double* __restrict__
     for (int ks = 0; ks < 8; ++ks) {
       double a[4], bb[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) a[i] = Xs[buf][wy * 32 + i * 8 + g][ks * 4 + t];
+      for (int i = 0; i < 4; ++i) a[i] = Xs[buf][rb * 32 + i * 8 + g][ks * 4 + t];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) bb[j] = Xs[buf][wx * 32 + j * 8 + g][ks * 4 + t];
+      for (int j = 0; j < 4; ++j) bb[j] = Xs[buf][cb * 32 + j * 8 + g][ks * 4 + t];
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) dmma(acc[i][j], a[i], bb[j]);
+        for (int j = 0; j < 4; ++j)
+          if ((mask >> (i * 4 + j)) & 1u) dmma(acc[i][j], a[i], bb[j]);
     }
     if (tile + 1 < tiles) stash(buf ^ 1);
     __syncthreads();
@@ -135,7 +141,8 @@ __global__ void __launch_bounds__(128) jb_gram_kernel(const double* __restrict__
   for (int i = 0; i < 4; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const int r = wy * 32 + i * 8 + g, c = wx * 32 + j * 8 + 2 * t;
+      if (!((mask >> (i * 4 + j)) & 1u)) continue;
+      const int r = rb * 32 + i * 8 + g, c = cb * 32 + j * 8 + 2 * t;
       *reinterpret_cast<double2*>(out + r * kPairRows + c) = make_double2(acc[i][j][0], acc[i][j][1]);
     }
 }
@@ -242,7 +249,11 @@ __global__ void __launch_bounds__(kSweepThreads, 2) jb_sweep_kernel(const double
       for (int j = 0; j < 4; ++j) {
         const double* sc = src + (int64_t)(c + j) * (kPairRows * kPairRows);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[j][i] = (c + j < chunks) ? sc[tid + kSweepThreads * i] : 0.0;
+        for (int i = 0; i < 8; ++i) {
+          const int idx = tid + kSweepThreads * i;
+          const bool upper = ((idx >> 9) <= ((idx >> 3) & 7));       // tile row <= tile column: the rest is not written
+          v[j][i] = (c + j < chunks && upper) ? sc[idx] : 0.0;
+        }
       }
 #pragma unroll
       for (int j = 0; j < 4; ++j)
