@@ -142,7 +142,8 @@ galore_status_t launch_gemm_dmma(int M, int N, int K, const TA* A, int64_t sAi, 
                                                                            batchB, epi, slots);
   } else {
     dim3 grid((unsigned)ceil_div(N, 128), (unsigned)ceil_div(M, 128), (unsigned)batch);
-    gemm_dmma_kernel<TA, TB, 128, 128, 32, 64, Epi><<<grid, 256, 0, stream>>>(M, N, K, A, sAi, sAk, batchA, B, sBk, sBj,
+    // sixteen warps of 32 x 32 (four per scheduler hide the latency of the fragment loads better than eight of 32 x 64)
+    gemm_dmma_kernel<TA, TB, 128, 128, 32, 32, Epi><<<grid, 512, 0, stream>>>(M, N, K, A, sAi, sAk, batchA, B, sBk, sBj,
                                                                              batchB, epi, slots);
   }
   GALORE_LAUNCH_CHECK();
