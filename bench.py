@@ -62,6 +62,10 @@ def algorithmic_cost(w, m, n):
     return by, 4 * m * n * r
 
 
+NOMINAL_HBM_GBS = 8000.0          # data-sheet HBM3e bandwidth
+NOMINAL_BF16_TFLOPS = 2250.0       # data-sheet dense bf16 tensor rate
+
+
 def state_bytes_per_step(w, nel, r, big):
     """Optimizer statistics read and written once per step: two fp32 moments, two 8-bit moments with their
     absmax values, or Adafactor's fp32 first moment with one value per row and per column of R."""
@@ -575,6 +579,10 @@ def time_workload(w, args, dev, dist, world, rank, full, mode=None):
             "scope": "whole step: algorithmic bytes and flops of every matrix / measured step time",
             "kernels": {k: v for k, v in kernels.items() if v},
             "step_roofline_ms": {"hbm": t_hbm * 1e3, "tensor" if uses_tc else "fp32_fma": t_tc * 1e3},
+            # the same fraction against the data-sheet figures (8 TB/s, 2250 dense bf16 TFLOP/s): context only
+            "nominal": ({"hbm_gbs": NOMINAL_HBM_GBS, "bf16_tflops": NOMINAL_BF16_TFLOPS,
+                         "frac": max(bytes_alg / (NOMINAL_HBM_GBS * 1e9), flops_alg / (NOMINAL_BF16_TFLOPS * 1e12)) * 1e3 / ms_step}
+                        if uses_tc else None),
             "algorithmic": {"bytes_per_step": bytes_alg, "flops_per_step": flops_alg}}
 
     out = {
