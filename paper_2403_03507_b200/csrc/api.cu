@@ -856,7 +856,8 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
   std::vector<std::vector<BatchMember>> groups, fgroups;
   const int fcap = std::min((int)kSimtGroup, std::min((int)kAdamGroup, (int)kAdafactorGroup));
   {
-    size_t used = 0, fused_bytes = 0;
+    size_t used = 0;
+    std::vector<size_t> fused_bytes_of;
     for (int32_t i = 0; i < count; ++i) {
       galore_layer* l = layers[i];
       const bool ok = batch_ws && batch_eligible(l, W[i], ldw[i], G[i], ldg[i]);
@@ -866,16 +867,19 @@ galore_status_t galore_step_batch(galore_layer_t* const* layers, void* const* W,
         const int fs = fma_splits(l, groupable);
         const size_t fneed = fma_layer_bytes(l, fs);
         if (fneed <= room) {
-          bool fresh = fgroups.empty();
-          if (!fresh)
-            fresh = !fma_same_kind(layers[fgroups.back()[0].index], l) || (int)fgroups.back().size() >= fcap ||
-                    fused_bytes + fneed > room;
-          if (fresh) {
+          // any open group of the same kind takes it (the layers are independent: their order in the list does
+          // not matter, so a list in model order, sides alternating, still gives full groups)
+          int at = -1;
+          for (int gi = (int)fgroups.size() - 1; gi >= 0 && at < 0; --gi)
+            if (fma_same_kind(layers[fgroups[gi][0].index], l) && (int)fgroups[gi].size() < fcap && fused_bytes_of[gi] + fneed <= room)
+              at = gi;
+          if (at < 0) {
             fgroups.emplace_back();
-            fused_bytes = 0;
+            fused_bytes_of.push_back(0);
+            at = (int)fgroups.size() - 1;
           }
-          fgroups.back().push_back(BatchMember{i, fused_bytes, fs});
-          fused_bytes += fneed;
+          fgroups[at].push_back(BatchMember{i, fused_bytes_of[at], fs});
+          fused_bytes_of[at] += fneed;
           continue;
         }
       }

@@ -119,13 +119,13 @@ def test_export_import_resumes_bit_identically():
 def test_fp32_path_layers_in_a_batch_match_the_oracle(state_fmt):
     """Nine fp32 layers (not on the tensor path) in one batched call: grouped launches of the FMA kernels for
     the two projections, one grouped launch for the inner optimizer; K is not sliced with this many in flight."""
-    shapes = [(192, 640, 48), (192, 640, 48), (256, 333, 32), (130, 301, 17), (192, 640, 48), (256, 512, 64),
-              (200, 304, 16), (384, 1000, 128), (256, 333, 32)]
+    shapes = [(192, 640, 48), (640, 192, 48), (256, 333, 32), (130, 301, 17), (192, 640, 48), (512, 256, 64),
+              (200, 304, 16), (384, 1000, 128), (333, 256, 32)]          # both sides, in no particular order
     inner = "adafactor" if state_fmt == "adafactor" else "adam"
     layers, orcs, Wg, Wo = [], [], [], []
     for i, (m, n, r) in enumerate(shapes):
         layer = gb.Layer(gb.make_config(m, n, r, w_dtype="f32", g_dtype="f32", state_fmt=state_fmt, auto_refresh=False))
-        P = wl.random_orthonormal(m, r, np.random.default_rng(i)).astype(np.float32)
+        P = wl.random_orthonormal(min(m, n), r, np.random.default_rng(i)).astype(np.float32)
         layer.set_projector(torch.from_numpy(P))
         o = go.GaLoreOracle(m, n, r, 0.25, 1000, w_store="f32", state="f32", inner=inner)
         o.set_projector(P.astype(np.float64))
@@ -139,7 +139,7 @@ def test_fp32_path_layers_in_a_batch_match_the_oracle(state_fmt):
         Wo = [o.step(w, g, 1e-2, auto_refresh=False) for o, w, g in zip(orcs, Wo, Gh)]
     torch.cuda.synchronize()
     launches = gb.galore_launch_count() - before
-    assert launches <= 3 * (3 + (5 if state_fmt == "adafactor" else 2))          # one group per phase and step
+    assert launches <= 2 * 3 * (3 + (5 if state_fmt == "adafactor" else 2))      # one group per side, phase and step
     for i, (wg, wo) in enumerate(zip(Wg, Wo)):
         assert rel_err(to_host(wg), wo) < 1e-5, i
     assert all(l.step_count == 3 and l.device_status() == 0 for l in layers)
