@@ -110,9 +110,12 @@ typedef struct {
   /* refresh: block subspace iteration on a block of rank + refresh_oversample
    * columns (clipped to min(m, n); 0 = default: max(256, rank / 2) on the
    * tensor path, rank more columns elsewhere; negative = none),
-   * stopped when the predicted subspace error (theta_b / theta_r)^iterations
-   * falls below refresh_tol or after refresh_max_iters power iterations.
-   * 0 = defaults (1e-4, 96). */
+   * stopped when the predicted subspace error falls below refresh_tol or
+   * after refresh_max_iters power iterations.  The prediction is
+   * (theta_b / theta_r)^iterations for plain power steps; blocks that converge
+   * slowly finish with pairs of steps that apply the degree-2 Chebyshev
+   * polynomial of the operator over [0, theta_b], each pair counted with the
+   * polynomial's value at theta_r.  0 = defaults (1e-4, 96). */
   float refresh_tol;
   int32_t refresh_max_iters;
   int32_t refresh_oversample;
@@ -130,7 +133,8 @@ typedef struct {
    * columns for the oversampling) and run this many power steps before its Rayleigh-Ritz pass.  The
    * result is then judged by its own residual: residual over spectral gap bounds the angle to the
    * exact subspace; within 10 x refresh_tol the refresh ends there, otherwise it continues like a
-   * cold one.  0 = always start from a random block. */
+   * cold one (as it does at once when the Rayleigh quotients after those steps show no gap behind
+   * the block).  0 = always start from a random block. */
   int32_t refresh_warm_iters;
   int32_t reserved[5];
 } galore_config_t;
