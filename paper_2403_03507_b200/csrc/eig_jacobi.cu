@@ -24,7 +24,8 @@ constexpr int kGramChunk = 256;   // columns summed by one CTA of the Gram kerne
 constexpr int kApplyCols = 128;   // columns transformed by one CTA of the apply kernel
 constexpr int kGramLd = 36;       // shared-memory row strides, all = 4 mod 16 doubles: the 8 x 4 operand
 constexpr int kRotLd = 68;        // fragments of the fp64 MMA then fall on distinct banks
-constexpr int kTileLd = 132;
+constexpr int kApplyHalf = 64;    // columns in shared memory at a time
+constexpr int kHalfLd = 68;
 
 // D (8 x 8) += A (8 x 4, row) B (4 x 8, col), fp64.  Lane l holds A[l / 4][l % 4], B[l % 4][l / 4]
 // and D[l / 4][2 (l % 4) + {0, 1}].
@@ -349,12 +350,15 @@ __global__ void __launch_bounds__(kSweepThreads, 2) jb_sweep_kernel(const double
 }
 
 // rows(pair)[:, cols] <- Rot rows(pair)[:, cols]  for X (blockIdx.z = 0) and, if present, Vt (blockIdx.z = 1)
+// A CTA owns 128 columns and takes them in two halves of 64: while the first half is multiplied the second
+// is already on its way from global memory into registers, and with one half in shared memory three CTAs
+// fit on an SM.  Warp (wy, wx) forms rows 32 wy .. + 32, columns 16 wx .. + 16 of a half.
 __global__ void __launch_bounds__(256) jb_apply_kernel(double* __restrict__ X, double* __restrict__ Vt, int b, int nblk, int round,
                                                        const double* __restrict__ rot, const int* __restrict__ flags,
                                                        const SlotList slots, int matrices) {
   extern __shared__ __align__(16) double jb_smem[];
   double(*Rs)[kRotLd] = reinterpret_cast<double(*)[kRotLd]>(jb_smem);
-  double(*Xs)[kTileLd] = reinterpret_cast<double(*)[kTileLd]>(jb_smem + kPairRows * kRotLd);
+  double(*Xs)[kHalfLd] = reinterpret_cast<double(*)[kHalfLd]>(jb_smem + kPairRows * kRotLd);
   const int pair = blockIdx.x;
   const int which = blockIdx.z % matrices;                                  // 0: X, 1: Vt
   {
@@ -379,56 +383,76 @@ __global__ void __launch_bounds__(256) jb_apply_kernel(double* __restrict__ X, d
     const int l = id >> 5, m2 = (id & 31) * 2;
     *reinterpret_cast<double2*>(&Rs[l][m2]) = *reinterpret_cast<const double2*>(rsrc + l * kPairRows + m2);
   }
+  double2 stage[8];
+  auto fetch = [&](int half) {             // 64 rows x 64 columns: row id / 32, columns 2 (id % 32) of the half
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const int id = tid + 256 * i;
-    const int l = id >> 6, cl = (id & 63) * 2;
-    const int row = bp.row(l), col = c0 + cl;
-    double2 v = make_double2(0.0, 0.0);
-    if (row < b) {
-      const double* src = M + (int64_t)row * b + col;
-      if (vec && col + 1 < b) {
-        v = *reinterpret_cast<const double2*>(src);
-      } else {
-        if (col < b) v.x = src[0];
-        if (col + 1 < b) v.y = src[1];
+    for (int i = 0; i < 8; ++i) {
+      const int id = tid + 256 * i;
+      const int l = id >> 5, cl = (id & 31) * 2;
+      const int row = bp.row(l), col = c0 + half * kApplyHalf + cl;
+      double2 v = make_double2(0.0, 0.0);
+      if (row < b) {
+        const double* src = M + (int64_t)row * b + col;
+        if (vec && col + 1 < b) {
+          v = *reinterpret_cast<const double2*>(src);
+        } else {
+          if (col < b) v.x = src[0];
+          if (col + 1 < b) v.y = src[1];
+        }
       }
+      stage[i] = v;
     }
-    *reinterpret_cast<double2*>(&Xs[l][cl]) = v;
-  }
+  };
+  auto stash = [&]() {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int id = tid + 256 * i;
+      *reinterpret_cast<double2*>(&Xs[id >> 5][(id & 31) * 2]) = stage[i];
+    }
+  };
+  fetch(0);
+  stash();
   __syncthreads();
-  double acc[4][4][2];
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-#pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
-#pragma unroll 4
-  for (int ks = 0; ks < kPairRows / 4; ++ks) {
-    double a[4], bb[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) a[i] = Rs[wy * 32 + i * 8 + g][ks * 4 + t];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) bb[j] = Xs[ks * 4 + t][wx * 32 + j * 8 + g];
+  const bool second = c0 + kApplyHalf < b;        // the second half holds columns of the matrix
+  for (int half = 0; half < 2; ++half) {
+    if (half == 0 && second) fetch(1);
+    double acc[4][2][2];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
-      for (int j = 0; j < 4; ++j) dmma(acc[i][j], a[i], bb[j]);
-  }
+      for (int j = 0; j < 2; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
+#pragma unroll 4
+    for (int ks = 0; ks < kPairRows / 4; ++ks) {
+      double a[4], bb[2];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int row = bp.row(wy * 32 + i * 8 + g);
-    if (row >= b) continue;
+      for (int i = 0; i < 4; ++i) a[i] = Rs[wy * 32 + i * 8 + g][ks * 4 + t];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int col = c0 + wx * 32 + j * 8 + 2 * t;
-      double* dst = M + (int64_t)row * b + col;
-      if (vec && col + 1 < b) {
-        *reinterpret_cast<double2*>(dst) = make_double2(acc[i][j][0], acc[i][j][1]);
-      } else {
-        if (col < b) dst[0] = acc[i][j][0];
-        if (col + 1 < b) dst[1] = acc[i][j][1];
+      for (int j = 0; j < 2; ++j) bb[j] = Xs[ks * 4 + t][wx * 16 + j * 8 + g];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) dmma(acc[i][j], a[i], bb[j]);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int row = bp.row(wy * 32 + i * 8 + g);
+      if (row >= b) continue;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int col = c0 + half * kApplyHalf + wx * 16 + j * 8 + 2 * t;
+        double* dst = M + (int64_t)row * b + col;
+        if (vec && col + 1 < b) {
+          *reinterpret_cast<double2*>(dst) = make_double2(acc[i][j][0], acc[i][j][1]);
+        } else {
+          if (col < b) dst[0] = acc[i][j][0];
+          if (col + 1 < b) dst[1] = acc[i][j][1];
+        }
       }
     }
+    if (half == 1 || !second) break;
+    __syncthreads();                               // every warp has read the first half
+    stash();
+    __syncthreads();
   }
 }
 
@@ -445,7 +469,7 @@ JacobiGeometry jacobi_geometry(int b) {
   return g;
 }
 
-constexpr size_t kApplySmem = (size_t)(kPairRows * kRotLd + kPairRows * kTileLd) * sizeof(double);
+constexpr size_t kApplySmem = (size_t)(kPairRows * kRotLd + kPairRows * kHalfLd) * sizeof(double);
 
 }  // namespace
 
