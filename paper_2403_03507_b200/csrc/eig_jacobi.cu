@@ -71,9 +71,9 @@ __global__ void __launch_bounds__(128) jb_gram_kernel(const double* __restrict__
   // The Gram matrix is symmetric and the sweep reads its upper triangle only: of the 8 x 8 grid of 8 x 8
   // tiles the 36 with tile row <= tile column are formed.  Warps 0 and 3 take the upper halves of the two
   // diagonal 32 x 32 quadrants (10 tiles each), warps 1 and 2 the two column halves of the off-diagonal one.
-  const int rb = warp == 3 ? 1 : 0, cb = warp == 0 ? 0 : 1;
-  constexpr uint32_t kUpper = 0x8cefu;                           // bit 4 i + j set for i <= j
-  const uint32_t mask = (warp == 0 || warp == 3) ? kUpper : (warp == 1 ? 0x3333u : 0xccccu);
+  const bool diagonal = warp == 0 || warp == 3;
+  const int rb = warp == 3 ? 1 : 0, cb = rb;                     // the diagonal quadrant of warps 0 and 3
+  const int jbase = warp == 2 ? 2 : 0;                           // first tile column of warps 1 and 2
   const int c_begin = chunk * kGramChunk;
   const int c_end = min(b, c_begin + kGramChunk);
   const int tiles = (c_end - c_begin + 31) / 32;
@@ -121,31 +121,55 @@ __global__ void __launch_bounds__(128) jb_gram_kernel(const double* __restrict__
     const int buf = tile & 1;
     if (tile + 1 < tiles) fetch(tile + 1);
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-      double a[4], bb[4];
+    if (diagonal) {            // upper half of a diagonal quadrant: tiles (i, j) with i <= j
 #pragma unroll
-      for (int i = 0; i < 4; ++i) a[i] = Xs[buf][rb * 32 + i * 8 + g][ks * 4 + t];
+      for (int ks = 0; ks < 8; ++ks) {
+        double a[4], bb[4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) bb[j] = Xs[buf][cb * 32 + j * 8 + g][ks * 4 + t];
+        for (int i = 0; i < 4; ++i) a[i] = Xs[buf][rb * 32 + i * 8 + g][ks * 4 + t];
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+        for (int j = 0; j < 4; ++j) bb[j] = Xs[buf][cb * 32 + j * 8 + g][ks * 4 + t];
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-          if ((mask >> (i * 4 + j)) & 1u) dmma(acc[i][j], a[i], bb[j]);
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = i; j < 4; ++j) dmma(acc[i][j], a[i], bb[j]);
+      }
+    } else {                   // two of the four tile columns of the off-diagonal quadrant (kept in acc[.][0..1])
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        double a[4], bb[2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) a[i] = Xs[buf][i * 8 + g][ks * 4 + t];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) bb[j] = Xs[buf][32 + (jbase + j) * 8 + g][ks * 4 + t];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 2; ++j) dmma(acc[i][j], a[i], bb[j]);
+      }
     }
     if (tile + 1 < tiles) stash(buf ^ 1);
     __syncthreads();
   }
 
   double* out = part + ((int64_t)pair * chunks + chunk) * (kPairRows * kPairRows);
+  if (diagonal) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (!((mask >> (i * 4 + j)) & 1u)) continue;
-      const int r = rb * 32 + i * 8 + g, c = cb * 32 + j * 8 + 2 * t;
-      *reinterpret_cast<double2*>(out + r * kPairRows + c) = make_double2(acc[i][j][0], acc[i][j][1]);
-    }
+      for (int j = i; j < 4; ++j) {
+        const int r = rb * 32 + i * 8 + g, c = cb * 32 + j * 8 + 2 * t;
+        *reinterpret_cast<double2*>(out + r * kPairRows + c) = make_double2(acc[i][j][0], acc[i][j][1]);
+      }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int r = i * 8 + g, c = 32 + (jbase + j) * 8 + 2 * t;
+        *reinterpret_cast<double2*>(out + r * kPairRows + c) = make_double2(acc[i][j][0], acc[i][j][1]);
+      }
+  }
 }
 
 // One cyclic sweep over the 64 rows of a block pair, run on their Gram matrix A, with the rotations
