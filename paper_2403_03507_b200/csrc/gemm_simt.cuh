@@ -119,8 +119,9 @@ template <typename TA, typename TB, typename TAcc, int BM, int BN, int BK, int T
 __global__ void __launch_bounds__((BM / TM) * (BN / TN))
 gemm_simt_kernel(int M, int N, int K, const TA* __restrict__ A, int64_t sAi, int64_t sAk,
                  const TB* __restrict__ B, int64_t sBk, int64_t sBj, int kchunk, Epi epi_in, int batched,
-                 int64_t batchA, int64_t batchB, const SlotList slots) {
+                 int64_t batchA, int64_t batchB, const SlotList slots, int lower_only) {
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  if (lower_only && n0 > m0 + BM - 1) return;      // the tile lies strictly above the diagonal of a square result
   const int inner = gridDim.z / slots.n;
   const int zi = blockIdx.z % inner;
   const int64_t shift = (int64_t)slots.id[blockIdx.z / inner] * slots.bytes;
@@ -282,7 +283,8 @@ struct EpiApplyW {
 template <typename TA, typename TB, typename TAcc, class Epi>
 galore_status_t launch_gemm_simt(int M, int N, int K, const TA* A, int64_t sAi, int64_t sAk, const TB* B,
                                  int64_t sBk, int64_t sBj, int splits, Epi epi, cudaStream_t stream, int batch = 0,
-                                 int64_t batchA = 0, int64_t batchB = 0, const SlotList* slot_list = nullptr) {
+                                 int64_t batchA = 0, int64_t batchB = 0, const SlotList* slot_list = nullptr,
+                                 bool lower_only = false) {
   if (M <= 0 || N <= 0) return GALORE_OK;
   if (batch > 0) splits = 1;       // a batch uses blockIdx.z for the problem index
   if (splits < 1) splits = 1;
@@ -295,11 +297,11 @@ galore_status_t launch_gemm_simt(int M, int N, int K, const TA* A, int64_t sAi, 
   if (small) {
     dim3 grid((unsigned)ceil_div(N, 64), (unsigned)ceil_div(M, 64), gz);
     gemm_simt_kernel<TA, TB, TAcc, 64, 64, 16, 4, 4, Epi><<<grid, 256, 0, stream>>>(
-        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi, batch > 0 ? 1 : 0, batchA, batchB, slots);
+        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi, batch > 0 ? 1 : 0, batchA, batchB, slots, lower_only ? 1 : 0);
   } else {
     dim3 grid((unsigned)ceil_div(N, 128), (unsigned)ceil_div(M, 128), gz);
     gemm_simt_kernel<TA, TB, TAcc, 128, 128, 16, 8, 8, Epi><<<grid, 256, 0, stream>>>(
-        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi, batch > 0 ? 1 : 0, batchA, batchB, slots);
+        M, N, K, A, sAi, sAk, B, sBk, sBj, kchunk, epi, batch > 0 ? 1 : 0, batchA, batchB, slots, lower_only ? 1 : 0);
   }
   GALORE_LAUNCH_CHECK();
   return GALORE_OK;

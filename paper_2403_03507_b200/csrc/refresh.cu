@@ -636,11 +636,11 @@ static galore_status_t gram(const Ctx& c, const std::vector<Lane*>& lanes, Src s
 template <typename TA, typename TB, typename S, class Epi>
 static galore_status_t gemm_scalar(int M, int N, int K, const TA* A, int64_t sAi, int64_t sAk, const TB* B, int64_t sBk,
                                    int64_t sBj, Epi epi, cudaStream_t st, const SlotList& sl, int batch = 1, int64_t bA = 0,
-                                   int64_t bB = 0) {
+                                   int64_t bB = 0, bool lower_only = false) {
   if constexpr (std::is_same<S, double>::value)
     return launch_gemm_dmma<TA, TB>(M, N, K, A, sAi, sAk, B, sBk, sBj, epi, st, batch, bA, bB, &sl);
   else
-    return launch_gemm_simt<TA, TB, float>(M, N, K, A, sAi, sAk, B, sBk, sBj, 1, epi, st, batch, bA, bB, &sl);
+    return launch_gemm_simt<TA, TB, float>(M, N, K, A, sAi, sAk, B, sBk, sBj, 1, epi, st, batch, bA, bB, &sl, lower_only);
 }
 
 template <typename S>
@@ -660,9 +660,10 @@ static galore_status_t cholesky_inverse(const Ctx& c, const SlotList& sl, S* C, 
       // L[rest, J] = C[rest, J] Linv^T   (in place: one CTA column covers all nb columns)
       EpiStore<S, S> epi{panel, b, 0, S(1), S(0)};
       GALORE_TRY((gemm_scalar<S, S, S>(rem, nb, nb, panel, b, 1, slab, 1, 64, epi, st, sl)));
-      // C[rest, rest] -= L[rest, J] L[rest, J]^T
+      // C[rest, rest] -= L[rest, J] L[rest, J]^T  (only the lower triangle of C is ever read: tiles above the
+      // diagonal are left out where the kernel can)
       EpiStore<S, S> upd{C + (int64_t)j1 * b + j1, b, 0, S(-1), S(1)};
-      GALORE_TRY((gemm_scalar<S, S, S>(rem, rem, nb, panel, b, 1, panel, 1, b, upd, st, sl)));
+      GALORE_TRY((gemm_scalar<S, S, S>(rem, rem, nb, panel, b, 1, panel, 1, b, upd, st, sl, 1, 0, 0, true)));
     }
   }
   for (int i = 0; i < sl.n; ++i)
