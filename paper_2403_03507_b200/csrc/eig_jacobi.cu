@@ -256,7 +256,7 @@ __global__ void __launch_bounds__(kSweepThreads, 2) jb_sweep_kernel(const double
   }
   double* const As = jb_smem;                          // the Gram matrix (upper triangle used)
   double* const Rs = jb_smem + kPairRows * kALd;       // the accumulated rotation
-  __shared__ double2 cs[kSlots];
+  __shared__ double2 cs[2][kSlots];     // the rotations of the current round and of the next
   const int pair = blockIdx.x, tid = threadIdx.x;
   const BlockPair bp = block_pair(pair, round, nblk);
   if (bp.I * kBlockRows >= b) {
@@ -302,60 +302,69 @@ __global__ void __launch_bounds__(kSweepThreads, 2) jb_sweep_kernel(const double
   __syncthreads();
   int applied = 0;
   const double tol2 = tol * tol;
-  for (int rr = 0; rr < kSweepRounds; ++rr) {
-    const double* Ac = As;
-    if (tid < kSlots) {
-      const int f = tid, g = kPairRows - 1 - tid;
-      const double app = Ac[f * kALd + f], aqq = Ac[g * kALd + g], apq = Ac[f * kALd + g];
-      double c = 1.0, s = 0.0;
-      if (apq != 0.0 && apq * apq > tol2 * app * aqq) {
-        // tan(2 phi) = 2 apq / (aqq - app), |phi| <= pi/4.  With h = hypot(d, o): cos(2 phi) = |d| / h,
-        // c = sqrt((1 + |d|/h) / 2), s = sign(d) o / (2 h c).
-        const double d = aqq - app, o = 2.0 * apq;
-        const int ex = (__double2hiint(fmax(fabs(d), fabs(o))) >> 20) & 0x7ff;
-        if (ex >= 1 && ex <= 2045) {
-          const double sc = __hiloint2double((2046 - ex) << 20, 0);
-          const float df = (float)(d * sc), of = (float)(o * sc);
-          const float rh = rsqrtf(fmaf(df, df, of * of));
-          const float v = fmaf(0.5f * fabsf(df), rh, 0.5f);
-          const float rc = rsqrtf(v);
-          const float c0 = v * rc, s0 = (d >= 0.0 ? 0.5f : -0.5f) * of * rh * rc;
-          if (s0 != 0.0f) {
-            c = (double)c0;
-            s = (double)s0;
-            const double eps = fma(c, c, fma(s, s, -1.0));          // c0^2 + s0^2 = 1 + eps, |eps| ~ 1e-7
-            const double fix = fma(eps, fma(eps, 0.375, -0.5), 1.0);  // (1 + eps)^-1/2 to O(eps^3)
-            c *= fix;
-            s *= fix;
-            ++applied;
-          }
+  // the rotation of slot `tid` (positions tid and 63 - tid) from the current A
+  auto rotation = [&]() -> double2 {
+    const int f = tid, g = kPairRows - 1 - tid;
+    const double app = As[f * kALd + f], aqq = As[g * kALd + g], apq = As[f * kALd + g];
+    double c = 1.0, s = 0.0;
+    if (apq != 0.0 && apq * apq > tol2 * app * aqq) {
+      // tan(2 phi) = 2 apq / (aqq - app), |phi| <= pi/4.  With h = hypot(d, o): cos(2 phi) = |d| / h,
+      // c = sqrt((1 + |d|/h) / 2), s = sign(d) o / (2 h c).
+      const double d = aqq - app, o = 2.0 * apq;
+      const int ex = (__double2hiint(fmax(fabs(d), fabs(o))) >> 20) & 0x7ff;
+      if (ex >= 1 && ex <= 2045) {
+        const double sc = __hiloint2double((2046 - ex) << 20, 0);
+        const float df = (float)(d * sc), of = (float)(o * sc);
+        const float rh = rsqrtf(fmaf(df, df, of * of));
+        const float v = fmaf(0.5f * fabsf(df), rh, 0.5f);
+        const float rc = rsqrtf(v);
+        const float c0 = v * rc, s0 = (d >= 0.0 ? 0.5f : -0.5f) * of * rh * rc;
+        if (s0 != 0.0f) {
+          c = (double)c0;
+          s = (double)s0;
+          const double eps = fma(c, c, fma(s, s, -1.0));          // c0^2 + s0^2 = 1 + eps, |eps| ~ 1e-7
+          const double fix = fma(eps, fma(eps, 0.375, -0.5), 1.0);  // (1 + eps)^-1/2 to O(eps^3)
+          c *= fix;
+          s *= fix;
+          ++applied;
         }
       }
-      cs[tid] = make_double2(c, s);
     }
-    // every entry moves one position on (the round-robin order of the rows): read, barrier, write
+    return make_double2(c, s);
+  };
+  // A round: A <- rotated A (every entry also moves one position on, the round-robin order of the rows),
+  // then, side by side, the first warp works out the next round's rotations from the new A while everybody
+  // rotates Rot.  Both matrices are updated in place: read, barrier, write.
+  //   barrier X: this round's rotations are visible, every thread has read its entries of A, and the previous
+  //              round's writes of Rot have landed;
+  //   barrier Y: the new A is visible and every thread has read its entries of Rot.
+  if (tid < kSlots) cs[0][tid] = rotation();
+  for (int rr = 0; rr < kSweepRounds; ++rr) {
+    const double2* cur = cs[rr & 1];
     const BlockValues v0 = block_read(t0, As);
     BlockValues v1 = v0;
     if (second) v1 = block_read(t1, As);
+    __syncthreads();                                   // X
+    block_write(t0, cur, v0, As);
+    if (second) block_write(t1, cur, v1, As);
     double rx[4], ry[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       rx[i] = Rs[rf + 16 * i];
       ry[i] = Rs[rg + 16 * i];
     }
-    __syncthreads();
-    block_write(t0, cs, v0, As);
-    if (second) block_write(t1, cs, v1, As);
+    __syncthreads();                                   // Y
+    if (tid < kSlots && rr + 1 < kSweepRounds) cs[(rr + 1) & 1][tid] = rotation();
     {
-      const double2 r = cs[rslot];
+      const double2 r = cur[rslot];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         Rs[wf + 16 * i] = r.x * rx[i] - r.y * ry[i];
         Rs[wg + 16 * i] = r.y * rx[i] + r.x * ry[i];
       }
     }
-    __syncthreads();
   }
+  __syncthreads();
   if (tid < 32) {
     for (int o = 16; o > 0; o >>= 1) applied += __shfl_xor_sync(0xffffffffu, applied, o);
     applied = __shfl_sync(0xffffffffu, applied, 0);
@@ -363,10 +372,10 @@ __global__ void __launch_bounds__(kSweepThreads, 2) jb_sweep_kernel(const double
       flags[pair] = applied;
       if (applied) atomicAdd(rotations, applied);
     }
-    if (tid == 0) cs[0].x = (double)applied;
+    if (tid == 0) cs[0][0].x = (double)applied;
   }
   __syncthreads();
-  if (cs[0].x != 0.0) {   // all rows are back at their own positions after the 63 rounds
+  if (cs[0][0].x != 0.0) {   // all rows are back at their own positions after the 63 rounds
     const double* Rf = Rs;
     double* out = rot_out + (int64_t)pair * (kPairRows * kPairRows);
     for (int idx = tid; idx < kPairRows * kPairRows; idx += kSweepThreads) out[idx] = Rf[(idx >> 6) * kALd + (idx & 63)];
