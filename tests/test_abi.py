@@ -70,12 +70,18 @@ def test_query_bytes_follows_memory_model():
     (dict(beta1=1.0), gb.ERR_INVALID_ARG),
     (dict(q_block=1000), gb.ERR_INVALID_ARG),
     (dict(side=7), gb.ERR_INVALID_ARG),
+    (dict(raw_state_fmt=3), gb.ERR_INVALID_ARG),
+    (dict(adam_place=5), gb.ERR_INVALID_ARG),
+    (dict(refresh_warm_iters=-1), gb.ERR_INVALID_ARG),
     (dict(path=gb.PATH_TENSOR, g_dtype="f32"), gb.ERR_UNIMPLEMENTED),
 ])
 def test_invalid_configs_are_rejected(kw, status):
     base = dict(m=12, n=20, rank=4, refresh_gap=5, w_dtype="f32", g_dtype="f32")
     base.update(kw)
+    raw_state_fmt = base.pop("raw_state_fmt", None)
     cfg = gb.make_config(**base)
+    if raw_state_fmt is not None:
+        cfg.state_fmt = raw_state_fmt                 # a value the binding's names do not reach
     sb, wb = C.c_size_t(), C.c_size_t()
     assert gb.lib().galore_query_bytes(C.byref(cfg), C.byref(sb), C.byref(wb)) == status
     with pytest.raises(gb.GaloreError):
