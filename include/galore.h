@@ -108,7 +108,7 @@ typedef struct {
   int32_t auto_refresh;    /* 1: galore_step refreshes P when (completed steps) mod T == 0 */
   int32_t path;            /* galore_path_t */
   /* refresh: block subspace iteration on a block of rank + refresh_oversample
-   * columns (clipped to min(m, n); 0 = default: max(256, rank / 2) on the
+   * columns (clipped to min(m, n); 0 = default: max(256, rank / 4) on the
    * tensor path, rank more columns elsewhere; negative = none),
    * stopped when the predicted subspace error falls below refresh_tol or
    * after refresh_max_iters power iterations.  The prediction is

@@ -146,11 +146,13 @@ galore_status_t resolve(const galore_config_t* c, Sizes* s) {
   if (c->path == GALORE_PATH_TENSOR && !eligible) return GALORE_ERR_UNIMPLEMENTED;
   s->tensor_path = eligible && c->path != GALORE_PATH_FP32;
   // Extra columns of the refresh block.  More of them mean fewer power steps but a larger dense
-  // eigenproblem (cubic in the block); where the steps run on the tensor cores they are cheap and
-  // half the rank, at least 256, balances the two (a block only twice a small rank converges
-  // slowly on flat spectra); elsewhere the block is twice the rank.
+  // eigenproblem (cubic in the block).  Where the steps run on the tensor cores and slow blocks are
+  // finished by Chebyshev pairs they are cheap: a quarter of the rank, at least 256, balances the two
+  // (LLaMA-7B shapes at rank 1024, groups of eight: 168 / 295 ms with 256 extra columns against
+  // 205 / 318 ms with 512 and 165 / 308 ms with 192; a small rank needs the absolute floor to
+  // converge on flat spectra at all); elsewhere the block is twice the rank.
   int over = c->refresh_oversample;
-  if (over == 0) over = s->tensor_path ? std::max(256, r / 2) : r;
+  if (over == 0) over = s->tensor_path ? std::max(256, r / 4) : r;
   over = std::max(0, over);
   s->block = (int)std::min<int64_t>(s->d, (int64_t)r + over);
 

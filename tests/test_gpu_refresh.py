@@ -145,7 +145,7 @@ def test_tensor_core_refresh_gapped_and_low_rank():
 
 
 def test_full_size_7b_refresh_meets_the_angle_bound_before_rounding():
-    """4096 x 11008 at rank 1024 through the tensor-core refresh with its default block (rank + 512).  The
+    """4096 x 11008 at rank 1024 through the tensor-core refresh with its default block (rank + 256).  The
     1e-3 rad bound is checked on the projector before it is rounded to bf16 (the rounding alone moves the
     stored basis by about 2e-3).  Gapped planted spectrum: the top-r subspace is well defined."""
     m, n, r = 4096, 11008, 1024
@@ -154,7 +154,7 @@ def test_full_size_7b_refresh_meets_the_angle_bound_before_rounding():
     G, U, V = wl.make_planted(m, n, seed=21, spectrum=spectrum, dtype="bf16")
     st, info, P = _refresh_tc(G, r)
     Pu = _refresh_tc.unrounded
-    assert st == gb.OK and info["converged"] == 1 and info["block"] == r + 512
+    assert st == gb.OK and info["converged"] == 1 and info["block"] == r + 256
     assert np.abs(Pu.T @ Pu - np.eye(r)).max() < 1e-9
     P_orc, S = go.top_r_projector(G, r, "left", method="lapack")
     assert go.largest_principal_angle(P_orc, Pu) < ANGLE_TOL
